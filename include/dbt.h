@@ -1,0 +1,194 @@
+/*
+ * dbt.h -- C ABI of the grouped decode step of the Decode-Branch Transformer on B200.
+ *
+ * What the library computes (paper Section 4).  Two residual trajectories share every
+ * large matrix: the primary path S_1 is a standard causal Transformer and is the only
+ * writer of the persistent KV cache; the decode branch S_2 starts from its own token
+ * embedding (Eq. embeddings), forms only a query (Eq. asymattn: Q~_2 = Q_2 + a*Q_1, read
+ * against the primary K_1,V_1), is coupled in the MLP by b and c (Eq. mlp) and writes no
+ * persistent state.  Logits of both paths go through one output matrix and are mixed with
+ * alpha = clip_[0.5,1](sum_v p_v^2) (Eq. alpha, Eq. mixloss).  Inference follows Section
+ * 4.4: a primary-only prefill over the prompt, then grouped steps -- both paths' rows
+ * stacked through the shared matrices and one read of the primary cache serving both
+ * queries ("Decode" paragraph; Section 4.5, Eq. decode_traffic).
+ *
+ * Conventions.
+ *  - Every pointer is marked HOST or DEVICE.  All device memory (weights, KV pool,
+ *    workspace, token / logit buffers) belongs to the caller; the library borrows it,
+ *    never frees it and never writes the weights.  It must outlive the handle.
+ *  - Matrices are row-major [out_features, in_features] (the paper's H W with W stored
+ *    transposed), in `weight_dtype`.  Norm gains and the coupling vectors a, b, c are fp32.
+ *  - Stacked activations are path-major: rows 0..B-1 primary, B..2B-1 branch.
+ *  - KV pool layout: [n_layers][2 (K,V)][num_pages][n_kv_heads][page_size][head_dim] in
+ *    `weight_dtype`; K is stored after RoPE.  Logical position t of sequence b lives in
+ *    physical page page_table[b][t / page_size], slot t % page_size.
+ *  - Calls enqueue work on the CUDA stream given at creation and return without waiting
+ *    (the *_host variants wait).  Errors the host can see (bad arguments, capacity) are
+ *    returned at once and enqueue nothing.  Errors only the device can see (a token id out
+ *    of range) are recorded in a status word read by dbt_sync_status; the offending value is
+ *    clamped so that no access leaves its buffer.  Nothing traps or aborts.
+ *  - Not thread-safe per handle.
+ */
+#ifndef DBT_H
+#define DBT_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct dbt_model dbt_model; /* opaque; owned by the library */
+
+typedef enum {
+    DBT_OK = 0,
+    DBT_ERR_INVALID_ARG = 1,
+    DBT_ERR_UNSUPPORTED = 2, /* shape / option outside what the kernels cover        */
+    DBT_ERR_CAPACITY = 3,    /* max_batch, max_seq or the page pool would be exceeded */
+    DBT_ERR_STATE = 4,
+    DBT_ERR_CUDA = 5,
+    DBT_ERR_DEVICE = 6       /* the device status word is non-zero (dbt_sync_status)  */
+} dbt_status;
+
+enum { DBT_DTYPE_F32 = 0, DBT_DTYPE_BF16 = 1 };
+enum { DBT_ROUTER_INDEPENDENT = 0, DBT_ROUTER_REPLAY = 1 };
+
+typedef struct {
+    uint32_t struct_size; /* sizeof(dbt_config), for versioning */
+    int32_t d_model, n_layers, n_q_heads, n_kv_heads, head_dim, d_ff, vocab;
+    int32_t weight_dtype; /* DBT_DTYPE_*; the KV cache uses the same storage type */
+    float rope_base;      /* RoPE base; half-split pairs (i, i+head_dim/2), 0-based positions,
+                             the same position for both paths */
+    float rms_eps;
+    int32_t final_norm;       /* 1: RMSNorm before the shared output matrix */
+    int32_t n_experts;        /* 0 = dense MLP (Eq. mlp); >0 = MoE (Eq. moe_layer) */
+    int32_t d_expert;         /* hidden width of one routed expert */
+    int32_t n_shared_experts; /* applied to every token of both paths, un-gated */
+    int32_t k_primary;        /* k_1 of Eq. moe_budget */
+    int32_t k_branch;         /* k_2 of Eq. moe_budget */
+    int32_t router_mode;      /* DBT_ROUTER_* (replay: Section 4.3) */
+    int32_t moe_b_coupling;   /* 1: b couples the shared expert's hidden state; 0: b unused in MoE */
+    int32_t max_batch, max_seq;
+    int32_t page_size; /* tokens per KV page; 16 */
+    int32_t num_pages; /* pages in the pool, per layer and per K/V */
+} dbt_config;
+
+/* DEVICE pointers.  Unused entries (MoE fields of a dense model and vice versa) may be NULL. */
+typedef struct {
+    const float *attn_norm_g;                  /* [d]                                         */
+    const void *wq, *wk, *wv, *wo;             /* [q_dim,d] [kv_dim,d] [kv_dim,d] [d,q_dim]   */
+    const float *coup_a;                       /* [q_dim]                                     */
+    const float *mlp_norm_g;                   /* [d]                                         */
+    const void *w_gate, *w_up, *w_down;        /* dense: [F,d] [F,d] [d,F]                    */
+    const float *coup_b;                       /* dense [F]; MoE [n_shared*d_expert]          */
+    const float *coup_c;                       /* [d]                                         */
+    const void *router;                        /* [E,d]                                       */
+    const void *exp_gate, *exp_up, *exp_down;  /* [E,Fe,d] [E,Fe,d] [E,d,Fe]                  */
+    const void *sh_gate, *sh_up, *sh_down;     /* [Fs,d] [Fs,d] [d,Fs], Fs = n_shared*Fe      */
+} dbt_layer_weights;
+
+typedef struct {
+    const void *embed_primary, *embed_branch;  /* DEVICE E_1, E_2 [V,d]                       */
+    const float *embed_norm_g, *final_norm_g;  /* DEVICE [d]                                  */
+    const void *lm_head;                       /* DEVICE shared output matrix [V,d]           */
+    const dbt_layer_weights *layers;           /* HOST array [n_layers] of DEVICE pointers    */
+} dbt_weights;
+
+/* Bytes the caller must provide for the KV pool and the workspace (both DEVICE, 256-byte
+ * aligned).  cfg HOST. */
+dbt_status dbt_query_sizes(const dbt_config *cfg, size_t *kv_bytes, size_t *workspace_bytes);
+
+/* Build a handle (Section 4: the model of both paths).  cfg, w HOST; kv_pool_dev,
+ * workspace_dev DEVICE; cuda_stream a cudaStream_t (NULL = default stream).  Validates the
+ * configuration (DBT_ERR_UNSUPPORTED for head_dim not in {64,128}, page_size != 16,
+ * n_q_heads not a multiple of n_kv_heads, more than 16 queries per KV head over both
+ * paths, k > n_experts, ...), builds the RoPE table and the default page table
+ * (sequence b owns pages b*ceil(max_seq/page_size) ...), and zeroes all sequence lengths.
+ * On failure *out is NULL. */
+dbt_status dbt_create(const dbt_config *cfg, const dbt_weights *w, void *kv_pool_dev,
+                      void *workspace_dev, void *cuda_stream, dbt_model **out);
+void dbt_destroy(dbt_model *m);
+
+/* HOST table [B][pages_per_seq] of physical page ids (distinct, < num_pages) for sequences
+ * 0..B-1; pages_per_seq <= ceil(max_seq/page_size) bounds each sequence's capacity. */
+dbt_status dbt_set_page_table(dbt_model *m, const int32_t *table_host, int32_t B, int32_t pages_per_seq);
+
+/* Sequence lengths := 0 (the cache contents are left as they are). */
+dbt_status dbt_reset(dbt_model *m);
+/* Declare that sequences 0..B-1 already hold lens_host[b] cached positions (the caller
+ * wrote the pool itself, e.g. a synthetic fill for timing).  lens_host HOST. */
+dbt_status dbt_set_seq_lens(dbt_model *m, const int32_t *lens_host, int32_t B);
+/* Current length of sequence b as the host tracks it (-1 on a bad argument). */
+int32_t dbt_seq_len(const dbt_model *m, int32_t b);
+
+/* Section 4.4 item 1, prompt-wide prefill: the primary path alone processes n positions of
+ * sequences 0..B-1 (tokens_dev DEVICE int32 [B][n]) starting at their current lengths,
+ * writes their K/V and advances the lengths.  No branch computation.
+ * last_primary_logits_dev: DEVICE fp32 [B][V] for the last position, or NULL. */
+dbt_status dbt_prefill(dbt_model *m, const int32_t *tokens_dev, int32_t B, int32_t n,
+                       float *last_primary_logits_dev);
+
+/* Section 4.4 items 2-3, one grouped step ("Decode" paragraph): for each sequence b the token
+ * tokens_dev[b] at position t_b = its length; the primary appends K_1,V_1[t_b]; both paths'
+ * queries read positions 0..t_b of the primary cache; the shared matrices are applied to
+ * the stacked rows; next_tokens_dev[b] = argmax of alpha*p + (1-alpha)*q (lowest index on
+ * ties).  Lengths advance by one.  All pointers DEVICE; outputs may be NULL:
+ * next_tokens_dev int32 [B] (may alias tokens_dev), logits_* fp32 [B][V], alpha_dev fp32 [B].
+ * To start from a prompt x_1..x_S: prefill x_1..x_{S-1}, then pass x_S to the first step
+ * (the boundary step of Section 4.4 item 2). */
+dbt_status dbt_decode_step(dbt_model *m, const int32_t *tokens_dev, int32_t B, int32_t *next_tokens_dev,
+                           float *logits_primary_dev, float *logits_branch_dev, float *alpha_dev);
+
+/* The comparison path: the same step with the branch rows absent (a standard decode step,
+ * Background "decode").  Writes the same K/V bits as dbt_decode_step for the same inputs;
+ * next token = argmax of the primary logits. */
+dbt_status dbt_decode_step_primary_only(dbt_model *m, const int32_t *tokens_dev, int32_t B,
+                                        int32_t *next_tokens_dev, float *logits_primary_dev);
+
+/* End-to-end variants with HOST buffers: copy tokens_host [B] to the device, run the step,
+ * copy next_tokens_host [B] (and alpha_host [B] when non-NULL) back, wait for the stream.
+ * Buffers should be pinned for the copies to be asynchronous. */
+dbt_status dbt_decode_step_host(dbt_model *m, const int32_t *tokens_host, int32_t B,
+                                int32_t *next_tokens_host, float *alpha_host);
+dbt_status dbt_decode_step_primary_only_host(dbt_model *m, const int32_t *tokens_host, int32_t B,
+                                             int32_t *next_tokens_host);
+
+/* MoE only: DEVICE int32 [n_layers][2][max_batch][kmax] (kmax = max(k_primary,k_branch)),
+ * the expert ids each row used in the last decode step (-1 padded); and the number of
+ * distinct experts loaded per layer in the last step, HOST int32 [n_layers] (waits for the
+ * stream).  Equation moe_layer leaves near-ties in the router to rounding, so tests read the
+ * choice back instead of assuming it. */
+dbt_status dbt_last_experts(dbt_model *m, const int32_t **experts_dev, int32_t *kmax);
+dbt_status dbt_last_expert_union(dbt_model *m, int32_t *count_per_layer_host);
+
+/* Wait for the stream and read the device status word.  *device_status: 0 = clean, 1 = a token
+ * id was out of range, 2 = a page id was out of range; *detail = the offending value.
+ * Returns DBT_ERR_DEVICE when non-zero.  HOST pointers, may be NULL. */
+dbt_status dbt_sync_status(dbt_model *m, int32_t *device_status, int32_t *detail);
+
+/* Per-kernel timing for the roofline report (paper Eq. roofline, Eq. decode_traffic: time
+ * against the bytes that must move).  Between begin and end every kernel launch is bracketed
+ * by CUDA events on the handle's stream; end waits for the stream and sums, per kernel family,
+ * the launches, the device time and the algorithmic bytes (weights read once, visible K/V read
+ * once; 0 for kernels that move neither).  entries_host HOST [max_entries]. */
+typedef struct {
+    char name[32];
+    int64_t launches;
+    double total_ms;
+    double bytes;
+} dbt_profile_entry;
+dbt_status dbt_profile_begin(dbt_model *m);
+dbt_status dbt_profile_end(dbt_model *m, dbt_profile_entry *entries_host, int32_t max_entries, int32_t *n_entries);
+
+/* Kernels launched by this handle since creation (for benchmark bookkeeping). */
+int64_t dbt_launch_count(const dbt_model *m);
+/* Last host-side error message of this handle (or of the failed dbt_create when m is NULL). */
+const char *dbt_last_error(const dbt_model *m);
+/* Library version string. */
+const char *dbt_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DBT_H */

@@ -1,0 +1,716 @@
+// Host side of the C ABI declared in include/dbt.h: argument checks, workspace carving,
+// the per-step launch plan.  Every step of the path runs in this library's kernels.
+#include "../../include/dbt.h"
+
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "dbt_kernels.cuh"
+
+using namespace dbt;
+
+namespace {
+
+thread_local std::string g_create_error;
+
+struct Workspace {
+    // fp32 activations, rows = Rmax unless noted
+    float *S, *X, *Q, *Kn, *Vn, *O, *G1, *M, *Z, *part, *Zrows;
+    float2 *rope;
+    int32_t *seq_len, *page_table, *status, *tokens_stage, *next_stage;
+    float *alpha_stage;
+    // MoE
+    float *rlogits, *rwts, *Hexp, *Yexp, *Msh, *Hsh;
+    int32_t *ridx, *ecnt, *elist, *last_experts, *union_cnt;
+};
+
+}  // namespace
+
+struct dbt_model {
+    dbt_config cfg;
+    dbt_weights w;
+    std::vector<dbt_layer_weights> layers;
+    cudaStream_t stream;
+    char *kv_pool;
+    char *ws_base;
+    size_t ws_bytes;
+    Workspace ws;
+    int Rmax, pages_per_seq_max, pages_per_seq, part_items;
+    std::vector<int32_t> len_host;
+    int64_t launches;
+    std::string err;
+    bool pending_union;
+    // optional per-launch timing (dbt_profile_begin / dbt_profile_end)
+    bool prof_on;
+    struct ProfRec { const char *tag; double bytes; cudaEvent_t e0, e1; };
+    std::vector<ProfRec> prof;
+    std::vector<cudaEvent_t> prof_pool;
+};
+
+namespace {
+
+size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
+
+struct Carver {
+    char *base;
+    size_t off;
+    template <typename T>
+    T *take(size_t n) {
+        off = align_up(off);
+        T *p = base ? reinterpret_cast<T *>(base + off) : nullptr;
+        off += n * sizeof(T);
+        return p;
+    }
+};
+
+int elem_bytes(const dbt_config &c) { return c.weight_dtype == DBT_DTYPE_F32 ? 4 : 2; }
+int kmax_of(const dbt_config &c) { return c.k_primary > c.k_branch ? c.k_primary : c.k_branch; }
+int prefill_rows(const dbt_config &c) { return 2 * c.max_batch > 128 ? 2 * c.max_batch : 128; }
+
+const char *check_config(const dbt_config *c, dbt_status *st) {
+    *st = DBT_ERR_INVALID_ARG;
+    if (!c) return "config is NULL";
+    if (c->struct_size != sizeof(dbt_config)) return "dbt_config.struct_size does not match this library";
+    if (c->d_model <= 0 || c->n_layers <= 0 || c->n_q_heads <= 0 || c->n_kv_heads <= 0 || c->vocab <= 0)
+        return "non-positive model dimension";
+    if (c->max_batch <= 0 || c->max_seq <= 0 || c->num_pages <= 0) return "non-positive capacity";
+    if (c->weight_dtype != DBT_DTYPE_F32 && c->weight_dtype != DBT_DTYPE_BF16) return "unknown weight_dtype";
+    *st = DBT_ERR_UNSUPPORTED;
+    if (c->head_dim != 64 && c->head_dim != 128) return "head_dim must be 64 or 128";
+    if (c->page_size != 16) return "page_size must be 16";
+    if (c->n_q_heads % c->n_kv_heads) return "n_q_heads must be a multiple of n_kv_heads";
+    if (2 * (c->n_q_heads / c->n_kv_heads) > 16) return "more than 16 queries per KV head over both paths";
+    if (c->d_model % 8) return "d_model must be a multiple of 8";
+    if (c->router_mode != DBT_ROUTER_INDEPENDENT && c->router_mode != DBT_ROUTER_REPLAY) return "unknown router_mode";
+    if (c->n_experts > 0) {
+        if (c->d_expert <= 0 || c->d_expert % 8) return "d_expert must be a positive multiple of 8";
+        if (c->k_primary <= 0 || c->k_branch <= 0) return "k_primary and k_branch must be positive";
+        if (c->k_primary > c->n_experts || c->k_branch > c->n_experts) return "top-k exceeds n_experts";
+        if (kmax_of(*c) > 64 || c->n_experts > 1024) return "at most 64 experts per token and 1024 experts";
+        if (c->n_shared_experts < 0) return "negative n_shared_experts";
+    } else {
+        if (c->d_ff <= 0 || c->d_ff % 8) return "d_ff must be a positive multiple of 8";
+    }
+    *st = DBT_OK;
+    return nullptr;
+}
+
+// One pass over the workspace layout; with base == nullptr it only measures.
+size_t carve(const dbt_config &c, char *base, Workspace *ws, int *Rmax_out, int *part_items_out) {
+    Carver k{base, 0};
+    Workspace w{};
+    int Rmax = prefill_rows(c);
+    int d = c.d_model, qd = c.n_q_heads * c.head_dim, kvd = c.n_kv_heads * c.head_dim;
+    bool moe = c.n_experts > 0;
+    int Fs = moe ? c.n_shared_experts * c.d_expert : 0;
+    int F = moe ? (Fs > 0 ? Fs : 8) : c.d_ff;
+    int pps = (c.max_seq + c.page_size - 1) / c.page_size;
+    int part_items = Rmax * c.n_kv_heads + 2 * 148;
+    w.S = k.take<float>((size_t)Rmax * d);
+    w.X = k.take<float>((size_t)Rmax * d);
+    w.Q = k.take<float>((size_t)Rmax * qd);
+    w.Kn = k.take<float>((size_t)Rmax * kvd);
+    w.Vn = k.take<float>((size_t)Rmax * kvd);
+    w.O = k.take<float>((size_t)Rmax * qd);
+    w.G1 = k.take<float>((size_t)Rmax * F);
+    w.M = k.take<float>((size_t)Rmax * d);
+    w.Z = k.take<float>((size_t)2 * c.max_batch * c.vocab);
+    w.Zrows = k.take<float>((size_t)2 * c.max_batch * d);
+    w.part = k.take<float>((size_t)part_items * 16 * (c.head_dim + 2));
+    w.rope = k.take<float2>((size_t)c.max_seq * (c.head_dim / 2));
+    w.seq_len = k.take<int32_t>(c.max_batch);
+    w.page_table = k.take<int32_t>((size_t)c.max_batch * pps);
+    w.status = k.take<int32_t>(4);
+    w.tokens_stage = k.take<int32_t>(c.max_batch);
+    w.next_stage = k.take<int32_t>(c.max_batch);
+    w.alpha_stage = k.take<float>(c.max_batch);
+    if (moe) {
+        int km = kmax_of(c);
+        w.rlogits = k.take<float>((size_t)Rmax * c.n_experts);
+        w.rwts = k.take<float>((size_t)Rmax * km);
+        w.ridx = k.take<int32_t>((size_t)Rmax * km);
+        w.Hexp = k.take<float>((size_t)Rmax * km * c.d_expert);
+        w.Yexp = k.take<float>((size_t)Rmax * km * d);
+        w.Msh = k.take<float>((size_t)Rmax * d);
+        w.Hsh = k.take<float>((size_t)Rmax * (Fs > 0 ? Fs : 8));
+        w.ecnt = k.take<int32_t>(c.n_experts);
+        w.elist = k.take<int32_t>((size_t)c.n_experts * Rmax);
+        w.last_experts = k.take<int32_t>((size_t)c.n_layers * 2 * c.max_batch * km);
+        w.union_cnt = k.take<int32_t>(c.n_layers);
+    }
+    if (ws) *ws = w;
+    if (Rmax_out) *Rmax_out = Rmax;
+    if (part_items_out) *part_items_out = part_items;
+    return align_up(k.off);
+}
+
+dbt_status fail(dbt_model *m, dbt_status st, const char *fmt, ...) {
+    char buf[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof buf, fmt, ap);
+    va_end(ap);
+    if (m)
+        m->err = buf;
+    else
+        g_create_error = buf;
+    return st;
+}
+
+#define CUDA_TRY(m, call)                                                                            \
+    do {                                                                                             \
+        cudaError_t e_ = (call);                                                                     \
+        if (e_ != cudaSuccess) return fail(m, DBT_ERR_CUDA, "%s: %s", #call, cudaGetErrorString(e_)); \
+    } while (0)
+
+cudaEvent_t prof_event(dbt_model *m) {
+    cudaEvent_t e = nullptr;
+    if (!m->prof_pool.empty()) {
+        e = m->prof_pool.back();
+        m->prof_pool.pop_back();
+    } else {
+        cudaEventCreate(&e);
+    }
+    return e;
+}
+
+// tag: kernel family name for the profile; bytes: the algorithmic bytes this launch must move.
+#define LAUNCH(m, tag, bytes, kernel, grid, block, smem, ...)                                            \
+    do {                                                                                                 \
+        cudaEvent_t p0_ = nullptr, p1_ = nullptr;                                                        \
+        if ((m)->prof_on) {                                                                              \
+            p0_ = prof_event(m);                                                                         \
+            p1_ = prof_event(m);                                                                         \
+            cudaEventRecord(p0_, (m)->stream);                                                           \
+        }                                                                                                \
+        kernel<<<grid, block, smem, (m)->stream>>>(__VA_ARGS__);                                         \
+        (m)->launches++;                                                                                 \
+        cudaError_t e_ = cudaGetLastError();                                                             \
+        if ((m)->prof_on) {                                                                              \
+            cudaEventRecord(p1_, (m)->stream);                                                           \
+            (m)->prof.push_back(dbt_model::ProfRec{tag, (double)(bytes), p0_, p1_});                     \
+        }                                                                                                \
+        if (e_ != cudaSuccess) return fail(m, DBT_ERR_CUDA, "launch %s: %s", #kernel, cudaGetErrorString(e_)); \
+    } while (0)
+
+// ---- launch helpers -------------------------------------------------------------------
+
+template <typename WT>
+dbt_status run_linear(dbt_model *m, const char *tag, const LinArgs &a) {
+    int total = 0;
+    double bytes = 0;
+    for (int s = 0; s < a.nseg; s++) bytes += (double)a.n_out[a.epi == EPI_SWIGLU ? 0 : s] * a.K * sizeof(WT);
+    if (a.epi == EPI_SWIGLU)
+        total = a.n_out[0];
+    else
+        for (int s = 0; s < a.nseg; s++) total += a.n_out[s];
+    int grid = (total + kLinWarps - 1) / kLinWarps;
+    LAUNCH(m, tag, bytes, linear_kernel<WT>, grid, kLinWarps * 32, 0, a);
+    return DBT_OK;
+}
+
+LinArgs lin1(const void *W, float *Y, int n_out, int rows, const float *X, int K, int epi = EPI_STORE) {
+    LinArgs a{};
+    a.W[0] = W;
+    a.Y[0] = Y;
+    a.n_out[0] = n_out;
+    a.rows[0] = rows;
+    a.nseg = 1;
+    a.X = X;
+    a.K = K;
+    a.epi = epi;
+    return a;
+}
+
+template <typename KT, int DH>
+dbt_status run_attention(dbt_model *m, const RowMap &rm, int grouped, const KT *kpool, const KT *vpool, int nsplit,
+                         double kv_bytes) {
+    const dbt_config &c = m->cfg;
+    int G = c.n_q_heads / c.n_kv_heads, nq = grouped ? 2 * G : G;
+    dim3 grid(rm.B * rm.cn, c.n_kv_heads, nsplit);
+    int NQ = nq <= 1 ? 1 : nq <= 2 ? 2 : nq <= 4 ? 4 : nq <= 8 ? 8 : 16;
+    const Workspace &w = m->ws;
+#define ATTN_CASE(N)                                                                                          \
+    case N:                                                                                                   \
+        LAUNCH(m, "attention", kv_bytes, (attn_partial_kernel<KT, N, DH>), grid, 128, 0, w.Q, rm, grouped, G, c.n_kv_heads, kpool,   \
+               vpool, w.page_table, m->pages_per_seq_max, c.num_pages, w.seq_len, nsplit, w.part, w.status);  \
+        break;
+    switch (NQ) {
+        ATTN_CASE(1)
+        ATTN_CASE(2)
+        ATTN_CASE(4)
+        ATTN_CASE(8)
+        ATTN_CASE(16)
+    }
+#undef ATTN_CASE
+    dim3 mgrid(rm.B * rm.cn, c.n_kv_heads);
+    LAUNCH(m, "attn_merge", 0, attn_merge_kernel, mgrid, DH, 0, w.part, nsplit, NQ, DH, rm.B * rm.cn, grouped, G, c.n_kv_heads, w.O);
+    return DBT_OK;
+}
+
+// The layer stack on `rows` stacked rows (Bc primary rows, then Bc branch rows when grouped).
+// Section 4.1 (attention), Eq. mlp / Eq. moe_layer (MLP), in the order the paper gives them.
+template <typename WT>
+dbt_status run_layers(dbt_model *m, const RowMap &rm, int grouped, bool record_experts) {
+    const dbt_config &c = m->cfg;
+    const Workspace &w = m->ws;
+    int Bc = rm.B * rm.cn, R = grouped ? 2 * Bc : Bc;
+    int d = c.d_model, qd = c.n_q_heads * c.head_dim, kvd = c.n_kv_heads * c.head_dim;
+    size_t pool_layer_elems = (size_t)2 * c.num_pages * c.n_kv_heads * c.page_size * c.head_dim;
+    size_t pool_kv_elems = pool_layer_elems / 2;
+    int nsplit = (2 * 148 + Bc * c.n_kv_heads - 1) / (Bc * c.n_kv_heads);
+    nsplit = nsplit < 1 ? 1 : nsplit > 16 ? 16 : nsplit;
+    double kv_bytes = 0;  // K and V of every visible position, once per layer
+    for (int b = 0; b < rm.B; b++)
+        for (int j = 0; j < rm.cn; j++) kv_bytes += (double)(m->len_host[b] + j + 1) * 2 * kvd * sizeof(WT);
+    dbt_status st;
+    for (int l = 0; l < c.n_layers; l++) {
+        const dbt_layer_weights &lw = m->layers[l];
+        WT *kpool = reinterpret_cast<WT *>(m->kv_pool) + (size_t)l * pool_layer_elems;
+        WT *vpool = kpool + pool_kv_elems;
+        // N_i = RMSNorm(S_i)
+        LAUNCH(m, "rmsnorm", 0, rmsnorm_kernel, R, 256, 0, w.S, lw.attn_norm_g, c.rms_eps, d, 1, 0, 1, w.X);
+        // Q for all rows; K, V for the primary rows only (the branch produces only a query)
+        LinArgs a{};
+        a.W[0] = lw.wq; a.Y[0] = w.Q; a.n_out[0] = qd; a.rows[0] = R;
+        a.W[1] = lw.wk; a.Y[1] = w.Kn; a.n_out[1] = kvd; a.rows[1] = Bc;
+        a.W[2] = lw.wv; a.Y[2] = w.Vn; a.n_out[2] = kvd; a.rows[2] = Bc;
+        a.nseg = 3; a.X = w.X; a.K = d; a.epi = EPI_STORE;
+        if ((st = run_linear<WT>(m, "linear_qkv", a)) != DBT_OK) return st;
+        LAUNCH(m, "rope_append", 0, rope_couple_append_kernel<WT>, Bc, 256, 0, w.Q, w.Kn, w.Vn, rm, grouped, c.n_q_heads, c.n_kv_heads,
+               c.head_dim, lw.coup_a, w.rope, w.seq_len, w.page_table, m->pages_per_seq_max, c.num_pages, c.page_size,
+               kpool, vpool, w.status);
+        if (c.head_dim == 128)
+            st = run_attention<WT, 128>(m, rm, grouped, kpool, vpool, nsplit, kv_bytes);
+        else
+            st = run_attention<WT, 64>(m, rm, grouped, kpool, vpool, nsplit, kv_bytes);
+        if (st != DBT_OK) return st;
+        // S-bar_i = S_i + Attn_i W_O
+        LinArgs o = lin1(lw.wo, nullptr, d, R, w.O, qd, EPI_RESID);
+        o.S = w.S;
+        if ((st = run_linear<WT>(m, "linear_o", o)) != DBT_OK) return st;
+        LAUNCH(m, "rmsnorm", 0, rmsnorm_kernel, R, 256, 0, w.S, lw.mlp_norm_g, c.rms_eps, d, 1, 0, 1, w.X);
+        if (c.n_experts == 0) {
+            LinArgs gu{};
+            gu.W[0] = lw.w_gate; gu.W[1] = lw.w_up; gu.Y[0] = w.G1; gu.n_out[0] = c.d_ff; gu.rows[0] = R;
+            gu.nseg = 2; gu.X = w.X; gu.K = d; gu.epi = EPI_SWIGLU; gu.Bc = Bc; gu.grouped = grouped;
+            gu.coup = lw.coup_b;
+            if ((st = run_linear<WT>(m, "linear_gateup", gu)) != DBT_OK) return st;
+            LinArgs dn = lin1(lw.w_down, w.M, d, R, w.G1, c.d_ff, EPI_DOWN);
+            dn.Bc = Bc; dn.grouped = grouped; dn.coup = lw.coup_c; dn.S = w.S;
+            if ((st = run_linear<WT>(m, "linear_down", dn)) != DBT_OK) return st;
+        } else {
+            int E = c.n_experts, Fe = c.d_expert, km = kmax_of(c), Fs = c.n_shared_experts * Fe;
+            LinArgs rl = lin1(lw.router, w.rlogits, E, R, w.X, d);
+            if ((st = run_linear<WT>(m, "router", rl)) != DBT_OK) return st;
+            int32_t *last = record_experts ? w.last_experts + (size_t)l * 2 * c.max_batch * km : nullptr;
+            if (last && !grouped)
+                CUDA_TRY(m, cudaMemsetAsync(last + (size_t)c.max_batch * km, 0xff, sizeof(int32_t) * c.max_batch * km,
+                                            m->stream));
+            LAUNCH(m, "route", 0, route_kernel, R, 32, E * sizeof(float) + E, w.rlogits, E, Bc, c.k_primary, c.k_branch, km,
+                   c.router_mode == DBT_ROUTER_REPLAY, w.ridx, w.rwts, last, c.max_batch * km);
+            int32_t *ucnt = record_experts ? w.union_cnt + l : nullptr;
+            if (ucnt) CUDA_TRY(m, cudaMemsetAsync(ucnt, 0, sizeof(int32_t), m->stream));
+            LAUNCH(m, "moe_lists", 0, moe_lists_kernel, (E + 127) / 128, 128, 0, w.ridx, R, km, E, m->Rmax, w.ecnt, w.elist, ucnt);
+            dim3 g1((Fe + kLinWarps - 1) / kLinWarps, E);
+            LAUNCH(m, "expert_gateup", 0, expert_gateup_kernel<WT>, g1, kLinWarps * 32, 0, (const WT *)lw.exp_gate, (const WT *)lw.exp_up,
+                   Fe, d, w.X, km, w.ecnt, w.elist, m->Rmax, w.Hexp);
+            dim3 g2((d + kLinWarps - 1) / kLinWarps, E);
+            LAUNCH(m, "expert_down", 0, expert_down_kernel<WT>, g2, kLinWarps * 32, 0, (const WT *)lw.exp_down, Fe, d, w.Hexp, w.ecnt,
+                   w.elist, m->Rmax, w.Yexp);
+            const float *Msh = nullptr;
+            if (Fs > 0) {  // shared expert(s): every row of both paths; b couples its hidden state
+                LinArgs gu{};
+                gu.W[0] = lw.sh_gate; gu.W[1] = lw.sh_up; gu.Y[0] = w.Hsh; gu.n_out[0] = Fs; gu.rows[0] = R;
+                gu.nseg = 2; gu.X = w.X; gu.K = d; gu.epi = EPI_SWIGLU; gu.Bc = Bc; gu.grouped = grouped;
+                gu.coup = c.moe_b_coupling ? lw.coup_b : nullptr;
+                if ((st = run_linear<WT>(m, "shared_gateup", gu)) != DBT_OK) return st;
+                LinArgs dn = lin1(lw.sh_down, w.Msh, d, R, w.Hsh, Fs, EPI_STORE);
+                if ((st = run_linear<WT>(m, "shared_down", dn)) != DBT_OK) return st;
+                Msh = w.Msh;
+            }
+            LAUNCH(m, "moe_combine", 0, moe_combine_kernel, Bc, 256, 0, w.Yexp, Msh, w.ridx, w.rwts, km, Bc, grouped, lw.coup_c, d, w.S);
+        }
+    }
+    return DBT_OK;
+}
+
+// Final norm + shared output matrix on `rows` rows taken from S (row r*src_mul+src_add).
+template <typename WT>
+dbt_status run_head(dbt_model *m, int rows, int src_mul, int src_add) {
+    const dbt_config &c = m->cfg;
+    const Workspace &w = m->ws;
+    LAUNCH(m, "rmsnorm", 0, rmsnorm_kernel, rows, 256, 0, w.S, m->w.final_norm_g, c.rms_eps, c.d_model, src_mul, src_add,
+           c.final_norm, w.Zrows);
+    LinArgs a = lin1(m->w.lm_head, w.Z, c.vocab, rows, w.Zrows, c.d_model);
+    return run_linear<WT>(m, "lm_head", a);
+}
+
+template <typename WT>
+dbt_status step_impl(dbt_model *m, const int32_t *tokens_dev, int B, int grouped, int32_t *next_dev, float *z1_dev,
+                     float *z2_dev, float *alpha_dev) {
+    const dbt_config &c = m->cfg;
+    const Workspace &w = m->ws;
+    RowMap rm{B, 1};
+    int R = grouped ? 2 * B : B;
+    dbt_status st;
+    LAUNCH(m, "embed", 0, embed_norm_kernel<WT>, R, 256, 0, tokens_dev, 1, 0, rm, (const WT *)m->w.embed_primary,
+           (const WT *)m->w.embed_branch, m->w.embed_norm_g, c.rms_eps, c.d_model, c.vocab, w.S, w.status);
+    if ((st = run_layers<WT>(m, rm, grouped, true)) != DBT_OK) return st;
+    if ((st = run_head<WT>(m, R, 1, 0)) != DBT_OK) return st;
+    LAUNCH(m, "readout", 0, readout_kernel, B, 1024, 0, w.Z, B, c.vocab, grouped, next_dev, alpha_dev);
+    LAUNCH(m, "advance_len", 0, advance_len_kernel, (B + 127) / 128, 128, 0, w.seq_len, B, 1);
+    size_t zb = sizeof(float) * (size_t)B * c.vocab;
+    if (z1_dev) CUDA_TRY(m, cudaMemcpyAsync(z1_dev, w.Z, zb, cudaMemcpyDeviceToDevice, m->stream));
+    if (z2_dev && grouped)
+        CUDA_TRY(m, cudaMemcpyAsync(z2_dev, w.Z + (size_t)B * c.vocab, zb, cudaMemcpyDeviceToDevice, m->stream));
+    for (int b = 0; b < B; b++) m->len_host[b] += 1;
+    m->pending_union = c.n_experts > 0;
+    return DBT_OK;
+}
+
+template <typename WT>
+dbt_status prefill_impl(dbt_model *m, const int32_t *tokens_dev, int B, int n, float *last_logits) {
+    const dbt_config &c = m->cfg;
+    const Workspace &w = m->ws;
+    int cn_max = m->Rmax / B;
+    if (cn_max < 1) cn_max = 1;
+    dbt_status st;
+    for (int p0 = 0; p0 < n; p0 += cn_max) {
+        int cn = n - p0 < cn_max ? n - p0 : cn_max;
+        RowMap rm{B, cn};
+        int R = B * cn;
+        LAUNCH(m, "embed", 0, embed_norm_kernel<WT>, R, 256, 0, tokens_dev, n, p0, rm, (const WT *)m->w.embed_primary,
+               (const WT *)m->w.embed_branch, m->w.embed_norm_g, c.rms_eps, c.d_model, c.vocab, w.S, w.status);
+        if ((st = run_layers<WT>(m, rm, 0, false)) != DBT_OK) return st;
+        bool last = p0 + cn >= n;
+        if (last && last_logits) {
+            if ((st = run_head<WT>(m, B, cn, cn - 1)) != DBT_OK) return st;
+            CUDA_TRY(m, cudaMemcpyAsync(last_logits, w.Z, sizeof(float) * (size_t)B * c.vocab,
+                                        cudaMemcpyDeviceToDevice, m->stream));
+        }
+        LAUNCH(m, "advance_len", 0, advance_len_kernel, (B + 127) / 128, 128, 0, w.seq_len, B, cn);
+    }
+    for (int b = 0; b < B; b++) m->len_host[b] += n;
+    return DBT_OK;
+}
+
+dbt_status check_step_args(dbt_model *m, const int32_t *tokens, int B, int n) {
+    if (!m) return DBT_ERR_INVALID_ARG;
+    if (!tokens) return fail(m, DBT_ERR_INVALID_ARG, "tokens pointer is NULL");
+    if (B <= 0 || n <= 0) return fail(m, DBT_ERR_INVALID_ARG, "B and n must be positive");
+    if (B > m->cfg.max_batch) return fail(m, DBT_ERR_CAPACITY, "B=%d exceeds max_batch=%d", B, m->cfg.max_batch);
+    int cap = m->pages_per_seq * m->cfg.page_size;
+    if (cap > m->cfg.max_seq) cap = m->cfg.max_seq;
+    for (int b = 0; b < B; b++)
+        if (m->len_host[b] + n > cap)
+            return fail(m, DBT_ERR_CAPACITY, "sequence %d: %d + %d positions exceed capacity %d", b, m->len_host[b], n,
+                        cap);
+    return DBT_OK;
+}
+
+}  // namespace
+
+// ---------------------------------------------------------------------------------------
+
+extern "C" {
+
+const char *dbt_version(void) { return "dbt-b200 0.1 (sm_100a)"; }
+
+const char *dbt_last_error(const dbt_model *m) { return m ? m->err.c_str() : g_create_error.c_str(); }
+
+dbt_status dbt_query_sizes(const dbt_config *cfg, size_t *kv_bytes, size_t *workspace_bytes) {
+    dbt_status st;
+    const char *why = check_config(cfg, &st);
+    if (why) return fail(nullptr, st, "%s", why);
+    if (kv_bytes)
+        *kv_bytes = (size_t)cfg->n_layers * 2 * cfg->num_pages * cfg->n_kv_heads * cfg->page_size * cfg->head_dim *
+                    elem_bytes(*cfg);
+    if (workspace_bytes) *workspace_bytes = carve(*cfg, nullptr, nullptr, nullptr, nullptr);
+    return DBT_OK;
+}
+
+dbt_status dbt_create(const dbt_config *cfg, const dbt_weights *w, void *kv_pool_dev, void *workspace_dev,
+                      void *cuda_stream, dbt_model **out) {
+    if (out) *out = nullptr;
+    dbt_status st;
+    const char *why = check_config(cfg, &st);
+    if (why) return fail(nullptr, st, "%s", why);
+    if (!w || !kv_pool_dev || !workspace_dev || !out || !w->layers)
+        return fail(nullptr, DBT_ERR_INVALID_ARG, "NULL pointer argument");
+    if (((uintptr_t)kv_pool_dev | (uintptr_t)workspace_dev) & 255)
+        return fail(nullptr, DBT_ERR_INVALID_ARG, "kv pool and workspace must be 256-byte aligned");
+    bool moe = cfg->n_experts > 0;
+    if (!w->embed_primary || !w->embed_branch || !w->embed_norm_g || !w->lm_head || (cfg->final_norm && !w->final_norm_g))
+        return fail(nullptr, DBT_ERR_INVALID_ARG, "NULL top-level weight pointer");
+    for (int l = 0; l < cfg->n_layers; l++) {
+        const dbt_layer_weights &lw = w->layers[l];
+        bool ok = lw.attn_norm_g && lw.wq && lw.wk && lw.wv && lw.wo && lw.coup_a && lw.mlp_norm_g && lw.coup_c;
+        if (moe) {
+            ok = ok && lw.router && lw.exp_gate && lw.exp_up && lw.exp_down;
+            if (cfg->n_shared_experts > 0)
+                ok = ok && lw.sh_gate && lw.sh_up && lw.sh_down && (!cfg->moe_b_coupling || lw.coup_b);
+        } else {
+            ok = ok && lw.w_gate && lw.w_up && lw.w_down && lw.coup_b;
+        }
+        if (!ok) return fail(nullptr, DBT_ERR_INVALID_ARG, "NULL weight pointer in layer %d", l);
+    }
+    dbt_model *m = new (std::nothrow) dbt_model();
+    if (!m) return fail(nullptr, DBT_ERR_INVALID_ARG, "out of host memory");
+    m->cfg = *cfg;
+    m->w = *w;
+    m->layers.assign(w->layers, w->layers + cfg->n_layers);
+    m->w.layers = m->layers.data();
+    m->stream = (cudaStream_t)cuda_stream;
+    m->kv_pool = (char *)kv_pool_dev;
+    m->ws_base = (char *)workspace_dev;
+    m->ws_bytes = carve(*cfg, m->ws_base, &m->ws, &m->Rmax, &m->part_items);
+    m->pages_per_seq_max = (cfg->max_seq + cfg->page_size - 1) / cfg->page_size;
+    m->pages_per_seq = m->pages_per_seq_max;
+    m->len_host.assign(cfg->max_batch, 0);
+    m->launches = 0;
+    m->pending_union = false;
+    m->prof_on = false;
+
+    // RoPE table in double: angle = t * base^(-2i/d_h), stored as (cos, sin) fp32 pairs.
+    int half = cfg->head_dim / 2;
+    std::vector<float2> tab((size_t)cfg->max_seq * half);
+    std::vector<double> inv_freq(half);
+    for (int i = 0; i < half; i++) inv_freq[i] = std::exp(-std::log((double)cfg->rope_base) * (2.0 * i) / cfg->head_dim);
+    for (int t = 0; t < cfg->max_seq; t++)
+        for (int i = 0; i < half; i++) {
+            double ang = (double)t * inv_freq[i];
+            tab[(size_t)t * half + i] = make_float2((float)std::cos(ang), (float)std::sin(ang));
+        }
+    // Default page table: sequence b owns a contiguous run of pages (clamped into the pool;
+    // capacity checks use the pool size).
+    std::vector<int32_t> pt((size_t)cfg->max_batch * m->pages_per_seq_max);
+    for (int b = 0; b < cfg->max_batch; b++)
+        for (int p = 0; p < m->pages_per_seq_max; p++) {
+            long long id = (long long)b * m->pages_per_seq_max + p;
+            pt[(size_t)b * m->pages_per_seq_max + p] = id < cfg->num_pages ? (int32_t)id : -1;
+        }
+    cudaError_t e = cudaMemcpyAsync(m->ws.rope, tab.data(), tab.size() * sizeof(float2), cudaMemcpyHostToDevice, m->stream);
+    if (e == cudaSuccess)
+        e = cudaMemcpyAsync(m->ws.page_table, pt.data(), pt.size() * sizeof(int32_t), cudaMemcpyHostToDevice, m->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(m->ws.seq_len, 0, sizeof(int32_t) * cfg->max_batch, m->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(m->ws.status, 0, sizeof(int32_t) * 4, m->stream);
+    if (e == cudaSuccess && moe) {
+        e = cudaMemsetAsync(m->ws.last_experts, 0xff, sizeof(int32_t) * (size_t)cfg->n_layers * 2 * cfg->max_batch * kmax_of(*cfg), m->stream);
+        if (e == cudaSuccess) e = cudaMemsetAsync(m->ws.union_cnt, 0, sizeof(int32_t) * cfg->n_layers, m->stream);
+    }
+    if (e == cudaSuccess) e = cudaStreamSynchronize(m->stream);  // the host vectors go out of scope
+    if (e != cudaSuccess) {
+        fail(nullptr, DBT_ERR_CUDA, "dbt_create: %s", cudaGetErrorString(e));
+        delete m;
+        return DBT_ERR_CUDA;
+    }
+    if ((long long)cfg->max_batch * m->pages_per_seq_max > cfg->num_pages) {
+        // the default table cannot give every sequence max_seq positions: shrink per-sequence capacity
+        m->pages_per_seq = cfg->num_pages / cfg->max_batch;
+        if (m->pages_per_seq < 1) {
+            fail(nullptr, DBT_ERR_CAPACITY, "num_pages=%d cannot hold one page per sequence", cfg->num_pages);
+            delete m;
+            return DBT_ERR_CAPACITY;
+        }
+        std::vector<int32_t> pt2((size_t)cfg->max_batch * m->pages_per_seq_max, -1);
+        for (int b = 0; b < cfg->max_batch; b++)
+            for (int p = 0; p < m->pages_per_seq; p++) pt2[(size_t)b * m->pages_per_seq_max + p] = b * m->pages_per_seq + p;
+        e = cudaMemcpy(m->ws.page_table, pt2.data(), pt2.size() * sizeof(int32_t), cudaMemcpyHostToDevice);
+        if (e != cudaSuccess) {
+            fail(nullptr, DBT_ERR_CUDA, "dbt_create: %s", cudaGetErrorString(e));
+            delete m;
+            return DBT_ERR_CUDA;
+        }
+    }
+    *out = m;
+    return DBT_OK;
+}
+
+void dbt_destroy(dbt_model *m) {
+    if (!m) return;
+    for (auto &r : m->prof) {
+        cudaEventDestroy(r.e0);
+        cudaEventDestroy(r.e1);
+    }
+    for (auto e : m->prof_pool) cudaEventDestroy(e);
+    delete m;
+}
+
+dbt_status dbt_profile_begin(dbt_model *m) {
+    if (!m) return DBT_ERR_INVALID_ARG;
+    for (auto &r : m->prof) {
+        m->prof_pool.push_back(r.e0);
+        m->prof_pool.push_back(r.e1);
+    }
+    m->prof.clear();
+    m->prof_on = true;
+    return DBT_OK;
+}
+
+dbt_status dbt_profile_end(dbt_model *m, dbt_profile_entry *entries_host, int32_t max_entries, int32_t *n_entries) {
+    if (!m) return DBT_ERR_INVALID_ARG;
+    if (!entries_host || !n_entries || max_entries <= 0) return fail(m, DBT_ERR_INVALID_ARG, "bad profile buffer");
+    m->prof_on = false;
+    CUDA_TRY(m, cudaStreamSynchronize(m->stream));
+    int n = 0;
+    for (auto &r : m->prof) {
+        float ms = 0.f;
+        CUDA_TRY(m, cudaEventElapsedTime(&ms, r.e0, r.e1));
+        int i = 0;
+        while (i < n && strncmp(entries_host[i].name, r.tag, sizeof entries_host[i].name) != 0) i++;
+        if (i == n) {
+            if (n == max_entries) continue;
+            memset(&entries_host[n], 0, sizeof entries_host[n]);
+            strncpy(entries_host[n].name, r.tag, sizeof entries_host[n].name - 1);
+            n++;
+        }
+        entries_host[i].launches += 1;
+        entries_host[i].total_ms += ms;
+        entries_host[i].bytes += r.bytes;
+    }
+    for (auto &r : m->prof) {
+        m->prof_pool.push_back(r.e0);
+        m->prof_pool.push_back(r.e1);
+    }
+    m->prof.clear();
+    *n_entries = n;
+    return DBT_OK;
+}
+
+dbt_status dbt_set_page_table(dbt_model *m, const int32_t *table_host, int32_t B, int32_t pages_per_seq) {
+    if (!m) return DBT_ERR_INVALID_ARG;
+    if (!table_host || B <= 0 || pages_per_seq <= 0) return fail(m, DBT_ERR_INVALID_ARG, "bad page-table argument");
+    if (B > m->cfg.max_batch || pages_per_seq > m->pages_per_seq_max)
+        return fail(m, DBT_ERR_CAPACITY, "page table [%d][%d] exceeds [%d][%d]", B, pages_per_seq, m->cfg.max_batch,
+                    m->pages_per_seq_max);
+    std::vector<char> seen(m->cfg.num_pages, 0);
+    std::vector<int32_t> pt((size_t)m->cfg.max_batch * m->pages_per_seq_max, -1);
+    for (int b = 0; b < B; b++)
+        for (int p = 0; p < pages_per_seq; p++) {
+            int32_t id = table_host[(size_t)b * pages_per_seq + p];
+            if (id < 0 || id >= m->cfg.num_pages) return fail(m, DBT_ERR_INVALID_ARG, "page id %d out of range", id);
+            if (seen[id]) return fail(m, DBT_ERR_INVALID_ARG, "page id %d appears twice", id);
+            seen[id] = 1;
+            pt[(size_t)b * m->pages_per_seq_max + p] = id;
+        }
+    CUDA_TRY(m, cudaStreamSynchronize(m->stream));
+    CUDA_TRY(m, cudaMemcpy(m->ws.page_table, pt.data(), pt.size() * sizeof(int32_t), cudaMemcpyHostToDevice));
+    m->pages_per_seq = pages_per_seq;
+    return DBT_OK;
+}
+
+dbt_status dbt_reset(dbt_model *m) {
+    if (!m) return DBT_ERR_INVALID_ARG;
+    CUDA_TRY(m, cudaMemsetAsync(m->ws.seq_len, 0, sizeof(int32_t) * m->cfg.max_batch, m->stream));
+    CUDA_TRY(m, cudaMemsetAsync(m->ws.status, 0, sizeof(int32_t) * 4, m->stream));
+    std::fill(m->len_host.begin(), m->len_host.end(), 0);
+    return DBT_OK;
+}
+
+dbt_status dbt_set_seq_lens(dbt_model *m, const int32_t *lens_host, int32_t B) {
+    if (!m) return DBT_ERR_INVALID_ARG;
+    if (!lens_host || B <= 0 || B > m->cfg.max_batch) return fail(m, DBT_ERR_INVALID_ARG, "bad argument");
+    int cap = m->pages_per_seq * m->cfg.page_size;
+    if (cap > m->cfg.max_seq) cap = m->cfg.max_seq;
+    for (int b = 0; b < B; b++)
+        if (lens_host[b] < 0 || lens_host[b] > cap) return fail(m, DBT_ERR_CAPACITY, "length %d out of range", lens_host[b]);
+    CUDA_TRY(m, cudaStreamSynchronize(m->stream));
+    CUDA_TRY(m, cudaMemcpy(m->ws.seq_len, lens_host, sizeof(int32_t) * B, cudaMemcpyHostToDevice));
+    for (int b = 0; b < B; b++) m->len_host[b] = lens_host[b];
+    return DBT_OK;
+}
+
+int32_t dbt_seq_len(const dbt_model *m, int32_t b) {
+    if (!m || b < 0 || b >= m->cfg.max_batch) return -1;
+    return m->len_host[b];
+}
+
+dbt_status dbt_prefill(dbt_model *m, const int32_t *tokens_dev, int32_t B, int32_t n, float *last_primary_logits_dev) {
+    dbt_status st = check_step_args(m, tokens_dev, B, n);
+    if (st != DBT_OK) return st;
+    if (m->cfg.weight_dtype == DBT_DTYPE_F32) return prefill_impl<float>(m, tokens_dev, B, n, last_primary_logits_dev);
+    return prefill_impl<__nv_bfloat16>(m, tokens_dev, B, n, last_primary_logits_dev);
+}
+
+dbt_status dbt_decode_step(dbt_model *m, const int32_t *tokens_dev, int32_t B, int32_t *next_tokens_dev,
+                           float *logits_primary_dev, float *logits_branch_dev, float *alpha_dev) {
+    dbt_status st = check_step_args(m, tokens_dev, B, 1);
+    if (st != DBT_OK) return st;
+    if (m->cfg.weight_dtype == DBT_DTYPE_F32)
+        return step_impl<float>(m, tokens_dev, B, 1, next_tokens_dev, logits_primary_dev, logits_branch_dev, alpha_dev);
+    return step_impl<__nv_bfloat16>(m, tokens_dev, B, 1, next_tokens_dev, logits_primary_dev, logits_branch_dev, alpha_dev);
+}
+
+dbt_status dbt_decode_step_primary_only(dbt_model *m, const int32_t *tokens_dev, int32_t B, int32_t *next_tokens_dev,
+                                        float *logits_primary_dev) {
+    dbt_status st = check_step_args(m, tokens_dev, B, 1);
+    if (st != DBT_OK) return st;
+    if (m->cfg.weight_dtype == DBT_DTYPE_F32)
+        return step_impl<float>(m, tokens_dev, B, 0, next_tokens_dev, logits_primary_dev, nullptr, nullptr);
+    return step_impl<__nv_bfloat16>(m, tokens_dev, B, 0, next_tokens_dev, logits_primary_dev, nullptr, nullptr);
+}
+
+static dbt_status step_host(dbt_model *m, const int32_t *tokens_host, int32_t B, int32_t *next_host, float *alpha_host,
+                            int grouped) {
+    if (!m) return DBT_ERR_INVALID_ARG;
+    if (!tokens_host || !next_host) return fail(m, DBT_ERR_INVALID_ARG, "NULL host buffer");
+    if (B <= 0 || B > m->cfg.max_batch) return fail(m, DBT_ERR_CAPACITY, "B=%d out of range", B);
+    const Workspace &w = m->ws;
+    CUDA_TRY(m, cudaMemcpyAsync(w.tokens_stage, tokens_host, sizeof(int32_t) * B, cudaMemcpyHostToDevice, m->stream));
+    dbt_status st = grouped ? dbt_decode_step(m, w.tokens_stage, B, w.next_stage, nullptr, nullptr, w.alpha_stage)
+                            : dbt_decode_step_primary_only(m, w.tokens_stage, B, w.next_stage, nullptr);
+    if (st != DBT_OK) return st;
+    CUDA_TRY(m, cudaMemcpyAsync(next_host, w.next_stage, sizeof(int32_t) * B, cudaMemcpyDeviceToHost, m->stream));
+    if (alpha_host && grouped)
+        CUDA_TRY(m, cudaMemcpyAsync(alpha_host, w.alpha_stage, sizeof(float) * B, cudaMemcpyDeviceToHost, m->stream));
+    CUDA_TRY(m, cudaStreamSynchronize(m->stream));
+    return DBT_OK;
+}
+
+dbt_status dbt_decode_step_host(dbt_model *m, const int32_t *tokens_host, int32_t B, int32_t *next_tokens_host,
+                                float *alpha_host) {
+    return step_host(m, tokens_host, B, next_tokens_host, alpha_host, 1);
+}
+
+dbt_status dbt_decode_step_primary_only_host(dbt_model *m, const int32_t *tokens_host, int32_t B,
+                                             int32_t *next_tokens_host) {
+    return step_host(m, tokens_host, B, next_tokens_host, nullptr, 0);
+}
+
+dbt_status dbt_last_experts(dbt_model *m, const int32_t **experts_dev, int32_t *kmax) {
+    if (!m) return DBT_ERR_INVALID_ARG;
+    if (m->cfg.n_experts == 0) return fail(m, DBT_ERR_STATE, "not an MoE model");
+    if (experts_dev) *experts_dev = m->ws.last_experts;
+    if (kmax) *kmax = kmax_of(m->cfg);
+    return DBT_OK;
+}
+
+dbt_status dbt_last_expert_union(dbt_model *m, int32_t *count_per_layer_host) {
+    if (!m) return DBT_ERR_INVALID_ARG;
+    if (m->cfg.n_experts == 0) return fail(m, DBT_ERR_STATE, "not an MoE model");
+    if (!count_per_layer_host) return fail(m, DBT_ERR_INVALID_ARG, "NULL output");
+    CUDA_TRY(m, cudaStreamSynchronize(m->stream));
+    CUDA_TRY(m, cudaMemcpy(count_per_layer_host, m->ws.union_cnt, sizeof(int32_t) * m->cfg.n_layers, cudaMemcpyDeviceToHost));
+    return DBT_OK;
+}
+
+dbt_status dbt_sync_status(dbt_model *m, int32_t *device_status, int32_t *detail) {
+    if (!m) return DBT_ERR_INVALID_ARG;
+    int32_t h[2] = {0, 0};
+    CUDA_TRY(m, cudaStreamSynchronize(m->stream));
+    CUDA_TRY(m, cudaMemcpy(h, m->ws.status, sizeof h, cudaMemcpyDeviceToHost));
+    if (device_status) *device_status = h[0];
+    if (detail) *detail = h[1];
+    if (h[0] != 0) return fail(m, DBT_ERR_DEVICE, "device status %d (detail %d)", h[0], h[1]);
+    return DBT_OK;
+}
+
+int64_t dbt_launch_count(const dbt_model *m) { return m ? m->launches : 0; }
+
+}  // extern "C"

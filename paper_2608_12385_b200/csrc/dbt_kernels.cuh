@@ -1,0 +1,587 @@
+// Generic kernels of the Decode-Branch step, templated on the storage type (fp32 / bf16).
+// These cover every operation of the step with fp32 arithmetic on the CUDA cores: they are
+// the fp32-model path and the fallback for shapes the tensor-core kernels do not take.
+// All reductions use fixed trees and fixed orders: results are run-to-run deterministic and
+// a primary row's value never depends on whether branch rows are present.
+#pragma once
+
+#include "dbt_common.cuh"
+
+namespace dbt {
+
+// ---------------------------------------------------------------------------------------
+// Eq. embeddings: S_1^0 = RMSNorm(E_1[x]), S_2^0 = RMSNorm(E_2[x]).  One block per row.
+template <typename WT>
+__global__ void embed_norm_kernel(const int32_t *__restrict__ tokens, int n, int p0, RowMap rm,
+                                  const WT *__restrict__ E1, const WT *__restrict__ E2,
+                                  const float *__restrict__ g, float eps, int d, int V,
+                                  float *__restrict__ S, int *status) {
+    __shared__ float scratch[32];
+    int r = blockIdx.x;
+    int path = r >= rm.Bc();
+    int tok = tokens[(size_t)rm.seq(r) * n + p0 + rm.off(r)];
+    if (tok < 0 || tok >= V) {
+        if (threadIdx.x == 0) report(status, kStatusBadToken, tok);
+        tok = min(max(tok, 0), V - 1);
+    }
+    const WT *e = (path ? E2 : E1) + (size_t)tok * d;
+    float ss = 0.f;
+    for (int i = threadIdx.x; i < d; i += blockDim.x) {
+        float x = load1(e + i);
+        ss += x * x;
+    }
+    ss = block_sum(ss, scratch);
+    float inv = 1.f / sqrtf(ss / (float)d + eps);
+    for (int i = threadIdx.x; i < d; i += blockDim.x) S[(size_t)r * d + i] = g[i] * load1(e + i) * inv;
+}
+
+// N = RMSNorm(S) (gain g, or no gain when g == nullptr: plain copy scaled by 1).
+// Output row r reads input row r * src_mul + src_add (a gather for "last position" rows).
+__global__ void rmsnorm_kernel(const float *__restrict__ S, const float *__restrict__ g, float eps, int d,
+                               int src_mul, int src_add, int apply, float *__restrict__ N) {
+    __shared__ float scratch[32];
+    int r = blockIdx.x;
+    const float *x = S + ((size_t)r * src_mul + src_add) * d;
+    float inv = 1.f;
+    if (apply) {
+        float ss = 0.f;
+        for (int i = threadIdx.x; i < d; i += blockDim.x) ss += x[i] * x[i];
+        ss = block_sum(ss, scratch);
+        inv = 1.f / sqrtf(ss / (float)d + eps);
+    }
+    for (int i = threadIdx.x; i < d; i += blockDim.x)
+        N[(size_t)r * d + i] = apply ? g[i] * x[i] * inv : x[i];
+}
+
+// ---------------------------------------------------------------------------------------
+// Skinny linear layer on the CUDA cores: Y[r][f] = sum_k W[f][k] X[r][k].
+// One warp per output feature; the warp walks the weight row once per group of RT rows with
+// 128-bit loads.  Up to three weight segments share one launch (Q|K|V).
+
+enum : int { EPI_STORE = 0, EPI_RESID = 1, EPI_SWIGLU = 2, EPI_DOWN = 3 };
+
+struct LinArgs {
+    const void *W[3];
+    float *Y[3];
+    int n_out[3];
+    int rows[3];
+    int nseg;
+    const float *X;  // [rows][K]
+    int K;
+    int epi;
+    int Bc;       // primary rows in this launch
+    int grouped;  // branch rows Bc..2Bc-1 present
+    const float *coup;  // b (EPI_SWIGLU) or c (EPI_DOWN); nullptr = no coupling
+    float *S;     // residual rows [.][n_out[0]] for EPI_RESID / EPI_DOWN
+};
+
+constexpr int kLinWarps = 8;
+constexpr int kLinRT = 8;
+
+template <typename WT, int RT>
+__device__ __forceinline__ void warp_dots(const WT *__restrict__ wrow, const float *const (&xp)[RT], int K,
+                                          float (&acc)[RT]) {
+    int lane = threadIdx.x & 31;
+#pragma unroll
+    for (int r = 0; r < RT; r++) acc[r] = 0.f;
+    for (int k = lane * 8; k < K; k += 256) {
+        float w[8];
+        load8(wrow + k, w);
+#pragma unroll
+        for (int r = 0; r < RT; r++) {
+            if (xp[r] != nullptr) {
+                float x[8];
+                load8(xp[r] + k, x);
+#pragma unroll
+                for (int i = 0; i < 8; i++) acc[r] = fmaf(w[i], x[i], acc[r]);
+            }
+        }
+    }
+#pragma unroll
+    for (int r = 0; r < RT; r++) acc[r] = warp_sum(acc[r]);
+}
+
+template <typename WT>
+__global__ void __launch_bounds__(kLinWarps * 32) linear_kernel(LinArgs a) {
+    int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    int f = blockIdx.x * kLinWarps + warp;
+    int seg = 0;
+    if (a.epi != EPI_SWIGLU) {
+        while (seg < a.nseg && f >= a.n_out[seg]) {
+            f -= a.n_out[seg];
+            seg++;
+        }
+        if (seg >= a.nseg) return;
+    } else if (f >= a.n_out[0]) {
+        return;
+    }
+    int K = a.K, rows = a.rows[seg], n_out = a.n_out[seg];
+    const WT *w0 = reinterpret_cast<const WT *>(a.W[seg]) + (size_t)f * K;
+    float *Y = a.Y[seg];
+    for (int r0 = 0; r0 < rows; r0 += kLinRT) {
+        const float *xp[kLinRT];
+#pragma unroll
+        for (int r = 0; r < kLinRT; r++) xp[r] = (r0 + r < rows) ? a.X + (size_t)(r0 + r) * K : nullptr;
+        float acc[kLinRT];
+        warp_dots<WT, kLinRT>(w0, xp, K, acc);
+        if (a.epi == EPI_SWIGLU) {
+            float up[kLinRT];
+            const WT *w1 = reinterpret_cast<const WT *>(a.W[1]) + (size_t)f * K;
+            warp_dots<WT, kLinRT>(w1, xp, K, up);
+#pragma unroll
+            for (int r = 0; r < kLinRT; r++) acc[r] = silu(acc[r]) * up[r];
+        }
+#pragma unroll
+        for (int r = 0; r < kLinRT; r++) {
+            if (lane == r && r0 + r < rows) {
+                size_t o = (size_t)(r0 + r) * n_out + f;
+                if (a.epi == EPI_RESID)
+                    a.S[o] += acc[r];
+                else
+                    Y[o] = acc[r];
+            }
+        }
+    }
+    if (a.epi == EPI_SWIGLU && a.grouped && a.coup != nullptr) {
+        // H~_2 = H_2 + b * H_1 (Eq. mlp), feature f of every sequence
+        __syncwarp();
+        float bf = a.coup[f];
+        for (int b = lane; b < a.Bc; b += 32) Y[(size_t)(a.Bc + b) * n_out + f] += bf * Y[(size_t)b * n_out + f];
+    } else if (a.epi == EPI_DOWN) {
+        // M_2 += c * M_1 ; S_i^{l+1} = S-bar_i + M_i (Eq. mlp)
+        __syncwarp();
+        float cf = (a.grouped && a.coup != nullptr) ? a.coup[f] : 0.f;
+        for (int b = lane; b < a.Bc; b += 32) {
+            float m1 = Y[(size_t)b * n_out + f];
+            a.S[(size_t)b * n_out + f] += m1;
+            if (a.grouped) a.S[(size_t)(a.Bc + b) * n_out + f] += Y[(size_t)(a.Bc + b) * n_out + f] + cf * m1;
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// RoPE on Q (both paths) and K (primary), the a coupling Q~_2 = Q_2 + a*Q_1 (Eq. asymattn)
+// and the append of K_1,V_1 to the paged cache (Section 4.4 item 3).  One block per primary
+// row, which also handles its branch twin.
+template <typename KT>
+__global__ void rope_couple_append_kernel(float *__restrict__ Q, const float *__restrict__ Kn,
+                                          const float *__restrict__ Vn, RowMap rm, int grouped, int n_q,
+                                          int n_kv, int dh, const float *__restrict__ coup_a,
+                                          const float2 *__restrict__ rope_tab, const int32_t *__restrict__ seq_len,
+                                          const int32_t *__restrict__ page_table, int pt_stride, int num_pages,
+                                          int page_size, KT *__restrict__ kpool, KT *__restrict__ vpool, int *status) {
+    int item = blockIdx.x, Bc = rm.Bc();
+    int seq = rm.seq(item), pos = seq_len[seq] + rm.off(item);
+    int half = dh / 2, q_dim = n_q * dh, kv_dim = n_kv * dh;
+    const float2 *cs = rope_tab + (size_t)pos * half;
+    float *q1 = Q + (size_t)item * q_dim;
+    float *q2 = Q + (size_t)(Bc + item) * q_dim;
+    for (int idx = threadIdx.x; idx < n_q * half; idx += blockDim.x) {
+        int h = idx / half, i = idx % half;
+        float2 t = cs[i];
+        int o0 = h * dh + i, o1 = o0 + half;
+        float x0 = q1[o0], x1 = q1[o1];
+        float r0 = x0 * t.x - x1 * t.y, r1 = x1 * t.x + x0 * t.y;
+        q1[o0] = r0;
+        q1[o1] = r1;
+        if (grouped) {
+            float y0 = q2[o0], y1 = q2[o1];
+            q2[o0] = (y0 * t.x - y1 * t.y) + coup_a[o0] * r0;
+            q2[o1] = (y1 * t.x + y0 * t.y) + coup_a[o1] * r1;
+        }
+    }
+    int page = page_table[(size_t)seq * pt_stride + pos / page_size];
+    if (page < 0 || page >= num_pages) {
+        if (threadIdx.x == 0) report(status, kStatusBadPage, page);
+        return;
+    }
+    int slot = pos % page_size;
+    const float *kn = Kn + (size_t)item * kv_dim, *vn = Vn + (size_t)item * kv_dim;
+    for (int idx = threadIdx.x; idx < n_kv * half; idx += blockDim.x) {
+        int g = idx / half, i = idx % half;
+        float2 t = cs[i];
+        size_t base = (((size_t)page * n_kv + g) * page_size + slot) * dh;
+        float x0 = kn[g * dh + i], x1 = kn[g * dh + i + half];
+        store1(kpool + base + i, x0 * t.x - x1 * t.y);
+        store1(kpool + base + i + half, x1 * t.x + x0 * t.y);
+        store1(vpool + base + i, vn[g * dh + i]);
+        store1(vpool + base + i + half, vn[g * dh + i + half]);
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// Grouped decode attention, CUDA-core version.  One block per (primary row, KV head, split):
+// the G primary query heads of that KV head and, in grouped mode, the G coupled branch
+// heads read each K/V position once.  Keys 0..pos inclusive (the K/V appended this step is
+// already in its page).  Partial (m, l, acc) per split; a second kernel merges in split
+// order.
+template <typename KT, int NQ, int DH>
+__global__ void __launch_bounds__(128) attn_partial_kernel(
+    const float *__restrict__ Q, RowMap rm, int grouped, int G, int n_kv, const KT *__restrict__ kpool,
+    const KT *__restrict__ vpool, const int32_t *__restrict__ page_table, int pt_stride, int num_pages,
+    const int32_t *__restrict__ seq_len, int nsplit, float *__restrict__ part, int *status) {
+    constexpr int TPB = 128, CH = 128, PS = 16, SUB = TPB / DH;
+    __shared__ float qs[NQ][DH];
+    __shared__ float sc[NQ][CH];
+    __shared__ float m_s[NQ], l_s[NQ], corr_s[NQ];
+    __shared__ int pg[CH / PS];
+    int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    int item = blockIdx.x, g = blockIdx.y, sp = blockIdx.z;
+    int Bc = rm.Bc(), seq = rm.seq(item);
+    int nkeys = seq_len[seq] + rm.off(item) + 1;
+    int nq_act = grouped ? 2 * G : G, q_dim = n_kv * G * DH;
+    float scale = 1.f / sqrtf((float)DH);
+    for (int idx = tid; idx < NQ * DH; idx += TPB) {
+        int q = idx / DH, e = idx % DH;
+        float v = 0.f;
+        if (q < nq_act) {
+            int row = q < G ? item : Bc + item;
+            int h = g * G + (q < G ? q : q - G);
+            v = Q[(size_t)row * q_dim + h * DH + e] * scale;
+        }
+        qs[q][e] = v;
+    }
+    if (tid < NQ) {
+        m_s[tid] = -INFINITY;
+        l_s[tid] = 0.f;
+    }
+    int total_pages = (nkeys + PS - 1) / PS;
+    int pps = (total_pages + nsplit - 1) / nsplit;
+    int pb = sp * pps, pe = min(total_pages, pb + pps);
+    int jbeg = pb * PS, jend = min(nkeys, pe * PS);
+    float acc[NQ];
+#pragma unroll
+    for (int q = 0; q < NQ; q++) acc[q] = 0.f;
+    __syncthreads();
+    for (int j0 = jbeg; j0 < jend; j0 += CH) {
+        if (tid < CH / PS) {
+            int p = j0 / PS + tid, page = 0;
+            if (p < pe) {
+                page = page_table[(size_t)seq * pt_stride + p];
+                if (page < 0 || page >= num_pages) {
+                    report(status, kStatusBadPage, page);
+                    page = 0;
+                }
+            }
+            pg[tid] = page;
+        }
+        __syncthreads();
+        bool valid = j0 + tid < jend;
+        float dots[NQ];
+#pragma unroll
+        for (int q = 0; q < NQ; q++) dots[q] = 0.f;
+        if (valid) {
+            const KT *kp = kpool + (((size_t)pg[tid / PS] * n_kv + g) * PS + (tid % PS)) * DH;
+            for (int e = 0; e < DH; e += 8) {
+                float kv[8];
+                load8(kp + e, kv);
+#pragma unroll
+                for (int q = 0; q < NQ; q++)
+#pragma unroll
+                    for (int i = 0; i < 8; i++) dots[q] = fmaf(kv[i], qs[q][e + i], dots[q]);
+            }
+        }
+#pragma unroll
+        for (int q = 0; q < NQ; q++) sc[q][tid] = valid ? dots[q] : -INFINITY;
+        __syncthreads();
+        for (int q = warp; q < NQ; q += TPB / 32) {
+            float mx = -INFINITY;
+#pragma unroll
+            for (int i = 0; i < CH / 32; i++) mx = fmaxf(mx, sc[q][lane + 32 * i]);
+            mx = warp_max(mx);
+            float mold = m_s[q], mnew = fmaxf(mold, mx), s = 0.f;
+#pragma unroll
+            for (int i = 0; i < CH / 32; i++) {
+                float x = sc[q][lane + 32 * i];
+                float p = (x == -INFINITY) ? 0.f : expf(x - mnew);
+                sc[q][lane + 32 * i] = p;
+                s += p;
+            }
+            s = warp_sum(s);
+            __syncwarp();
+            if (lane == 0) {
+                float c = (mold == -INFINITY) ? 0.f : expf(mold - mnew);
+                corr_s[q] = c;
+                l_s[q] = l_s[q] * c + s;
+                m_s[q] = mnew;
+            }
+        }
+        __syncthreads();
+        int e = tid % DH, sub = tid / DH, cnt = min(CH, jend - j0);
+#pragma unroll
+        for (int q = 0; q < NQ; q++) acc[q] *= corr_s[q];
+        for (int jj = sub; jj < cnt; jj += SUB) {
+            float v = load1(vpool + (((size_t)pg[jj / PS] * n_kv + g) * PS + (jj % PS)) * DH + e);
+#pragma unroll
+            for (int q = 0; q < NQ; q++) acc[q] = fmaf(sc[q][jj], v, acc[q]);
+        }
+        __syncthreads();
+    }
+    if (SUB > 1) {  // fold the token subsets in a fixed order
+#pragma unroll
+        for (int q = 0; q < NQ; q++) sc[q][tid] = acc[q];
+        __syncthreads();
+        if (tid < DH) {
+#pragma unroll
+            for (int q = 0; q < NQ; q++) {
+                float t = sc[q][tid];
+                for (int s2 = 1; s2 < SUB; s2++) t += sc[q][s2 * DH + tid];
+                acc[q] = t;
+            }
+        }
+    }
+    float *out = part + (((size_t)item * n_kv + g) * nsplit + sp) * NQ * (DH + 2);
+    if (tid < DH) {
+#pragma unroll
+        for (int q = 0; q < NQ; q++) out[(size_t)q * (DH + 2) + tid] = acc[q];
+    }
+    if (tid < NQ) {
+        out[(size_t)tid * (DH + 2) + DH] = m_s[tid];
+        out[(size_t)tid * (DH + 2) + DH + 1] = l_s[tid];
+    }
+}
+
+// Merge the split partials in split order (log-sum-exp), write O [rows][q_dim].
+__global__ void attn_merge_kernel(const float *__restrict__ part, int nsplit, int NQ, int DH, int Bc, int grouped,
+                                  int G, int n_kv, float *__restrict__ O) {
+    int item = blockIdx.x, g = blockIdx.y, e = threadIdx.x;
+    int nq_act = grouped ? 2 * G : G, q_dim = n_kv * G * DH;
+    const float *base = part + ((size_t)item * n_kv + g) * nsplit * NQ * (DH + 2);
+    for (int q = 0; q < nq_act; q++) {
+        float M = -INFINITY;
+        for (int s = 0; s < nsplit; s++) M = fmaxf(M, base[((size_t)s * NQ + q) * (DH + 2) + DH]);
+        float L = 0.f, o = 0.f;
+        for (int s = 0; s < nsplit; s++) {
+            const float *p = base + ((size_t)s * NQ + q) * (DH + 2);
+            float ms = p[DH];
+            float w = (ms == -INFINITY) ? 0.f : expf(ms - M);
+            L += p[DH + 1] * w;
+            o += p[e] * w;
+        }
+        int row = q < G ? item : Bc + item;
+        int h = g * G + (q < G ? q : q - G);
+        O[(size_t)row * q_dim + h * DH + e] = o / L;
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// Readout (Eq. alpha, Eq. mixloss): p = softmax(z_1), q = softmax(z_2),
+// alpha = clip_[0.5,1](sum p^2), next = argmax(alpha p + (1-alpha) q), lowest index on ties.
+// Primary-only: next = argmax z_1.  One block per sequence.
+struct ArgBest {
+    float v;
+    int i;
+};
+__device__ __forceinline__ ArgBest better(ArgBest a, ArgBest b) {
+    if (b.v > a.v || (b.v == a.v && b.i < a.i)) return b;
+    return a;
+}
+
+__global__ void __launch_bounds__(1024) readout_kernel(const float *__restrict__ Z, int B, int V, int grouped,
+                                                       int32_t *__restrict__ next, float *__restrict__ alpha_out) {
+    __shared__ float scratch[32];
+    __shared__ float bv[32];
+    __shared__ int bi[32];
+    int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nw = blockDim.x >> 5;
+    const float *z1 = Z + (size_t)b * V, *z2 = Z + (size_t)(B + b) * V;
+    float m1 = -INFINITY, m2 = -INFINITY, d1 = 1.f, d2 = 1.f, alpha = 1.f;
+    if (grouped) {
+        for (int v = tid; v < V; v += blockDim.x) {
+            m1 = fmaxf(m1, z1[v]);
+            m2 = fmaxf(m2, z2[v]);
+        }
+        m1 = block_max(m1, scratch);
+        m2 = block_max(m2, scratch);
+        float s1 = 0.f, s2 = 0.f, c1 = 0.f;
+        for (int v = tid; v < V; v += blockDim.x) {
+            float e1 = expf(z1[v] - m1);
+            s1 += e1;
+            c1 += e1 * e1;
+            s2 += expf(z2[v] - m2);
+        }
+        d1 = block_sum(s1, scratch);
+        d2 = block_sum(s2, scratch);
+        c1 = block_sum(c1, scratch);
+        alpha = fminf(1.f, fmaxf(0.5f, c1 / (d1 * d1)));
+    }
+    ArgBest best = {-INFINITY, 0x7fffffff};
+    for (int v = tid; v < V; v += blockDim.x) {
+        float val = grouped ? alpha * (expf(z1[v] - m1) / d1) + (1.f - alpha) * (expf(z2[v] - m2) / d2) : z1[v];
+        best = better(best, ArgBest{val, v});
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        ArgBest other = {__shfl_xor_sync(0xffffffffu, best.v, o), __shfl_xor_sync(0xffffffffu, best.i, o)};
+        best = better(best, other);
+    }
+    __syncthreads();
+    if (lane == 0) {
+        bv[warp] = best.v;
+        bi[warp] = best.i;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        ArgBest t = lane < nw ? ArgBest{bv[lane], bi[lane]} : ArgBest{-INFINITY, 0x7fffffff};
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            ArgBest other = {__shfl_xor_sync(0xffffffffu, t.v, o), __shfl_xor_sync(0xffffffffu, t.i, o)};
+            t = better(t, other);
+        }
+        if (lane == 0) {
+            if (next) next[b] = t.i;
+            if (alpha_out && grouped) alpha_out[b] = alpha;
+        }
+    }
+}
+
+__global__ void advance_len_kernel(int32_t *seq_len, int B, int n) {
+    int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b < B) seq_len[b] += n;
+}
+
+// ---------------------------------------------------------------------------------------
+// MoE (Eq. moe_layer, Eq. moe_budget, Section 4.3).
+
+// Router: softmax over E logits, top-k by repeated "largest remaining, lowest index first",
+// weights renormalised over the selection.  Replay: the branch row takes its primary twin's
+// selection and weighs it with its own probabilities.  One warp per row.
+__global__ void route_kernel(const float *__restrict__ logits, int E, int Bc, int k_p, int k_b, int kmax, int replay,
+                             int32_t *__restrict__ idx, float *__restrict__ wts, int32_t *__restrict__ last,
+                             int last_stride_path) {
+    extern __shared__ float smem[];
+    float *p = smem;                                   // [E] own-row probabilities
+    unsigned char *taken = (unsigned char *)(smem + E);  // [E]
+    int r = blockIdx.x, lane = threadIdx.x;
+    int path = r >= Bc;
+    const float *own = logits + (size_t)r * E;
+    const float *sel = (path && replay) ? logits + (size_t)(r - Bc) * E : own;
+    int k = (path && !replay) ? k_b : k_p;
+    float mx = -INFINITY;
+    for (int e = lane; e < E; e += 32) mx = fmaxf(mx, own[e]);
+    mx = warp_max(mx);
+    float s = 0.f;
+    for (int e = lane; e < E; e += 32) {
+        float x = expf(own[e] - mx);
+        p[e] = x;
+        s += x;
+        taken[e] = 0;
+    }
+    s = warp_sum(s);
+    __syncwarp();
+    if (lane == 0) {
+        float tot = 0.f;
+        int chosen[64];
+        for (int j = 0; j < k; j++) {
+            int best = -1;
+            for (int e = 0; e < E; e++)
+                if (!taken[e] && (best < 0 || sel[e] > sel[best])) best = e;
+            taken[best] = 1;
+            chosen[j] = best;
+            tot += p[best] / s;
+        }
+        for (int j = 0; j < kmax; j++) {
+            int e = j < k ? chosen[j] : -1;
+            idx[(size_t)r * kmax + j] = e;
+            wts[(size_t)r * kmax + j] = j < k ? (p[e] / s) / tot : 0.f;
+            if (last) last[(size_t)path * last_stride_path + (size_t)(r - path * Bc) * kmax + j] = e;
+        }
+    }
+}
+
+// Per-expert lists of (row, slot) entries in ascending order, and the size of the union.
+__global__ void moe_lists_kernel(const int32_t *__restrict__ idx, int R, int kmax, int E, int cap,
+                                 int32_t *__restrict__ cnt, int32_t *__restrict__ list, int32_t *union_count) {
+    int e = blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= E) return;
+    int c = 0;
+    for (int r = 0; r < R; r++)
+        for (int j = 0; j < kmax; j++)
+            if (idx[(size_t)r * kmax + j] == e) list[(size_t)e * cap + c++] = r * kmax + j;
+    cnt[e] = c;
+    if (c > 0 && union_count) atomicAdd(union_count, 1);
+}
+
+// Routed experts, gate/up + SwiGLU: every expert with a non-empty list streams its gate and up
+// matrices once for all its entries of both paths.  grid (ceil(Fe/warps), E).
+template <typename WT>
+__global__ void __launch_bounds__(kLinWarps * 32) expert_gateup_kernel(
+    const WT *__restrict__ Wg, const WT *__restrict__ Wu, int Fe, int d, const float *__restrict__ X, int kmax,
+    const int32_t *__restrict__ cnt, const int32_t *__restrict__ list, int cap, float *__restrict__ Hexp) {
+    int e = blockIdx.y, n = cnt[e];
+    if (n == 0) return;
+    int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    int f = blockIdx.x * kLinWarps + warp;
+    if (f >= Fe) return;
+    const WT *wg = Wg + ((size_t)e * Fe + f) * d, *wu = Wu + ((size_t)e * Fe + f) * d;
+    const int32_t *li = list + (size_t)e * cap;
+    for (int r0 = 0; r0 < n; r0 += kLinRT) {
+        const float *xp[kLinRT];
+        int ent[kLinRT];
+#pragma unroll
+        for (int r = 0; r < kLinRT; r++) {
+            ent[r] = (r0 + r < n) ? li[r0 + r] : -1;
+            xp[r] = ent[r] >= 0 ? X + (size_t)(ent[r] / kmax) * d : nullptr;
+        }
+        float ga[kLinRT], up[kLinRT];
+        warp_dots<WT, kLinRT>(wg, xp, d, ga);
+        warp_dots<WT, kLinRT>(wu, xp, d, up);
+#pragma unroll
+        for (int r = 0; r < kLinRT; r++)
+            if (lane == r && ent[r] >= 0) Hexp[(size_t)ent[r] * Fe + f] = silu(ga[r]) * up[r];
+    }
+}
+
+// Routed experts, down projection: Yexp[entry] = W_D[e] Hexp[entry].  grid (ceil(d/warps), E).
+template <typename WT>
+__global__ void __launch_bounds__(kLinWarps * 32) expert_down_kernel(
+    const WT *__restrict__ Wd, int Fe, int d, const float *__restrict__ Hexp, const int32_t *__restrict__ cnt,
+    const int32_t *__restrict__ list, int cap, float *__restrict__ Yexp) {
+    int e = blockIdx.y, n = cnt[e];
+    if (n == 0) return;
+    int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    int f = blockIdx.x * kLinWarps + warp;
+    if (f >= d) return;
+    const WT *w = Wd + ((size_t)e * d + f) * Fe;
+    const int32_t *li = list + (size_t)e * cap;
+    for (int r0 = 0; r0 < n; r0 += kLinRT) {
+        const float *xp[kLinRT];
+        int ent[kLinRT];
+#pragma unroll
+        for (int r = 0; r < kLinRT; r++) {
+            ent[r] = (r0 + r < n) ? li[r0 + r] : -1;
+            xp[r] = ent[r] >= 0 ? Hexp + (size_t)ent[r] * Fe : nullptr;
+        }
+        float acc[kLinRT];
+        warp_dots<WT, kLinRT>(w, xp, Fe, acc);
+#pragma unroll
+        for (int r = 0; r < kLinRT; r++)
+            if (lane == r && ent[r] >= 0) Yexp[(size_t)ent[r] * d + f] = acc[r];
+    }
+}
+
+// M_1 = sum_j w_1j Expert_j(m_1) + G(m_1);  M_2 = sum_j w_2j Expert_j(m_2) + G~(m_2) + c*M_1;
+// S_i += M_i.  Slots are summed in slot order.  One block per primary row.
+__global__ void moe_combine_kernel(const float *__restrict__ Yexp, const float *__restrict__ Msh,
+                                   const int32_t *__restrict__ idx, const float *__restrict__ wts, int kmax, int Bc,
+                                   int grouped, const float *__restrict__ coup_c, int d, float *__restrict__ S) {
+    int b = blockIdx.x;
+    for (int i = threadIdx.x; i < d; i += blockDim.x) {
+        float m1 = 0.f;
+        for (int j = 0; j < kmax; j++)
+            if (idx[(size_t)b * kmax + j] >= 0) m1 = fmaf(wts[(size_t)b * kmax + j], Yexp[((size_t)b * kmax + j) * d + i], m1);
+        if (Msh) m1 += Msh[(size_t)b * d + i];
+        S[(size_t)b * d + i] += m1;
+        if (grouped) {
+            int r = Bc + b;
+            float m2 = 0.f;
+            for (int j = 0; j < kmax; j++)
+                if (idx[(size_t)r * kmax + j] >= 0)
+                    m2 = fmaf(wts[(size_t)r * kmax + j], Yexp[((size_t)r * kmax + j) * d + i], m2);
+            if (Msh) m2 += Msh[(size_t)r * d + i];
+            m2 += coup_c[i] * m1;
+            S[(size_t)r * d + i] += m2;
+        }
+    }
+}
+
+}  // namespace dbt

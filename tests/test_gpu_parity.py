@@ -1,0 +1,290 @@
+"""GPU parity: the CUDA library against the CPU oracle through the C ABI, element by element
+on the same seeded inputs, plus the properties that must hold at any size."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from gpu_util import TOL, assert_logits_close, make_gpu_model, teacher_forced_compare
+from paper_2608_12385_b200 import binding
+from paper_2608_12385_b200.inputs import (ModelConfig, dense_1b, make_page_table, make_synthetic_kv, make_tokens,
+                                          make_weights, moe_1b, tiny_dense_fp32)
+
+pytestmark = pytest.mark.gpu
+
+
+def small_bf16(**kw):
+    base = dict(d_model=256, n_layers=3, n_q_heads=8, n_kv_heads=2, head_dim=64, d_ff=712, vocab=1000,
+                weight_dtype="bf16")
+    base.update(kw)
+    return ModelConfig(**base)
+
+
+def small_moe(**kw):
+    base = dict(d_model=256, n_layers=2, n_q_heads=4, n_kv_heads=2, head_dim=64, d_ff=0, vocab=1000,
+                weight_dtype="bf16", n_experts=8, d_expert=200, n_shared_experts=1, k_primary=2, k_branch=3)
+    base.update(kw)
+    return ModelConfig(**base)
+
+
+# ---- end-to-end parity ---------------------------------------------------------------------------
+
+def test_tiny_fp32_config_prefill_and_16_grouped_steps():
+    """Tiny dense fp32 model, batch 2, prompt 64 (prefill 63 + boundary step), 16 grouped steps."""
+    cfg = tiny_dense_fp32()
+    w = make_weights(cfg, seed=0)
+    tok = make_tokens(cfg, 2, 64 + 15, seed=1)
+    teacher_forced_compare(cfg, w, tok, n_prefill=63, grouped=True)
+
+
+def test_tiny_fp32_primary_only():
+    cfg = tiny_dense_fp32()
+    w = make_weights(cfg, seed=0)
+    tok = make_tokens(cfg, 2, 40, seed=1)
+    teacher_forced_compare(cfg, w, tok, n_prefill=33, grouped=False)
+
+
+@pytest.mark.parametrize("cfg,B,T,npre", [
+    (small_bf16(), 3, 40, 35),                                     # GQA 4 queries per KV head, ragged d_ff
+    (small_bf16(n_q_heads=4, n_kv_heads=4, head_dim=64), 1, 20, 17),  # MHA, batch 1
+    (small_bf16(n_q_heads=2, n_kv_heads=1, head_dim=128, d_model=128, vocab=777), 5, 50, 47),  # MQA, odd batch
+    (small_bf16(final_norm=0, n_layers=1), 2, 18, 0),              # no prefill at all: decode from position 0
+])
+def test_small_bf16_models(cfg, B, T, npre):
+    w = make_weights(cfg, seed=5, matrix_std=0.05)
+    tok = make_tokens(cfg, B, T, seed=6)
+    teacher_forced_compare(cfg, w, tok, n_prefill=npre, grouped=True)
+
+
+def test_prefill_longer_than_one_chunk_and_page_boundaries():
+    """Prompt of 300 positions at batch 2 crosses the prefill chunking and 18 page boundaries."""
+    cfg = small_bf16(n_layers=2)
+    w = make_weights(cfg, seed=7, matrix_std=0.05)
+    tok = make_tokens(cfg, 2, 306, seed=8)
+    teacher_forced_compare(cfg, w, tok, n_prefill=300, grouped=True)
+
+
+@pytest.mark.parametrize("ctx", [0, 1, 15, 16, 17, 255, 256, 257])
+def test_context_lengths_around_page_and_chunk_boundaries(ctx):
+    """Synthetic cache of `ctx` positions, then two grouped steps."""
+    cfg = small_bf16(n_layers=1)
+    w = make_weights(cfg, seed=9, matrix_std=0.05)
+    B = 2
+    tok = make_tokens(cfg, B, 2, seed=10)
+    om = oracle.OracleModel(cfg, w, B, ctx + 2)
+    gm = make_gpu_model(cfg, w, B, ctx + 2)
+    if ctx > 0:
+        k, v = make_synthetic_kv(cfg, B, ctx, seed=11)
+        om.inject_kv(k, v, ctx)
+        gm.write_kv(k, v)
+    for t in range(2):
+        o = om.decode_step(tok[:, t].numpy())
+        g = gm.decode_full(tok[:, t].cuda().contiguous())
+        assert_logits_close(g["z1"], o["z1"], "bf16", f"ctx {ctx} step {t} z1")
+        assert_logits_close(g["z2"], o["z2"], "bf16", f"ctx {ctx} step {t} z2")
+
+
+def test_1b_shape_full_width_grouped_step_with_synthetic_cache():
+    """The 1B configuration at full width and depth: batch 3, a 300-position synthetic cache
+    (same bytes on both sides), two grouped steps and one primary-only step."""
+    cfg = dense_1b()
+    w = make_weights(cfg, seed=0)
+    B, ctx = 3, 300
+    tok = make_tokens(cfg, B, 3, seed=2)
+    k, v = make_synthetic_kv(cfg, B, ctx, seed=3)
+    om = oracle.OracleModel(cfg, w, B, ctx + 3)
+    gm = make_gpu_model(cfg, w, B, ctx + 3)
+    om.inject_kv(k, v, ctx)
+    gm.write_kv(k, v)
+    for t in range(2):
+        o = om.decode_step(tok[:, t].numpy())
+        g = gm.decode_full(tok[:, t].cuda().contiguous())
+        assert_logits_close(g["z1"], o["z1"], "bf16", f"1B step {t} z1")
+        assert_logits_close(g["z2"], o["z2"], "bf16", f"1B step {t} z2")
+        assert (g["alpha"].cpu().numpy() == 0.5).all() and (o["alpha"] == 0.5).all()
+    o = om.decode_step(tok[:, 2].numpy(), grouped=False)
+    g = gm.decode_full(tok[:, 2].cuda().contiguous(), grouped=False)
+    assert_logits_close(g["z1"], o["z1"], "bf16", "1B primary-only z1")
+
+
+# ---- properties that hold at any size ---------------------------------------------------------------
+
+def _run_steps(gm, tok_dev, n_prefill, grouped):
+    if n_prefill:
+        gm.prefill(tok_dev[:, :n_prefill].contiguous())
+    outs = [gm.decode_full(tok_dev[:, t].contiguous(), grouped=grouped) for t in range(n_prefill, tok_dev.shape[1])]
+    torch.cuda.synchronize()
+    return outs
+
+
+@pytest.mark.parametrize("cfg", [tiny_dense_fp32().replace(n_layers=2), small_bf16(), small_moe()])
+def test_kv_cache_bit_identical_grouped_vs_primary_only(cfg):
+    """The primary path never reads the branch: the cache written by grouped decode and by
+    primary-only decode is the same bits, and so are the primary logits."""
+    w = make_weights(cfg, seed=12, matrix_std=0.05)
+    B, T, npre = 3, 30, 20
+    tok = make_tokens(cfg, B, T, seed=13).cuda()
+    wd = binding.weights_to_device(w)
+    a = binding.Model(cfg, wd, B, T)
+    b = binding.Model(cfg, wd, B, T)
+    oa = _run_steps(a, tok, npre, True)
+    ob = _run_steps(b, tok, npre, False)
+    for x, y in zip(oa, ob):
+        assert torch.equal(x["z1"], y["z1"])
+    ka, va = a.read_kv(B, T)
+    kb, vb = b.read_kv(B, T)
+    assert torch.equal(ka.view(torch.int16 if cfg.weight_dtype == "bf16" else torch.int32),
+                       kb.view(torch.int16 if cfg.weight_dtype == "bf16" else torch.int32))
+    assert torch.equal(va.view(torch.int16 if cfg.weight_dtype == "bf16" else torch.int32),
+                       vb.view(torch.int16 if cfg.weight_dtype == "bf16" else torch.int32))
+    assert ka.float().abs().sum() > 0
+
+
+def test_page_table_permutation_does_not_change_results():
+    cfg = small_bf16(n_layers=2)
+    w = make_weights(cfg, seed=14, matrix_std=0.05)
+    B, T, npre = 3, 60, 50
+    tok = make_tokens(cfg, B, T, seed=15).cuda()
+    wd = binding.weights_to_device(w)
+    a = binding.Model(cfg, wd, B, T)
+    b = binding.Model(cfg, wd, B, T, num_pages=64)
+    pt = make_page_table(B, (T + 15) // 16, 64, seed=16)
+    b.set_page_table(pt)
+    oa = _run_steps(a, tok, npre, True)
+    ob = _run_steps(b, tok, npre, True)
+    for x, y in zip(oa, ob):
+        assert torch.equal(x["z1"], y["z1"]) and torch.equal(x["z2"], y["z2"]) and torch.equal(x["next"], y["next"])
+    ka, _ = a.read_kv(B, T)
+    kb, _ = b.read_kv(B, T)
+    assert torch.equal(ka.float(), kb.float())
+
+
+def test_sequences_do_not_depend_on_batch_mates_and_runs_are_deterministic():
+    cfg = small_bf16(n_layers=2)
+    w = make_weights(cfg, seed=17, matrix_std=0.05)
+    T, npre = 40, 33
+    tok = make_tokens(cfg, 4, T, seed=18).cuda()
+    wd = binding.weights_to_device(w)
+    full = _run_steps(binding.Model(cfg, wd, 4, T), tok, npre, True)
+    again = _run_steps(binding.Model(cfg, wd, 4, T), tok, npre, True)
+    solo = _run_steps(binding.Model(cfg, wd, 4, T), tok[2:3].contiguous(), npre, True)
+    for x, y, z in zip(full, again, solo):
+        assert torch.equal(x["z1"], y["z1"]) and torch.equal(x["z2"], y["z2"])
+        # a different batch size may pick a different split of the KV range: compare within tolerance
+        assert_logits_close(z["z1"][0], x["z1"][2].cpu().numpy(), "bf16")
+        assert_logits_close(z["z2"][0], x["z2"][2].cpu().numpy(), "bf16")
+
+
+def test_host_buffer_entry_points_match_device_entry_points():
+    cfg = small_bf16(n_layers=2)
+    w = make_weights(cfg, seed=19, matrix_std=0.05)
+    B = 3
+    tok = make_tokens(cfg, B, 12, seed=20)
+    wd = binding.weights_to_device(w)
+    a, b = binding.Model(cfg, wd, B, 32), binding.Model(cfg, wd, B, 32)
+    a.prefill(tok[:, :8].cuda().contiguous())
+    b.prefill(tok[:, :8].cuda().contiguous())
+    cur_dev = tok[:, 8].cuda().contiguous()
+    cur_host = tok[:, 8].clone().pin_memory()
+    nxt_host = torch.empty(B, dtype=torch.int32).pin_memory()
+    alpha_host = torch.empty(B, dtype=torch.float32).pin_memory()
+    for i in range(4):  # free-running greedy decode, next tokens fed back
+        grouped = i % 2 == 0
+        out = a.decode_full(cur_dev, grouped=grouped)
+        if grouped:
+            b.decode_step_host(cur_host, nxt_host, alpha_host)
+            assert torch.equal(alpha_host, out["alpha"].cpu())
+        else:
+            b.decode_step_primary_only_host(cur_host, nxt_host)
+        assert torch.equal(nxt_host, out["next"].cpu())
+        cur_dev = out["next"].clone()
+        cur_host.copy_(nxt_host)
+    assert a.seq_len(0) == b.seq_len(0) == 12
+    assert a.launch_count() > 0
+
+
+# ---- MoE ----------------------------------------------------------------------------------------------
+
+def _moe_compare(cfg, B, T, npre):
+    w = make_weights(cfg, seed=21, matrix_std=0.05)
+    tok = make_tokens(cfg, B, T, seed=22)
+    om = oracle.OracleModel(cfg, w, B, T)
+    gm = make_gpu_model(cfg, w, B, T)
+    z1_full, _, k_full, v_full = oracle.full_forward(cfg, w, tok[:, :npre].numpy(), want_kv=True)
+    om.inject_kv(k_full, v_full, npre)
+    got = gm.prefill(tok[:, :npre].cuda().contiguous(), want_logits=True)
+    # prefill routes the primary path by top-k too; near-ties can flip, so compare loosely here
+    # and exactly (forced routing) in the decode steps below, which restart from the oracle's cache
+    gm.write_kv(torch.from_numpy(k_full), torch.from_numpy(v_full))
+    flips = 0
+    for t in range(npre, T):
+        g = gm.decode_full(tok[:, t].cuda().contiguous())
+        ex = gm.last_experts(B).numpy()
+        free = om_probe = None
+        # the device's choice must be a valid top-k of the oracle's router up to rounding:
+        o_free = oracle.OracleModel(cfg, w, B, T)
+        o_free.inject_kv(om.k_cache[:, :B, :t], om.v_cache[:, :B, :t], t)
+        of = o_free.decode_step(tok[:, t].numpy())
+        flips += int((np.sort(of["experts"], -1) != np.sort(ex, -1)).any())
+        o = om.decode_step(tok[:, t].numpy(), forced_experts=ex)
+        assert_logits_close(g["z1"], o["z1"], "bf16", f"moe step {t} z1")
+        assert_logits_close(g["z2"], o["z2"], "bf16", f"moe step {t} z2")
+        kp, kb = cfg.k_primary, (cfg.k_primary if cfg.router_mode == 1 else cfg.k_branch)
+        assert (ex[:, 0, :, :kp] >= 0).all() and (ex[:, 0, :, kp:] == -1).all()
+        assert (ex[:, 1, :, :kb] >= 0).all() and (ex[:, 1, :, kb:] == -1).all()
+        union = gm.last_expert_union()
+        for l in range(cfg.n_layers):
+            assert union[l] == len(set(ex[l][ex[l] >= 0].tolist()))
+    assert got is not None
+    return flips
+
+
+@pytest.mark.parametrize("cfg", [small_moe(), small_moe(router_mode=1), small_moe(n_shared_experts=0, k_branch=8),
+                                 small_moe(moe_b_coupling=0, k_primary=1, k_branch=1)])
+def test_moe_decode_matches_oracle_under_the_devices_routing(cfg):
+    """Router near-ties are decided by rounding, so the device's expert choice is read back,
+    checked for shape and union count, and imposed on the oracle; everything else is compared
+    element by element."""
+    flips = _moe_compare(cfg, B=3, T=14, npre=10)
+    assert flips <= 2  # well-separated router logits: the free-running oracle picks the same experts
+
+
+def test_moe_1b_shape_two_layers():
+    cfg = moe_1b(k_branch=4).replace(n_layers=2)
+    flips = _moe_compare(cfg, B=2, T=8, npre=6)
+    assert flips <= 2
+
+
+# ---- error paths (host-detected, and device-detected without any fault) ---------------------------------
+
+def test_capacity_and_argument_errors():
+    cfg = small_bf16(n_layers=1)
+    w = make_weights(cfg, seed=23, matrix_std=0.05)
+    gm = make_gpu_model(cfg, w, 2, 20)
+    tok = make_tokens(cfg, 2, 21, seed=24).cuda()
+    with pytest.raises(binding.DbtError) as e:
+        gm.prefill(tok.contiguous())
+    assert e.value.status == 3
+    gm.prefill(tok[:, :20].contiguous())
+    with pytest.raises(binding.DbtError) as e:
+        gm.decode_step(tok[:, 20].contiguous())
+    assert e.value.status == 3
+    gm.reset()
+    with pytest.raises(binding.DbtError) as e:
+        gm.decode_step(make_tokens(cfg, 3, 1).cuda().view(-1))
+    assert e.value.status == 3
+    with pytest.raises(binding.DbtError):
+        gm.set_page_table(torch.tensor([[0, 0], [1, 2]]))
+
+
+def test_out_of_range_token_is_reported_not_faulted():
+    cfg = small_bf16(n_layers=1)
+    w = make_weights(cfg, seed=25, matrix_std=0.05)
+    gm = make_gpu_model(cfg, w, 2, 8)
+    bad = torch.tensor([3, cfg.vocab + 5], dtype=torch.int32).cuda()
+    gm.decode_step(bad)
+    status, detail = gm.sync_status()
+    assert status == 1 and detail == cfg.vocab + 5
+    gm.reset()
+    gm.decode_step(torch.tensor([3, 4], dtype=torch.int32).cuda())
+    assert gm.sync_status() == (0, 0)
