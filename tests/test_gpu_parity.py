@@ -205,8 +205,8 @@ def test_host_buffer_entry_points_match_device_entry_points():
 
 # ---- MoE ----------------------------------------------------------------------------------------------
 
-def _moe_compare(cfg, B, T, npre):
-    w = make_weights(cfg, seed=21, matrix_std=0.05)
+def _moe_compare(cfg, B, T, npre, matrix_std=0.05):
+    w = make_weights(cfg, seed=21, matrix_std=matrix_std)
     tok = make_tokens(cfg, B, T, seed=22)
     om = oracle.OracleModel(cfg, w, B, T)
     gm = make_gpu_model(cfg, w, B, T)
@@ -220,7 +220,6 @@ def _moe_compare(cfg, B, T, npre):
     for t in range(npre, T):
         g = gm.decode_full(tok[:, t].cuda().contiguous())
         ex = gm.last_experts(B).numpy()
-        free = om_probe = None
         # the device's choice must be a valid top-k of the oracle's router up to rounding:
         o_free = oracle.OracleModel(cfg, w, B, T)
         o_free.inject_kv(om.k_cache[:, :B, :t], om.v_cache[:, :B, :t], t)
@@ -251,7 +250,7 @@ def test_moe_decode_matches_oracle_under_the_devices_routing(cfg):
 
 def test_moe_1b_shape_two_layers():
     cfg = moe_1b(k_branch=4).replace(n_layers=2)
-    flips = _moe_compare(cfg, B=2, T=8, npre=6)
+    flips = _moe_compare(cfg, B=2, T=8, npre=6, matrix_std=0.02)
     assert flips <= 2
 
 
