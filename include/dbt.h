@@ -167,6 +167,19 @@ dbt_status dbt_last_expert_union(dbt_model *m, int32_t *count_per_layer_host);
  * Returns DBT_ERR_DEVICE when non-zero.  HOST pointers, may be NULL. */
 dbt_status dbt_sync_status(dbt_model *m, int32_t *device_status, int32_t *detail);
 
+/* Operator-level entry: the grouped skinny GEMM alone (Section 4.4 "Decode": the stacked rows
+ * of both paths go through one shared matrix, each weight tile fetched once).
+ * Y[r][f] = sum_k W[f][k] X[r][k] with W_dev DEVICE bf16 [n_out][K], X_dev DEVICE bf16 [R][K]
+ * (1 <= R <= 256, K a multiple of 8, both 16-byte aligned), Y_dev DEVICE fp32 [R][n_out].
+ * scratch_dev: DEVICE fp32 workspace of scratch_floats elements for the split-K partials
+ * (at least splits * roundup(R) * n_out with roundup to 16/32/64/128/256); status_dev DEVICE
+ * int32[2] (zeroed by the caller; non-zero afterwards = a bounded device wait expired).
+ * force_split > 0 fixes the split-K factor, 0 lets the library choose; *split_used (HOST,
+ * nullable) receives it.  Runs on the tensor cores (TMA + tcgen05); enqueues on cuda_stream. */
+dbt_status dbt_op_gemm_tc(const void *W_dev, const void *X_dev, int32_t n_out, int32_t K, int32_t R,
+                          int32_t force_split, float *Y_dev, float *scratch_dev, size_t scratch_floats,
+                          int32_t *status_dev, void *cuda_stream, int32_t *split_used);
+
 /* Per-kernel timing for the roofline report (paper Eq. roofline, Eq. decode_traffic: time
  * against the bytes that must move).  Between begin and end every kernel launch is bracketed
  * by CUDA events on the handle's stream; end waits for the stream and sums, per kernel family,

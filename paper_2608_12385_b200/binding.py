@@ -23,7 +23,7 @@ STATUS_NAMES = {0: "DBT_OK", 1: "DBT_ERR_INVALID_ARG", 2: "DBT_ERR_UNSUPPORTED",
 EXPORTS = ["dbt_query_sizes", "dbt_create", "dbt_destroy", "dbt_set_page_table", "dbt_reset", "dbt_set_seq_lens",
            "dbt_seq_len", "dbt_prefill", "dbt_decode_step", "dbt_decode_step_primary_only", "dbt_decode_step_host",
            "dbt_decode_step_primary_only_host", "dbt_last_experts", "dbt_last_expert_union", "dbt_sync_status",
-           "dbt_launch_count", "dbt_last_error", "dbt_version", "dbt_profile_begin", "dbt_profile_end"]
+           "dbt_launch_count", "dbt_last_error", "dbt_version", "dbt_profile_begin", "dbt_profile_end", "dbt_op_gemm_tc"]
 
 
 class DbtError(RuntimeError):
@@ -89,6 +89,7 @@ def load_library():
     L.dbt_last_experts.argtypes = [vp, C.POINTER(vp), i32p]
     L.dbt_last_expert_union.argtypes = [vp, vp]
     L.dbt_sync_status.argtypes = [vp, i32p, i32p]
+    L.dbt_op_gemm_tc.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, C.c_size_t, vp, vp, i32p]
     L.dbt_profile_begin.argtypes = [vp]
     L.dbt_profile_end.argtypes = [vp, C.POINTER(DbtProfileEntry), i32, i32p]
     L.dbt_launch_count.argtypes = [vp]
@@ -121,6 +122,30 @@ def query_sizes(cfg: ModelConfig, max_batch: int, max_seq: int, num_pages: int) 
     if st != DBT_OK:
         raise DbtError(st, L.dbt_last_error(None).decode())
     return kv.value, ws.value
+
+
+def op_gemm_tc(W: torch.Tensor, X: torch.Tensor, force_split: int = 0, scratch: torch.Tensor | None = None):
+    """Y = X W^T on the tensor cores.  W bf16 [n_out, K], X bf16 [R, K] on the GPU.
+    Returns (Y fp32 [R, n_out], split used)."""
+    L = load_library()
+    assert W.dtype == torch.bfloat16 and X.dtype == torch.bfloat16 and W.is_cuda and X.is_cuda
+    n_out, K = W.shape
+    R = X.shape[0]
+    Y = torch.empty(R, n_out, dtype=torch.float32, device=W.device)
+    if scratch is None:
+        scratch = torch.empty(max(force_split, 16) * 256 * n_out if R > 128 else max(force_split, 16) * 128 * n_out,
+                              dtype=torch.float32, device=W.device)
+    status = torch.zeros(2, dtype=torch.int32, device=W.device)
+    used = C.c_int32(0)
+    st = L.dbt_op_gemm_tc(W.data_ptr(), X.data_ptr(), n_out, K, R, force_split, Y.data_ptr(), scratch.data_ptr(),
+                          scratch.numel(), status.data_ptr(), torch.cuda.current_stream().cuda_stream, C.byref(used))
+    if st != DBT_OK:
+        raise DbtError(st, L.dbt_last_error(None).decode())
+    torch.cuda.synchronize()
+    code = status.cpu().tolist()
+    if code[0] != 0:
+        raise DbtError(6, f"device status {code}")
+    return Y, used.value
 
 
 def weights_to_device(weights: dict, device="cuda") -> dict:
@@ -239,17 +264,25 @@ class Model:
                                                              next_host.data_ptr()))
 
     def decode_full(self, tokens_dev: torch.Tensor, grouped: bool = True) -> dict:
-        """One step returning every output (test convenience)."""
+        """One step returning every output (test convenience).  The library replays a step as
+        a CUDA graph keyed by its buffer addresses, so the buffers are kept and reused; the
+        returned tensors are copies."""
         B, V = tokens_dev.shape[0], self.cfg.vocab
-        out = {"next": torch.empty(B, dtype=torch.int32, device=self.device),
-               "z1": torch.empty(B, V, dtype=torch.float32, device=self.device)}
+        cache = self.__dict__.setdefault("_full_bufs", {})
+        buf = cache.get(B)
+        if buf is None:
+            buf = {"tok": torch.empty(B, dtype=torch.int32, device=self.device),
+                   "next": torch.empty(B, dtype=torch.int32, device=self.device),
+                   "z1": torch.empty(B, V, dtype=torch.float32, device=self.device),
+                   "z2": torch.empty(B, V, dtype=torch.float32, device=self.device),
+                   "alpha": torch.empty(B, dtype=torch.float32, device=self.device)}
+            cache[B] = buf
+        buf["tok"].copy_(tokens_dev)
         if grouped:
-            out["z2"] = torch.empty(B, V, dtype=torch.float32, device=self.device)
-            out["alpha"] = torch.empty(B, dtype=torch.float32, device=self.device)
-            self.decode_step(tokens_dev, out["next"], out["z1"], out["z2"], out["alpha"])
-        else:
-            self.decode_step_primary_only(tokens_dev, out["next"], out["z1"])
-        return out
+            self.decode_step(buf["tok"], buf["next"], buf["z1"], buf["z2"], buf["alpha"])
+            return {k: buf[k].clone() for k in ("next", "z1", "z2", "alpha")}
+        self.decode_step_primary_only(buf["tok"], buf["next"], buf["z1"])
+        return {k: buf[k].clone() for k in ("next", "z1")}
 
     # -- diagnostics ----------------------------------------------------------------------
     def last_experts(self, batch: int) -> torch.Tensor:

@@ -5,11 +5,14 @@
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <string>
 #include <vector>
 
+#include "dbt_fused.cuh"
+#include "dbt_gemm_tc.cuh"
 #include "dbt_kernels.cuh"
 
 using namespace dbt;
@@ -27,6 +30,14 @@ struct Workspace {
     // MoE
     float *rlogits, *rwts, *Hexp, *Yexp, *Msh, *Hsh;
     int32_t *ridx, *ecnt, *elist, *last_experts, *union_cnt;
+    // bf16 tensor-core path: bf16 GEMM inputs and the fp32 split-K partial buffer
+    __nv_bfloat16 *Xb, *Ob, *Hb;
+    float *P;
+    size_t P_floats;
+};
+
+struct LayerMaps {
+    CUtensorMap wq, wk, wv, wo, wg, wu, wd;
 };
 
 }  // namespace
@@ -50,6 +61,22 @@ struct dbt_model {
     struct ProfRec { const char *tag; double bytes; cudaEvent_t e0, e1; };
     std::vector<ProfRec> prof;
     std::vector<cudaEvent_t> prof_pool;
+    // tensor-core path (bf16 models): TMA descriptors of every weight matrix and GEMM input
+    bool tc;
+    std::vector<LayerMaps> maps;
+    CUtensorMap map_lm, map_Xb, map_Ob, map_Hb;
+    int act_parts;  // 2: GEMM inputs carried as hi + lo bf16 terms; 1: plain bf16
+    // a decode step is captured once per (batch, mode, buffer set) and replayed as a CUDA graph
+    struct GraphEntry {
+        int B, grouped;
+        const void *ptr[5];
+        cudaGraph_t graph;
+        cudaGraphExec_t exec;
+        int64_t launches;
+    };
+    bool use_graph;
+    cudaStream_t cap_stream;
+    std::vector<GraphEntry> graphs;
 };
 
 namespace {
@@ -143,6 +170,19 @@ size_t carve(const dbt_config &c, char *base, Workspace *ws, int *Rmax_out, int 
         w.last_experts = k.take<int32_t>((size_t)c.n_layers * 2 * c.max_batch * km);
         w.union_cnt = k.take<int32_t>(c.n_layers);
     }
+    if (c.weight_dtype == DBT_DTYPE_BF16) {
+        // two planes each: rows [0,Rmax) hold hi = bf16(x), rows [Rmax,2Rmax) hold lo = bf16(x - hi)
+        w.Xb = k.take<__nv_bfloat16>((size_t)2 * Rmax * d);
+        w.Ob = k.take<__nv_bfloat16>((size_t)2 * Rmax * qd);
+        w.Hb = k.take<__nv_bfloat16>((size_t)2 * Rmax * F);
+        // room for the widest GEMM output at a few splits, capped
+        size_t widest = (size_t)(moe ? (qd + 2 * kvd > 2 * F ? qd + 2 * kvd : 2 * F) : (2 * F > qd + 2 * kvd ? 2 * F : qd + 2 * kvd));
+        size_t want = (size_t)Rmax * widest * 6;
+        size_t cap = (size_t)24 << 20;  // floats (96 MB)
+        w.P_floats = want < cap ? want : cap;
+        if (w.P_floats < (size_t)Rmax * widest) w.P_floats = (size_t)Rmax * widest;
+        w.P = k.take<float>(w.P_floats);
+    }
     if (ws) *ws = w;
     if (Rmax_out) *Rmax_out = Rmax;
     if (part_items_out) *part_items_out = part_items;
@@ -229,7 +269,7 @@ LinArgs lin1(const void *W, float *Y, int n_out, int rows, const float *X, int K
 
 template <typename KT, int DH>
 dbt_status run_attention(dbt_model *m, const RowMap &rm, int grouped, const KT *kpool, const KT *vpool, int nsplit,
-                         double kv_bytes) {
+                         double kv_bytes, bool out_bf16 = false) {
     const dbt_config &c = m->cfg;
     int G = c.n_q_heads / c.n_kv_heads, nq = grouped ? 2 * G : G;
     dim3 grid(rm.B * rm.cn, c.n_kv_heads, nsplit);
@@ -249,7 +289,53 @@ dbt_status run_attention(dbt_model *m, const RowMap &rm, int grouped, const KT *
     }
 #undef ATTN_CASE
     dim3 mgrid(rm.B * rm.cn, c.n_kv_heads);
-    LAUNCH(m, "attn_merge", 0, attn_merge_kernel, mgrid, DH, 0, w.part, nsplit, NQ, DH, rm.B * rm.cn, grouped, G, c.n_kv_heads, w.O);
+    LAUNCH(m, "attn_merge", 0, attn_merge_kernel, mgrid, DH, 0, w.part, nsplit, NQ, DH, rm.B * rm.cn, grouped, G, c.n_kv_heads,
+           out_bf16 ? (float *)nullptr : w.O, out_bf16 ? w.Ob : (__nv_bfloat16 *)nullptr,
+           (out_bf16 && m->act_parts == 2) ? (size_t)m->Rmax * c.n_q_heads * c.head_dim : (size_t)0);
+    return DBT_OK;
+}
+
+// MoE sub-layer (Eq. moe_layer, Eq. moe_budget, Section 4.3) on the normalised rows in X:
+// router, per-expert row lists, routed experts (each selected expert's matrices streamed once
+// for all its rows of both paths), shared expert with the b coupling, weighted combine with
+// the c coupling and the residual add into S.
+template <typename WT>
+dbt_status run_moe(dbt_model *m, int l, const RowMap &rm, int grouped, bool record_experts) {
+    const dbt_config &c = m->cfg;
+    const Workspace &w = m->ws;
+    const dbt_layer_weights &lw = m->layers[l];
+    int Bc = rm.B * rm.cn, R = grouped ? 2 * Bc : Bc, d = c.d_model;
+    dbt_status st;
+    int E = c.n_experts, Fe = c.d_expert, km = kmax_of(c), Fs = c.n_shared_experts * Fe;
+    LinArgs rl = lin1(lw.router, w.rlogits, E, R, w.X, d);
+    if ((st = run_linear<WT>(m, "router", rl)) != DBT_OK) return st;
+    int32_t *last = record_experts ? w.last_experts + (size_t)l * 2 * c.max_batch * km : nullptr;
+    if (last && !grouped)
+        CUDA_TRY(m, cudaMemsetAsync(last + (size_t)c.max_batch * km, 0xff, sizeof(int32_t) * c.max_batch * km,
+                                    m->stream));
+    LAUNCH(m, "route", 0, route_kernel, R, 32, E * sizeof(float) + E, w.rlogits, E, Bc, c.k_primary, c.k_branch, km,
+           c.router_mode == DBT_ROUTER_REPLAY, w.ridx, w.rwts, last, c.max_batch * km);
+    int32_t *ucnt = record_experts ? w.union_cnt + l : nullptr;
+    if (ucnt) CUDA_TRY(m, cudaMemsetAsync(ucnt, 0, sizeof(int32_t), m->stream));
+    LAUNCH(m, "moe_lists", 0, moe_lists_kernel, (E + 127) / 128, 128, 0, w.ridx, R, km, E, m->Rmax, w.ecnt, w.elist, ucnt);
+    dim3 g1((Fe + kLinWarps - 1) / kLinWarps, E);
+    LAUNCH(m, "expert_gateup", 0, expert_gateup_kernel<WT>, g1, kLinWarps * 32, 0, (const WT *)lw.exp_gate, (const WT *)lw.exp_up,
+           Fe, d, w.X, km, w.ecnt, w.elist, m->Rmax, w.Hexp);
+    dim3 g2((d + kLinWarps - 1) / kLinWarps, E);
+    LAUNCH(m, "expert_down", 0, expert_down_kernel<WT>, g2, kLinWarps * 32, 0, (const WT *)lw.exp_down, Fe, d, w.Hexp, w.ecnt,
+           w.elist, m->Rmax, w.Yexp);
+    const float *Msh = nullptr;
+    if (Fs > 0) {  // shared expert(s): every row of both paths; b couples its hidden state
+        LinArgs gu{};
+        gu.W[0] = lw.sh_gate; gu.W[1] = lw.sh_up; gu.Y[0] = w.Hsh; gu.n_out[0] = Fs; gu.rows[0] = R;
+        gu.nseg = 2; gu.X = w.X; gu.K = d; gu.epi = EPI_SWIGLU; gu.Bc = Bc; gu.grouped = grouped;
+        gu.coup = c.moe_b_coupling ? lw.coup_b : nullptr;
+        if ((st = run_linear<WT>(m, "shared_gateup", gu)) != DBT_OK) return st;
+        LinArgs dn = lin1(lw.sh_down, w.Msh, d, R, w.Hsh, Fs, EPI_STORE);
+        if ((st = run_linear<WT>(m, "shared_down", dn)) != DBT_OK) return st;
+        Msh = w.Msh;
+    }
+    LAUNCH(m, "moe_combine", 0, moe_combine_kernel, Bc, 256, 0, w.Yexp, Msh, w.ridx, w.rwts, km, Bc, grouped, lw.coup_c, d, w.S);
     return DBT_OK;
 }
 
@@ -305,36 +391,7 @@ dbt_status run_layers(dbt_model *m, const RowMap &rm, int grouped, bool record_e
             dn.Bc = Bc; dn.grouped = grouped; dn.coup = lw.coup_c; dn.S = w.S;
             if ((st = run_linear<WT>(m, "linear_down", dn)) != DBT_OK) return st;
         } else {
-            int E = c.n_experts, Fe = c.d_expert, km = kmax_of(c), Fs = c.n_shared_experts * Fe;
-            LinArgs rl = lin1(lw.router, w.rlogits, E, R, w.X, d);
-            if ((st = run_linear<WT>(m, "router", rl)) != DBT_OK) return st;
-            int32_t *last = record_experts ? w.last_experts + (size_t)l * 2 * c.max_batch * km : nullptr;
-            if (last && !grouped)
-                CUDA_TRY(m, cudaMemsetAsync(last + (size_t)c.max_batch * km, 0xff, sizeof(int32_t) * c.max_batch * km,
-                                            m->stream));
-            LAUNCH(m, "route", 0, route_kernel, R, 32, E * sizeof(float) + E, w.rlogits, E, Bc, c.k_primary, c.k_branch, km,
-                   c.router_mode == DBT_ROUTER_REPLAY, w.ridx, w.rwts, last, c.max_batch * km);
-            int32_t *ucnt = record_experts ? w.union_cnt + l : nullptr;
-            if (ucnt) CUDA_TRY(m, cudaMemsetAsync(ucnt, 0, sizeof(int32_t), m->stream));
-            LAUNCH(m, "moe_lists", 0, moe_lists_kernel, (E + 127) / 128, 128, 0, w.ridx, R, km, E, m->Rmax, w.ecnt, w.elist, ucnt);
-            dim3 g1((Fe + kLinWarps - 1) / kLinWarps, E);
-            LAUNCH(m, "expert_gateup", 0, expert_gateup_kernel<WT>, g1, kLinWarps * 32, 0, (const WT *)lw.exp_gate, (const WT *)lw.exp_up,
-                   Fe, d, w.X, km, w.ecnt, w.elist, m->Rmax, w.Hexp);
-            dim3 g2((d + kLinWarps - 1) / kLinWarps, E);
-            LAUNCH(m, "expert_down", 0, expert_down_kernel<WT>, g2, kLinWarps * 32, 0, (const WT *)lw.exp_down, Fe, d, w.Hexp, w.ecnt,
-                   w.elist, m->Rmax, w.Yexp);
-            const float *Msh = nullptr;
-            if (Fs > 0) {  // shared expert(s): every row of both paths; b couples its hidden state
-                LinArgs gu{};
-                gu.W[0] = lw.sh_gate; gu.W[1] = lw.sh_up; gu.Y[0] = w.Hsh; gu.n_out[0] = Fs; gu.rows[0] = R;
-                gu.nseg = 2; gu.X = w.X; gu.K = d; gu.epi = EPI_SWIGLU; gu.Bc = Bc; gu.grouped = grouped;
-                gu.coup = c.moe_b_coupling ? lw.coup_b : nullptr;
-                if ((st = run_linear<WT>(m, "shared_gateup", gu)) != DBT_OK) return st;
-                LinArgs dn = lin1(lw.sh_down, w.Msh, d, R, w.Hsh, Fs, EPI_STORE);
-                if ((st = run_linear<WT>(m, "shared_down", dn)) != DBT_OK) return st;
-                Msh = w.Msh;
-            }
-            LAUNCH(m, "moe_combine", 0, moe_combine_kernel, Bc, 256, 0, w.Yexp, Msh, w.ridx, w.rwts, km, Bc, grouped, lw.coup_c, d, w.S);
+            if ((st = run_moe<WT>(m, l, rm, grouped, record_experts)) != DBT_OK) return st;
         }
     }
     return DBT_OK;
@@ -349,6 +406,281 @@ dbt_status run_head(dbt_model *m, int rows, int src_mul, int src_add) {
            c.final_norm, w.Zrows);
     LinArgs a = lin1(m->w.lm_head, w.Z, c.vocab, rows, w.Zrows, c.d_model);
     return run_linear<WT>(m, "lm_head", a);
+}
+
+// ---- tensor-core path (bf16 weights) -----------------------------------------------------
+
+struct TcCall {
+    const CUtensorMap *W[3];
+    int n_out[3];
+    int rows[3];
+    int nseg;
+    const CUtensorMap *X;
+    int K;
+    int R;  // activation rows whose outputs are stored
+    float *P;
+    size_t P_floats;
+    const char *tag;
+    int parts;    // 1 or 2 bf16 terms per activation
+    int lo_row0;  // row of the lo plane in the activation buffer
+};
+
+int norm_threads(int d) { return d >= 1024 ? 1024 : d >= 512 ? 512 : 256; }
+int pad_rows(int r) { return r <= 16 ? 16 : r <= 32 ? 32 : r <= 64 ? 64 : r <= 128 ? 128 : 256; }
+
+// Split-K factor from the tile count and K only (never from the mode), so that grouped and
+// primary-only steps add the same partials in the same order.
+int choose_split(int tiles, int total_kt) {
+    int best = 1;
+    double best_cost = 1e30;
+    for (int s = 1; s <= total_kt && s <= 16; s++) {
+        int kt = (total_kt + s - 1) / s;
+        int s_eff = (total_kt + kt - 1) / kt;
+        int waves = (tiles * s_eff + 147) / 148;
+        double cost = waves * (kt + 3.0);
+        if (cost < best_cost - 1e-9) {
+            best_cost = cost;
+            best = s_eff;
+        }
+    }
+    return best;
+}
+
+template <int N_TILE>
+dbt_status launch_gemm_tc(dbt_model *m, const TcCall &c, const TcParams &p, dim3 grid, double bytes) {
+    const CUtensorMap *w1 = c.nseg > 1 ? c.W[1] : c.W[0], *w2 = c.nseg > 2 ? c.W[2] : c.W[0];
+    LAUNCH(m, c.tag, bytes, gemm_tc_kernel<N_TILE>, grid, 128, TcCfg<N_TILE>::kSmemBytes, *c.W[0], *w1, *w2, *c.X, p);
+    return DBT_OK;
+}
+
+// Y partials P[split][R][ldp]; returns the split count and stride the consumer must use.
+dbt_status run_gemm_tc(dbt_model *m, const TcCall &c, int n_tile, int *nsplit_out, size_t *split_stride_out,
+                       int force_split = 0) {
+    TcParams p{};
+    int tiles = 0, col = 0;
+    double bytes = 0;
+    for (int s = 0; s < c.nseg; s++) {
+        p.seg[s] = TcSeg{tiles, c.n_out[s], c.rows[s], col};
+        tiles += (c.n_out[s] + kTcM - 1) / kTcM;
+        col += c.n_out[s];
+        bytes += (double)c.n_out[s] * c.K * 2;
+    }
+    p.nseg = c.nseg;
+    p.K = c.K;
+    p.ldp = col;
+    p.R = c.R;
+    p.parts = c.parts;
+    p.lo_row0 = c.lo_row0;
+    p.P = c.P;
+    p.status = m->ws.status;
+    int total_kt = (c.K + kTcK - 1) / kTcK;
+    int split = force_split > 0 ? (force_split < total_kt ? force_split : total_kt) : choose_split(tiles, total_kt);
+    while (split > 1 && (size_t)split * n_tile * col > c.P_floats) split--;
+    if ((size_t)c.R * col > c.P_floats) return fail(m, DBT_ERR_CAPACITY, "partial buffer too small for %s", c.tag);
+    p.kt_per_split = (total_kt + split - 1) / split;
+    split = (total_kt + p.kt_per_split - 1) / p.kt_per_split;
+    dim3 grid(tiles, split);
+    if (nsplit_out) *nsplit_out = split;
+    if (split_stride_out) *split_stride_out = (size_t)c.R * col;
+    switch (n_tile) {
+        case 16: return launch_gemm_tc<16>(m, c, p, grid, bytes);
+        case 32: return launch_gemm_tc<32>(m, c, p, grid, bytes);
+        case 64: return launch_gemm_tc<64>(m, c, p, grid, bytes);
+        case 128: return launch_gemm_tc<128>(m, c, p, grid, bytes);
+        case 256: return launch_gemm_tc<256>(m, c, p, grid, bytes);
+    }
+    return fail(m, DBT_ERR_UNSUPPORTED, "row tile %d", n_tile);
+}
+
+// bf16 layer stack: TMA + tcgen05 GEMMs with the elementwise work between them fused into
+// three small kernels.  On return the last layer's MLP output is still pending in P (dense
+// models): `pending` tells the caller how to fold it into S (mode of resid_norm_kernel).
+dbt_status run_layers_tc(dbt_model *m, const RowMap &rm, int grouped, int n_tile, bool record_experts, int *pending_mode,
+                         int *pending_split, size_t *pending_stride) {
+    typedef __nv_bfloat16 WT;
+    const dbt_config &c = m->cfg;
+    const Workspace &w = m->ws;
+    int Bc = rm.B * rm.cn, R = grouped ? 2 * Bc : Bc;
+    int d = c.d_model, qd = c.n_q_heads * c.head_dim, kvd = c.n_kv_heads * c.head_dim;
+    size_t pool_layer_elems = (size_t)2 * c.num_pages * c.n_kv_heads * c.page_size * c.head_dim;
+    size_t pool_kv_elems = pool_layer_elems / 2;
+    int att_split = (2 * 148 + Bc * c.n_kv_heads - 1) / (Bc * c.n_kv_heads);
+    att_split = att_split < 1 ? 1 : att_split > 16 ? 16 : att_split;
+    double kv_bytes = 0;
+    for (int b = 0; b < rm.B; b++)
+        for (int j = 0; j < rm.cn; j++) kv_bytes += (double)(m->len_host[b] + j + 1) * 2 * kvd * sizeof(WT);
+    bool moe = c.n_experts > 0;
+    size_t lo_x = m->act_parts == 2 ? (size_t)m->Rmax * d : 0;
+    dbt_status st;
+    int mode = 0, nsp = 1;
+    size_t sstride = 0;
+    for (int l = 0; l < c.n_layers; l++) {
+        const dbt_layer_weights &lw = m->layers[l];
+        const LayerMaps &mp = m->maps[l];
+        WT *kpool = reinterpret_cast<WT *>(m->kv_pool) + (size_t)l * pool_layer_elems;
+        WT *vpool = kpool + pool_kv_elems;
+        // fold the previous layer's MLP output into S (Eq. mlp), N_i = RMSNorm(S_i)
+        LAUNCH(m, "resid_norm", 0, resid_norm_kernel, Bc, norm_threads(d), 0, w.S, w.P, nsp, sstride, mode,
+               l > 0 ? m->layers[l - 1].coup_c : nullptr, Bc, grouped, lw.attn_norm_g, c.rms_eps, d, 1, 1, 0, w.Xb,
+               lo_x, (float *)nullptr);
+        TcCall qkv{};
+        qkv.W[0] = &mp.wq; qkv.n_out[0] = qd; qkv.rows[0] = R;
+        qkv.W[1] = &mp.wk; qkv.n_out[1] = kvd; qkv.rows[1] = Bc;
+        qkv.W[2] = &mp.wv; qkv.n_out[2] = kvd; qkv.rows[2] = Bc;
+        qkv.nseg = 3; qkv.X = &m->map_Xb; qkv.K = d; qkv.R = R; qkv.P = w.P; qkv.P_floats = w.P_floats; qkv.parts = m->act_parts; qkv.lo_row0 = m->Rmax; qkv.tag = "gemm_qkv";
+        if ((st = run_gemm_tc(m, qkv, n_tile, &nsp, &sstride)) != DBT_OK) return st;
+        LAUNCH(m, "qkv_epilogue", 0, qkv_epilogue_kernel<WT>, dim3(Bc, c.n_q_heads + c.n_kv_heads), 64, 0, w.P, nsp, sstride, w.Q, rm, grouped, c.n_q_heads,
+               c.n_kv_heads, c.head_dim, lw.coup_a, w.rope, w.seq_len, w.page_table, m->pages_per_seq_max, c.num_pages,
+               c.page_size, kpool, vpool, w.status);
+        if (c.head_dim == 128)
+            st = run_attention<WT, 128>(m, rm, grouped, kpool, vpool, att_split, kv_bytes, true);
+        else
+            st = run_attention<WT, 64>(m, rm, grouped, kpool, vpool, att_split, kv_bytes, true);
+        if (st != DBT_OK) return st;
+        TcCall op{};
+        op.W[0] = &mp.wo; op.n_out[0] = d; op.rows[0] = R; op.nseg = 1; op.X = &m->map_Ob; op.K = qd; op.R = R;
+        op.P = w.P; op.P_floats = w.P_floats; op.parts = m->act_parts; op.lo_row0 = m->Rmax; op.tag = "gemm_o";
+        if ((st = run_gemm_tc(m, op, n_tile, &nsp, &sstride)) != DBT_OK) return st;
+        // S-bar_i = S_i + Attn_i W_O ; RMSNorm for the MLP
+        LAUNCH(m, "resid_norm", 0, resid_norm_kernel, Bc, norm_threads(d), 0, w.S, w.P, nsp, sstride, 1, (const float *)nullptr, Bc,
+               grouped, lw.mlp_norm_g, c.rms_eps, d, 1, 1, 0, w.Xb, lo_x, moe ? w.X : (float *)nullptr);
+        if (!moe) {
+            int F = c.d_ff;
+            TcCall gu{};
+            gu.W[0] = &mp.wg; gu.n_out[0] = F; gu.rows[0] = R;
+            gu.W[1] = &mp.wu; gu.n_out[1] = F; gu.rows[1] = R;
+            gu.nseg = 2; gu.X = &m->map_Xb; gu.K = d; gu.R = R; gu.P = w.P; gu.P_floats = w.P_floats; gu.parts = m->act_parts; gu.lo_row0 = m->Rmax; gu.tag = "gemm_gateup";
+            if ((st = run_gemm_tc(m, gu, n_tile, &nsp, &sstride)) != DBT_OK) return st;
+            dim3 sg(Bc, (F + 255) / 256);
+            LAUNCH(m, "swiglu_couple", 0, swiglu_couple_kernel, sg, 256, 0, w.P, nsp, sstride, F, Bc, grouped, lw.coup_b,
+                   w.Hb, m->act_parts == 2 ? (size_t)m->Rmax * F : (size_t)0);
+            TcCall dn{};
+            dn.W[0] = &mp.wd; dn.n_out[0] = d; dn.rows[0] = R; dn.nseg = 1; dn.X = &m->map_Hb; dn.K = F; dn.R = R;
+            dn.P = w.P; dn.P_floats = w.P_floats; dn.parts = m->act_parts; dn.lo_row0 = m->Rmax; dn.tag = "gemm_down";
+            if ((st = run_gemm_tc(m, dn, n_tile, &nsp, &sstride)) != DBT_OK) return st;
+            mode = 2;
+        } else {
+            if ((st = run_moe<WT>(m, l, rm, grouped, record_experts)) != DBT_OK) return st;
+            mode = 0;
+        }
+    }
+    *pending_mode = mode;
+    *pending_split = nsp;
+    *pending_stride = sstride;
+    return DBT_OK;
+}
+
+// Fold the pending MLP output, final norm, shared output matrix on tensor cores -> Z.
+dbt_status run_head_tc(dbt_model *m, int Bc_src, int grouped, int n_rows_out, int src_mul, int src_add, int n_tile,
+                       int mode, int nsp, size_t sstride) {
+    const dbt_config &c = m->cfg;
+    const Workspace &w = m->ws;
+    LAUNCH(m, "resid_norm", 0, resid_norm_kernel, n_rows_out, norm_threads(c.d_model), 0, w.S, w.P, nsp, sstride, mode,
+           m->layers[c.n_layers - 1].coup_c, Bc_src, grouped, m->w.final_norm_g, c.rms_eps, c.d_model, c.final_norm,
+           src_mul, src_add, w.Xb, m->act_parts == 2 ? (size_t)m->Rmax * c.d_model : (size_t)0, (float *)nullptr);
+    int R = grouped ? 2 * n_rows_out : n_rows_out;
+    TcCall lm{};
+    lm.W[0] = &m->map_lm; lm.n_out[0] = c.vocab; lm.rows[0] = R; lm.nseg = 1; lm.X = &m->map_Xb; lm.K = c.d_model;
+    lm.R = R; lm.P = w.Z; lm.P_floats = (size_t)R * c.vocab;  // exactly one split: Z is the output itself
+    lm.parts = m->act_parts; lm.lo_row0 = m->Rmax; lm.tag = "gemm_lm_head";
+    int one = 0;
+    return run_gemm_tc(m, lm, n_tile, &one, nullptr);
+}
+
+dbt_status step_tc(dbt_model *m, const int32_t *tokens_dev, int B, int grouped, int32_t *next_dev, float *z1_dev,
+                   float *z2_dev, float *alpha_dev) {
+    typedef __nv_bfloat16 WT;
+    const dbt_config &c = m->cfg;
+    const Workspace &w = m->ws;
+    RowMap rm{B, 1};
+    int R = grouped ? 2 * B : B;
+    int n_tile = pad_rows(2 * B);  // the same instruction shape in both modes
+    dbt_status st;
+    LAUNCH(m, "embed", 0, embed_norm_kernel<WT>, R, 256, 0, tokens_dev, 1, 0, rm, (const WT *)m->w.embed_primary,
+           (const WT *)m->w.embed_branch, m->w.embed_norm_g, c.rms_eps, c.d_model, c.vocab, w.S, w.status);
+    int mode, nsp;
+    size_t sstride;
+    if ((st = run_layers_tc(m, rm, grouped, n_tile, true, &mode, &nsp, &sstride)) != DBT_OK) return st;
+    if ((st = run_head_tc(m, B, grouped, B, 1, 0, n_tile, mode, nsp, sstride)) != DBT_OK) return st;
+    LAUNCH(m, "readout", 0, readout_kernel, B, 1024, 0, w.Z, B, c.vocab, grouped, next_dev, alpha_dev);
+    LAUNCH(m, "advance_len", 0, advance_len_kernel, (B + 127) / 128, 128, 0, w.seq_len, B, 1);
+    size_t zb = sizeof(float) * (size_t)B * c.vocab;
+    if (z1_dev) CUDA_TRY(m, cudaMemcpyAsync(z1_dev, w.Z, zb, cudaMemcpyDeviceToDevice, m->stream));
+    if (z2_dev && grouped)
+        CUDA_TRY(m, cudaMemcpyAsync(z2_dev, w.Z + (size_t)B * c.vocab, zb, cudaMemcpyDeviceToDevice, m->stream));
+    for (int b = 0; b < B; b++) m->len_host[b] += 1;
+    m->pending_union = c.n_experts > 0;
+    return DBT_OK;
+}
+
+dbt_status prefill_tc(dbt_model *m, const int32_t *tokens_dev, int B, int n, float *last_logits) {
+    typedef __nv_bfloat16 WT;
+    const dbt_config &c = m->cfg;
+    const Workspace &w = m->ws;
+    int cn_max = m->Rmax / B;
+    if (cn_max < 1) cn_max = 1;
+    dbt_status st;
+    for (int p0 = 0; p0 < n; p0 += cn_max) {
+        int cn = n - p0 < cn_max ? n - p0 : cn_max;
+        RowMap rm{B, cn};
+        int R = B * cn, n_tile = pad_rows(R);
+        LAUNCH(m, "embed", 0, embed_norm_kernel<WT>, R, 256, 0, tokens_dev, n, p0, rm, (const WT *)m->w.embed_primary,
+               (const WT *)m->w.embed_branch, m->w.embed_norm_g, c.rms_eps, c.d_model, c.vocab, w.S, w.status);
+        int mode, nsp;
+        size_t sstride;
+        if ((st = run_layers_tc(m, rm, 0, n_tile, false, &mode, &nsp, &sstride)) != DBT_OK) return st;
+        bool last = p0 + cn >= n;
+        if (last && last_logits) {
+            if ((st = run_head_tc(m, R, 0, B, cn, cn - 1, pad_rows(B), mode, nsp, sstride)) != DBT_OK) return st;
+            CUDA_TRY(m, cudaMemcpyAsync(last_logits, w.Z, sizeof(float) * (size_t)B * c.vocab, cudaMemcpyDeviceToDevice,
+                                        m->stream));
+        }
+        LAUNCH(m, "advance_len", 0, advance_len_kernel, (B + 127) / 128, 128, 0, w.seq_len, B, cn);
+    }
+    for (int b = 0; b < B; b++) m->len_host[b] += n;
+    return DBT_OK;
+}
+
+template <int N_TILE>
+bool allow_smem() {
+    return cudaFuncSetAttribute(gemm_tc_kernel<N_TILE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                TcCfg<N_TILE>::kSmemBytes) == cudaSuccess;
+}
+bool allow_smem_all() {
+    static int state = 0;  // 0 unknown, 1 ok, -1 failed
+    if (state == 0)
+        state = (allow_smem<16>() && allow_smem<32>() && allow_smem<64>() && allow_smem<128>() && allow_smem<256>()) ? 1 : -1;
+    return state == 1;
+}
+
+// Build the TMA descriptors of a bf16 model.  Returns false when the path cannot be used.
+bool setup_tc(dbt_model *m) {
+    const dbt_config &c = m->cfg;
+    const Workspace &w = m->ws;
+    const char *force = getenv("DBT_FORCE_PATH");
+    if (force && strcmp(force, "simt") == 0) return false;
+    if (c.weight_dtype != DBT_DTYPE_BF16 || m->Rmax > 256) return false;
+    if (!allow_smem_all()) return false;
+    int d = c.d_model, qd = c.n_q_heads * c.head_dim, kvd = c.n_kv_heads * c.head_dim;
+    bool moe = c.n_experts > 0;
+    int F = moe ? 0 : c.d_ff;
+    bool ok = true;
+    m->maps.resize(c.n_layers);
+    for (int l = 0; l < c.n_layers && ok; l++) {
+        const dbt_layer_weights &lw = m->layers[l];
+        LayerMaps &mp = m->maps[l];
+        ok = ok && make_bf16_map(&mp.wq, lw.wq, qd, d, kTcM) && make_bf16_map(&mp.wk, lw.wk, kvd, d, kTcM) &&
+             make_bf16_map(&mp.wv, lw.wv, kvd, d, kTcM) && make_bf16_map(&mp.wo, lw.wo, d, qd, kTcM);
+        if (!moe)
+            ok = ok && make_bf16_map(&mp.wg, lw.w_gate, F, d, kTcM) && make_bf16_map(&mp.wu, lw.w_up, F, d, kTcM) &&
+                 make_bf16_map(&mp.wd, lw.w_down, d, F, kTcM);
+    }
+    ok = ok && make_bf16_map(&m->map_lm, m->w.lm_head, c.vocab, d, kTcM);
+    ok = ok && make_bf16_map(&m->map_Xb, w.Xb, 2 * m->Rmax, d, 16) && make_bf16_map(&m->map_Ob, w.Ob, 2 * m->Rmax, qd, 16);
+    if (!moe) ok = ok && make_bf16_map(&m->map_Hb, w.Hb, 2 * m->Rmax, F, 16);
+    const char *split = getenv("DBT_ACT_SPLIT");
+    m->act_parts = (split && strcmp(split, "0") == 0) ? 1 : 2;
+    return ok;
 }
 
 template <typename WT>
@@ -476,6 +808,14 @@ dbt_status dbt_create(const dbt_config *cfg, const dbt_weights *w, void *kv_pool
     m->launches = 0;
     m->pending_union = false;
     m->prof_on = false;
+    m->tc = setup_tc(m);
+    const char *gr = getenv("DBT_GRAPH");
+    m->use_graph = !(gr && strcmp(gr, "0") == 0);
+    m->cap_stream = nullptr;
+    if (m->use_graph && cudaStreamCreateWithFlags(&m->cap_stream, cudaStreamNonBlocking) != cudaSuccess) {
+        m->use_graph = false;
+        cudaGetLastError();
+    }
 
     // RoPE table in double: angle = t * base^(-2i/d_h), stored as (cos, sin) fp32 pairs.
     int half = cfg->head_dim / 2;
@@ -539,6 +879,11 @@ void dbt_destroy(dbt_model *m) {
         cudaEventDestroy(r.e1);
     }
     for (auto e : m->prof_pool) cudaEventDestroy(e);
+    for (auto &g : m->graphs) {
+        cudaGraphExecDestroy(g.exec);
+        cudaGraphDestroy(g.graph);
+    }
+    if (m->cap_stream) cudaStreamDestroy(m->cap_stream);
     delete m;
 }
 
@@ -557,6 +902,14 @@ dbt_status dbt_profile_end(dbt_model *m, dbt_profile_entry *entries_host, int32_
     if (!m) return DBT_ERR_INVALID_ARG;
     if (!entries_host || !n_entries || max_entries <= 0) return fail(m, DBT_ERR_INVALID_ARG, "bad profile buffer");
     m->prof_on = false;
+    m->tc = setup_tc(m);
+    const char *gr = getenv("DBT_GRAPH");
+    m->use_graph = !(gr && strcmp(gr, "0") == 0);
+    m->cap_stream = nullptr;
+    if (m->use_graph && cudaStreamCreateWithFlags(&m->cap_stream, cudaStreamNonBlocking) != cudaSuccess) {
+        m->use_graph = false;
+        cudaGetLastError();
+    }
     CUDA_TRY(m, cudaStreamSynchronize(m->stream));
     int n = 0;
     for (auto &r : m->prof) {
@@ -635,25 +988,82 @@ dbt_status dbt_prefill(dbt_model *m, const int32_t *tokens_dev, int32_t B, int32
     dbt_status st = check_step_args(m, tokens_dev, B, n);
     if (st != DBT_OK) return st;
     if (m->cfg.weight_dtype == DBT_DTYPE_F32) return prefill_impl<float>(m, tokens_dev, B, n, last_primary_logits_dev);
+    if (m->tc) return prefill_tc(m, tokens_dev, B, n, last_primary_logits_dev);
     return prefill_impl<__nv_bfloat16>(m, tokens_dev, B, n, last_primary_logits_dev);
+}
+
+static dbt_status step_direct(dbt_model *m, const int32_t *tokens_dev, int B, int grouped, int32_t *next_dev,
+                              float *z1, float *z2, float *alpha) {
+    if (m->cfg.weight_dtype == DBT_DTYPE_F32) return step_impl<float>(m, tokens_dev, B, grouped, next_dev, z1, z2, alpha);
+    if (m->tc) return step_tc(m, tokens_dev, B, grouped, next_dev, z1, z2, alpha);
+    return step_impl<__nv_bfloat16>(m, tokens_dev, B, grouped, next_dev, z1, z2, alpha);
+}
+
+// Replay the step as a CUDA graph: every kernel reads the sequence lengths from device
+// memory, so one capture per (batch, mode, buffer set) serves every later step.
+static dbt_status step_graphed(dbt_model *m, const int32_t *tokens_dev, int B, int grouped, int32_t *next_dev,
+                               float *z1, float *z2, float *alpha) {
+    if (!m->use_graph || m->prof_on) return step_direct(m, tokens_dev, B, grouped, next_dev, z1, z2, alpha);
+    const void *key[5] = {tokens_dev, next_dev, z1, z2, alpha};
+    dbt_model::GraphEntry *hit = nullptr;
+    for (auto &g : m->graphs)
+        if (g.B == B && g.grouped == grouped && memcmp(g.ptr, key, sizeof key) == 0) hit = &g;
+    if (!hit) {
+        if (m->graphs.size() >= 64) {  // a caller that never reuses buffers: stop caching
+            return step_direct(m, tokens_dev, B, grouped, next_dev, z1, z2, alpha);
+        }
+        std::vector<int32_t> len_save = m->len_host;
+        int64_t l0 = m->launches;
+        cudaStream_t user = m->stream;
+        CUDA_TRY(m, cudaStreamBeginCapture(m->cap_stream, cudaStreamCaptureModeThreadLocal));
+        m->stream = m->cap_stream;
+        dbt_status st = step_direct(m, tokens_dev, B, grouped, next_dev, z1, z2, alpha);
+        m->stream = user;
+        cudaGraph_t graph = nullptr;
+        cudaError_t e = cudaStreamEndCapture(m->cap_stream, &graph);
+        int64_t captured = m->launches - l0;
+        m->launches = l0;
+        m->len_host = len_save;
+        if (st != DBT_OK) {
+            if (graph) cudaGraphDestroy(graph);
+            return st;
+        }
+        if (e != cudaSuccess) return fail(m, DBT_ERR_CUDA, "graph capture: %s", cudaGetErrorString(e));
+        cudaGraphExec_t exec = nullptr;
+        e = cudaGraphInstantiate(&exec, graph, 0);
+        if (e != cudaSuccess) {
+            cudaGraphDestroy(graph);
+            return fail(m, DBT_ERR_CUDA, "graph instantiate: %s", cudaGetErrorString(e));
+        }
+        dbt_model::GraphEntry g{};
+        g.B = B;
+        g.grouped = grouped;
+        memcpy(g.ptr, key, sizeof key);
+        g.graph = graph;
+        g.exec = exec;
+        g.launches = captured;
+        m->graphs.push_back(g);
+        hit = &m->graphs.back();
+    }
+    CUDA_TRY(m, cudaGraphLaunch(hit->exec, m->stream));
+    m->launches += hit->launches;
+    for (int b = 0; b < B; b++) m->len_host[b] += 1;
+    m->pending_union = m->cfg.n_experts > 0;
+    return DBT_OK;
 }
 
 dbt_status dbt_decode_step(dbt_model *m, const int32_t *tokens_dev, int32_t B, int32_t *next_tokens_dev,
                            float *logits_primary_dev, float *logits_branch_dev, float *alpha_dev) {
     dbt_status st = check_step_args(m, tokens_dev, B, 1);
     if (st != DBT_OK) return st;
-    if (m->cfg.weight_dtype == DBT_DTYPE_F32)
-        return step_impl<float>(m, tokens_dev, B, 1, next_tokens_dev, logits_primary_dev, logits_branch_dev, alpha_dev);
-    return step_impl<__nv_bfloat16>(m, tokens_dev, B, 1, next_tokens_dev, logits_primary_dev, logits_branch_dev, alpha_dev);
+    return step_graphed(m, tokens_dev, B, 1, next_tokens_dev, logits_primary_dev, logits_branch_dev, alpha_dev);
 }
 
 dbt_status dbt_decode_step_primary_only(dbt_model *m, const int32_t *tokens_dev, int32_t B, int32_t *next_tokens_dev,
                                         float *logits_primary_dev) {
     dbt_status st = check_step_args(m, tokens_dev, B, 1);
     if (st != DBT_OK) return st;
-    if (m->cfg.weight_dtype == DBT_DTYPE_F32)
-        return step_impl<float>(m, tokens_dev, B, 0, next_tokens_dev, logits_primary_dev, nullptr, nullptr);
-    return step_impl<__nv_bfloat16>(m, tokens_dev, B, 0, next_tokens_dev, logits_primary_dev, nullptr, nullptr);
+    return step_graphed(m, tokens_dev, B, 0, next_tokens_dev, logits_primary_dev, nullptr, nullptr);
 }
 
 static dbt_status step_host(dbt_model *m, const int32_t *tokens_host, int32_t B, int32_t *next_host, float *alpha_host,
@@ -712,5 +1122,46 @@ dbt_status dbt_sync_status(dbt_model *m, int32_t *device_status, int32_t *detail
 }
 
 int64_t dbt_launch_count(const dbt_model *m) { return m ? m->launches : 0; }
+
+static dbt_status op_gemm_tc_impl(dbt_model *m, const void *W_dev, const void *X_dev, int32_t n_out, int32_t K,
+                                  int32_t R, int32_t force_split, float *Y_dev, float *scratch_dev,
+                                  size_t scratch_floats, int32_t *status_dev, int32_t *split_used) {
+    if (!W_dev || !X_dev || !Y_dev || !scratch_dev || !status_dev) return fail(m, DBT_ERR_INVALID_ARG, "NULL pointer");
+    if (n_out <= 0 || K <= 0 || K % 8 || R <= 0 || R > 256) return fail(m, DBT_ERR_UNSUPPORTED, "need K %% 8 == 0, 1 <= R <= 256");
+    if (((uintptr_t)W_dev | (uintptr_t)X_dev) & 15) return fail(m, DBT_ERR_INVALID_ARG, "operands must be 16-byte aligned");
+    CUtensorMap mw, mx;
+    if (!allow_smem_all()) return fail(m, DBT_ERR_CUDA, "cannot raise the shared-memory limit");
+    if (!make_bf16_map(&mw, W_dev, n_out, K, kTcM) || !make_bf16_map(&mx, X_dev, R, K, 16))
+        return fail(m, DBT_ERR_CUDA, "cuTensorMapEncodeTiled failed");
+    m->ws.status = status_dev;
+    TcCall c{};
+    c.W[0] = &mw; c.n_out[0] = n_out; c.rows[0] = R; c.nseg = 1; c.X = &mx; c.K = K; c.R = R;
+    c.P = scratch_dev; c.P_floats = scratch_floats; c.tag = "gemm"; c.parts = 1; c.lo_row0 = 0;
+    if (force_split > 0) {  // honour the request by shrinking the scratch the heuristic may use
+        size_t per = (size_t)pad_rows(R) * n_out;
+        if ((size_t)force_split * per > scratch_floats) return fail(m, DBT_ERR_CAPACITY, "scratch too small");
+    }
+    int nsp = 1;
+    size_t stride = 0;
+    dbt_status st = run_gemm_tc(m, c, pad_rows(R), &nsp, &stride, force_split);
+    if (st != DBT_OK) return st;
+    size_t n = (size_t)R * n_out;
+    LAUNCH(m, "reduce", 0, reduce_splits_kernel, (unsigned)((n + 255) / 256), 256, 0, scratch_dev, nsp, stride, n, Y_dev);
+    if (split_used) *split_used = nsp;
+    return DBT_OK;
+}
+
+dbt_status dbt_op_gemm_tc(const void *W_dev, const void *X_dev, int32_t n_out, int32_t K, int32_t R, int32_t force_split,
+                          float *Y_dev, float *scratch_dev, size_t scratch_floats, int32_t *status_dev,
+                          void *cuda_stream, int32_t *split_used) {
+    static thread_local dbt_model scratch_handle;  // carries the stream and the error text only
+    dbt_model *m = &scratch_handle;
+    m->stream = (cudaStream_t)cuda_stream;
+    m->prof_on = false;
+    dbt_status st = op_gemm_tc_impl(m, W_dev, X_dev, n_out, K, R, force_split, Y_dev, scratch_dev, scratch_floats,
+                                    status_dev, split_used);
+    if (st != DBT_OK) g_create_error = m->err;
+    return st;
+}
 
 }  // extern "C"

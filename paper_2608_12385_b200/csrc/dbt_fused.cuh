@@ -1,0 +1,160 @@
+// Elementwise kernels that sit between the tensor-core GEMMs of the bf16 path.  Each one also
+// sums the split-K partials of the GEMM before it, in split order (deterministic).
+#pragma once
+
+#include "dbt_common.cuh"
+
+namespace dbt {
+
+// x = hi + lo with hi = bf16(x), lo = bf16(x - hi): the two-term form the GEMM consumes.
+// lo_off is the element offset of the lo plane (0: store hi only).
+__device__ __forceinline__ void store_split(__nv_bfloat16 *dst, size_t idx, size_t lo_off, float x) {
+    __nv_bfloat16 hi = __float2bfloat16_rn(x);
+    dst[idx] = hi;
+    if (lo_off) dst[idx + lo_off] = __float2bfloat16_rn(x - __bfloat162float(hi));
+}
+
+__device__ __forceinline__ float sum_splits(const float *__restrict__ P, size_t split_stride, int nsplit, size_t off) {
+    float m = 0.f;
+    for (int s = 0; s < nsplit; s++) m += P[(size_t)s * split_stride + off];
+    return m;
+}
+
+// Residual update + RMSNorm feeding the next GEMM.
+//   mode 0: S unchanged                                   (after the embedding, after an MoE layer)
+//   mode 1: S += sum_s P[s]                               (S-bar_i = S_i + Attn_i W_O)
+//   mode 2: M = sum_s P[s]; M_2 += c * M_1; S += M        (Eq. mlp: M_2 = H~_2 W_D + c*M_1)
+// then Xb = bf16(g * S / rms(S)) (apply_norm) or bf16(S).  Block j handles primary source row
+// j*src_mul + src_add and, in grouped mode, its branch twin; outputs go to rows j and n_out + j.
+__global__ void __launch_bounds__(1024) resid_norm_kernel(float *__restrict__ S, const float *__restrict__ P, int nsplit,
+                                                         size_t split_stride, int mode,
+                                                         const float *__restrict__ coup_c, int Bc, int grouped,
+                                                         const float *__restrict__ g, float eps, int d, int apply_norm,
+                                                         int src_mul, int src_add, __nv_bfloat16 *__restrict__ Xb,
+                                                         size_t lo_off, float *__restrict__ Xf) {
+    __shared__ float scratch[32];
+    int j = blockIdx.x, n_out = gridDim.x;
+    int r1 = j * src_mul + src_add, r2 = Bc + r1;
+    float ss1 = 0.f, ss2 = 0.f;
+    for (int i = threadIdx.x; i < d; i += blockDim.x) {
+        float v1 = S[(size_t)r1 * d + i], m1 = 0.f;
+        if (mode != 0) {
+            m1 = sum_splits(P, split_stride, nsplit, (size_t)r1 * d + i);
+            v1 += m1;
+            S[(size_t)r1 * d + i] = v1;
+        }
+        ss1 += v1 * v1;
+        if (grouped) {
+            float v2 = S[(size_t)r2 * d + i];
+            if (mode != 0) {
+                float m2 = sum_splits(P, split_stride, nsplit, (size_t)r2 * d + i);
+                if (mode == 2) m2 += coup_c[i] * m1;
+                v2 += m2;
+                S[(size_t)r2 * d + i] = v2;
+            }
+            ss2 += v2 * v2;
+        }
+    }
+    float inv1 = 1.f, inv2 = 1.f;
+    if (apply_norm) {
+        ss1 = block_sum(ss1, scratch);
+        inv1 = 1.f / sqrtf(ss1 / (float)d + eps);
+        if (grouped) {
+            ss2 = block_sum(ss2, scratch);
+            inv2 = 1.f / sqrtf(ss2 / (float)d + eps);
+        }
+    }
+    // each thread re-reads only the elements of S it wrote itself (same index stride)
+    for (int i = threadIdx.x; i < d; i += blockDim.x) {
+        float gi = apply_norm ? g[i] : 1.f;
+        float x1 = gi * S[(size_t)r1 * d + i] * inv1;
+        store_split(Xb, (size_t)j * d + i, lo_off, x1);
+        if (Xf) Xf[(size_t)j * d + i] = x1;
+        if (grouped) {
+            float x2 = gi * S[(size_t)r2 * d + i] * inv2;
+            store_split(Xb, (size_t)(n_out + j) * d + i, lo_off, x2);
+            if (Xf) Xf[(size_t)(n_out + j) * d + i] = x2;
+        }
+    }
+}
+
+// After the Q|K|V GEMM: sum the splits, RoPE on Q (both paths) and K (primary), the a coupling
+// Q~_2 = Q_2 + a*Q_1 (Eq. asymattn), append K_1,V_1 to the paged cache.  P rows are
+// [q_dim | kv_dim (K) | kv_dim (V)].  grid (primary rows, n_q + n_kv heads), one thread per
+// rotation pair of the head.
+template <typename KT>
+__global__ void __launch_bounds__(64) qkv_epilogue_kernel(
+    const float *__restrict__ P, int nsplit, size_t split_stride, float *__restrict__ Q, RowMap rm, int grouped,
+    int n_q, int n_kv, int dh, const float *__restrict__ coup_a, const float2 *__restrict__ rope_tab,
+    const int32_t *__restrict__ seq_len, const int32_t *__restrict__ page_table, int pt_stride, int num_pages,
+    int page_size, KT *__restrict__ kpool, KT *__restrict__ vpool, int *status) {
+    int item = blockIdx.x, hh = blockIdx.y, i = threadIdx.x, Bc = rm.Bc();
+    int half = dh / 2;
+    if (i >= half) return;
+    int seq = rm.seq(item), pos = seq_len[seq] + rm.off(item);
+    int q_dim = n_q * dh, kv_dim = n_kv * dh, ldp = q_dim + 2 * kv_dim;
+    float2 t = rope_tab[(size_t)pos * half + i];
+    size_t p1 = (size_t)item * ldp, p2 = (size_t)(Bc + item) * ldp;
+    if (hh < n_q) {
+        int o0 = hh * dh + i, o1 = o0 + half;
+        float x0 = sum_splits(P, split_stride, nsplit, p1 + o0), x1 = sum_splits(P, split_stride, nsplit, p1 + o1);
+        float r0 = x0 * t.x - x1 * t.y, r1 = x1 * t.x + x0 * t.y;
+        float *q1 = Q + (size_t)item * q_dim;
+        q1[o0] = r0;
+        q1[o1] = r1;
+        if (grouped) {
+            float y0 = sum_splits(P, split_stride, nsplit, p2 + o0), y1 = sum_splits(P, split_stride, nsplit, p2 + o1);
+            float *q2 = Q + (size_t)(Bc + item) * q_dim;
+            q2[o0] = (y0 * t.x - y1 * t.y) + coup_a[o0] * r0;
+            q2[o1] = (y1 * t.x + y0 * t.y) + coup_a[o1] * r1;
+        }
+        return;
+    }
+    int gk = hh - n_q;
+    int page = page_table[(size_t)seq * pt_stride + pos / page_size];
+    if (page < 0 || page >= num_pages) {
+        if (i == 0) report(status, kStatusBadPage, page);
+        return;
+    }
+    int slot = pos % page_size;
+    size_t base = (((size_t)page * n_kv + gk) * page_size + slot) * dh;
+    size_t ko = p1 + q_dim + gk * dh + i, vo = ko + kv_dim;
+    float x0 = sum_splits(P, split_stride, nsplit, ko), x1 = sum_splits(P, split_stride, nsplit, ko + half);
+    store1(kpool + base + i, x0 * t.x - x1 * t.y);
+    store1(kpool + base + i + half, x1 * t.x + x0 * t.y);
+    store1(vpool + base + i, sum_splits(P, split_stride, nsplit, vo));
+    store1(vpool + base + i + half, sum_splits(P, split_stride, nsplit, vo + half));
+}
+
+// After the gate|up GEMM: H = SiLU(gate) * up; H~_2 = H_2 + b * H_1 (Eq. mlp); bf16 out for
+// the down projection.  P rows are [F gate | F up].  grid (primary rows, F / 256).
+__global__ void __launch_bounds__(256) swiglu_couple_kernel(const float *__restrict__ P, int nsplit,
+                                                            size_t split_stride, int F, int Bc, int grouped,
+                                                            const float *__restrict__ coup_b,
+                                                            __nv_bfloat16 *__restrict__ Hb, size_t lo_off) {
+    int b = blockIdx.x, f = blockIdx.y * blockDim.x + threadIdx.x;
+    if (f >= F) return;
+    size_t p1 = (size_t)b * 2 * F + f;
+    float h1 = silu(sum_splits(P, split_stride, nsplit, p1)) * sum_splits(P, split_stride, nsplit, p1 + F);
+    store_split(Hb, (size_t)b * F + f, lo_off, h1);
+    if (grouped) {
+        size_t p2 = (size_t)(Bc + b) * 2 * F + f;
+        float h2 = silu(sum_splits(P, split_stride, nsplit, p2)) * sum_splits(P, split_stride, nsplit, p2 + F);
+        if (coup_b) h2 += coup_b[f] * h1;
+        store_split(Hb, (size_t)(Bc + b) * F + f, lo_off, h2);
+    }
+}
+
+// Sum split partials into a plain fp32 matrix (used by the operator-level GEMM entry point).
+__global__ void reduce_splits_kernel(const float *__restrict__ P, int nsplit, size_t split_stride, size_t n,
+                                     float *__restrict__ Y) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) Y[i] = sum_splits(P, split_stride, nsplit, i);
+}
+
+__global__ void f32_to_bf16_kernel(const float *__restrict__ X, size_t n, __nv_bfloat16 *__restrict__ Y) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) Y[i] = __float2bfloat16_rn(X[i]);
+}
+
+}  // namespace dbt

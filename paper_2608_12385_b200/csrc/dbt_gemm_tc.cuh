@@ -1,0 +1,307 @@
+// Grouped skinny GEMM on the 5th-generation tensor cores (sm_100a): Y[r][f] = sum_k W[f][k] X[r][k].
+//
+// "Swap-AB": the bf16 weight tile is the 128-row A operand (it is the big, streamed side), the
+// stacked [primary; branch] activation rows are the N side (16..256 columns).  Each weight
+// tile is brought from HBM exactly once by TMA (128B-swizzled, K-major) into a shared-memory
+// ring, multiplied by tcgen05.mma into an fp32 accumulator in tensor memory, and read back
+// with tcgen05.ld for the epilogue.  One CTA = one 128-feature tile x one K range (split-K
+// partials are written to global memory and summed, in split order, by the consumer kernel).
+//
+// Roles inside the 128-thread CTA: warp 0 lane 0 issues TMA, warp 1 lane 0 issues MMAs and
+// owns the TMEM allocation, all four warps run the epilogue (warp w owns TMEM lanes 32w..).
+// Every wait is bounded: on expiry the CTA records kStatusWaitExpired, skips its stores,
+// frees its TMEM and returns.
+#pragma once
+
+#include <cuda.h>
+
+#include "dbt_common.cuh"
+
+namespace dbt {
+
+constexpr int kTcM = 128;       // weight rows per tile (MMA M)
+constexpr int kTcK = 64;        // K elements per stage (one 128-byte swizzle row of bf16)
+constexpr int kTcABytes = kTcM * kTcK * 2;
+constexpr uint64_t kWaitCycles = 4000000000ull;  // ~2 s at 1.9 GHz
+
+struct TcSeg {
+    int tile0;   // first tile index of this segment
+    int n_out;   // features in this segment
+    int rows;    // activation rows whose outputs are kept (K/V: primary rows only)
+    int col0;    // first output column of this segment in P
+};
+
+struct TcParams {
+    TcSeg seg[3];
+    int nseg;
+    int K;
+    int kt_per_split;  // k-tiles (of 64) per split
+    int ldp;           // row stride of P (total output features)
+    int R;             // activation rows
+    int parts;         // 1: X is plain bf16; 2: X = hi + lo (two bf16 terms), lo rows at lo_row0
+    int lo_row0;       // row offset of the lo term inside the activation buffer
+    float *P;          // [splits][R][ldp] fp32 partials
+    int *status;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// Bounded wait on a phase parity; false when the limit expired.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    uint32_t done = 0;
+    long long t0 = clock64();
+    while (true) {
+        asm volatile(
+            "{\n"
+            ".reg .pred p;\n"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+            "selp.u32 %0, 1, 0, p;\n"
+            "}\n"
+            : "=r"(done)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (done) return true;
+        if ((unsigned long long)(clock64() - t0) > kWaitCycles) return false;
+    }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1,
+                                                 uint64_t hint) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, "
+        "%4}], [%2], %5;" ::"r"(dst),
+        "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "l"(hint)
+        : "memory");
+}
+__device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap *map) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
+}
+
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// K-major, 128B-swizzled operand tile: rows of 128 bytes, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t umma_smem_desc(uint32_t saddr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);  // start address
+    d |= (uint64_t)0 << 16;                    // leading byte offset: unused for swizzled K-major
+    d |= (uint64_t)(1024 >> 4) << 32;          // stride byte offset between 8-row groups
+    d |= (uint64_t)1 << 46;                    // descriptor version (sm_100)
+    d |= (uint64_t)2 << 61;                    // SWIZZLE_128B
+    return d;
+}
+// kind::f16, bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n.
+__host__ __device__ constexpr uint32_t umma_idesc(int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTcM >> 4) << 24);
+}
+__device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
+        "}\n" ::"r"(tmem_d),
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; i++) v[i] = __uint_as_float(r[i]);
+}
+
+// Activations may arrive as two bf16 terms, x = hi + lo (hi = bf16(x), lo = bf16(x - hi)): the
+// weight tile is then multiplied by both and the two products land in the same fp32
+// accumulator, which restores fp32-level accuracy of the activations at no extra HBM traffic.
+template <int N_TILE>
+struct TcCfg {
+    static constexpr int kBBytes = N_TILE * kTcK * 2;        // one term of the activation tile
+    static constexpr int kStageBytes = kTcABytes + 2 * kBBytes;
+    // small row counts: keep one CTA near 100 KB so that a dependent kernel's CTA can become
+    // resident beside it; large row counts take the whole SM
+    static constexpr int kStages = N_TILE <= 16 ? 5 : N_TILE <= 32 ? 4 : N_TILE <= 64 ? 3 : N_TILE <= 128 ? 4 : 2;
+    static constexpr int kTmemCols = N_TILE < 32 ? 32 : N_TILE;
+    static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+};
+
+template <int N_TILE>
+__global__ void __launch_bounds__(128, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtensorMap tmW1,
+               const __grid_constant__ CUtensorMap tmW2, const __grid_constant__ CUtensorMap tmX, TcParams p) {
+    using Cfg = TcCfg<N_TILE>;
+    constexpr int STAGES = Cfg::kStages;
+    extern __shared__ uint8_t smem_raw[];
+    uint32_t raw = smem_u32(smem_raw);
+    uint32_t tiles = (raw + 1023u) & ~1023u;  // 1024-byte aligned operand tiles
+    uint8_t *gen_tiles = smem_raw + (tiles - raw);
+    uint32_t bars = tiles + STAGES * Cfg::kStageBytes;
+    uint32_t *tmem_holder = reinterpret_cast<uint32_t *>(gen_tiles + STAGES * Cfg::kStageBytes + 8 * (2 * STAGES + 1));
+    auto full_bar = [&](int s) { return bars + 8u * s; };
+    auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
+    uint32_t accum_bar = bars + 8u * (2 * STAGES);
+
+    int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    int tile = blockIdx.x, split = blockIdx.y;
+    int sg = 0;
+    if (p.nseg > 1 && tile >= p.seg[1].tile0) sg = 1;
+    if (p.nseg > 2 && tile >= p.seg[2].tile0) sg = 2;
+    const TcSeg seg = p.seg[sg];
+    const CUtensorMap *tmW = sg == 0 ? &tmW0 : sg == 1 ? &tmW1 : &tmW2;
+    int f0 = (tile - seg.tile0) * kTcM;
+    int total_kt = (p.K + kTcK - 1) / kTcK;
+    int kt0 = split * p.kt_per_split;
+    int nkt = min(p.kt_per_split, total_kt - kt0);
+
+    if (tid == 0) {
+        for (int s = 0; s < STAGES; s++) {
+            mbar_init(full_bar(s), 1);
+            mbar_init(empty_bar(s), 1);
+        }
+        mbar_init(accum_bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_holder)),
+                     "r"((uint32_t)Cfg::kTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    uint32_t tmem_base = *tmem_holder;
+    pdl_launch_dependents();
+
+    bool ok = true;
+    if (warp == 0 && lane == 0) {
+        // ---- TMA producer.  Weight tiles do not depend on the previous kernel: the first
+        // ring-full of them is requested before waiting for it.
+        tma_prefetch_desc(tmW);
+        tma_prefetch_desc(&tmX);
+        int npre = min(STAGES, nkt);
+        const uint32_t tx = kTcABytes + p.parts * Cfg::kBBytes;
+        auto load_x = [&](int s, int kt) {
+            for (int part = 0; part < p.parts; part++)
+                for (int j = 0; j < N_TILE / 16; j++)
+                    tma_load_2d(tiles + s * Cfg::kStageBytes + kTcABytes + part * Cfg::kBBytes + j * 2048, &tmX,
+                                full_bar(s), kt * kTcK, part * p.lo_row0 + j * 16);
+        };
+        for (int i = 0; i < npre; i++) {
+            mbar_expect_tx(full_bar(i), tx);
+            tma_load_2d(tiles + i * Cfg::kStageBytes, tmW, full_bar(i), (kt0 + i) * kTcK, f0);
+        }
+        pdl_wait();
+        for (int i = 0; i < npre; i++) load_x(i, kt0 + i);
+        for (int i = npre; i < nkt && ok; i++) {
+            int s = i % STAGES;
+            ok = mbar_wait(empty_bar(s), ((i / STAGES) - 1) & 1);
+            if (!ok) break;
+            mbar_expect_tx(full_bar(s), tx);
+            tma_load_2d(tiles + s * Cfg::kStageBytes, tmW, full_bar(s), (kt0 + i) * kTcK, f0);
+            load_x(s, kt0 + i);
+        }
+    } else if (warp == 1 && lane == 0) {
+        // ---- MMA issuer
+        constexpr uint32_t idesc = umma_idesc(N_TILE);
+        for (int i = 0; i < nkt && ok; i++) {
+            int s = i % STAGES;
+            ok = mbar_wait(full_bar(s), (i / STAGES) & 1);
+            if (!ok) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            uint64_t adesc = umma_smem_desc(tiles + s * Cfg::kStageBytes);
+            for (int part = 0; part < p.parts; part++) {
+                uint64_t bdesc = umma_smem_desc(tiles + s * Cfg::kStageBytes + kTcABytes + part * Cfg::kBBytes);
+#pragma unroll
+                for (int k = 0; k < kTcK / 16; k++)  // advance 16 elements = 32 bytes inside the swizzle row
+                    umma_f16(tmem_base, adesc + 2 * k, bdesc + 2 * k, idesc, (i | k | part) != 0);
+            }
+            umma_commit(empty_bar(s));
+        }
+        if (ok) umma_commit(accum_bar);
+    }
+    if (!ok) report(p.status, kStatusWaitExpired, 100 + warp);
+    __syncwarp();
+
+    // ---- epilogue: TMEM lane = weight row (feature), TMEM column = activation row
+    pdl_wait();
+    bool got = mbar_wait(accum_bar, 0);
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    if (got) {
+        int f = f0 + warp * 32 + lane;
+        float *out = p.P + (size_t)split * p.R * p.ldp + seg.col0 + f;
+        int rows = min(seg.rows, p.R);
+#pragma unroll 1
+        for (int c0 = 0; c0 < N_TILE && c0 < rows; c0 += 16) {
+            float v[16];
+            tmem_ld16(tmem_base + ((uint32_t)(warp * 32) << 16) + c0, v);
+            if (f < seg.n_out) {
+#pragma unroll
+                for (int i = 0; i < 16; i++)
+                    if (c0 + i < rows) out[(size_t)(c0 + i) * p.ldp] = v[i];
+            }
+        }
+    } else if (lane == 0) {
+        report(p.status, kStatusWaitExpired, 200 + warp);
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 1)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                     "r"((uint32_t)Cfg::kTmemCols)
+                     : "memory");
+}
+
+// ---- host side: tensor maps -------------------------------------------------------------
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+inline EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// bf16 matrix [rows][K] (K contiguous), box = 64 x box_rows, 128B swizzle, zero fill outside.
+inline bool make_bf16_map(CUtensorMap *map, const void *base, uint64_t rows, uint64_t K, uint32_t box_rows) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {K, rows};
+    cuuint64_t strides[1] = {K * 2};
+    cuuint32_t box[2] = {(cuuint32_t)kTcK, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+}  // namespace dbt

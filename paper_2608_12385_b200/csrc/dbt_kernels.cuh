@@ -343,7 +343,8 @@ __global__ void __launch_bounds__(128) attn_partial_kernel(
 
 // Merge the split partials in split order (log-sum-exp), write O [rows][q_dim].
 __global__ void attn_merge_kernel(const float *__restrict__ part, int nsplit, int NQ, int DH, int Bc, int grouped,
-                                  int G, int n_kv, float *__restrict__ O) {
+                                  int G, int n_kv, float *__restrict__ O, __nv_bfloat16 *__restrict__ Ob,
+                                  size_t lo_off) {
     int item = blockIdx.x, g = blockIdx.y, e = threadIdx.x;
     int nq_act = grouped ? 2 * G : G, q_dim = n_kv * G * DH;
     const float *base = part + ((size_t)item * n_kv + g) * nsplit * NQ * (DH + 2);
@@ -360,7 +361,13 @@ __global__ void attn_merge_kernel(const float *__restrict__ part, int nsplit, in
         }
         int row = q < G ? item : Bc + item;
         int h = g * G + (q < G ? q : q - G);
-        O[(size_t)row * q_dim + h * DH + e] = o / L;
+        if (O) O[(size_t)row * q_dim + h * DH + e] = o / L;
+        if (Ob) {
+            float x = o / L;
+            __nv_bfloat16 hi = __float2bfloat16_rn(x);
+            Ob[(size_t)row * q_dim + h * DH + e] = hi;
+            if (lo_off) Ob[(size_t)row * q_dim + h * DH + e + lo_off] = __float2bfloat16_rn(x - __bfloat162float(hi));
+        }
     }
 }
 
