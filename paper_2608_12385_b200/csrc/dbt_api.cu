@@ -11,6 +11,7 @@
 #include <string>
 #include <vector>
 
+#include "dbt_attn_mma.cuh"
 #include "dbt_fused.cuh"
 #include "dbt_gemm_tc.cuh"
 #include "dbt_kernels.cuh"
@@ -64,7 +65,8 @@ struct dbt_model {
     // tensor-core path (bf16 models): TMA descriptors of every weight matrix and GEMM input
     bool tc;
     std::vector<LayerMaps> maps;
-    CUtensorMap map_lm, map_Xb, map_Ob, map_Hb;
+    CUtensorMap map_lm, map_Xb, map_Ob, map_Hb, map_kv;
+    bool att_fast;  // TMA + mma.sync attention over the bf16 pool
     int act_parts;  // 2: GEMM inputs carried as hi + lo bf16 terms; 1: plain bf16
     // a decode step is captured once per (batch, mode, buffer set) and replayed as a CUDA graph
     struct GraphEntry {
@@ -137,7 +139,7 @@ size_t carve(const dbt_config &c, char *base, Workspace *ws, int *Rmax_out, int 
     int Fs = moe ? c.n_shared_experts * c.d_expert : 0;
     int F = moe ? (Fs > 0 ? Fs : 8) : c.d_ff;
     int pps = (c.max_seq + c.page_size - 1) / c.page_size;
-    int part_items = Rmax * c.n_kv_heads + 2 * 148;
+    int part_items = Rmax * c.n_kv_heads + 4 * 148;
     w.S = k.take<float>((size_t)Rmax * d);
     w.X = k.take<float>((size_t)Rmax * d);
     w.Q = k.take<float>((size_t)Rmax * qd);
@@ -492,6 +494,41 @@ dbt_status run_gemm_tc(dbt_model *m, const TcCall &c, int n_tile, int *nsplit_ou
     return fail(m, DBT_ERR_UNSUPPORTED, "row tile %d", n_tile);
 }
 
+// Split count of the attention grid: a function of the row count and head count only.
+int attn_splits(int items, int n_kv) {
+    int ns = (4 * 148 + items * n_kv - 1) / (items * n_kv);
+    return ns < 1 ? 1 : ns > 32 ? 32 : ns;
+}
+
+template <int DH>
+dbt_status run_attention_mma(dbt_model *m, const RowMap &rm, int grouped, int layer, double kv_bytes) {
+    const dbt_config &c = m->cfg;
+    const Workspace &w = m->ws;
+    int items = rm.B * rm.cn, G = c.n_q_heads / c.n_kv_heads;
+    AttnParams p{};
+    p.Q = w.Q;
+    p.rm = rm;
+    p.grouped = grouped;
+    p.G = G;
+    p.n_kv = c.n_kv_heads;
+    p.nsplit = attn_splits(items, c.n_kv_heads);
+    p.num_pages = c.num_pages;
+    p.pt_stride = m->pages_per_seq_max;
+    long long plane = (long long)c.num_pages * c.n_kv_heads * c.page_size;
+    p.k_row0 = (long long)layer * 2 * plane;
+    p.v_row0 = p.k_row0 + plane;
+    p.page_table = w.page_table;
+    p.seq_len = w.seq_len;
+    p.part = w.part;
+    p.status = w.status;
+    dim3 grid(items, c.n_kv_heads, p.nsplit);
+    LAUNCH(m, "attention", kv_bytes, attn_mma_kernel<DH>, grid, 160, AttCfg<DH>::kSmemBytes, m->map_kv, p);
+    dim3 mgrid(items, c.n_kv_heads);
+    LAUNCH(m, "attn_merge", 0, attn_merge_kernel, mgrid, DH, 0, w.part, p.nsplit, 16, DH, items, grouped, G, c.n_kv_heads,
+           (float *)nullptr, w.Ob, m->act_parts == 2 ? (size_t)m->Rmax * c.n_q_heads * c.head_dim : (size_t)0);
+    return DBT_OK;
+}
+
 // bf16 layer stack: TMA + tcgen05 GEMMs with the elementwise work between them fused into
 // three small kernels.  On return the last layer's MLP output is still pending in P (dense
 // models): `pending` tells the caller how to fold it into S (mode of resid_norm_kernel).
@@ -532,7 +569,10 @@ dbt_status run_layers_tc(dbt_model *m, const RowMap &rm, int grouped, int n_tile
         LAUNCH(m, "qkv_epilogue", 0, qkv_epilogue_kernel<WT>, dim3(Bc, c.n_q_heads + c.n_kv_heads), 64, 0, w.P, nsp, sstride, w.Q, rm, grouped, c.n_q_heads,
                c.n_kv_heads, c.head_dim, lw.coup_a, w.rope, w.seq_len, w.page_table, m->pages_per_seq_max, c.num_pages,
                c.page_size, kpool, vpool, w.status);
-        if (c.head_dim == 128)
+        if (m->att_fast)
+            st = c.head_dim == 128 ? run_attention_mma<128>(m, rm, grouped, l, kv_bytes)
+                                   : run_attention_mma<64>(m, rm, grouped, l, kv_bytes);
+        else if (c.head_dim == 128)
             st = run_attention<WT, 128>(m, rm, grouped, kpool, vpool, att_split, kv_bytes, true);
         else
             st = run_attention<WT, 64>(m, rm, grouped, kpool, vpool, att_split, kv_bytes, true);
@@ -678,6 +718,14 @@ bool setup_tc(dbt_model *m) {
     ok = ok && make_bf16_map(&m->map_lm, m->w.lm_head, c.vocab, d, kTcM);
     ok = ok && make_bf16_map(&m->map_Xb, w.Xb, 2 * m->Rmax, d, 16) && make_bf16_map(&m->map_Ob, w.Ob, 2 * m->Rmax, qd, 16);
     if (!moe) ok = ok && make_bf16_map(&m->map_Hb, w.Hb, 2 * m->Rmax, F, 16);
+    const char *fa = getenv("DBT_ATTN");
+    m->att_fast = ok && !(fa && strcmp(fa, "simt") == 0) &&
+                  make_kv_map(&m->map_kv, m->kv_pool, (uint64_t)c.n_layers * 2 * c.num_pages * c.n_kv_heads * c.page_size,
+                              c.head_dim) &&
+                  cudaFuncSetAttribute(attn_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       AttCfg<128>::kSmemBytes) == cudaSuccess &&
+                  cudaFuncSetAttribute(attn_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       AttCfg<64>::kSmemBytes) == cudaSuccess;
     const char *split = getenv("DBT_ACT_SPLIT");
     m->act_parts = (split && strcmp(split, "0") == 0) ? 1 : 2;
     return ok;
