@@ -9,6 +9,7 @@
 #include <cstring>
 #include <new>
 #include <string>
+#include <utility>
 #include <vector>
 
 #include "dbt_attn_mma.cuh"
@@ -76,7 +77,8 @@ struct dbt_model {
         cudaGraphExec_t exec;
         int64_t launches;
     };
-    bool use_graph;
+    bool use_graph, use_pdl;
+    std::string pdl_off;
     cudaStream_t cap_stream;
     std::vector<GraphEntry> graphs;
 };
@@ -210,6 +212,38 @@ dbt_status fail(dbt_model *m, dbt_status st, const char *fmt, ...) {
         if (e_ != cudaSuccess) return fail(m, DBT_ERR_CUDA, "%s: %s", #call, cudaGetErrorString(e_)); \
     } while (0)
 
+// Every kernel goes through cudaLaunchKernelEx; with `pdl` the launch carries the programmatic
+// stream-serialization attribute, so the kernel may start while its predecessor drains.  Each
+// kernel calls griddepcontrol.wait before it touches anything its predecessor produced.
+template <typename... Params, typename... Args>
+cudaError_t launch_kernel(cudaStream_t stream, bool pdl, dim3 grid, dim3 block, size_t smem, void (*kernel)(Params...),
+                          Args &&...args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, Params(std::forward<Args>(args))...);
+}
+
+// Debug aid: DBT_PDL_OFF=tag1,tag2 launches those kernel families fully serialized.
+bool pdl_disabled_for(const dbt_model *m, const char *tag) {
+    if (m->pdl_off.empty()) return false;
+    size_t n = strlen(tag), pos = 0;
+    while ((pos = m->pdl_off.find(tag, pos)) != std::string::npos) {
+        bool left = pos == 0 || m->pdl_off[pos - 1] == ',';
+        bool right = pos + n == m->pdl_off.size() || m->pdl_off[pos + n] == ',';
+        if (left && right) return true;
+        pos += n;
+    }
+    return false;
+}
+
 cudaEvent_t prof_event(dbt_model *m) {
     cudaEvent_t e = nullptr;
     if (!m->prof_pool.empty()) {
@@ -230,9 +264,9 @@ cudaEvent_t prof_event(dbt_model *m) {
             p1_ = prof_event(m);                                                                         \
             cudaEventRecord(p0_, (m)->stream);                                                           \
         }                                                                                                \
-        kernel<<<grid, block, smem, (m)->stream>>>(__VA_ARGS__);                                         \
+        cudaError_t e_ = launch_kernel((m)->stream, (m)->use_pdl && !pdl_disabled_for(m, tag), dim3(grid), dim3(block), \
+                                       smem, kernel, __VA_ARGS__);                                       \
         (m)->launches++;                                                                                 \
-        cudaError_t e_ = cudaGetLastError();                                                             \
         if ((m)->prof_on) {                                                                              \
             cudaEventRecord(p1_, (m)->stream);                                                           \
             (m)->prof.push_back(dbt_model::ProfRec{tag, (double)(bytes), p0_, p1_});                     \
@@ -857,6 +891,10 @@ dbt_status dbt_create(const dbt_config *cfg, const dbt_weights *w, void *kv_pool
     m->pending_union = false;
     m->prof_on = false;
     m->tc = setup_tc(m);
+    const char *pd = getenv("DBT_PDL");
+    m->use_pdl = !(pd && strcmp(pd, "0") == 0);
+    const char *po = getenv("DBT_PDL_OFF");
+    m->pdl_off = po ? po : "";
     const char *gr = getenv("DBT_GRAPH");
     m->use_graph = !(gr && strcmp(gr, "0") == 0);
     m->cap_stream = nullptr;
@@ -951,6 +989,10 @@ dbt_status dbt_profile_end(dbt_model *m, dbt_profile_entry *entries_host, int32_
     if (!entries_host || !n_entries || max_entries <= 0) return fail(m, DBT_ERR_INVALID_ARG, "bad profile buffer");
     m->prof_on = false;
     m->tc = setup_tc(m);
+    const char *pd = getenv("DBT_PDL");
+    m->use_pdl = !(pd && strcmp(pd, "0") == 0);
+    const char *po = getenv("DBT_PDL_OFF");
+    m->pdl_off = po ? po : "";
     const char *gr = getenv("DBT_GRAPH");
     m->use_graph = !(gr && strcmp(gr, "0") == 0);
     m->cap_stream = nullptr;
@@ -1206,6 +1248,7 @@ dbt_status dbt_op_gemm_tc(const void *W_dev, const void *X_dev, int32_t n_out, i
     dbt_model *m = &scratch_handle;
     m->stream = (cudaStream_t)cuda_stream;
     m->prof_on = false;
+    m->use_pdl = false;
     dbt_status st = op_gemm_tc_impl(m, W_dev, X_dev, n_out, K, R, force_split, Y_dev, scratch_dev, scratch_floats,
                                     status_dev, split_used);
     if (st != DBT_OK) g_create_error = m->err;

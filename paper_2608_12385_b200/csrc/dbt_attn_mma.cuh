@@ -80,12 +80,6 @@ __global__ void __launch_bounds__(160) attn_mma_kernel(const __grid_constant__ C
     int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     int item = blockIdx.x, g = blockIdx.y, sp = blockIdx.z;
     int Bc = p.rm.Bc(), seq = p.rm.seq(item);
-    int nkeys = p.seq_len[seq] + p.rm.off(item) + 1;
-    int total_pages = (nkeys + 15) >> 4;
-    int pps = (total_pages + p.nsplit - 1) / p.nsplit;
-    int pb = sp * pps, pe = min(total_pages, pb + pps);
-    int jbeg = pb * 16, jend = min(nkeys, pe * 16);
-    int ntiles = jend > jbeg ? (jend - jbeg + kAttTile - 1) / kAttTile : 0;
     int nq_act = p.grouped ? 2 * p.G : p.G, q_dim = p.n_kv * p.G * DH;
 
     if (tid == 0) {
@@ -97,7 +91,13 @@ __global__ void __launch_bounds__(160) attn_mma_kernel(const __grid_constant__ C
     }
     __syncthreads();
     pdl_launch_dependents();
-    pdl_wait();  // Q and the freshly appended K/V come from the previous kernel
+    pdl_wait();  // sequence lengths, Q and the freshly appended K/V come from earlier kernels of the step
+    int nkeys = ld_mut(p.seq_len + seq) + p.rm.off(item) + 1;
+    int total_pages = (nkeys + 15) >> 4;
+    int pps = (total_pages + p.nsplit - 1) / p.nsplit;
+    int pb = sp * pps, pe = min(total_pages, pb + pps);
+    int jbeg = pb * 16, jend = min(nkeys, pe * 16);
+    int ntiles = jend > jbeg ? (jend - jbeg + kAttTile - 1) / kAttTile : 0;
 
     float *out = p.part + (((size_t)item * p.n_kv + g) * p.nsplit + sp) * 16 * (DH + 2);
 
@@ -146,10 +146,10 @@ __global__ void __launch_bounds__(160) attn_mma_kernel(const __grid_constant__ C
 #pragma unroll
         for (int ks = 0; ks < KS; ks++) {
             int k = ks * 16 + c;
-            qa[ks][0] = q0 ? pack_bf16(q0[k] * scale, q0[k + 1] * scale) : 0u;
-            qa[ks][1] = q1 ? pack_bf16(q1[k] * scale, q1[k + 1] * scale) : 0u;
-            qa[ks][2] = q0 ? pack_bf16(q0[k + 8] * scale, q0[k + 9] * scale) : 0u;
-            qa[ks][3] = q1 ? pack_bf16(q1[k + 8] * scale, q1[k + 9] * scale) : 0u;
+            qa[ks][0] = q0 ? pack_bf16(__ldcg(q0 + k) * scale, __ldcg(q0 + k + 1) * scale) : 0u;
+            qa[ks][1] = q1 ? pack_bf16(__ldcg(q1 + k) * scale, __ldcg(q1 + k + 1) * scale) : 0u;
+            qa[ks][2] = q0 ? pack_bf16(__ldcg(q0 + k + 8) * scale, __ldcg(q0 + k + 9) * scale) : 0u;
+            qa[ks][3] = q1 ? pack_bf16(__ldcg(q1 + k + 8) * scale, __ldcg(q1 + k + 9) * scale) : 0u;
         }
     }
     float o[NB][4];

@@ -16,6 +16,24 @@ __device__ __forceinline__ void report(int *status, int code, int detail) {
     if (atomicCAS(status, 0, code) == 0) status[1] = detail;
 }
 
+// Programmatic dependent launch: a kernel lets its successor start early, and waits for its
+// predecessor's results before reading or writing anything that predecessor touches.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_enter() {
+    pdl_launch_dependents();
+    pdl_wait();
+}
+// Under programmatic dependent launch a kernel is resident before its predecessors have
+// finished, so "read-only for the lifetime of the kernel" does not hold for anything another
+// kernel of the step writes (sequence lengths, tokens, activations, partials, the KV pool):
+// such pointers carry no `const __restrict__` (which would permit non-coherent loads), and
+// scalars are read with ld_mut.
+template <typename T>
+__device__ __forceinline__ T ld_mut(const T *p) {
+    return __ldcg(p);
+}
+
 // ---- storage-type loads: 8 consecutive elements widened to fp32 -------------------------
 __device__ __forceinline__ void load8(const float *p, float (&v)[8]) {
     float4 a = *reinterpret_cast<const float4 *>(p);

@@ -14,7 +14,7 @@ __device__ __forceinline__ void store_split(__nv_bfloat16 *dst, size_t idx, size
     if (lo_off) dst[idx + lo_off] = __float2bfloat16_rn(x - __bfloat162float(hi));
 }
 
-__device__ __forceinline__ float sum_splits(const float *__restrict__ P, size_t split_stride, int nsplit, size_t off) {
+__device__ __forceinline__ float sum_splits(const float *P, size_t split_stride, int nsplit, size_t off) {
     float m = 0.f;
     for (int s = 0; s < nsplit; s++) m += P[(size_t)s * split_stride + off];
     return m;
@@ -26,12 +26,13 @@ __device__ __forceinline__ float sum_splits(const float *__restrict__ P, size_t 
 //   mode 2: M = sum_s P[s]; M_2 += c * M_1; S += M        (Eq. mlp: M_2 = H~_2 W_D + c*M_1)
 // then Xb = bf16(g * S / rms(S)) (apply_norm) or bf16(S).  Block j handles primary source row
 // j*src_mul + src_add and, in grouped mode, its branch twin; outputs go to rows j and n_out + j.
-__global__ void __launch_bounds__(1024) resid_norm_kernel(float *__restrict__ S, const float *__restrict__ P, int nsplit,
+__global__ void __launch_bounds__(1024) resid_norm_kernel(float *S, const float *P, int nsplit,
                                                          size_t split_stride, int mode,
                                                          const float *__restrict__ coup_c, int Bc, int grouped,
                                                          const float *__restrict__ g, float eps, int d, int apply_norm,
-                                                         int src_mul, int src_add, __nv_bfloat16 *__restrict__ Xb,
-                                                         size_t lo_off, float *__restrict__ Xf) {
+                                                         int src_mul, int src_add, __nv_bfloat16 *Xb,
+                                                         size_t lo_off, float *Xf) {
+    pdl_enter();
     __shared__ float scratch[32];
     int j = blockIdx.x, n_out = gridDim.x;
     int r1 = j * src_mul + src_add, r2 = Bc + r1;
@@ -84,14 +85,15 @@ __global__ void __launch_bounds__(1024) resid_norm_kernel(float *__restrict__ S,
 // rotation pair of the head.
 template <typename KT>
 __global__ void __launch_bounds__(64) qkv_epilogue_kernel(
-    const float *__restrict__ P, int nsplit, size_t split_stride, float *__restrict__ Q, RowMap rm, int grouped,
+    const float *P, int nsplit, size_t split_stride, float *Q, RowMap rm, int grouped,
     int n_q, int n_kv, int dh, const float *__restrict__ coup_a, const float2 *__restrict__ rope_tab,
-    const int32_t *__restrict__ seq_len, const int32_t *__restrict__ page_table, int pt_stride, int num_pages,
-    int page_size, KT *__restrict__ kpool, KT *__restrict__ vpool, int *status) {
+    const int32_t *seq_len, const int32_t *__restrict__ page_table, int pt_stride, int num_pages,
+    int page_size, KT *kpool, KT *vpool, int *status) {
+    pdl_enter();
     int item = blockIdx.x, hh = blockIdx.y, i = threadIdx.x, Bc = rm.Bc();
     int half = dh / 2;
     if (i >= half) return;
-    int seq = rm.seq(item), pos = seq_len[seq] + rm.off(item);
+    int seq = rm.seq(item), pos = ld_mut(seq_len + seq) + rm.off(item);
     int q_dim = n_q * dh, kv_dim = n_kv * dh, ldp = q_dim + 2 * kv_dim;
     float2 t = rope_tab[(size_t)pos * half + i];
     size_t p1 = (size_t)item * ldp, p2 = (size_t)(Bc + item) * ldp;
@@ -128,10 +130,11 @@ __global__ void __launch_bounds__(64) qkv_epilogue_kernel(
 
 // After the gate|up GEMM: H = SiLU(gate) * up; H~_2 = H_2 + b * H_1 (Eq. mlp); bf16 out for
 // the down projection.  P rows are [F gate | F up].  grid (primary rows, F / 256).
-__global__ void __launch_bounds__(256) swiglu_couple_kernel(const float *__restrict__ P, int nsplit,
+__global__ void __launch_bounds__(256) swiglu_couple_kernel(const float *P, int nsplit,
                                                             size_t split_stride, int F, int Bc, int grouped,
                                                             const float *__restrict__ coup_b,
-                                                            __nv_bfloat16 *__restrict__ Hb, size_t lo_off) {
+                                                            __nv_bfloat16 *Hb, size_t lo_off) {
+    pdl_enter();
     int b = blockIdx.x, f = blockIdx.y * blockDim.x + threadIdx.x;
     if (f >= F) return;
     size_t p1 = (size_t)b * 2 * F + f;
@@ -146,13 +149,15 @@ __global__ void __launch_bounds__(256) swiglu_couple_kernel(const float *__restr
 }
 
 // Sum split partials into a plain fp32 matrix (used by the operator-level GEMM entry point).
-__global__ void reduce_splits_kernel(const float *__restrict__ P, int nsplit, size_t split_stride, size_t n,
-                                     float *__restrict__ Y) {
+__global__ void reduce_splits_kernel(const float *P, int nsplit, size_t split_stride, size_t n,
+                                     float *Y) {
+    pdl_enter();
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i < n) Y[i] = sum_splits(P, split_stride, nsplit, i);
 }
 
-__global__ void f32_to_bf16_kernel(const float *__restrict__ X, size_t n, __nv_bfloat16 *__restrict__ Y) {
+__global__ void f32_to_bf16_kernel(const float *X, size_t n, __nv_bfloat16 *Y) {
+    pdl_enter();
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i < n) Y[i] = __float2bfloat16_rn(X[i]);
 }

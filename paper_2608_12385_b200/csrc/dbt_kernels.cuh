@@ -12,14 +12,15 @@ namespace dbt {
 // ---------------------------------------------------------------------------------------
 // Eq. embeddings: S_1^0 = RMSNorm(E_1[x]), S_2^0 = RMSNorm(E_2[x]).  One block per row.
 template <typename WT>
-__global__ void embed_norm_kernel(const int32_t *__restrict__ tokens, int n, int p0, RowMap rm,
+__global__ void embed_norm_kernel(const int32_t *tokens, int n, int p0, RowMap rm,
                                   const WT *__restrict__ E1, const WT *__restrict__ E2,
                                   const float *__restrict__ g, float eps, int d, int V,
-                                  float *__restrict__ S, int *status) {
+                                  float *S, int *status) {
+    pdl_enter();
     __shared__ float scratch[32];
     int r = blockIdx.x;
     int path = r >= rm.Bc();
-    int tok = tokens[(size_t)rm.seq(r) * n + p0 + rm.off(r)];
+    int tok = ld_mut(tokens + (size_t)rm.seq(r) * n + p0 + rm.off(r));
     if (tok < 0 || tok >= V) {
         if (threadIdx.x == 0) report(status, kStatusBadToken, tok);
         tok = min(max(tok, 0), V - 1);
@@ -37,8 +38,9 @@ __global__ void embed_norm_kernel(const int32_t *__restrict__ tokens, int n, int
 
 // N = RMSNorm(S) (gain g, or no gain when g == nullptr: plain copy scaled by 1).
 // Output row r reads input row r * src_mul + src_add (a gather for "last position" rows).
-__global__ void rmsnorm_kernel(const float *__restrict__ S, const float *__restrict__ g, float eps, int d,
-                               int src_mul, int src_add, int apply, float *__restrict__ N) {
+__global__ void rmsnorm_kernel(const float *S, const float *__restrict__ g, float eps, int d,
+                               int src_mul, int src_add, int apply, float *N) {
+    pdl_enter();
     __shared__ float scratch[32];
     int r = blockIdx.x;
     const float *x = S + ((size_t)r * src_mul + src_add) * d;
@@ -103,6 +105,7 @@ __device__ __forceinline__ void warp_dots(const WT *__restrict__ wrow, const flo
 
 template <typename WT>
 __global__ void __launch_bounds__(kLinWarps * 32) linear_kernel(LinArgs a) {
+    pdl_enter();
     int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     int f = blockIdx.x * kLinWarps + warp;
     int seg = 0;
@@ -164,14 +167,15 @@ __global__ void __launch_bounds__(kLinWarps * 32) linear_kernel(LinArgs a) {
 // and the append of K_1,V_1 to the paged cache (Section 4.4 item 3).  One block per primary
 // row, which also handles its branch twin.
 template <typename KT>
-__global__ void rope_couple_append_kernel(float *__restrict__ Q, const float *__restrict__ Kn,
-                                          const float *__restrict__ Vn, RowMap rm, int grouped, int n_q,
+__global__ void rope_couple_append_kernel(float *Q, const float *Kn,
+                                          const float *Vn, RowMap rm, int grouped, int n_q,
                                           int n_kv, int dh, const float *__restrict__ coup_a,
-                                          const float2 *__restrict__ rope_tab, const int32_t *__restrict__ seq_len,
+                                          const float2 *__restrict__ rope_tab, const int32_t *seq_len,
                                           const int32_t *__restrict__ page_table, int pt_stride, int num_pages,
-                                          int page_size, KT *__restrict__ kpool, KT *__restrict__ vpool, int *status) {
+                                          int page_size, KT *kpool, KT *vpool, int *status) {
+    pdl_enter();
     int item = blockIdx.x, Bc = rm.Bc();
-    int seq = rm.seq(item), pos = seq_len[seq] + rm.off(item);
+    int seq = rm.seq(item), pos = ld_mut(seq_len + seq) + rm.off(item);
     int half = dh / 2, q_dim = n_q * dh, kv_dim = n_kv * dh;
     const float2 *cs = rope_tab + (size_t)pos * half;
     float *q1 = Q + (size_t)item * q_dim;
@@ -217,9 +221,10 @@ __global__ void rope_couple_append_kernel(float *__restrict__ Q, const float *__
 // order.
 template <typename KT, int NQ, int DH>
 __global__ void __launch_bounds__(128) attn_partial_kernel(
-    const float *__restrict__ Q, RowMap rm, int grouped, int G, int n_kv, const KT *__restrict__ kpool,
-    const KT *__restrict__ vpool, const int32_t *__restrict__ page_table, int pt_stride, int num_pages,
-    const int32_t *__restrict__ seq_len, int nsplit, float *__restrict__ part, int *status) {
+    const float *Q, RowMap rm, int grouped, int G, int n_kv, const KT *kpool,
+    const KT *vpool, const int32_t *__restrict__ page_table, int pt_stride, int num_pages,
+    const int32_t *seq_len, int nsplit, float *part, int *status) {
+    pdl_enter();
     constexpr int TPB = 128, CH = 128, PS = 16, SUB = TPB / DH;
     __shared__ float qs[NQ][DH];
     __shared__ float sc[NQ][CH];
@@ -228,7 +233,7 @@ __global__ void __launch_bounds__(128) attn_partial_kernel(
     int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     int item = blockIdx.x, g = blockIdx.y, sp = blockIdx.z;
     int Bc = rm.Bc(), seq = rm.seq(item);
-    int nkeys = seq_len[seq] + rm.off(item) + 1;
+    int nkeys = ld_mut(seq_len + seq) + rm.off(item) + 1;
     int nq_act = grouped ? 2 * G : G, q_dim = n_kv * G * DH;
     float scale = 1.f / sqrtf((float)DH);
     for (int idx = tid; idx < NQ * DH; idx += TPB) {
@@ -342,9 +347,10 @@ __global__ void __launch_bounds__(128) attn_partial_kernel(
 }
 
 // Merge the split partials in split order (log-sum-exp), write O [rows][q_dim].
-__global__ void attn_merge_kernel(const float *__restrict__ part, int nsplit, int NQ, int DH, int Bc, int grouped,
-                                  int G, int n_kv, float *__restrict__ O, __nv_bfloat16 *__restrict__ Ob,
+__global__ void attn_merge_kernel(const float *part, int nsplit, int NQ, int DH, int Bc, int grouped,
+                                  int G, int n_kv, float *O, __nv_bfloat16 *Ob,
                                   size_t lo_off) {
+    pdl_enter();
     int item = blockIdx.x, g = blockIdx.y, e = threadIdx.x;
     int nq_act = grouped ? 2 * G : G, q_dim = n_kv * G * DH;
     const float *base = part + ((size_t)item * n_kv + g) * nsplit * NQ * (DH + 2);
@@ -384,8 +390,9 @@ __device__ __forceinline__ ArgBest better(ArgBest a, ArgBest b) {
     return a;
 }
 
-__global__ void __launch_bounds__(1024) readout_kernel(const float *__restrict__ Z, int B, int V, int grouped,
-                                                       int32_t *__restrict__ next, float *__restrict__ alpha_out) {
+__global__ void __launch_bounds__(1024) readout_kernel(const float *Z, int B, int V, int grouped,
+                                                       int32_t *next, float *alpha_out) {
+    pdl_enter();
     __shared__ float scratch[32];
     __shared__ float bv[32];
     __shared__ int bi[32];
@@ -442,6 +449,7 @@ __global__ void __launch_bounds__(1024) readout_kernel(const float *__restrict__
 }
 
 __global__ void advance_len_kernel(int32_t *seq_len, int B, int n) {
+    pdl_enter();
     int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b < B) seq_len[b] += n;
 }
@@ -452,9 +460,10 @@ __global__ void advance_len_kernel(int32_t *seq_len, int B, int n) {
 // Router: softmax over E logits, top-k by repeated "largest remaining, lowest index first",
 // weights renormalised over the selection.  Replay: the branch row takes its primary twin's
 // selection and weighs it with its own probabilities.  One warp per row.
-__global__ void route_kernel(const float *__restrict__ logits, int E, int Bc, int k_p, int k_b, int kmax, int replay,
-                             int32_t *__restrict__ idx, float *__restrict__ wts, int32_t *__restrict__ last,
+__global__ void route_kernel(const float *logits, int E, int Bc, int k_p, int k_b, int kmax, int replay,
+                             int32_t *idx, float *wts, int32_t *__restrict__ last,
                              int last_stride_path) {
+    pdl_enter();
     extern __shared__ float smem[];
     float *p = smem;                                   // [E] own-row probabilities
     unsigned char *taken = (unsigned char *)(smem + E);  // [E]
@@ -496,8 +505,9 @@ __global__ void route_kernel(const float *__restrict__ logits, int E, int Bc, in
 }
 
 // Per-expert lists of (row, slot) entries in ascending order, and the size of the union.
-__global__ void moe_lists_kernel(const int32_t *__restrict__ idx, int R, int kmax, int E, int cap,
-                                 int32_t *__restrict__ cnt, int32_t *__restrict__ list, int32_t *union_count) {
+__global__ void moe_lists_kernel(const int32_t *idx, int R, int kmax, int E, int cap,
+                                 int32_t *cnt, int32_t *list, int32_t *union_count) {
+    pdl_enter();
     int e = blockIdx.x * blockDim.x + threadIdx.x;
     if (e >= E) return;
     int c = 0;
@@ -512,8 +522,9 @@ __global__ void moe_lists_kernel(const int32_t *__restrict__ idx, int R, int kma
 // matrices once for all its entries of both paths.  grid (ceil(Fe/warps), E).
 template <typename WT>
 __global__ void __launch_bounds__(kLinWarps * 32) expert_gateup_kernel(
-    const WT *__restrict__ Wg, const WT *__restrict__ Wu, int Fe, int d, const float *__restrict__ X, int kmax,
-    const int32_t *__restrict__ cnt, const int32_t *__restrict__ list, int cap, float *__restrict__ Hexp) {
+    const WT *__restrict__ Wg, const WT *__restrict__ Wu, int Fe, int d, const float *X, int kmax,
+    const int32_t *cnt, const int32_t *list, int cap, float *Hexp) {
+    pdl_enter();
     int e = blockIdx.y, n = cnt[e];
     if (n == 0) return;
     int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -541,8 +552,9 @@ __global__ void __launch_bounds__(kLinWarps * 32) expert_gateup_kernel(
 // Routed experts, down projection: Yexp[entry] = W_D[e] Hexp[entry].  grid (ceil(d/warps), E).
 template <typename WT>
 __global__ void __launch_bounds__(kLinWarps * 32) expert_down_kernel(
-    const WT *__restrict__ Wd, int Fe, int d, const float *__restrict__ Hexp, const int32_t *__restrict__ cnt,
-    const int32_t *__restrict__ list, int cap, float *__restrict__ Yexp) {
+    const WT *__restrict__ Wd, int Fe, int d, const float *Hexp, const int32_t *cnt,
+    const int32_t *list, int cap, float *Yexp) {
+    pdl_enter();
     int e = blockIdx.y, n = cnt[e];
     if (n == 0) return;
     int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -568,9 +580,10 @@ __global__ void __launch_bounds__(kLinWarps * 32) expert_down_kernel(
 
 // M_1 = sum_j w_1j Expert_j(m_1) + G(m_1);  M_2 = sum_j w_2j Expert_j(m_2) + G~(m_2) + c*M_1;
 // S_i += M_i.  Slots are summed in slot order.  One block per primary row.
-__global__ void moe_combine_kernel(const float *__restrict__ Yexp, const float *__restrict__ Msh,
-                                   const int32_t *__restrict__ idx, const float *__restrict__ wts, int kmax, int Bc,
-                                   int grouped, const float *__restrict__ coup_c, int d, float *__restrict__ S) {
+__global__ void moe_combine_kernel(const float *Yexp, const float *Msh,
+                                   const int32_t *idx, const float *wts, int kmax, int Bc,
+                                   int grouped, const float *__restrict__ coup_c, int d, float *S) {
+    pdl_enter();
     int b = blockIdx.x;
     for (int i = threadIdx.x; i < d; i += blockDim.x) {
         float m1 = 0.f;
