@@ -27,7 +27,7 @@ struct Workspace {
     // fp32 activations, rows = Rmax unless noted
     float *S, *X, *Q, *Kn, *Vn, *O, *G1, *M, *Z, *part, *Zrows;
     float2 *rope;
-    int32_t *seq_len, *page_table, *status, *tokens_stage, *next_stage;
+    int32_t *seq_len, *page_table, *status, *tokens_stage, *next_stage, *att_tickets, *gemm_tickets;
     float *alpha_stage;
     // MoE
     float *rlogits, *rwts, *Hexp, *Yexp, *Msh, *Hsh;
@@ -157,6 +157,8 @@ size_t carve(const dbt_config &c, char *base, Workspace *ws, int *Rmax_out, int 
     w.seq_len = k.take<int32_t>(c.max_batch);
     w.page_table = k.take<int32_t>((size_t)c.max_batch * pps);
     w.status = k.take<int32_t>(4);
+    w.att_tickets = k.take<int32_t>((size_t)Rmax * c.n_kv_heads);
+    w.gemm_tickets = k.take<int32_t>(4096);
     w.tokens_stage = k.take<int32_t>(c.max_batch);
     w.next_stage = k.take<int32_t>(c.max_batch);
     w.alpha_stage = k.take<float>(c.max_batch);
@@ -554,12 +556,12 @@ dbt_status run_attention_mma(dbt_model *m, const RowMap &rm, int grouped, int la
     p.page_table = w.page_table;
     p.seq_len = w.seq_len;
     p.part = w.part;
+    p.tickets = w.att_tickets;
+    p.Ob = w.Ob;
+    p.lo_off = m->act_parts == 2 ? (size_t)m->Rmax * c.n_q_heads * c.head_dim : (size_t)0;
     p.status = w.status;
     dim3 grid(items, c.n_kv_heads, p.nsplit);
     LAUNCH(m, "attention", kv_bytes, attn_mma_kernel<DH>, grid, 160, AttCfg<DH>::kSmemBytes, m->map_kv, p);
-    dim3 mgrid(items, c.n_kv_heads);
-    LAUNCH(m, "attn_merge", 0, attn_merge_kernel, mgrid, DH, 0, w.part, p.nsplit, 16, DH, items, grouped, G, c.n_kv_heads,
-           (float *)nullptr, w.Ob, m->act_parts == 2 ? (size_t)m->Rmax * c.n_q_heads * c.head_dim : (size_t)0);
     return DBT_OK;
 }
 
@@ -926,6 +928,8 @@ dbt_status dbt_create(const dbt_config *cfg, const dbt_weights *w, void *kv_pool
         e = cudaMemcpyAsync(m->ws.page_table, pt.data(), pt.size() * sizeof(int32_t), cudaMemcpyHostToDevice, m->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(m->ws.seq_len, 0, sizeof(int32_t) * cfg->max_batch, m->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(m->ws.status, 0, sizeof(int32_t) * 4, m->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(m->ws.att_tickets, 0, sizeof(int32_t) * (size_t)m->Rmax * cfg->n_kv_heads, m->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(m->ws.gemm_tickets, 0, sizeof(int32_t) * 4096, m->stream);
     if (e == cudaSuccess && moe) {
         e = cudaMemsetAsync(m->ws.last_experts, 0xff, sizeof(int32_t) * (size_t)cfg->n_layers * 2 * cfg->max_batch * kmax_of(*cfg), m->stream);
         if (e == cudaSuccess) e = cudaMemsetAsync(m->ws.union_cnt, 0, sizeof(int32_t) * cfg->n_layers, m->stream);

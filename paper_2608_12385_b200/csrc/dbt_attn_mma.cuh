@@ -27,6 +27,9 @@ struct AttnParams {
     long long k_row0, v_row0;  // first row of this layer's K / V planes in the pool's 2-D view
     const int32_t *page_table, *seq_len;
     float *part;  // [items][n_kv][nsplit][16][DH + 2]
+    int *tickets;  // [items][n_kv] arrival counters (zero between launches)
+    __nv_bfloat16 *Ob;  // [rows][q_dim] attention output, hi plane (+ lo plane at lo_off)
+    size_t lo_off;
     int *status;
 };
 
@@ -66,7 +69,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 }
 
 template <int DH>
-__global__ void __launch_bounds__(160) attn_mma_kernel(const __grid_constant__ CUtensorMap tmKV, AttnParams p) {
+__global__ void __launch_bounds__(160, 3) attn_mma_kernel(const __grid_constant__ CUtensorMap tmKV, AttnParams p) {
     using Cfg = AttCfg<DH>;
     constexpr int STAGES = Cfg::kStages, HALVES = Cfg::kHalves, KS = DH / 16, NB = DH / 8;
     extern __shared__ uint8_t smem_raw[];
@@ -293,9 +296,44 @@ __global__ void __launch_bounds__(160) attn_mma_kernel(const __grid_constant__ C
         }
         out[(size_t)q * (DH + 2) + e] = ok ? acc : 0.f;
         if (e == 0) {
-            out[(size_t)q * (DH + 2) + DH] = ok ? M * kLn2 : -INFINITY;  // natural-log units for the merge
+            out[(size_t)q * (DH + 2) + DH] = ok ? M * kLn2 : -INFINITY;  // natural-log units
             out[(size_t)q * (DH + 2) + DH + 1] = ok ? L : 0.f;
         }
+    }
+    // ---- the last split to arrive for this (row, KV head) folds all splits in split order
+    __threadfence();
+    asm volatile("bar.sync 1, 128;" ::: "memory");
+    int *flag = reinterpret_cast<int *>(sc_l + kAttWarps * 16);
+    if (tid == 0) {
+        int *tk = p.tickets + (size_t)item * p.n_kv + g;
+        int t = atomicAdd(tk, 1);
+        int last = t == p.nsplit - 1;
+        if (last) atomicExch(tk, 0);
+        *flag = last;
+    }
+    asm volatile("bar.sync 1, 128;" ::: "memory");
+    if (!*flag) return;
+    __threadfence();
+    const float *base = p.part + ((size_t)item * p.n_kv + g) * p.nsplit * 16 * (DH + 2);
+    for (int idx = tid; idx < nq_act * DH; idx += 128) {
+        int q = idx / DH, e = idx % DH;
+        float M = -INFINITY;
+        for (int s2 = 0; s2 < p.nsplit; s2++) M = fmaxf(M, __ldcg(base + ((size_t)s2 * 16 + q) * (DH + 2) + DH));
+        float L = 0.f, acc = 0.f;
+        for (int s2 = 0; s2 < p.nsplit; s2++) {
+            const float *pp = base + ((size_t)s2 * 16 + q) * (DH + 2);
+            float ms = __ldcg(pp + DH);
+            float f = ms == -INFINITY ? 0.f : expf(ms - M);
+            L += __ldcg(pp + DH + 1) * f;
+            acc += __ldcg(pp + e) * f;
+        }
+        float x = acc / L;
+        int row = q < p.G ? item : Bc + item;
+        int h = g * p.G + (q < p.G ? q : q - p.G);
+        size_t o_idx = (size_t)row * q_dim + (size_t)h * DH + e;
+        __nv_bfloat16 hi = __float2bfloat16_rn(x);
+        p.Ob[o_idx] = hi;
+        if (p.lo_off) p.Ob[o_idx + p.lo_off] = __float2bfloat16_rn(x - __bfloat162float(hi));
     }
 }
 
