@@ -68,6 +68,7 @@ struct dbt_model {
     std::vector<LayerMaps> maps;
     CUtensorMap map_lm, map_Xb, map_Ob, map_Hb, map_kv;
     bool att_fast;  // TMA + mma.sync attention over the bf16 pool
+    int num_sms;
     int act_parts;  // 2: GEMM inputs carried as hi + lo bf16 terms; 1: plain bf16
     // a decode step is captured once per (batch, mode, buffer set) and replayed as a CUDA graph
     struct GraphEntry {
@@ -530,12 +531,6 @@ dbt_status run_gemm_tc(dbt_model *m, const TcCall &c, int n_tile, int *nsplit_ou
     return fail(m, DBT_ERR_UNSUPPORTED, "row tile %d", n_tile);
 }
 
-// Split count of the attention grid: a function of the row count and head count only.
-int attn_splits(int items, int n_kv) {
-    int ns = (4 * 148 + items * n_kv - 1) / (items * n_kv);
-    return ns < 1 ? 1 : ns > 32 ? 32 : ns;
-}
-
 template <int DH>
 dbt_status run_attention_mma(dbt_model *m, const RowMap &rm, int grouped, int layer, double kv_bytes) {
     const dbt_config &c = m->cfg;
@@ -547,7 +542,6 @@ dbt_status run_attention_mma(dbt_model *m, const RowMap &rm, int grouped, int la
     p.grouped = grouped;
     p.G = G;
     p.n_kv = c.n_kv_heads;
-    p.nsplit = attn_splits(items, c.n_kv_heads);
     p.num_pages = c.num_pages;
     p.pt_stride = m->pages_per_seq_max;
     long long plane = (long long)c.num_pages * c.n_kv_heads * c.page_size;
@@ -560,7 +554,8 @@ dbt_status run_attention_mma(dbt_model *m, const RowMap &rm, int grouped, int la
     p.Ob = w.Ob;
     p.lo_off = m->act_parts == 2 ? (size_t)m->Rmax * c.n_q_heads * c.head_dim : (size_t)0;
     p.status = w.status;
-    dim3 grid(items, c.n_kv_heads, p.nsplit);
+    if (items > kAttMaxItems) return fail(m, DBT_ERR_CAPACITY, "attention rows %d exceed %d", items, kAttMaxItems);
+    dim3 grid(2 * m->num_sms);  // two resident CTAs per SM; each takes an equal share of all K/V tiles
     LAUNCH(m, "attention", kv_bytes, attn_mma_kernel<DH>, grid, 160, AttCfg<DH>::kSmemBytes, m->map_kv, p);
     return DBT_OK;
 }
@@ -892,6 +887,11 @@ dbt_status dbt_create(const dbt_config *cfg, const dbt_weights *w, void *kv_pool
     m->launches = 0;
     m->pending_union = false;
     m->prof_on = false;
+    {
+        int dev = 0, sms = 148;
+        if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        m->num_sms = sms > 0 && sms <= 148 ? sms : 148;  // the partial buffer is sized for 2 x 148 CTAs
+    }
     m->tc = setup_tc(m);
     const char *pd = getenv("DBT_PDL");
     m->use_pdl = !(pd && strcmp(pd, "0") == 0);
@@ -992,18 +992,6 @@ dbt_status dbt_profile_end(dbt_model *m, dbt_profile_entry *entries_host, int32_
     if (!m) return DBT_ERR_INVALID_ARG;
     if (!entries_host || !n_entries || max_entries <= 0) return fail(m, DBT_ERR_INVALID_ARG, "bad profile buffer");
     m->prof_on = false;
-    m->tc = setup_tc(m);
-    const char *pd = getenv("DBT_PDL");
-    m->use_pdl = !(pd && strcmp(pd, "0") == 0);
-    const char *po = getenv("DBT_PDL_OFF");
-    m->pdl_off = po ? po : "";
-    const char *gr = getenv("DBT_GRAPH");
-    m->use_graph = !(gr && strcmp(gr, "0") == 0);
-    m->cap_stream = nullptr;
-    if (m->use_graph && cudaStreamCreateWithFlags(&m->cap_stream, cudaStreamNonBlocking) != cudaSuccess) {
-        m->use_graph = false;
-        cudaGetLastError();
-    }
     CUDA_TRY(m, cudaStreamSynchronize(m->stream));
     int n = 0;
     for (auto &r : m->prof) {

@@ -1,19 +1,26 @@
 // Grouped decode attention for a bf16 paged KV cache (sm_100a).
 //
-// One CTA per (primary row, KV head, split of the context).  The G primary query heads of
-// that KV head and, in grouped mode, the G coupled branch heads (Q~_2 = Q_2 + a*Q_1) form one
-// 16-row query tile, so every K/V page is fetched from HBM once and serves both paths
-// (Section 4.1: "grouped or fused query execution lets the two paths share reads of the
-// primary keys and values").  Keys 0..pos inclusive: the K_1,V_1 appended this step is
-// already in its page.
+// The G primary query heads of a KV head and, in grouped mode, the G coupled branch heads
+// (Q~_2 = Q_2 + a*Q_1) form one 16-row query tile, so every K/V page is fetched from HBM once
+// and serves both paths (Section 4.1: "grouped or fused query execution lets the two paths
+// share reads of the primary keys and values").  Keys 0..pos inclusive: the K_1,V_1 appended
+// this step is already in its page.
+//
+// Work decomposition.  All (row, KV head) pairs are laid end to end in units of one 64-token
+// tile; the grid is a fixed number of CTAs (two per SM) and CTA c takes the contiguous unit
+// range [c*q, (c+1)*q), q = max(ceil(units / CTAs), 4, ceil(longest pair / 31)).  A range may
+// end inside a pair or cover several short pairs: each (CTA, pair) intersection is one
+// segment, whose un-normalised partial (m, l, O) goes to slot c + pair (unique, and consecutive
+// for one pair).  The last segment of a pair to arrive folds all of that pair's segments in
+// segment order, so the result does not depend on arrival order.  Every SM therefore streams
+// the same number of K/V bytes (to within one tile) whatever the batch and context mix.
 //
 // Data movement: a producer warp walks the page table and brings 16-token pages in with
-// tiled TMA copies (128B swizzle) into a shared-memory ring, 64 tokens per stage.  Math:
-// four consumer warps, one page each per stage; S = Q K^T and O += P V with mma.sync
-// m16n8k16 (bf16 in, fp32 accumulate), operands read with ldmatrix through the swizzle; each
-// warp keeps its own running (max, sum, O) and the four are folded in warp order at the end.
-// The CTA writes an un-normalised partial (m, l, O) per split; attn_merge_kernel folds the
-// splits in split order.  All waits are bounded.
+// tiled TMA copies (128B swizzle) into a shared-memory ring, 64 tokens per stage, ~190 KB in
+// flight per SM.  Math: four consumer warps, one page each per stage; S = Q K^T and O += P V
+// with mma.sync m16n8k16 (bf16 in, fp32 accumulate), operands read with ldmatrix through the
+// swizzle; each warp keeps its own running (max, sum, O) and the four are folded in a fixed
+// order at the end of a segment.  All waits are bounded.
 #pragma once
 
 #include "dbt_gemm_tc.cuh"
@@ -23,28 +30,32 @@ namespace dbt {
 struct AttnParams {
     const float *Q;  // [rows][q_dim] fp32, post-RoPE, branch rows already coupled
     RowMap rm;
-    int grouped, G, n_kv, nsplit, num_pages, pt_stride;
+    int grouped, G, n_kv, num_pages, pt_stride;
     long long k_row0, v_row0;  // first row of this layer's K / V planes in the pool's 2-D view
     const int32_t *page_table, *seq_len;
-    float *part;  // [items][n_kv][nsplit][16][DH + 2]
-    int *tickets;  // [items][n_kv] arrival counters (zero between launches)
+    float *part;        // [CTAs + pairs][16][DH + 2] segment partials
+    int *tickets;       // [rows][n_kv] arrival counters (zero between launches)
     __nv_bfloat16 *Ob;  // [rows][q_dim] attention output, hi plane (+ lo plane at lo_off)
     size_t lo_off;
     int *status;
 };
 
-constexpr int kAttTile = 64;      // tokens per pipeline stage (4 pages)
-constexpr int kAttWarps = 4;      // consumer warps, one page each
+constexpr int kAttTile = 64;       // tokens per pipeline stage (4 pages)
+constexpr int kAttWarps = 4;       // consumer warps, one page each
+constexpr int kAttMaxItems = 256;  // rows per launch (prefill chunks and batches stay below)
+constexpr int kAttMinUnits = 4;    // a CTA takes at least 4 tiles (256 tokens)
+constexpr int kAttMaxSeg = 32;     // segments per pair the final fold handles at once
 constexpr float kLog2e = 1.4426950408889634f;
-constexpr float kLn2 = 0.6931471805599453f;
 
 template <int DH>
 struct AttCfg {
     static constexpr int kHalves = DH / 64;                 // 128-byte column groups per row
     static constexpr int kPageBytes = 16 * DH * 2;          // one page of K (or V) for one head
     static constexpr int kStageBytes = 2 * 4 * kPageBytes;  // K + V, 4 pages
-    static constexpr int kStages = DH == 128 ? 2 : 4;
-    static constexpr int kSmemBytes = kStages * kStageBytes + 1024 + 128;
+    static constexpr int kStages = DH == 128 ? 3 : 6;       // 96 KB ring: two CTAs keep ~190 KB in flight per SM
+    // scratch: one [16][DH] fp32 slot (Q tile / warp fold / fold weights), m, l, flag, row tables
+    static constexpr int kScratchBytes = (16 * DH + 2 * 16 + 8 + 2 * kAttMaxItems + 8) * 4;
+    static constexpr int kSmemBytes = kStages * kStageBytes + 1024 + 128 + kScratchBytes;
 };
 
 __device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4]) {
@@ -67,9 +78,10 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t *>(&v);
 }
+__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
 template <int DH>
-__global__ void __launch_bounds__(160, 3) attn_mma_kernel(const __grid_constant__ CUtensorMap tmKV, AttnParams p) {
+__global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant__ CUtensorMap tmKV, AttnParams p) {
     using Cfg = AttCfg<DH>;
     constexpr int STAGES = Cfg::kStages, HALVES = Cfg::kHalves, KS = DH / 16, NB = DH / 8;
     extern __shared__ uint8_t smem_raw[];
@@ -79,10 +91,15 @@ __global__ void __launch_bounds__(160, 3) attn_mma_kernel(const __grid_constant_
     uint32_t bars = tiles + STAGES * Cfg::kStageBytes;
     auto full_bar = [&](int s) { return bars + 8u * s; };
     auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
+    float *sc_o = reinterpret_cast<float *>(gen + STAGES * Cfg::kStageBytes + 128);  // [16][DH]
+    float *sc_m = sc_o + 16 * DH;                                                   // [16]
+    float *sc_l = sc_m + 16;                                                        // [16]
+    int *flag = reinterpret_cast<int *>(sc_l + 16);                                 // [0] last?, [1] longest pair
+    int *cum = flag + 8;                 // [items + 1] prefix of tiles per row
+    int *nk_s = cum + kAttMaxItems + 1;  // [items] visible keys per row
 
     int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    int item = blockIdx.x, g = blockIdx.y, sp = blockIdx.z;
-    int Bc = p.rm.Bc(), seq = p.rm.seq(item);
+    int items = p.rm.Bc(), Bc = items;
     int nq_act = p.grouped ? 2 * p.G : p.G, q_dim = p.n_kv * p.G * DH;
 
     if (tid == 0) {
@@ -92,248 +109,339 @@ __global__ void __launch_bounds__(160, 3) attn_mma_kernel(const __grid_constant_
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    __syncthreads();
     pdl_launch_dependents();
     pdl_wait();  // sequence lengths, Q and the freshly appended K/V come from earlier kernels of the step
-    int nkeys = ld_mut(p.seq_len + seq) + p.rm.off(item) + 1;
-    int total_pages = (nkeys + 15) >> 4;
-    int pps = (total_pages + p.nsplit - 1) / p.nsplit;
-    int pb = sp * pps, pe = min(total_pages, pb + pps);
-    int jbeg = pb * 16, jend = min(nkeys, pe * 16);
-    int ntiles = jend > jbeg ? (jend - jbeg + kAttTile - 1) / kAttTile : 0;
-
-    float *out = p.part + (((size_t)item * p.n_kv + g) * p.nsplit + sp) * 16 * (DH + 2);
+    if (warp == 0) {
+        int running = 0, longest = 0;
+        if (lane == 0) cum[0] = 0;
+        for (int base = 0; base < items; base += 32) {
+            int i = base + lane, nk = 0, u = 0;
+            if (i < items) {
+                nk = ld_mut(p.seq_len + p.rm.seq(i)) + p.rm.off(i) + 1;
+                u = (nk + kAttTile - 1) / kAttTile;
+                nk_s[i] = nk;
+            }
+            int incl = u, mx = u;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                int t = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += t;
+                mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+            }
+            longest = max(longest, mx);
+            if (i < items) cum[i + 1] = running + incl;
+            running += __shfl_sync(0xffffffffu, incl, 31);
+        }
+        if (lane == 0) flag[1] = longest;
+    }
+    __syncthreads();
+    const int U = cum[items] * p.n_kv, C = gridDim.x;
+    const int quota = max(max((U + C - 1) / C, kAttMinUnits), (flag[1] + kAttMaxSeg - 2) / (kAttMaxSeg - 1));
+    const int u0 = blockIdx.x * quota, u1 = min(U, u0 + quota);
+    if (u0 >= U) return;
+    int item = 0;
+    while (cum[item + 1] * p.n_kv <= u0) item++;
 
     if (warp == kAttWarps) {
-        // ---- producer: page table walk + TMA
+        // ---- producer: walks the same segments as the consumers; page table walk + TMA
         if (lane == 0) {
             tma_prefetch_desc(&tmKV);
             bool ok = true;
-            for (int i = 0; i < ntiles && ok; i++) {
-                int s = i % STAGES;
-                if (i >= STAGES) ok = mbar_wait(empty_bar(s), ((i / STAGES) - 1) & 1);
-                if (!ok) break;
-                int p0 = pb + i * 4, np = min(4, pe - p0);
-                mbar_expect_tx(full_bar(s), (uint32_t)np * 2 * Cfg::kPageBytes);
-                uint32_t kdst = tiles + s * Cfg::kStageBytes, vdst = kdst + 4 * Cfg::kPageBytes;
-                for (int j = 0; j < np; j++) {
-                    int page = p.page_table[(size_t)seq * p.pt_stride + p0 + j];
-                    if (page < 0 || page >= p.num_pages) {
-                        report(p.status, kStatusBadPage, page);
-                        page = 0;
-                    }
-                    int row = (int)(((long long)page * p.n_kv + g) * 16);
-                    for (int h = 0; h < HALVES; h++) {
-                        tma_load_2d(kdst + (j * HALVES + h) * 2048, &tmKV, full_bar(s), h * 64, (int)(p.k_row0 + row));
-                        tma_load_2d(vdst + (j * HALVES + h) * 2048, &tmKV, full_bar(s), h * 64, (int)(p.v_row0 + row));
+            int it = 0;
+            for (int u = u0; u < u1 && ok;) {
+                int ui = cum[item + 1] - cum[item], base = cum[item] * p.n_kv;
+                int g = (u - base) / ui, t0 = (u - base) % ui;
+                int pair_end = base + (g + 1) * ui, t1 = t0 + min(u1, pair_end) - u;
+                int seq = p.rm.seq(item), total_pages = (nk_s[item] + 15) >> 4;
+                for (int t = t0; t < t1 && ok; t++, it++) {
+                    int s = it % STAGES;
+                    if (it >= STAGES) ok = mbar_wait(empty_bar(s), ((it / STAGES) - 1) & 1);
+                    if (!ok) break;
+                    int p0 = t * 4, np = min(4, total_pages - p0);
+                    mbar_expect_tx(full_bar(s), (uint32_t)np * 2 * Cfg::kPageBytes);
+                    uint32_t kdst = tiles + s * Cfg::kStageBytes, vdst = kdst + 4 * Cfg::kPageBytes;
+                    for (int j = 0; j < np; j++) {
+                        int page = p.page_table[(size_t)seq * p.pt_stride + p0 + j];
+                        if (page < 0 || page >= p.num_pages) {
+                            report(p.status, kStatusBadPage, page);
+                            page = 0;
+                        }
+                        int row = (int)(((long long)page * p.n_kv + g) * 16);
+                        for (int h = 0; h < HALVES; h++) {
+                            tma_load_2d(kdst + (j * HALVES + h) * 2048, &tmKV, full_bar(s), h * 64, (int)(p.k_row0 + row));
+                            tma_load_2d(vdst + (j * HALVES + h) * 2048, &tmKV, full_bar(s), h * 64, (int)(p.v_row0 + row));
+                        }
                     }
                 }
+                u += t1 - t0;
+                if (u == pair_end && g == p.n_kv - 1) item++;
             }
             if (!ok) report(p.status, kStatusWaitExpired, 300);
         }
         return;
     }
 
-    // ---- consumers.  Query tile as mma A fragments (bf16), pre-scaled by log2(e)/sqrt(d_h).
-    uint32_t qa[KS][4];
-    {
-        float scale = kLog2e / sqrtf((float)DH);
-        int r0 = lane >> 2, r1 = r0 + 8, c = (lane & 3) * 2;
-        auto qrow = [&](int q) -> const float * {
-            if (q >= nq_act) return nullptr;
-            int row = q < p.G ? item : Bc + item;
-            int h = g * p.G + (q < p.G ? q : q - p.G);
-            return p.Q + (size_t)row * q_dim + (size_t)h * DH;
-        };
-        const float *q0 = qrow(r0), *q1 = qrow(r1);
-#pragma unroll
-        for (int ks = 0; ks < KS; ks++) {
-            int k = ks * 16 + c;
-            qa[ks][0] = q0 ? pack_bf16(__ldcg(q0 + k) * scale, __ldcg(q0 + k + 1) * scale) : 0u;
-            qa[ks][1] = q1 ? pack_bf16(__ldcg(q1 + k) * scale, __ldcg(q1 + k + 1) * scale) : 0u;
-            qa[ks][2] = q0 ? pack_bf16(__ldcg(q0 + k + 8) * scale, __ldcg(q0 + k + 9) * scale) : 0u;
-            qa[ks][3] = q1 ? pack_bf16(__ldcg(q1 + k + 8) * scale, __ldcg(q1 + k + 9) * scale) : 0u;
-        }
-    }
-    float o[NB][4];
-#pragma unroll
-    for (int nb = 0; nb < NB; nb++) o[nb][0] = o[nb][1] = o[nb][2] = o[nb][3] = 0.f;
-    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
-
+    // ---- consumers
     bool ok = true;
-    for (int i = 0; i < ntiles; i++) {
-        int s = i % STAGES;
-        ok = mbar_wait(full_bar(s), (i / STAGES) & 1);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-        int tile_j0 = jbeg + i * kAttTile;
-        int valid = min(16, jend - (tile_j0 + warp * 16));  // valid tokens in this warp's page
-        if (valid > 0) {
-            uint32_t kpage = tiles + s * Cfg::kStageBytes + warp * HALVES * 2048;
-            uint32_t vpage = kpage + 4 * Cfg::kPageBytes;
-            if (valid < 16) {
-                // stale slots past the end of the sequence: their scores are masked below, and
-                // their V rows are zeroed here so that 0 * garbage cannot produce a NaN
-                for (int idx = lane; idx < (16 - valid) * HALVES * 8; idx += 32) {
-                    int r = valid + idx / (HALVES * 8), rest = idx % (HALVES * 8);
-                    uint32_t a = vpage + (rest / 8) * 2048 + r * 128 + (rest % 8) * 16;
-                    asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(a), "r"(0u) : "memory");
-                }
-                __syncwarp();
-            }
-            // S = Q K^T for this warp's 16 tokens: two 8-token column blocks
-            float sacc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-            {
-                int r = (lane & 7) + ((lane >> 4) << 3);  // token row this lane addresses
-                int cb = (lane >> 3) & 1;                 // which 8-dim chunk of the k-step
-#pragma unroll
-                for (int ks = 0; ks < KS; ks++) {
-                    int chunk = ks * 2 + cb;  // 16-byte chunk index within the row
-                    uint32_t a = kpage + (chunk >> 3) * 2048 + r * 128 + (((chunk & 7) ^ (r & 7)) << 4);
-                    uint32_t kb[4];
-                    ldsm_x4(a, kb);
-                    mma_bf16(sacc[0], qa[ks], kb[0], kb[1]);
-                    mma_bf16(sacc[1], qa[ks], kb[2], kb[3]);
-                }
-            }
-            // mask, online softmax (base 2), pack P as the A operand of P V
-            int col = (lane & 3) * 2;
-            float rmax[2] = {-INFINITY, -INFINITY};
-#pragma unroll
-            for (int nb = 0; nb < 2; nb++)
-#pragma unroll
-                for (int e = 0; e < 4; e++) {
-                    int t = nb * 8 + col + (e & 1);
-                    if (t >= valid) sacc[nb][e] = -INFINITY;
-                    rmax[e >> 1] = fmaxf(rmax[e >> 1], sacc[nb][e]);
-                }
-            float corr[2], msub[2];
-#pragma unroll
-            for (int h = 0; h < 2; h++) {
-                rmax[h] = fmaxf(rmax[h], __shfl_xor_sync(0xffffffffu, rmax[h], 1));
-                rmax[h] = fmaxf(rmax[h], __shfl_xor_sync(0xffffffffu, rmax[h], 2));
-                float mnew = fmaxf(m_run[h], rmax[h]);
-                msub[h] = mnew == -INFINITY ? 0.f : mnew;
-                corr[h] = m_run[h] == -INFINITY ? 0.f : exp2f(m_run[h] - msub[h]);
-                m_run[h] = mnew;
-            }
-            float rsum[2] = {0.f, 0.f};
-            uint32_t pa[4];
-#pragma unroll
-            for (int nb = 0; nb < 2; nb++) {
-                float p0 = exp2f(sacc[nb][0] - msub[0]), p1 = exp2f(sacc[nb][1] - msub[0]);
-                float p2 = exp2f(sacc[nb][2] - msub[1]), p3 = exp2f(sacc[nb][3] - msub[1]);
-                rsum[0] += p0 + p1;
-                rsum[1] += p2 + p3;
-                pa[nb * 2 + 0] = pack_bf16(p0, p1);
-                pa[nb * 2 + 1] = pack_bf16(p2, p3);
-            }
-#pragma unroll
-            for (int h = 0; h < 2; h++) {
-                rsum[h] += __shfl_xor_sync(0xffffffffu, rsum[h], 1);
-                rsum[h] += __shfl_xor_sync(0xffffffffu, rsum[h], 2);
-                l_run[h] = l_run[h] * corr[h] + rsum[h];
-            }
-#pragma unroll
-            for (int nb = 0; nb < NB; nb++) {
-                o[nb][0] *= corr[0];
-                o[nb][1] *= corr[0];
-                o[nb][2] *= corr[1];
-                o[nb][3] *= corr[1];
-            }
-            // O += P V: V read transposed, two 8-dim column blocks per ldmatrix
-            {
-                int r = (lane & 7) + (((lane >> 3) & 1) << 3);  // token row
-                int cb = lane >> 4;                              // which of the two dim blocks
-#pragma unroll
-                for (int np = 0; np < NB / 2; np++) {
-                    int chunk = np * 2 + cb;
-                    uint32_t a = vpage + (chunk >> 3) * 2048 + r * 128 + (((chunk & 7) ^ (r & 7)) << 4);
-                    uint32_t vb[4];
-                    ldsm_x4_trans(a, vb);
-                    mma_bf16(o[np * 2], pa, vb[0], vb[1]);
-                    mma_bf16(o[np * 2 + 1], pa, vb[2], vb[3]);
-                }
-            }
-        }
-        __syncwarp();
-        if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(empty_bar(s)) : "memory");
-    }
-    if (!ok && lane == 0) report(p.status, kStatusWaitExpired, 310 + warp);
+    int it = 0;
+    const float qscale = kLog2e / sqrtf((float)DH);
+    for (int u = u0; u < u1;) {
+        int ui = cum[item + 1] - cum[item], base = cum[item] * p.n_kv;
+        int g = (u - base) / ui, t0 = (u - base) % ui;
+        int pair_start = base + g * ui, pair_end = pair_start + ui, t1 = t0 + min(u1, pair_end) - u;
+        int nkeys = nk_s[item];
 
-    // ---- fold the four warps' states in warp order and write this split's partial
-    asm volatile("bar.sync 1, 128;" ::: "memory");  // every consumer is done with the ring
-    float *sc_o = reinterpret_cast<float *>(gen);            // [4][16][DH]
-    float *sc_m = sc_o + kAttWarps * 16 * DH;                // [4][16]
-    float *sc_l = sc_m + kAttWarps * 16;                     // [4][16]
-    {
-        int r0 = lane >> 2, c = (lane & 3) * 2;
+        // Query tile (16 rows x DH, fp32) into shared memory, then mma A fragments (bf16),
+        // pre-scaled by log2(e)/sqrt(d_h).  Rows: G primary heads, then G coupled branch heads.
+        consumer_sync();  // the previous segment is done with the scratch
+        for (int idx = tid; idx < 16 * DH / 4; idx += 128) {
+            int q = idx / (DH / 4), c4 = idx % (DH / 4);
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (q < nq_act) {
+                int row = q < p.G ? item : Bc + item;
+                int h = g * p.G + (q < p.G ? q : q - p.G);
+                v = __ldcg(reinterpret_cast<const float4 *>(p.Q + (size_t)row * q_dim + (size_t)h * DH) + c4);
+            }
+            reinterpret_cast<float4 *>(sc_o)[idx] = v;
+        }
+        consumer_sync();
+        uint32_t qa[KS][4];
+        {
+            int r0 = lane >> 2, c = (lane & 3) * 2;
+            const float *q0 = sc_o + r0 * DH, *q1 = sc_o + (r0 + 8) * DH;
 #pragma unroll
-        for (int nb = 0; nb < NB; nb++) {
-            *reinterpret_cast<float2 *>(sc_o + ((size_t)warp * 16 + r0) * DH + nb * 8 + c) = make_float2(o[nb][0], o[nb][1]);
-            *reinterpret_cast<float2 *>(sc_o + ((size_t)warp * 16 + r0 + 8) * DH + nb * 8 + c) = make_float2(o[nb][2], o[nb][3]);
+            for (int ks = 0; ks < KS; ks++) {
+                int k = ks * 16 + c;
+                qa[ks][0] = pack_bf16(q0[k] * qscale, q0[k + 1] * qscale);
+                qa[ks][1] = pack_bf16(q1[k] * qscale, q1[k + 1] * qscale);
+                qa[ks][2] = pack_bf16(q0[k + 8] * qscale, q0[k + 9] * qscale);
+                qa[ks][3] = pack_bf16(q1[k + 8] * qscale, q1[k + 9] * qscale);
+            }
         }
-        if ((lane & 3) == 0) {
-            sc_m[warp * 16 + r0] = m_run[0];
-            sc_m[warp * 16 + r0 + 8] = m_run[1];
-            sc_l[warp * 16 + r0] = l_run[0];
-            sc_l[warp * 16 + r0 + 8] = l_run[1];
-        }
-    }
-    asm volatile("bar.sync 1, 128;" ::: "memory");
-    for (int idx = tid; idx < nq_act * DH; idx += 128) {
-        int q = idx / DH, e = idx % DH;
-        float M = -INFINITY;
+        consumer_sync();  // everyone has its fragments: the scratch is free again
+        float o[NB][4];
 #pragma unroll
-        for (int w = 0; w < kAttWarps; w++) M = fmaxf(M, sc_m[w * 16 + q]);
-        float L = 0.f, acc = 0.f;
+        for (int nb = 0; nb < NB; nb++) o[nb][0] = o[nb][1] = o[nb][2] = o[nb][3] = 0.f;
+        float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+
+        for (int t = t0; t < t1 && ok; t++, it++) {
+            int s = it % STAGES;
+            ok = mbar_wait(full_bar(s), (it / STAGES) & 1);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            int valid = min(16, nkeys - (t * kAttTile + warp * 16));  // valid tokens in this warp's page
+            if (valid > 0) {
+                uint32_t kpage = tiles + s * Cfg::kStageBytes + warp * HALVES * 2048;
+                uint32_t vpage = kpage + 4 * Cfg::kPageBytes;
+                if (valid < 16) {
+                    // stale slots past the end of the sequence: their scores are masked below, and
+                    // their V rows are zeroed here so that 0 * garbage cannot produce a NaN
+                    for (int idx = lane; idx < (16 - valid) * HALVES * 8; idx += 32) {
+                        int r = valid + idx / (HALVES * 8), rest = idx % (HALVES * 8);
+                        uint32_t a = vpage + (rest / 8) * 2048 + r * 128 + (rest % 8) * 16;
+                        asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(a), "r"(0u) : "memory");
+                    }
+                    __syncwarp();
+                }
+                // S = Q K^T for this warp's 16 tokens: two 8-token column blocks
+                float sacc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+                {
+                    int r = (lane & 7) + ((lane >> 4) << 3);  // token row this lane addresses
+                    int cb = (lane >> 3) & 1;                 // which 8-dim chunk of the k-step
 #pragma unroll
-        for (int w = 0; w < kAttWarps; w++) {
-            float mw = sc_m[w * 16 + q];
-            float f = mw == -INFINITY ? 0.f : exp2f(mw - M);
-            L += sc_l[w * 16 + q] * f;
-            acc += sc_o[((size_t)w * 16 + q) * DH + e] * f;
+                    for (int ks = 0; ks < KS; ks++) {
+                        int chunk = ks * 2 + cb;  // 16-byte chunk index within the row
+                        uint32_t a = kpage + (chunk >> 3) * 2048 + r * 128 + (((chunk & 7) ^ (r & 7)) << 4);
+                        uint32_t kb[4];
+                        ldsm_x4(a, kb);
+                        mma_bf16(sacc[0], qa[ks], kb[0], kb[1]);
+                        mma_bf16(sacc[1], qa[ks], kb[2], kb[3]);
+                    }
+                }
+                // mask, online softmax (base 2), pack P as the A operand of P V
+                int col = (lane & 3) * 2;
+                float rmax[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+                for (int nb = 0; nb < 2; nb++)
+#pragma unroll
+                    for (int e = 0; e < 4; e++) {
+                        int tk = nb * 8 + col + (e & 1);
+                        if (tk >= valid) sacc[nb][e] = -INFINITY;
+                        rmax[e >> 1] = fmaxf(rmax[e >> 1], sacc[nb][e]);
+                    }
+                float corr[2], msub[2];
+#pragma unroll
+                for (int h = 0; h < 2; h++) {
+                    rmax[h] = fmaxf(rmax[h], __shfl_xor_sync(0xffffffffu, rmax[h], 1));
+                    rmax[h] = fmaxf(rmax[h], __shfl_xor_sync(0xffffffffu, rmax[h], 2));
+                    float mnew = fmaxf(m_run[h], rmax[h]);
+                    msub[h] = mnew == -INFINITY ? 0.f : mnew;
+                    corr[h] = m_run[h] == -INFINITY ? 0.f : exp2f(m_run[h] - msub[h]);
+                    m_run[h] = mnew;
+                }
+                float rsum[2] = {0.f, 0.f};
+                uint32_t pa[4];
+#pragma unroll
+                for (int nb = 0; nb < 2; nb++) {
+                    float p0 = exp2f(sacc[nb][0] - msub[0]), p1 = exp2f(sacc[nb][1] - msub[0]);
+                    float p2 = exp2f(sacc[nb][2] - msub[1]), p3 = exp2f(sacc[nb][3] - msub[1]);
+                    rsum[0] += p0 + p1;
+                    rsum[1] += p2 + p3;
+                    pa[nb * 2 + 0] = pack_bf16(p0, p1);
+                    pa[nb * 2 + 1] = pack_bf16(p2, p3);
+                }
+#pragma unroll
+                for (int h = 0; h < 2; h++) {
+                    rsum[h] += __shfl_xor_sync(0xffffffffu, rsum[h], 1);
+                    rsum[h] += __shfl_xor_sync(0xffffffffu, rsum[h], 2);
+                    l_run[h] = l_run[h] * corr[h] + rsum[h];
+                }
+#pragma unroll
+                for (int nb = 0; nb < NB; nb++) {
+                    o[nb][0] *= corr[0];
+                    o[nb][1] *= corr[0];
+                    o[nb][2] *= corr[1];
+                    o[nb][3] *= corr[1];
+                }
+                // O += P V: V read transposed, two 8-dim column blocks per ldmatrix
+                {
+                    int r = (lane & 7) + (((lane >> 3) & 1) << 3);  // token row
+                    int cb = lane >> 4;                              // which of the two dim blocks
+#pragma unroll
+                    for (int np = 0; np < NB / 2; np++) {
+                        int chunk = np * 2 + cb;
+                        uint32_t a = vpage + (chunk >> 3) * 2048 + r * 128 + (((chunk & 7) ^ (r & 7)) << 4);
+                        uint32_t vb[4];
+                        ldsm_x4_trans(a, vb);
+                        mma_bf16(o[np * 2], pa, vb[0], vb[1]);
+                        mma_bf16(o[np * 2 + 1], pa, vb[2], vb[3]);
+                    }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(empty_bar(s)) : "memory");
         }
-        out[(size_t)q * (DH + 2) + e] = ok ? acc : 0.f;
-        if (e == 0) {
-            out[(size_t)q * (DH + 2) + DH] = ok ? M * kLn2 : -INFINITY;  // natural-log units
-            out[(size_t)q * (DH + 2) + DH + 1] = ok ? L : 0.f;
+        if (!ok) {
+            // a ring that stopped filling stops for all four warps: every consumer leaves here
+            if (lane == 0) report(p.status, kStatusWaitExpired, 310 + warp);
+            return;
         }
-    }
-    // ---- the last split to arrive for this (row, KV head) folds all splits in split order
-    __threadfence();
-    asm volatile("bar.sync 1, 128;" ::: "memory");
-    int *flag = reinterpret_cast<int *>(sc_l + kAttWarps * 16);
-    if (tid == 0) {
-        int *tk = p.tickets + (size_t)item * p.n_kv + g;
-        int t = atomicAdd(tk, 1);
-        int last = t == p.nsplit - 1;
-        if (last) atomicExch(tk, 0);
-        *flag = last;
-    }
-    asm volatile("bar.sync 1, 128;" ::: "memory");
-    if (!*flag) return;
-    __threadfence();
-    const float *base = p.part + ((size_t)item * p.n_kv + g) * p.nsplit * 16 * (DH + 2);
-    for (int idx = tid; idx < nq_act * DH; idx += 128) {
-        int q = idx / DH, e = idx % DH;
-        float M = -INFINITY;
-        for (int s2 = 0; s2 < p.nsplit; s2++) M = fmaxf(M, __ldcg(base + ((size_t)s2 * 16 + q) * (DH + 2) + DH));
-        float L = 0.f, acc = 0.f;
-        for (int s2 = 0; s2 < p.nsplit; s2++) {
-            const float *pp = base + ((size_t)s2 * 16 + q) * (DH + 2);
-            float ms = __ldcg(pp + DH);
-            float f = ms == -INFINITY ? 0.f : expf(ms - M);
-            L += __ldcg(pp + DH + 1) * f;
-            acc += __ldcg(pp + e) * f;
+
+        // ---- fold the four warps' states, (0+2) + (1+3), in registers through the one-slot
+        // scratch; warp 0 then writes this segment's partial
+        int pair = item * p.n_kv + g;
+        int first_cta = pair_start / quota, nseg = (pair_end - 1) / quota - first_cta + 1;
+        float *out = p.part + (size_t)(blockIdx.x + pair) * 16 * (DH + 2);
+        {
+            int r0 = lane >> 2, c = (lane & 3) * 2;
+            auto put = [&]() {
+#pragma unroll
+                for (int nb = 0; nb < NB; nb++) {
+                    *reinterpret_cast<float2 *>(sc_o + (size_t)r0 * DH + nb * 8 + c) = make_float2(o[nb][0], o[nb][1]);
+                    *reinterpret_cast<float2 *>(sc_o + (size_t)(r0 + 8) * DH + nb * 8 + c) = make_float2(o[nb][2], o[nb][3]);
+                }
+                if ((lane & 3) == 0) {
+                    sc_m[r0] = m_run[0];
+                    sc_m[r0 + 8] = m_run[1];
+                    sc_l[r0] = l_run[0];
+                    sc_l[r0 + 8] = l_run[1];
+                }
+            };
+            auto take = [&]() {  // this warp's state := this warp's state (+) the slot's state
+#pragma unroll
+                for (int h = 0; h < 2; h++) {
+                    int r = r0 + 8 * h;
+                    float mb = sc_m[r], lb = sc_l[r];
+                    float M = fmaxf(m_run[h], mb);
+                    float fa = m_run[h] == -INFINITY ? 0.f : exp2f(m_run[h] - M);
+                    float fb = mb == -INFINITY ? 0.f : exp2f(mb - M);
+                    l_run[h] = l_run[h] * fa + lb * fb;
+                    m_run[h] = M;
+#pragma unroll
+                    for (int nb = 0; nb < NB; nb++) {
+                        float2 ob = *reinterpret_cast<const float2 *>(sc_o + (size_t)r * DH + nb * 8 + c);
+                        o[nb][2 * h] = o[nb][2 * h] * fa + ob.x * fb;
+                        o[nb][2 * h + 1] = o[nb][2 * h + 1] * fa + ob.y * fb;
+                    }
+                }
+            };
+            for (int step = 0; step < 3; step++) {  // 2 -> 0, 3 -> 1, 1 -> 0
+                int src = step == 0 ? 2 : step == 1 ? 3 : 1, dst = step == 1 ? 1 : 0;
+                if (warp == src) put();
+                consumer_sync();
+                if (warp == dst) take();
+                consumer_sync();
+            }
+            if (warp == 0) {
+#pragma unroll
+                for (int h = 0; h < 2; h++) {
+                    int q = r0 + 8 * h;
+                    if (q < nq_act) {
+#pragma unroll
+                        for (int nb = 0; nb < NB; nb++)
+                            *reinterpret_cast<float2 *>(out + (size_t)q * (DH + 2) + nb * 8 + c) =
+                                make_float2(o[nb][2 * h], o[nb][2 * h + 1]);
+                        if ((lane & 3) == 0) {
+                            out[(size_t)q * (DH + 2) + DH] = m_run[h];  // base-2 units
+                            out[(size_t)q * (DH + 2) + DH + 1] = l_run[h];
+                        }
+                    }
+                }
+            }
         }
-        float x = acc / L;
-        int row = q < p.G ? item : Bc + item;
-        int h = g * p.G + (q < p.G ? q : q - p.G);
-        size_t o_idx = (size_t)row * q_dim + (size_t)h * DH + e;
-        __nv_bfloat16 hi = __float2bfloat16_rn(x);
-        p.Ob[o_idx] = hi;
-        if (p.lo_off) p.Ob[o_idx + p.lo_off] = __float2bfloat16_rn(x - __bfloat162float(hi));
+        // ---- the last segment of this pair to arrive folds all of them in segment order
+        __threadfence();
+        consumer_sync();
+        if (tid == 0) {
+            int last = 1;
+            if (nseg > 1) {
+                int *tk = p.tickets + pair;
+                int tkt = atomicAdd(tk, 1);
+                last = tkt == nseg - 1;
+                if (last) atomicExch(tk, 0);
+            }
+            flag[0] = last;
+        }
+        consumer_sync();
+        if (flag[0]) {
+            __threadfence();
+            const float *pbase = p.part + (size_t)(first_cta + pair) * 16 * (DH + 2);
+            float *wt = sc_o, *ml = sc_o + 16 * kAttMaxSeg;  // fold weights [16][32], (m, l) staging
+            for (int t = tid; t < nq_act * nseg; t += 128) {  // all (m, l) pairs in one round of loads
+                int q = t / nseg, s2 = t % nseg;
+                const float *pp = pbase + ((size_t)s2 * 16 + q) * (DH + 2) + DH;
+                wt[q * kAttMaxSeg + s2] = __ldcg(pp);
+                ml[q * kAttMaxSeg + s2] = __ldcg(pp + 1);
+            }
+            consumer_sync();
+            if (tid < nq_act) {
+                float M = -INFINITY, L = 0.f;
+                for (int s2 = 0; s2 < nseg; s2++) M = fmaxf(M, wt[tid * kAttMaxSeg + s2]);
+                for (int s2 = 0; s2 < nseg; s2++) {
+                    float ms = wt[tid * kAttMaxSeg + s2];
+                    float f = ms == -INFINITY ? 0.f : exp2f(ms - M);
+                    L += ml[tid * kAttMaxSeg + s2] * f;
+                    wt[tid * kAttMaxSeg + s2] = f;
+                }
+                float inv = 1.f / L;
+                for (int s2 = 0; s2 < nseg; s2++) wt[tid * kAttMaxSeg + s2] *= inv;
+            }
+            consumer_sync();
+            for (int idx = tid; idx < nq_act * DH; idx += 128) {
+                int q = idx / DH, e = idx % DH;
+                float x = 0.f;
+                for (int s2 = 0; s2 < nseg; s2++)
+                    x = fmaf(__ldcg(pbase + ((size_t)s2 * 16 + q) * (DH + 2) + e), wt[q * kAttMaxSeg + s2], x);
+                int row = q < p.G ? item : Bc + item;
+                int h = g * p.G + (q < p.G ? q : q - p.G);
+                size_t o_idx = (size_t)row * q_dim + (size_t)h * DH + e;
+                __nv_bfloat16 hi = __float2bfloat16_rn(x);
+                p.Ob[o_idx] = hi;
+                if (p.lo_off) p.Ob[o_idx + p.lo_off] = __float2bfloat16_rn(x - __bfloat162float(hi));
+            }
+        }
+        u += t1 - t0;
+        if (u == pair_end && g == p.n_kv - 1) item++;
     }
 }
 
