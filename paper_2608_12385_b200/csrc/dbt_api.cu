@@ -34,7 +34,7 @@ struct Workspace {
     int32_t *ridx, *ecnt, *elist, *last_experts, *union_cnt;
     // bf16 tensor-core path: bf16 GEMM inputs and the fp32 split-K partial buffer
     __nv_bfloat16 *Xb, *Ob, *Hb;
-    float *P;
+    float *P, *ss;
     size_t P_floats;
 };
 
@@ -68,6 +68,7 @@ struct dbt_model {
     std::vector<LayerMaps> maps;
     CUtensorMap map_lm, map_Xb, map_Ob, map_Hb, map_kv;
     bool att_fast;  // TMA + mma.sync attention over the bf16 pool
+    bool fused;     // dense bf16: elementwise work fused into the GEMM epilogues
     int num_sms;
     int act_parts;  // 2: GEMM inputs carried as hi + lo bf16 terms; 1: plain bf16
     // a decode step is captured once per (batch, mode, buffer set) and replayed as a CUDA graph
@@ -189,6 +190,7 @@ size_t carve(const dbt_config &c, char *base, Workspace *ws, int *Rmax_out, int 
         w.P_floats = want < cap ? want : cap;
         if (w.P_floats < (size_t)Rmax * widest) w.P_floats = (size_t)Rmax * widest;
         w.P = k.take<float>(w.P_floats);
+        w.ss = k.take<float>((size_t)((d + 127) / 128) * Rmax);
     }
     if (ws) *ws = w;
     if (Rmax_out) *Rmax_out = Rmax;
@@ -486,15 +488,15 @@ int choose_split(int tiles, int total_kt) {
 }
 
 template <int N_TILE>
-dbt_status launch_gemm_tc(dbt_model *m, const TcCall &c, const TcParams &p, dim3 grid, double bytes) {
+dbt_status launch_gemm_tc(dbt_model *m, const TcCall &c, const TcParams &p, const FusedEpi &e, dim3 grid, double bytes) {
     const CUtensorMap *w1 = c.nseg > 1 ? c.W[1] : c.W[0], *w2 = c.nseg > 2 ? c.W[2] : c.W[0];
-    LAUNCH(m, c.tag, bytes, gemm_tc_kernel<N_TILE>, grid, 128, TcCfg<N_TILE>::kSmemBytes, *c.W[0], *w1, *w2, *c.X, p);
+    LAUNCH(m, c.tag, bytes, gemm_tc_kernel<N_TILE>, grid, 128, TcCfg<N_TILE>::kSmemBytes, *c.W[0], *w1, *w2, *c.X, p, e);
     return DBT_OK;
 }
 
 // Y partials P[split][R][ldp]; returns the split count and stride the consumer must use.
 dbt_status run_gemm_tc(dbt_model *m, const TcCall &c, int n_tile, int *nsplit_out, size_t *split_stride_out,
-                       int force_split = 0) {
+                       int force_split = 0, FusedEpi e = FusedEpi{}) {
     TcParams p{};
     int tiles = 0, col = 0;
     double bytes = 0;
@@ -518,15 +520,21 @@ dbt_status run_gemm_tc(dbt_model *m, const TcCall &c, int n_tile, int *nsplit_ou
     if ((size_t)c.R * col > c.P_floats) return fail(m, DBT_ERR_CAPACITY, "partial buffer too small for %s", c.tag);
     p.kt_per_split = (total_kt + split - 1) / split;
     split = (total_kt + p.kt_per_split - 1) / p.kt_per_split;
+    if (e.mode == FE_LMHEAD) {
+        split = 1;
+        p.kt_per_split = total_kt;
+    }
+    e.arrivals = (e.mode == FE_GATEUP ? 2 : 1) * split;
+    if (e.mode != FE_NONE && tiles > 4096) return fail(m, DBT_ERR_UNSUPPORTED, "too many output tiles for %s", c.tag);
     dim3 grid(tiles, split);
     if (nsplit_out) *nsplit_out = split;
     if (split_stride_out) *split_stride_out = (size_t)c.R * col;
     switch (n_tile) {
-        case 16: return launch_gemm_tc<16>(m, c, p, grid, bytes);
-        case 32: return launch_gemm_tc<32>(m, c, p, grid, bytes);
-        case 64: return launch_gemm_tc<64>(m, c, p, grid, bytes);
-        case 128: return launch_gemm_tc<128>(m, c, p, grid, bytes);
-        case 256: return launch_gemm_tc<256>(m, c, p, grid, bytes);
+        case 16: return launch_gemm_tc<16>(m, c, p, e, grid, bytes);
+        case 32: return launch_gemm_tc<32>(m, c, p, e, grid, bytes);
+        case 64: return launch_gemm_tc<64>(m, c, p, e, grid, bytes);
+        case 128: return launch_gemm_tc<128>(m, c, p, e, grid, bytes);
+        case 256: return launch_gemm_tc<256>(m, c, p, e, grid, bytes);
     }
     return fail(m, DBT_ERR_UNSUPPORTED, "row tile %d", n_tile);
 }
@@ -712,6 +720,160 @@ dbt_status prefill_tc(dbt_model *m, const int32_t *tokens_dev, int B, int n, flo
     return DBT_OK;
 }
 
+// ---- fused dense path: 4 GEMMs + attention per layer, no kernel between them ----------------
+
+FusedEpi epi_base(dbt_model *m, const RowMap &rm, int grouped, int mode) {
+    const dbt_config &c = m->cfg;
+    FusedEpi e{};
+    e.mode = mode;
+    e.Bc = rm.B * rm.cn;
+    e.grouped = grouped;
+    e.rm = rm;
+    e.tickets = m->ws.gemm_tickets;
+    e.ss_in = m->ws.ss;
+    e.ss_tiles = (c.d_model + 127) / 128;
+    e.ss_ld = m->Rmax;
+    e.d_norm = c.d_model;
+    e.eps = c.rms_eps;
+    e.use_scale = 1;
+    return e;
+}
+
+dbt_status run_layers_fused(dbt_model *m, const RowMap &rm, int grouped, int n_tile) {
+    typedef __nv_bfloat16 WT;
+    const dbt_config &c = m->cfg;
+    const Workspace &w = m->ws;
+    int Bc = rm.B * rm.cn, R = grouped ? 2 * Bc : Bc;
+    int d = c.d_model, qd = c.n_q_heads * c.head_dim, kvd = c.n_kv_heads * c.head_dim, F = c.d_ff;
+    size_t pool_layer_elems = (size_t)2 * c.num_pages * c.n_kv_heads * c.page_size * c.head_dim;
+    size_t lo_x = m->act_parts == 2 ? (size_t)m->Rmax * d : 0, lo_h = m->act_parts == 2 ? (size_t)m->Rmax * F : 0;
+    double kv_bytes = 0;
+    for (int b = 0; b < rm.B; b++)
+        for (int j = 0; j < rm.cn; j++) kv_bytes += (double)(m->len_host[b] + j + 1) * 2 * kvd * sizeof(WT);
+    dbt_status st;
+    auto call = [&](const char *tag, const CUtensorMap *X, int K) {
+        TcCall t{};
+        t.X = X; t.K = K; t.R = R; t.P = w.P; t.P_floats = w.P_floats; t.tag = tag;
+        t.parts = m->act_parts; t.lo_row0 = m->Rmax;
+        return t;
+    };
+    for (int l = 0; l < c.n_layers; l++) {
+        const dbt_layer_weights &lw = m->layers[l];
+        const LayerMaps &mp = m->maps[l];
+        WT *kpool = reinterpret_cast<WT *>(m->kv_pool) + (size_t)l * pool_layer_elems;
+        // Q|K|V with 1/rms, RoPE, the a coupling and the cache append in the epilogue
+        TcCall qkv = call("gemm_qkv", &m->map_Xb, d);
+        qkv.W[0] = &mp.wq; qkv.n_out[0] = qd; qkv.rows[0] = R;
+        qkv.W[1] = &mp.wk; qkv.n_out[1] = kvd; qkv.rows[1] = Bc;
+        qkv.W[2] = &mp.wv; qkv.n_out[2] = kvd; qkv.rows[2] = Bc;
+        qkv.nseg = 3;
+        FusedEpi eq = epi_base(m, rm, grouped, FE_QKV);
+        eq.coup = lw.coup_a; eq.Q = w.Q; eq.rope = w.rope; eq.seq_len = w.seq_len; eq.page_table = w.page_table;
+        eq.pt_stride = m->pages_per_seq_max; eq.num_pages = c.num_pages; eq.n_q = c.n_q_heads; eq.n_kv = c.n_kv_heads;
+        eq.dh = c.head_dim; eq.kpool = kpool; eq.vpool = kpool + pool_layer_elems / 2;
+        if ((st = run_gemm_tc(m, qkv, n_tile, nullptr, nullptr, 0, eq)) != DBT_OK) return st;
+        st = c.head_dim == 128 ? run_attention_mma<128>(m, rm, grouped, l, kv_bytes)
+                               : run_attention_mma<64>(m, rm, grouped, l, kv_bytes);
+        if (st != DBT_OK) return st;
+        // S-bar = S + Attn W_O; next input g_mlp * S-bar
+        TcCall op = call("gemm_o", &m->map_Ob, qd);
+        op.W[0] = &mp.wo; op.n_out[0] = d; op.rows[0] = R; op.nseg = 1;
+        FusedEpi eo = epi_base(m, rm, grouped, FE_RESID);
+        eo.use_scale = 0; eo.S = w.S; eo.g_next = lw.mlp_norm_g; eo.Xout = w.Xb; eo.lo_off = lo_x; eo.ld_out = d; eo.ss_out = w.ss;
+        if ((st = run_gemm_tc(m, op, n_tile, nullptr, nullptr, 0, eo)) != DBT_OK) return st;
+        // gate|up with 1/rms, SwiGLU and the b coupling
+        TcCall gu = call("gemm_gateup", &m->map_Xb, d);
+        gu.W[0] = &mp.wg; gu.n_out[0] = F; gu.rows[0] = R;
+        gu.W[1] = &mp.wu; gu.n_out[1] = F; gu.rows[1] = R;
+        gu.nseg = 2;
+        FusedEpi eg = epi_base(m, rm, grouped, FE_GATEUP);
+        eg.coup = lw.coup_b; eg.Xout = w.Hb; eg.lo_off = lo_h; eg.ld_out = F;
+        if ((st = run_gemm_tc(m, gu, n_tile, nullptr, nullptr, 0, eg)) != DBT_OK) return st;
+        // down with the c coupling and the residual; next input for layer l+1 (or the output matrix)
+        TcCall dn = call("gemm_down", &m->map_Hb, F);
+        dn.W[0] = &mp.wd; dn.n_out[0] = d; dn.rows[0] = R; dn.nseg = 1;
+        FusedEpi ed = epi_base(m, rm, grouped, FE_DOWN);
+        ed.use_scale = 0; ed.coup = lw.coup_c; ed.S = w.S; ed.Xout = w.Xb; ed.lo_off = lo_x; ed.ld_out = d; ed.ss_out = w.ss;
+        ed.g_next = l + 1 < c.n_layers ? m->layers[l + 1].attn_norm_g : (c.final_norm ? m->w.final_norm_g : nullptr);
+        if ((st = run_gemm_tc(m, dn, n_tile, nullptr, nullptr, 0, ed)) != DBT_OK) return st;
+    }
+    return DBT_OK;
+}
+
+dbt_status run_head_fused(dbt_model *m, const RowMap &rm, int grouped, int n_tile) {
+    const dbt_config &c = m->cfg;
+    const Workspace &w = m->ws;
+    int R = (grouped ? 2 : 1) * rm.B * rm.cn;
+    TcCall lm{};
+    lm.W[0] = &m->map_lm; lm.n_out[0] = c.vocab; lm.rows[0] = R; lm.nseg = 1; lm.X = &m->map_Xb; lm.K = c.d_model;
+    lm.R = R; lm.P = w.Z; lm.P_floats = (size_t)R * c.vocab; lm.tag = "gemm_lm_head";
+    lm.parts = m->act_parts; lm.lo_row0 = m->Rmax;
+    FusedEpi e = epi_base(m, rm, grouped, FE_LMHEAD);
+    e.use_scale = c.final_norm;
+    e.Z = w.Z;
+    return run_gemm_tc(m, lm, n_tile, nullptr, nullptr, 0, e);
+}
+
+template <typename WT>
+dbt_status run_embed_fused(dbt_model *m, const int32_t *tokens_dev, int n, int p0, const RowMap &rm, int R) {
+    const dbt_config &c = m->cfg;
+    const Workspace &w = m->ws;
+    LAUNCH(m, "embed", 0, embed_fused_kernel<WT>, R, 256, 0, tokens_dev, n, p0, rm, (const WT *)m->w.embed_primary,
+           (const WT *)m->w.embed_branch, m->w.embed_norm_g, c.rms_eps, c.d_model, c.vocab, w.S,
+           m->layers[0].attn_norm_g, w.Xb, m->act_parts == 2 ? (size_t)m->Rmax * c.d_model : (size_t)0, w.ss, m->Rmax,
+           (c.d_model + 127) / 128, w.status);
+    return DBT_OK;
+}
+
+dbt_status step_fused(dbt_model *m, const int32_t *tokens_dev, int B, int grouped, int32_t *next_dev, float *z1_dev,
+                      float *z2_dev, float *alpha_dev) {
+    typedef __nv_bfloat16 WT;
+    const dbt_config &c = m->cfg;
+    const Workspace &w = m->ws;
+    RowMap rm{B, 1};
+    int R = grouped ? 2 * B : B, n_tile = pad_rows(2 * B);
+    dbt_status st;
+    if ((st = run_embed_fused<WT>(m, tokens_dev, 1, 0, rm, R)) != DBT_OK) return st;
+    if ((st = run_layers_fused(m, rm, grouped, n_tile)) != DBT_OK) return st;
+    if ((st = run_head_fused(m, rm, grouped, n_tile)) != DBT_OK) return st;
+    LAUNCH(m, "readout", 0, readout_kernel, B, 1024, 0, w.Z, B, c.vocab, grouped, next_dev, alpha_dev);
+    LAUNCH(m, "advance_len", 0, advance_len_kernel, (B + 127) / 128, 128, 0, w.seq_len, B, 1);
+    size_t zb = sizeof(float) * (size_t)B * c.vocab;
+    if (z1_dev) CUDA_TRY(m, cudaMemcpyAsync(z1_dev, w.Z, zb, cudaMemcpyDeviceToDevice, m->stream));
+    if (z2_dev && grouped)
+        CUDA_TRY(m, cudaMemcpyAsync(z2_dev, w.Z + (size_t)B * c.vocab, zb, cudaMemcpyDeviceToDevice, m->stream));
+    for (int b = 0; b < B; b++) m->len_host[b] += 1;
+    return DBT_OK;
+}
+
+dbt_status prefill_fused(dbt_model *m, const int32_t *tokens_dev, int B, int n, float *last_logits) {
+    typedef __nv_bfloat16 WT;
+    const dbt_config &c = m->cfg;
+    const Workspace &w = m->ws;
+    int cn_max = (m->Rmax < kAttMaxItems ? m->Rmax : kAttMaxItems) / B;
+    if (cn_max < 1) cn_max = 1;
+    // when logits are wanted the last position runs as its own chunk, so that the rows of the
+    // output-matrix GEMM are exactly the B last positions
+    int n_bulk = last_logits ? n - 1 : n;
+    dbt_status st;
+    for (int p0 = 0; p0 < n;) {
+        int cn = p0 < n_bulk ? (n_bulk - p0 < cn_max ? n_bulk - p0 : cn_max) : 1;
+        RowMap rm{B, cn};
+        int R = B * cn, n_tile = pad_rows(R);
+        if ((st = run_embed_fused<WT>(m, tokens_dev, n, p0, rm, R)) != DBT_OK) return st;
+        if ((st = run_layers_fused(m, rm, 0, n_tile)) != DBT_OK) return st;
+        if (last_logits && p0 + cn >= n) {
+            if ((st = run_head_fused(m, rm, 0, n_tile)) != DBT_OK) return st;
+            CUDA_TRY(m, cudaMemcpyAsync(last_logits, w.Z, sizeof(float) * (size_t)B * c.vocab, cudaMemcpyDeviceToDevice,
+                                        m->stream));
+        }
+        LAUNCH(m, "advance_len", 0, advance_len_kernel, (B + 127) / 128, 128, 0, w.seq_len, B, cn);
+        for (int b = 0; b < B; b++) m->len_host[b] += cn;  // the next chunk's byte accounting sees the new lengths
+        p0 += cn;
+    }
+    return DBT_OK;
+}
+
 template <int N_TILE>
 bool allow_smem() {
     return cudaFuncSetAttribute(gemm_tc_kernel<N_TILE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -757,6 +919,12 @@ bool setup_tc(dbt_model *m) {
                                        AttCfg<128>::kSmemBytes) == cudaSuccess &&
                   cudaFuncSetAttribute(attn_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        AttCfg<64>::kSmemBytes) == cudaSuccess;
+    const char *fu = getenv("DBT_FUSED");
+    // Opt-in (DBT_FUSED=1): measured slower than the separate elementwise kernels at batch 16
+    // (1.96 ms vs 1.55 ms per step on the 1B model): the tile's last CTA folds the split-K
+    // partials alone, on 16..44 SMs, while the separate kernels spread that work over the GPU
+    // and overlap with their neighbours through programmatic dependent launch.
+    m->fused = ok && m->att_fast && !moe && (fu && strcmp(fu, "1") == 0);
     const char *split = getenv("DBT_ACT_SPLIT");
     m->act_parts = (split && strcmp(split, "0") == 0) ? 1 : 2;
     return ok;
@@ -1044,6 +1212,8 @@ dbt_status dbt_reset(dbt_model *m) {
     if (!m) return DBT_ERR_INVALID_ARG;
     CUDA_TRY(m, cudaMemsetAsync(m->ws.seq_len, 0, sizeof(int32_t) * m->cfg.max_batch, m->stream));
     CUDA_TRY(m, cudaMemsetAsync(m->ws.status, 0, sizeof(int32_t) * 4, m->stream));
+    CUDA_TRY(m, cudaMemsetAsync(m->ws.att_tickets, 0, sizeof(int32_t) * (size_t)m->Rmax * m->cfg.n_kv_heads, m->stream));
+    CUDA_TRY(m, cudaMemsetAsync(m->ws.gemm_tickets, 0, sizeof(int32_t) * 4096, m->stream));
     std::fill(m->len_host.begin(), m->len_host.end(), 0);
     return DBT_OK;
 }
@@ -1070,6 +1240,7 @@ dbt_status dbt_prefill(dbt_model *m, const int32_t *tokens_dev, int32_t B, int32
     dbt_status st = check_step_args(m, tokens_dev, B, n);
     if (st != DBT_OK) return st;
     if (m->cfg.weight_dtype == DBT_DTYPE_F32) return prefill_impl<float>(m, tokens_dev, B, n, last_primary_logits_dev);
+    if (m->fused) return prefill_fused(m, tokens_dev, B, n, last_primary_logits_dev);
     if (m->tc) return prefill_tc(m, tokens_dev, B, n, last_primary_logits_dev);
     return prefill_impl<__nv_bfloat16>(m, tokens_dev, B, n, last_primary_logits_dev);
 }
@@ -1077,6 +1248,7 @@ dbt_status dbt_prefill(dbt_model *m, const int32_t *tokens_dev, int32_t B, int32
 static dbt_status step_direct(dbt_model *m, const int32_t *tokens_dev, int B, int grouped, int32_t *next_dev,
                               float *z1, float *z2, float *alpha) {
     if (m->cfg.weight_dtype == DBT_DTYPE_F32) return step_impl<float>(m, tokens_dev, B, grouped, next_dev, z1, z2, alpha);
+    if (m->fused) return step_fused(m, tokens_dev, B, grouped, next_dev, z1, z2, alpha);
     if (m->tc) return step_tc(m, tokens_dev, B, grouped, next_dev, z1, z2, alpha);
     return step_impl<__nv_bfloat16>(m, tokens_dev, B, grouped, next_dev, z1, z2, alpha);
 }

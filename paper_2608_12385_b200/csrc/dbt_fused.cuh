@@ -148,6 +148,43 @@ __global__ void __launch_bounds__(256) swiglu_couple_kernel(const float *P, int 
     }
 }
 
+// Eq. embeddings for the fused path: S^0 = RMSNorm(E[x]) and, for the first layer's Q|K|V GEMM,
+// the input g_next * S^0 as two bf16 planes plus sum(S^0 ^2) per row (tile 0 carries the whole
+// sum, the other tile slots are zeroed).  One block per row.
+template <typename WT>
+__global__ void __launch_bounds__(256) embed_fused_kernel(const int32_t *tokens, int n, int p0, RowMap rm,
+                                                          const WT *__restrict__ E1, const WT *__restrict__ E2,
+                                                          const float *__restrict__ g, float eps, int d, int V,
+                                                          float *S, const float *__restrict__ g_next,
+                                                          __nv_bfloat16 *Xb, size_t lo_off, float *ss_out, int ss_ld,
+                                                          int ss_tiles, int *status) {
+    pdl_enter();
+    __shared__ float scratch[32];
+    int r = blockIdx.x;
+    int path = r >= rm.Bc();
+    int tok = ld_mut(tokens + (size_t)rm.seq(r) * n + p0 + rm.off(r));
+    if (tok < 0 || tok >= V) {
+        if (threadIdx.x == 0) report(status, kStatusBadToken, tok);
+        tok = min(max(tok, 0), V - 1);
+    }
+    const WT *e = (path ? E2 : E1) + (size_t)tok * d;
+    float ss = 0.f;
+    for (int i = threadIdx.x; i < d; i += blockDim.x) {
+        float x = load1(e + i);
+        ss += x * x;
+    }
+    ss = block_sum(ss, scratch);
+    float inv = 1.f / sqrtf(ss / (float)d + eps), sq = 0.f;
+    for (int i = threadIdx.x; i < d; i += blockDim.x) {
+        float s0 = g[i] * load1(e + i) * inv;
+        S[(size_t)r * d + i] = s0;
+        store_split(Xb, (size_t)r * d + i, lo_off, g_next[i] * s0);
+        sq += s0 * s0;
+    }
+    sq = block_sum(sq, scratch);
+    for (int t = threadIdx.x; t < ss_tiles; t += blockDim.x) ss_out[(size_t)t * ss_ld + r] = t == 0 ? sq : 0.f;
+}
+
 // Sum split partials into a plain fp32 matrix (used by the operator-level GEMM entry point).
 __global__ void reduce_splits_kernel(const float *P, int nsplit, size_t split_stride, size_t n,
                                      float *Y) {

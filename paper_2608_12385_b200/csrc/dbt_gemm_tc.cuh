@@ -16,6 +16,7 @@
 #include <cuda.h>
 
 #include "dbt_common.cuh"
+#include "dbt_gemm_epi.cuh"
 
 namespace dbt {
 
@@ -146,7 +147,8 @@ struct TcCfg {
 template <int N_TILE>
 __global__ void __launch_bounds__(128, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtensorMap tmW1,
-               const __grid_constant__ CUtensorMap tmW2, const __grid_constant__ CUtensorMap tmX, TcParams p) {
+               const __grid_constant__ CUtensorMap tmW2, const __grid_constant__ CUtensorMap tmX, TcParams p,
+               FusedEpi e) {
     using Cfg = TcCfg<N_TILE>;
     constexpr int STAGES = Cfg::kStages;
     extern __shared__ uint8_t smem_raw[];
@@ -245,10 +247,26 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
     pdl_wait();
     bool got = mbar_wait(accum_bar, 0);
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    if (got) {
+    if (!got && lane == 0) report(p.status, kStatusWaitExpired, 200 + warp);
+    got = __syncthreads_and(got);  // the ring is idle from here on: its memory serves as scratch
+    float *scratch = reinterpret_cast<float *>(gen_tiles);
+    int rows = min(seg.rows, p.R);
+    if (got && e.mode == FE_LMHEAD) {
+        epi_row_scales(e, p.R, scratch);
+        int f = f0 + warp * 32 + lane;
+#pragma unroll 1
+        for (int c0 = 0; c0 < N_TILE && c0 < rows; c0 += 16) {
+            float v[16];
+            tmem_ld16(tmem_base + ((uint32_t)(warp * 32) << 16) + c0, v);
+            if (f < seg.n_out) {
+#pragma unroll
+                for (int i = 0; i < 16; i++)
+                    if (c0 + i < rows) e.Z[(size_t)(c0 + i) * p.ldp + seg.col0 + f] = v[i] * scratch[c0 + i];
+            }
+        }
+    } else if (got) {
         int f = f0 + warp * 32 + lane;
         float *out = p.P + (size_t)split * p.R * p.ldp + seg.col0 + f;
-        int rows = min(seg.rows, p.R);
 #pragma unroll 1
         for (int c0 = 0; c0 < N_TILE && c0 < rows; c0 += 16) {
             float v[16];
@@ -259,8 +277,26 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
                     if (c0 + i < rows) out[(size_t)(c0 + i) * p.ldp] = v[i];
             }
         }
-    } else if (lane == 0) {
-        report(p.status, kStatusWaitExpired, 200 + warp);
+        if (e.mode != FE_NONE) {
+            // arrival ticket of this output tile; the last CTA folds the splits and finishes the tile
+            __threadfence();
+            __syncthreads();
+            int *flag = reinterpret_cast<int *>(scratch);
+            if (tid == 0) {
+                int *tk = e.tickets + (e.mode == FE_GATEUP ? tile - seg.tile0 : tile);
+                int t = atomicAdd(tk, 1);
+                int last = t == e.arrivals - 1;
+                if (last) atomicExch(tk, 0);
+                *flag = last;
+            }
+            __syncthreads();
+            int last = *flag;
+            __syncthreads();
+            if (last) {
+                __threadfence();
+                fused_epilogue(e, p.P, gridDim.y, p.R, p.ldp, f0, seg.col0, seg.n_out, sg, tile, scratch);
+            }
+        }
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();

@@ -305,3 +305,14 @@ def test_fresh_models_give_bitwise_identical_results():
     for other in runs[1:]:
         for x, y in zip(runs[0], other):
             assert torch.equal(x["z1"], y["z1"]) and torch.equal(x["z2"], y["z2"])
+
+
+def test_fused_epilogue_path_matches_oracle(monkeypatch):
+    """The opt-in variant that folds the elementwise work into the GEMM epilogues (last-arriving
+    CTA per output tile) computes the same step."""
+    monkeypatch.setenv("DBT_FUSED", "1")
+    cfg = small_bf16()
+    w = make_weights(cfg, seed=5, matrix_std=0.05)
+    tok = make_tokens(cfg, 3, 40, seed=6)
+    teacher_forced_compare(cfg, w, tok, n_prefill=35, grouped=True)
+    teacher_forced_compare(cfg, w, tok, n_prefill=35, grouped=False)
