@@ -180,6 +180,31 @@ dbt_status dbt_op_gemm_tc(const void *W_dev, const void *X_dev, int32_t n_out, i
                           int32_t force_split, float *Y_dev, float *scratch_dev, size_t scratch_floats,
                           int32_t *status_dev, void *cuda_stream, int32_t *split_used);
 
+/* The same GEMM for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this entry exists for the integration, not for the method.)  Some hosts of this
+ * library run where cudaMalloc is off limits -- inside a region that is being captured into a
+ * CUDA graph, in a process whose memory pool is owned and fully handed out by another runtime,
+ * or under a policy that forbids allocation after start-up -- and so cannot provide the split-K
+ * workspace that dbt_op_gemm_tc asks for.  Here that workspace is a fixed array inside the
+ * library's device image: 2^21 floats (8 MiB), resident on every GPU that has loaded the
+ * library until the process exits.  The call allocates nothing and frees nothing.
+ *   - Arguments as dbt_op_gemm_tc without the scratch pair; inputs, Y_dev and status_dev are
+ *     still the caller's.  Results are identical to dbt_op_gemm_tc for the same split factor.
+ *   - Limit: roundup(R) * n_out * splits <= 2^21 (roundup to 16/32/64/128/256).  The library
+ *     lowers its own split choice to fit; a request that cannot fit even unsplit, or a
+ *     force_split that does not fit, returns DBT_ERR_CAPACITY with a message and enqueues
+ *     nothing.
+ *   - The first call on each device looks up the array's device address (no allocation, but a
+ *     runtime query): make that first call outside any stream capture, with the target device
+ *     current.
+ *   - All calls on a device share the one array and leave their partial sums in it.  Nothing in
+ *     it needs to start at zero -- every element that is read has been written by the same
+ *     call -- but two calls whose kernels overlap on the GPU (different streams, or a second
+ *     process thread) race on it: serialise them. */
+dbt_status dbt_op_gemm_tc_static(const void *W_dev, const void *X_dev, int32_t n_out, int32_t K, int32_t R,
+                                 int32_t force_split, float *Y_dev, int32_t *status_dev, void *cuda_stream,
+                                 int32_t *split_used);
+
 /* Per-kernel timing for the roofline report (paper Eq. roofline, Eq. decode_traffic: time
  * against the bytes that must move).  Between begin and end every kernel launch is bracketed
  * by CUDA events on the handle's stream; end waits for the stream and sums, per kernel family,

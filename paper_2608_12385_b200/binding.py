@@ -23,7 +23,8 @@ STATUS_NAMES = {0: "DBT_OK", 1: "DBT_ERR_INVALID_ARG", 2: "DBT_ERR_UNSUPPORTED",
 EXPORTS = ["dbt_query_sizes", "dbt_create", "dbt_destroy", "dbt_set_page_table", "dbt_reset", "dbt_set_seq_lens",
            "dbt_seq_len", "dbt_prefill", "dbt_decode_step", "dbt_decode_step_primary_only", "dbt_decode_step_host",
            "dbt_decode_step_primary_only_host", "dbt_last_experts", "dbt_last_expert_union", "dbt_sync_status",
-           "dbt_launch_count", "dbt_last_error", "dbt_version", "dbt_profile_begin", "dbt_profile_end", "dbt_op_gemm_tc"]
+           "dbt_launch_count", "dbt_last_error", "dbt_version", "dbt_profile_begin", "dbt_profile_end", "dbt_op_gemm_tc",
+           "dbt_op_gemm_tc_static"]
 
 
 class DbtError(RuntimeError):
@@ -90,6 +91,7 @@ def load_library():
     L.dbt_last_expert_union.argtypes = [vp, vp]
     L.dbt_sync_status.argtypes = [vp, i32p, i32p]
     L.dbt_op_gemm_tc.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, C.c_size_t, vp, vp, i32p]
+    L.dbt_op_gemm_tc_static.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, vp, i32p]
     L.dbt_profile_begin.argtypes = [vp]
     L.dbt_profile_end.argtypes = [vp, C.POINTER(DbtProfileEntry), i32, i32p]
     L.dbt_launch_count.argtypes = [vp]
@@ -139,6 +141,31 @@ def op_gemm_tc(W: torch.Tensor, X: torch.Tensor, force_split: int = 0, scratch: 
     used = C.c_int32(0)
     st = L.dbt_op_gemm_tc(W.data_ptr(), X.data_ptr(), n_out, K, R, force_split, Y.data_ptr(), scratch.data_ptr(),
                           scratch.numel(), status.data_ptr(), torch.cuda.current_stream().cuda_stream, C.byref(used))
+    if st != DBT_OK:
+        raise DbtError(st, L.dbt_last_error(None).decode())
+    torch.cuda.synchronize()
+    code = status.cpu().tolist()
+    if code[0] != 0:
+        raise DbtError(6, f"device status {code}")
+    return Y, used.value
+
+
+def op_gemm_tc_static(W: torch.Tensor, X: torch.Tensor, force_split: int = 0, Y: torch.Tensor | None = None,
+                      status: torch.Tensor | None = None):
+    """Y = X W^T through the entry point that allocates no device memory: its split-K workspace
+    is a fixed 8 MiB array inside the library.  Pass Y and status to make the call itself
+    allocation-free on the Python side too.  Returns (Y, split used)."""
+    L = load_library()
+    assert W.dtype == torch.bfloat16 and X.dtype == torch.bfloat16 and W.is_cuda and X.is_cuda
+    n_out, K = W.shape
+    R = X.shape[0]
+    if Y is None:
+        Y = torch.empty(R, n_out, dtype=torch.float32, device=W.device)
+    if status is None:
+        status = torch.zeros(2, dtype=torch.int32, device=W.device)
+    used = C.c_int32(0)
+    st = L.dbt_op_gemm_tc_static(W.data_ptr(), X.data_ptr(), n_out, K, R, force_split, Y.data_ptr(), status.data_ptr(),
+                                 torch.cuda.current_stream().cuda_stream, C.byref(used))
     if st != DBT_OK:
         raise DbtError(st, L.dbt_last_error(None).decode())
     torch.cuda.synchronize()

@@ -7,6 +7,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <string>
 #include <utility>
@@ -1403,6 +1404,64 @@ static dbt_status op_gemm_tc_impl(dbt_model *m, const void *W_dev, const void *X
     LAUNCH(m, "reduce", 0, reduce_splits_kernel, (unsigned)((n + 255) / 256), 256, 0, scratch_dev, nsp, stride, n, Y_dev);
     if (split_used) *split_used = nsp;
     return DBT_OK;
+}
+
+// ---- no-allocation variant -----------------------------------------------------------------
+// Split-K scratch for dbt_op_gemm_tc_static lives in this file-scope device array: 2^21 floats
+// (8 MiB), held by every GPU that loads the library until the process exits.  Host code may
+// not pass the symbol to a kernel (on the host it is only a stand-in for the device array):
+// its device address is looked up once per device with cudaGetSymbolAddress.
+constexpr size_t kStaticScratchFloats = (size_t)1 << 21;
+static __device__ __align__(256) float g_static_scratch[kStaticScratchFloats];
+
+static float *static_scratch_for_current_device(cudaError_t *err) {
+    static std::mutex mu;
+    static float *ptr_of_device[64] = {nullptr};
+    int dev = -1;
+    *err = cudaGetDevice(&dev);
+    if (*err != cudaSuccess) return nullptr;
+    if (dev < 0 || dev >= 64) {
+        *err = cudaErrorInvalidDevice;
+        return nullptr;
+    }
+    std::lock_guard<std::mutex> lock(mu);
+    if (!ptr_of_device[dev]) {
+        void *p = nullptr;
+        *err = cudaGetSymbolAddress(&p, g_static_scratch);  // resolved for the current device
+        if (*err != cudaSuccess) return nullptr;
+        ptr_of_device[dev] = static_cast<float *>(p);
+    }
+    return ptr_of_device[dev];
+}
+
+dbt_status dbt_op_gemm_tc_static(const void *W_dev, const void *X_dev, int32_t n_out, int32_t K, int32_t R,
+                                 int32_t force_split, float *Y_dev, int32_t *status_dev, void *cuda_stream,
+                                 int32_t *split_used) {
+    static thread_local dbt_model scratch_handle;  // carries the stream and the error text only
+    dbt_model *m = &scratch_handle;
+    m->stream = (cudaStream_t)cuda_stream;
+    m->prof_on = false;
+    m->use_pdl = false;
+    dbt_status st;
+    cudaError_t ce = cudaSuccess;
+    float *scratch = static_scratch_for_current_device(&ce);
+    if (!scratch) {
+        st = fail(m, DBT_ERR_CUDA, "cudaGetSymbolAddress(static scratch): %s", cudaGetErrorString(ce));
+    } else if (n_out > 0 && R > 0 && R <= 256 && (size_t)pad_rows(R) * (size_t)n_out > kStaticScratchFloats) {
+        st = fail(m, DBT_ERR_CAPACITY,
+                  "roundup(R)=%d rows x n_out=%d = %zu floats exceed the static scratch of %zu floats (8 MiB); "
+                  "use dbt_op_gemm_tc with caller-provided scratch",
+                  pad_rows(R), n_out, (size_t)pad_rows(R) * (size_t)n_out, kStaticScratchFloats);
+    } else if (force_split > 0 && (size_t)force_split * pad_rows(R > 0 && R <= 256 ? R : 1) * (size_t)(n_out > 0 ? n_out : 0) >
+                                      kStaticScratchFloats) {
+        st = fail(m, DBT_ERR_CAPACITY, "force_split=%d needs more than the static scratch of %zu floats (8 MiB)",
+                  force_split, kStaticScratchFloats);
+    } else {
+        st = op_gemm_tc_impl(m, W_dev, X_dev, n_out, K, R, force_split, Y_dev, scratch, kStaticScratchFloats, status_dev,
+                             split_used);
+    }
+    if (st != DBT_OK) g_create_error = m->err;
+    return st;
 }
 
 dbt_status dbt_op_gemm_tc(const void *W_dev, const void *X_dev, int32_t n_out, int32_t K, int32_t R, int32_t force_split,
