@@ -92,11 +92,13 @@ class ClockSampler:
         return out
 
 
-def step_bytes(cfg, B: int, ctx_keys_first: int, steps: int) -> float:
+def step_bytes(cfg, B: int, ctx_keys_first: int, steps: int, union=None) -> float:
     """Algorithmic bytes of one step, averaged over `steps` steps whose first reads
-    ctx_keys_first keys per sequence: every shared matrix once + every visible K/V once."""
+    ctx_keys_first keys per sequence: every shared matrix once + every visible K/V once.
+    MoE: `union` = routed experts loaded per layer (realised, read back from the device)."""
     avg_keys = ctx_keys_first + (steps - 1) / 2.0
-    return cfg.matrix_bytes_dense_step() + B * avg_keys * cfg.kv_bytes_per_token()
+    mats = cfg.matrix_bytes_moe_step(union) if cfg.is_moe else cfg.matrix_bytes_dense_step()
+    return mats + B * avg_keys * cfg.kv_bytes_per_token()
 
 
 def run_ours(args) -> dict | None:
@@ -108,7 +110,7 @@ def run_ours(args) -> dict | None:
     build.build()
     cfg = PRESETS[args.model]()
     if cfg.is_moe:
-        raise SystemExit("bench.py times the dense configurations; MoE timing lives in the tests' sweep")
+        cfg = cfg.replace(k_branch=args.k_branch, router_mode=args.router_mode)
     B, S, K, W = args.batch, args.ctx, args.steps, args.warmup
     t0 = time.time()
     w = make_weights(cfg, seed=0)
@@ -156,11 +158,15 @@ def run_ours(args) -> dict | None:
         clocks = sampler.stop() if sampler else None
         return e0.elapsed_time(e1), m.launch_count() - launches0, clocks
 
-    ms_total, launches, clocks = timed(True, K, W, True)
     ms_po, _, _ = timed(False, K, W, False)
+    po_union_m = m.last_expert_union() if cfg.is_moe else None
+    ms_total, launches, clocks = timed(True, K, W, True)
     value, ms_max = replicas.aggregate_throughput(B * K, ms_total, dev)
     ms_step = ms_max / K
-    bytes_step = step_bytes(cfg, B, S + W, K)
+    union = po_union = None
+    if cfg.is_moe:  # the routed experts actually loaded by the last grouped step, per layer
+        union = m.last_expert_union()
+    bytes_step = step_bytes(cfg, B, S + W, K, union)
 
     # per-kernel device time, on the launching stream, for the roofline of the dominant kernel
     m.set_seq_lens([S - 1] * B)
@@ -207,7 +213,7 @@ def run_ours(args) -> dict | None:
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if cfg.weight_dtype == "bf16" else "f32", "data": "synthetic",
-        "config": {"workload": f"dense-{args.model} bf16 grouped decode, batch {B}/GPU, prompt {S}, "
+        "config": {"workload": f"{'moe' if cfg.is_moe else 'dense'}-{args.model} bf16 grouped decode, batch {B}/GPU, prompt {S}, "
                                f"{K} steps (paged KV, 16-token pages)",
                    "batch_per_gpu": B, "prompt": S, "kv_population": kv_mode,
                    "l2_policy": "inputs larger than L2 (weights + KV >= 1.7 GB per step vs 126 MB)",
@@ -223,7 +229,11 @@ def run_ours(args) -> dict | None:
                      "kernel_bytes_per_launch": dom["bytes"] / max(dom["launches"], 1)},
         "step_roofline": {"algorithmic_bytes_per_step": bytes_step, "achieved_gbs": achieved_step_gbs,
                           "frac_of_measured_copy": achieved_step_gbs / hbm, "frac_of_8tbs_nominal": achieved_step_gbs / 8000.0},
-        "primary_only": {"ms_per_step": ms_po / K, "grouped_over_primary_only": (ms_total / K) / (ms_po / K)},
+        "primary_only": {"ms_per_step": ms_po / K, "grouped_over_primary_only": (ms_total / K) / (ms_po / K),
+                         "experts_loaded_per_layer": po_union_m},
+        "moe": None if not cfg.is_moe else {"k_primary": cfg.k_primary, "k_branch": cfg.k_branch,
+                                            "router_mode": cfg.router_mode, "experts_loaded_per_layer": union,
+                                            "mean_union": sum(union) / len(union)},
         "kernels": [{"name": r["name"], "launches_per_step": r["launches"] / nprof,
                      "us_per_step": 1e3 * r["total_ms"] / nprof,
                      "gbs": (r["bytes"] / (r["total_ms"] * 1e-3) / 1e9) if r["bytes"] > 0 and r["total_ms"] > 0 else None}
@@ -284,6 +294,8 @@ def main():
     ap.add_argument("--batch", type=int, default=16)
     ap.add_argument("--ctx", type=int, default=2048)
     ap.add_argument("--kv", default="prefill", choices=["prefill", "synthetic"])
+    ap.add_argument("--k-branch", type=int, default=2, help="MoE: branch top-k")
+    ap.add_argument("--router-mode", type=int, default=0, help="MoE: 0 independent routing, 1 router replay")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--reference-max-steps", type=int, default=128)
     args = ap.parse_args()

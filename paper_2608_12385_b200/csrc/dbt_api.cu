@@ -36,11 +36,17 @@ struct Workspace {
     // bf16 tensor-core path: bf16 GEMM inputs and the fp32 split-K partial buffer
     __nv_bfloat16 *Xb, *Ob, *Hb;
     float *P, *ss;
+    // MoE on tensor cores: activation rows sorted by expert
+    __nv_bfloat16 *Xs, *Hs;
+    float *Pe;
+    int32_t *epos, *eoff;
     size_t P_floats;
 };
 
 struct LayerMaps {
-    CUtensorMap wq, wk, wv, wo, wg, wu, wd;
+    CUtensorMap wq, wk, wv, wo, wg, wu, wd;  // dense MLP; for MoE wg/wu/wd hold the shared expert
+    CUtensorMap eg, eu, ed;                  // all routed experts as [E*Fe, d], [E*Fe, d], [E*d, Fe]
+    CUtensorMap rt;                          // router [E, d]
 };
 
 }  // namespace
@@ -67,7 +73,8 @@ struct dbt_model {
     // tensor-core path (bf16 models): TMA descriptors of every weight matrix and GEMM input
     bool tc;
     std::vector<LayerMaps> maps;
-    CUtensorMap map_lm, map_Xb, map_Ob, map_Hb, map_kv;
+    CUtensorMap map_lm, map_Xb, map_Ob, map_Hb, map_kv, map_Xs, map_Hs;
+    bool moe_tc;  // MoE experts on the tensor cores
     bool att_fast;  // TMA + mma.sync attention over the bf16 pool
     bool fused;     // dense bf16: elementwise work fused into the GEMM epilogues
     int num_sms;
@@ -192,6 +199,14 @@ size_t carve(const dbt_config &c, char *base, Workspace *ws, int *Rmax_out, int 
         if (w.P_floats < (size_t)Rmax * widest) w.P_floats = (size_t)Rmax * widest;
         w.P = k.take<float>(w.P_floats);
         w.ss = k.take<float>((size_t)((d + 127) / 128) * Rmax);
+        if (moe) {
+            size_t Rk = (size_t)Rmax * kmax_of(c);
+            w.Xs = k.take<__nv_bfloat16>(2 * Rk * d);
+            w.Hs = k.take<__nv_bfloat16>(2 * Rk * c.d_expert);
+            w.Pe = k.take<float>(Rk * 2 * c.d_expert);
+            w.epos = k.take<int32_t>(Rk);
+            w.eoff = k.take<int32_t>(c.n_experts + 1);
+        }
     }
     if (ws) *ws = w;
     if (Rmax_out) *Rmax_out = Rmax;
@@ -355,7 +370,7 @@ dbt_status run_moe(dbt_model *m, int l, const RowMap &rm, int grouped, bool reco
     if (last && !grouped)
         CUDA_TRY(m, cudaMemsetAsync(last + (size_t)c.max_batch * km, 0xff, sizeof(int32_t) * c.max_batch * km,
                                     m->stream));
-    LAUNCH(m, "route", 0, route_kernel, R, 32, E * sizeof(float) + E, w.rlogits, E, Bc, c.k_primary, c.k_branch, km,
+    LAUNCH(m, "route", 0, route_kernel, R, 32, 2 * E * sizeof(float), w.rlogits, 1, (size_t)0, E, Bc, c.k_primary, c.k_branch, km,
            c.router_mode == DBT_ROUTER_REPLAY, w.ridx, w.rwts, last, c.max_batch * km);
     int32_t *ucnt = record_experts ? w.union_cnt + l : nullptr;
     if (ucnt) CUDA_TRY(m, cudaMemsetAsync(ucnt, 0, sizeof(int32_t), m->stream));
@@ -465,6 +480,8 @@ struct TcCall {
     const char *tag;
     int parts;    // 1 or 2 bf16 terms per activation
     int lo_row0;  // row of the lo plane in the activation buffer
+    const int *grp_cnt, *grp_off;  // per-expert mode (see TcParams); n_groups experts
+    int grp_w_rows, n_groups;
 };
 
 int norm_threads(int d) { return d >= 1024 ? 1024 : d >= 512 ? 512 : 256; }
@@ -505,7 +522,7 @@ dbt_status run_gemm_tc(dbt_model *m, const TcCall &c, int n_tile, int *nsplit_ou
         p.seg[s] = TcSeg{tiles, c.n_out[s], c.rows[s], col};
         tiles += (c.n_out[s] + kTcM - 1) / kTcM;
         col += c.n_out[s];
-        bytes += (double)c.n_out[s] * c.K * 2;
+        if (!c.grp_cnt) bytes += (double)c.n_out[s] * c.K * 2;  // per-expert launches: the loaded set is known on the device only
     }
     p.nseg = c.nseg;
     p.K = c.K;
@@ -513,9 +530,13 @@ dbt_status run_gemm_tc(dbt_model *m, const TcCall &c, int n_tile, int *nsplit_ou
     p.R = c.R;
     p.parts = c.parts;
     p.lo_row0 = c.lo_row0;
+    p.grp_cnt = c.grp_cnt;
+    p.grp_off = c.grp_off;
+    p.grp_w_rows = c.grp_w_rows;
     p.P = c.P;
     p.status = m->ws.status;
     int total_kt = (c.K + kTcK - 1) / kTcK;
+    if (c.grp_cnt) force_split = 1;  // enough CTAs already: tiles x selected experts
     int split = force_split > 0 ? (force_split < total_kt ? force_split : total_kt) : choose_split(tiles, total_kt);
     while (split > 1 && (size_t)split * n_tile * col > c.P_floats) split--;
     if ((size_t)c.R * col > c.P_floats) return fail(m, DBT_ERR_CAPACITY, "partial buffer too small for %s", c.tag);
@@ -527,7 +548,7 @@ dbt_status run_gemm_tc(dbt_model *m, const TcCall &c, int n_tile, int *nsplit_ou
     }
     e.arrivals = (e.mode == FE_GATEUP ? 2 : 1) * split;
     if (e.mode != FE_NONE && tiles > 4096) return fail(m, DBT_ERR_UNSUPPORTED, "too many output tiles for %s", c.tag);
-    dim3 grid(tiles, split);
+    dim3 grid(tiles, split, c.grp_cnt ? c.n_groups : 1);
     if (nsplit_out) *nsplit_out = split;
     if (split_stride_out) *split_stride_out = (size_t)c.R * col;
     switch (n_tile) {
@@ -566,6 +587,78 @@ dbt_status run_attention_mma(dbt_model *m, const RowMap &rm, int grouped, int la
     if (items > kAttMaxItems) return fail(m, DBT_ERR_CAPACITY, "attention rows %d exceed %d", items, kAttMaxItems);
     dim3 grid(2 * m->num_sms);  // two resident CTAs per SM; each takes an equal share of all K/V tiles
     LAUNCH(m, "attention", kv_bytes, attn_mma_kernel<DH>, grid, 160, AttCfg<DH>::kSmemBytes, m->map_kv, p);
+    return DBT_OK;
+}
+
+// MoE sub-layer on the tensor cores (Eq. moe_layer, Eq. moe_budget, Section 4.3).  Rows of both
+// paths are sorted by expert; one grouped GEMM launch covers all experts (blockIdx.z), CTAs of
+// experts nobody selected exit before touching their weights, so each selected expert's
+// matrices are read once for the union of the primary top-k_1 and branch top-k_2 rows.
+dbt_status run_moe_tc(dbt_model *m, int l, const RowMap &rm, int grouped, bool record_experts) {
+    typedef __nv_bfloat16 WT;
+    const dbt_config &c = m->cfg;
+    const Workspace &w = m->ws;
+    const dbt_layer_weights &lw = m->layers[l];
+    const LayerMaps &mp = m->maps[l];
+    int Bc = rm.B * rm.cn, R = grouped ? 2 * Bc : Bc, d = c.d_model;
+    int E = c.n_experts, Fe = c.d_expert, km = kmax_of(c), Fs = c.n_shared_experts * Fe, Rk = m->Rmax * km;
+    int n_tile = pad_rows(R);
+    size_t lo_x = m->act_parts == 2 ? (size_t)m->Rmax * d : 0;
+    size_t lo_xs = m->act_parts == 2 ? (size_t)Rk * d : 0, lo_hs = m->act_parts == 2 ? (size_t)Rk * Fe : 0;
+    dbt_status st;
+    // router logits on the tensor cores (split-K partials summed by the routing kernel), then
+    // top-k per path and renormalised weights
+    int rnsp = 1;
+    size_t rstride = 0;
+    TcCall rt{};
+    rt.W[0] = &mp.rt; rt.n_out[0] = E; rt.rows[0] = R; rt.nseg = 1; rt.X = &m->map_Xb; rt.K = d; rt.R = R;
+    rt.P = w.P; rt.P_floats = w.P_floats; rt.tag = "router"; rt.parts = m->act_parts; rt.lo_row0 = m->Rmax;
+    if ((st = run_gemm_tc(m, rt, n_tile, &rnsp, &rstride)) != DBT_OK) return st;
+    int32_t *last = record_experts ? w.last_experts + (size_t)l * 2 * c.max_batch * km : nullptr;
+    if (last && !grouped)
+        CUDA_TRY(m, cudaMemsetAsync(last + (size_t)c.max_batch * km, 0xff, sizeof(int32_t) * c.max_batch * km, m->stream));
+    LAUNCH(m, "route", 0, route_kernel, R, 32, 2 * E * sizeof(float), w.P, rnsp, rstride, E, Bc, c.k_primary, c.k_branch, km,
+           c.router_mode == DBT_ROUTER_REPLAY, w.ridx, w.rwts, last, c.max_batch * km);
+    LAUNCH(m, "moe_sort", 0, moe_sort_kernel, 1, 1024, 0, w.ridx, R, km, E, w.ecnt, w.eoff, w.epos,
+           record_experts ? w.union_cnt + l : (int32_t *)nullptr);
+    LAUNCH(m, "moe_gather", 0, moe_gather_kernel, R * km, 256, 0, w.Xb, lo_x, w.ridx, w.epos, km, d, w.Xs, lo_xs);
+    // routed experts: gate|up, SwiGLU, down
+    TcCall gu{};
+    gu.W[0] = &mp.eg; gu.n_out[0] = Fe; gu.rows[0] = Rk;
+    gu.W[1] = &mp.eu; gu.n_out[1] = Fe; gu.rows[1] = Rk;
+    gu.nseg = 2; gu.X = &m->map_Xs; gu.K = d; gu.R = Rk; gu.P = w.Pe; gu.P_floats = (size_t)Rk * 2 * Fe;
+    gu.tag = "expert_gateup"; gu.parts = m->act_parts; gu.lo_row0 = Rk;
+    gu.grp_cnt = w.ecnt; gu.grp_off = w.eoff; gu.grp_w_rows = Fe; gu.n_groups = E;
+    if ((st = run_gemm_tc(m, gu, n_tile, nullptr, nullptr)) != DBT_OK) return st;
+    LAUNCH(m, "moe_swiglu", 0, moe_swiglu_kernel, dim3(R * km, (Fe + 255) / 256), 256, 0, w.Pe, w.eoff + E, Fe, w.Hs, lo_hs);
+    TcCall dn{};
+    dn.W[0] = &mp.ed; dn.n_out[0] = d; dn.rows[0] = Rk; dn.nseg = 1; dn.X = &m->map_Hs; dn.K = Fe; dn.R = Rk;
+    dn.P = w.Yexp; dn.P_floats = (size_t)Rk * d; dn.tag = "expert_down"; dn.parts = m->act_parts; dn.lo_row0 = Rk;
+    dn.grp_cnt = w.ecnt; dn.grp_off = w.eoff; dn.grp_w_rows = d; dn.n_groups = E;
+    if ((st = run_gemm_tc(m, dn, n_tile, nullptr, nullptr)) != DBT_OK) return st;
+    // shared expert(s) on every row of both paths; b couples its hidden state
+    const float *Psh = nullptr;
+    int nsp = 1;
+    size_t sstride = 0;
+    if (Fs > 0) {
+        int nt = pad_rows(R);
+        TcCall sg{};
+        sg.W[0] = &mp.wg; sg.n_out[0] = Fs; sg.rows[0] = R;
+        sg.W[1] = &mp.wu; sg.n_out[1] = Fs; sg.rows[1] = R;
+        sg.nseg = 2; sg.X = &m->map_Xb; sg.K = d; sg.R = R; sg.P = w.P; sg.P_floats = w.P_floats; sg.tag = "shared_gateup";
+        sg.parts = m->act_parts; sg.lo_row0 = m->Rmax;
+        if ((st = run_gemm_tc(m, sg, nt, &nsp, &sstride)) != DBT_OK) return st;
+        LAUNCH(m, "swiglu_couple", 0, swiglu_couple_kernel, dim3(Bc, (Fs + 255) / 256), 256, 0, w.P, nsp, sstride, Fs, Bc,
+               grouped, c.moe_b_coupling ? lw.coup_b : (const float *)nullptr, w.Hb,
+               m->act_parts == 2 ? (size_t)m->Rmax * Fs : (size_t)0);
+        TcCall sd{};
+        sd.W[0] = &mp.wd; sd.n_out[0] = d; sd.rows[0] = R; sd.nseg = 1; sd.X = &m->map_Hb; sd.K = Fs; sd.R = R;
+        sd.P = w.P; sd.P_floats = w.P_floats; sd.tag = "shared_down"; sd.parts = m->act_parts; sd.lo_row0 = m->Rmax;
+        if ((st = run_gemm_tc(m, sd, nt, &nsp, &sstride)) != DBT_OK) return st;
+        Psh = w.P;
+    }
+    LAUNCH(m, "moe_combine", 0, moe_combine_sorted_kernel, dim3(Bc, (d + 255) / 256), 256, 0, w.Yexp, Psh, nsp, sstride, w.ridx, w.epos, w.rwts, km,
+           Bc, grouped, lw.coup_c, d, w.S);
     return DBT_OK;
 }
 
@@ -640,7 +733,8 @@ dbt_status run_layers_tc(dbt_model *m, const RowMap &rm, int grouped, int n_tile
             if ((st = run_gemm_tc(m, dn, n_tile, &nsp, &sstride)) != DBT_OK) return st;
             mode = 2;
         } else {
-            if ((st = run_moe<WT>(m, l, rm, grouped, record_experts)) != DBT_OK) return st;
+            st = m->moe_tc ? run_moe_tc(m, l, rm, grouped, record_experts) : run_moe<WT>(m, l, rm, grouped, record_experts);
+            if (st != DBT_OK) return st;
             mode = 0;
         }
     }
@@ -908,6 +1002,30 @@ bool setup_tc(dbt_model *m) {
         if (!moe)
             ok = ok && make_bf16_map(&mp.wg, lw.w_gate, F, d, kTcM) && make_bf16_map(&mp.wu, lw.w_up, F, d, kTcM) &&
                  make_bf16_map(&mp.wd, lw.w_down, d, F, kTcM);
+    }
+    m->moe_tc = false;
+    if (moe && ok) {
+        int E = c.n_experts, Fe = c.d_expert, Fs = c.n_shared_experts * Fe, Rk = m->Rmax * kmax_of(c);
+        const char *mo = getenv("DBT_MOE");
+        bool want = !(mo && strcmp(mo, "simt") == 0);
+        bool mok = want;
+        for (int l = 0; l < c.n_layers && mok; l++) {
+            const dbt_layer_weights &lw = m->layers[l];
+            LayerMaps &mp = m->maps[l];
+            mok = make_bf16_map(&mp.eg, lw.exp_gate, (uint64_t)E * Fe, d, kTcM) &&
+                  make_bf16_map(&mp.eu, lw.exp_up, (uint64_t)E * Fe, d, kTcM) &&
+                  make_bf16_map(&mp.ed, lw.exp_down, (uint64_t)E * d, Fe, kTcM) &&
+                  make_bf16_map(&mp.rt, lw.router, E, d, kTcM);
+            if (mok && Fs > 0)
+                mok = make_bf16_map(&mp.wg, lw.sh_gate, Fs, d, kTcM) && make_bf16_map(&mp.wu, lw.sh_up, Fs, d, kTcM) &&
+                      make_bf16_map(&mp.wd, lw.sh_down, d, Fs, kTcM);
+        }
+        mok = mok && make_bf16_map(&m->map_Xs, w.Xs, 2 * (uint64_t)Rk, d, 16) &&
+              make_bf16_map(&m->map_Hs, w.Hs, 2 * (uint64_t)Rk, Fe, 16);
+        if (mok && Fs > 0) mok = make_bf16_map(&m->map_Hb, w.Hb, 2 * m->Rmax, Fs, 16);
+        // (a weight tile that runs past its expert's last row only computes features that the
+        // epilogue never stores)
+        m->moe_tc = mok;
     }
     ok = ok && make_bf16_map(&m->map_lm, m->w.lm_head, c.vocab, d, kTcM);
     ok = ok && make_bf16_map(&m->map_Xb, w.Xb, 2 * m->Rmax, d, 16) && make_bf16_map(&m->map_Ob, w.Ob, 2 * m->Rmax, qd, 16);

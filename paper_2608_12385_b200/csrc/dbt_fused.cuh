@@ -185,6 +185,96 @@ __global__ void __launch_bounds__(256) embed_fused_kernel(const int32_t *tokens,
     for (int t = threadIdx.x; t < ss_tiles; t += blockDim.x) ss_out[(size_t)t * ss_ld + r] = t == 0 ? sq : 0.f;
 }
 
+// ---- MoE on tensor cores: rows sorted by expert ---------------------------------------------
+
+// Per-expert row lists -> offsets and the sorted position of every (row, slot) entry.  Entries of
+// one expert keep ascending (row, slot) order; experts follow each other in index order.
+// One block, one thread per expert (E <= 1024).
+__global__ void __launch_bounds__(1024) moe_sort_kernel(const int32_t *idx, int R, int kmax, int E, int32_t *cnt,
+                                                        int32_t *off, int32_t *pos, int32_t *union_count) {
+    pdl_enter();
+    __shared__ int s_cnt[1024], s_off[1025];
+    int e = threadIdx.x, c = 0;
+    if (e < E)
+        for (int i = 0; i < R * kmax; i++) c += idx[i] == e;
+    s_cnt[e] = e < E ? c : 0;
+    __syncthreads();
+    if (e == 0) {
+        int run = 0, uni = 0;
+        for (int i = 0; i < E; i++) {
+            s_off[i] = run;
+            run += s_cnt[i];
+            uni += s_cnt[i] > 0;
+        }
+        s_off[E] = run;
+        if (union_count) *union_count = uni;
+    }
+    __syncthreads();
+    if (e < E) {
+        cnt[e] = c;
+        off[e] = s_off[e];
+        int k = 0;
+        for (int i = 0; i < R * kmax && k < c; i++)
+            if (idx[i] == e) pos[i] = s_off[e] + k++;
+    }
+    if (e == 0) off[E] = s_off[E];
+}
+
+// Copy each entry's activation row (both bf16 planes) to its sorted position.
+__global__ void __launch_bounds__(256) moe_gather_kernel(const __nv_bfloat16 *Xb, size_t lo_in, const int32_t *idx,
+                                                         const int32_t *pos, int kmax, int d, __nv_bfloat16 *Xs,
+                                                         size_t lo_out) {
+    pdl_enter();
+    int entry = blockIdx.x;
+    if (idx[entry] < 0) return;
+    const uint4 *src = reinterpret_cast<const uint4 *>(Xb + (size_t)(entry / kmax) * d);
+    uint4 *dst = reinterpret_cast<uint4 *>(Xs + (size_t)pos[entry] * d);
+    for (int i = threadIdx.x; i < d / 8; i += blockDim.x) {
+        dst[i] = src[i];
+        if (lo_out) dst[i + lo_out / 8] = src[i + lo_in / 8];
+    }
+}
+
+// H = SiLU(gate) * up on the sorted rows; Pe rows are [Fe gate | Fe up] (one split).
+__global__ void __launch_bounds__(256) moe_swiglu_kernel(const float *Pe, const int32_t *off_total, int Fe,
+                                                         __nv_bfloat16 *Hs, size_t lo_off) {
+    pdl_enter();
+    int p = blockIdx.x, f = blockIdx.y * blockDim.x + threadIdx.x;
+    if (p >= *off_total || f >= Fe) return;
+    float h = silu(Pe[(size_t)p * 2 * Fe + f]) * Pe[(size_t)p * 2 * Fe + Fe + f];
+    store_split(Hs, (size_t)p * Fe + f, lo_off, h);
+}
+
+// M_1 = sum_j w_1j Expert_j(m_1) + G(m_1);  M_2 = sum_j w_2j Expert_j(m_2) + G~(m_2) + c*M_1;
+// S_i += M_i.  Ys: expert outputs at sorted positions; Psh: split-K partials of the shared
+// expert's down projection (nullptr: no shared expert).  One block per primary row.
+__global__ void __launch_bounds__(256) moe_combine_sorted_kernel(const float *Ys, const float *Psh, int nsplit,
+                                                                 size_t split_stride, const int32_t *idx,
+                                                                 const int32_t *pos, const float *wts, int kmax, int Bc,
+                                                                 int grouped, const float *__restrict__ coup_c, int d,
+                                                                 float *S) {
+    pdl_enter();
+    int b = blockIdx.x;
+    for (int i = blockIdx.y * blockDim.x + threadIdx.x; i < d; i += gridDim.y * blockDim.x) {
+        float m1 = 0.f;
+        for (int j = 0; j < kmax; j++)
+            if (idx[(size_t)b * kmax + j] >= 0)
+                m1 = fmaf(wts[(size_t)b * kmax + j], Ys[(size_t)pos[(size_t)b * kmax + j] * d + i], m1);
+        if (Psh) m1 += sum_splits(Psh, split_stride, nsplit, (size_t)b * d + i);
+        S[(size_t)b * d + i] += m1;
+        if (grouped) {
+            int r = Bc + b;
+            float m2 = 0.f;
+            for (int j = 0; j < kmax; j++)
+                if (idx[(size_t)r * kmax + j] >= 0)
+                    m2 = fmaf(wts[(size_t)r * kmax + j], Ys[(size_t)pos[(size_t)r * kmax + j] * d + i], m2);
+            if (Psh) m2 += sum_splits(Psh, split_stride, nsplit, (size_t)r * d + i);
+            m2 += coup_c[i] * m1;
+            S[(size_t)r * d + i] += m2;
+        }
+    }
+}
+
 // Sum split partials into a plain fp32 matrix (used by the operator-level GEMM entry point).
 __global__ void reduce_splits_kernel(const float *P, int nsplit, size_t split_stride, size_t n,
                                      float *Y) {

@@ -43,6 +43,10 @@ struct TcParams {
     int lo_row0;       // row offset of the lo term inside the activation buffer
     float *P;          // [splits][R][ldp] fp32 partials
     int *status;
+    // grouped (per-expert) mode: blockIdx.z = expert; its rows are grp_cnt[e] consecutive rows of
+    // X and P starting at grp_off[e]; its weight rows start at e * grp_w_rows.  nullptr = off.
+    const int *grp_cnt, *grp_off;
+    int grp_w_rows;
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -163,6 +167,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
 
     int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     int tile = blockIdx.x, split = blockIdx.y;
+    int x_row0 = 0, w_row0 = 0, grp_n = -1;
+    if (p.grp_cnt) {
+        // the expert's row list comes from the previous kernel: nothing can start before it is known
+        pdl_wait();
+        grp_n = ld_mut(p.grp_cnt + blockIdx.z);
+        if (grp_n == 0) return;  // expert not selected by any row of either path: its weights are not read
+        x_row0 = ld_mut(p.grp_off + blockIdx.z);
+        w_row0 = blockIdx.z * p.grp_w_rows;
+    }
     int sg = 0;
     if (p.nseg > 1 && tile >= p.seg[1].tile0) sg = 1;
     if (p.nseg > 2 && tile >= p.seg[2].tile0) sg = 2;
@@ -205,11 +218,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
             for (int part = 0; part < p.parts; part++)
                 for (int j = 0; j < N_TILE / 16; j++)
                     tma_load_2d(tiles + s * Cfg::kStageBytes + kTcABytes + part * Cfg::kBBytes + j * 2048, &tmX,
-                                full_bar(s), kt * kTcK, part * p.lo_row0 + j * 16);
+                                full_bar(s), kt * kTcK, part * p.lo_row0 + x_row0 + j * 16);
         };
         for (int i = 0; i < npre; i++) {
             mbar_expect_tx(full_bar(i), tx);
-            tma_load_2d(tiles + i * Cfg::kStageBytes, tmW, full_bar(i), (kt0 + i) * kTcK, f0);
+            tma_load_2d(tiles + i * Cfg::kStageBytes, tmW, full_bar(i), (kt0 + i) * kTcK, w_row0 + f0);
         }
         pdl_wait();
         for (int i = 0; i < npre; i++) load_x(i, kt0 + i);
@@ -218,7 +231,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
             ok = mbar_wait(empty_bar(s), ((i / STAGES) - 1) & 1);
             if (!ok) break;
             mbar_expect_tx(full_bar(s), tx);
-            tma_load_2d(tiles + s * Cfg::kStageBytes, tmW, full_bar(s), (kt0 + i) * kTcK, f0);
+            tma_load_2d(tiles + s * Cfg::kStageBytes, tmW, full_bar(s), (kt0 + i) * kTcK, w_row0 + f0);
             load_x(s, kt0 + i);
         }
     } else if (warp == 1 && lane == 0) {
@@ -250,7 +263,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
     if (!got && lane == 0) report(p.status, kStatusWaitExpired, 200 + warp);
     got = __syncthreads_and(got);  // the ring is idle from here on: its memory serves as scratch
     float *scratch = reinterpret_cast<float *>(gen_tiles);
-    int rows = min(seg.rows, p.R);
+    int rows = grp_n >= 0 ? min(grp_n, N_TILE) : min(seg.rows, p.R);
     if (got && e.mode == FE_LMHEAD) {
         epi_row_scales(e, p.R, scratch);
         int f = f0 + warp * 32 + lane;
@@ -266,7 +279,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
         }
     } else if (got) {
         int f = f0 + warp * 32 + lane;
-        float *out = p.P + (size_t)split * p.R * p.ldp + seg.col0 + f;
+        float *out = p.P + ((size_t)split * p.R + x_row0) * p.ldp + seg.col0 + f;
 #pragma unroll 1
         for (int c0 = 0; c0 < N_TILE && c0 < rows; c0 += 16) {
             float v[16];

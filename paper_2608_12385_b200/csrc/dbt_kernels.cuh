@@ -459,48 +459,71 @@ __global__ void advance_len_kernel(int32_t *seq_len, int B, int n) {
 
 // Router: softmax over E logits, top-k by repeated "largest remaining, lowest index first",
 // weights renormalised over the selection.  Replay: the branch row takes its primary twin's
-// selection and weighs it with its own probabilities.  One warp per row.
-__global__ void route_kernel(const float *logits, int E, int Bc, int k_p, int k_b, int kmax, int replay,
-                             int32_t *idx, float *wts, int32_t *__restrict__ last,
-                             int last_stride_path) {
+// selection and weighs it with its own probabilities.  One warp per row; logits may arrive
+// as split-K partials [nsplit][R][E] (summed in split order).
+__global__ void __launch_bounds__(32) route_kernel(const float *logits, int nsplit, size_t split_stride, int E, int Bc,
+                                                   int k_p, int k_b, int kmax, int replay, int32_t *idx, float *wts,
+                                                   int32_t *last, int last_stride_path) {
     pdl_enter();
     extern __shared__ float smem[];
-    float *p = smem;                                   // [E] own-row probabilities
-    unsigned char *taken = (unsigned char *)(smem + E);  // [E]
+    float *own = smem, *sel = smem + E;  // own-row logits -> probabilities; selection-row logits
     int r = blockIdx.x, lane = threadIdx.x;
     int path = r >= Bc;
-    const float *own = logits + (size_t)r * E;
-    const float *sel = (path && replay) ? logits + (size_t)(r - Bc) * E : own;
+    int sel_row = (path && replay) ? r - Bc : r;
     int k = (path && !replay) ? k_b : k_p;
     float mx = -INFINITY;
-    for (int e = lane; e < E; e += 32) mx = fmaxf(mx, own[e]);
+    for (int e = lane; e < E; e += 32) {
+        float a = 0.f, b2 = 0.f;
+        for (int s = 0; s < nsplit; s++) {
+            a += logits[(size_t)s * split_stride + (size_t)r * E + e];
+            b2 += logits[(size_t)s * split_stride + (size_t)sel_row * E + e];
+        }
+        own[e] = a;
+        sel[e] = b2;
+        mx = fmaxf(mx, a);
+    }
     mx = warp_max(mx);
-    float s = 0.f;
+    float sum = 0.f;
     for (int e = lane; e < E; e += 32) {
         float x = expf(own[e] - mx);
-        p[e] = x;
-        s += x;
-        taken[e] = 0;
+        own[e] = x;
+        sum += x;
     }
-    s = warp_sum(s);
+    sum = warp_sum(sum);
     __syncwarp();
-    if (lane == 0) {
-        float tot = 0.f;
-        int chosen[64];
-        for (int j = 0; j < k; j++) {
-            int best = -1;
-            for (int e = 0; e < E; e++)
-                if (!taken[e] && (best < 0 || sel[e] > sel[best])) best = e;
-            taken[best] = 1;
-            chosen[j] = best;
-            tot += p[best] / s;
+    float tot = 0.f;
+    int mine = -1;  // lane j keeps the j-th selection (k <= 64: two rounds of lanes at most)
+    int mine2 = -1;
+    for (int j = 0; j < k; j++) {
+        float bv = -INFINITY;
+        int bi = 0x7fffffff;
+        for (int e = lane; e < E; e += 32) {
+            float v = sel[e];
+            if (v > bv || (v == bv && e < bi)) {  // NaN-free: taken entries are -inf
+                bv = v;
+                bi = e;
+            }
         }
-        for (int j = 0; j < kmax; j++) {
-            int e = j < k ? chosen[j] : -1;
-            idx[(size_t)r * kmax + j] = e;
-            wts[(size_t)r * kmax + j] = j < k ? (p[e] / s) / tot : 0.f;
-            if (last) last[(size_t)path * last_stride_path + (size_t)(r - path * Bc) * kmax + j] = e;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+            int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+            if (ov > bv || (ov == bv && oi < bi)) {
+                bv = ov;
+                bi = oi;
+            }
         }
+        if (lane == 0) sel[bi] = -INFINITY;
+        __syncwarp();
+        tot += own[bi] / sum;
+        if (j == lane) mine = bi;
+        if (j == lane + 32) mine2 = bi;
+    }
+    for (int j = lane; j < kmax; j += 32) {
+        int e = j < k ? (j < 32 ? mine : mine2) : -1;
+        idx[(size_t)r * kmax + j] = e;
+        wts[(size_t)r * kmax + j] = j < k ? (own[e] / sum) / tot : 0.f;
+        if (last) last[(size_t)path * last_stride_path + (size_t)(r - path * Bc) * kmax + j] = e;
     }
 }
 

@@ -72,6 +72,18 @@ class ModelConfig:
         per_layer += 3 * self.d_ff * self.d_model if not self.is_moe else 0
         return (self.n_layers * per_layer + self.vocab * self.d_model) * self.elem_bytes
 
+    def matrix_bytes_moe_step(self, experts_loaded_per_layer) -> int:
+        """Bytes of the matrices one MoE decode step must read once each: attention projections,
+        router, shared expert, output matrix, and the routed experts actually selected
+        (`experts_loaded_per_layer`: the size of the union over all rows of both paths)."""
+        attn = (self.q_dim + 2 * self.kv_dim) * self.d_model + self.d_model * self.q_dim
+        router = self.n_experts * self.d_model
+        shared = 3 * self.n_shared_experts * self.d_expert * self.d_model
+        expert = 3 * self.d_expert * self.d_model
+        total = self.n_layers * (attn + router + shared) + self.vocab * self.d_model
+        total += expert * int(sum(experts_loaded_per_layer))
+        return total * self.elem_bytes
+
     def kv_bytes_per_token(self) -> int:
         return 2 * self.kv_dim * self.n_layers * self.elem_bytes
 
