@@ -143,7 +143,11 @@ struct TcCfg {
     static constexpr int kStageBytes = kTcABytes + 2 * kBBytes;
     // small row counts: keep one CTA near 100 KB so that a dependent kernel's CTA can become
     // resident beside it; large row counts take the whole SM
+#ifdef DBT_TC_DEEP
+    static constexpr int kStages = N_TILE <= 16 ? 10 : N_TILE <= 32 ? 8 : N_TILE <= 64 ? 6 : N_TILE <= 128 ? 4 : 2;
+#else
     static constexpr int kStages = N_TILE <= 16 ? 5 : N_TILE <= 32 ? 4 : N_TILE <= 64 ? 3 : N_TILE <= 128 ? 4 : 2;
+#endif
     static constexpr int kTmemCols = N_TILE < 32 ? 32 : N_TILE;
     static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };

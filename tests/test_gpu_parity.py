@@ -316,3 +316,26 @@ def test_fused_epilogue_path_matches_oracle(monkeypatch):
     tok = make_tokens(cfg, 3, 40, seed=6)
     teacher_forced_compare(cfg, w, tok, n_prefill=35, grouped=True)
     teacher_forced_compare(cfg, w, tok, n_prefill=35, grouped=False)
+
+
+def test_8b_shape_two_layers_paged_with_shuffled_pages():
+    """The 8B-shaped configuration at full width (d 4096, 32 query / 8 KV heads, F 14336, vocab
+    128256) with two layers: batch 2, a 100-position synthetic cache scattered over a shuffled
+    page table, two grouped steps."""
+    from paper_2608_12385_b200.inputs import dense_8b
+    cfg = dense_8b().replace(n_layers=2)
+    w = make_weights(cfg, seed=0)
+    B, ctx = 2, 100
+    tok = make_tokens(cfg, B, 2, seed=2)
+    k, v = make_synthetic_kv(cfg, B, ctx, seed=3)
+    om = oracle.OracleModel(cfg, w, B, ctx + 2)
+    gm = make_gpu_model(cfg, w, B, ctx + 2, num_pages=40)
+    pt = make_page_table(B, (ctx + 2 + 15) // 16, 40, seed=4)
+    gm.set_page_table(pt)
+    om.inject_kv(k, v, ctx)
+    gm.write_kv(k, v)
+    for t in range(2):
+        o = om.decode_step(tok[:, t].numpy())
+        g = gm.decode_full(tok[:, t].cuda().contiguous())
+        assert_logits_close(g["z1"], o["z1"], "bf16", f"8B-shape step {t} z1")
+        assert_logits_close(g["z2"], o["z2"], "bf16", f"8B-shape step {t} z2")
