@@ -77,6 +77,7 @@ struct dbt_model {
     bool moe_tc;  // MoE experts on the tensor cores
     bool att_fast;  // TMA + mma.sync attention over the bf16 pool
     bool fused;     // dense bf16: elementwise work fused into the GEMM epilogues
+    bool wide;      // dense bf16: RMSNorm factor applied after the GEMM, no row-wide reduction kernel
     int num_sms;
     int act_parts;  // 2: GEMM inputs carried as hi + lo bf16 terms; 1: plain bf16
     // a decode step is captured once per (batch, mode, buffer set) and replayed as a CUDA graph
@@ -650,7 +651,7 @@ dbt_status run_moe_tc(dbt_model *m, int l, const RowMap &rm, int grouped, bool r
         if ((st = run_gemm_tc(m, sg, nt, &nsp, &sstride)) != DBT_OK) return st;
         LAUNCH(m, "swiglu_couple", 0, swiglu_couple_kernel, dim3(Bc, (Fs + 255) / 256), 256, 0, w.P, nsp, sstride, Fs, Bc,
                grouped, c.moe_b_coupling ? lw.coup_b : (const float *)nullptr, w.Hb,
-               m->act_parts == 2 ? (size_t)m->Rmax * Fs : (size_t)0);
+               m->act_parts == 2 ? (size_t)m->Rmax * Fs : (size_t)0, (const float *)nullptr, 0, 0, d, c.rms_eps);
         TcCall sd{};
         sd.W[0] = &mp.wd; sd.n_out[0] = d; sd.rows[0] = R; sd.nseg = 1; sd.X = &m->map_Hb; sd.K = Fs; sd.R = R;
         sd.P = w.P; sd.P_floats = w.P_floats; sd.tag = "shared_down"; sd.parts = m->act_parts; sd.lo_row0 = m->Rmax;
@@ -701,7 +702,7 @@ dbt_status run_layers_tc(dbt_model *m, const RowMap &rm, int grouped, int n_tile
         if ((st = run_gemm_tc(m, qkv, n_tile, &nsp, &sstride)) != DBT_OK) return st;
         LAUNCH(m, "qkv_epilogue", 0, qkv_epilogue_kernel<WT>, dim3(Bc, c.n_q_heads + c.n_kv_heads), 64, 0, w.P, nsp, sstride, w.Q, rm, grouped, c.n_q_heads,
                c.n_kv_heads, c.head_dim, lw.coup_a, w.rope, w.seq_len, w.page_table, m->pages_per_seq_max, c.num_pages,
-               c.page_size, kpool, vpool, w.status);
+               c.page_size, kpool, vpool, w.status, (const float *)nullptr, 0, 0, d, c.rms_eps);
         if (m->att_fast)
             st = c.head_dim == 128 ? run_attention_mma<128>(m, rm, grouped, l, kv_bytes)
                                    : run_attention_mma<64>(m, rm, grouped, l, kv_bytes);
@@ -726,7 +727,7 @@ dbt_status run_layers_tc(dbt_model *m, const RowMap &rm, int grouped, int n_tile
             if ((st = run_gemm_tc(m, gu, n_tile, &nsp, &sstride)) != DBT_OK) return st;
             dim3 sg(Bc, (F + 255) / 256);
             LAUNCH(m, "swiglu_couple", 0, swiglu_couple_kernel, sg, 256, 0, w.P, nsp, sstride, F, Bc, grouped, lw.coup_b,
-                   w.Hb, m->act_parts == 2 ? (size_t)m->Rmax * F : (size_t)0);
+                   w.Hb, m->act_parts == 2 ? (size_t)m->Rmax * F : (size_t)0, (const float *)nullptr, 0, 0, d, c.rms_eps);
             TcCall dn{};
             dn.W[0] = &mp.wd; dn.n_out[0] = d; dn.rows[0] = R; dn.nseg = 1; dn.X = &m->map_Hb; dn.K = F; dn.R = R;
             dn.P = w.P; dn.P_floats = w.P_floats; dn.parts = m->act_parts; dn.lo_row0 = m->Rmax; dn.tag = "gemm_down";
@@ -969,6 +970,148 @@ dbt_status prefill_fused(dbt_model *m, const int32_t *tokens_dev, int B, int n, 
     return DBT_OK;
 }
 
+// ---- dense bf16 path with the RMSNorm factor applied after the GEMM ---------------------------
+// No kernel of this chain reduces over a whole row: the residual kernel is column-parallel and
+// leaves per-block shares of sum(S^2); the kernels after the Q|K|V and gate|up GEMMs (and the
+// output-matrix GEMM's own epilogue) multiply by 1/rms.  9 kernels per layer.
+
+dbt_status run_layers_wide(dbt_model *m, const RowMap &rm, int grouped, int n_tile) {
+    typedef __nv_bfloat16 WT;
+    const dbt_config &c = m->cfg;
+    const Workspace &w = m->ws;
+    int Bc = rm.B * rm.cn, R = grouped ? 2 * Bc : Bc;
+    int d = c.d_model, qd = c.n_q_heads * c.head_dim, kvd = c.n_kv_heads * c.head_dim, F = c.d_ff;
+    size_t pool_layer_elems = (size_t)2 * c.num_pages * c.n_kv_heads * c.page_size * c.head_dim;
+    size_t lo_x = m->act_parts == 2 ? (size_t)m->Rmax * d : 0, lo_h = m->act_parts == 2 ? (size_t)m->Rmax * F : 0;
+    int ss_tiles = (d + 255) / 256, ss_ld = m->Rmax;
+    double kv_bytes = 0;
+    for (int b = 0; b < rm.B; b++)
+        for (int j = 0; j < rm.cn; j++) kv_bytes += (double)(m->len_host[b] + j + 1) * 2 * kvd * sizeof(WT);
+    dbt_status st;
+    int nsp = 1;
+    size_t sstride = 0;
+    auto call = [&](const char *tag, const CUtensorMap *X, int K) {
+        TcCall t{};
+        t.X = X; t.K = K; t.R = R; t.P = w.P; t.P_floats = w.P_floats; t.tag = tag;
+        t.parts = m->act_parts; t.lo_row0 = m->Rmax;
+        return t;
+    };
+    for (int l = 0; l < c.n_layers; l++) {
+        const dbt_layer_weights &lw = m->layers[l];
+        const LayerMaps &mp = m->maps[l];
+        WT *kpool = reinterpret_cast<WT *>(m->kv_pool) + (size_t)l * pool_layer_elems;
+        WT *vpool = kpool + pool_layer_elems / 2;
+        TcCall qkv = call("gemm_qkv", &m->map_Xb, d);
+        qkv.W[0] = &mp.wq; qkv.n_out[0] = qd; qkv.rows[0] = R;
+        qkv.W[1] = &mp.wk; qkv.n_out[1] = kvd; qkv.rows[1] = Bc;
+        qkv.W[2] = &mp.wv; qkv.n_out[2] = kvd; qkv.rows[2] = Bc;
+        qkv.nseg = 3;
+        if ((st = run_gemm_tc(m, qkv, n_tile, &nsp, &sstride)) != DBT_OK) return st;
+        LAUNCH(m, "qkv_epilogue", 0, qkv_epilogue_kernel<WT>, dim3(Bc, c.n_q_heads + c.n_kv_heads), 64, 0, w.P, nsp, sstride,
+               w.Q, rm, grouped, c.n_q_heads, c.n_kv_heads, c.head_dim, lw.coup_a, w.rope, w.seq_len, w.page_table,
+               m->pages_per_seq_max, c.num_pages, c.page_size, kpool, vpool, w.status, (const float *)w.ss, ss_tiles, ss_ld, d,
+               c.rms_eps);
+        st = c.head_dim == 128 ? run_attention_mma<128>(m, rm, grouped, l, kv_bytes)
+                               : run_attention_mma<64>(m, rm, grouped, l, kv_bytes);
+        if (st != DBT_OK) return st;
+        TcCall op = call("gemm_o", &m->map_Ob, qd);
+        op.W[0] = &mp.wo; op.n_out[0] = d; op.rows[0] = R; op.nseg = 1;
+        if ((st = run_gemm_tc(m, op, n_tile, &nsp, &sstride)) != DBT_OK) return st;
+        LAUNCH(m, "resid_wide", 0, resid_wide_kernel, dim3(Bc, ss_tiles), 256, 0, w.S, w.P, nsp, sstride, 1,
+               (const float *)nullptr, Bc, grouped, lw.mlp_norm_g, d, w.Xb, lo_x, w.ss, ss_ld);
+        TcCall gu = call("gemm_gateup", &m->map_Xb, d);
+        gu.W[0] = &mp.wg; gu.n_out[0] = F; gu.rows[0] = R;
+        gu.W[1] = &mp.wu; gu.n_out[1] = F; gu.rows[1] = R;
+        gu.nseg = 2;
+        if ((st = run_gemm_tc(m, gu, n_tile, &nsp, &sstride)) != DBT_OK) return st;
+        LAUNCH(m, "swiglu_couple", 0, swiglu_couple_kernel, dim3(Bc, (F + 255) / 256), 256, 0, w.P, nsp, sstride, F, Bc,
+               grouped, lw.coup_b, w.Hb, lo_h, (const float *)w.ss, ss_tiles, ss_ld, d, c.rms_eps);
+        TcCall dn = call("gemm_down", &m->map_Hb, F);
+        dn.W[0] = &mp.wd; dn.n_out[0] = d; dn.rows[0] = R; dn.nseg = 1;
+        if ((st = run_gemm_tc(m, dn, n_tile, &nsp, &sstride)) != DBT_OK) return st;
+        const float *g_next = l + 1 < c.n_layers ? m->layers[l + 1].attn_norm_g
+                                                 : (c.final_norm ? m->w.final_norm_g : (const float *)nullptr);
+        LAUNCH(m, "resid_wide", 0, resid_wide_kernel, dim3(Bc, ss_tiles), 256, 0, w.S, w.P, nsp, sstride, 2, lw.coup_c, Bc,
+               grouped, g_next, d, w.Xb, lo_x, w.ss, ss_ld);
+    }
+    return DBT_OK;
+}
+
+dbt_status run_head_wide(dbt_model *m, const RowMap &rm, int grouped, int n_tile) {
+    const dbt_config &c = m->cfg;
+    const Workspace &w = m->ws;
+    int R = (grouped ? 2 : 1) * rm.B * rm.cn;
+    TcCall lm{};
+    lm.W[0] = &m->map_lm; lm.n_out[0] = c.vocab; lm.rows[0] = R; lm.nseg = 1; lm.X = &m->map_Xb; lm.K = c.d_model;
+    lm.R = R; lm.P = w.Z; lm.P_floats = (size_t)R * c.vocab; lm.tag = "gemm_lm_head";
+    lm.parts = m->act_parts; lm.lo_row0 = m->Rmax;
+    FusedEpi e = epi_base(m, rm, grouped, FE_LMHEAD);
+    e.ss_tiles = (c.d_model + 255) / 256;
+    e.use_scale = c.final_norm;
+    e.Z = w.Z;
+    return run_gemm_tc(m, lm, n_tile, nullptr, nullptr, 0, e);
+}
+
+template <typename WT>
+dbt_status run_embed_wide(dbt_model *m, const int32_t *tokens_dev, int n, int p0, const RowMap &rm, int R) {
+    const dbt_config &c = m->cfg;
+    const Workspace &w = m->ws;
+    LAUNCH(m, "embed", 0, embed_fused_kernel<WT>, R, 256, 0, tokens_dev, n, p0, rm, (const WT *)m->w.embed_primary,
+           (const WT *)m->w.embed_branch, m->w.embed_norm_g, c.rms_eps, c.d_model, c.vocab, w.S,
+           m->layers[0].attn_norm_g, w.Xb, m->act_parts == 2 ? (size_t)m->Rmax * c.d_model : (size_t)0, w.ss, m->Rmax,
+           (c.d_model + 255) / 256, w.status);
+    return DBT_OK;
+}
+
+dbt_status step_wide(dbt_model *m, const int32_t *tokens_dev, int B, int grouped, int32_t *next_dev, float *z1_dev,
+                     float *z2_dev, float *alpha_dev) {
+    typedef __nv_bfloat16 WT;
+    const dbt_config &c = m->cfg;
+    const Workspace &w = m->ws;
+    RowMap rm{B, 1};
+    int R = grouped ? 2 * B : B, n_tile = pad_rows(2 * B);
+    dbt_status st;
+    if ((st = run_embed_wide<WT>(m, tokens_dev, 1, 0, rm, R)) != DBT_OK) return st;
+    if ((st = run_layers_wide(m, rm, grouped, n_tile)) != DBT_OK) return st;
+    if ((st = run_head_wide(m, rm, grouped, n_tile)) != DBT_OK) return st;
+    LAUNCH(m, "readout", 0, readout_kernel, B, 1024, 0, w.Z, B, c.vocab, grouped, next_dev, alpha_dev);
+    LAUNCH(m, "advance_len", 0, advance_len_kernel, (B + 127) / 128, 128, 0, w.seq_len, B, 1);
+    size_t zb = sizeof(float) * (size_t)B * c.vocab;
+    if (z1_dev) CUDA_TRY(m, cudaMemcpyAsync(z1_dev, w.Z, zb, cudaMemcpyDeviceToDevice, m->stream));
+    if (z2_dev && grouped)
+        CUDA_TRY(m, cudaMemcpyAsync(z2_dev, w.Z + (size_t)B * c.vocab, zb, cudaMemcpyDeviceToDevice, m->stream));
+    for (int b = 0; b < B; b++) m->len_host[b] += 1;
+    return DBT_OK;
+}
+
+dbt_status prefill_wide(dbt_model *m, const int32_t *tokens_dev, int B, int n, float *last_logits) {
+    typedef __nv_bfloat16 WT;
+    const dbt_config &c = m->cfg;
+    const Workspace &w = m->ws;
+    int cn_max = (m->Rmax < kAttMaxItems ? m->Rmax : kAttMaxItems) / B;
+    if (cn_max < 1) cn_max = 1;
+    // when logits are wanted the last position runs as its own chunk, so that the rows of the
+    // output-matrix GEMM are exactly the B last positions
+    int n_bulk = last_logits ? n - 1 : n;
+    dbt_status st;
+    for (int p0 = 0; p0 < n;) {
+        int cn = p0 < n_bulk ? (n_bulk - p0 < cn_max ? n_bulk - p0 : cn_max) : 1;
+        RowMap rm{B, cn};
+        int R = B * cn, n_tile = pad_rows(R);
+        if ((st = run_embed_wide<WT>(m, tokens_dev, n, p0, rm, R)) != DBT_OK) return st;
+        if ((st = run_layers_wide(m, rm, 0, n_tile)) != DBT_OK) return st;
+        if (last_logits && p0 + cn >= n) {
+            if ((st = run_head_wide(m, rm, 0, n_tile)) != DBT_OK) return st;
+            CUDA_TRY(m, cudaMemcpyAsync(last_logits, w.Z, sizeof(float) * (size_t)B * c.vocab, cudaMemcpyDeviceToDevice,
+                                        m->stream));
+        }
+        LAUNCH(m, "advance_len", 0, advance_len_kernel, (B + 127) / 128, 128, 0, w.seq_len, B, cn);
+        for (int b = 0; b < B; b++) m->len_host[b] += cn;
+        p0 += cn;
+    }
+    return DBT_OK;
+}
+
 template <int N_TILE>
 bool allow_smem() {
     return cudaFuncSetAttribute(gemm_tc_kernel<N_TILE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -1044,6 +1187,11 @@ bool setup_tc(dbt_model *m) {
     // partials alone, on 16..44 SMs, while the separate kernels spread that work over the GPU
     // and overlap with their neighbours through programmatic dependent launch.
     m->fused = ok && m->att_fast && !moe && (fu && strcmp(fu, "1") == 0);
+    const char *wi = getenv("DBT_WIDE");
+    // Opt-in (DBT_WIDE=1): 9 instead of 10 kernels per layer and no row-wide reduction, but measured
+    // no faster (1.62 vs 1.55 ms per step at batch 16 on the 1B model): the step is bound by the
+    // kernel-to-kernel dependency latency, not by these kernels' bodies.
+    m->wide = ok && m->att_fast && !moe && (wi && strcmp(wi, "1") == 0);
     const char *split = getenv("DBT_ACT_SPLIT");
     m->act_parts = (split && strcmp(split, "0") == 0) ? 1 : 2;
     return ok;
@@ -1360,6 +1508,7 @@ dbt_status dbt_prefill(dbt_model *m, const int32_t *tokens_dev, int32_t B, int32
     if (st != DBT_OK) return st;
     if (m->cfg.weight_dtype == DBT_DTYPE_F32) return prefill_impl<float>(m, tokens_dev, B, n, last_primary_logits_dev);
     if (m->fused) return prefill_fused(m, tokens_dev, B, n, last_primary_logits_dev);
+    if (m->wide) return prefill_wide(m, tokens_dev, B, n, last_primary_logits_dev);
     if (m->tc) return prefill_tc(m, tokens_dev, B, n, last_primary_logits_dev);
     return prefill_impl<__nv_bfloat16>(m, tokens_dev, B, n, last_primary_logits_dev);
 }
@@ -1368,6 +1517,7 @@ static dbt_status step_direct(dbt_model *m, const int32_t *tokens_dev, int B, in
                               float *z1, float *z2, float *alpha) {
     if (m->cfg.weight_dtype == DBT_DTYPE_F32) return step_impl<float>(m, tokens_dev, B, grouped, next_dev, z1, z2, alpha);
     if (m->fused) return step_fused(m, tokens_dev, B, grouped, next_dev, z1, z2, alpha);
+    if (m->wide) return step_wide(m, tokens_dev, B, grouped, next_dev, z1, z2, alpha);
     if (m->tc) return step_tc(m, tokens_dev, B, grouped, next_dev, z1, z2, alpha);
     return step_impl<__nv_bfloat16>(m, tokens_dev, B, grouped, next_dev, z1, z2, alpha);
 }

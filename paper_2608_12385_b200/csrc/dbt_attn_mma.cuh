@@ -98,6 +98,7 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
     int *cum = flag + 8;                 // [items + 1] prefix of tiles per row
     int *nk_s = cum + kAttMaxItems + 1;  // [items] visible keys per row
 
+    DBT_TL_DECL;
     int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     int items = p.rm.Bc(), Bc = items;
     int nq_act = p.grouped ? 2 * p.G : p.G, q_dim = p.n_kv * p.G * DH;
@@ -111,6 +112,7 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
     }
     pdl_launch_dependents();
     pdl_wait();  // sequence lengths, Q and the freshly appended K/V come from earlier kernels of the step
+    DBT_TL_WAITED;
     if (warp == 0) {
         int running = 0, longest = 0;
         if (lane == 0) cum[0] = 0;
@@ -443,6 +445,7 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
         u += t1 - t0;
         if (u == pair_end && g == p.n_kv - 1) item++;
     }
+    DBT_TL_END("attention");
 }
 
 // The whole pool as one 2-D bf16 tensor [rows][head_dim], rows = (layer, K|V, page, head, slot).

@@ -4,6 +4,7 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <stdio.h>
 
 namespace dbt {
 
@@ -20,6 +21,22 @@ __device__ __forceinline__ void report(int *status, int code, int detail) {
 // predecessor's results before reading or writing anything that predecessor touches.
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+#ifdef DBT_TIMELINE
+__device__ __forceinline__ unsigned long long gtime() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+#define DBT_TL_DECL unsigned long long tl0_ = gtime(), tl1_ = 0
+#define DBT_TL_WAITED tl1_ = gtime()
+#define DBT_TL_END(name)                                                                                   \
+    if (threadIdx.x == 0 && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0)                         \
+    printf("TL %s entry %llu waited %llu end %llu\n", name, tl0_, tl1_, gtime())
+#else
+#define DBT_TL_DECL
+#define DBT_TL_WAITED
+#define DBT_TL_END(name)
+#endif
 __device__ __forceinline__ void pdl_enter() {
     pdl_launch_dependents();
     pdl_wait();

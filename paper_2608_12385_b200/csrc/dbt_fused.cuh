@@ -20,6 +20,56 @@ __device__ __forceinline__ float sum_splits(const float *P, size_t split_stride,
     return m;
 }
 
+// 1/rms of a row from its per-tile shares of sum(x^2) (ss[t][ss_ld], summed in tile order);
+// 1 when ss == nullptr (the GEMM input was already normalised).
+__device__ __forceinline__ float row_scale(const float *ss, int ss_tiles, int ss_ld, int row, int d_norm, float eps) {
+    if (!ss) return 1.f;
+    float a = 0.f;
+    for (int t = 0; t < ss_tiles; t++) a += __ldcg(ss + (size_t)t * ss_ld + row);
+    return 1.f / sqrtf(a / (float)d_norm + eps);
+}
+
+// Residual update without the row-wide reduction: S += sum_s P[s] (mode 1) or, with the c
+// coupling, M_2 += c*M_1 first (mode 2); the next GEMM's input is g * S (un-normalised, two bf16
+// planes) and each 256-column block leaves its share of sum(S^2) per row in ss_out[tile][row].
+// The consumer of that GEMM multiplies by 1/rms (the GEMM is linear), see row_scale.
+// grid (primary rows, d / 256): every thread owns one column of a row and of its branch twin.
+__global__ void __launch_bounds__(256) resid_wide_kernel(float *S, const float *P, int nsplit, size_t split_stride,
+                                                         int mode, const float *__restrict__ coup_c, int Bc, int grouped,
+                                                         const float *__restrict__ g_next, int d, __nv_bfloat16 *Xb,
+                                                         size_t lo_off, float *ss_out, int ss_ld) {
+    DBT_TL_DECL;
+    pdl_enter();
+    DBT_TL_WAITED;
+    __shared__ float scratch[32];
+    int b = blockIdx.x, i = blockIdx.y * blockDim.x + threadIdx.x;
+    float q1 = 0.f, q2 = 0.f;
+    if (i < d) {
+        float gn = g_next ? g_next[i] : 1.f;
+        size_t o1 = (size_t)b * d + i, o2 = (size_t)(Bc + b) * d + i;
+        float m1 = sum_splits(P, split_stride, nsplit, o1);
+        float s1 = S[o1] + m1;
+        S[o1] = s1;
+        store_split(Xb, o1, lo_off, gn * s1);
+        q1 = s1 * s1;
+        if (grouped) {
+            float m2 = sum_splits(P, split_stride, nsplit, o2);
+            if (mode == 2) m2 += coup_c[i] * m1;
+            float s2 = S[o2] + m2;
+            S[o2] = s2;
+            store_split(Xb, o2, lo_off, gn * s2);
+            q2 = s2 * s2;
+        }
+    }
+    q1 = block_sum(q1, scratch);
+    if (grouped) q2 = block_sum(q2, scratch);
+    if (threadIdx.x == 0) {
+        ss_out[(size_t)blockIdx.y * ss_ld + b] = q1;
+        if (grouped) ss_out[(size_t)blockIdx.y * ss_ld + Bc + b] = q2;
+    }
+    DBT_TL_END("resid_wide");
+}
+
 // Residual update + RMSNorm feeding the next GEMM.
 //   mode 0: S unchanged                                   (after the embedding, after an MoE layer)
 //   mode 1: S += sum_s P[s]                               (S-bar_i = S_i + Attn_i W_O)
@@ -32,7 +82,9 @@ __global__ void __launch_bounds__(1024) resid_norm_kernel(float *S, const float 
                                                          const float *__restrict__ g, float eps, int d, int apply_norm,
                                                          int src_mul, int src_add, __nv_bfloat16 *Xb,
                                                          size_t lo_off, float *Xf) {
+    DBT_TL_DECL;
     pdl_enter();
+    DBT_TL_WAITED;
     __shared__ float scratch[32];
     int j = blockIdx.x, n_out = gridDim.x;
     int r1 = j * src_mul + src_add, r2 = Bc + r1;
@@ -77,6 +129,7 @@ __global__ void __launch_bounds__(1024) resid_norm_kernel(float *S, const float 
             if (Xf) Xf[(size_t)(n_out + j) * d + i] = x2;
         }
     }
+    DBT_TL_END("resid_norm");
 }
 
 // After the Q|K|V GEMM: sum the splits, RoPE on Q (both paths) and K (primary), the a coupling
@@ -88,8 +141,11 @@ __global__ void __launch_bounds__(64) qkv_epilogue_kernel(
     const float *P, int nsplit, size_t split_stride, float *Q, RowMap rm, int grouped,
     int n_q, int n_kv, int dh, const float *__restrict__ coup_a, const float2 *__restrict__ rope_tab,
     const int32_t *seq_len, const int32_t *__restrict__ page_table, int pt_stride, int num_pages,
-    int page_size, KT *kpool, KT *vpool, int *status) {
+    int page_size, KT *kpool, KT *vpool, int *status, const float *ss, int ss_tiles, int ss_ld, int d_norm,
+    float eps) {
+    DBT_TL_DECL;
     pdl_enter();
+    DBT_TL_WAITED;
     int item = blockIdx.x, hh = blockIdx.y, i = threadIdx.x, Bc = rm.Bc();
     int half = dh / 2;
     if (i >= half) return;
@@ -97,19 +153,22 @@ __global__ void __launch_bounds__(64) qkv_epilogue_kernel(
     int q_dim = n_q * dh, kv_dim = n_kv * dh, ldp = q_dim + 2 * kv_dim;
     float2 t = rope_tab[(size_t)pos * half + i];
     size_t p1 = (size_t)item * ldp, p2 = (size_t)(Bc + item) * ldp;
+    const float rs1 = row_scale(ss, ss_tiles, ss_ld, item, d_norm, eps);  // 1/rms when the GEMM input was g*S
     if (hh < n_q) {
         int o0 = hh * dh + i, o1 = o0 + half;
-        float x0 = sum_splits(P, split_stride, nsplit, p1 + o0), x1 = sum_splits(P, split_stride, nsplit, p1 + o1);
+        float x0 = rs1 * sum_splits(P, split_stride, nsplit, p1 + o0), x1 = rs1 * sum_splits(P, split_stride, nsplit, p1 + o1);
         float r0 = x0 * t.x - x1 * t.y, r1 = x1 * t.x + x0 * t.y;
         float *q1 = Q + (size_t)item * q_dim;
         q1[o0] = r0;
         q1[o1] = r1;
         if (grouped) {
-            float y0 = sum_splits(P, split_stride, nsplit, p2 + o0), y1 = sum_splits(P, split_stride, nsplit, p2 + o1);
+            const float rs2 = row_scale(ss, ss_tiles, ss_ld, Bc + item, d_norm, eps);
+            float y0 = rs2 * sum_splits(P, split_stride, nsplit, p2 + o0), y1 = rs2 * sum_splits(P, split_stride, nsplit, p2 + o1);
             float *q2 = Q + (size_t)(Bc + item) * q_dim;
             q2[o0] = (y0 * t.x - y1 * t.y) + coup_a[o0] * r0;
             q2[o1] = (y1 * t.x + y0 * t.y) + coup_a[o1] * r1;
         }
+        DBT_TL_END("qkv_epilogue");
         return;
     }
     int gk = hh - n_q;
@@ -121,11 +180,11 @@ __global__ void __launch_bounds__(64) qkv_epilogue_kernel(
     int slot = pos % page_size;
     size_t base = (((size_t)page * n_kv + gk) * page_size + slot) * dh;
     size_t ko = p1 + q_dim + gk * dh + i, vo = ko + kv_dim;
-    float x0 = sum_splits(P, split_stride, nsplit, ko), x1 = sum_splits(P, split_stride, nsplit, ko + half);
+    float x0 = rs1 * sum_splits(P, split_stride, nsplit, ko), x1 = rs1 * sum_splits(P, split_stride, nsplit, ko + half);
     store1(kpool + base + i, x0 * t.x - x1 * t.y);
     store1(kpool + base + i + half, x1 * t.x + x0 * t.y);
-    store1(vpool + base + i, sum_splits(P, split_stride, nsplit, vo));
-    store1(vpool + base + i + half, sum_splits(P, split_stride, nsplit, vo + half));
+    store1(vpool + base + i, rs1 * sum_splits(P, split_stride, nsplit, vo));
+    store1(vpool + base + i + half, rs1 * sum_splits(P, split_stride, nsplit, vo + half));
 }
 
 // After the gate|up GEMM: H = SiLU(gate) * up; H~_2 = H_2 + b * H_1 (Eq. mlp); bf16 out for
@@ -133,19 +192,25 @@ __global__ void __launch_bounds__(64) qkv_epilogue_kernel(
 __global__ void __launch_bounds__(256) swiglu_couple_kernel(const float *P, int nsplit,
                                                             size_t split_stride, int F, int Bc, int grouped,
                                                             const float *__restrict__ coup_b,
-                                                            __nv_bfloat16 *Hb, size_t lo_off) {
+                                                            __nv_bfloat16 *Hb, size_t lo_off, const float *ss,
+                                                            int ss_tiles, int ss_ld, int d_norm, float eps) {
+    DBT_TL_DECL;
     pdl_enter();
+    DBT_TL_WAITED;
     int b = blockIdx.x, f = blockIdx.y * blockDim.x + threadIdx.x;
     if (f >= F) return;
     size_t p1 = (size_t)b * 2 * F + f;
-    float h1 = silu(sum_splits(P, split_stride, nsplit, p1)) * sum_splits(P, split_stride, nsplit, p1 + F);
+    const float rs1 = row_scale(ss, ss_tiles, ss_ld, b, d_norm, eps);
+    float h1 = silu(rs1 * sum_splits(P, split_stride, nsplit, p1)) * (rs1 * sum_splits(P, split_stride, nsplit, p1 + F));
     store_split(Hb, (size_t)b * F + f, lo_off, h1);
     if (grouped) {
         size_t p2 = (size_t)(Bc + b) * 2 * F + f;
-        float h2 = silu(sum_splits(P, split_stride, nsplit, p2)) * sum_splits(P, split_stride, nsplit, p2 + F);
+        const float rs2 = row_scale(ss, ss_tiles, ss_ld, Bc + b, d_norm, eps);
+        float h2 = silu(rs2 * sum_splits(P, split_stride, nsplit, p2)) * (rs2 * sum_splits(P, split_stride, nsplit, p2 + F));
         if (coup_b) h2 += coup_b[f] * h1;
         store_split(Hb, (size_t)(Bc + b) * F + f, lo_off, h2);
     }
+    DBT_TL_END("swiglu");
 }
 
 // Eq. embeddings for the fused path: S^0 = RMSNorm(E[x]) and, for the first layer's Q|K|V GEMM,

@@ -169,6 +169,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
     auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
     uint32_t accum_bar = bars + 8u * (2 * STAGES);
 
+    DBT_TL_DECL;
     int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     int tile = blockIdx.x, split = blockIdx.y;
     int x_row0 = 0, w_row0 = 0, grp_n = -1;
@@ -262,6 +263,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
 
     // ---- epilogue: TMEM lane = weight row (feature), TMEM column = activation row
     pdl_wait();
+    DBT_TL_WAITED;
     bool got = mbar_wait(accum_bar, 0);
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (!got && lane == 0) report(p.status, kStatusWaitExpired, 200 + warp);
@@ -321,6 +323,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
                      "r"((uint32_t)Cfg::kTmemCols)
                      : "memory");
+    DBT_TL_END("gemm");
 }
 
 // ---- host side: tensor maps -------------------------------------------------------------

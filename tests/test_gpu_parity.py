@@ -307,10 +307,12 @@ def test_fresh_models_give_bitwise_identical_results():
             assert torch.equal(x["z1"], y["z1"]) and torch.equal(x["z2"], y["z2"])
 
 
-def test_fused_epilogue_path_matches_oracle(monkeypatch):
-    """The opt-in variant that folds the elementwise work into the GEMM epilogues (last-arriving
-    CTA per output tile) computes the same step."""
-    monkeypatch.setenv("DBT_FUSED", "1")
+@pytest.mark.parametrize("knob", ["DBT_FUSED", "DBT_WIDE"])
+def test_opt_in_kernel_chains_match_oracle(monkeypatch, knob):
+    """The two opt-in variants of the dense chain -- elementwise work folded into the GEMM
+    epilogues (last-arriving CTA per output tile), and the RMSNorm factor applied after the GEMM
+    (no row-wide reduction kernel) -- compute the same step."""
+    monkeypatch.setenv(knob, "1")
     cfg = small_bf16()
     w = make_weights(cfg, seed=5, matrix_std=0.05)
     tok = make_tokens(cfg, 3, 40, seed=6)
