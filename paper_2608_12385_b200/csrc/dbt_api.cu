@@ -17,6 +17,7 @@
 #include "dbt_fused.cuh"
 #include "dbt_gemm_tc.cuh"
 #include "dbt_kernels.cuh"
+#include "dbt_mega.cuh"
 
 using namespace dbt;
 
@@ -41,7 +42,13 @@ struct Workspace {
     float *Pe;
     int32_t *epos, *eoff;
     size_t P_floats;
+    // single-kernel decode step: plans (one per batch size and mode), descriptor array, counters
+    char *mega_plans;
+    CUtensorMap *mega_maps;
+    unsigned int *mega_sync;  // [0] barrier arrivals, [1] CTAs done, [2] error flag
+    float *rd_part, *rd_best;
 };
+constexpr int kMegaPlanSlots = 16;
 
 struct LayerMaps {
     CUtensorMap wq, wk, wv, wo, wg, wu, wd;  // dense MLP; for MoE wg/wu/wd hold the shared expert
@@ -78,6 +85,9 @@ struct dbt_model {
     bool att_fast;  // TMA + mma.sync attention over the bf16 pool
     bool fused;     // dense bf16: elementwise work fused into the GEMM epilogues
     bool wide;      // dense bf16: RMSNorm factor applied after the GEMM, no row-wide reduction kernel
+    bool mega;      // dense bf16, small batch: the whole decode step as one persistent kernel
+    struct MegaSlot { int B, grouped; };
+    std::vector<MegaSlot> mega_slots;
     int num_sms;
     int act_parts;  // 2: GEMM inputs carried as hi + lo bf16 terms; 1: plain bf16
     // a decode step is captured once per (batch, mode, buffer set) and replayed as a CUDA graph
@@ -200,6 +210,13 @@ size_t carve(const dbt_config &c, char *base, Workspace *ws, int *Rmax_out, int 
         if (w.P_floats < (size_t)Rmax * widest) w.P_floats = (size_t)Rmax * widest;
         w.P = k.take<float>(w.P_floats);
         w.ss = k.take<float>((size_t)((d + 127) / 128) * Rmax);
+        if (!moe) {
+            w.mega_plans = k.take<char>((size_t)kMegaPlanSlots * align_up(sizeof(MegaPlan)));
+            w.mega_maps = k.take<CUtensorMap>((size_t)c.n_layers * 7 + 5);
+            w.mega_sync = k.take<unsigned int>(8);
+            w.rd_part = k.take<float>((size_t)kMegaMaxCtas * 64 * 4);
+            w.rd_best = k.take<float>((size_t)kMegaMaxCtas * 64 * 2);
+        }
         if (moe) {
             size_t Rk = (size_t)Rmax * kmax_of(c);
             w.Xs = k.take<__nv_bfloat16>(2 * Rk * d);
@@ -1112,6 +1129,169 @@ dbt_status prefill_wide(dbt_model *m, const int32_t *tokens_dev, int B, int n, f
     return DBT_OK;
 }
 
+
+// ---- dense bf16, small batch: the whole decode step as one persistent kernel -------------------
+
+template <int N_TILE, int DH>
+bool mega_allow() {
+    if (cudaFuncSetAttribute(mega_decode_kernel<N_TILE, DH>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             MegaCfg<N_TILE, DH>::kSmemBytes) != cudaSuccess)
+        return false;
+    int per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, mega_decode_kernel<N_TILE, DH>, kMegaThreads,
+                                                      MegaCfg<N_TILE, DH>::kSmemBytes) != cudaSuccess)
+        return false;
+    return per_sm >= 1;
+}
+
+bool mega_eligible(const dbt_model *m, int B) {
+    if (!m->mega) return false;
+    const dbt_config &c = m->cfg;
+    int n_tile = pad_rows(2 * B);
+    if (n_tile > 64 || B > 32) return false;
+    int vt = (c.vocab + 127) / 128, ft = 2 * ((c.d_ff + 127) / 128);
+    int qt = (c.n_q_heads * c.head_dim + 127) / 128 + 2 * ((c.n_kv_heads * c.head_dim + 127) / 128);
+    int tiles = vt > ft ? vt : ft;
+    if (qt > tiles) tiles = qt;
+    if ((size_t)(m->num_sms + tiles) * n_tile * 128 > m->ws.P_floats) return false;
+    if (m->num_sms + B * c.n_kv_heads > m->part_items) return false;
+    return true;
+}
+
+// The plan of a (batch, mode) pair lives in device memory; it is written once, outside any capture.
+dbt_status mega_prepare(dbt_model *m, int B, int grouped, int *slot_out) {
+    for (size_t i = 0; i < m->mega_slots.size(); i++)
+        if (m->mega_slots[i].B == B && m->mega_slots[i].grouped == grouped) {
+            *slot_out = (int)i;
+            return DBT_OK;
+        }
+    if ((int)m->mega_slots.size() >= kMegaPlanSlots) {
+        *slot_out = -1;
+        return DBT_OK;
+    }
+    const dbt_config &c = m->cfg;
+    const Workspace &w = m->ws;
+    MegaPlan p;
+    memset(&p, 0, sizeof p);
+    int d = c.d_model, qd = c.n_q_heads * c.head_dim;
+    p.B = B; p.grouped = grouped; p.R = grouped ? 2 * B : B; p.L = c.n_layers; p.d = d; p.n_q = c.n_q_heads;
+    p.n_kv = c.n_kv_heads; p.dh = c.head_dim; p.F = c.d_ff; p.V = c.vocab; p.Rmax = m->Rmax; p.final_norm = c.final_norm;
+    p.num_pages = c.num_pages; p.pt_stride = m->pages_per_seq_max; p.eps = c.rms_eps;
+    p.S = w.S; p.Q = w.Q; p.P = w.P; p.ss = w.ss; p.Z = w.Z; p.part = w.part; p.rd_part = w.rd_part; p.rd_best = w.rd_best;
+    p.Xb = w.Xb; p.Ob = w.Ob; p.Hb = w.Hb; p.pool = reinterpret_cast<__nv_bfloat16 *>(m->kv_pool);
+    p.lo_x = (size_t)m->Rmax * d; p.lo_o = (size_t)m->Rmax * qd; p.lo_h = (size_t)m->Rmax * c.d_ff;
+    p.rope = w.rope; p.seq_len = w.seq_len; p.page_table = w.page_table; p.att_tickets = w.att_tickets; p.status = w.status;
+    p.bar_count = w.mega_sync; p.done_count = w.mega_sync + 1; p.err = reinterpret_cast<int *>(w.mega_sync + 2);
+    p.maps = w.mega_maps;
+    p.E1 = (const __nv_bfloat16 *)m->w.embed_primary; p.E2 = (const __nv_bfloat16 *)m->w.embed_branch;
+    p.g_e = m->w.embed_norm_g; p.g_first = m->layers[0].attn_norm_g;
+    p.plane_rows = (long long)c.num_pages * c.n_kv_heads * c.page_size;
+    for (int l = 0; l < c.n_layers; l++) {
+        const dbt_layer_weights &lw = m->layers[l];
+        p.layer[l].coup_a = lw.coup_a; p.layer[l].coup_b = lw.coup_b; p.layer[l].coup_c = lw.coup_c;
+        p.layer[l].g_mlp = lw.mlp_norm_g;
+        p.layer[l].g_next = l + 1 < c.n_layers ? m->layers[l + 1].attn_norm_g
+                                               : (c.final_norm ? m->w.final_norm_g : (const float *)nullptr);
+    }
+    int slot = (int)m->mega_slots.size();
+    CUDA_TRY(m, cudaMemcpy(w.mega_plans + (size_t)slot * align_up(sizeof(MegaPlan)), &p, sizeof p, cudaMemcpyHostToDevice));
+    m->mega_slots.push_back(dbt_model::MegaSlot{B, grouped});
+    *slot_out = slot;
+    return DBT_OK;
+}
+
+template <int N_TILE, int DH>
+cudaError_t mega_launch(dbt_model *m, const MegaPlan *plan, const int32_t *tokens, int32_t *next, float *alpha) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(m->num_sms);
+    cfg.blockDim = dim3(kMegaThreads);
+    cfg.dynamicSmemBytes = MegaCfg<N_TILE, DH>::kSmemBytes;
+    cfg.stream = m->stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;  // all CTAs resident at once: they meet at grid barriers
+    attr[0].val.cooperative = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, mega_decode_kernel<N_TILE, DH>, plan, tokens, next, alpha);
+}
+
+dbt_status step_mega(dbt_model *m, int slot, const int32_t *tokens_dev, int B, int grouped, int32_t *next_dev,
+                     float *z1_dev, float *z2_dev, float *alpha_dev) {
+    const dbt_config &c = m->cfg;
+    const Workspace &w = m->ws;
+    const MegaPlan *plan = reinterpret_cast<const MegaPlan *>(w.mega_plans + (size_t)slot * align_up(sizeof(MegaPlan)));
+    int n_tile = pad_rows(2 * B);
+    double bytes = 0;
+    if (m->prof_on) {
+        int qd = c.n_q_heads * c.head_dim, kvd = c.n_kv_heads * c.head_dim;
+        bytes = ((double)c.n_layers * ((double)(qd + 2 * kvd) * c.d_model + (double)c.d_model * qd + 3.0 * c.d_ff * c.d_model) +
+                 (double)c.vocab * c.d_model) * 2;
+        for (int b = 0; b < B; b++) bytes += (double)(m->len_host[b] + 1) * 2 * kvd * 2 * c.n_layers;
+    }
+    cudaEvent_t p0 = nullptr, p1 = nullptr;
+    if (m->prof_on) {
+        p0 = prof_event(m);
+        p1 = prof_event(m);
+        cudaEventRecord(p0, m->stream);
+    }
+    cudaError_t e = cudaErrorInvalidValue;
+    if (c.head_dim == 128) {
+        if (n_tile == 16) e = mega_launch<16, 128>(m, plan, tokens_dev, next_dev, alpha_dev);
+        else if (n_tile == 32) e = mega_launch<32, 128>(m, plan, tokens_dev, next_dev, alpha_dev);
+        else e = mega_launch<64, 128>(m, plan, tokens_dev, next_dev, alpha_dev);
+    } else {
+        if (n_tile == 16) e = mega_launch<16, 64>(m, plan, tokens_dev, next_dev, alpha_dev);
+        else if (n_tile == 32) e = mega_launch<32, 64>(m, plan, tokens_dev, next_dev, alpha_dev);
+        else e = mega_launch<64, 64>(m, plan, tokens_dev, next_dev, alpha_dev);
+    }
+    m->launches++;
+    if (m->prof_on) {
+        cudaEventRecord(p1, m->stream);
+        m->prof.push_back(dbt_model::ProfRec{"mega_decode_step", bytes, p0, p1});
+    }
+    if (e != cudaSuccess) return fail(m, DBT_ERR_CUDA, "launch mega_decode_kernel: %s", cudaGetErrorString(e));
+    size_t zb = sizeof(float) * (size_t)B * c.vocab;
+    if (z1_dev) CUDA_TRY(m, cudaMemcpyAsync(z1_dev, w.Z, zb, cudaMemcpyDeviceToDevice, m->stream));
+    if (z2_dev && grouped)
+        CUDA_TRY(m, cudaMemcpyAsync(z2_dev, w.Z + (size_t)B * c.vocab, zb, cudaMemcpyDeviceToDevice, m->stream));
+    for (int b = 0; b < B; b++) m->len_host[b] += 1;
+    return DBT_OK;
+}
+
+bool setup_mega(dbt_model *m) {
+    const dbt_config &c = m->cfg;
+    const char *mg = getenv("DBT_MEGA");
+    if (!(mg && strcmp(mg, "1") == 0)) return false;
+    if (!m->tc || !m->att_fast || c.n_experts > 0 || m->act_parts != 2 || c.n_layers > kMegaMaxLayers) return false;
+    if (c.head_dim != 64 && c.head_dim != 128) return false;
+    if (c.page_size != 16 || m->num_sms > kMegaMaxCtas) return false;
+    int dev = 0, coop = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return false;
+    cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
+    if (!coop) return false;
+    bool ok = c.head_dim == 128 ? (mega_allow<16, 128>() && mega_allow<32, 128>() && mega_allow<64, 128>())
+                                : (mega_allow<16, 64>() && mega_allow<32, 64>() && mega_allow<64, 64>());
+    if (!ok) {
+        cudaGetLastError();
+        return false;
+    }
+    const Workspace &w = m->ws;
+    std::vector<CUtensorMap> maps((size_t)c.n_layers * 7 + 5);
+    for (int l = 0; l < c.n_layers; l++) {
+        const LayerMaps &mp = m->maps[l];
+        CUtensorMap *o = maps.data() + (size_t)l * 7;
+        o[0] = mp.wq; o[1] = mp.wk; o[2] = mp.wv; o[3] = mp.wo; o[4] = mp.wg; o[5] = mp.wu; o[6] = mp.wd;
+    }
+    CUtensorMap *t = maps.data() + (size_t)c.n_layers * 7;
+    t[0] = m->map_lm; t[1] = m->map_Xb; t[2] = m->map_Ob; t[3] = m->map_Hb; t[4] = m->map_kv;
+    if (cudaMemcpy(w.mega_maps, maps.data(), maps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice) != cudaSuccess ||
+        cudaMemset(w.mega_sync, 0, sizeof(unsigned int) * 8) != cudaSuccess) {
+        cudaGetLastError();
+        return false;
+    }
+    return true;
+}
+
 template <int N_TILE>
 bool allow_smem() {
     return cudaFuncSetAttribute(gemm_tc_kernel<N_TILE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -1328,6 +1508,8 @@ dbt_status dbt_create(const dbt_config *cfg, const dbt_weights *w, void *kv_pool
         m->num_sms = sms > 0 && sms <= 148 ? sms : 148;  // the partial buffer is sized for 2 x 148 CTAs
     }
     m->tc = setup_tc(m);
+    m->mega = false;
+    m->mega = setup_mega(m);
     const char *pd = getenv("DBT_PDL");
     m->use_pdl = !(pd && strcmp(pd, "0") == 0);
     const char *po = getenv("DBT_PDL_OFF");
@@ -1481,6 +1663,7 @@ dbt_status dbt_reset(dbt_model *m) {
     CUDA_TRY(m, cudaMemsetAsync(m->ws.status, 0, sizeof(int32_t) * 4, m->stream));
     CUDA_TRY(m, cudaMemsetAsync(m->ws.att_tickets, 0, sizeof(int32_t) * (size_t)m->Rmax * m->cfg.n_kv_heads, m->stream));
     CUDA_TRY(m, cudaMemsetAsync(m->ws.gemm_tickets, 0, sizeof(int32_t) * 4096, m->stream));
+    if (m->ws.mega_sync) CUDA_TRY(m, cudaMemsetAsync(m->ws.mega_sync, 0, sizeof(unsigned int) * 8, m->stream));
     std::fill(m->len_host.begin(), m->len_host.end(), 0);
     return DBT_OK;
 }
@@ -1516,6 +1699,12 @@ dbt_status dbt_prefill(dbt_model *m, const int32_t *tokens_dev, int32_t B, int32
 static dbt_status step_direct(dbt_model *m, const int32_t *tokens_dev, int B, int grouped, int32_t *next_dev,
                               float *z1, float *z2, float *alpha) {
     if (m->cfg.weight_dtype == DBT_DTYPE_F32) return step_impl<float>(m, tokens_dev, B, grouped, next_dev, z1, z2, alpha);
+    if (mega_eligible(m, B)) {
+        int slot = -1;
+        dbt_status st = mega_prepare(m, B, grouped, &slot);
+        if (st != DBT_OK) return st;
+        if (slot >= 0) return step_mega(m, slot, tokens_dev, B, grouped, next_dev, z1, z2, alpha);
+    }
     if (m->fused) return step_fused(m, tokens_dev, B, grouped, next_dev, z1, z2, alpha);
     if (m->wide) return step_wide(m, tokens_dev, B, grouped, next_dev, z1, z2, alpha);
     if (m->tc) return step_tc(m, tokens_dev, B, grouped, next_dev, z1, z2, alpha);
@@ -1534,6 +1723,11 @@ static dbt_status step_graphed(dbt_model *m, const int32_t *tokens_dev, int B, i
     if (!hit) {
         if (m->graphs.size() >= 64) {  // a caller that never reuses buffers: stop caching
             return step_direct(m, tokens_dev, B, grouped, next_dev, z1, z2, alpha);
+        }
+        if (mega_eligible(m, B)) {  // the plan upload must not fall inside the capture
+            int slot = -1;
+            dbt_status pst = mega_prepare(m, B, grouped, &slot);
+            if (pst != DBT_OK) return pst;
         }
         std::vector<int32_t> len_save = m->len_host;
         int64_t l0 = m->launches;

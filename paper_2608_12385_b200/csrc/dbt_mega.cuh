@@ -1,0 +1,946 @@
+// The whole grouped decode step of a dense bf16 model as ONE persistent kernel (sm_100a).
+//
+// Why: run as separate kernels, a layer is ten launches of a few microseconds each, and the
+// dependency latency between them (grid drain, flush, wake-up of the next grid) costs more
+// than the kernels themselves at small batch.  Here one CTA per SM stays resident for the
+// whole step; the phases of a layer are separated by grid barriers (an arrival counter in
+// global memory, every wait bounded), and a single producer warp per CTA streams, through one
+// shared-memory ring, everything the step reads from HBM in program order: the weight tiles
+// of the Q|K|V GEMM, the K/V pages of the attention, the weight tiles of the O, gate|up and
+// down GEMMs, the next layer's..., and finally the output matrix.  Weight tiles do not depend
+// on activations, so the producer runs ahead of the barriers and the ring is full when a GEMM
+// phase begins; only the (small, L2-resident) activation tiles wait for the barrier.
+//
+// Roles (192 threads): warp 0 = producer (TMA), warp 1 = tcgen05 MMA issuer and TMEM owner,
+// warps 2..5 = workers (GEMM epilogues out of tensor memory, the elementwise phases, the
+// attention math with mma.sync).
+//
+// GEMM phases are split "stream-K": all (tile, k-tile) units of a GEMM are laid end to end
+// and CTA c takes units [c*q, (c+1)*q): every SM streams the same number of weight bytes
+// whatever the shape.  A CTA's run of units inside one 128-feature tile is a segment; its
+// partial tile goes to slot c + tile, and the elementwise phase after the barrier adds a
+// tile's segments in CTA order (deterministic, and identical for grouped and primary-only
+// steps because q depends on the shape only).  RMSNorm is split around the GEMMs: the gain
+// is folded into the GEMM input, sum(S^2) is kept as per-block shares, and the phase after
+// the GEMM multiplies by 1/rms.
+//
+// Phases per layer (Section 4.1, Eq. asymattn, Eq. mlp):
+//   G1 Q|K|V  | E1 1/rms, RoPE, Q~_2 = Q_2 + a*Q_1, append K_1,V_1 | A attention (both paths'
+//   queries on one pass over the pages) | G2 O | E2 S-bar = S + ., next input | G3 gate|up |
+//   E3 SiLU*up, H~_2 = H_2 + b*H_1 | G4 down | E4 M_2 += c*M_1, S += M, next input
+// then the output matrix and the readout (Eq. alpha, Eq. mixloss) spread over all CTAs.
+#pragma once
+
+#include "dbt_attn_mma.cuh"
+#include "dbt_fused.cuh"
+#include "dbt_kernels.cuh"
+
+namespace dbt {
+
+constexpr int kMegaMaxLayers = 128;
+constexpr int kMegaSlots = 6;
+constexpr int kMegaSlotBytes = 32768;
+constexpr int kMegaThreads = 192;
+constexpr int kMegaMaxCtas = 160;
+constexpr unsigned long long kMegaWaitCycles = 4000000000ull;
+
+struct MegaLayer {
+    const float *coup_a, *coup_b, *coup_c, *g_mlp, *g_next;  // g_next: gain folded into the input after this layer
+};
+
+struct MegaPlan {
+    int B, grouped, R, L, d, n_q, n_kv, dh, F, V, Rmax, final_norm;
+    int num_pages, pt_stride;
+    float eps;
+    float *S, *Q, *P, *ss, *Z, *part, *rd_part, *rd_best;
+    __nv_bfloat16 *Xb, *Ob, *Hb, *pool;
+    size_t lo_x, lo_o, lo_h;  // element offset of the lo plane of each GEMM input
+    const float2 *rope;
+    int32_t *seq_len;
+    const int32_t *page_table;
+    int *att_tickets, *status;
+    unsigned int *bar_count, *done_count;
+    int *err;
+    const CUtensorMap *maps;  // per layer wq wk wv wo wg wu wd; then lm_head, Xb, Ob, Hb, kv pool
+    const __nv_bfloat16 *E1, *E2;
+    const float *g_e, *g_first;
+    long long plane_rows;  // rows of one K (or V) plane of one layer in the pool's 2-D view
+    MegaLayer layer[kMegaMaxLayers];
+};
+
+template <int N_TILE, int DH>
+struct MegaCfg {
+    static constexpr int kBBytes = N_TILE * kTcK * 2;
+    static constexpr int kScratchFloats = 16 * DH + 1024;
+    static constexpr int kSmemBytes = kMegaSlots * kMegaSlotBytes + 1024 + 256 + kScratchFloats * 4;
+    static_assert(kTcABytes + 2 * kBBytes <= kMegaSlotBytes, "GEMM stage must fit a ring slot");
+    static_assert(2 * 4 * 16 * DH * 2 <= kMegaSlotBytes, "attention stage must fit a ring slot");
+};
+
+__device__ __forceinline__ unsigned ld_acquire_u32(const unsigned *p) {
+    unsigned v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+template <int N_TILE, int DH>
+__global__ void __launch_bounds__(kMegaThreads, 1)
+mega_decode_kernel(const MegaPlan *__restrict__ pl, const int32_t *tokens, int32_t *next, float *alpha_out) {
+    using Cfg = MegaCfg<N_TILE, DH>;
+    constexpr int SLOTS = kMegaSlots, HALVES = DH / 64, KS = DH / 16, NB = DH / 8;
+    constexpr int PAGE_BYTES = 16 * DH * 2;
+    constexpr int SLOT_FLOATS = N_TILE * 128;  // one partial tile [N_TILE rows][128 features]
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t ring = (raw + 1023u) & ~1023u;
+    uint8_t *gen_ring = smem_raw + (ring - raw);
+    const uint32_t bars = ring + SLOTS * kMegaSlotBytes;
+    auto full_bar = [&](int s) { return bars + 8u * s; };
+    auto empty_bar = [&](int s) { return bars + 8u * (SLOTS + s); };
+    auto accf_bar = [&](int b) { return bars + 8u * (2 * SLOTS + b); };
+    auto acce_bar = [&](int b) { return bars + 8u * (2 * SLOTS + 2 + b); };
+    uint32_t *tmem_holder = reinterpret_cast<uint32_t *>(gen_ring + SLOTS * kMegaSlotBytes + 192);
+    volatile unsigned *gen_s = reinterpret_cast<volatile unsigned *>(gen_ring + SLOTS * kMegaSlotBytes + 200);
+    volatile int *abort_s = reinterpret_cast<volatile int *>(gen_ring + SLOTS * kMegaSlotBytes + 204);
+    float *sc_o = reinterpret_cast<float *>(gen_ring + SLOTS * kMegaSlotBytes + 256);  // [16][DH]
+    float *sc_m = sc_o + 16 * DH, *sc_l = sc_m + 16;
+    int *flag = reinterpret_cast<int *>(sc_l + 16);
+    int *cum = flag + 8, *nk_s = cum + kAttMaxItems + 1;
+    float *red = reinterpret_cast<float *>(nk_s + kAttMaxItems);  // [64] worker reductions
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const bool is_prod = warp == 0, is_mma = warp == 1, is_worker = warp >= 2;
+    const int wt = tid - 64, ww = warp - 2;  // worker thread / warp index
+    const int C = gridDim.x, cta = blockIdx.x;
+    const int B = pl->B, grouped = pl->grouped, R = pl->R, d = pl->d, dh = DH, n_q = pl->n_q, n_kv = pl->n_kv;
+    const int F = pl->F, V = pl->V, qd = n_q * dh, kvd = n_kv * dh, G = n_q / n_kv, half = dh / 2;
+    const int ss_tiles = (d + 255) / 256, ss_ld = pl->Rmax;
+    const float eps = pl->eps;
+    const CUtensorMap *maps = pl->maps;
+    const CUtensorMap *map_tail = maps + (size_t)pl->L * 7;
+
+    if (tid == 0) {
+        for (int s = 0; s < SLOTS; s++) {
+            mbar_init(full_bar(s), 1);
+            mbar_init(empty_bar(s), 4);
+        }
+        for (int b = 0; b < 2; b++) {
+            mbar_init(accf_bar(b), 1);
+            mbar_init(acce_bar(b), 4);
+        }
+        *gen_s = 0;
+        *abort_s = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (is_mma) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_holder)),
+                     "r"((uint32_t)(2 * N_TILE < 32 ? 32 : 2 * N_TILE))
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = *tmem_holder;
+
+    // ---- shared bookkeeping: every role walks the same schedule and keeps the same counters
+    unsigned k_bar = 0;  // grid barriers in program order
+    int it = 0;          // ring slots in program order
+    int seg_it = 0;      // GEMM segments (TMEM buffers) in program order
+    bool ok = true;
+
+    auto fail_here = [&](int site) {
+        ok = false;
+        *abort_s = 1;
+        atomicExch(pl->err, 1);
+        report(pl->status, kStatusWaitExpired, site);
+    };
+    // bounded waits that also give up as soon as any role of any CTA has failed
+    auto wait_bar = [&](uint32_t bar, uint32_t parity, int site) {
+        if (!ok) return;
+        uint32_t done = 0;
+        long long t0 = clock64();
+        unsigned spins = 0;
+        while (true) {
+            asm volatile(
+                "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
+                : "=r"(done)
+                : "r"(bar), "r"(parity)
+                : "memory");
+            if (done) return;
+            if ((++spins & 1023u) == 0) {
+                if (*abort_s || (unsigned long long)(clock64() - t0) > kMegaWaitCycles) {
+                    fail_here(site);
+                    return;
+                }
+            }
+        }
+    };
+    auto worker_sync = [&]() { consumer_sync(); };
+    // Grid barrier.  Workers arrive and wait; the other roles only count it.
+    auto grid_barrier = [&]() {
+        k_bar++;
+        if (!is_worker) return;
+        asm volatile("fence.proxy.async;" ::: "memory");  // this phase's stores are read by other SMs' TMA next
+        worker_sync();
+        if (wt == 0) {
+            __threadfence();
+            atomicAdd(pl->bar_count, 1u);
+            const unsigned target = k_bar * (unsigned)C;
+            long long t0 = clock64();
+            unsigned spins = 0;
+            while (ok && ld_acquire_u32(pl->bar_count) < target) {
+                if ((++spins & 255u) == 0) {
+                    if (*abort_s || *(volatile int *)pl->err || (unsigned long long)(clock64() - t0) > kMegaWaitCycles)
+                        fail_here(900 + (int)(k_bar & 63));
+                }
+            }
+            *gen_s = k_bar;
+        }
+        worker_sync();
+        __threadfence();
+        if (*abort_s) ok = false;
+    };
+    // the producer learns from its own CTA's workers that barrier k has been passed
+    auto wait_gen = [&](unsigned k, int site) {
+        if (!ok) return;
+        long long t0 = clock64();
+        unsigned spins = 0;
+        while (*gen_s < k) {
+            if ((++spins & 255u) == 0) {
+                if (*abort_s || (unsigned long long)(clock64() - t0) > kMegaWaitCycles) {
+                    fail_here(site);
+                    return;
+                }
+            }
+        }
+        __threadfence();
+        asm volatile("fence.proxy.async;" ::: "memory");  // other SMs' stores, now visible, are read next by TMA
+    };
+    // sum / max over the 128 worker threads (result to all)
+    auto worker_sum = [&](float v) {
+        v = warp_sum(v);
+        worker_sync();
+        if (lane == 0) red[ww] = v;
+        worker_sync();
+        return red[0] + red[1] + red[2] + red[3];
+    };
+
+    // ---- stream-K bookkeeping of one GEMM
+    struct Gemm {
+        const CUtensorMap *w[3];
+        int n_out[3], nseg, K, tiles, KT, U, q, lo_row0;
+        const CUtensorMap *x;
+    };
+    auto make_gemm = [&](const CUtensorMap *w0, int n0, const CUtensorMap *w1, int n1, const CUtensorMap *w2, int n2,
+                         const CUtensorMap *x, int K) {
+        Gemm g;
+        g.w[0] = w0; g.w[1] = w1; g.w[2] = w2;
+        g.n_out[0] = n0; g.n_out[1] = n1; g.n_out[2] = n2;
+        g.nseg = w2 ? 3 : w1 ? 2 : 1;
+        g.K = K;
+        g.tiles = (n0 + 127) / 128 + (w1 ? (n1 + 127) / 128 : 0) + (w2 ? (n2 + 127) / 128 : 0);
+        g.KT = (K + kTcK - 1) / kTcK;
+        g.U = g.tiles * g.KT;
+        g.q = (g.U + C - 1) / C;
+        g.lo_row0 = pl->Rmax;
+        g.x = x;
+        return g;
+    };
+    // sum of a tile's segment partials, in CTA order
+    auto tile_sum = [&](const Gemm &g, int tile, int r, int f) {
+        int first = (tile * g.KT) / g.q, last = ((tile + 1) * g.KT - 1) / g.q;
+        float a = 0.f;
+        for (int c = first; c <= last; c++) a += __ldcg(pl->P + ((size_t)(c + tile) * N_TILE + r) * 128 + f);
+        return a;
+    };
+
+    // ---- one GEMM phase; the activations are ready once grid barrier `gate` has been passed
+    auto gemm_phase = [&](const Gemm &g, unsigned gate) {
+        const int u0 = min(g.U, cta * g.q), u1 = min(g.U, u0 + g.q), nun = u1 - u0;
+        const int nsegs = nun > 0 ? (u1 - 1) / g.KT - u0 / g.KT + 1 : 0;
+        const int it0 = it, seg0 = seg_it;
+        auto seg_of = [&](int tile, int &row0) {
+            int t1 = (g.n_out[0] + 127) / 128, t2 = t1 + (g.nseg > 1 ? (g.n_out[1] + 127) / 128 : 0);
+            int sg = tile < t1 ? 0 : (tile < t2 ? 1 : 2);
+            row0 = (tile - (sg == 0 ? 0 : sg == 1 ? t1 : t2)) * 128;
+            return sg;
+        };
+        if (is_prod) {
+            if (lane == 0) {
+                int pend_s[SLOTS], pend_kt[SLOTS], npend = 0;
+                bool gated = true;
+                const uint32_t tx = kTcABytes + 2 * Cfg::kBBytes;
+                auto load_x = [&](int s, int kt) {
+                    for (int part = 0; part < 2; part++)
+                        for (int j = 0; j < N_TILE / 16; j++)
+                            tma_load_2d(ring + s * kMegaSlotBytes + kTcABytes + part * Cfg::kBBytes + j * 2048, g.x,
+                                        full_bar(s), kt * kTcK, part * g.lo_row0 + j * 16);
+                };
+                for (int u = u0; u < u1 && ok; u++, it++) {
+                    int s = it % SLOTS;
+                    if (it >= SLOTS) wait_bar(empty_bar(s), ((it / SLOTS) - 1) & 1, 400);
+                    if (!ok) break;
+                    int tile = u / g.KT, kt = u % g.KT, row0;
+                    int sg = seg_of(tile, row0);
+                    mbar_expect_tx(full_bar(s), tx);
+                    tma_load_2d(ring + s * kMegaSlotBytes, g.w[sg], full_bar(s), kt * kTcK, row0);
+                    if (gated) {
+                        pend_s[npend] = s;
+                        pend_kt[npend] = kt;
+                        npend++;
+                        if (npend == SLOTS || u == u1 - 1) {
+                            wait_gen(gate, 410);
+                            if (ok)
+                                for (int i = 0; i < npend; i++) load_x(pend_s[i], pend_kt[i]);
+                            gated = false;
+                        }
+                    } else {
+                        load_x(s, kt);
+                    }
+                }
+            }
+        } else if (is_mma) {
+            if (lane == 0) {
+                constexpr uint32_t idesc = umma_idesc(N_TILE);
+                for (int u = u0; u < u1 && ok; u++, it++) {
+                    int s = it % SLOTS, kt = u % g.KT;
+                    int buf = seg_it & 1;
+                    bool first = (u == u0) || kt == 0, last = (u == u1 - 1) || kt == g.KT - 1;
+                    if (first && seg_it >= 2) wait_bar(acce_bar(buf), ((seg_it >> 1) - 1) & 1, 420);
+                    wait_bar(full_bar(s), (it / SLOTS) & 1, 421);
+                    if (!ok) break;
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    uint64_t adesc = umma_smem_desc(ring + s * kMegaSlotBytes);
+                    for (int part = 0; part < 2; part++) {
+                        uint64_t bdesc = umma_smem_desc(ring + s * kMegaSlotBytes + kTcABytes + part * Cfg::kBBytes);
+#pragma unroll
+                        for (int k = 0; k < kTcK / 16; k++)
+                            umma_f16(tmem_base + buf * N_TILE, adesc + 2 * k, bdesc + 2 * k, idesc, !(first && part == 0 && k == 0));
+                    }
+                    // the slot is free when these MMAs have read it: three plain arrivals plus the commit's
+                    for (int a = 0; a < 3; a++)
+                        asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(empty_bar(s)) : "memory");
+                    umma_commit(empty_bar(s));
+                    if (last) {
+                        umma_commit(accf_bar(buf));
+                        seg_it++;
+                    }
+                }
+            }
+        } else {
+            // workers: each finished segment out of tensor memory into its partial slot
+            for (int sgi = 0; sgi < nsegs; sgi++, seg_it++) {
+                int tile = u0 / g.KT + sgi, buf = seg_it & 1;
+                wait_bar(accf_bar(buf), (seg_it >> 1) & 1, 430);
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                if (ok) {
+                    float *out = pl->P + (size_t)(cta + tile) * SLOT_FLOATS + (warp & 3) * 32 + lane;
+#pragma unroll 1
+                    for (int c0 = 0; c0 < N_TILE && c0 < R; c0 += 16) {
+                        float v[16];
+                        tmem_ld16(tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + buf * N_TILE + c0, v);
+#pragma unroll
+                        for (int i = 0; i < 16; i++)
+                            if (c0 + i < R) out[(size_t)(c0 + i) * 128] = v[i];
+                    }
+                }
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(acce_bar(buf)) : "memory");
+            }
+        }
+        it = it0 + nun;
+        seg_it = seg0 + nsegs;
+    };
+
+    // ---- attention phase (same decomposition as the stand-alone kernel, CTAs = the grid)
+    auto attn_phase = [&](int layer, unsigned gate) {
+        const int items = B, Bc = B, nq_act = grouped ? 2 * G : G;
+        if (is_prod && lane == 0) wait_gen(gate, 500);
+        if (warp == 2) {
+            int running = 0, longest = 0;
+            if (lane == 0) cum[0] = 0;
+            for (int base = 0; base < items; base += 32) {
+                int i = base + lane, nk = 0, u = 0;
+                if (i < items) {
+                    nk = ld_mut(pl->seq_len + i) + 1;
+                    u = (nk + kAttTile - 1) / kAttTile;
+                    nk_s[i] = nk;
+                }
+                int incl = u, mx = u;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    int t = __shfl_up_sync(0xffffffffu, incl, o);
+                    if (lane >= o) incl += t;
+                    mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+                }
+                longest = max(longest, mx);
+                if (i < items) cum[i + 1] = running + incl;
+                running += __shfl_sync(0xffffffffu, incl, 31);
+            }
+            if (lane == 0) flag[1] = longest;
+        }
+        __syncthreads();
+        const int U = cum[items] * n_kv;
+        const int quota = max(max((U + C - 1) / C, kAttMinUnits), (flag[1] + kAttMaxSeg - 2) / (kAttMaxSeg - 1));
+        const int u0 = min(U, cta * quota), u1 = min(U, u0 + quota);
+        const int it0 = it;
+        const long long k_row0 = (long long)layer * 2 * pl->plane_rows, v_row0 = k_row0 + pl->plane_rows;
+        const CUtensorMap *tmKV = map_tail + 4;
+        int item = 0;
+        if (u0 < u1)
+            while (cum[item + 1] * n_kv <= u0) item++;
+
+        if (is_prod) {
+            if (lane == 0) {
+                for (int u = u0; u < u1 && ok;) {
+                    int ui = cum[item + 1] - cum[item], base = cum[item] * n_kv;
+                    int g = (u - base) / ui, t0 = (u - base) % ui;
+                    int pair_end = base + (g + 1) * ui, t1 = t0 + min(u1, pair_end) - u;
+                    int total_pages = (nk_s[item] + 15) >> 4;
+                    for (int t = t0; t < t1 && ok; t++, it++) {
+                        int s = it % SLOTS;
+                        if (it >= SLOTS) wait_bar(empty_bar(s), ((it / SLOTS) - 1) & 1, 510);
+                        if (!ok) break;
+                        int p0 = t * 4, np = min(4, total_pages - p0);
+                        mbar_expect_tx(full_bar(s), (uint32_t)np * 2 * PAGE_BYTES);
+                        uint32_t kdst = ring + s * kMegaSlotBytes, vdst = kdst + 4 * PAGE_BYTES;
+                        for (int j = 0; j < np; j++) {
+                            int page = pl->page_table[(size_t)item * pl->pt_stride + p0 + j];
+                            if (page < 0 || page >= pl->num_pages) {
+                                report(pl->status, kStatusBadPage, page);
+                                page = 0;
+                            }
+                            int row = (int)(((long long)page * n_kv + g) * 16);
+                            for (int h = 0; h < HALVES; h++) {
+                                tma_load_2d(kdst + (j * HALVES + h) * 2048, tmKV, full_bar(s), h * 64, (int)(k_row0 + row));
+                                tma_load_2d(vdst + (j * HALVES + h) * 2048, tmKV, full_bar(s), h * 64, (int)(v_row0 + row));
+                            }
+                        }
+                    }
+                    u += t1 - t0;
+                    if (u == pair_end && g == n_kv - 1) item++;
+                }
+            }
+        } else if (is_worker) {
+            const float qscale = kLog2e / sqrtf((float)DH);
+            for (int u = u0; u < u1;) {
+                int ui = cum[item + 1] - cum[item], base = cum[item] * n_kv;
+                int g = (u - base) / ui, t0 = (u - base) % ui;
+                int pair_start = base + g * ui, pair_end = pair_start + ui, t1 = t0 + min(u1, pair_end) - u;
+                int nkeys = nk_s[item];
+                worker_sync();
+                for (int idx = wt; idx < 16 * DH / 4; idx += 128) {
+                    int q = idx / (DH / 4), c4 = idx % (DH / 4);
+                    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (q < nq_act) {
+                        int row = q < G ? item : Bc + item;
+                        int h = g * G + (q < G ? q : q - G);
+                        v = __ldcg(reinterpret_cast<const float4 *>(pl->Q + (size_t)row * qd + (size_t)h * DH) + c4);
+                    }
+                    reinterpret_cast<float4 *>(sc_o)[idx] = v;
+                }
+                worker_sync();
+                uint32_t qa[KS][4];
+                {
+                    int r0 = lane >> 2, c = (lane & 3) * 2;
+                    const float *q0 = sc_o + r0 * DH, *q1 = sc_o + (r0 + 8) * DH;
+#pragma unroll
+                    for (int ks = 0; ks < KS; ks++) {
+                        int k = ks * 16 + c;
+                        qa[ks][0] = pack_bf16(q0[k] * qscale, q0[k + 1] * qscale);
+                        qa[ks][1] = pack_bf16(q1[k] * qscale, q1[k + 1] * qscale);
+                        qa[ks][2] = pack_bf16(q0[k + 8] * qscale, q0[k + 9] * qscale);
+                        qa[ks][3] = pack_bf16(q1[k + 8] * qscale, q1[k + 9] * qscale);
+                    }
+                }
+                worker_sync();
+                float o[NB][4];
+#pragma unroll
+                for (int nb = 0; nb < NB; nb++) o[nb][0] = o[nb][1] = o[nb][2] = o[nb][3] = 0.f;
+                float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+                for (int t = t0; t < t1; t++, it++) {
+                    int s = it % SLOTS;
+                    wait_bar(full_bar(s), (it / SLOTS) & 1, 520);
+                    bool live = __all_sync(0xffffffffu, ok);
+                    int valid = min(16, nkeys - (t * kAttTile + ww * 16));
+                    if (live && valid > 0) {
+                        uint32_t kpage = ring + s * kMegaSlotBytes + ww * HALVES * 2048;
+                        uint32_t vpage = kpage + 4 * PAGE_BYTES;
+                        if (valid < 16) {
+                            for (int idx = lane; idx < (16 - valid) * HALVES * 8; idx += 32) {
+                                int r = valid + idx / (HALVES * 8), rest = idx % (HALVES * 8);
+                                uint32_t a = vpage + (rest / 8) * 2048 + r * 128 + (rest % 8) * 16;
+                                asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(a), "r"(0u) : "memory");
+                            }
+                            __syncwarp();
+                        }
+                        float sacc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+                        {
+                            int r = (lane & 7) + ((lane >> 4) << 3), cb = (lane >> 3) & 1;
+#pragma unroll
+                            for (int ks = 0; ks < KS; ks++) {
+                                int chunk = ks * 2 + cb;
+                                uint32_t a = kpage + (chunk >> 3) * 2048 + r * 128 + (((chunk & 7) ^ (r & 7)) << 4);
+                                uint32_t kb[4];
+                                ldsm_x4(a, kb);
+                                mma_bf16(sacc[0], qa[ks], kb[0], kb[1]);
+                                mma_bf16(sacc[1], qa[ks], kb[2], kb[3]);
+                            }
+                        }
+                        int col = (lane & 3) * 2;
+                        float rmax[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+                        for (int nb = 0; nb < 2; nb++)
+#pragma unroll
+                            for (int e = 0; e < 4; e++) {
+                                int tk = nb * 8 + col + (e & 1);
+                                if (tk >= valid) sacc[nb][e] = -INFINITY;
+                                rmax[e >> 1] = fmaxf(rmax[e >> 1], sacc[nb][e]);
+                            }
+                        float corr[2], msub[2];
+#pragma unroll
+                        for (int h = 0; h < 2; h++) {
+                            rmax[h] = fmaxf(rmax[h], __shfl_xor_sync(0xffffffffu, rmax[h], 1));
+                            rmax[h] = fmaxf(rmax[h], __shfl_xor_sync(0xffffffffu, rmax[h], 2));
+                            float mnew = fmaxf(m_run[h], rmax[h]);
+                            msub[h] = mnew == -INFINITY ? 0.f : mnew;
+                            corr[h] = m_run[h] == -INFINITY ? 0.f : exp2f(m_run[h] - msub[h]);
+                            m_run[h] = mnew;
+                        }
+                        float rsum[2] = {0.f, 0.f};
+                        uint32_t pa[4];
+#pragma unroll
+                        for (int nb = 0; nb < 2; nb++) {
+                            float p0 = exp2f(sacc[nb][0] - msub[0]), p1 = exp2f(sacc[nb][1] - msub[0]);
+                            float p2 = exp2f(sacc[nb][2] - msub[1]), p3 = exp2f(sacc[nb][3] - msub[1]);
+                            rsum[0] += p0 + p1;
+                            rsum[1] += p2 + p3;
+                            pa[nb * 2 + 0] = pack_bf16(p0, p1);
+                            pa[nb * 2 + 1] = pack_bf16(p2, p3);
+                        }
+#pragma unroll
+                        for (int h = 0; h < 2; h++) {
+                            rsum[h] += __shfl_xor_sync(0xffffffffu, rsum[h], 1);
+                            rsum[h] += __shfl_xor_sync(0xffffffffu, rsum[h], 2);
+                            l_run[h] = l_run[h] * corr[h] + rsum[h];
+                        }
+#pragma unroll
+                        for (int nb = 0; nb < NB; nb++) {
+                            o[nb][0] *= corr[0];
+                            o[nb][1] *= corr[0];
+                            o[nb][2] *= corr[1];
+                            o[nb][3] *= corr[1];
+                        }
+                        {
+                            int r = (lane & 7) + (((lane >> 3) & 1) << 3), cb = lane >> 4;
+#pragma unroll
+                            for (int np = 0; np < NB / 2; np++) {
+                                int chunk = np * 2 + cb;
+                                uint32_t a = vpage + (chunk >> 3) * 2048 + r * 128 + (((chunk & 7) ^ (r & 7)) << 4);
+                                uint32_t vb[4];
+                                ldsm_x4_trans(a, vb);
+                                mma_bf16(o[np * 2], pa, vb[0], vb[1]);
+                                mma_bf16(o[np * 2 + 1], pa, vb[2], vb[3]);
+                            }
+                        }
+                    }
+                    __syncwarp();
+                    if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(empty_bar(s)) : "memory");
+                }
+                // fold the four warps' states (0+2) + (1+3) through the one-slot scratch
+                int pair = item * n_kv + g;
+                int first_cta = pair_start / quota, nseg = (pair_end - 1) / quota - first_cta + 1;
+                float *out = pl->part + (size_t)(cta + pair) * 16 * (DH + 2);
+                {
+                    int r0 = lane >> 2, c = (lane & 3) * 2;
+                    auto put = [&]() {
+#pragma unroll
+                        for (int nb = 0; nb < NB; nb++) {
+                            *reinterpret_cast<float2 *>(sc_o + (size_t)r0 * DH + nb * 8 + c) = make_float2(o[nb][0], o[nb][1]);
+                            *reinterpret_cast<float2 *>(sc_o + (size_t)(r0 + 8) * DH + nb * 8 + c) = make_float2(o[nb][2], o[nb][3]);
+                        }
+                        if ((lane & 3) == 0) {
+                            sc_m[r0] = m_run[0];
+                            sc_m[r0 + 8] = m_run[1];
+                            sc_l[r0] = l_run[0];
+                            sc_l[r0 + 8] = l_run[1];
+                        }
+                    };
+                    auto take = [&]() {
+#pragma unroll
+                        for (int h = 0; h < 2; h++) {
+                            int r = r0 + 8 * h;
+                            float mb = sc_m[r], lb = sc_l[r];
+                            float M = fmaxf(m_run[h], mb);
+                            float fa = m_run[h] == -INFINITY ? 0.f : exp2f(m_run[h] - M);
+                            float fb = mb == -INFINITY ? 0.f : exp2f(mb - M);
+                            l_run[h] = l_run[h] * fa + lb * fb;
+                            m_run[h] = M;
+#pragma unroll
+                            for (int nb = 0; nb < NB; nb++) {
+                                float2 ob = *reinterpret_cast<const float2 *>(sc_o + (size_t)r * DH + nb * 8 + c);
+                                o[nb][2 * h] = o[nb][2 * h] * fa + ob.x * fb;
+                                o[nb][2 * h + 1] = o[nb][2 * h + 1] * fa + ob.y * fb;
+                            }
+                        }
+                    };
+                    for (int step = 0; step < 3; step++) {
+                        int src = step == 0 ? 2 : step == 1 ? 3 : 1, dst = step == 1 ? 1 : 0;
+                        if (ww == src) put();
+                        worker_sync();
+                        if (ww == dst) take();
+                        worker_sync();
+                    }
+                    if (ww == 0) {
+#pragma unroll
+                        for (int h = 0; h < 2; h++) {
+                            int q = r0 + 8 * h;
+                            if (q < nq_act) {
+#pragma unroll
+                                for (int nb = 0; nb < NB; nb++)
+                                    *reinterpret_cast<float2 *>(out + (size_t)q * (DH + 2) + nb * 8 + c) =
+                                        make_float2(o[nb][2 * h], o[nb][2 * h + 1]);
+                                if ((lane & 3) == 0) {
+                                    out[(size_t)q * (DH + 2) + DH] = m_run[h];
+                                    out[(size_t)q * (DH + 2) + DH + 1] = l_run[h];
+                                }
+                            }
+                        }
+                    }
+                }
+                __threadfence();
+                worker_sync();
+                if (wt == 0) {
+                    int last = 1;
+                    if (nseg > 1) {
+                        int *tk = pl->att_tickets + pair;
+                        int tkt = atomicAdd(tk, 1);
+                        last = tkt == nseg - 1;
+                        if (last) atomicExch(tk, 0);
+                    }
+                    flag[0] = last;
+                }
+                worker_sync();
+                if (flag[0]) {
+                    __threadfence();
+                    const float *pbase = pl->part + (size_t)(first_cta + pair) * 16 * (DH + 2);
+                    float *wgt = sc_o, *ml = sc_o + 16 * kAttMaxSeg;
+                    for (int t = wt; t < nq_act * nseg; t += 128) {
+                        int q = t / nseg, s2 = t % nseg;
+                        const float *pp = pbase + ((size_t)s2 * 16 + q) * (DH + 2) + DH;
+                        wgt[q * kAttMaxSeg + s2] = __ldcg(pp);
+                        ml[q * kAttMaxSeg + s2] = __ldcg(pp + 1);
+                    }
+                    worker_sync();
+                    if (wt < nq_act) {
+                        float M = -INFINITY, L = 0.f;
+                        for (int s2 = 0; s2 < nseg; s2++) M = fmaxf(M, wgt[wt * kAttMaxSeg + s2]);
+                        for (int s2 = 0; s2 < nseg; s2++) {
+                            float ms = wgt[wt * kAttMaxSeg + s2];
+                            float f = ms == -INFINITY ? 0.f : exp2f(ms - M);
+                            L += ml[wt * kAttMaxSeg + s2] * f;
+                            wgt[wt * kAttMaxSeg + s2] = f;
+                        }
+                        float inv = 1.f / L;
+                        for (int s2 = 0; s2 < nseg; s2++) wgt[wt * kAttMaxSeg + s2] *= inv;
+                    }
+                    worker_sync();
+                    for (int idx = wt; idx < nq_act * DH; idx += 128) {
+                        int q = idx / DH, e = idx % DH;
+                        float x = 0.f;
+                        for (int s2 = 0; s2 < nseg; s2++)
+                            x = fmaf(__ldcg(pbase + ((size_t)s2 * 16 + q) * (DH + 2) + e), wgt[q * kAttMaxSeg + s2], x);
+                        int row = q < G ? item : Bc + item;
+                        int h = g * G + (q < G ? q : q - G);
+                        store_split(pl->Ob, (size_t)row * qd + (size_t)h * DH + e, pl->lo_o, x);
+                    }
+                }
+                u += t1 - t0;
+                if (u == pair_end && g == n_kv - 1) item++;
+            }
+        }
+        it = it0 + (u1 - u0);
+    };
+
+    // =========================== the step ===========================================
+    // E0: embeddings (Eq. embeddings), one row per CTA
+    if (is_worker) {
+        for (int r = cta; r < R; r += C) {
+            int path = r >= B;
+            int tok = ld_mut(tokens + (r % B));
+            if (tok < 0 || tok >= V) {
+                if (wt == 0) report(pl->status, kStatusBadToken, tok);
+                tok = min(max(tok, 0), V - 1);
+            }
+            const __nv_bfloat16 *e = (path ? pl->E2 : pl->E1) + (size_t)tok * d;
+            float ssq = 0.f;
+            for (int i = wt; i < d; i += 128) {
+                float x = __bfloat162float(e[i]);
+                ssq += x * x;
+            }
+            ssq = worker_sum(ssq);
+            float inv = 1.f / sqrtf(ssq / (float)d + eps), sq = 0.f;
+            for (int i = wt; i < d; i += 128) {
+                float s0 = pl->g_e[i] * __bfloat162float(e[i]) * inv;
+                pl->S[(size_t)r * d + i] = s0;
+                store_split(pl->Xb, (size_t)r * d + i, pl->lo_x, pl->g_first[i] * s0);
+                sq += s0 * s0;
+            }
+            sq = worker_sum(sq);
+            for (int t = wt; t < ss_tiles; t += 128) pl->ss[(size_t)t * ss_ld + r] = t == 0 ? sq : 0.f;
+        }
+    }
+    grid_barrier();
+
+    const int tQ = (qd + 127) / 128, tK = (kvd + 127) / 128, tG = (F + 127) / 128;
+    for (int l = 0; l < pl->L; l++) {
+        const MegaLayer &ly = pl->layer[l];
+        const CUtensorMap *mp = maps + (size_t)l * 7;
+        const long long plane = pl->plane_rows;
+        __nv_bfloat16 *kpool = pl->pool + (size_t)l * 2 * plane * DH, *vpool = kpool + (size_t)plane * DH;
+
+        // G1: Q | K | V
+        Gemm g1 = make_gemm(mp + 0, qd, mp + 1, kvd, mp + 2, kvd, map_tail + 1, d);
+        gemm_phase(g1, k_bar);
+        grid_barrier();
+        // E1: 1/rms, RoPE, a coupling, cache append
+        if (is_worker) {
+            const int per_row = (n_q + n_kv) * half, total = B * per_row;
+            for (int idx = cta * 128 + wt; idx < total; idx += C * 128) {
+                int b = idx / per_row, rem = idx % per_row, hh = rem / half, i = rem % half;
+                int pos = ld_mut(pl->seq_len + b);
+                float2 t = pl->rope[(size_t)pos * half + i];
+                float rs1 = row_scale(pl->ss, ss_tiles, ss_ld, b, d, eps);
+                if (hh < n_q) {
+                    int o0 = hh * dh + i, o1 = o0 + half, tile = o0 / 128;
+                    float x0 = rs1 * tile_sum(g1, tile, b, o0 % 128), x1 = rs1 * tile_sum(g1, tile, b, o1 % 128);
+                    float r0 = x0 * t.x - x1 * t.y, r1 = x1 * t.x + x0 * t.y;
+                    pl->Q[(size_t)b * qd + o0] = r0;
+                    pl->Q[(size_t)b * qd + o1] = r1;
+                    if (grouped) {
+                        float rs2 = row_scale(pl->ss, ss_tiles, ss_ld, B + b, d, eps);
+                        float y0 = rs2 * tile_sum(g1, tile, B + b, o0 % 128), y1 = rs2 * tile_sum(g1, tile, B + b, o1 % 128);
+                        pl->Q[(size_t)(B + b) * qd + o0] = (y0 * t.x - y1 * t.y) + ly.coup_a[o0] * r0;
+                        pl->Q[(size_t)(B + b) * qd + o1] = (y1 * t.x + y0 * t.y) + ly.coup_a[o1] * r1;
+                    }
+                } else {
+                    int gk = hh - n_q, c0 = gk * dh + i, c1 = c0 + half;
+                    int page = pl->page_table[(size_t)b * pl->pt_stride + pos / 16];
+                    if (page < 0 || page >= pl->num_pages) {
+                        report(pl->status, kStatusBadPage, page);
+                    } else {
+                        size_t base = (((size_t)page * n_kv + gk) * 16 + (pos & 15)) * dh;
+                        int tk = tQ + c0 / 128, tv = tQ + tK + c0 / 128;
+                        float x0 = rs1 * tile_sum(g1, tk, b, c0 % 128), x1 = rs1 * tile_sum(g1, tk, b, c1 % 128);
+                        kpool[base + i] = __float2bfloat16_rn(x0 * t.x - x1 * t.y);
+                        kpool[base + i + half] = __float2bfloat16_rn(x1 * t.x + x0 * t.y);
+                        vpool[base + i] = __float2bfloat16_rn(rs1 * tile_sum(g1, tv, b, c0 % 128));
+                        vpool[base + i + half] = __float2bfloat16_rn(rs1 * tile_sum(g1, tv, b, c1 % 128));
+                    }
+                }
+            }
+        }
+        grid_barrier();
+        // A: attention of both paths over the primary cache
+        attn_phase(l, k_bar);
+        grid_barrier();
+        // G2: O projection
+        Gemm g2 = make_gemm(mp + 3, d, nullptr, 0, nullptr, 0, map_tail + 2, qd);
+        gemm_phase(g2, k_bar);
+        grid_barrier();
+        // E2 / E4 share this: residual update, next GEMM input, shares of sum(S^2)
+        auto resid = [&](const Gemm &g, int mode, const float *coup_c, const float *g_next) {
+            if (!is_worker) return;
+            for (int unit = cta; unit < B * ss_tiles; unit += C) {
+                int b = unit / ss_tiles, blk = unit % ss_tiles;
+                float q1 = 0.f, q2 = 0.f;
+                for (int j = 0; j < 2; j++) {
+                    int i = blk * 256 + j * 128 + wt;
+                    if (i < d) {
+                        float gn = g_next ? g_next[i] : 1.f;
+                        size_t o1 = (size_t)b * d + i, o2 = (size_t)(B + b) * d + i;
+                        float m1 = tile_sum(g, i / 128, b, i % 128);
+                        float s1 = __ldcg(pl->S + o1) + m1;
+                        pl->S[o1] = s1;
+                        store_split(pl->Xb, o1, pl->lo_x, gn * s1);
+                        q1 += s1 * s1;
+                        if (grouped) {
+                            float m2 = tile_sum(g, i / 128, B + b, i % 128);
+                            if (mode == 2) m2 += coup_c[i] * m1;
+                            float s2 = __ldcg(pl->S + o2) + m2;
+                            pl->S[o2] = s2;
+                            store_split(pl->Xb, o2, pl->lo_x, gn * s2);
+                            q2 += s2 * s2;
+                        }
+                    }
+                }
+                q1 = worker_sum(q1);
+                q2 = worker_sum(q2);
+                if (wt == 0) {
+                    pl->ss[(size_t)blk * ss_ld + b] = q1;
+                    if (grouped) pl->ss[(size_t)blk * ss_ld + B + b] = q2;
+                }
+            }
+        };
+        resid(g2, 1, nullptr, ly.g_mlp);
+        grid_barrier();
+        // G3: gate | up
+        Gemm g3 = make_gemm(mp + 4, F, mp + 5, F, nullptr, 0, map_tail + 1, d);
+        gemm_phase(g3, k_bar);
+        grid_barrier();
+        // E3: SwiGLU and the b coupling
+        if (is_worker) {
+            for (int idx = cta * 128 + wt; idx < B * F; idx += C * 128) {
+                int b = idx / F, f = idx % F;
+                float rs1 = row_scale(pl->ss, ss_tiles, ss_ld, b, d, eps);
+                float h1 = silu(rs1 * tile_sum(g3, f / 128, b, f % 128)) * (rs1 * tile_sum(g3, tG + f / 128, b, f % 128));
+                store_split(pl->Hb, (size_t)b * F + f, pl->lo_h, h1);
+                if (grouped) {
+                    float rs2 = row_scale(pl->ss, ss_tiles, ss_ld, B + b, d, eps);
+                    float h2 = silu(rs2 * tile_sum(g3, f / 128, B + b, f % 128)) *
+                               (rs2 * tile_sum(g3, tG + f / 128, B + b, f % 128));
+                    store_split(pl->Hb, (size_t)(B + b) * F + f, pl->lo_h, h2 + ly.coup_b[f] * h1);
+                }
+            }
+        }
+        grid_barrier();
+        // G4: down
+        Gemm g4 = make_gemm(mp + 6, d, nullptr, 0, nullptr, 0, map_tail + 3, F);
+        gemm_phase(g4, k_bar);
+        grid_barrier();
+        resid(g4, 2, ly.coup_c, ly.g_next);
+        grid_barrier();
+    }
+
+    // ---- output matrix and readout (Eq. alpha, Eq. mixloss)
+    Gemm g5 = make_gemm(map_tail + 0, V, nullptr, 0, nullptr, 0, map_tail + 1, d);
+    gemm_phase(g5, k_bar);
+    grid_barrier();
+    const int chunk = (V + C - 1) / C, v0 = min(V, cta * chunk), v1 = min(V, v0 + chunk);
+    if (is_worker) {
+        // logits of this CTA's vocabulary chunk, and per-row (max, sum exp, sum exp^2) of the chunk
+        for (int r = ww; r < R; r += 4) {
+            float rs = pl->final_norm ? row_scale(pl->ss, ss_tiles, ss_ld, r, d, eps) : 1.f;
+            float mx = -INFINITY;
+            for (int v = v0 + lane; v < v1; v += 32) {
+                float z = rs * tile_sum(g5, v / 128, r, v % 128);
+                pl->Z[(size_t)r * V + v] = z;
+                mx = fmaxf(mx, z);
+            }
+            mx = warp_max(mx);
+            float s1 = 0.f, c1 = 0.f;
+            __syncwarp();
+            for (int v = v0 + lane; v < v1; v += 32) {
+                float e1 = expf(pl->Z[(size_t)r * V + v] - mx);
+                s1 += e1;
+                c1 += e1 * e1;
+            }
+            s1 = warp_sum(s1);
+            c1 = warp_sum(c1);
+            if (lane == 0) {
+                float *o = pl->rd_part + ((size_t)cta * 64 + r) * 4;
+                o[0] = mx;
+                o[1] = s1;
+                o[2] = c1;
+            }
+        }
+    }
+    grid_barrier();
+    if (is_worker) {
+        // global softmax statistics per row from the chunk partials (CTA order), then this chunk's
+        // best candidate of the mixture per sequence
+        for (int b = ww; b < B; b += 4) {
+            float M[2] = {0.f, 0.f}, D[2] = {1.f, 1.f}, alpha = 1.f;
+            if (grouped) {
+                float Cq = 0.f;
+                for (int p = 0; p < 2; p++) {
+                    int r = p * B + b;
+                    float mx = -INFINITY;
+                    for (int c = lane; c < C; c += 32) mx = fmaxf(mx, __ldcg(pl->rd_part + ((size_t)c * 64 + r) * 4));
+                    mx = warp_max(mx);
+                    float s = 0.f, cq = 0.f;
+                    for (int c = lane; c < C; c += 32) {
+                        const float *o = pl->rd_part + ((size_t)c * 64 + r) * 4;
+                        float mc = __ldcg(o);
+                        if (mc != -INFINITY) {
+                            float f = expf(mc - mx);
+                            s += __ldcg(o + 1) * f;
+                            cq += __ldcg(o + 2) * f * f;
+                        }
+                    }
+                    M[p] = mx;
+                    D[p] = warp_sum(s);
+                    if (p == 0) Cq = warp_sum(cq);
+                }
+                alpha = fminf(1.f, fmaxf(0.5f, Cq / (D[0] * D[0])));
+            }
+            ArgBest best = {-INFINITY, 0x7fffffff};
+            for (int v = v0 + lane; v < v1; v += 32) {
+                float z1 = __ldcg(pl->Z + (size_t)b * V + v);
+                float val = z1;
+                if (grouped) {
+                    float z2 = __ldcg(pl->Z + (size_t)(B + b) * V + v);
+                    val = alpha * (expf(z1 - M[0]) / D[0]) + (1.f - alpha) * (expf(z2 - M[1]) / D[1]);
+                }
+                best = better(best, ArgBest{val, v});
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                ArgBest other = {__shfl_xor_sync(0xffffffffu, best.v, o), __shfl_xor_sync(0xffffffffu, best.i, o)};
+                best = better(best, other);
+            }
+            if (lane == 0) {
+                float *o = pl->rd_best + ((size_t)cta * 64 + b) * 2;
+                o[0] = best.v;
+                o[1] = __int_as_float(best.i);
+                if (cta == 0 && grouped && alpha_out) alpha_out[b] = alpha;
+            }
+        }
+    }
+    grid_barrier();
+    if (is_worker && cta == 0) {
+        for (int b = ww; b < B; b += 4) {
+            ArgBest best = {-INFINITY, 0x7fffffff};
+            for (int c = lane; c < C; c += 32) {
+                const float *o = pl->rd_best + ((size_t)c * 64 + b) * 2;
+                best = better(best, ArgBest{__ldcg(o), __float_as_int(__ldcg(o + 1))});
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                ArgBest other = {__shfl_xor_sync(0xffffffffu, best.v, o), __shfl_xor_sync(0xffffffffu, best.i, o)};
+                best = better(best, other);
+            }
+            if (lane == 0) {
+                if (next) next[b] = best.i;
+                pl->seq_len[b] += 1;
+            }
+        }
+    }
+
+    // ---- teardown: nothing of this CTA may still be in flight
+    if (is_prod && lane == 0 && !ok) {
+        // give copies that were issued a bounded time to land before the shared memory goes away
+        long long t0 = clock64();
+        while ((unsigned long long)(clock64() - t0) < 200000ull) {
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (is_mma)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                     "r"((uint32_t)(2 * N_TILE < 32 ? 32 : 2 * N_TILE))
+                     : "memory");
+    if (tid == 0) {
+        // the last CTA out re-arms the barrier counters for the next launch
+        __threadfence();
+        unsigned n = atomicAdd(pl->done_count, 1u);
+        if (n == (unsigned)C - 1) {
+            atomicExch(pl->bar_count, 0u);
+            atomicExch(pl->done_count, 0u);
+        }
+    }
+}
+
+}  // namespace dbt
