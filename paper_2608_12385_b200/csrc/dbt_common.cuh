@@ -21,12 +21,12 @@ __device__ __forceinline__ void report(int *status, int code, int detail) {
 // predecessor's results before reading or writing anything that predecessor touches.
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-#ifdef DBT_TIMELINE
 __device__ __forceinline__ unsigned long long gtime() {
     unsigned long long t;
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
+#ifdef DBT_TIMELINE
 #define DBT_TL_DECL unsigned long long tl0_ = gtime(), tl1_ = 0
 #define DBT_TL_WAITED tl1_ = gtime()
 #define DBT_TL_END(name)                                                                                   \

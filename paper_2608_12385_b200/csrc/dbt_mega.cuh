@@ -71,7 +71,7 @@ struct MegaPlan {
 template <int N_TILE, int DH>
 struct MegaCfg {
     static constexpr int kBBytes = N_TILE * kTcK * 2;
-    static constexpr int kScratchFloats = 16 * DH + 1024;
+    static constexpr int kScratchFloats = 16 * DH + 1024 + 768;
     static constexpr int kSmemBytes = kMegaSlots * kMegaSlotBytes + 1024 + 256 + kScratchFloats * 4;
     static_assert(kTcABytes + 2 * kBBytes <= kMegaSlotBytes, "GEMM stage must fit a ring slot");
     static_assert(2 * 4 * 16 * DH * 2 <= kMegaSlotBytes, "attention stage must fit a ring slot");
@@ -108,6 +108,9 @@ mega_decode_kernel(const MegaPlan *__restrict__ pl, const int32_t *tokens, int32
     int *cum = flag + 8, *nk_s = cum + kAttMaxItems + 1;
     float *red = reinterpret_cast<float *>(nk_s + kAttMaxItems);  // [64] worker reductions
 
+#ifdef DBT_MEGA_TL
+    unsigned long long *tl = reinterpret_cast<unsigned long long *>(sc_o + 16 * DH + 640);  // debug: barrier timestamps
+#endif
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const bool is_prod = warp == 0, is_mma = warp == 1, is_worker = warp >= 2;
     const int wt = tid - 64, ww = warp - 2;  // worker thread / warp index
@@ -196,6 +199,9 @@ mega_decode_kernel(const MegaPlan *__restrict__ pl, const int32_t *tokens, int32
                 }
             }
             *gen_s = k_bar;
+#ifdef DBT_MEGA_TL
+            if (cta == 0 && k_bar < 380) tl[k_bar] = gtime();
+#endif
         }
         worker_sync();
         __threadfence();
@@ -303,6 +309,10 @@ mega_decode_kernel(const MegaPlan *__restrict__ pl, const int32_t *tokens, int32
         } else if (is_mma) {
             if (lane == 0) {
                 constexpr uint32_t idesc = umma_idesc(N_TILE);
+                // Not before this CTA's workers are through the preceding phases: a wait posted on a
+                // full barrier while the attention phase still cycles the same slot would be two
+                // phases ahead of it and could match the parity of an attention stage.
+                wait_gen(gate, 415);
                 for (int u = u0; u < u1 && ok; u++, it++) {
                     int s = it % SLOTS, kt = u % g.KT;
                     int buf = seg_it & 1;
@@ -919,6 +929,11 @@ mega_decode_kernel(const MegaPlan *__restrict__ pl, const int32_t *tokens, int32
         }
     }
 
+#ifdef DBT_MEGA_TL
+    if (cta == 0 && wt == 0) {
+        for (unsigned k = 2; k <= k_bar && k < 380; k++) printf("TL %u %llu\n", k, tl[k] - tl[k - 1]);
+    }
+#endif
     // ---- teardown: nothing of this CTA may still be in flight
     if (is_prod && lane == 0 && !ok) {
         // give copies that were issued a bounded time to land before the shared memory goes away
