@@ -49,6 +49,7 @@ struct Workspace {
     float *rd_part, *rd_best;
 };
 constexpr int kMegaPlanSlots = 16;
+constexpr int kMegaTailMaps = 11;  // lm_head, K/V pages, {Xb, Ob, Hb} x row-tile width {16, 32, 64}
 
 struct LayerMaps {
     CUtensorMap wq, wk, wv, wo, wg, wu, wd;  // dense MLP; for MoE wg/wu/wd hold the shared expert
@@ -212,7 +213,7 @@ size_t carve(const dbt_config &c, char *base, Workspace *ws, int *Rmax_out, int 
         w.ss = k.take<float>((size_t)((d + 127) / 128) * Rmax);
         if (!moe) {
             w.mega_plans = k.take<char>((size_t)kMegaPlanSlots * align_up(sizeof(MegaPlan)));
-            w.mega_maps = k.take<CUtensorMap>((size_t)c.n_layers * 7 + 5);
+            w.mega_maps = k.take<CUtensorMap>((size_t)c.n_layers * 7 + kMegaTailMaps);
             w.mega_sync = k.take<unsigned int>(8);
             w.rd_part = k.take<float>((size_t)kMegaMaxCtas * 64 * 4);
             w.rd_best = k.take<float>((size_t)kMegaMaxCtas * 64 * 2);
@@ -1276,14 +1277,23 @@ bool setup_mega(dbt_model *m) {
         return false;
     }
     const Workspace &w = m->ws;
-    std::vector<CUtensorMap> maps((size_t)c.n_layers * 7 + 5);
+    std::vector<CUtensorMap> maps((size_t)c.n_layers * 7 + kMegaTailMaps);
     for (int l = 0; l < c.n_layers; l++) {
         const LayerMaps &mp = m->maps[l];
         CUtensorMap *o = maps.data() + (size_t)l * 7;
         o[0] = mp.wq; o[1] = mp.wk; o[2] = mp.wv; o[3] = mp.wo; o[4] = mp.wg; o[5] = mp.wu; o[6] = mp.wd;
     }
     CUtensorMap *t = maps.data() + (size_t)c.n_layers * 7;
-    t[0] = m->map_lm; t[1] = m->map_Xb; t[2] = m->map_Ob; t[3] = m->map_Hb; t[4] = m->map_kv;
+    t[0] = m->map_lm;
+    uint64_t plane_rows = (uint64_t)c.num_pages * c.n_kv_heads * c.page_size;
+    bool mok = make_kv_page_map(&t[1], m->kv_pool, (uint64_t)c.n_layers * 2 * plane_rows, plane_rows, c.head_dim);
+    for (int i = 0; i < 3 && mok; i++) {
+        uint32_t nt = 16u << i;
+        mok = make_act_map(&t[2 + 3 * i + 0], w.Xb, m->Rmax, c.d_model, nt) &&
+              make_act_map(&t[2 + 3 * i + 1], w.Ob, m->Rmax, (uint64_t)c.n_q_heads * c.head_dim, nt) &&
+              make_act_map(&t[2 + 3 * i + 2], w.Hb, m->Rmax, c.d_ff, nt);
+    }
+    if (!mok) return false;
     if (cudaMemcpy(w.mega_maps, maps.data(), maps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice) != cudaSuccess ||
         cudaMemset(w.mega_sync, 0, sizeof(unsigned int) * 8) != cudaSuccess) {
         cudaGetLastError();
