@@ -1285,8 +1285,8 @@ bool setup_mega(dbt_model *m) {
     }
     CUtensorMap *t = maps.data() + (size_t)c.n_layers * 7;
     t[0] = m->map_lm;
-    uint64_t plane_rows = (uint64_t)c.num_pages * c.n_kv_heads * c.page_size;
-    bool mok = make_kv_page_map(&t[1], m->kv_pool, (uint64_t)c.n_layers * 2 * plane_rows, plane_rows, c.head_dim);
+    t[1] = m->map_kv;
+    bool mok = true;
     for (int i = 0; i < 3 && mok; i++) {
         uint32_t nt = 16u << i;
         mok = make_act_map(&t[2 + 3 * i + 0], w.Xb, m->Rmax, c.d_model, nt) &&
@@ -1365,8 +1365,8 @@ bool setup_tc(dbt_model *m) {
     if (!moe) ok = ok && make_bf16_map(&m->map_Hb, w.Hb, 2 * m->Rmax, F, 16);
     const char *fa = getenv("DBT_ATTN");
     m->att_fast = ok && !(fa && strcmp(fa, "simt") == 0) &&
-                  make_kv_map(&m->map_kv, m->kv_pool, (uint64_t)c.n_layers * 2 * c.num_pages * c.n_kv_heads * c.page_size,
-                              c.head_dim) &&
+                  make_kv_page_map(&m->map_kv, m->kv_pool, (uint64_t)c.n_layers * 2 * c.num_pages * c.n_kv_heads * c.page_size,
+                                   (uint64_t)c.num_pages * c.n_kv_heads * c.page_size, c.head_dim) &&
                   cudaFuncSetAttribute(attn_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        AttCfg<128>::kSmemBytes) == cudaSuccess &&
                   cudaFuncSetAttribute(attn_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,

@@ -53,8 +53,10 @@ struct AttCfg {
     static constexpr int kPageBytes = 16 * DH * 2;          // one page of K (or V) for one head
     static constexpr int kStageBytes = 2 * 4 * kPageBytes;  // K + V, 4 pages
     static constexpr int kStages = DH == 128 ? 3 : 6;       // 96 KB ring: two CTAs keep ~190 KB in flight per SM
-    // scratch: one [16][DH] fp32 slot (Q tile / warp fold / fold weights), m, l, flag, row tables
-    static constexpr int kScratchBytes = (16 * DH + 2 * 16 + 8 + 2 * kAttMaxItems + 8) * 4;
+    // scratch: one [16][DH + 8] fp32 slot (Q tile / warp fold; the padding keeps the fold's
+    // fragment-shaped accesses off a single bank), m, l, flag, row tables
+    static constexpr int kFoldStride = DH + 8;
+    static constexpr int kScratchBytes = (16 * kFoldStride + 2 * 16 + 8 + 2 * kAttMaxItems + 8) * 4;
     static constexpr int kSmemBytes = kStages * kStageBytes + 1024 + 128 + kScratchBytes;
 };
 
@@ -78,6 +80,12 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t *>(&v);
 }
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2, int c3) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];" ::"r"(dst),
+        "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        : "memory");
+}
 __device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
 template <int DH>
@@ -91,8 +99,9 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
     uint32_t bars = tiles + STAGES * Cfg::kStageBytes;
     auto full_bar = [&](int s) { return bars + 8u * s; };
     auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
-    float *sc_o = reinterpret_cast<float *>(gen + STAGES * Cfg::kStageBytes + 128);  // [16][DH]
-    float *sc_m = sc_o + 16 * DH;                                                   // [16]
+    constexpr int FS = Cfg::kFoldStride;
+    float *sc_o = reinterpret_cast<float *>(gen + STAGES * Cfg::kStageBytes + 128);  // [16][FS]
+    float *sc_m = sc_o + 16 * FS;                                                   // [16]
     float *sc_l = sc_m + 16;                                                        // [16]
     int *flag = reinterpret_cast<int *>(sc_l + 16);                                 // [0] last?, [1] longest pair
     int *cum = flag + 8;                 // [items + 1] prefix of tiles per row
@@ -145,41 +154,41 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
     while (cum[item + 1] * p.n_kv <= u0) item++;
 
     if (warp == kAttWarps) {
-        // ---- producer: walks the same segments as the consumers; page table walk + TMA
-        if (lane == 0) {
-            tma_prefetch_desc(&tmKV);
-            bool ok = true;
-            int it = 0;
-            for (int u = u0; u < u1 && ok;) {
-                int ui = cum[item + 1] - cum[item], base = cum[item] * p.n_kv;
-                int g = (u - base) / ui, t0 = (u - base) % ui;
-                int pair_end = base + (g + 1) * ui, t1 = t0 + min(u1, pair_end) - u;
-                int seq = p.rm.seq(item), total_pages = (nk_s[item] + 15) >> 4;
-                for (int t = t0; t < t1 && ok; t++, it++) {
-                    int s = it % STAGES;
+        // ---- producer: walks the same segments as the consumers.  Lane 0 waits for the stage and
+        // arms its barrier; up to four lanes then issue one box each (a page's K and V, both
+        // 64-column pieces: 8 KB at d_h = 128), each after its own page-table lookup.
+        if (lane == 0) tma_prefetch_desc(&tmKV);
+        bool ok = true;
+        int it = 0;
+        for (int u = u0; u < u1 && ok;) {
+            int ui = cum[item + 1] - cum[item], base = cum[item] * p.n_kv;
+            int g = (u - base) / ui, t0 = (u - base) % ui;
+            int pair_end = base + (g + 1) * ui, t1 = t0 + min(u1, pair_end) - u;
+            int seq = p.rm.seq(item), total_pages = (nk_s[item] + 15) >> 4;
+            for (int t = t0; t < t1; t++, it++) {
+                int s = it % STAGES;
+                int p0 = t * 4, np = min(4, total_pages - p0);
+                if (lane == 0) {
                     if (it >= STAGES) ok = mbar_wait(empty_bar(s), ((it / STAGES) - 1) & 1);
-                    if (!ok) break;
-                    int p0 = t * 4, np = min(4, total_pages - p0);
-                    mbar_expect_tx(full_bar(s), (uint32_t)np * 2 * Cfg::kPageBytes);
-                    uint32_t kdst = tiles + s * Cfg::kStageBytes, vdst = kdst + 4 * Cfg::kPageBytes;
-                    for (int j = 0; j < np; j++) {
-                        int page = p.page_table[(size_t)seq * p.pt_stride + p0 + j];
-                        if (page < 0 || page >= p.num_pages) {
-                            report(p.status, kStatusBadPage, page);
-                            page = 0;
-                        }
-                        int row = (int)(((long long)page * p.n_kv + g) * 16);
-                        for (int h = 0; h < HALVES; h++) {
-                            tma_load_2d(kdst + (j * HALVES + h) * 2048, &tmKV, full_bar(s), h * 64, (int)(p.k_row0 + row));
-                            tma_load_2d(vdst + (j * HALVES + h) * 2048, &tmKV, full_bar(s), h * 64, (int)(p.v_row0 + row));
-                        }
-                    }
+                    if (ok) mbar_expect_tx(full_bar(s), (uint32_t)np * 2 * Cfg::kPageBytes);
                 }
-                u += t1 - t0;
-                if (u == pair_end && g == p.n_kv - 1) item++;
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) break;
+                if (lane < np) {
+                    int page = __ldg(p.page_table + (size_t)seq * p.pt_stride + p0 + lane);
+                    if (page < 0 || page >= p.num_pages) {
+                        report(p.status, kStatusBadPage, page);
+                        page = 0;
+                    }
+                    int row = (int)(((long long)page * p.n_kv + g) * 16);
+                    tma_load_4d(tiles + s * Cfg::kStageBytes + lane * 2 * Cfg::kPageBytes, &tmKV, full_bar(s), 0, 0,
+                                (int)(p.k_row0 + row), 0);
+                }
             }
-            if (!ok) report(p.status, kStatusWaitExpired, 300);
+            u += t1 - t0;
+            if (u == pair_end && g == p.n_kv - 1) item++;
         }
+        if (!ok && lane == 0) report(p.status, kStatusWaitExpired, 300);
         return;
     }
 
@@ -233,14 +242,14 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
             if (!ok) break;
             int valid = min(16, nkeys - (t * kAttTile + warp * 16));  // valid tokens in this warp's page
             if (valid > 0) {
-                uint32_t kpage = tiles + s * Cfg::kStageBytes + warp * HALVES * 2048;
-                uint32_t vpage = kpage + 4 * Cfg::kPageBytes;
+                // a page's box: K then V, each [16 rows][DH], the 128-byte pieces of a row swizzled
+                uint32_t kpage = tiles + s * Cfg::kStageBytes + warp * 2 * Cfg::kPageBytes;
+                uint32_t vpage = kpage + Cfg::kPageBytes;
                 if (valid < 16) {
                     // stale slots past the end of the sequence: their scores are masked below, and
                     // their V rows are zeroed here so that 0 * garbage cannot produce a NaN
                     for (int idx = lane; idx < (16 - valid) * HALVES * 8; idx += 32) {
-                        int r = valid + idx / (HALVES * 8), rest = idx % (HALVES * 8);
-                        uint32_t a = vpage + (rest / 8) * 2048 + r * 128 + (rest % 8) * 16;
+                        uint32_t a = vpage + valid * HALVES * 128 + idx * 16;
                         asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(a), "r"(0u) : "memory");
                     }
                     __syncwarp();
@@ -253,7 +262,8 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
 #pragma unroll
                     for (int ks = 0; ks < KS; ks++) {
                         int chunk = ks * 2 + cb;  // 16-byte chunk index within the row
-                        uint32_t a = kpage + (chunk >> 3) * 2048 + r * 128 + (((chunk & 7) ^ (r & 7)) << 4);
+                        int sg = r * HALVES + (chunk >> 3);
+                        uint32_t a = kpage + sg * 128 + (((chunk & 7) ^ (sg & 7)) << 4);
                         uint32_t kb[4];
                         ldsm_x4(a, kb);
                         mma_bf16(sacc[0], qa[ks], kb[0], kb[1]);
@@ -312,7 +322,8 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
 #pragma unroll
                     for (int np = 0; np < NB / 2; np++) {
                         int chunk = np * 2 + cb;
-                        uint32_t a = vpage + (chunk >> 3) * 2048 + r * 128 + (((chunk & 7) ^ (r & 7)) << 4);
+                        int sg = r * HALVES + (chunk >> 3);
+                        uint32_t a = vpage + sg * 128 + (((chunk & 7) ^ (sg & 7)) << 4);
                         uint32_t vb[4];
                         ldsm_x4_trans(a, vb);
                         mma_bf16(o[np * 2], pa, vb[0], vb[1]);
@@ -339,8 +350,8 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
             auto put = [&]() {
 #pragma unroll
                 for (int nb = 0; nb < NB; nb++) {
-                    *reinterpret_cast<float2 *>(sc_o + (size_t)r0 * DH + nb * 8 + c) = make_float2(o[nb][0], o[nb][1]);
-                    *reinterpret_cast<float2 *>(sc_o + (size_t)(r0 + 8) * DH + nb * 8 + c) = make_float2(o[nb][2], o[nb][3]);
+                    *reinterpret_cast<float2 *>(sc_o + (size_t)r0 * FS + nb * 8 + c) = make_float2(o[nb][0], o[nb][1]);
+                    *reinterpret_cast<float2 *>(sc_o + (size_t)(r0 + 8) * FS + nb * 8 + c) = make_float2(o[nb][2], o[nb][3]);
                 }
                 if ((lane & 3) == 0) {
                     sc_m[r0] = m_run[0];
@@ -361,7 +372,7 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
                     m_run[h] = M;
 #pragma unroll
                     for (int nb = 0; nb < NB; nb++) {
-                        float2 ob = *reinterpret_cast<const float2 *>(sc_o + (size_t)r * DH + nb * 8 + c);
+                        float2 ob = *reinterpret_cast<const float2 *>(sc_o + (size_t)r * FS + nb * 8 + c);
                         o[nb][2 * h] = o[nb][2 * h] * fa + ob.x * fb;
                         o[nb][2 * h + 1] = o[nb][2 * h + 1] * fa + ob.y * fb;
                     }
@@ -379,67 +390,112 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
                 for (int h = 0; h < 2; h++) {
                     int q = r0 + 8 * h;
                     if (q < nq_act) {
+                        if (nseg == 1) {
+                            // the pair's only segment: normalise and write the head's output
+                            int row = q < p.G ? item : Bc + item;
+                            int hq = g * p.G + (q < p.G ? q : q - p.G);
+                            size_t ob = (size_t)row * q_dim + (size_t)hq * DH;
+                            float inv = 1.f / l_run[h];
 #pragma unroll
-                        for (int nb = 0; nb < NB; nb++)
-                            *reinterpret_cast<float2 *>(out + (size_t)q * (DH + 2) + nb * 8 + c) =
-                                make_float2(o[nb][2 * h], o[nb][2 * h + 1]);
-                        if ((lane & 3) == 0) {
-                            out[(size_t)q * (DH + 2) + DH] = m_run[h];  // base-2 units
-                            out[(size_t)q * (DH + 2) + DH + 1] = l_run[h];
+                            for (int nb = 0; nb < NB; nb++)
+#pragma unroll
+                                for (int e = 0; e < 2; e++) {
+                                    float x = o[nb][2 * h + e] * inv;
+                                    __nv_bfloat16 hi = __float2bfloat16_rn(x);
+                                    p.Ob[ob + nb * 8 + c + e] = hi;
+                                    if (p.lo_off) p.Ob[ob + nb * 8 + c + e + p.lo_off] = __float2bfloat16_rn(x - __bfloat162float(hi));
+                                }
+                        } else {
+#pragma unroll
+                            for (int nb = 0; nb < NB; nb++)
+                                *reinterpret_cast<float2 *>(out + (size_t)q * (DH + 2) + nb * 8 + c) =
+                                    make_float2(o[nb][2 * h], o[nb][2 * h + 1]);
+                            if ((lane & 3) == 0) {
+                                out[(size_t)q * (DH + 2) + DH] = m_run[h];  // base-2 units
+                                out[(size_t)q * (DH + 2) + DH + 1] = l_run[h];
+                            }
                         }
                     }
                 }
+                if (nseg > 1) __threadfence();
             }
         }
         // ---- the last segment of this pair to arrive folds all of them in segment order
-        __threadfence();
-        consumer_sync();
-        if (tid == 0) {
-            int last = 1;
-            if (nseg > 1) {
+        int is_last = 0;
+        if (nseg > 1) {
+            consumer_sync();
+            if (tid == 0) {
                 int *tk = p.tickets + pair;
                 int tkt = atomicAdd(tk, 1);
-                last = tkt == nseg - 1;
-                if (last) atomicExch(tk, 0);
-            }
-            flag[0] = last;
-        }
-        consumer_sync();
-        if (flag[0]) {
-            __threadfence();
-            const float *pbase = p.part + (size_t)(first_cta + pair) * 16 * (DH + 2);
-            float *wt = sc_o, *ml = sc_o + 16 * kAttMaxSeg;  // fold weights [16][32], (m, l) staging
-            for (int t = tid; t < nq_act * nseg; t += 128) {  // all (m, l) pairs in one round of loads
-                int q = t / nseg, s2 = t % nseg;
-                const float *pp = pbase + ((size_t)s2 * 16 + q) * (DH + 2) + DH;
-                wt[q * kAttMaxSeg + s2] = __ldcg(pp);
-                ml[q * kAttMaxSeg + s2] = __ldcg(pp + 1);
-            }
-            consumer_sync();
-            if (tid < nq_act) {
-                float M = -INFINITY, L = 0.f;
-                for (int s2 = 0; s2 < nseg; s2++) M = fmaxf(M, wt[tid * kAttMaxSeg + s2]);
-                for (int s2 = 0; s2 < nseg; s2++) {
-                    float ms = wt[tid * kAttMaxSeg + s2];
-                    float f = ms == -INFINITY ? 0.f : exp2f(ms - M);
-                    L += ml[tid * kAttMaxSeg + s2] * f;
-                    wt[tid * kAttMaxSeg + s2] = f;
+                int last = tkt == nseg - 1;
+                if (last) {
+                    atomicExch(tk, 0);
+                    __threadfence();
                 }
-                float inv = 1.f / L;
-                for (int s2 = 0; s2 < nseg; s2++) wt[tid * kAttMaxSeg + s2] *= inv;
+                flag[0] = last;
             }
             consumer_sync();
-            for (int idx = tid; idx < nq_act * DH; idx += 128) {
-                int q = idx / DH, e = idx % DH;
-                float x = 0.f;
-                for (int s2 = 0; s2 < nseg; s2++)
-                    x = fmaf(__ldcg(pbase + ((size_t)s2 * 16 + q) * (DH + 2) + e), wt[q * kAttMaxSeg + s2], x);
-                int row = q < p.G ? item : Bc + item;
-                int h = g * p.G + (q < p.G ? q : q - p.G);
-                size_t o_idx = (size_t)row * q_dim + (size_t)h * DH + e;
-                __nv_bfloat16 hi = __float2bfloat16_rn(x);
-                p.Ob[o_idx] = hi;
-                if (p.lo_off) p.Ob[o_idx + p.lo_off] = __float2bfloat16_rn(x - __bfloat162float(hi));
+            is_last = flag[0];
+        }
+        if (is_last) {
+            const float *pbase = p.part + (size_t)(first_cta + pair) * 16 * (DH + 2);
+            for (int idx0 = tid; idx0 < nq_act * DH; idx0 += 2 * 128) {
+                // two outputs per thread, eight segments of each in flight
+                const float *pq[2];
+                float M[2] = {-INFINITY, -INFINITY}, L[2] = {0.f, 0.f}, X[2] = {0.f, 0.f};
+                bool act[2];
+                int ee[2];
+#pragma unroll
+                for (int a = 0; a < 2; a++) {
+                    int idx = idx0 + a * 128;
+                    act[a] = idx < nq_act * DH;
+                    int q = act[a] ? idx / DH : 0;
+                    ee[a] = act[a] ? idx % DH : 0;
+                    pq[a] = pbase + (size_t)q * (DH + 2);
+                }
+                for (int sb = 0; sb < nseg; sb += 8) {
+                    float mv[2][8], lv[2][8], ov[2][8];
+#pragma unroll
+                    for (int a = 0; a < 2; a++)
+#pragma unroll
+                        for (int j = 0; j < 8; j++) {
+                            bool on = act[a] && sb + j < nseg;
+                            const float *pp = pq[a] + (size_t)(sb + j) * 16 * (DH + 2);
+                            mv[a][j] = on ? __ldcg(pp + DH) : -INFINITY;
+                            lv[a][j] = on ? __ldcg(pp + DH + 1) : 0.f;
+                            ov[a][j] = on ? __ldcg(pp + ee[a]) : 0.f;
+                        }
+#pragma unroll
+                    for (int a = 0; a < 2; a++) {
+                        float Mn = M[a];
+#pragma unroll
+                        for (int j = 0; j < 8; j++) Mn = fmaxf(Mn, mv[a][j]);
+                        float sc = M[a] == -INFINITY ? 0.f : exp2f(M[a] - Mn);
+                        L[a] *= sc;
+                        X[a] *= sc;
+#pragma unroll
+                        for (int j = 0; j < 8; j++) {
+                            float f = mv[a][j] == -INFINITY ? 0.f : exp2f(mv[a][j] - Mn);
+                            L[a] = fmaf(lv[a][j], f, L[a]);
+                            X[a] = fmaf(ov[a][j], f, X[a]);
+                        }
+                        M[a] = Mn;
+                    }
+                }
+#pragma unroll
+                for (int a = 0; a < 2; a++) {
+                    int idx = idx0 + a * 128;
+                    if (act[a]) {
+                        int q = idx / DH;
+                        int row = q < p.G ? item : Bc + item;
+                        int h = g * p.G + (q < p.G ? q : q - p.G);
+                        size_t o_idx = (size_t)row * q_dim + (size_t)h * DH + ee[a];
+                        float x = X[a] / L[a];
+                        __nv_bfloat16 hi = __float2bfloat16_rn(x);
+                        p.Ob[o_idx] = hi;
+                        if (p.lo_off) p.Ob[o_idx + p.lo_off] = __float2bfloat16_rn(x - __bfloat162float(hi));
+                    }
+                }
             }
         }
         u += t1 - t0;
@@ -448,15 +504,18 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
     DBT_TL_END("attention");
 }
 
-// The whole pool as one 2-D bf16 tensor [rows][head_dim], rows = (layer, K|V, page, head, slot).
-inline bool make_kv_map(CUtensorMap *map, const void *pool, uint64_t total_rows, int head_dim) {
+// The K/V pool as a 4-D bf16 tensor (64 columns, 64-column piece of a row, row, K|V plane of a
+// layer); rows = (layer, K|V, page, head, slot).  One box {64, d_h/64, 16, 2} brings a page's K and V
+// of one KV head.  The row extent stops one plane short so that plane 1 of the last layer stays
+// inside the allocation.
+inline bool make_kv_page_map(CUtensorMap *map, const void *pool, uint64_t total_rows, uint64_t plane_rows, int head_dim) {
     EncodeTiledFn fn = encode_tiled_fn();
-    if (!fn || total_rows >= (1ull << 31)) return false;
-    cuuint64_t dims[2] = {(cuuint64_t)head_dim, total_rows};
-    cuuint64_t strides[1] = {(cuuint64_t)head_dim * 2};
-    cuuint32_t box[2] = {64, 16};
-    cuuint32_t estr[2] = {1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(pool), dims, strides, box, estr,
+    if (!fn || total_rows >= (1ull << 31) || total_rows <= plane_rows) return false;
+    cuuint64_t dims[4] = {64, (cuuint64_t)head_dim / 64, total_rows - plane_rows, 2};
+    cuuint64_t strides[3] = {128, (cuuint64_t)head_dim * 2, plane_rows * (cuuint64_t)head_dim * 2};
+    cuuint32_t box[4] = {64, (cuuint32_t)head_dim / 64, 16, 2};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(pool), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }

@@ -14,10 +14,59 @@ __device__ __forceinline__ void store_split(__nv_bfloat16 *dst, size_t idx, size
     if (lo_off) dst[idx + lo_off] = __float2bfloat16_rn(x - __bfloat162float(hi));
 }
 
+// Sum of one output's split-K partials, in split order; the loads go out four at a time so that
+// the sum costs one or two L2 round trips instead of one per split.
 __device__ __forceinline__ float sum_splits(const float *P, size_t split_stride, int nsplit, size_t off) {
+    const float *p = P + off;
     float m = 0.f;
-    for (int s = 0; s < nsplit; s++) m += P[(size_t)s * split_stride + off];
+    int s = 0;
+    for (; s + 4 <= nsplit; s += 4) {
+        float a = __ldcg(p), b = __ldcg(p + split_stride), c = __ldcg(p + 2 * split_stride), e = __ldcg(p + 3 * split_stride);
+        m += a;
+        m += b;
+        m += c;
+        m += e;
+        p += 4 * split_stride;
+    }
+    if (s + 2 <= nsplit) {
+        float a = __ldcg(p), b = __ldcg(p + split_stride);
+        m += a;
+        m += b;
+        p += 2 * split_stride;
+        s += 2;
+    }
+    if (s < nsplit) m += __ldcg(p);
     return m;
+}
+
+// The same for K outputs at once: the loads of all K outputs (two splits of each) are in flight
+// together.  Each output is still added in split order.
+template <int K>
+__device__ __forceinline__ void sum_splits_k(const float *P, size_t split_stride, int nsplit, const size_t (&off)[K],
+                                             float (&out)[K]) {
+#pragma unroll
+    for (int k = 0; k < K; k++) out[k] = 0.f;
+    int s = 0;
+    for (; s + 2 <= nsplit; s += 2) {
+        float a[K], b[K];
+#pragma unroll
+        for (int k = 0; k < K; k++) {
+            a[k] = __ldcg(P + (size_t)s * split_stride + off[k]);
+            b[k] = __ldcg(P + (size_t)(s + 1) * split_stride + off[k]);
+        }
+#pragma unroll
+        for (int k = 0; k < K; k++) {
+            out[k] += a[k];
+            out[k] += b[k];
+        }
+    }
+    if (s < nsplit) {
+        float a[K];
+#pragma unroll
+        for (int k = 0; k < K; k++) a[k] = __ldcg(P + (size_t)s * split_stride + off[k]);
+#pragma unroll
+        for (int k = 0; k < K; k++) out[k] += a[k];
+    }
 }
 
 // 1/rms of a row from its per-tile shares of sum(x^2) (ss[t][ss_ld], summed in tile order);
@@ -91,16 +140,19 @@ __global__ void __launch_bounds__(1024) resid_norm_kernel(float *S, const float 
     float ss1 = 0.f, ss2 = 0.f;
     for (int i = threadIdx.x; i < d; i += blockDim.x) {
         float v1 = S[(size_t)r1 * d + i], m1 = 0.f;
+        float v2 = grouped ? S[(size_t)r2 * d + i] : 0.f;
+        float sm[2] = {0.f, 0.f};
         if (mode != 0) {
-            m1 = sum_splits(P, split_stride, nsplit, (size_t)r1 * d + i);
+            const size_t offs[2] = {(size_t)r1 * d + i, (size_t)(grouped ? r2 : r1) * d + i};
+            sum_splits_k<2>(P, split_stride, nsplit, offs, sm);
+            m1 = sm[0];
             v1 += m1;
             S[(size_t)r1 * d + i] = v1;
         }
         ss1 += v1 * v1;
         if (grouped) {
-            float v2 = S[(size_t)r2 * d + i];
             if (mode != 0) {
-                float m2 = sum_splits(P, split_stride, nsplit, (size_t)r2 * d + i);
+                float m2 = sm[1];
                 if (mode == 2) m2 += coup_c[i] * m1;
                 v2 += m2;
                 S[(size_t)r2 * d + i] = v2;
@@ -156,14 +208,17 @@ __global__ void __launch_bounds__(64) qkv_epilogue_kernel(
     const float rs1 = row_scale(ss, ss_tiles, ss_ld, item, d_norm, eps);  // 1/rms when the GEMM input was g*S
     if (hh < n_q) {
         int o0 = hh * dh + i, o1 = o0 + half;
-        float x0 = rs1 * sum_splits(P, split_stride, nsplit, p1 + o0), x1 = rs1 * sum_splits(P, split_stride, nsplit, p1 + o1);
+        const size_t offs[4] = {p1 + o0, p1 + o1, grouped ? p2 + o0 : p1 + o0, grouped ? p2 + o1 : p1 + o1};
+        float sm[4];
+        sum_splits_k<4>(P, split_stride, nsplit, offs, sm);
+        float x0 = rs1 * sm[0], x1 = rs1 * sm[1];
         float r0 = x0 * t.x - x1 * t.y, r1 = x1 * t.x + x0 * t.y;
         float *q1 = Q + (size_t)item * q_dim;
         q1[o0] = r0;
         q1[o1] = r1;
         if (grouped) {
             const float rs2 = row_scale(ss, ss_tiles, ss_ld, Bc + item, d_norm, eps);
-            float y0 = rs2 * sum_splits(P, split_stride, nsplit, p2 + o0), y1 = rs2 * sum_splits(P, split_stride, nsplit, p2 + o1);
+            float y0 = rs2 * sm[2], y1 = rs2 * sm[3];
             float *q2 = Q + (size_t)(Bc + item) * q_dim;
             q2[o0] = (y0 * t.x - y1 * t.y) + coup_a[o0] * r0;
             q2[o1] = (y1 * t.x + y0 * t.y) + coup_a[o1] * r1;
@@ -180,11 +235,14 @@ __global__ void __launch_bounds__(64) qkv_epilogue_kernel(
     int slot = pos % page_size;
     size_t base = (((size_t)page * n_kv + gk) * page_size + slot) * dh;
     size_t ko = p1 + q_dim + gk * dh + i, vo = ko + kv_dim;
-    float x0 = rs1 * sum_splits(P, split_stride, nsplit, ko), x1 = rs1 * sum_splits(P, split_stride, nsplit, ko + half);
+    const size_t offs[4] = {ko, ko + half, vo, vo + half};
+    float sm[4];
+    sum_splits_k<4>(P, split_stride, nsplit, offs, sm);
+    float x0 = rs1 * sm[0], x1 = rs1 * sm[1];
     store1(kpool + base + i, x0 * t.x - x1 * t.y);
     store1(kpool + base + i + half, x1 * t.x + x0 * t.y);
-    store1(vpool + base + i, rs1 * sum_splits(P, split_stride, nsplit, vo));
-    store1(vpool + base + i + half, rs1 * sum_splits(P, split_stride, nsplit, vo + half));
+    store1(vpool + base + i, rs1 * sm[2]);
+    store1(vpool + base + i + half, rs1 * sm[3]);
 }
 
 // After the gate|up GEMM: H = SiLU(gate) * up; H~_2 = H_2 + b * H_1 (Eq. mlp); bf16 out for
@@ -201,12 +259,15 @@ __global__ void __launch_bounds__(256) swiglu_couple_kernel(const float *P, int 
     if (f >= F) return;
     size_t p1 = (size_t)b * 2 * F + f;
     const float rs1 = row_scale(ss, ss_tiles, ss_ld, b, d_norm, eps);
-    float h1 = silu(rs1 * sum_splits(P, split_stride, nsplit, p1)) * (rs1 * sum_splits(P, split_stride, nsplit, p1 + F));
+    size_t p2 = grouped ? (size_t)(Bc + b) * 2 * F + f : p1;
+    const size_t offs[4] = {p1, p1 + F, p2, p2 + F};
+    float sm[4];
+    sum_splits_k<4>(P, split_stride, nsplit, offs, sm);
+    float h1 = silu(rs1 * sm[0]) * (rs1 * sm[1]);
     store_split(Hb, (size_t)b * F + f, lo_off, h1);
     if (grouped) {
-        size_t p2 = (size_t)(Bc + b) * 2 * F + f;
         const float rs2 = row_scale(ss, ss_tiles, ss_ld, Bc + b, d_norm, eps);
-        float h2 = silu(rs2 * sum_splits(P, split_stride, nsplit, p2)) * (rs2 * sum_splits(P, split_stride, nsplit, p2 + F));
+        float h2 = silu(rs2 * sm[2]) * (rs2 * sm[3]);
         if (coup_b) h2 += coup_b[f] * h1;
         store_split(Hb, (size_t)(Bc + b) * F + f, lo_off, h2);
     }

@@ -95,12 +95,6 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map
         "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
         : "memory");
 }
-__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2, int c3) {
-    asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];" ::"r"(dst),
-        "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
-        : "memory");
-}
 __device__ __forceinline__ void worker_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
 // stream-K bookkeeping of one GEMM phase
@@ -1284,22 +1278,7 @@ mega_decode_kernel(const MegaPlan *__restrict__ pl, const int32_t *tokens, int32
     }
 }
 
-// ---- host side: the two tensor maps only this kernel uses ---------------------------------
-
-// The K/V pool as a 4-D tensor (64 columns, 64-column piece of a row, row, K|V plane of a layer):
-// one box {64, d_h/64, 16, 2} brings a page's K and V of one KV head.  The row extent stops one
-// plane short so that plane 1 of the last layer stays inside the allocation.
-inline bool make_kv_page_map(CUtensorMap *map, const void *pool, uint64_t total_rows, uint64_t plane_rows, int head_dim) {
-    EncodeTiledFn fn = encode_tiled_fn();
-    if (!fn || total_rows >= (1ull << 31) || total_rows <= plane_rows) return false;
-    cuuint64_t dims[4] = {64, (cuuint64_t)head_dim / 64, total_rows - plane_rows, 2};
-    cuuint64_t strides[3] = {128, (cuuint64_t)head_dim * 2, plane_rows * (cuuint64_t)head_dim * 2};
-    cuuint32_t box[4] = {64, (cuuint32_t)head_dim / 64, 16, 2};
-    cuuint32_t estr[4] = {1, 1, 1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(pool), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
+// ---- host side: the tensor map only this kernel uses ---------------------------------
 
 // A GEMM input held as two bf16 planes [2][plane_rows][K]: one box {64, n_tile, 2} brings a k-tile
 // of the first n_tile rows of both planes.
