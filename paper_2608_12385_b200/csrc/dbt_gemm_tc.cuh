@@ -33,6 +33,11 @@ struct TcSeg {
 };
 
 struct TcParams {
+    // up to three byte ranges (the next GEMM's weights) that this launch asks the L2 to fetch while it
+    // and the small kernels after it run: HBM is otherwise idle between the GEMMs of a decode step
+    const char *pf_ptr[3];
+    unsigned long long pf_bytes[3];
+    int x3d;  // tmX is the 3-D {64, N_TILE, 2} view of a two-plane input: one box per stage
     TcSeg seg[3];
     int nseg;
     int K;
@@ -60,6 +65,16 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 // Bounded wait on a phase parity; false when the limit expired.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
     uint32_t done = 0;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(done)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    if (done) return true;  // the common case costs one probe and no clock read
     long long t0 = clock64();
     while (true) {
         asm volatile(
@@ -80,6 +95,12 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];" ::"r"(dst),
+        "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
         : "memory");
 }
 __device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1,
@@ -211,6 +232,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
     uint32_t tmem_base = *tmem_holder;
     pdl_launch_dependents();
 
+    if (warp == 2 && lane == 0) {
+        constexpr unsigned long long kChunk = 16384;
+        const unsigned ncta = gridDim.x * gridDim.y * gridDim.z;
+        const unsigned cid = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);
+        for (int j = 0; j < 3; j++) {
+            const unsigned long long bytes = p.pf_bytes[j];
+            for (unsigned long long off = (unsigned long long)cid * kChunk; off < bytes; off += (unsigned long long)ncta * kChunk) {
+                unsigned sz = (unsigned)min(kChunk, bytes - off) & ~15u;
+                if (sz) asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p.pf_ptr[j] + off), "r"(sz) : "memory");
+            }
+        }
+    }
     bool ok = true;
     if (warp == 0 && lane == 0) {
         // ---- TMA producer.  Weight tiles do not depend on the previous kernel: the first
@@ -220,6 +253,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
         int npre = min(STAGES, nkt);
         const uint32_t tx = kTcABytes + p.parts * Cfg::kBBytes;
         auto load_x = [&](int s, int kt) {
+            if (p.x3d) {
+                tma_load_3d(tiles + s * Cfg::kStageBytes + kTcABytes, &tmX, full_bar(s), kt * kTcK, x_row0, 0);
+                return;
+            }
             for (int part = 0; part < p.parts; part++)
                 for (int j = 0; j < N_TILE / 16; j++)
                     tma_load_2d(tiles + s * Cfg::kStageBytes + kTcABytes + part * Cfg::kBBytes + j * 2048, &tmX,
@@ -356,6 +393,20 @@ inline bool make_bf16_map(CUtensorMap *map, const void *base, uint64_t rows, uin
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
+}
+
+// A GEMM input held as two bf16 planes [2][plane_rows][K]: one box {64, n_tile, 2} brings a k-tile
+// of n_tile rows of both planes.
+inline bool make_act_map(CUtensorMap *map, const void *base, uint64_t plane_rows, uint64_t K, uint32_t n_tile) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    cuuint64_t dims[3] = {K, plane_rows, 2};
+    cuuint64_t strides[2] = {K * 2, plane_rows * K * 2};
+    cuuint32_t box[3] = {(cuuint32_t)kTcK, n_tile, 2};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 }  // namespace dbt

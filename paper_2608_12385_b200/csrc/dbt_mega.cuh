@@ -89,12 +89,6 @@ __device__ __forceinline__ unsigned ld_acquire_u32(const unsigned *p) {
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
 }
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2) {
-    asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];" ::"r"(dst),
-        "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
-        : "memory");
-}
 __device__ __forceinline__ void worker_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
 // stream-K bookkeeping of one GEMM phase
@@ -1276,22 +1270,6 @@ mega_decode_kernel(const MegaPlan *__restrict__ pl, const int32_t *tokens, int32
             atomicExch(pl->done_count, 0u);
         }
     }
-}
-
-// ---- host side: the tensor map only this kernel uses ---------------------------------
-
-// A GEMM input held as two bf16 planes [2][plane_rows][K]: one box {64, n_tile, 2} brings a k-tile
-// of the first n_tile rows of both planes.
-inline bool make_act_map(CUtensorMap *map, const void *base, uint64_t plane_rows, uint64_t K, uint32_t n_tile) {
-    EncodeTiledFn fn = encode_tiled_fn();
-    if (!fn) return false;
-    cuuint64_t dims[3] = {K, plane_rows, 2};
-    cuuint64_t strides[2] = {K * 2, plane_rows * K * 2};
-    cuuint32_t box[3] = {(cuuint32_t)kTcK, n_tile, 2};
-    cuuint32_t estr[3] = {1, 1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 }  // namespace dbt
