@@ -634,7 +634,12 @@ dbt_status run_attention_mma(dbt_model *m, const RowMap &rm, int grouped, int la
     p.status = w.status;
     if (items > kAttMaxItems) return fail(m, DBT_ERR_CAPACITY, "attention rows %d exceed %d", items, kAttMaxItems);
     dim3 grid(2 * m->num_sms);  // two resident CTAs per SM; each takes an equal share of all K/V tiles
-    LAUNCH(m, "attention", kv_bytes, attn_mma_kernel<DH>, grid, 160, AttCfg<DH>::kSmemBytes, m->map_kv, p);
+    // up to 8 query rows per KV head over both paths: the transposed-product variant (fixed per
+    // model, so that grouped and primary-only steps run the same arithmetic on the primary rows)
+    if (2 * G <= 8)
+        LAUNCH(m, "attention", kv_bytes, (attn_mma_kernel<DH, true>), grid, 160, AttCfg<DH>::kSmemBytes, m->map_kv, p);
+    else
+        LAUNCH(m, "attention", kv_bytes, (attn_mma_kernel<DH, false>), grid, 160, AttCfg<DH>::kSmemBytes, m->map_kv, p);
     return DBT_OK;
 }
 
@@ -1419,9 +1424,13 @@ bool setup_tc(dbt_model *m) {
     m->att_fast = ok && !(fa && strcmp(fa, "simt") == 0) &&
                   make_kv_page_map(&m->map_kv, m->kv_pool, (uint64_t)c.n_layers * 2 * c.num_pages * c.n_kv_heads * c.page_size,
                                    (uint64_t)c.num_pages * c.n_kv_heads * c.page_size, c.head_dim) &&
-                  cudaFuncSetAttribute(attn_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                  cudaFuncSetAttribute(attn_mma_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        AttCfg<128>::kSmemBytes) == cudaSuccess &&
-                  cudaFuncSetAttribute(attn_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                  cudaFuncSetAttribute(attn_mma_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       AttCfg<128>::kSmemBytes) == cudaSuccess &&
+                  cudaFuncSetAttribute(attn_mma_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       AttCfg<64>::kSmemBytes) == cudaSuccess &&
+                  cudaFuncSetAttribute(attn_mma_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        AttCfg<64>::kSmemBytes) == cudaSuccess;
     const char *fu = getenv("DBT_FUSED");
     // Opt-in (DBT_FUSED=1): measured slower than the separate elementwise kernels at batch 16

@@ -76,6 +76,13 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], 
         : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
+// Transpose of an 8x8 matrix of 16-bit elements held one row pair per lane (the layout of an
+// accumulator's 8x8 block packed to bf16).
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
+    uint32_t d;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+    return d;
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t *>(&v);
@@ -88,7 +95,7 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map
 }
 __device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
-template <int DH>
+template <int DH, bool NARROW>
 __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant__ CUtensorMap tmKV, AttnParams p) {
     using Cfg = AttCfg<DH>;
     constexpr int STAGES = Cfg::kStages, HALVES = Cfg::kHalves, KS = DH / 16, NB = DH / 8;
@@ -216,208 +223,407 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
             reinterpret_cast<float4 *>(sc_o)[idx] = v;
         }
         consumer_sync();
-        uint32_t qa[KS][4];
-        {
-            int r0 = lane >> 2, c = (lane & 3) * 2;
-            const float *q0 = sc_o + r0 * DH, *q1 = sc_o + (r0 + 8) * DH;
-#pragma unroll
-            for (int ks = 0; ks < KS; ks++) {
-                int k = ks * 16 + c;
-                qa[ks][0] = pack_bf16(q0[k] * qscale, q0[k + 1] * qscale);
-                qa[ks][1] = pack_bf16(q1[k] * qscale, q1[k + 1] * qscale);
-                qa[ks][2] = pack_bf16(q0[k + 8] * qscale, q0[k + 9] * qscale);
-                qa[ks][3] = pack_bf16(q1[k + 8] * qscale, q1[k + 9] * qscale);
-            }
-        }
-        consumer_sync();  // everyone has its fragments: the scratch is free again
-        float o[NB][4];
-#pragma unroll
-        for (int nb = 0; nb < NB; nb++) o[nb][0] = o[nb][1] = o[nb][2] = o[nb][3] = 0.f;
-        float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
-
-        for (int t = t0; t < t1 && ok; t++, it++) {
-            int s = it % STAGES;
-            ok = mbar_wait(full_bar(s), (it / STAGES) & 1);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            int valid = min(16, nkeys - (t * kAttTile + warp * 16));  // valid tokens in this warp's page
-            if (valid > 0) {
-                // a page's box: K then V, each [16 rows][DH], the 128-byte pieces of a row swizzled
-                uint32_t kpage = tiles + s * Cfg::kStageBytes + warp * 2 * Cfg::kPageBytes;
-                uint32_t vpage = kpage + Cfg::kPageBytes;
-                if (valid < 16) {
-                    // stale slots past the end of the sequence: their scores are masked below, and
-                    // their V rows are zeroed here so that 0 * garbage cannot produce a NaN
-                    for (int idx = lane; idx < (16 - valid) * HALVES * 8; idx += 32) {
-                        uint32_t a = vpage + valid * HALVES * 128 + idx * 16;
-                        asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(a), "r"(0u) : "memory");
-                    }
-                    __syncwarp();
-                }
-                // S = Q K^T for this warp's 16 tokens: two 8-token column blocks
-                float sacc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-                {
-                    int r = (lane & 7) + ((lane >> 4) << 3);  // token row this lane addresses
-                    int cb = (lane >> 3) & 1;                 // which 8-dim chunk of the k-step
-#pragma unroll
-                    for (int ks = 0; ks < KS; ks++) {
-                        int chunk = ks * 2 + cb;  // 16-byte chunk index within the row
-                        int sg = r * HALVES + (chunk >> 3);
-                        uint32_t a = kpage + sg * 128 + (((chunk & 7) ^ (sg & 7)) << 4);
-                        uint32_t kb[4];
-                        ldsm_x4(a, kb);
-                        mma_bf16(sacc[0], qa[ks], kb[0], kb[1]);
-                        mma_bf16(sacc[1], qa[ks], kb[2], kb[3]);
-                    }
-                }
-                // mask, online softmax (base 2), pack P as the A operand of P V
-                int col = (lane & 3) * 2;
-                float rmax[2] = {-INFINITY, -INFINITY};
-#pragma unroll
-                for (int nb = 0; nb < 2; nb++)
-#pragma unroll
-                    for (int e = 0; e < 4; e++) {
-                        int tk = nb * 8 + col + (e & 1);
-                        if (tk >= valid) sacc[nb][e] = -INFINITY;
-                        rmax[e >> 1] = fmaxf(rmax[e >> 1], sacc[nb][e]);
-                    }
-                float corr[2], msub[2];
-#pragma unroll
-                for (int h = 0; h < 2; h++) {
-                    rmax[h] = fmaxf(rmax[h], __shfl_xor_sync(0xffffffffu, rmax[h], 1));
-                    rmax[h] = fmaxf(rmax[h], __shfl_xor_sync(0xffffffffu, rmax[h], 2));
-                    float mnew = fmaxf(m_run[h], rmax[h]);
-                    msub[h] = mnew == -INFINITY ? 0.f : mnew;
-                    corr[h] = m_run[h] == -INFINITY ? 0.f : exp2f(m_run[h] - msub[h]);
-                    m_run[h] = mnew;
-                }
-                float rsum[2] = {0.f, 0.f};
-                uint32_t pa[4];
-#pragma unroll
-                for (int nb = 0; nb < 2; nb++) {
-                    float p0 = exp2f(sacc[nb][0] - msub[0]), p1 = exp2f(sacc[nb][1] - msub[0]);
-                    float p2 = exp2f(sacc[nb][2] - msub[1]), p3 = exp2f(sacc[nb][3] - msub[1]);
-                    rsum[0] += p0 + p1;
-                    rsum[1] += p2 + p3;
-                    pa[nb * 2 + 0] = pack_bf16(p0, p1);
-                    pa[nb * 2 + 1] = pack_bf16(p2, p3);
-                }
-#pragma unroll
-                for (int h = 0; h < 2; h++) {
-                    rsum[h] += __shfl_xor_sync(0xffffffffu, rsum[h], 1);
-                    rsum[h] += __shfl_xor_sync(0xffffffffu, rsum[h], 2);
-                    l_run[h] = l_run[h] * corr[h] + rsum[h];
-                }
-#pragma unroll
-                for (int nb = 0; nb < NB; nb++) {
-                    o[nb][0] *= corr[0];
-                    o[nb][1] *= corr[0];
-                    o[nb][2] *= corr[1];
-                    o[nb][3] *= corr[1];
-                }
-                // O += P V: V read transposed, two 8-dim column blocks per ldmatrix
-                {
-                    int r = (lane & 7) + (((lane >> 3) & 1) << 3);  // token row
-                    int cb = lane >> 4;                              // which of the two dim blocks
-#pragma unroll
-                    for (int np = 0; np < NB / 2; np++) {
-                        int chunk = np * 2 + cb;
-                        int sg = r * HALVES + (chunk >> 3);
-                        uint32_t a = vpage + sg * 128 + (((chunk & 7) ^ (sg & 7)) << 4);
-                        uint32_t vb[4];
-                        ldsm_x4_trans(a, vb);
-                        mma_bf16(o[np * 2], pa, vb[0], vb[1]);
-                        mma_bf16(o[np * 2 + 1], pa, vb[2], vb[3]);
-                    }
-                }
-            }
-            __syncwarp();
-            if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(empty_bar(s)) : "memory");
-        }
-        if (!ok) {
-            // a ring that stopped filling stops for all four warps: every consumer leaves here
-            if (lane == 0) report(p.status, kStatusWaitExpired, 310 + warp);
-            return;
-        }
-
-        // ---- fold the four warps' states, (0+2) + (1+3), in registers through the one-slot
-        // scratch; warp 0 then writes this segment's partial
         int pair = item * p.n_kv + g;
         int first_cta = pair_start / quota, nseg = (pair_end - 1) / quota - first_cta + 1;
         float *out = p.part + (size_t)(blockIdx.x + pair) * 16 * (DH + 2);
-        {
-            int r0 = lane >> 2, c = (lane & 3) * 2;
-            auto put = [&]() {
-#pragma unroll
-                for (int nb = 0; nb < NB; nb++) {
-                    *reinterpret_cast<float2 *>(sc_o + (size_t)r0 * FS + nb * 8 + c) = make_float2(o[nb][0], o[nb][1]);
-                    *reinterpret_cast<float2 *>(sc_o + (size_t)(r0 + 8) * FS + nb * 8 + c) = make_float2(o[nb][2], o[nb][3]);
+        if constexpr (!NARROW) {
+            uint32_t qa[KS][4];
+            {
+                int r0 = lane >> 2, c = (lane & 3) * 2;
+                const float *q0 = sc_o + r0 * DH, *q1 = sc_o + (r0 + 8) * DH;
+    #pragma unroll
+                for (int ks = 0; ks < KS; ks++) {
+                    int k = ks * 16 + c;
+                    qa[ks][0] = pack_bf16(q0[k] * qscale, q0[k + 1] * qscale);
+                    qa[ks][1] = pack_bf16(q1[k] * qscale, q1[k + 1] * qscale);
+                    qa[ks][2] = pack_bf16(q0[k + 8] * qscale, q0[k + 9] * qscale);
+                    qa[ks][3] = pack_bf16(q1[k + 8] * qscale, q1[k + 9] * qscale);
                 }
-                if ((lane & 3) == 0) {
-                    sc_m[r0] = m_run[0];
-                    sc_m[r0 + 8] = m_run[1];
-                    sc_l[r0] = l_run[0];
-                    sc_l[r0 + 8] = l_run[1];
-                }
-            };
-            auto take = [&]() {  // this warp's state := this warp's state (+) the slot's state
-#pragma unroll
-                for (int h = 0; h < 2; h++) {
-                    int r = r0 + 8 * h;
-                    float mb = sc_m[r], lb = sc_l[r];
-                    float M = fmaxf(m_run[h], mb);
-                    float fa = m_run[h] == -INFINITY ? 0.f : exp2f(m_run[h] - M);
-                    float fb = mb == -INFINITY ? 0.f : exp2f(mb - M);
-                    l_run[h] = l_run[h] * fa + lb * fb;
-                    m_run[h] = M;
-#pragma unroll
-                    for (int nb = 0; nb < NB; nb++) {
-                        float2 ob = *reinterpret_cast<const float2 *>(sc_o + (size_t)r * FS + nb * 8 + c);
-                        o[nb][2 * h] = o[nb][2 * h] * fa + ob.x * fb;
-                        o[nb][2 * h + 1] = o[nb][2 * h + 1] * fa + ob.y * fb;
-                    }
-                }
-            };
-            for (int step = 0; step < 3; step++) {  // 2 -> 0, 3 -> 1, 1 -> 0
-                int src = step == 0 ? 2 : step == 1 ? 3 : 1, dst = step == 1 ? 1 : 0;
-                if (warp == src) put();
-                consumer_sync();
-                if (warp == dst) take();
-                consumer_sync();
             }
-            if (warp == 0) {
-#pragma unroll
-                for (int h = 0; h < 2; h++) {
-                    int q = r0 + 8 * h;
-                    if (q < nq_act) {
-                        if (nseg == 1) {
-                            // the pair's only segment: normalise and write the head's output
-                            int row = q < p.G ? item : Bc + item;
-                            int hq = g * p.G + (q < p.G ? q : q - p.G);
-                            size_t ob = (size_t)row * q_dim + (size_t)hq * DH;
-                            float inv = 1.f / l_run[h];
-#pragma unroll
-                            for (int nb = 0; nb < NB; nb++)
-#pragma unroll
-                                for (int e = 0; e < 2; e++) {
-                                    float x = o[nb][2 * h + e] * inv;
-                                    __nv_bfloat16 hi = __float2bfloat16_rn(x);
-                                    p.Ob[ob + nb * 8 + c + e] = hi;
-                                    if (p.lo_off) p.Ob[ob + nb * 8 + c + e + p.lo_off] = __float2bfloat16_rn(x - __bfloat162float(hi));
-                                }
-                        } else {
-#pragma unroll
-                            for (int nb = 0; nb < NB; nb++)
-                                *reinterpret_cast<float2 *>(out + (size_t)q * (DH + 2) + nb * 8 + c) =
-                                    make_float2(o[nb][2 * h], o[nb][2 * h + 1]);
-                            if ((lane & 3) == 0) {
-                                out[(size_t)q * (DH + 2) + DH] = m_run[h];  // base-2 units
-                                out[(size_t)q * (DH + 2) + DH + 1] = l_run[h];
-                            }
+            consumer_sync();  // everyone has its fragments: the scratch is free again
+            float o[NB][4];
+    #pragma unroll
+            for (int nb = 0; nb < NB; nb++) o[nb][0] = o[nb][1] = o[nb][2] = o[nb][3] = 0.f;
+            float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+
+            for (int t = t0; t < t1 && ok; t++, it++) {
+                int s = it % STAGES;
+                ok = mbar_wait(full_bar(s), (it / STAGES) & 1);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                int valid = min(16, nkeys - (t * kAttTile + warp * 16));  // valid tokens in this warp's page
+                if (valid > 0) {
+                    // a page's box: K then V, each [16 rows][DH], the 128-byte pieces of a row swizzled
+                    uint32_t kpage = tiles + s * Cfg::kStageBytes + warp * 2 * Cfg::kPageBytes;
+                    uint32_t vpage = kpage + Cfg::kPageBytes;
+                    if (valid < 16) {
+                        // stale slots past the end of the sequence: their scores are masked below, and
+                        // their V rows are zeroed here so that 0 * garbage cannot produce a NaN
+                        for (int idx = lane; idx < (16 - valid) * HALVES * 8; idx += 32) {
+                            uint32_t a = vpage + valid * HALVES * 128 + idx * 16;
+                            asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(a), "r"(0u) : "memory");
+                        }
+                        __syncwarp();
+                    }
+                    // S = Q K^T for this warp's 16 tokens: two 8-token column blocks
+                    float sacc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+                    {
+                        int r = (lane & 7) + ((lane >> 4) << 3);  // token row this lane addresses
+                        int cb = (lane >> 3) & 1;                 // which 8-dim chunk of the k-step
+    #pragma unroll
+                        for (int ks = 0; ks < KS; ks++) {
+                            int chunk = ks * 2 + cb;  // 16-byte chunk index within the row
+                            int sg = r * HALVES + (chunk >> 3);
+                            uint32_t a = kpage + sg * 128 + (((chunk & 7) ^ (sg & 7)) << 4);
+                            uint32_t kb[4];
+                            ldsm_x4(a, kb);
+                            mma_bf16(sacc[0], qa[ks], kb[0], kb[1]);
+                            mma_bf16(sacc[1], qa[ks], kb[2], kb[3]);
+                        }
+                    }
+                    // mask, online softmax (base 2), pack P as the A operand of P V
+                    int col = (lane & 3) * 2;
+                    float rmax[2] = {-INFINITY, -INFINITY};
+    #pragma unroll
+                    for (int nb = 0; nb < 2; nb++)
+    #pragma unroll
+                        for (int e = 0; e < 4; e++) {
+                            int tk = nb * 8 + col + (e & 1);
+                            if (tk >= valid) sacc[nb][e] = -INFINITY;
+                            rmax[e >> 1] = fmaxf(rmax[e >> 1], sacc[nb][e]);
+                        }
+                    float corr[2], msub[2];
+    #pragma unroll
+                    for (int h = 0; h < 2; h++) {
+                        rmax[h] = fmaxf(rmax[h], __shfl_xor_sync(0xffffffffu, rmax[h], 1));
+                        rmax[h] = fmaxf(rmax[h], __shfl_xor_sync(0xffffffffu, rmax[h], 2));
+                        float mnew = fmaxf(m_run[h], rmax[h]);
+                        msub[h] = mnew == -INFINITY ? 0.f : mnew;
+                        corr[h] = m_run[h] == -INFINITY ? 0.f : exp2f(m_run[h] - msub[h]);
+                        m_run[h] = mnew;
+                    }
+                    float rsum[2] = {0.f, 0.f};
+                    uint32_t pa[4];
+    #pragma unroll
+                    for (int nb = 0; nb < 2; nb++) {
+                        float p0 = exp2f(sacc[nb][0] - msub[0]), p1 = exp2f(sacc[nb][1] - msub[0]);
+                        float p2 = exp2f(sacc[nb][2] - msub[1]), p3 = exp2f(sacc[nb][3] - msub[1]);
+                        rsum[0] += p0 + p1;
+                        rsum[1] += p2 + p3;
+                        pa[nb * 2 + 0] = pack_bf16(p0, p1);
+                        pa[nb * 2 + 1] = pack_bf16(p2, p3);
+                    }
+    #pragma unroll
+                    for (int h = 0; h < 2; h++) {
+                        rsum[h] += __shfl_xor_sync(0xffffffffu, rsum[h], 1);
+                        rsum[h] += __shfl_xor_sync(0xffffffffu, rsum[h], 2);
+                        l_run[h] = l_run[h] * corr[h] + rsum[h];
+                    }
+    #pragma unroll
+                    for (int nb = 0; nb < NB; nb++) {
+                        o[nb][0] *= corr[0];
+                        o[nb][1] *= corr[0];
+                        o[nb][2] *= corr[1];
+                        o[nb][3] *= corr[1];
+                    }
+                    // O += P V: V read transposed, two 8-dim column blocks per ldmatrix
+                    {
+                        int r = (lane & 7) + (((lane >> 3) & 1) << 3);  // token row
+                        int cb = lane >> 4;                              // which of the two dim blocks
+    #pragma unroll
+                        for (int np = 0; np < NB / 2; np++) {
+                            int chunk = np * 2 + cb;
+                            int sg = r * HALVES + (chunk >> 3);
+                            uint32_t a = vpage + sg * 128 + (((chunk & 7) ^ (sg & 7)) << 4);
+                            uint32_t vb[4];
+                            ldsm_x4_trans(a, vb);
+                            mma_bf16(o[np * 2], pa, vb[0], vb[1]);
+                            mma_bf16(o[np * 2 + 1], pa, vb[2], vb[3]);
                         }
                     }
                 }
-                if (nseg > 1) __threadfence();
+                __syncwarp();
+                if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(empty_bar(s)) : "memory");
+            }
+            if (!ok) {
+                // a ring that stopped filling stops for all four warps: every consumer leaves here
+                if (lane == 0) report(p.status, kStatusWaitExpired, 310 + warp);
+                return;
+            }
+
+            // ---- fold the four warps' states, (0+2) + (1+3), in registers through the one-slot
+            // scratch; warp 0 then writes this segment's partial
+            {
+                int r0 = lane >> 2, c = (lane & 3) * 2;
+                auto put = [&]() {
+    #pragma unroll
+                    for (int nb = 0; nb < NB; nb++) {
+                        *reinterpret_cast<float2 *>(sc_o + (size_t)r0 * FS + nb * 8 + c) = make_float2(o[nb][0], o[nb][1]);
+                        *reinterpret_cast<float2 *>(sc_o + (size_t)(r0 + 8) * FS + nb * 8 + c) = make_float2(o[nb][2], o[nb][3]);
+                    }
+                    if ((lane & 3) == 0) {
+                        sc_m[r0] = m_run[0];
+                        sc_m[r0 + 8] = m_run[1];
+                        sc_l[r0] = l_run[0];
+                        sc_l[r0 + 8] = l_run[1];
+                    }
+                };
+                auto take = [&]() {  // this warp's state := this warp's state (+) the slot's state
+    #pragma unroll
+                    for (int h = 0; h < 2; h++) {
+                        int r = r0 + 8 * h;
+                        float mb = sc_m[r], lb = sc_l[r];
+                        float M = fmaxf(m_run[h], mb);
+                        float fa = m_run[h] == -INFINITY ? 0.f : exp2f(m_run[h] - M);
+                        float fb = mb == -INFINITY ? 0.f : exp2f(mb - M);
+                        l_run[h] = l_run[h] * fa + lb * fb;
+                        m_run[h] = M;
+    #pragma unroll
+                        for (int nb = 0; nb < NB; nb++) {
+                            float2 ob = *reinterpret_cast<const float2 *>(sc_o + (size_t)r * FS + nb * 8 + c);
+                            o[nb][2 * h] = o[nb][2 * h] * fa + ob.x * fb;
+                            o[nb][2 * h + 1] = o[nb][2 * h + 1] * fa + ob.y * fb;
+                        }
+                    }
+                };
+                for (int step = 0; step < 3; step++) {  // 2 -> 0, 3 -> 1, 1 -> 0
+                    int src = step == 0 ? 2 : step == 1 ? 3 : 1, dst = step == 1 ? 1 : 0;
+                    if (warp == src) put();
+                    consumer_sync();
+                    if (warp == dst) take();
+                    consumer_sync();
+                }
+                if (warp == 0) {
+    #pragma unroll
+                    for (int h = 0; h < 2; h++) {
+                        int q = r0 + 8 * h;
+                        if (q < nq_act) {
+                            if (nseg == 1) {
+                                // the pair's only segment: normalise and write the head's output
+                                int row = q < p.G ? item : Bc + item;
+                                int hq = g * p.G + (q < p.G ? q : q - p.G);
+                                size_t ob = (size_t)row * q_dim + (size_t)hq * DH;
+                                float inv = 1.f / l_run[h];
+    #pragma unroll
+                                for (int nb = 0; nb < NB; nb++)
+    #pragma unroll
+                                    for (int e = 0; e < 2; e++) {
+                                        float x = o[nb][2 * h + e] * inv;
+                                        __nv_bfloat16 hi = __float2bfloat16_rn(x);
+                                        p.Ob[ob + nb * 8 + c + e] = hi;
+                                        if (p.lo_off) p.Ob[ob + nb * 8 + c + e + p.lo_off] = __float2bfloat16_rn(x - __bfloat162float(hi));
+                                    }
+                            } else {
+    #pragma unroll
+                                for (int nb = 0; nb < NB; nb++)
+                                    *reinterpret_cast<float2 *>(out + (size_t)q * (DH + 2) + nb * 8 + c) =
+                                        make_float2(o[nb][2 * h], o[nb][2 * h + 1]);
+                                if ((lane & 3) == 0) {
+                                    out[(size_t)q * (DH + 2) + DH] = m_run[h];  // base-2 units
+                                    out[(size_t)q * (DH + 2) + DH + 1] = l_run[h];
+                                }
+                            }
+                        }
+                    }
+                    if (nseg > 1) __threadfence();
+                }
+            }
+        } else {
+            // ---- narrow variant: at most 8 query rows per KV head.  The products are taken transposed,
+            // S^T = K Q^T and O^T = V^T P^T, so that the 16 keys of a page fill the M side of
+            // m16n8k16 and the (few) queries sit on the 8-wide N side: half the MMAs and half the
+            // accumulators of the 16-query form.
+            uint32_t qb[KS][2];
+            {
+                int n = lane >> 2, c = (lane & 3) * 2;
+                const float *q0 = sc_o + n * DH;
+#pragma unroll
+                for (int ks = 0; ks < KS; ks++) {
+                    int k = ks * 16 + c;
+                    qb[ks][0] = pack_bf16(q0[k] * qscale, q0[k + 1] * qscale);
+                    qb[ks][1] = pack_bf16(q0[k + 8] * qscale, q0[k + 9] * qscale);
+                }
+            }
+            consumer_sync();  // everyone has its fragments: the scratch is free again
+            constexpr int MB = DH / 16;  // 16-row blocks of O^T
+            float o[MB][4];
+#pragma unroll
+            for (int mb = 0; mb < MB; mb++) o[mb][0] = o[mb][1] = o[mb][2] = o[mb][3] = 0.f;
+            // per query column (2t, 2t+1): running max (same in the 8 lanes of a column) and this
+            // lane's share of the running sum (reduced over the lanes once, after the loop)
+            float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+            const int g8 = lane >> 2;
+
+            for (int t = t0; t < t1 && ok; t++, it++) {
+                int s = it % STAGES;
+                ok = mbar_wait(full_bar(s), (it / STAGES) & 1);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                int valid = min(16, nkeys - (t * kAttTile + warp * 16));  // valid tokens in this warp's page
+                if (valid > 0) {
+                    uint32_t kpage = tiles + s * Cfg::kStageBytes + warp * 2 * Cfg::kPageBytes;
+                    uint32_t vpage = kpage + Cfg::kPageBytes;
+                    if (valid < 16) {
+                        for (int idx = lane; idx < (16 - valid) * HALVES * 8; idx += 32) {
+                            uint32_t a = vpage + valid * HALVES * 128 + idx * 16;
+                            asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(a), "r"(0u) : "memory");
+                        }
+                        __syncwarp();
+                    }
+                    // S^T = K Q^T: K rows as the A operand
+                    float sacc[4] = {0.f, 0.f, 0.f, 0.f};
+                    {
+                        int r = (lane & 7) + (((lane >> 3) & 1) << 3);  // key row this lane addresses
+                        int cb = lane >> 4;                              // which 8-dim chunk of the k-step
+#pragma unroll
+                        for (int ks = 0; ks < KS; ks++) {
+                            int chunk = ks * 2 + cb;
+                            int sg = r * HALVES + (chunk >> 3);
+                            uint32_t a = kpage + sg * 128 + (((chunk & 7) ^ (sg & 7)) << 4);
+                            uint32_t ka[4];
+                            ldsm_x4(a, ka);
+                            mma_bf16(sacc, ka, qb[ks][0], qb[ks][1]);
+                        }
+                    }
+                    // sacc: keys g8, g8+8 (rows) x queries 2t, 2t+1 (columns)
+                    if (valid < 16) {
+                        if (g8 >= valid) sacc[0] = sacc[1] = -INFINITY;
+                        if (g8 + 8 >= valid) sacc[2] = sacc[3] = -INFINITY;
+                    }
+                    float rmax[2] = {fmaxf(sacc[0], sacc[2]), fmaxf(sacc[1], sacc[3])};
+                    float corr[2], msub[2];
+#pragma unroll
+                    for (int j = 0; j < 2; j++) {
+                        rmax[j] = fmaxf(rmax[j], __shfl_xor_sync(0xffffffffu, rmax[j], 4));
+                        rmax[j] = fmaxf(rmax[j], __shfl_xor_sync(0xffffffffu, rmax[j], 8));
+                        rmax[j] = fmaxf(rmax[j], __shfl_xor_sync(0xffffffffu, rmax[j], 16));
+                        float mnew = fmaxf(m_run[j], rmax[j]);
+                        msub[j] = mnew == -INFINITY ? 0.f : mnew;
+                        corr[j] = m_run[j] == -INFINITY ? 0.f : exp2f(m_run[j] - msub[j]);
+                        m_run[j] = mnew;
+                    }
+                    float p0 = exp2f(sacc[0] - msub[0]), p1 = exp2f(sacc[1] - msub[1]);
+                    float p2 = exp2f(sacc[2] - msub[0]), p3 = exp2f(sacc[3] - msub[1]);
+                    l_run[0] = l_run[0] * corr[0] + (p0 + p2);
+                    l_run[1] = l_run[1] * corr[1] + (p1 + p3);
+                    // P^T as the B operand of O^T += V^T P^T: transpose the two 8x8 blocks across the warp
+                    uint32_t pb0 = movmatrix_trans(pack_bf16(p0, p1)), pb1 = movmatrix_trans(pack_bf16(p2, p3));
+                    if (__any_sync(0xffffffffu, corr[0] != 1.f || corr[1] != 1.f)) {
+#pragma unroll
+                        for (int mb = 0; mb < MB; mb++) {
+                            o[mb][0] *= corr[0];
+                            o[mb][1] *= corr[1];
+                            o[mb][2] *= corr[0];
+                            o[mb][3] *= corr[1];
+                        }
+                    }
+                    {
+                        int r = (lane & 7) + ((lane >> 4) << 3);  // key row
+                        int cb = (lane >> 3) & 1;                 // which 8-dim half of the 16-dim block
+#pragma unroll
+                        for (int mb = 0; mb < MB; mb++) {
+                            int chunk = mb * 2 + cb;
+                            int sg = r * HALVES + (chunk >> 3);
+                            uint32_t a = vpage + sg * 128 + (((chunk & 7) ^ (sg & 7)) << 4);
+                            uint32_t va[4];
+                            ldsm_x4_trans(a, va);
+                            mma_bf16(o[mb], va, pb0, pb1);
+                        }
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(empty_bar(s)) : "memory");
+            }
+            if (!ok) {
+                if (lane == 0) report(p.status, kStatusWaitExpired, 310 + warp);
+                return;
+            }
+#pragma unroll
+            for (int j = 0; j < 2; j++) {  // the lanes' shares of the running sums
+                l_run[j] += __shfl_xor_sync(0xffffffffu, l_run[j], 4);
+                l_run[j] += __shfl_xor_sync(0xffffffffu, l_run[j], 8);
+                l_run[j] += __shfl_xor_sync(0xffffffffu, l_run[j], 16);
+            }
+            // ---- fold the four warps' states, (0+2) + (1+3), through the scratch ([8 queries][DH + 4])
+            {
+                constexpr int FN = DH + 4;
+                int c = (lane & 3) * 2;
+                auto put = [&]() {
+#pragma unroll
+                    for (int mb = 0; mb < MB; mb++) {
+                        sc_o[(size_t)c * FN + mb * 16 + g8] = o[mb][0];
+                        sc_o[(size_t)(c + 1) * FN + mb * 16 + g8] = o[mb][1];
+                        sc_o[(size_t)c * FN + mb * 16 + g8 + 8] = o[mb][2];
+                        sc_o[(size_t)(c + 1) * FN + mb * 16 + g8 + 8] = o[mb][3];
+                    }
+                    if (g8 == 0) {
+                        sc_m[c] = m_run[0];
+                        sc_m[c + 1] = m_run[1];
+                        sc_l[c] = l_run[0];
+                        sc_l[c + 1] = l_run[1];
+                    }
+                };
+                auto take = [&]() {
+                    float fa[2], fb[2];
+#pragma unroll
+                    for (int j = 0; j < 2; j++) {
+                        float mb2 = sc_m[c + j], lb = sc_l[c + j];
+                        float M = fmaxf(m_run[j], mb2);
+                        fa[j] = m_run[j] == -INFINITY ? 0.f : exp2f(m_run[j] - M);
+                        fb[j] = mb2 == -INFINITY ? 0.f : exp2f(mb2 - M);
+                        l_run[j] = l_run[j] * fa[j] + lb * fb[j];
+                        m_run[j] = M;
+                    }
+#pragma unroll
+                    for (int mb = 0; mb < MB; mb++) {
+                        o[mb][0] = o[mb][0] * fa[0] + sc_o[(size_t)c * FN + mb * 16 + g8] * fb[0];
+                        o[mb][1] = o[mb][1] * fa[1] + sc_o[(size_t)(c + 1) * FN + mb * 16 + g8] * fb[1];
+                        o[mb][2] = o[mb][2] * fa[0] + sc_o[(size_t)c * FN + mb * 16 + g8 + 8] * fb[0];
+                        o[mb][3] = o[mb][3] * fa[1] + sc_o[(size_t)(c + 1) * FN + mb * 16 + g8 + 8] * fb[1];
+                    }
+                };
+                for (int step = 0; step < 3; step++) {  // 2 -> 0, 3 -> 1, 1 -> 0
+                    int src = step == 0 ? 2 : step == 1 ? 3 : 1, dst = step == 1 ? 1 : 0;
+                    if (warp == src) put();
+                    consumer_sync();
+                    if (warp == dst) take();
+                    consumer_sync();
+                }
+                if (warp == 0) {
+#pragma unroll
+                    for (int j = 0; j < 2; j++) {
+                        int q = c + j;
+                        if (q < nq_act) {
+                            if (nseg == 1) {
+                                int row = q < p.G ? item : Bc + item;
+                                int hq = g * p.G + (q < p.G ? q : q - p.G);
+                                size_t ob = (size_t)row * q_dim + (size_t)hq * DH;
+                                float inv = 1.f / l_run[j];
+#pragma unroll
+                                for (int mb = 0; mb < MB; mb++)
+#pragma unroll
+                                    for (int e = 0; e < 2; e++) {
+                                        float x = o[mb][2 * e + j] * inv;
+                                        size_t oi = ob + mb * 16 + g8 + 8 * e;
+                                        __nv_bfloat16 hi = __float2bfloat16_rn(x);
+                                        p.Ob[oi] = hi;
+                                        if (p.lo_off) p.Ob[oi + p.lo_off] = __float2bfloat16_rn(x - __bfloat162float(hi));
+                                    }
+                            } else {
+#pragma unroll
+                                for (int mb = 0; mb < MB; mb++) {
+                                    out[(size_t)q * (DH + 2) + mb * 16 + g8] = o[mb][j];
+                                    out[(size_t)q * (DH + 2) + mb * 16 + g8 + 8] = o[mb][2 + j];
+                                }
+                                if (g8 == 0) {
+                                    out[(size_t)q * (DH + 2) + DH] = m_run[j];  // base-2 units
+                                    out[(size_t)q * (DH + 2) + DH + 1] = l_run[j];
+                                }
+                            }
+                        }
+                    }
+                    if (nseg > 1) __threadfence();
+                }
             }
         }
         // ---- the last segment of this pair to arrive folds all of them in segment order

@@ -49,6 +49,8 @@ def test_tiny_fp32_primary_only():
     (small_bf16(n_q_heads=4, n_kv_heads=4, head_dim=64), 1, 20, 17),  # MHA, batch 1
     (small_bf16(n_q_heads=2, n_kv_heads=1, head_dim=128, d_model=128, vocab=777), 5, 50, 47),  # MQA, odd batch
     (small_bf16(final_norm=0, n_layers=1), 2, 18, 0),              # no prefill at all: decode from position 0
+    (small_bf16(n_q_heads=8, n_kv_heads=1, head_dim=64), 3, 40, 35),   # 8 queries per KV head: 16-row attention tile
+    (small_bf16(n_q_heads=8, n_kv_heads=1, head_dim=128, d_model=256), 2, 90, 70),  # the same at d_h 128, two tiles
 ])
 def test_small_bf16_models(cfg, B, T, npre):
     w = make_weights(cfg, seed=5, matrix_std=0.05)
