@@ -1439,10 +1439,10 @@ bool setup_tc(dbt_model *m) {
     // and overlap with their neighbours through programmatic dependent launch.
     m->fused = ok && m->att_fast && !moe && (fu && strcmp(fu, "1") == 0);
     const char *wi = getenv("DBT_WIDE");
-    // Opt-in (DBT_WIDE=1): 9 instead of 10 kernels per layer and no row-wide reduction, but measured
-    // no faster (1.62 vs 1.55 ms per step at batch 16 on the 1B model): the step is bound by the
-    // kernel-to-kernel dependency latency, not by these kernels' bodies.
-    m->wide = ok && m->att_fast && !moe && (wi && strcmp(wi, "1") == 0);
+    // Default chain of a dense bf16 model: the RMSNorm factor is applied after the GEMM, so no kernel
+    // reduces over a whole row (9 kernels per layer; 1.37 vs 1.42 ms per step at batch 16 on the 1B
+    // model against the chain with a row-wide residual+norm kernel, which DBT_WIDE=0 selects).
+    m->wide = ok && m->att_fast && !moe && !m->fused && !(wi && strcmp(wi, "0") == 0);
     const char *split = getenv("DBT_ACT_SPLIT");
     m->act_parts = (split && strcmp(split, "0") == 0) ? 1 : 2;
     return ok;

@@ -74,7 +74,13 @@ __device__ __forceinline__ void sum_splits_k(const float *P, size_t split_stride
 __device__ __forceinline__ float row_scale(const float *ss, int ss_tiles, int ss_ld, int row, int d_norm, float eps) {
     if (!ss) return 1.f;
     float a = 0.f;
-    for (int t = 0; t < ss_tiles; t++) a += __ldcg(ss + (size_t)t * ss_ld + row);
+    for (int t0 = 0; t0 < ss_tiles; t0 += 8) {  // eight shares in flight at a time, added in tile order
+        float v[8];
+#pragma unroll
+        for (int j = 0; j < 8; j++) v[j] = t0 + j < ss_tiles ? __ldcg(ss + (size_t)(t0 + j) * ss_ld + row) : 0.f;
+#pragma unroll
+        for (int j = 0; j < 8; j++) a += v[j];
+    }
     return 1.f / sqrtf(a / (float)d_norm + eps);
 }
 

@@ -309,17 +309,36 @@ def test_fresh_models_give_bitwise_identical_results():
             assert torch.equal(x["z1"], y["z1"]) and torch.equal(x["z2"], y["z2"])
 
 
-@pytest.mark.parametrize("knob", ["DBT_FUSED", "DBT_WIDE"])
-def test_opt_in_kernel_chains_match_oracle(monkeypatch, knob):
-    """The two opt-in variants of the dense chain -- elementwise work folded into the GEMM
-    epilogues (last-arriving CTA per output tile), and the RMSNorm factor applied after the GEMM
-    (no row-wide reduction kernel) -- compute the same step."""
-    monkeypatch.setenv(knob, "1")
+@pytest.mark.parametrize("knob,value", [("DBT_FUSED", "1"), ("DBT_WIDE", "0"), ("DBT_MEGA", "1"), ("DBT_L2_PREFETCH", "1")])
+def test_alternative_kernel_chains_match_oracle(monkeypatch, knob, value):
+    """The variants of the dense chain that are not the default -- elementwise work folded into the
+    GEMM epilogues (last-arriving CTA per output tile), a row-wide residual+RMSNorm kernel before
+    each GEMM, the whole step as one persistent kernel, L2 prefetch requests riding on the GEMM
+    launches -- compute the same step."""
+    monkeypatch.setenv(knob, value)
     cfg = small_bf16()
     w = make_weights(cfg, seed=5, matrix_std=0.05)
     tok = make_tokens(cfg, 3, 40, seed=6)
     teacher_forced_compare(cfg, w, tok, n_prefill=35, grouped=True)
     teacher_forced_compare(cfg, w, tok, n_prefill=35, grouped=False)
+
+
+def test_single_kernel_step_across_row_tile_widths(monkeypatch):
+    """The persistent single-kernel step at batch sizes that select each of its row-tile widths
+    (16, 32, 64), with enough context for several attention stages per CTA."""
+    monkeypatch.setenv("DBT_MEGA", "1")
+    cfg = small_bf16(n_q_heads=2, n_kv_heads=1, head_dim=128, d_model=128, vocab=777, n_layers=2)
+    w = make_weights(cfg, seed=5, matrix_std=0.05)
+    for B, T, npre in [(5, 140, 132), (12, 24, 20), (30, 24, 20)]:
+        tok = make_tokens(cfg, B, T, seed=6)
+        teacher_forced_compare(cfg, w, tok, n_prefill=npre, grouped=True)
+    # and it is the path that ran: one launch per decode step
+    gm = make_gpu_model(cfg, w, 5, 32)
+    tok = make_tokens(cfg, 5, 8, seed=6).cuda()
+    gm.prefill(tok[:, :6].contiguous())
+    before = gm.launch_count()
+    gm.decode_step(tok[:, 6].contiguous())
+    assert gm.launch_count() - before == 1
 
 
 def test_8b_shape_two_layers_paged_with_shuffled_pages():
