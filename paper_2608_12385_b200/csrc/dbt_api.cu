@@ -518,13 +518,13 @@ int pad_rows(int r) { return r <= 16 ? 16 : r <= 32 ? 32 : r <= 64 ? 64 : r <= 1
 
 // Split-K factor from the tile count and K only (never from the mode), so that grouped and
 // primary-only steps add the same partials in the same order.
-int choose_split(int tiles, int total_kt) {
+int choose_split(int tiles, int total_kt, int slots) {
     int best = 1;
     double best_cost = 1e30;
     for (int s = 1; s <= total_kt && s <= 16; s++) {
         int kt = (total_kt + s - 1) / s;
         int s_eff = (total_kt + kt - 1) / kt;
-        int waves = (tiles * s_eff + 147) / 148;
+        int waves = (tiles * s_eff + slots - 1) / slots;
         double cost = waves * (kt + 3.0);
         if (cost < best_cost - 1e-9) {
             best_cost = cost;
@@ -532,6 +532,18 @@ int choose_split(int tiles, int total_kt) {
         }
     }
     return best;
+}
+
+// CTAs of the GEMM kernel that are resident at once: two per SM up to a row tile of 64 (96 KB of
+// ring each), one above.  DBT_SPLIT_SLOTS overrides (experiments).
+int split_slots(const dbt_model *m, int n_tile) {
+    static int forced = -1;
+    if (forced < 0) {
+        const char *e = getenv("DBT_SPLIT_SLOTS");
+        forced = e ? atoi(e) : 0;
+    }
+    if (forced > 0) return forced;
+    return (n_tile <= 64 ? 2 : 1) * m->num_sms;
 }
 
 template <int N_TILE>
@@ -585,7 +597,7 @@ dbt_status run_gemm_tc(dbt_model *m, const TcCall &c, int n_tile, int *nsplit_ou
     }
     int total_kt = (c.K + kTcK - 1) / kTcK;
     if (c.grp_cnt) force_split = 1;  // enough CTAs already: tiles x selected experts
-    int split = force_split > 0 ? (force_split < total_kt ? force_split : total_kt) : choose_split(tiles, total_kt);
+    int split = force_split > 0 ? (force_split < total_kt ? force_split : total_kt) : choose_split(tiles, total_kt, split_slots(m, n_tile));
     while (split > 1 && (size_t)split * n_tile * col > c.P_floats) split--;
     if ((size_t)c.R * col > c.P_floats) return fail(m, DBT_ERR_CAPACITY, "partial buffer too small for %s", c.tag);
     p.kt_per_split = (total_kt + split - 1) / split;

@@ -44,28 +44,19 @@ __device__ __forceinline__ float sum_splits(const float *P, size_t split_stride,
 template <int K>
 __device__ __forceinline__ void sum_splits_k(const float *P, size_t split_stride, int nsplit, const size_t (&off)[K],
                                              float (&out)[K]) {
+    constexpr int NB = K <= 2 ? 4 : 2;  // splits per batch: eight loads in flight
 #pragma unroll
     for (int k = 0; k < K; k++) out[k] = 0.f;
-    int s = 0;
-    for (; s + 2 <= nsplit; s += 2) {
-        float a[K], b[K];
+    for (int s = 0; s < nsplit; s += NB) {
+        float v[NB][K];
 #pragma unroll
-        for (int k = 0; k < K; k++) {
-            a[k] = __ldcg(P + (size_t)s * split_stride + off[k]);
-            b[k] = __ldcg(P + (size_t)(s + 1) * split_stride + off[k]);
-        }
+        for (int j = 0; j < NB; j++)
 #pragma unroll
-        for (int k = 0; k < K; k++) {
-            out[k] += a[k];
-            out[k] += b[k];
-        }
-    }
-    if (s < nsplit) {
-        float a[K];
+            for (int k = 0; k < K; k++) v[j][k] = s + j < nsplit ? __ldcg(P + (size_t)(s + j) * split_stride + off[k]) : 0.f;
 #pragma unroll
-        for (int k = 0; k < K; k++) a[k] = __ldcg(P + (size_t)s * split_stride + off[k]);
+        for (int j = 0; j < NB; j++)
 #pragma unroll
-        for (int k = 0; k < K; k++) out[k] += a[k];
+            for (int k = 0; k < K; k++) out[k] += v[j][k];
     }
 }
 
