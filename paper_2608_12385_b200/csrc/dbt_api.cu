@@ -93,6 +93,7 @@ struct dbt_model {
     struct ActBase { const void *base; };
     std::map<const CUtensorMap *, ActBase> act_base;
     std::map<std::tuple<const CUtensorMap *, int, int>, CUtensorMap> act3d;
+    bool fuse_qkv;     // decode steps: the attention kernel does the Q|K|V epilogue itself (DBT_FUSE_QKV=0 keeps the kernel)
     bool l2_prefetch;  // GEMM launches ask the L2 for the next GEMM's weights (opt-in, DBT_L2_PREFETCH=1)
     bool mega;      // dense bf16, small batch: the whole decode step as one persistent kernel
     struct MegaSlot { int B, grouped; };
@@ -543,7 +544,8 @@ int split_slots(const dbt_model *m, int n_tile) {
         forced = e ? atoi(e) : 0;
     }
     if (forced > 0) return forced;
-    return (n_tile <= 64 ? 2 : 1) * m->num_sms;
+    int sms = m->num_sms > 0 ? m->num_sms : 148;  // the operator-level entry points carry no device query
+    return (n_tile <= 64 ? 2 : 1) * sms;
 }
 
 template <int N_TILE>
@@ -621,8 +623,19 @@ dbt_status run_gemm_tc(dbt_model *m, const TcCall &c, int n_tile, int *nsplit_ou
     return fail(m, DBT_ERR_UNSUPPORTED, "row tile %d", n_tile);
 }
 
+// Inputs of the Q|K|V epilogue when the attention kernel does that work itself (decode steps).
+struct QkvFuse {
+    const float *P;
+    int nsplit;
+    size_t stride;
+    const float *ss;
+    int ss_tiles, ss_ld;
+    const float *coup_a;
+};
+
 template <int DH>
-dbt_status run_attention_mma(dbt_model *m, const RowMap &rm, int grouped, int layer, double kv_bytes) {
+dbt_status run_attention_mma(dbt_model *m, const RowMap &rm, int grouped, int layer, double kv_bytes,
+                             const QkvFuse *qf = nullptr) {
     const dbt_config &c = m->cfg;
     const Workspace &w = m->ws;
     int items = rm.B * rm.cn, G = c.n_q_heads / c.n_kv_heads;
@@ -644,6 +657,20 @@ dbt_status run_attention_mma(dbt_model *m, const RowMap &rm, int grouped, int la
     p.Ob = w.Ob;
     p.lo_off = m->act_parts == 2 ? (size_t)m->Rmax * c.n_q_heads * c.head_dim : (size_t)0;
     p.status = w.status;
+    if (qf) {
+        p.qkv_P = qf->P;
+        p.qkv_nsplit = qf->nsplit;
+        p.qkv_stride = qf->stride;
+        p.ss = qf->ss;
+        p.ss_tiles = qf->ss_tiles;
+        p.ss_ld = qf->ss_ld;
+        p.d_norm = c.d_model;
+        p.eps = c.rms_eps;
+        p.coup_a = qf->coup_a;
+        p.rope = w.rope;
+        p.kpool = reinterpret_cast<__nv_bfloat16 *>(m->kv_pool) + (size_t)layer * 2 * plane * c.head_dim;
+        p.vpool = p.kpool + (size_t)plane * c.head_dim;
+    }
     if (items > kAttMaxItems) return fail(m, DBT_ERR_CAPACITY, "attention rows %d exceed %d", items, kAttMaxItems);
     dim3 grid(2 * m->num_sms);  // two resident CTAs per SM; each takes an equal share of all K/V tiles
     // up to 8 query rows per KV head over both paths: the transposed-product variant (fixed per
@@ -765,12 +792,15 @@ dbt_status run_layers_tc(dbt_model *m, const RowMap &rm, int grouped, int n_tile
         qkv.nseg = 3; qkv.X = &m->map_Xb; qkv.K = d; qkv.R = R; qkv.P = w.P; qkv.P_floats = w.P_floats; qkv.parts = m->act_parts; qkv.lo_row0 = m->Rmax; qkv.tag = "gemm_qkv";
         qkv.pf_ptr[0] = lw.wo; qkv.pf_bytes[0] = (size_t)d * qd * sizeof(WT);
         if ((st = run_gemm_tc(m, qkv, n_tile, &nsp, &sstride)) != DBT_OK) return st;
-        LAUNCH(m, "qkv_epilogue", 0, qkv_epilogue_kernel<WT>, dim3(Bc, c.n_q_heads + c.n_kv_heads), 64, 0, w.P, nsp, sstride, w.Q, rm, grouped, c.n_q_heads,
-               c.n_kv_heads, c.head_dim, lw.coup_a, w.rope, w.seq_len, w.page_table, m->pages_per_seq_max, c.num_pages,
-               c.page_size, kpool, vpool, w.status, (const float *)nullptr, 0, 0, d, c.rms_eps);
+        const bool fuse = m->fuse_qkv && m->att_fast && rm.cn == 1;
+        QkvFuse qf{w.P, nsp, sstride, nullptr, 0, 0, lw.coup_a};
+        if (!fuse)
+            LAUNCH(m, "qkv_epilogue", 0, qkv_epilogue_kernel<WT>, dim3(Bc, c.n_q_heads + c.n_kv_heads), 64, 0, w.P, nsp, sstride, w.Q, rm, grouped, c.n_q_heads,
+                   c.n_kv_heads, c.head_dim, lw.coup_a, w.rope, w.seq_len, w.page_table, m->pages_per_seq_max, c.num_pages,
+                   c.page_size, kpool, vpool, w.status, (const float *)nullptr, 0, 0, d, c.rms_eps);
         if (m->att_fast)
-            st = c.head_dim == 128 ? run_attention_mma<128>(m, rm, grouped, l, kv_bytes)
-                                   : run_attention_mma<64>(m, rm, grouped, l, kv_bytes);
+            st = c.head_dim == 128 ? run_attention_mma<128>(m, rm, grouped, l, kv_bytes, fuse ? &qf : nullptr)
+                                   : run_attention_mma<64>(m, rm, grouped, l, kv_bytes, fuse ? &qf : nullptr);
         else if (c.head_dim == 128)
             st = run_attention<WT, 128>(m, rm, grouped, kpool, vpool, att_split, kv_bytes, true);
         else
@@ -857,8 +887,8 @@ dbt_status step_tc(dbt_model *m, const int32_t *tokens_dev, int B, int grouped, 
     size_t sstride;
     if ((st = run_layers_tc(m, rm, grouped, n_tile, true, &mode, &nsp, &sstride)) != DBT_OK) return st;
     if ((st = run_head_tc(m, B, grouped, B, 1, 0, n_tile, mode, nsp, sstride)) != DBT_OK) return st;
-    LAUNCH(m, "readout", 0, readout_kernel, B, 1024, 0, w.Z, B, c.vocab, grouped, next_dev, alpha_dev);
-    LAUNCH(m, "advance_len", 0, advance_len_kernel, (B + 127) / 128, 128, 0, w.seq_len, B, 1);
+    // the readout also bumps the sequence lengths: nothing after it in the step reads them
+    LAUNCH(m, "readout", 0, readout_kernel, B, 1024, 0, w.Z, B, c.vocab, grouped, next_dev, alpha_dev, w.seq_len, 1);
     size_t zb = sizeof(float) * (size_t)B * c.vocab;
     if (z1_dev) CUDA_TRY(m, cudaMemcpyAsync(z1_dev, w.Z, zb, cudaMemcpyDeviceToDevice, m->stream));
     if (z2_dev && grouped)
@@ -1012,8 +1042,8 @@ dbt_status step_fused(dbt_model *m, const int32_t *tokens_dev, int B, int groupe
     if ((st = run_embed_fused<WT>(m, tokens_dev, 1, 0, rm, R)) != DBT_OK) return st;
     if ((st = run_layers_fused(m, rm, grouped, n_tile)) != DBT_OK) return st;
     if ((st = run_head_fused(m, rm, grouped, n_tile)) != DBT_OK) return st;
-    LAUNCH(m, "readout", 0, readout_kernel, B, 1024, 0, w.Z, B, c.vocab, grouped, next_dev, alpha_dev);
-    LAUNCH(m, "advance_len", 0, advance_len_kernel, (B + 127) / 128, 128, 0, w.seq_len, B, 1);
+    // the readout also bumps the sequence lengths: nothing after it in the step reads them
+    LAUNCH(m, "readout", 0, readout_kernel, B, 1024, 0, w.Z, B, c.vocab, grouped, next_dev, alpha_dev, w.seq_len, 1);
     size_t zb = sizeof(float) * (size_t)B * c.vocab;
     if (z1_dev) CUDA_TRY(m, cudaMemcpyAsync(z1_dev, w.Z, zb, cudaMemcpyDeviceToDevice, m->stream));
     if (z2_dev && grouped)
@@ -1087,12 +1117,15 @@ dbt_status run_layers_wide(dbt_model *m, const RowMap &rm, int grouped, int n_ti
         qkv.W[2] = &mp.wv; qkv.n_out[2] = kvd; qkv.rows[2] = Bc;
         qkv.nseg = 3;
         if ((st = run_gemm_tc(m, qkv, n_tile, &nsp, &sstride)) != DBT_OK) return st;
-        LAUNCH(m, "qkv_epilogue", 0, qkv_epilogue_kernel<WT>, dim3(Bc, c.n_q_heads + c.n_kv_heads), 64, 0, w.P, nsp, sstride,
-               w.Q, rm, grouped, c.n_q_heads, c.n_kv_heads, c.head_dim, lw.coup_a, w.rope, w.seq_len, w.page_table,
-               m->pages_per_seq_max, c.num_pages, c.page_size, kpool, vpool, w.status, (const float *)w.ss, ss_tiles, ss_ld, d,
-               c.rms_eps);
-        st = c.head_dim == 128 ? run_attention_mma<128>(m, rm, grouped, l, kv_bytes)
-                               : run_attention_mma<64>(m, rm, grouped, l, kv_bytes);
+        const bool fuse = m->fuse_qkv && rm.cn == 1;
+        QkvFuse qf{w.P, nsp, sstride, w.ss, ss_tiles, ss_ld, lw.coup_a};
+        if (!fuse)
+            LAUNCH(m, "qkv_epilogue", 0, qkv_epilogue_kernel<WT>, dim3(Bc, c.n_q_heads + c.n_kv_heads), 64, 0, w.P, nsp, sstride,
+                   w.Q, rm, grouped, c.n_q_heads, c.n_kv_heads, c.head_dim, lw.coup_a, w.rope, w.seq_len, w.page_table,
+                   m->pages_per_seq_max, c.num_pages, c.page_size, kpool, vpool, w.status, (const float *)w.ss, ss_tiles, ss_ld, d,
+                   c.rms_eps);
+        st = c.head_dim == 128 ? run_attention_mma<128>(m, rm, grouped, l, kv_bytes, fuse ? &qf : nullptr)
+                               : run_attention_mma<64>(m, rm, grouped, l, kv_bytes, fuse ? &qf : nullptr);
         if (st != DBT_OK) return st;
         TcCall op = call("gemm_o", &m->map_Ob, qd);
         op.W[0] = &mp.wo; op.n_out[0] = d; op.rows[0] = R; op.nseg = 1;
@@ -1154,8 +1187,8 @@ dbt_status step_wide(dbt_model *m, const int32_t *tokens_dev, int B, int grouped
     if ((st = run_embed_wide<WT>(m, tokens_dev, 1, 0, rm, R)) != DBT_OK) return st;
     if ((st = run_layers_wide(m, rm, grouped, n_tile)) != DBT_OK) return st;
     if ((st = run_head_wide(m, rm, grouped, n_tile)) != DBT_OK) return st;
-    LAUNCH(m, "readout", 0, readout_kernel, B, 1024, 0, w.Z, B, c.vocab, grouped, next_dev, alpha_dev);
-    LAUNCH(m, "advance_len", 0, advance_len_kernel, (B + 127) / 128, 128, 0, w.seq_len, B, 1);
+    // the readout also bumps the sequence lengths: nothing after it in the step reads them
+    LAUNCH(m, "readout", 0, readout_kernel, B, 1024, 0, w.Z, B, c.vocab, grouped, next_dev, alpha_dev, w.seq_len, 1);
     size_t zb = sizeof(float) * (size_t)B * c.vocab;
     if (z1_dev) CUDA_TRY(m, cudaMemcpyAsync(z1_dev, w.Z, zb, cudaMemcpyDeviceToDevice, m->stream));
     if (z2_dev && grouped)
@@ -1472,8 +1505,8 @@ dbt_status step_impl(dbt_model *m, const int32_t *tokens_dev, int B, int grouped
            (const WT *)m->w.embed_branch, m->w.embed_norm_g, c.rms_eps, c.d_model, c.vocab, w.S, w.status);
     if ((st = run_layers<WT>(m, rm, grouped, true)) != DBT_OK) return st;
     if ((st = run_head<WT>(m, R, 1, 0)) != DBT_OK) return st;
-    LAUNCH(m, "readout", 0, readout_kernel, B, 1024, 0, w.Z, B, c.vocab, grouped, next_dev, alpha_dev);
-    LAUNCH(m, "advance_len", 0, advance_len_kernel, (B + 127) / 128, 128, 0, w.seq_len, B, 1);
+    // the readout also bumps the sequence lengths: nothing after it in the step reads them
+    LAUNCH(m, "readout", 0, readout_kernel, B, 1024, 0, w.Z, B, c.vocab, grouped, next_dev, alpha_dev, w.seq_len, 1);
     size_t zb = sizeof(float) * (size_t)B * c.vocab;
     if (z1_dev) CUDA_TRY(m, cudaMemcpyAsync(z1_dev, w.Z, zb, cudaMemcpyDeviceToDevice, m->stream));
     if (z2_dev && grouped)
@@ -1596,6 +1629,8 @@ dbt_status dbt_create(const dbt_config *cfg, const dbt_weights *w, void *kv_pool
     {
         // Opt-in (DBT_L2_PREFETCH=1): measured no faster (1.49 vs 1.45 ms per step at batch 16 on the
         // 1B model); the GEMMs of a decode step wait on dependency latency, not on HBM bandwidth.
+        const char *fq = getenv("DBT_FUSE_QKV");
+        m->fuse_qkv = m->att_fast && !(fq && strcmp(fq, "0") == 0);
         const char *pf = getenv("DBT_L2_PREFETCH");
         m->l2_prefetch = pf && strcmp(pf, "1") == 0;
     }

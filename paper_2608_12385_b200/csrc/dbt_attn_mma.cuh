@@ -23,6 +23,7 @@
 // order at the end of a segment.  All waits are bounded.
 #pragma once
 
+#include "dbt_fused.cuh"
 #include "dbt_gemm_tc.cuh"
 
 namespace dbt {
@@ -38,6 +39,19 @@ struct AttnParams {
     __nv_bfloat16 *Ob;  // [rows][q_dim] attention output, hi plane (+ lo plane at lo_off)
     size_t lo_off;
     int *status;
+    // Decode steps take the Q|K|V GEMM's split-K partials directly (no kernel in between): each CTA
+    // builds its pair's queries itself (1/rms, RoPE, Q~_2 = Q_2 + a*Q_1, Eq. asymattn), and the CTA that
+    // owns the pair's last stage computes the new K_1, V_1 row, writes it to the pool for later steps
+    // and patches it into the staged page.  qkv_P == nullptr: Q comes from `Q`, the cache is complete.
+    const float *qkv_P;  // [nsplit][rows][q_dim | kv_dim | kv_dim]
+    int qkv_nsplit;
+    size_t qkv_stride;
+    const float *ss;  // shares of sum(S^2) per row (nullptr: the GEMM input was already normalised)
+    int ss_tiles, ss_ld, d_norm;
+    float eps;
+    const float *coup_a;
+    const float2 *rope;
+    __nv_bfloat16 *kpool, *vpool;  // this layer's K and V planes
 };
 
 constexpr int kAttTile = 64;       // tokens per pipeline stage (4 pages)
@@ -56,7 +70,7 @@ struct AttCfg {
     // scratch: one [16][DH + 8] fp32 slot (Q tile / warp fold; the padding keeps the fold's
     // fragment-shaped accesses off a single bank), m, l, flag, row tables
     static constexpr int kFoldStride = DH + 8;
-    static constexpr int kScratchBytes = (16 * kFoldStride + 2 * 16 + 8 + 2 * kAttMaxItems + 8) * 4;
+    static constexpr int kScratchBytes = (16 * kFoldStride + 2 * 16 + 8 + 2 * kAttMaxItems + 8) * 4 + 2 * DH * 2 + 32;
     static constexpr int kSmemBytes = kStages * kStageBytes + 1024 + 128 + kScratchBytes;
 };
 
@@ -113,6 +127,8 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
     int *flag = reinterpret_cast<int *>(sc_l + 16);                                 // [0] last?, [1] longest pair
     int *cum = flag + 8;                 // [items + 1] prefix of tiles per row
     int *nk_s = cum + kAttMaxItems + 1;  // [items] visible keys per row
+    __nv_bfloat16 *kv_new =  // [2][DH] this step's K, V row (16-byte aligned)
+        reinterpret_cast<__nv_bfloat16 *>((reinterpret_cast<uintptr_t>(nk_s + kAttMaxItems) + 15) & ~(uintptr_t)15);
 
     DBT_TL_DECL;
     int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -203,6 +219,19 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
     bool ok = true;
     int it = 0;
     const float qscale = kLog2e / sqrtf((float)DH);
+    // The staged copy of the page that holds this step's position was read while the row was being
+    // written: overwrite the row in shared memory with the values computed here (16-byte pieces,
+    // lanes 0..15 the K row, lanes 16..31 the V row; DH = 64 uses half of each).
+    auto patch_new_row = [&](uint32_t kpage, uint32_t vpage, int row) {
+        int piece = lane & 15;
+        if (piece < DH / 8) {
+            int sg = row * HALVES + (piece >> 3);
+            uint32_t dst = (lane < 16 ? kpage : vpage) + sg * 128 + (((piece & 7) ^ (sg & 7)) << 4);
+            const uint4 v = *reinterpret_cast<const uint4 *>(kv_new + (lane < 16 ? 0 : DH) + piece * 8);
+            asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(dst), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+        }
+        __syncwarp();
+    };
     for (int u = u0; u < u1;) {
         int ui = cum[item + 1] - cum[item], base = cum[item] * p.n_kv;
         int g = (u - base) / ui, t0 = (u - base) % ui;
@@ -212,15 +241,69 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
         // Query tile (16 rows x DH, fp32) into shared memory, then mma A fragments (bf16),
         // pre-scaled by log2(e)/sqrt(d_h).  Rows: G primary heads, then G coupled branch heads.
         consumer_sync();  // the previous segment is done with the scratch
-        for (int idx = tid; idx < 16 * DH / 4; idx += 128) {
-            int q = idx / (DH / 4), c4 = idx % (DH / 4);
-            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (q < nq_act) {
-                int row = q < p.G ? item : Bc + item;
-                int h = g * p.G + (q < p.G ? q : q - p.G);
-                v = __ldcg(reinterpret_cast<const float4 *>(p.Q + (size_t)row * q_dim + (size_t)h * DH) + c4);
+        const bool owns_last = p.qkv_P != nullptr && u + (t1 - t0) == pair_end;  // this segment ends the pair
+        if (p.qkv_P == nullptr) {
+            for (int idx = tid; idx < 16 * DH / 4; idx += 128) {
+                int q = idx / (DH / 4), c4 = idx % (DH / 4);
+                float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (q < nq_act) {
+                    int row = q < p.G ? item : Bc + item;
+                    int h = g * p.G + (q < p.G ? q : q - p.G);
+                    v = __ldcg(reinterpret_cast<const float4 *>(p.Q + (size_t)row * q_dim + (size_t)h * DH) + c4);
+                }
+                reinterpret_cast<float4 *>(sc_o)[idx] = v;
             }
-            reinterpret_cast<float4 *>(sc_o)[idx] = v;
+        } else {
+            constexpr int half = DH / 2;
+            const int kv_dim = p.n_kv * DH, ldp = q_dim + 2 * kv_dim, pos = nkeys - 1;
+            const size_t p1 = (size_t)item * ldp, p2 = (size_t)(p.grouped ? Bc + item : item) * ldp;
+            float rs1, rs2;
+            row_scale2(p.ss, p.ss_tiles, p.ss_ld, item, p.grouped ? Bc + item : item, p.d_norm, p.eps, rs1, rs2);
+            for (int idx = tid; idx < (16 - nq_act) * DH / 4; idx += 128)  // unused query rows
+                reinterpret_cast<float4 *>(sc_o + (size_t)nq_act * DH)[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int idx = tid; idx < p.G * half; idx += 128) {
+                int j = idx / half, i = idx % half;
+                int o0 = (g * p.G + j) * DH + i, o1 = o0 + half;
+                float2 t = p.rope[(size_t)pos * half + i];
+                const size_t offs[4] = {p1 + o0, p1 + o1, p2 + o0, p2 + o1};
+                float sm[4];
+                sum_splits_k<4, 8>(p.qkv_P, p.qkv_stride, p.qkv_nsplit, offs, sm);
+                float x0 = rs1 * sm[0], x1 = rs1 * sm[1];
+                float r0 = x0 * t.x - x1 * t.y, r1 = x1 * t.x + x0 * t.y;
+                sc_o[(size_t)j * DH + i] = r0;
+                sc_o[(size_t)j * DH + i + half] = r1;
+                if (p.grouped) {
+                    float y0 = rs2 * sm[2], y1 = rs2 * sm[3];
+                    sc_o[(size_t)(p.G + j) * DH + i] = (y0 * t.x - y1 * t.y) + p.coup_a[o0] * r0;
+                    sc_o[(size_t)(p.G + j) * DH + i + half] = (y1 * t.x + y0 * t.y) + p.coup_a[o1] * r1;
+                }
+            }
+            if (owns_last && tid < half) {
+                // K_1 = RoPE(N_1 W_K), V_1 = N_1 W_V of this step's token, for this KV head
+                int i = tid;
+                float2 t = p.rope[(size_t)pos * half + i];
+                size_t ko = p1 + q_dim + (size_t)g * DH + i, vo = ko + kv_dim;
+                const size_t offs[4] = {ko, ko + half, vo, vo + half};
+                float sm[4];
+                sum_splits_k<4, 8>(p.qkv_P, p.qkv_stride, p.qkv_nsplit, offs, sm);
+                float x0 = rs1 * sm[0], x1 = rs1 * sm[1];
+                __nv_bfloat16 k0 = __float2bfloat16_rn(x0 * t.x - x1 * t.y), k1 = __float2bfloat16_rn(x1 * t.x + x0 * t.y);
+                __nv_bfloat16 v0 = __float2bfloat16_rn(rs1 * sm[2]), v1 = __float2bfloat16_rn(rs1 * sm[3]);
+                kv_new[i] = k0;
+                kv_new[i + half] = k1;
+                kv_new[DH + i] = v0;
+                kv_new[DH + i + half] = v1;
+                int page = __ldg(p.page_table + (size_t)p.rm.seq(item) * p.pt_stride + (pos >> 4));
+                if (page < 0 || page >= p.num_pages) {
+                    if (i == 0) report(p.status, kStatusBadPage, page);
+                } else {
+                    size_t base = (((size_t)page * p.n_kv + g) * 16 + (pos & 15)) * DH;
+                    p.kpool[base + i] = k0;
+                    p.kpool[base + i + half] = k1;
+                    p.vpool[base + i] = v0;
+                    p.vpool[base + i + half] = v1;
+                }
+            }
         }
         consumer_sync();
         int pair = item * p.n_kv + g;
@@ -265,7 +348,8 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
                         }
                         __syncwarp();
                     }
-                    // S = Q K^T for this warp's 16 tokens: two 8-token column blocks
+                    if (owns_last && t == ui - 1 && ((nkeys - 1) >> 4 & 3) == warp) patch_new_row(kpage, vpage, (nkeys - 1) & 15);
+                // S = Q K^T for this warp's 16 tokens: two 8-token column blocks
                     float sacc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
                     {
                         int r = (lane & 7) + ((lane >> 4) << 3);  // token row this lane addresses
@@ -470,6 +554,7 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
                         }
                         __syncwarp();
                     }
+                    if (owns_last && t == ui - 1 && ((nkeys - 1) >> 4 & 3) == warp) patch_new_row(kpage, vpage, (nkeys - 1) & 15);
                     // S^T = K Q^T: K rows as the A operand
                     float sacc[4] = {0.f, 0.f, 0.f, 0.f};
                     {

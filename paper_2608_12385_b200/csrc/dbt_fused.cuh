@@ -41,10 +41,9 @@ __device__ __forceinline__ float sum_splits(const float *P, size_t split_stride,
 
 // The same for K outputs at once: the loads of all K outputs (two splits of each) are in flight
 // together.  Each output is still added in split order.
-template <int K>
+template <int K, int NB = (K <= 2 ? 4 : 2)>  // NB splits per batch: K * NB loads in flight
 __device__ __forceinline__ void sum_splits_k(const float *P, size_t split_stride, int nsplit, const size_t (&off)[K],
                                              float (&out)[K]) {
-    constexpr int NB = K <= 2 ? 4 : 2;  // splits per batch: eight loads in flight
 #pragma unroll
     for (int k = 0; k < K; k++) out[k] = 0.f;
     for (int s = 0; s < nsplit; s += NB) {
@@ -73,6 +72,29 @@ __device__ __forceinline__ float row_scale(const float *ss, int ss_tiles, int ss
         for (int j = 0; j < 8; j++) a += v[j];
     }
     return 1.f / sqrtf(a / (float)d_norm + eps);
+}
+
+// The same for two rows at once (a primary row and its branch twin), their loads in flight together.
+__device__ __forceinline__ void row_scale2(const float *ss, int ss_tiles, int ss_ld, int row_a, int row_b, int d_norm,
+                                           float eps, float &rs_a, float &rs_b) {
+    rs_a = rs_b = 1.f;
+    if (!ss) return;
+    float a = 0.f, b = 0.f;
+    for (int t0 = 0; t0 < ss_tiles; t0 += 8) {
+        float va[8], vb[8];
+#pragma unroll
+        for (int j = 0; j < 8; j++) {
+            va[j] = t0 + j < ss_tiles ? __ldcg(ss + (size_t)(t0 + j) * ss_ld + row_a) : 0.f;
+            vb[j] = t0 + j < ss_tiles ? __ldcg(ss + (size_t)(t0 + j) * ss_ld + row_b) : 0.f;
+        }
+#pragma unroll
+        for (int j = 0; j < 8; j++) {
+            a += va[j];
+            b += vb[j];
+        }
+    }
+    rs_a = 1.f / sqrtf(a / (float)d_norm + eps);
+    rs_b = 1.f / sqrtf(b / (float)d_norm + eps);
 }
 
 // Residual update without the row-wide reduction: S += sum_s P[s] (mode 1) or, with the c
@@ -202,7 +224,8 @@ __global__ void __launch_bounds__(64) qkv_epilogue_kernel(
     int q_dim = n_q * dh, kv_dim = n_kv * dh, ldp = q_dim + 2 * kv_dim;
     float2 t = rope_tab[(size_t)pos * half + i];
     size_t p1 = (size_t)item * ldp, p2 = (size_t)(Bc + item) * ldp;
-    const float rs1 = row_scale(ss, ss_tiles, ss_ld, item, d_norm, eps);  // 1/rms when the GEMM input was g*S
+    float rs1, rs2;  // 1/rms when the GEMM input was g*S
+    row_scale2(ss, ss_tiles, ss_ld, item, grouped ? Bc + item : item, d_norm, eps, rs1, rs2);
     if (hh < n_q) {
         int o0 = hh * dh + i, o1 = o0 + half;
         const size_t offs[4] = {p1 + o0, p1 + o1, grouped ? p2 + o0 : p1 + o0, grouped ? p2 + o1 : p1 + o1};
@@ -214,7 +237,6 @@ __global__ void __launch_bounds__(64) qkv_epilogue_kernel(
         q1[o0] = r0;
         q1[o1] = r1;
         if (grouped) {
-            const float rs2 = row_scale(ss, ss_tiles, ss_ld, Bc + item, d_norm, eps);
             float y0 = rs2 * sm[2], y1 = rs2 * sm[3];
             float *q2 = Q + (size_t)(Bc + item) * q_dim;
             q2[o0] = (y0 * t.x - y1 * t.y) + coup_a[o0] * r0;
@@ -255,7 +277,8 @@ __global__ void __launch_bounds__(256) swiglu_couple_kernel(const float *P, int 
     int b = blockIdx.x, f = blockIdx.y * blockDim.x + threadIdx.x;
     if (f >= F) return;
     size_t p1 = (size_t)b * 2 * F + f;
-    const float rs1 = row_scale(ss, ss_tiles, ss_ld, b, d_norm, eps);
+    float rs1, rs2;
+    row_scale2(ss, ss_tiles, ss_ld, b, grouped ? Bc + b : b, d_norm, eps, rs1, rs2);
     size_t p2 = grouped ? (size_t)(Bc + b) * 2 * F + f : p1;
     const size_t offs[4] = {p1, p1 + F, p2, p2 + F};
     float sm[4];
@@ -263,7 +286,6 @@ __global__ void __launch_bounds__(256) swiglu_couple_kernel(const float *P, int 
     float h1 = silu(rs1 * sm[0]) * (rs1 * sm[1]);
     store_split(Hb, (size_t)b * F + f, lo_off, h1);
     if (grouped) {
-        const float rs2 = row_scale(ss, ss_tiles, ss_ld, Bc + b, d_norm, eps);
         float h2 = silu(rs2 * sm[2]) * (rs2 * sm[3]);
         if (coup_b) h2 += coup_b[f] * h1;
         store_split(Hb, (size_t)(Bc + b) * F + f, lo_off, h2);

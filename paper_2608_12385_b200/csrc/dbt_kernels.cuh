@@ -380,7 +380,8 @@ __global__ void attn_merge_kernel(const float *part, int nsplit, int NQ, int DH,
 // ---------------------------------------------------------------------------------------
 // Readout (Eq. alpha, Eq. mixloss): p = softmax(z_1), q = softmax(z_2),
 // alpha = clip_[0.5,1](sum p^2), next = argmax(alpha p + (1-alpha) q), lowest index on ties.
-// Primary-only: next = argmax z_1.  One block per sequence.
+// Primary-only: next = argmax z_1.  One block per sequence; the block also advances its sequence's
+// length when asked to (the last kernel of a decode step).
 struct ArgBest {
     float v;
     int i;
@@ -391,7 +392,7 @@ __device__ __forceinline__ ArgBest better(ArgBest a, ArgBest b) {
 }
 
 __global__ void __launch_bounds__(1024) readout_kernel(const float *Z, int B, int V, int grouped,
-                                                       int32_t *next, float *alpha_out) {
+                                                       int32_t *next, float *alpha_out, int32_t *seq_len, int advance) {
     pdl_enter();
     __shared__ float scratch[32];
     __shared__ float bv[32];
@@ -444,6 +445,7 @@ __global__ void __launch_bounds__(1024) readout_kernel(const float *Z, int B, in
         if (lane == 0) {
             if (next) next[b] = t.i;
             if (alpha_out && grouped) alpha_out[b] = alpha;
+            if (seq_len) seq_len[b] += advance;  // the step's last use of the lengths was the last layer's attention
         }
     }
 }
