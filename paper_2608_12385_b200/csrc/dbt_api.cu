@@ -31,7 +31,7 @@ struct Workspace {
     // fp32 activations, rows = Rmax unless noted
     float *S, *X, *Q, *Kn, *Vn, *O, *G1, *M, *Z, *part, *Zrows;
     float2 *rope;
-    int32_t *seq_len, *page_table, *status, *tokens_stage, *next_stage, *att_tickets, *gemm_tickets;
+    int32_t *seq_len, *page_table, *status, *tokens_stage, *next_stage, *att_tickets, *att_tickets2, *gemm_tickets;
     float *alpha_stage;
     // MoE
     float *rlogits, *rwts, *Hexp, *Yexp, *Msh, *Hsh;
@@ -189,6 +189,7 @@ size_t carve(const dbt_config &c, char *base, Workspace *ws, int *Rmax_out, int 
     w.page_table = k.take<int32_t>((size_t)c.max_batch * pps);
     w.status = k.take<int32_t>(4);
     w.att_tickets = k.take<int32_t>((size_t)Rmax * c.n_kv_heads);
+    w.att_tickets2 = k.take<int32_t>((size_t)Rmax * c.n_kv_heads * kAttMaxGroups);
     w.gemm_tickets = k.take<int32_t>(4096);
     w.tokens_stage = k.take<int32_t>(c.max_batch);
     w.next_stage = k.take<int32_t>(c.max_batch);
@@ -654,6 +655,7 @@ dbt_status run_attention_mma(dbt_model *m, const RowMap &rm, int grouped, int la
     p.seq_len = w.seq_len;
     p.part = w.part;
     p.tickets = w.att_tickets;
+    p.tickets2 = w.att_tickets2;
     p.Ob = w.Ob;
     p.lo_off = m->act_parts == 2 ? (size_t)m->Rmax * c.n_q_heads * c.head_dim : (size_t)0;
     p.status = w.status;
@@ -1670,6 +1672,7 @@ dbt_status dbt_create(const dbt_config *cfg, const dbt_weights *w, void *kv_pool
     if (e == cudaSuccess) e = cudaMemsetAsync(m->ws.seq_len, 0, sizeof(int32_t) * cfg->max_batch, m->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(m->ws.status, 0, sizeof(int32_t) * 4, m->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(m->ws.att_tickets, 0, sizeof(int32_t) * (size_t)m->Rmax * cfg->n_kv_heads, m->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(m->ws.att_tickets2, 0, sizeof(int32_t) * (size_t)m->Rmax * cfg->n_kv_heads * kAttMaxGroups, m->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(m->ws.gemm_tickets, 0, sizeof(int32_t) * 4096, m->stream);
     if (e == cudaSuccess && moe) {
         e = cudaMemsetAsync(m->ws.last_experts, 0xff, sizeof(int32_t) * (size_t)cfg->n_layers * 2 * cfg->max_batch * kmax_of(*cfg), m->stream);
@@ -1786,6 +1789,7 @@ dbt_status dbt_reset(dbt_model *m) {
     CUDA_TRY(m, cudaMemsetAsync(m->ws.seq_len, 0, sizeof(int32_t) * m->cfg.max_batch, m->stream));
     CUDA_TRY(m, cudaMemsetAsync(m->ws.status, 0, sizeof(int32_t) * 4, m->stream));
     CUDA_TRY(m, cudaMemsetAsync(m->ws.att_tickets, 0, sizeof(int32_t) * (size_t)m->Rmax * m->cfg.n_kv_heads, m->stream));
+    CUDA_TRY(m, cudaMemsetAsync(m->ws.att_tickets2, 0, sizeof(int32_t) * (size_t)m->Rmax * m->cfg.n_kv_heads * kAttMaxGroups, m->stream));
     CUDA_TRY(m, cudaMemsetAsync(m->ws.gemm_tickets, 0, sizeof(int32_t) * 4096, m->stream));
     if (m->ws.mega_sync) CUDA_TRY(m, cudaMemsetAsync(m->ws.mega_sync, 0, sizeof(unsigned int) * 8, m->stream));
     std::fill(m->len_host.begin(), m->len_host.end(), 0);

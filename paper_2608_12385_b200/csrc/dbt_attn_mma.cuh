@@ -36,6 +36,7 @@ struct AttnParams {
     const int32_t *page_table, *seq_len;
     float *part;        // [CTAs + pairs][16][DH + 2] segment partials
     int *tickets;       // [rows][n_kv] arrival counters (zero between launches)
+    int *tickets2;      // [rows][n_kv][kAttMaxGroups] arrival counters of the segment groups
     __nv_bfloat16 *Ob;  // [rows][q_dim] attention output, hi plane (+ lo plane at lo_off)
     size_t lo_off;
     int *status;
@@ -58,7 +59,9 @@ constexpr int kAttTile = 64;       // tokens per pipeline stage (4 pages)
 constexpr int kAttWarps = 4;       // consumer warps, one page each
 constexpr int kAttMaxItems = 256;  // rows per launch (prefill chunks and batches stay below)
 constexpr int kAttMinUnits = 4;    // a CTA takes at least 4 tiles (256 tokens)
-constexpr int kAttMaxSeg = 32;     // segments per pair the final fold handles at once
+constexpr int kAttMaxSeg = 256;    // most segments a (sequence, KV head) pair is split into
+constexpr int kAttGroup = 8;       // segments merged at once (one round of loads)
+constexpr int kAttMaxGroups = kAttMaxSeg / kAttGroup;
 constexpr float kLog2e = 1.4426950408889634f;
 
 template <int DH>
@@ -711,47 +714,37 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
                 }
             }
         }
-        // ---- the last segment of this pair to arrive folds all of them in segment order
-        int is_last = 0;
-        if (nseg > 1) {
-            consumer_sync();
-            if (tid == 0) {
-                int *tk = p.tickets + pair;
-                int tkt = atomicAdd(tk, 1);
-                int last = tkt == nseg - 1;
-                if (last) {
-                    atomicExch(tk, 0);
-                    __threadfence();
-                }
-                flag[0] = last;
-            }
-            consumer_sync();
-            is_last = flag[0];
-        }
-        if (is_last) {
-            const float *pbase = p.part + (size_t)(first_cta + pair) * 16 * (DH + 2);
+        // ---- merging a pair's segments.  Up to kAttGroup segments: the last one to arrive merges them
+        // all, in segment order, and writes the output.  More: the segments form groups of kAttGroup;
+        // the last arrival of a group merges it in place into the group's first slot, and the last
+        // group to finish merges the group results: two short merges on several CTAs instead of one
+        // long one on a single CTA (a pair of a 32k-token sequence has ~35 segments).
+        // merge n partials at slots pbase + j * slot_stride; final: normalise and write the output,
+        // else leave the merged (unnormalised) state in the first slot
+        auto merge = [&](float *pbase, int slot_stride, int n, bool final) {
+            const size_t sstr = (size_t)slot_stride * 16 * (DH + 2);
             for (int idx0 = tid; idx0 < nq_act * DH; idx0 += 2 * 128) {
-                // two outputs per thread, eight segments of each in flight
+                // two outputs per thread, eight partials of each in flight
                 const float *pq[2];
                 float M[2] = {-INFINITY, -INFINITY}, L[2] = {0.f, 0.f}, X[2] = {0.f, 0.f};
                 bool act[2];
-                int ee[2];
+                int ee[2], qq[2];
 #pragma unroll
                 for (int a = 0; a < 2; a++) {
                     int idx = idx0 + a * 128;
                     act[a] = idx < nq_act * DH;
-                    int q = act[a] ? idx / DH : 0;
+                    qq[a] = act[a] ? idx / DH : 0;
                     ee[a] = act[a] ? idx % DH : 0;
-                    pq[a] = pbase + (size_t)q * (DH + 2);
+                    pq[a] = pbase + (size_t)qq[a] * (DH + 2);
                 }
-                for (int sb = 0; sb < nseg; sb += 8) {
+                for (int sb = 0; sb < n; sb += 8) {
                     float mv[2][8], lv[2][8], ov[2][8];
 #pragma unroll
                     for (int a = 0; a < 2; a++)
 #pragma unroll
                         for (int j = 0; j < 8; j++) {
-                            bool on = act[a] && sb + j < nseg;
-                            const float *pp = pq[a] + (size_t)(sb + j) * 16 * (DH + 2);
+                            bool on = act[a] && sb + j < n;
+                            const float *pp = pq[a] + (size_t)(sb + j) * sstr;
                             mv[a][j] = on ? __ldcg(pp + DH) : -INFINITY;
                             lv[a][j] = on ? __ldcg(pp + DH + 1) : 0.f;
                             ov[a][j] = on ? __ldcg(pp + ee[a]) : 0.f;
@@ -775,17 +768,58 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
                 }
 #pragma unroll
                 for (int a = 0; a < 2; a++) {
-                    int idx = idx0 + a * 128;
-                    if (act[a]) {
-                        int q = idx / DH;
-                        int row = q < p.G ? item : Bc + item;
-                        int h = g * p.G + (q < p.G ? q : q - p.G);
+                    if (!act[a]) continue;
+                    if (final) {
+                        int row = qq[a] < p.G ? item : Bc + item;
+                        int h = g * p.G + (qq[a] < p.G ? qq[a] : qq[a] - p.G);
                         size_t o_idx = (size_t)row * q_dim + (size_t)h * DH + ee[a];
                         float x = X[a] / L[a];
                         __nv_bfloat16 hi = __float2bfloat16_rn(x);
                         p.Ob[o_idx] = hi;
                         if (p.lo_off) p.Ob[o_idx + p.lo_off] = __float2bfloat16_rn(x - __bfloat162float(hi));
+                    } else {
+                        // this thread is the only reader of the first slot's element (q, e)
+                        pbase[(size_t)qq[a] * (DH + 2) + ee[a]] = X[a];
+                        if (ee[a] == 0) {
+                            sc_m[qq[a]] = M[a];
+                            sc_l[qq[a]] = L[a];
+                        }
                     }
+                }
+            }
+            if (!final) {
+                consumer_sync();  // every thread has read the first slot's (m, l): now they may change
+                if (tid < nq_act) {
+                    pbase[(size_t)tid * (DH + 2) + DH] = sc_m[tid];
+                    pbase[(size_t)tid * (DH + 2) + DH + 1] = sc_l[tid];
+                }
+                __threadfence();
+            }
+        };
+        auto arrive = [&](int *counter, int arrivals) {  // true in the CTA that arrives last
+            consumer_sync();
+            if (tid == 0) {
+                int tkt = atomicAdd(counter, 1);
+                int last = tkt == arrivals - 1;
+                if (last) {
+                    atomicExch(counter, 0);
+                    __threadfence();
+                }
+                flag[0] = last;
+            }
+            consumer_sync();
+            return flag[0] != 0;
+        };
+        if (nseg > 1) {
+            float *slot0 = p.part + (size_t)(first_cta + pair) * 16 * (DH + 2);
+            if (nseg <= kAttGroup) {
+                if (arrive(p.tickets + pair, nseg)) merge(slot0, 1, nseg, true);
+            } else {
+                int gi = ((int)blockIdx.x - first_cta) / kAttGroup, ngroups = (nseg + kAttGroup - 1) / kAttGroup;
+                int gs = min(kAttGroup, nseg - gi * kAttGroup);
+                if (arrive(p.tickets2 + (size_t)pair * kAttMaxGroups + gi, gs)) {
+                    merge(slot0 + (size_t)gi * kAttGroup * 16 * (DH + 2), 1, gs, false);
+                    if (arrive(p.tickets + pair, ngroups)) merge(slot0, kAttGroup, ngroups, true);
                 }
             }
         }

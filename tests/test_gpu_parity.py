@@ -66,7 +66,7 @@ def test_prefill_longer_than_one_chunk_and_page_boundaries():
     teacher_forced_compare(cfg, w, tok, n_prefill=300, grouped=True)
 
 
-@pytest.mark.parametrize("ctx", [0, 1, 15, 16, 17, 63, 64, 65, 255, 256, 257, 2047, 4100])
+@pytest.mark.parametrize("ctx", [0, 1, 15, 16, 17, 63, 64, 65, 255, 256, 257, 2047, 4100, 8200])
 def test_context_lengths_around_page_and_chunk_boundaries(ctx):
     """Synthetic cache of `ctx` positions, then two grouped steps."""
     cfg = small_bf16(n_layers=1)
