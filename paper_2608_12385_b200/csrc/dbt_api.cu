@@ -93,6 +93,7 @@ struct dbt_model {
     struct ActBase { const void *base; };
     std::map<const CUtensorMap *, ActBase> act_base;
     std::map<std::tuple<const CUtensorMap *, int, int>, CUtensorMap> act3d;
+    bool evict_first;  // weight tiles and K/V pages carry the evict-first L2 hint (DBT_EVICT_FIRST=0 turns it off)
     bool fuse_qkv;     // decode steps: the attention kernel does the Q|K|V epilogue itself (DBT_FUSE_QKV=0 keeps the kernel)
     bool l2_prefetch;  // GEMM launches ask the L2 for the next GEMM's weights (opt-in, DBT_L2_PREFETCH=1)
     bool mega;      // dense bf16, small batch: the whole decode step as one persistent kernel
@@ -594,6 +595,7 @@ dbt_status run_gemm_tc(dbt_model *m, const TcCall &c, int n_tile, int *nsplit_ou
     p.grp_w_rows = c.grp_w_rows;
     p.P = c.P;
     p.status = m->ws.status;
+    p.evict_first = m->evict_first ? 1 : 0;
     for (int j = 0; j < 3; j++) {
         p.pf_ptr[j] = m->l2_prefetch ? (const char *)c.pf_ptr[j] : nullptr;
         p.pf_bytes[j] = m->l2_prefetch && c.pf_ptr[j] ? c.pf_bytes[j] : 0;
@@ -659,6 +661,7 @@ dbt_status run_attention_mma(dbt_model *m, const RowMap &rm, int grouped, int la
     p.Ob = w.Ob;
     p.lo_off = m->act_parts == 2 ? (size_t)m->Rmax * c.n_q_heads * c.head_dim : (size_t)0;
     p.status = w.status;
+    p.evict_first = m->evict_first ? 1 : 0;
     if (qf) {
         p.qkv_P = qf->P;
         p.qkv_nsplit = qf->nsplit;
@@ -1631,6 +1634,8 @@ dbt_status dbt_create(const dbt_config *cfg, const dbt_weights *w, void *kv_pool
     {
         // Opt-in (DBT_L2_PREFETCH=1): measured no faster (1.49 vs 1.45 ms per step at batch 16 on the
         // 1B model); the GEMMs of a decode step wait on dependency latency, not on HBM bandwidth.
+        const char *ef = getenv("DBT_EVICT_FIRST");
+        m->evict_first = !(ef && strcmp(ef, "0") == 0);
         const char *fq = getenv("DBT_FUSE_QKV");
         m->fuse_qkv = m->att_fast && !(fq && strcmp(fq, "0") == 0);
         const char *pf = getenv("DBT_L2_PREFETCH");
@@ -2069,3 +2074,18 @@ dbt_status dbt_op_gemm_tc(const void *W_dev, const void *X_dev, int32_t n_out, i
 }
 
 }  // extern "C"
+
+#ifdef DBT_TIMELINE
+// Instrumentation builds only: copies the kernels' timeline records out and clears the list.
+extern "C" int dbt_debug_timeline(unsigned long long *out_host, int max_records) {
+    unsigned int n = 0;
+    cudaDeviceSynchronize();
+    if (cudaMemcpyFromSymbol(&n, dbt::g_tl_n, sizeof n) != cudaSuccess) return -1;
+    if ((int)n > max_records) n = max_records;
+    if (n > (unsigned)dbt::kTlMax) n = dbt::kTlMax;
+    if (n && cudaMemcpyFromSymbol(out_host, dbt::g_tl, sizeof(unsigned long long) * 8 * n) != cudaSuccess) return -1;
+    unsigned int zero = 0;
+    cudaMemcpyToSymbol(dbt::g_tl_n, &zero, sizeof zero);
+    return (int)n;
+}
+#endif

@@ -40,6 +40,7 @@ struct AttnParams {
     __nv_bfloat16 *Ob;  // [rows][q_dim] attention output, hi plane (+ lo plane at lo_off)
     size_t lo_off;
     int *status;
+    int evict_first;  // K/V pages carry the evict-first L2 hint (read once per step)
     // Decode steps take the Q|K|V GEMM's split-K partials directly (no kernel in between): each CTA
     // builds its pair's queries itself (1/rms, RoPE, Q~_2 = Q_2 + a*Q_1, Eq. asymattn), and the CTA that
     // owns the pair's last stage computes the new K_1, V_1 row, writes it to the pool for later steps
@@ -108,6 +109,14 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map
     asm volatile(
         "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];" ::"r"(dst),
         "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_4d_hint(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2, int c3,
+                                                 uint64_t hint) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4, %5, "
+        "%6}], [%2], %7;" ::"r"(dst),
+        "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "l"(hint)
         : "memory");
 }
 __device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
@@ -184,6 +193,7 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
         // arms its barrier; up to four lanes then issue one box each (a page's K and V, both
         // 64-column pieces: 8 KB at d_h = 128), each after its own page-table lookup.
         if (lane == 0) tma_prefetch_desc(&tmKV);
+        const uint64_t pol = l2_evict_first_policy();
         bool ok = true;
         int it = 0;
         for (int u = u0; u < u1 && ok;) {
@@ -207,9 +217,17 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
                         page = 0;
                     }
                     int row = (int)(((long long)page * p.n_kv + g) * 16);
-                    tma_load_4d(tiles + s * Cfg::kStageBytes + lane * 2 * Cfg::kPageBytes, &tmKV, full_bar(s), 0, 0,
-                                (int)(p.k_row0 + row), 0);
+                    if (p.evict_first)
+                        tma_load_4d_hint(tiles + s * Cfg::kStageBytes + lane * 2 * Cfg::kPageBytes, &tmKV, full_bar(s), 0, 0,
+                                         (int)(p.k_row0 + row), 0, pol);
+                    else
+                        tma_load_4d(tiles + s * Cfg::kStageBytes + lane * 2 * Cfg::kPageBytes, &tmKV, full_bar(s), 0, 0,
+                                    (int)(p.k_row0 + row), 0);
                 }
+                // After the first stage the stream pauses until the consumers have their queries: their
+                // few small loads would otherwise queue behind hundreds of CTAs' page traffic for several
+                // microseconds, and nothing can be consumed before they return anyway.
+                if (it == 0) asm volatile("bar.sync 2, 160;" ::: "memory");
             }
             u += t1 - t0;
             if (u == pair_end && g == p.n_kv - 1) item++;
@@ -259,39 +277,70 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
         } else {
             constexpr int half = DH / 2;
             const int kv_dim = p.n_kv * DH, ldp = q_dim + 2 * kv_dim, pos = nkeys - 1;
-            const size_t p1 = (size_t)item * ldp, p2 = (size_t)(p.grouped ? Bc + item : item) * ldp;
-            float rs1, rs2;
-            row_scale2(p.ss, p.ss_tiles, p.ss_ld, item, p.grouped ? Bc + item : item, p.d_norm, p.eps, rs1, rs2);
+            const int twin = p.grouped ? Bc + item : item;
+            const size_t p1 = (size_t)item * ldp, p2 = (size_t)twin * ldp;
+            // One round of loads: the first warp requests the norm shares of the two rows (lanes
+            // 0..15 the primary row, 16..31 its twin) and hands 1/rms to the others through shared
+            // memory; every thread requests the partials, the rotation and the coupling of its
+            // outputs before anyone waits.
+            float myss = 0.f;
+            if (p.ss && warp == 0)
+                for (int t = lane & 15; t < p.ss_tiles; t += 16) myss += __ldcg(p.ss + (size_t)t * p.ss_ld + (lane < 16 ? item : twin));
             for (int idx = tid; idx < (16 - nq_act) * DH / 4; idx += 128)  // unused query rows
                 reinterpret_cast<float4 *>(sc_o + (size_t)nq_act * DH)[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
-            for (int idx = tid; idx < p.G * half; idx += 128) {
-                int j = idx / half, i = idx % half;
+            const int nitems = p.G * half;
+            const bool do_kv = owns_last && tid < half;
+            float *rs_s = reinterpret_cast<float *>(flag + 2);
+            float rs1 = 1.f, rs2 = 1.f, kvs[4] = {0.f, 0.f, 0.f, 0.f};
+            float2 t_kv = make_float2(1.f, 0.f);
+            for (int it0 = 0; it0 * 128 < nitems; it0++) {
+                int idx = it0 * 128 + tid;
+                bool act = idx < nitems;
+                int j = act ? idx / half : 0, i = act ? idx % half : tid % half;
                 int o0 = (g * p.G + j) * DH + i, o1 = o0 + half;
                 float2 t = p.rope[(size_t)pos * half + i];
+                float ca0 = p.grouped ? p.coup_a[o0] : 0.f, ca1 = p.grouped ? p.coup_a[o1] : 0.f;
                 const size_t offs[4] = {p1 + o0, p1 + o1, p2 + o0, p2 + o1};
-                float sm[4];
-                sum_splits_k<4, 8>(p.qkv_P, p.qkv_stride, p.qkv_nsplit, offs, sm);
-                float x0 = rs1 * sm[0], x1 = rs1 * sm[1];
-                float r0 = x0 * t.x - x1 * t.y, r1 = x1 * t.x + x0 * t.y;
-                sc_o[(size_t)j * DH + i] = r0;
-                sc_o[(size_t)j * DH + i + half] = r1;
-                if (p.grouped) {
-                    float y0 = rs2 * sm[2], y1 = rs2 * sm[3];
-                    sc_o[(size_t)(p.G + j) * DH + i] = (y0 * t.x - y1 * t.y) + p.coup_a[o0] * r0;
-                    sc_o[(size_t)(p.G + j) * DH + i + half] = (y1 * t.x + y0 * t.y) + p.coup_a[o1] * r1;
+                float sm[4] = {0.f, 0.f, 0.f, 0.f};
+                if (act) sum_splits_k<4, 8>(p.qkv_P, p.qkv_stride, p.qkv_nsplit, offs, sm);
+                if (it0 == 0) {
+                    if (do_kv) {  // K_1 and V_1 of this step's token for this KV head (tid = rotation pair)
+                        size_t ko = p1 + q_dim + (size_t)g * DH + tid, vo = ko + kv_dim;
+                        const size_t koffs[4] = {ko, ko + half, vo, vo + half};
+                        sum_splits_k<4, 8>(p.qkv_P, p.qkv_stride, p.qkv_nsplit, koffs, kvs);
+                        t_kv = t;  // idx = tid < half in the first round: the same rotation pair
+                    }
+                    if (warp == 0) {
+                        sc_m[lane] = myss;  // sc_m[0..15], sc_l[0..15] are contiguous
+                        __syncwarp();
+                        if ((lane & 15) == 0) {
+                            float a = 0.f;
+                            for (int k = 0; k < 16; k++) a += sc_m[lane + k];
+                            rs_s[lane >> 4] = p.ss ? 1.f / sqrtf(a / (float)p.d_norm + p.eps) : 1.f;
+                        }
+                    }
+                    consumer_sync();
+                    rs1 = rs_s[0];
+                    rs2 = rs_s[1];
+                }
+                if (act) {
+                    float x0 = rs1 * sm[0], x1 = rs1 * sm[1];
+                    float r0 = x0 * t.x - x1 * t.y, r1 = x1 * t.x + x0 * t.y;
+                    sc_o[(size_t)j * DH + i] = r0;
+                    sc_o[(size_t)j * DH + i + half] = r1;
+                    if (p.grouped) {
+                        float y0 = rs2 * sm[2], y1 = rs2 * sm[3];
+                        sc_o[(size_t)(p.G + j) * DH + i] = (y0 * t.x - y1 * t.y) + ca0 * r0;
+                        sc_o[(size_t)(p.G + j) * DH + i + half] = (y1 * t.x + y0 * t.y) + ca1 * r1;
+                    }
                 }
             }
-            if (owns_last && tid < half) {
-                // K_1 = RoPE(N_1 W_K), V_1 = N_1 W_V of this step's token, for this KV head
+            if (do_kv) {
+                // K_1 = RoPE(N_1 W_K), V_1 = N_1 W_V: to the staging row for the patch and to the pool
                 int i = tid;
-                float2 t = p.rope[(size_t)pos * half + i];
-                size_t ko = p1 + q_dim + (size_t)g * DH + i, vo = ko + kv_dim;
-                const size_t offs[4] = {ko, ko + half, vo, vo + half};
-                float sm[4];
-                sum_splits_k<4, 8>(p.qkv_P, p.qkv_stride, p.qkv_nsplit, offs, sm);
-                float x0 = rs1 * sm[0], x1 = rs1 * sm[1];
-                __nv_bfloat16 k0 = __float2bfloat16_rn(x0 * t.x - x1 * t.y), k1 = __float2bfloat16_rn(x1 * t.x + x0 * t.y);
-                __nv_bfloat16 v0 = __float2bfloat16_rn(rs1 * sm[2]), v1 = __float2bfloat16_rn(rs1 * sm[3]);
+                float x0 = rs1 * kvs[0], x1 = rs1 * kvs[1];
+                __nv_bfloat16 k0 = __float2bfloat16_rn(x0 * t_kv.x - x1 * t_kv.y), k1 = __float2bfloat16_rn(x1 * t_kv.x + x0 * t_kv.y);
+                __nv_bfloat16 v0 = __float2bfloat16_rn(rs1 * kvs[2]), v1 = __float2bfloat16_rn(rs1 * kvs[3]);
                 kv_new[i] = k0;
                 kv_new[i + half] = k1;
                 kv_new[DH + i] = v0;
@@ -309,6 +358,10 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
             }
         }
         consumer_sync();
+        if (u == u0) {
+            asm volatile("bar.arrive 2, 160;" ::: "memory");  // the producer may stream on
+            DBT_TL_MARK(0);
+        }
         int pair = item * p.n_kv + g;
         int first_cta = pair_start / quota, nseg = (pair_end - 1) / quota - first_cta + 1;
         float *out = p.part + (size_t)(blockIdx.x + pair) * 16 * (DH + 2);
@@ -714,6 +767,7 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
                 }
             }
         }
+        if (u == u0) DBT_TL_MARK(1);
         // ---- merging a pair's segments.  Up to kAttGroup segments: the last one to arrive merges them
         // all, in segment order, and writes the output.  More: the segments form groups of kAttGroup;
         // the last arrival of a group merges it in place into the group's first slot, and the last
@@ -823,10 +877,11 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
                 }
             }
         }
+        if (u == u0) DBT_TL_MARK(2);
         u += t1 - t0;
         if (u == pair_end && g == p.n_kv - 1) item++;
     }
-    DBT_TL_END("attention");
+    DBT_TL_END_IF(blockIdx.x == 0 || blockIdx.x == 99 || blockIdx.x == 200 || blockIdx.x == 281, blockIdx.x == 0 ? "attentio" : blockIdx.x == 99 ? "att99" : blockIdx.x == 200 ? "att200" : "att281");
 }
 
 // The K/V pool as a 4-D bf16 tensor (64 columns, 64-column piece of a row, row, K|V plane of a

@@ -26,16 +26,40 @@ __device__ __forceinline__ unsigned long long gtime() {
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
+// Timeline instrumentation (compile with -DDBT_TIMELINE): block 0 of every instrumented kernel
+// appends (name tag, entry, after the dependency wait, end, four optional marks) in nanoseconds of %globaltimer to a
+// device array that dbt_debug_timeline copies out.  Stores only: a printf would itself delay the
+// end of the kernel and with it the next one's start.
 #ifdef DBT_TIMELINE
-#define DBT_TL_DECL unsigned long long tl0_ = gtime(), tl1_ = 0
+constexpr int kTlMax = 16384;
+__device__ unsigned long long g_tl[kTlMax * 8];
+__device__ unsigned int g_tl_n;
+__device__ __forceinline__ unsigned long long tl_tag(const char *s) {
+    unsigned long long t = 0;
+    for (int i = 0; i < 8 && s[i]; i++) t |= (unsigned long long)(unsigned char)s[i] << (8 * i);
+    return t;
+}
+#define DBT_TL_DECL unsigned long long tl0_ = gtime(), tl1_ = 0, tlx_[4] = {0, 0, 0, 0}
 #define DBT_TL_WAITED tl1_ = gtime()
-#define DBT_TL_END(name)                                                                                   \
-    if (threadIdx.x == 0 && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0)                         \
-    printf("TL %s entry %llu waited %llu end %llu\n", name, tl0_, tl1_, gtime())
+#define DBT_TL_MARK(k) tlx_[k] = gtime()
+#define DBT_TL_END(name) DBT_TL_END_IF(blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0, name)
+#define DBT_TL_END_IF(cond, name)                                                          \
+    if (threadIdx.x == 0 && (cond)) {                                                      \
+        unsigned int i_ = atomicAdd(&g_tl_n, 1u);                                          \
+        if (i_ < (unsigned)kTlMax) {                                                       \
+            g_tl[8 * i_] = tl_tag(name);                                                   \
+            g_tl[8 * i_ + 1] = tl0_;                                                       \
+            g_tl[8 * i_ + 2] = tl1_;                                                       \
+            g_tl[8 * i_ + 3] = gtime();                                                    \
+            for (int k_ = 0; k_ < 4; k_++) g_tl[8 * i_ + 4 + k_] = tlx_[k_];               \
+        }                                                                                  \
+    }
 #else
 #define DBT_TL_DECL
 #define DBT_TL_WAITED
+#define DBT_TL_MARK(k)
 #define DBT_TL_END(name)
+#define DBT_TL_END_IF(cond, name)
 #endif
 __device__ __forceinline__ void pdl_enter() {
     pdl_launch_dependents();

@@ -109,31 +109,48 @@ __global__ void __launch_bounds__(256) resid_wide_kernel(float *S, const float *
     DBT_TL_DECL;
     pdl_enter();
     DBT_TL_WAITED;
-    __shared__ float scratch[32];
+    __shared__ float scratch[64];
     int b = blockIdx.x, i = blockIdx.y * blockDim.x + threadIdx.x;
     float q1 = 0.f, q2 = 0.f;
     if (i < d) {
-        float gn = g_next ? g_next[i] : 1.f;
+        // every load of this thread goes out before the first use: S of both rows, the gain, the
+        // coupling, and all splits of both rows' partials (up to 16 splits in one round)
         size_t o1 = (size_t)b * d + i, o2 = (size_t)(Bc + b) * d + i;
-        float m1 = sum_splits(P, split_stride, nsplit, o1);
-        float s1 = S[o1] + m1;
+        float s1 = __ldcg(S + o1), s2 = grouped ? __ldcg(S + o2) : 0.f;
+        float gn = g_next ? g_next[i] : 1.f, cc = mode == 2 ? coup_c[i] : 0.f;
+        const size_t offs[2] = {o1, grouped ? o2 : o1};
+        float mm[2];
+        sum_splits_k<2, 16>(P, split_stride, nsplit, offs, mm);
+        s1 += mm[0];
         S[o1] = s1;
         store_split(Xb, o1, lo_off, gn * s1);
         q1 = s1 * s1;
         if (grouped) {
-            float m2 = sum_splits(P, split_stride, nsplit, o2);
-            if (mode == 2) m2 += coup_c[i] * m1;
-            float s2 = S[o2] + m2;
+            float m2 = mm[1];
+            if (mode == 2) m2 += cc * mm[0];
+            s2 += m2;
             S[o2] = s2;
             store_split(Xb, o2, lo_off, gn * s2);
             q2 = s2 * s2;
         }
     }
-    q1 = block_sum(q1, scratch);
-    if (grouped) q2 = block_sum(q2, scratch);
+    // both rows' shares in one pass over the block
+    q1 = warp_sum(q1);
+    q2 = warp_sum(q2);
+    int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    if (lane == 0) {
+        scratch[warp] = q1;
+        scratch[32 + warp] = q2;
+    }
+    __syncthreads();
     if (threadIdx.x == 0) {
-        ss_out[(size_t)blockIdx.y * ss_ld + b] = q1;
-        if (grouped) ss_out[(size_t)blockIdx.y * ss_ld + Bc + b] = q2;
+        float a1 = 0.f, a2 = 0.f;
+        for (int w2 = 0; w2 < nw; w2++) {
+            a1 += scratch[w2];
+            a2 += scratch[32 + w2];
+        }
+        ss_out[(size_t)blockIdx.y * ss_ld + b] = a1;
+        if (grouped) ss_out[(size_t)blockIdx.y * ss_ld + Bc + b] = a2;
     }
     DBT_TL_END("resid_wide");
 }
@@ -274,21 +291,41 @@ __global__ void __launch_bounds__(256) swiglu_couple_kernel(const float *P, int 
     DBT_TL_DECL;
     pdl_enter();
     DBT_TL_WAITED;
+    __shared__ float sh[34];
     int b = blockIdx.x, f = blockIdx.y * blockDim.x + threadIdx.x;
-    if (f >= F) return;
-    size_t p1 = (size_t)b * 2 * F + f;
-    float rs1, rs2;
-    row_scale2(ss, ss_tiles, ss_ld, b, grouped ? Bc + b : b, d_norm, eps, rs1, rs2);
-    size_t p2 = grouped ? (size_t)(Bc + b) * 2 * F + f : p1;
+    const bool act = f < F;
+    const int rb = grouped ? Bc + b : b, lane = threadIdx.x & 31;
+    // The norm shares of the block's two rows are fetched once, by the first warp (lanes 0..15 the
+    // primary row, 16..31 its twin), requested before the partials so that they travel together,
+    // and handed to the block through shared memory: a few hundred blocks would otherwise all
+    // hammer the same few lines.
+    float myss = 0.f;
+    if (ss && threadIdx.x < 32)
+        for (int t = lane & 15; t < ss_tiles; t += 16) myss += __ldcg(ss + (size_t)t * ss_ld + (lane < 16 ? b : rb));
+    size_t p1 = (size_t)b * 2 * F + (act ? f : 0);
+    size_t p2 = grouped ? (size_t)(Bc + b) * 2 * F + (act ? f : 0) : p1;
     const size_t offs[4] = {p1, p1 + F, p2, p2 + F};
-    float sm[4];
-    sum_splits_k<4>(P, split_stride, nsplit, offs, sm);
-    float h1 = silu(rs1 * sm[0]) * (rs1 * sm[1]);
-    store_split(Hb, (size_t)b * F + f, lo_off, h1);
-    if (grouped) {
-        float h2 = silu(rs2 * sm[2]) * (rs2 * sm[3]);
-        if (coup_b) h2 += coup_b[f] * h1;
-        store_split(Hb, (size_t)(Bc + b) * F + f, lo_off, h2);
+    float sm[4] = {0.f, 0.f, 0.f, 0.f};
+    if (act) sum_splits_k<4, 4>(P, split_stride, nsplit, offs, sm);
+    if (threadIdx.x < 32) {
+        sh[lane] = myss;
+        __syncwarp();
+        if ((lane & 15) == 0) {
+            float a = 0.f;
+            for (int j = 0; j < 16; j++) a += sh[lane + j];
+            sh[32 + (lane >> 4)] = ss ? 1.f / sqrtf(a / (float)d_norm + eps) : 1.f;
+        }
+    }
+    __syncthreads();
+    if (act) {
+        float rs1 = sh[32], rs2 = sh[33];
+        float h1 = silu(rs1 * sm[0]) * (rs1 * sm[1]);
+        store_split(Hb, (size_t)b * F + f, lo_off, h1);
+        if (grouped) {
+            float h2 = silu(rs2 * sm[2]) * (rs2 * sm[3]);
+            if (coup_b) h2 += coup_b[f] * h1;
+            store_split(Hb, (size_t)(Bc + b) * F + f, lo_off, h2);
+        }
     }
     DBT_TL_END("swiglu");
 }

@@ -33,6 +33,7 @@ struct TcSeg {
 };
 
 struct TcParams {
+    int evict_first;  // weight tiles carry the evict-first L2 hint
     // up to three byte ranges (the next GEMM's weights) that this launch asks the L2 to fetch while it
     // and the small kernels after it run: HBM is otherwise idle between the GEMMs of a decode step
     const char *pf_ptr[3];
@@ -102,6 +103,13 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map
         "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];" ::"r"(dst),
         "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
         : "memory");
+}
+// L2 eviction policy for data that is read once per step (weight tiles, K/V pages): evict first, so
+// that the stream does not push the small reused data (activations, partials, gains, tables) out.
+__device__ __forceinline__ uint64_t l2_evict_first_policy() {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
 }
 __device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1,
                                                  uint64_t hint) {
@@ -262,18 +270,26 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
                     tma_load_2d(tiles + s * Cfg::kStageBytes + kTcABytes + part * Cfg::kBBytes + j * 2048, &tmX,
                                 full_bar(s), kt * kTcK, part * p.lo_row0 + x_row0 + j * 16);
         };
+        const uint64_t pol = l2_evict_first_policy();
+        auto load_w = [&](int s, int kt) {
+            if (p.evict_first)
+                tma_load_2d_hint(tiles + s * Cfg::kStageBytes, tmW, full_bar(s), kt * kTcK, w_row0 + f0, pol);
+            else
+                tma_load_2d(tiles + s * Cfg::kStageBytes, tmW, full_bar(s), kt * kTcK, w_row0 + f0);
+        };
         for (int i = 0; i < npre; i++) {
             mbar_expect_tx(full_bar(i), tx);
-            tma_load_2d(tiles + i * Cfg::kStageBytes, tmW, full_bar(i), (kt0 + i) * kTcK, w_row0 + f0);
+            load_w(i, kt0 + i);
         }
         pdl_wait();
+        DBT_TL_MARK(0);
         for (int i = 0; i < npre; i++) load_x(i, kt0 + i);
         for (int i = npre; i < nkt && ok; i++) {
             int s = i % STAGES;
             ok = mbar_wait(empty_bar(s), ((i / STAGES) - 1) & 1);
             if (!ok) break;
             mbar_expect_tx(full_bar(s), tx);
-            tma_load_2d(tiles + s * Cfg::kStageBytes, tmW, full_bar(s), (kt0 + i) * kTcK, w_row0 + f0);
+            load_w(s, kt0 + i);
             load_x(s, kt0 + i);
         }
     } else if (warp == 1 && lane == 0) {
@@ -295,6 +311,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
         }
         if (ok) umma_commit(accum_bar);
     }
+    if (warp == 0 && lane == 0) DBT_TL_MARK(1);
     if (!ok) report(p.status, kStatusWaitExpired, 100 + warp);
     __syncwarp();
 
@@ -302,6 +319,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
     pdl_wait();
     DBT_TL_WAITED;
     bool got = mbar_wait(accum_bar, 0);
+    DBT_TL_MARK(2);
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (!got && lane == 0) report(p.status, kStatusWaitExpired, 200 + warp);
     got = __syncthreads_and(got);  // the ring is idle from here on: its memory serves as scratch
@@ -354,6 +372,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
             }
         }
     }
+    DBT_TL_MARK(3);
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     if (warp == 1)
