@@ -93,6 +93,7 @@ struct dbt_model {
     struct ActBase { const void *base; };
     std::map<const CUtensorMap *, ActBase> act_base;
     std::map<std::tuple<const CUtensorMap *, int, int>, CUtensorMap> act3d;
+    bool stack_planes;  // GEMM: one MMA per k16 step over both activation planes (DBT_STACK=0 issues two)
     bool evict_first;  // weight tiles and K/V pages carry the evict-first L2 hint (DBT_EVICT_FIRST=0 turns it off)
     bool fuse_qkv;     // decode steps: the attention kernel does the Q|K|V epilogue itself (DBT_FUSE_QKV=0 keeps the kernel)
     bool l2_prefetch;  // GEMM launches ask the L2 for the next GEMM's weights (opt-in, DBT_L2_PREFETCH=1)
@@ -566,6 +567,7 @@ dbt_status launch_gemm_tc(dbt_model *m, const TcCall &c, const TcParams &p, cons
         if (hit != m->act3d.end()) {
             x = &hit->second;
             pp.x3d = 1;
+            pp.stacked = m->stack_planes && N_TILE <= 128 ? 1 : 0;
         }
     }
     LAUNCH(m, c.tag, bytes, gemm_tc_kernel<N_TILE>, grid, 128, TcCfg<N_TILE>::kSmemBytes, *c.W[0], *w1, *w2, *x, pp, e);
@@ -1634,6 +1636,8 @@ dbt_status dbt_create(const dbt_config *cfg, const dbt_weights *w, void *kv_pool
     {
         // Opt-in (DBT_L2_PREFETCH=1): measured no faster (1.49 vs 1.45 ms per step at batch 16 on the
         // 1B model); the GEMMs of a decode step wait on dependency latency, not on HBM bandwidth.
+        const char *sp = getenv("DBT_STACK");
+        m->stack_planes = !(sp && strcmp(sp, "0") == 0);
         const char *ef = getenv("DBT_EVICT_FIRST");
         m->evict_first = !(ef && strcmp(ef, "0") == 0);
         const char *fq = getenv("DBT_FUSE_QKV");

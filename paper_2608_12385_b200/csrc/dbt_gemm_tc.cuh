@@ -39,6 +39,7 @@ struct TcParams {
     const char *pf_ptr[3];
     unsigned long long pf_bytes[3];
     int x3d;  // tmX is the 3-D {64, N_TILE, 2} view of a two-plane input: one box per stage
+    int stacked;  // with x3d: one MMA per k16 step over both planes (N = 2 * N_TILE), halves added in the epilogue
     TcSeg seg[3];
     int nseg;
     int K;
@@ -177,7 +178,9 @@ struct TcCfg {
 #else
     static constexpr int kStages = N_TILE <= 16 ? 5 : N_TILE <= 32 ? 4 : N_TILE <= 64 ? 3 : N_TILE <= 128 ? 4 : 2;
 #endif
-    static constexpr int kTmemCols = N_TILE < 32 ? 32 : N_TILE;
+    // room for the two planes' accumulators side by side (see `stacked` in the kernel)
+    static constexpr int kStackable = N_TILE <= 128;
+    static constexpr int kTmemCols = kStackable ? (2 * N_TILE < 32 ? 32 : 2 * N_TILE) : N_TILE;
     static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
 
@@ -295,17 +298,29 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
     } else if (warp == 1 && lane == 0) {
         // ---- MMA issuer
         constexpr uint32_t idesc = umma_idesc(N_TILE);
+        // Stacked form: the 3-D box leaves the hi rows and the lo rows of a k-tile next to each other,
+        // so they can serve as ONE B operand of 2 * N_TILE rows: hi and lo products land in separate
+        // accumulator columns (added in the epilogue) and the narrow MMAs, whose cost is mostly
+        // fixed, are issued once per k16 step instead of twice.
+        constexpr uint32_t idesc2 = umma_idesc(Cfg::kStackable ? 2 * N_TILE : N_TILE);
+        const bool stacked = Cfg::kStackable && p.stacked;
         for (int i = 0; i < nkt && ok; i++) {
             int s = i % STAGES;
             ok = mbar_wait(full_bar(s), (i / STAGES) & 1);
             if (!ok) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             uint64_t adesc = umma_smem_desc(tiles + s * Cfg::kStageBytes);
-            for (int part = 0; part < p.parts; part++) {
-                uint64_t bdesc = umma_smem_desc(tiles + s * Cfg::kStageBytes + kTcABytes + part * Cfg::kBBytes);
+            if (stacked) {
+                uint64_t bdesc = umma_smem_desc(tiles + s * Cfg::kStageBytes + kTcABytes);
 #pragma unroll
-                for (int k = 0; k < kTcK / 16; k++)  // advance 16 elements = 32 bytes inside the swizzle row
-                    umma_f16(tmem_base, adesc + 2 * k, bdesc + 2 * k, idesc, (i | k | part) != 0);
+                for (int k = 0; k < kTcK / 16; k++) umma_f16(tmem_base, adesc + 2 * k, bdesc + 2 * k, idesc2, (i | k) != 0);
+            } else {
+                for (int part = 0; part < p.parts; part++) {
+                    uint64_t bdesc = umma_smem_desc(tiles + s * Cfg::kStageBytes + kTcABytes + part * Cfg::kBBytes);
+#pragma unroll
+                    for (int k = 0; k < kTcK / 16; k++)  // advance 16 elements = 32 bytes inside the swizzle row
+                        umma_f16(tmem_base, adesc + 2 * k, bdesc + 2 * k, idesc, (i | k | part) != 0);
+                }
             }
             umma_commit(empty_bar(s));
         }
@@ -325,13 +340,23 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
     got = __syncthreads_and(got);  // the ring is idle from here on: its memory serves as scratch
     float *scratch = reinterpret_cast<float *>(gen_tiles);
     int rows = grp_n >= 0 ? min(grp_n, N_TILE) : min(seg.rows, p.R);
+    const bool stacked_acc = Cfg::kStackable && p.stacked;
+    auto ld_acc = [&](int c0, float (&v)[16]) {  // 16 accumulator columns of this thread's feature
+        tmem_ld16(tmem_base + ((uint32_t)(warp * 32) << 16) + c0, v);
+        if (stacked_acc) {
+            float t[16];
+            tmem_ld16(tmem_base + ((uint32_t)(warp * 32) << 16) + N_TILE + c0, t);
+#pragma unroll
+            for (int i = 0; i < 16; i++) v[i] += t[i];
+        }
+    };
     if (got && e.mode == FE_LMHEAD) {
         epi_row_scales(e, p.R, scratch);
         int f = f0 + warp * 32 + lane;
 #pragma unroll 1
         for (int c0 = 0; c0 < N_TILE && c0 < rows; c0 += 16) {
             float v[16];
-            tmem_ld16(tmem_base + ((uint32_t)(warp * 32) << 16) + c0, v);
+            ld_acc(c0, v);
             if (f < seg.n_out) {
 #pragma unroll
                 for (int i = 0; i < 16; i++)
@@ -344,7 +369,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
 #pragma unroll 1
         for (int c0 = 0; c0 < N_TILE && c0 < rows; c0 += 16) {
             float v[16];
-            tmem_ld16(tmem_base + ((uint32_t)(warp * 32) << 16) + c0, v);
+            ld_acc(c0, v);
             if (f < seg.n_out) {
 #pragma unroll
                 for (int i = 0; i < 16; i++)
