@@ -6,21 +6,23 @@
 // share reads of the primary keys and values").  Keys 0..pos inclusive: the K_1,V_1 appended
 // this step is already in its page.
 //
-// Work decomposition.  All (row, KV head) pairs are laid end to end in units of one 64-token
-// tile; the grid is a fixed number of CTAs (two per SM) and CTA c takes the contiguous unit
-// range [c*q, (c+1)*q), q = max(ceil(units / CTAs), 4, ceil(longest pair / 31)).  A range may
-// end inside a pair or cover several short pairs: each (CTA, pair) intersection is one
-// segment, whose un-normalised partial (m, l, O) goes to slot c + pair (unique, and consecutive
-// for one pair).  The last segment of a pair to arrive folds all of that pair's segments in
-// segment order, so the result does not depend on arrival order.  Every SM therefore streams
-// the same number of K/V bytes (to within one tile) whatever the batch and context mix.
+// Work decomposition.  A (row, KV head) pair of u 64-token stages is cut into n = round(u / q)
+// equal segments, q = the per-CTA share of all stages (at least 4); the segments of all pairs,
+// in (row, KV head, segment) order, are dealt to a fixed grid of CTAs (two per SM) round robin.
+// A CTA never straddles two pairs (the per-segment costs -- building the queries, folding the
+// warps, the merge -- are then paid once per CTA for equal-length batches), and the split depends
+// on the lengths only.  A segment's un-normalised partial (m, l, O) goes to the slot of its
+// index, consecutive for one pair; the last segment of a pair to arrive merges them in segment
+// order (in two levels above 8 segments), so the result does not depend on arrival order.
 //
-// Data movement: a producer warp walks the page table and brings 16-token pages in with
-// tiled TMA copies (128B swizzle) into a shared-memory ring, 64 tokens per stage, ~190 KB in
-// flight per SM.  Math: four consumer warps, one page each per stage; S = Q K^T and O += P V
-// with mma.sync m16n8k16 (bf16 in, fp32 accumulate), operands read with ldmatrix through the
-// swizzle; each warp keeps its own running (max, sum, O) and the four are folded in a fixed
-// order at the end of a segment.  All waits are bounded.
+// Data movement: a producer warp walks the page table and brings 16-token pages in with one 4-D
+// TMA box per page (K and V, 128B swizzle) into a shared-memory ring, 64 tokens per stage, ~190 KB
+// in flight per SM, with the evict-first L2 hint.  Math: four consumer warps, one page each per
+// stage, mma.sync m16n8k16 (bf16 in, fp32 accumulate), operands read with ldmatrix through the
+// swizzle; with at most 8 query rows per KV head the products are taken transposed (keys on the
+// M side).  Each warp keeps its own running (max, sum, O) and the four are folded in a fixed
+// order at the end of a segment.  In decode steps the kernel also builds its queries and the
+// new K,V row from the Q|K|V GEMM's split-K partials.  All waits are bounded.
 #pragma once
 
 #include "dbt_fused.cuh"
@@ -74,7 +76,7 @@ struct AttCfg {
     // scratch: one [16][DH + 8] fp32 slot (Q tile / warp fold; the padding keeps the fold's
     // fragment-shaped accesses off a single bank), m, l, flag, row tables
     static constexpr int kFoldStride = DH + 8;
-    static constexpr int kScratchBytes = (16 * kFoldStride + 2 * 16 + 8 + 2 * kAttMaxItems + 8) * 4 + 2 * DH * 2 + 32;
+    static constexpr int kScratchBytes = (16 * kFoldStride + 2 * 16 + 8 + 3 * kAttMaxItems + 12) * 4 + 2 * DH * 2 + 32;
     static constexpr int kSmemBytes = kStages * kStageBytes + 1024 + 128 + kScratchBytes;
 };
 
@@ -139,8 +141,9 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
     int *flag = reinterpret_cast<int *>(sc_l + 16);                                 // [0] last?, [1] longest pair
     int *cum = flag + 8;                 // [items + 1] prefix of tiles per row
     int *nk_s = cum + kAttMaxItems + 1;  // [items] visible keys per row
+    int *segcum = nk_s + kAttMaxItems;   // [items + 1] prefix of segments per row (per KV head)
     __nv_bfloat16 *kv_new =  // [2][DH] this step's K, V row (16-byte aligned)
-        reinterpret_cast<__nv_bfloat16 *>((reinterpret_cast<uintptr_t>(nk_s + kAttMaxItems) + 15) & ~(uintptr_t)15);
+        reinterpret_cast<__nv_bfloat16 *>((reinterpret_cast<uintptr_t>(segcum + kAttMaxItems + 1) + 15) & ~(uintptr_t)15);
 
     DBT_TL_DECL;
     int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -179,14 +182,49 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
             running += __shfl_sync(0xffffffffu, incl, 31);
         }
         if (lane == 0) flag[1] = longest;
+        __syncwarp();
+        // Work split: a (row, KV head) pair of u stages is cut into n = round(u / q) equal segments,
+        // q = the per-CTA share of all stages; CTA c takes segments c, c + gridDim.x, ...  A CTA thus
+        // never straddles two pairs, equal-length batches give every CTA one segment, and the split
+        // depends on the lengths only.
+        const int C0 = gridDim.x, U0 = cum[items] * p.n_kv, q0 = max((U0 + C0 - 1) / C0, kAttMinUnits);
+        int run2 = 0;
+        if (lane == 0) segcum[0] = 0;
+        for (int base = 0; base < items; base += 32) {
+            int i = base + lane, n = 0;
+            if (i < items) {
+                int u = cum[i + 1] - cum[i];
+                n = min(max((2 * u + q0) / (2 * q0), 1), min(max(u, 1), kAttMaxSeg));
+            }
+            int incl = n;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                int t = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += t;
+            }
+            if (i < items) segcum[i + 1] = run2 + incl;
+            run2 += __shfl_sync(0xffffffffu, incl, 31);
+        }
     }
     __syncthreads();
-    const int U = cum[items] * p.n_kv, C = gridDim.x;
-    const int quota = max(max((U + C - 1) / C, kAttMinUnits), (flag[1] + kAttMaxSeg - 2) / (kAttMaxSeg - 1));
-    const int u0 = blockIdx.x * quota, u1 = min(U, u0 + quota);
-    if (u0 >= U) return;
-    int item = 0;
-    while (cum[item + 1] * p.n_kv <= u0) item++;
+    const int C = gridDim.x, Sg = segcum[items] * p.n_kv;  // all segments, ordered (row, KV head, segment)
+    if ((int)blockIdx.x >= Sg) return;
+    // segment sidx -> its row, KV head, stage range and the pair's segment count
+    auto locate = [&](int sidx, int &item, int &g, int &seg, int &n, int &ui, int &t0, int &t1) {
+        int lo = 0, hi = items - 1;
+        while (lo < hi) {  // largest row whose first segment is <= sidx
+            int mid = (lo + hi + 1) >> 1;
+            if (segcum[mid] * p.n_kv <= sidx) lo = mid; else hi = mid - 1;
+        }
+        item = lo;
+        n = segcum[item + 1] - segcum[item];
+        int rel = sidx - segcum[item] * p.n_kv;
+        g = rel / n;
+        seg = rel % n;
+        ui = cum[item + 1] - cum[item];
+        t0 = (int)(((long long)seg * ui) / n);
+        t1 = (int)(((long long)(seg + 1) * ui) / n);
+    };
 
     if (warp == kAttWarps) {
         // ---- producer: walks the same segments as the consumers.  Lane 0 waits for the stage and
@@ -196,10 +234,9 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
         const uint64_t pol = l2_evict_first_policy();
         bool ok = true;
         int it = 0;
-        for (int u = u0; u < u1 && ok;) {
-            int ui = cum[item + 1] - cum[item], base = cum[item] * p.n_kv;
-            int g = (u - base) / ui, t0 = (u - base) % ui;
-            int pair_end = base + (g + 1) * ui, t1 = t0 + min(u1, pair_end) - u;
+        for (int sidx = blockIdx.x; sidx < Sg && ok; sidx += C) {
+            int item, g, seg, n, ui, t0, t1;
+            locate(sidx, item, g, seg, n, ui, t0, t1);
             int seq = p.rm.seq(item), total_pages = (nk_s[item] + 15) >> 4;
             for (int t = t0; t < t1; t++, it++) {
                 int s = it % STAGES;
@@ -229,8 +266,6 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
                 // microseconds, and nothing can be consumed before they return anyway.
                 if (it == 0) asm volatile("bar.sync 2, 160;" ::: "memory");
             }
-            u += t1 - t0;
-            if (u == pair_end && g == p.n_kv - 1) item++;
         }
         if (!ok && lane == 0) report(p.status, kStatusWaitExpired, 300);
         return;
@@ -253,16 +288,15 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
         }
         __syncwarp();
     };
-    for (int u = u0; u < u1;) {
-        int ui = cum[item + 1] - cum[item], base = cum[item] * p.n_kv;
-        int g = (u - base) / ui, t0 = (u - base) % ui;
-        int pair_start = base + g * ui, pair_end = pair_start + ui, t1 = t0 + min(u1, pair_end) - u;
+    for (int sidx = blockIdx.x; sidx < Sg; sidx += C) {
+        int item, g, seg, nseg, ui, t0, t1;
+        locate(sidx, item, g, seg, nseg, ui, t0, t1);
         int nkeys = nk_s[item];
 
         // Query tile (16 rows x DH, fp32) into shared memory, then mma A fragments (bf16),
         // pre-scaled by log2(e)/sqrt(d_h).  Rows: G primary heads, then G coupled branch heads.
         consumer_sync();  // the previous segment is done with the scratch
-        const bool owns_last = p.qkv_P != nullptr && u + (t1 - t0) == pair_end;  // this segment ends the pair
+        const bool owns_last = p.qkv_P != nullptr && seg == nseg - 1;  // this segment ends the pair
         if (p.qkv_P == nullptr) {
             for (int idx = tid; idx < 16 * DH / 4; idx += 128) {
                 int q = idx / (DH / 4), c4 = idx % (DH / 4);
@@ -358,13 +392,13 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
             }
         }
         consumer_sync();
-        if (u == u0) {
+        if (sidx == (int)blockIdx.x) {
             asm volatile("bar.arrive 2, 160;" ::: "memory");  // the producer may stream on
             DBT_TL_MARK(0);
         }
         int pair = item * p.n_kv + g;
-        int first_cta = pair_start / quota, nseg = (pair_end - 1) / quota - first_cta + 1;
-        float *out = p.part + (size_t)(blockIdx.x + pair) * 16 * (DH + 2);
+        int first_slot = sidx - seg;  // the pair's segments occupy consecutive partial slots
+        float *out = p.part + (size_t)sidx * 16 * (DH + 2);
         if constexpr (!NARROW) {
             uint32_t qa[KS][4];
             {
@@ -767,7 +801,7 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
                 }
             }
         }
-        if (u == u0) DBT_TL_MARK(1);
+        if (sidx == (int)blockIdx.x) DBT_TL_MARK(1);
         // ---- merging a pair's segments.  Up to kAttGroup segments: the last one to arrive merges them
         // all, in segment order, and writes the output.  More: the segments form groups of kAttGroup;
         // the last arrival of a group merges it in place into the group's first slot, and the last
@@ -865,11 +899,11 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
             return flag[0] != 0;
         };
         if (nseg > 1) {
-            float *slot0 = p.part + (size_t)(first_cta + pair) * 16 * (DH + 2);
+            float *slot0 = p.part + (size_t)first_slot * 16 * (DH + 2);
             if (nseg <= kAttGroup) {
                 if (arrive(p.tickets + pair, nseg)) merge(slot0, 1, nseg, true);
             } else {
-                int gi = ((int)blockIdx.x - first_cta) / kAttGroup, ngroups = (nseg + kAttGroup - 1) / kAttGroup;
+                int gi = seg / kAttGroup, ngroups = (nseg + kAttGroup - 1) / kAttGroup;
                 int gs = min(kAttGroup, nseg - gi * kAttGroup);
                 if (arrive(p.tickets2 + (size_t)pair * kAttMaxGroups + gi, gs)) {
                     merge(slot0 + (size_t)gi * kAttGroup * 16 * (DH + 2), 1, gs, false);
@@ -877,9 +911,7 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
                 }
             }
         }
-        if (u == u0) DBT_TL_MARK(2);
-        u += t1 - t0;
-        if (u == pair_end && g == p.n_kv - 1) item++;
+        if (sidx == (int)blockIdx.x) DBT_TL_MARK(2);
     }
     DBT_TL_END_IF(blockIdx.x == 0 || blockIdx.x == 99 || blockIdx.x == 200 || blockIdx.x == 281, blockIdx.x == 0 ? "attentio" : blockIdx.x == 99 ? "att99" : blockIdx.x == 200 ? "att200" : "att281");
 }
