@@ -208,6 +208,7 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
     }
     __syncthreads();
     const int C = gridDim.x, Sg = segcum[items] * p.n_kv;  // all segments, ordered (row, KV head, segment)
+    DBT_TL_MARK(3);
     if ((int)blockIdx.x >= Sg) return;
     // segment sidx -> its row, KV head, stage range and the pair's segment count
     auto locate = [&](int sidx, int &item, int &g, int &seg, int &n, int &ui, int &t0, int &t1) {
