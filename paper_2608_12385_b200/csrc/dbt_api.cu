@@ -174,7 +174,7 @@ size_t carve(const dbt_config &c, char *base, Workspace *ws, int *Rmax_out, int 
     int Fs = moe ? c.n_shared_experts * c.d_expert : 0;
     int F = moe ? (Fs > 0 ? Fs : 8) : c.d_ff;
     int pps = (c.max_seq + c.page_size - 1) / c.page_size;
-    int part_items = Rmax * c.n_kv_heads + 4 * 148;
+    int part_items = Rmax * c.n_kv_heads + 8 * 148;  // attention partial slots: up to three rounds of 2 x 148 segments plus one per pair
     w.S = k.take<float>((size_t)Rmax * d);
     w.X = k.take<float>((size_t)Rmax * d);
     w.Q = k.take<float>((size_t)Rmax * qd);

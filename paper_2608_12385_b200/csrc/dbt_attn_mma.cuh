@@ -6,9 +6,10 @@
 // share reads of the primary keys and values").  Keys 0..pos inclusive: the K_1,V_1 appended
 // this step is already in its page.
 //
-// Work decomposition.  A (row, KV head) pair of u 64-token stages is cut into n = round(u / q)
-// equal segments, q = the per-CTA share of all stages (at least 4); the segments of all pairs,
-// in (row, KV head, segment) order, are dealt to a fixed grid of CTAs (two per SM) round robin.
+// Work decomposition.  A (row, KV head) pair of u 64-token stages is cut into n ~ u / q equal
+// segments (q: a target length chosen so that the segments fill one to three rounds of the
+// grid); the segments of all pairs, in (row, KV head, segment) order, are dealt to a fixed grid
+// of CTAs (two per SM) round robin.
 // A CTA never straddles two pairs (the per-segment costs -- building the queries, folding the
 // warps, the merge -- are then paid once per CTA for equal-length batches), and the split depends
 // on the lengths only.  A segment's un-normalised partial (m, l, O) goes to the slot of its
@@ -183,19 +184,52 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
         }
         if (lane == 0) flag[1] = longest;
         __syncwarp();
-        // Work split: a (row, KV head) pair of u stages is cut into n = round(u / q) equal segments,
-        // q = the per-CTA share of all stages; CTA c takes segments c, c + gridDim.x, ...  A CTA thus
-        // never straddles two pairs, equal-length batches give every CTA one segment, and the split
-        // depends on the lengths only.
-        const int C0 = gridDim.x, U0 = cum[items] * p.n_kv, q0 = max((U0 + C0 - 1) / C0, kAttMinUnits);
+        // Work split: a (row, KV head) pair of u stages is cut into n equal segments and CTA c takes
+        // segments c, c + gridDim.x, ...: a CTA never straddles two pairs, and the split depends on
+        // the lengths only.  n = round or floor of u / q for a target segment length q = all stages /
+        // (k * CTAs), k = 1..3 rounds; of these six candidates the one with the smallest estimated
+        // time (rounds x (longest segment + a fixed per-segment cost of ~6 stages)) is taken, fewer
+        // segments on ties.
+        const int C0 = gridDim.x, U0 = cum[items] * p.n_kv;
+        auto seg_count = [&](int u, int q, int mode) {  // mode 0: round, 1: floor
+            int n = mode == 0 ? (2 * u + q) / (2 * q) : u / q;
+            return min(max(n, 1), min(max(u, 1), kAttMaxSeg));
+        };
+        int best_q = max((U0 + C0 - 1) / C0, kAttMinUnits), best_mode = 0;
+        int best_cost = -1, best_sg = 0;
+        for (int cand = 0; cand < 6; cand++) {
+            const int k = cand / 2 + 1, mode = cand & 1;
+            const int q = max((U0 + k * C0 - 1) / (k * C0), kAttMinUnits);
+            int sg = 0, longest_seg = 0;
+            for (int base = 0; base < items; base += 32) {
+                int i = base + lane;
+                if (i < items) {
+                    int u = cum[i + 1] - cum[i], n = seg_count(u, q, mode);
+                    sg += n;
+                    longest_seg = max(longest_seg, (u + n - 1) / n);
+                }
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                sg += __shfl_xor_sync(0xffffffffu, sg, o);
+                longest_seg = max(longest_seg, __shfl_xor_sync(0xffffffffu, longest_seg, o));
+            }
+            sg *= p.n_kv;
+            int rounds = (sg + C0 - 1) / C0, cost = rounds * (longest_seg + 6);
+            if (best_cost < 0 || cost < best_cost || (cost == best_cost && sg < best_sg)) {
+                best_cost = cost;
+                best_q = q;
+                best_mode = mode;
+                best_sg = sg;
+            }
+            // the plain split fits one round, or every pair is already whole: take it (the common cases)
+            if (cand == 0 && (rounds == 1 || sg == items * p.n_kv)) break;
+        }
         int run2 = 0;
         if (lane == 0) segcum[0] = 0;
         for (int base = 0; base < items; base += 32) {
             int i = base + lane, n = 0;
-            if (i < items) {
-                int u = cum[i + 1] - cum[i];
-                n = min(max((2 * u + q0) / (2 * q0), 1), min(max(u, 1), kAttMaxSeg));
-            }
+            if (i < items) n = seg_count(cum[i + 1] - cum[i], best_q, best_mode);
             int incl = n;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {

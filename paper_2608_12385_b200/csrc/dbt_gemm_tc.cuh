@@ -152,6 +152,15 @@ __device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t adesc, uint64
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
+// The same without waiting for the data: several loads can be in flight before one tmem_ld_wait().
+__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
     uint32_t r[16];
     asm volatile(
@@ -342,13 +351,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
     int rows = grp_n >= 0 ? min(grp_n, N_TILE) : min(seg.rows, p.R);
     const bool stacked_acc = Cfg::kStackable && p.stacked;
     auto ld_acc = [&](int c0, float (&v)[16]) {  // 16 accumulator columns of this thread's feature
-        tmem_ld16(tmem_base + ((uint32_t)(warp * 32) << 16) + c0, v);
-        if (stacked_acc) {
-            float t[16];
-            tmem_ld16(tmem_base + ((uint32_t)(warp * 32) << 16) + N_TILE + c0, t);
+        uint32_t a[16], b[16];
+        tmem_ld16_issue(tmem_base + ((uint32_t)(warp * 32) << 16) + c0, a);
+        if (stacked_acc) tmem_ld16_issue(tmem_base + ((uint32_t)(warp * 32) << 16) + N_TILE + c0, b);
+        tmem_ld_wait();  // both halves travel together
 #pragma unroll
-            for (int i = 0; i < 16; i++) v[i] += t[i];
-        }
+        for (int i = 0; i < 16; i++) v[i] = __uint_as_float(a[i]) + (stacked_acc ? __uint_as_float(b[i]) : 0.f);
     };
     if (got && e.mode == FE_LMHEAD) {
         epi_row_scales(e, p.R, scratch);
