@@ -371,12 +371,12 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
                 float ca0 = p.grouped ? p.coup_a[o0] : 0.f, ca1 = p.grouped ? p.coup_a[o1] : 0.f;
                 const size_t offs[4] = {p1 + o0, p1 + o1, p2 + o0, p2 + o1};
                 float sm[4] = {0.f, 0.f, 0.f, 0.f};
-                if (act) sum_splits_k<4, 8>(p.qkv_P, p.qkv_stride, p.qkv_nsplit, offs, sm);
+                if (act) sum_splits_k<4, 12>(p.qkv_P, p.qkv_stride, p.qkv_nsplit, offs, sm);
                 if (it0 == 0) {
                     if (do_kv) {  // K_1 and V_1 of this step's token for this KV head (tid = rotation pair)
                         size_t ko = p1 + q_dim + (size_t)g * DH + tid, vo = ko + kv_dim;
                         const size_t koffs[4] = {ko, ko + half, vo, vo + half};
-                        sum_splits_k<4, 8>(p.qkv_P, p.qkv_stride, p.qkv_nsplit, koffs, kvs);
+                        sum_splits_k<4, 12>(p.qkv_P, p.qkv_stride, p.qkv_nsplit, koffs, kvs);
                         t_kv = t;  // idx = tid < half in the first round: the same rotation pair
                     }
                     if (warp == 0) {

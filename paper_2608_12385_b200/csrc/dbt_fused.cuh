@@ -180,7 +180,7 @@ __global__ void __launch_bounds__(1024) resid_norm_kernel(float *S, const float 
         float sm[2] = {0.f, 0.f};
         if (mode != 0) {
             const size_t offs[2] = {(size_t)r1 * d + i, (size_t)(grouped ? r2 : r1) * d + i};
-            sum_splits_k<2>(P, split_stride, nsplit, offs, sm);
+            sum_splits_k<2, 8>(P, split_stride, nsplit, offs, sm);  // (1024 threads per block: 64 registers each)
             m1 = sm[0];
             v1 += m1;
             S[(size_t)r1 * d + i] = v1;
@@ -374,11 +374,20 @@ __global__ void __launch_bounds__(256) embed_fused_kernel(const int32_t *tokens,
 // One block, one thread per expert (E <= 1024).
 __global__ void __launch_bounds__(1024) moe_sort_kernel(const int32_t *idx, int R, int kmax, int E, int32_t *cnt,
                                                         int32_t *off, int32_t *pos, int32_t *union_count) {
+    DBT_TL_DECL;
     pdl_enter();
+    DBT_TL_WAITED;
     __shared__ int s_cnt[1024], s_off[1025];
+    __shared__ int s_idx[4096];  // the selections, staged once (larger lists are read from global memory)
+    const int n = R * kmax;
+    const bool staged = n <= 4096;
+    if (staged)
+        for (int i = threadIdx.x; i < n; i += blockDim.x) s_idx[i] = idx[i];
+    __syncthreads();
+    const int32_t *src = staged ? s_idx : idx;
     int e = threadIdx.x, c = 0;
     if (e < E)
-        for (int i = 0; i < R * kmax; i++) c += idx[i] == e;
+        for (int i = 0; i < n; i++) c += src[i] == e;
     s_cnt[e] = e < E ? c : 0;
     __syncthreads();
     if (e == 0) {
@@ -396,17 +405,20 @@ __global__ void __launch_bounds__(1024) moe_sort_kernel(const int32_t *idx, int 
         cnt[e] = c;
         off[e] = s_off[e];
         int k = 0;
-        for (int i = 0; i < R * kmax && k < c; i++)
-            if (idx[i] == e) pos[i] = s_off[e] + k++;
+        for (int i = 0; i < n && k < c; i++)
+            if (src[i] == e) pos[i] = s_off[e] + k++;
     }
     if (e == 0) off[E] = s_off[E];
+    DBT_TL_END("moe_sort");
 }
 
 // Copy each entry's activation row (both bf16 planes) to its sorted position.
 __global__ void __launch_bounds__(256) moe_gather_kernel(const __nv_bfloat16 *Xb, size_t lo_in, const int32_t *idx,
                                                          const int32_t *pos, int kmax, int d, __nv_bfloat16 *Xs,
                                                          size_t lo_out) {
+    DBT_TL_DECL;
     pdl_enter();
+    DBT_TL_WAITED;
     int entry = blockIdx.x;
     if (idx[entry] < 0) return;
     const uint4 *src = reinterpret_cast<const uint4 *>(Xb + (size_t)(entry / kmax) * d);
@@ -415,16 +427,20 @@ __global__ void __launch_bounds__(256) moe_gather_kernel(const __nv_bfloat16 *Xb
         dst[i] = src[i];
         if (lo_out) dst[i + lo_out / 8] = src[i + lo_in / 8];
     }
+    DBT_TL_END("moe_gath");
 }
 
 // H = SiLU(gate) * up on the sorted rows; Pe rows are [Fe gate | Fe up] (one split).
 __global__ void __launch_bounds__(256) moe_swiglu_kernel(const float *Pe, const int32_t *off_total, int Fe,
                                                          __nv_bfloat16 *Hs, size_t lo_off) {
+    DBT_TL_DECL;
     pdl_enter();
+    DBT_TL_WAITED;
     int p = blockIdx.x, f = blockIdx.y * blockDim.x + threadIdx.x;
     if (p >= *off_total || f >= Fe) return;
     float h = silu(Pe[(size_t)p * 2 * Fe + f]) * Pe[(size_t)p * 2 * Fe + Fe + f];
     store_split(Hs, (size_t)p * Fe + f, lo_off, h);
+    DBT_TL_END("moe_swig");
 }
 
 // M_1 = sum_j w_1j Expert_j(m_1) + G(m_1);  M_2 = sum_j w_2j Expert_j(m_2) + G~(m_2) + c*M_1;
@@ -435,26 +451,47 @@ __global__ void __launch_bounds__(256) moe_combine_sorted_kernel(const float *Ys
                                                                  const int32_t *pos, const float *wts, int kmax, int Bc,
                                                                  int grouped, const float *__restrict__ coup_c, int d,
                                                                  float *S) {
+    DBT_TL_DECL;
     pdl_enter();
+    DBT_TL_WAITED;
     int b = blockIdx.x;
+    // the row's selections (weights, sorted positions) once, then all expert rows of a column in
+    // flight together; terms are added in slot order
+    constexpr int KM = 16;
+    const int r2 = Bc + b;
     for (int i = blockIdx.y * blockDim.x + threadIdx.x; i < d; i += gridDim.y * blockDim.x) {
-        float m1 = 0.f;
-        for (int j = 0; j < kmax; j++)
-            if (idx[(size_t)b * kmax + j] >= 0)
-                m1 = fmaf(wts[(size_t)b * kmax + j], Ys[(size_t)pos[(size_t)b * kmax + j] * d + i], m1);
-        if (Psh) m1 += sum_splits(Psh, split_stride, nsplit, (size_t)b * d + i);
+        float m1 = 0.f, m2 = 0.f;
+        for (int j0 = 0; j0 < kmax; j0 += KM) {
+            float y1[KM], w1[KM], y2[KM], w2[KM];
+#pragma unroll
+            for (int j = 0; j < KM; j++) {
+                bool on1 = j0 + j < kmax && idx[(size_t)b * kmax + j0 + j] >= 0;
+                bool on2 = grouped && j0 + j < kmax && idx[(size_t)r2 * kmax + j0 + j] >= 0;
+                w1[j] = on1 ? wts[(size_t)b * kmax + j0 + j] : 0.f;
+                y1[j] = on1 ? __ldcg(Ys + (size_t)pos[(size_t)b * kmax + j0 + j] * d + i) : 0.f;
+                w2[j] = on2 ? wts[(size_t)r2 * kmax + j0 + j] : 0.f;
+                y2[j] = on2 ? __ldcg(Ys + (size_t)pos[(size_t)r2 * kmax + j0 + j] * d + i) : 0.f;
+            }
+#pragma unroll
+            for (int j = 0; j < KM; j++) {
+                if (j0 + j < kmax && w1[j] != 0.f) m1 = fmaf(w1[j], y1[j], m1);
+                if (j0 + j < kmax && w2[j] != 0.f) m2 = fmaf(w2[j], y2[j], m2);
+            }
+        }
+        if (Psh) {
+            const size_t offs[2] = {(size_t)b * d + i, (size_t)(grouped ? r2 : b) * d + i};
+            float sm[2];
+            sum_splits_k<2, 8>(Psh, split_stride, nsplit, offs, sm);
+            m1 += sm[0];
+            m2 += sm[1];
+        }
         S[(size_t)b * d + i] += m1;
         if (grouped) {
-            int r = Bc + b;
-            float m2 = 0.f;
-            for (int j = 0; j < kmax; j++)
-                if (idx[(size_t)r * kmax + j] >= 0)
-                    m2 = fmaf(wts[(size_t)r * kmax + j], Ys[(size_t)pos[(size_t)r * kmax + j] * d + i], m2);
-            if (Psh) m2 += sum_splits(Psh, split_stride, nsplit, (size_t)r * d + i);
             m2 += coup_c[i] * m1;
-            S[(size_t)r * d + i] += m2;
+            S[(size_t)r2 * d + i] += m2;
         }
     }
+    DBT_TL_END("moe_comb");
 }
 
 // Sum split partials into a plain fp32 matrix (used by the operator-level GEMM entry point).

@@ -466,7 +466,9 @@ __global__ void advance_len_kernel(int32_t *seq_len, int B, int n) {
 __global__ void __launch_bounds__(32) route_kernel(const float *logits, int nsplit, size_t split_stride, int E, int Bc,
                                                    int k_p, int k_b, int kmax, int replay, int32_t *idx, float *wts,
                                                    int32_t *last, int last_stride_path) {
+    DBT_TL_DECL;
     pdl_enter();
+    DBT_TL_WAITED;
     extern __shared__ float smem[];
     float *own = smem, *sel = smem + E;  // own-row logits -> probabilities; selection-row logits
     int r = blockIdx.x, lane = threadIdx.x;
@@ -476,9 +478,19 @@ __global__ void __launch_bounds__(32) route_kernel(const float *logits, int nspl
     float mx = -INFINITY;
     for (int e = lane; e < E; e += 32) {
         float a = 0.f, b2 = 0.f;
-        for (int s = 0; s < nsplit; s++) {
-            a += logits[(size_t)s * split_stride + (size_t)r * E + e];
-            b2 += logits[(size_t)s * split_stride + (size_t)sel_row * E + e];
+        for (int s0 = 0; s0 < nsplit; s0 += 8) {  // eight splits of both rows in flight, added in split order
+            float va[8], vb[8];
+#pragma unroll
+            for (int j = 0; j < 8; j++) {
+                bool on = s0 + j < nsplit;
+                va[j] = on ? __ldcg(logits + (size_t)(s0 + j) * split_stride + (size_t)r * E + e) : 0.f;
+                vb[j] = on ? __ldcg(logits + (size_t)(s0 + j) * split_stride + (size_t)sel_row * E + e) : 0.f;
+            }
+#pragma unroll
+            for (int j = 0; j < 8; j++) {
+                a += va[j];
+                b2 += vb[j];
+            }
         }
         own[e] = a;
         sel[e] = b2;
@@ -527,6 +539,7 @@ __global__ void __launch_bounds__(32) route_kernel(const float *logits, int nspl
         wts[(size_t)r * kmax + j] = j < k ? (own[e] / sum) / tot : 0.f;
         if (last) last[(size_t)path * last_stride_path + (size_t)(r - path * Bc) * kmax + j] = e;
     }
+    DBT_TL_END("route");
 }
 
 // Per-expert lists of (row, slot) entries in ascending order, and the size of the union.
