@@ -28,10 +28,10 @@ sys.path.insert(0, ROOT)
 from paper_2608_12385_b200 import replicas  # noqa: E402
 from paper_2608_12385_b200.inputs import PRESETS, make_synthetic_kv, make_tokens, make_weights  # noqa: E402
 
-# ncu DRAM traffic / algorithmic bytes per launch (captures summarised under profiles/): attention 141.9 MB
+# ncu DRAM traffic / algorithmic bytes per launch (captures summarised under profiles/): attention 140.8 MB
 # read+written for 134.6 MB of visible K/V (the rest is the Q|K|V partials it consumes and its output); the GEMMs
 # read their weights once (46.47 MB for 46.14 MB of gate|up weights).
-NCU_TRAFFIC_OVER_ALGORITHMIC = {"attention": 141.9 / 134.58, "gemm_gateup": 1.007, "gemm_down": 1.034, "gemm_qkv": 1.02,
+NCU_TRAFFIC_OVER_ALGORITHMIC = {"attention": 140.8 / 134.58, "gemm_gateup": 1.007, "gemm_down": 1.034, "gemm_qkv": 1.02,
                                 "gemm_o": 1.04}
 METRIC = "grouped_decode_tokens_per_s"
 UNIT = "tokens/s"
