@@ -654,7 +654,6 @@ dbt_status run_attention_mma(dbt_model *m, const RowMap &rm, int grouped, int la
     p.pt_stride = m->pages_per_seq_max;
     long long plane = (long long)c.num_pages * c.n_kv_heads * c.page_size;
     p.k_row0 = (long long)layer * 2 * plane;
-    p.v_row0 = p.k_row0 + plane;
     p.page_table = w.page_table;
     p.seq_len = w.seq_len;
     p.part = w.part;

@@ -35,7 +35,7 @@ struct AttnParams {
     const float *Q;  // [rows][q_dim] fp32, post-RoPE, branch rows already coupled
     RowMap rm;
     int grouped, G, n_kv, num_pages, pt_stride;
-    long long k_row0, v_row0;  // first row of this layer's K / V planes in the pool's 2-D view
+    long long k_row0;  // first row of this layer's K plane in the pool's row numbering (the V plane is one plane further)
     const int32_t *page_table, *seq_len;
     float *part;        // [CTAs + pairs][16][DH + 2] segment partials
     int *tickets;       // [rows][n_kv] arrival counters (zero between launches)
