@@ -93,6 +93,9 @@ struct dbt_model {
     struct ActBase { const void *base; };
     std::map<const CUtensorMap *, ActBase> act_base;
     std::map<std::tuple<const CUtensorMap *, int, int>, CUtensorMap> act3d;
+    int cluster_max;     // largest cluster the GEMM kernel may be launched with (16 when the opt-in size is granted, else 8)
+    int next_cluster_y;  // cluster size along y for the next launch (0: none); consumed by LAUNCH
+    bool cluster_epi;    // opt-in: O and down projections reduce their split-K partials inside a cluster and apply the residual there
     bool stack_planes;  // GEMM: one MMA per k16 step over both activation planes (DBT_STACK=0 issues two)
     bool evict_first;  // weight tiles and K/V pages carry the evict-first L2 hint (DBT_EVICT_FIRST=0 turns it off)
     bool fuse_qkv;     // decode steps: the attention kernel does the Q|K|V epilogue itself (DBT_FUSE_QKV=0 keeps the kernel)
@@ -268,18 +271,29 @@ dbt_status fail(dbt_model *m, dbt_status st, const char *fmt, ...) {
 // stream-serialization attribute, so the kernel may start while its predecessor drains.  Each
 // kernel calls griddepcontrol.wait before it touches anything its predecessor produced.
 template <typename... Params, typename... Args>
-cudaError_t launch_kernel(cudaStream_t stream, bool pdl, dim3 grid, dim3 block, size_t smem, void (*kernel)(Params...),
-                          Args &&...args) {
+cudaError_t launch_kernel(cudaStream_t stream, bool pdl, int cluster_y, dim3 grid, dim3 block, size_t smem,
+                          void (*kernel)(Params...), Args &&...args) {
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = grid;
     cfg.blockDim = block;
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchAttribute attr[2];
+    int n = 0;
+    if (pdl) {
+        attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[n].val.programmaticStreamSerializationAllowed = 1;
+        n++;
+    }
+    if (cluster_y > 1) {  // the CTAs (x, 0..cluster_y-1) of the grid form one thread-block cluster
+        attr[n].id = cudaLaunchAttributeClusterDimension;
+        attr[n].val.clusterDim.x = 1;
+        attr[n].val.clusterDim.y = (unsigned)cluster_y;
+        attr[n].val.clusterDim.z = 1;
+        n++;
+    }
     cfg.attrs = attr;
-    cfg.numAttrs = pdl ? 1 : 0;
+    cfg.numAttrs = n;
     return cudaLaunchKernelEx(&cfg, kernel, Params(std::forward<Args>(args))...);
 }
 
@@ -316,8 +330,9 @@ cudaEvent_t prof_event(dbt_model *m) {
             p1_ = prof_event(m);                                                                         \
             cudaEventRecord(p0_, (m)->stream);                                                           \
         }                                                                                                \
-        cudaError_t e_ = launch_kernel((m)->stream, (m)->use_pdl && !pdl_disabled_for(m, tag), dim3(grid), dim3(block), \
-                                       smem, kernel, __VA_ARGS__);                                       \
+        cudaError_t e_ = launch_kernel((m)->stream, (m)->use_pdl && !pdl_disabled_for(m, tag), (m)->next_cluster_y,     \
+                                       dim3(grid), dim3(block), smem, kernel, __VA_ARGS__);               \
+        (m)->next_cluster_y = 0;                                                                         \
         (m)->launches++;                                                                                 \
         if ((m)->prof_on) {                                                                              \
             cudaEventRecord(p1_, (m)->stream);                                                           \
@@ -613,9 +628,16 @@ dbt_status run_gemm_tc(dbt_model *m, const TcCall &c, int n_tile, int *nsplit_ou
         split = 1;
         p.kt_per_split = total_kt;
     }
+    if (e.cluster) {  // the splits of a tile are one cluster: at most 16 CTAs (the opt-in cluster size)
+        int cap = m->cluster_max;
+        split = total_kt < cap ? total_kt : cap;
+        p.kt_per_split = (total_kt + split - 1) / split;
+        split = (total_kt + p.kt_per_split - 1) / p.kt_per_split;
+    }
     e.arrivals = (e.mode == FE_GATEUP ? 2 : 1) * split;
     if (e.mode != FE_NONE && tiles > 4096) return fail(m, DBT_ERR_UNSUPPORTED, "too many output tiles for %s", c.tag);
     dim3 grid(tiles, split, c.grp_cnt ? c.n_groups : 1);
+    m->next_cluster_y = e.cluster ? split : 0;
     if (nsplit_out) *nsplit_out = split;
     if (split_stride_out) *split_stride_out = (size_t)c.R * col;
     switch (n_tile) {
@@ -1091,6 +1113,13 @@ dbt_status prefill_fused(dbt_model *m, const int32_t *tokens_dev, int B, int n, 
 // leaves per-block shares of sum(S^2); the kernels after the Q|K|V and gate|up GEMMs (and the
 // output-matrix GEMM's own epilogue) multiply by 1/rms.  9 kernels per layer.
 
+// Up to a row tile of 64 the O and down projections finish their own output (cluster reduction of the
+// split-K partials + residual epilogue); their shares of sum(S^2) are then per 128-column tile.
+bool wide_cluster(const dbt_model *m, int n_tile) { return m->cluster_epi && n_tile <= 64; }
+int wide_ss_tiles(const dbt_model *m, int n_tile) {
+    return wide_cluster(m, n_tile) ? (m->cfg.d_model + 127) / 128 : (m->cfg.d_model + 255) / 256;
+}
+
 dbt_status run_layers_wide(dbt_model *m, const RowMap &rm, int grouped, int n_tile) {
     typedef __nv_bfloat16 WT;
     const dbt_config &c = m->cfg;
@@ -1099,7 +1128,8 @@ dbt_status run_layers_wide(dbt_model *m, const RowMap &rm, int grouped, int n_ti
     int d = c.d_model, qd = c.n_q_heads * c.head_dim, kvd = c.n_kv_heads * c.head_dim, F = c.d_ff;
     size_t pool_layer_elems = (size_t)2 * c.num_pages * c.n_kv_heads * c.page_size * c.head_dim;
     size_t lo_x = m->act_parts == 2 ? (size_t)m->Rmax * d : 0, lo_h = m->act_parts == 2 ? (size_t)m->Rmax * F : 0;
-    int ss_tiles = (d + 255) / 256, ss_ld = m->Rmax;
+    const bool clustered = wide_cluster(m, n_tile);
+    int ss_tiles = wide_ss_tiles(m, n_tile), ss_ld = m->Rmax;
     double kv_bytes = 0;
     for (int b = 0; b < rm.B; b++)
         for (int j = 0; j < rm.cn; j++) kv_bytes += (double)(m->len_host[b] + j + 1) * 2 * kvd * sizeof(WT);
@@ -1135,9 +1165,15 @@ dbt_status run_layers_wide(dbt_model *m, const RowMap &rm, int grouped, int n_ti
         if (st != DBT_OK) return st;
         TcCall op = call("gemm_o", &m->map_Ob, qd);
         op.W[0] = &mp.wo; op.n_out[0] = d; op.rows[0] = R; op.nseg = 1;
-        if ((st = run_gemm_tc(m, op, n_tile, &nsp, &sstride)) != DBT_OK) return st;
-        LAUNCH(m, "resid_wide", 0, resid_wide_kernel, dim3(Bc, ss_tiles), 256, 0, w.S, w.P, nsp, sstride, 1,
-               (const float *)nullptr, Bc, grouped, lw.mlp_norm_g, d, w.Xb, lo_x, w.ss, ss_ld);
+        if (clustered) {
+            FusedEpi eo = epi_base(m, rm, grouped, FE_RESID);
+            eo.cluster = 1; eo.S = w.S; eo.g_next = lw.mlp_norm_g; eo.Xout = w.Xb; eo.lo_off = lo_x; eo.ld_out = d; eo.ss_out = w.ss;
+            if ((st = run_gemm_tc(m, op, n_tile, nullptr, nullptr, 0, eo)) != DBT_OK) return st;
+        } else {
+            if ((st = run_gemm_tc(m, op, n_tile, &nsp, &sstride)) != DBT_OK) return st;
+            LAUNCH(m, "resid_wide", 0, resid_wide_kernel, dim3(Bc, ss_tiles), 256, 0, w.S, w.P, nsp, sstride, 1,
+                   (const float *)nullptr, Bc, grouped, lw.mlp_norm_g, d, w.Xb, lo_x, w.ss, ss_ld);
+        }
         TcCall gu = call("gemm_gateup", &m->map_Xb, d);
         gu.W[0] = &mp.wg; gu.n_out[0] = F; gu.rows[0] = R;
         gu.W[1] = &mp.wu; gu.n_out[1] = F; gu.rows[1] = R;
@@ -1147,11 +1183,18 @@ dbt_status run_layers_wide(dbt_model *m, const RowMap &rm, int grouped, int n_ti
                grouped, lw.coup_b, w.Hb, lo_h, (const float *)w.ss, ss_tiles, ss_ld, d, c.rms_eps);
         TcCall dn = call("gemm_down", &m->map_Hb, F);
         dn.W[0] = &mp.wd; dn.n_out[0] = d; dn.rows[0] = R; dn.nseg = 1;
-        if ((st = run_gemm_tc(m, dn, n_tile, &nsp, &sstride)) != DBT_OK) return st;
         const float *g_next = l + 1 < c.n_layers ? m->layers[l + 1].attn_norm_g
                                                  : (c.final_norm ? m->w.final_norm_g : (const float *)nullptr);
-        LAUNCH(m, "resid_wide", 0, resid_wide_kernel, dim3(Bc, ss_tiles), 256, 0, w.S, w.P, nsp, sstride, 2, lw.coup_c, Bc,
-               grouped, g_next, d, w.Xb, lo_x, w.ss, ss_ld);
+        if (clustered) {
+            FusedEpi ed = epi_base(m, rm, grouped, FE_DOWN);
+            ed.cluster = 1; ed.coup = lw.coup_c; ed.S = w.S; ed.g_next = g_next; ed.Xout = w.Xb; ed.lo_off = lo_x; ed.ld_out = d;
+            ed.ss_out = w.ss;
+            if ((st = run_gemm_tc(m, dn, n_tile, nullptr, nullptr, 0, ed)) != DBT_OK) return st;
+        } else {
+            if ((st = run_gemm_tc(m, dn, n_tile, &nsp, &sstride)) != DBT_OK) return st;
+            LAUNCH(m, "resid_wide", 0, resid_wide_kernel, dim3(Bc, ss_tiles), 256, 0, w.S, w.P, nsp, sstride, 2, lw.coup_c, Bc,
+                   grouped, g_next, d, w.Xb, lo_x, w.ss, ss_ld);
+        }
     }
     return DBT_OK;
 }
@@ -1165,20 +1208,20 @@ dbt_status run_head_wide(dbt_model *m, const RowMap &rm, int grouped, int n_tile
     lm.R = R; lm.P = w.Z; lm.P_floats = (size_t)R * c.vocab; lm.tag = "gemm_lm_head";
     lm.parts = m->act_parts; lm.lo_row0 = m->Rmax;
     FusedEpi e = epi_base(m, rm, grouped, FE_LMHEAD);
-    e.ss_tiles = (c.d_model + 255) / 256;
+    e.ss_tiles = wide_ss_tiles(m, n_tile);
     e.use_scale = c.final_norm;
     e.Z = w.Z;
     return run_gemm_tc(m, lm, n_tile, nullptr, nullptr, 0, e);
 }
 
 template <typename WT>
-dbt_status run_embed_wide(dbt_model *m, const int32_t *tokens_dev, int n, int p0, const RowMap &rm, int R) {
+dbt_status run_embed_wide(dbt_model *m, const int32_t *tokens_dev, int n, int p0, const RowMap &rm, int R, int n_tile) {
     const dbt_config &c = m->cfg;
     const Workspace &w = m->ws;
     LAUNCH(m, "embed", 0, embed_fused_kernel<WT>, R, 256, 0, tokens_dev, n, p0, rm, (const WT *)m->w.embed_primary,
            (const WT *)m->w.embed_branch, m->w.embed_norm_g, c.rms_eps, c.d_model, c.vocab, w.S,
            m->layers[0].attn_norm_g, w.Xb, m->act_parts == 2 ? (size_t)m->Rmax * c.d_model : (size_t)0, w.ss, m->Rmax,
-           (c.d_model + 255) / 256, w.status);
+           wide_ss_tiles(m, n_tile), w.status);
     return DBT_OK;
 }
 
@@ -1190,7 +1233,7 @@ dbt_status step_wide(dbt_model *m, const int32_t *tokens_dev, int B, int grouped
     RowMap rm{B, 1};
     int R = grouped ? 2 * B : B, n_tile = pad_rows(2 * B);
     dbt_status st;
-    if ((st = run_embed_wide<WT>(m, tokens_dev, 1, 0, rm, R)) != DBT_OK) return st;
+    if ((st = run_embed_wide<WT>(m, tokens_dev, 1, 0, rm, R, n_tile)) != DBT_OK) return st;
     if ((st = run_layers_wide(m, rm, grouped, n_tile)) != DBT_OK) return st;
     if ((st = run_head_wide(m, rm, grouped, n_tile)) != DBT_OK) return st;
     // the readout also bumps the sequence lengths: nothing after it in the step reads them
@@ -1217,7 +1260,7 @@ dbt_status prefill_wide(dbt_model *m, const int32_t *tokens_dev, int B, int n, f
         int cn = p0 < n_bulk ? (n_bulk - p0 < cn_max ? n_bulk - p0 : cn_max) : 1;
         RowMap rm{B, cn};
         int R = B * cn, n_tile = pad_rows(R);
-        if ((st = run_embed_wide<WT>(m, tokens_dev, n, p0, rm, R)) != DBT_OK) return st;
+        if ((st = run_embed_wide<WT>(m, tokens_dev, n, p0, rm, R, n_tile)) != DBT_OK) return st;
         if ((st = run_layers_wide(m, rm, 0, n_tile)) != DBT_OK) return st;
         if (last_logits && p0 + cn >= n) {
             if ((st = run_head_wide(m, rm, 0, n_tile)) != DBT_OK) return st;
@@ -1407,6 +1450,18 @@ template <int N_TILE>
 bool allow_smem() {
     return cudaFuncSetAttribute(gemm_tc_kernel<N_TILE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 TcCfg<N_TILE>::kSmemBytes) == cudaSuccess;
+}
+// Clusters of 16 CTAs need an opt-in per kernel; without it the clustered epilogue uses 8.
+bool allow_cluster16() {
+    static int state = 0;
+    if (state == 0) {
+        bool ok = cudaFuncSetAttribute(gemm_tc_kernel<16>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess &&
+                  cudaFuncSetAttribute(gemm_tc_kernel<32>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess &&
+                  cudaFuncSetAttribute(gemm_tc_kernel<64>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess;
+        if (!ok) cudaGetLastError();
+        state = ok ? 1 : -1;
+    }
+    return state == 1;
 }
 bool allow_smem_all() {
     static int state = 0;  // 0 unknown, 1 ok, -1 failed
@@ -1635,6 +1690,19 @@ dbt_status dbt_create(const dbt_config *cfg, const dbt_weights *w, void *kv_pool
     {
         // Opt-in (DBT_L2_PREFETCH=1): measured no faster (1.49 vs 1.45 ms per step at batch 16 on the
         // 1B model); the GEMMs of a decode step wait on dependency latency, not on HBM bandwidth.
+        // Opt-in (DBT_CLUSTER=1): the splits of an O / down projection tile as one thread-block cluster that
+        // reduces through distributed shared memory and applies the residual itself.  Measured equal to
+        // the separate residual kernel (1.12 vs 1.12 ms per step at batch 16 on the 1B model): a cluster
+        // is at most 8 CTAs, so the projections run with 8 splits instead of 15-16 and their longer
+        // chains cost what the removed kernel saves; 16-CTA clusters (DBT_CLUSTER_MAX=16) schedule
+        // badly (1.29 ms).
+        const char *cl = getenv("DBT_CLUSTER");
+        m->cluster_epi = cl && strcmp(cl, "1") == 0;
+        m->next_cluster_y = 0;
+        const char *cm = getenv("DBT_CLUSTER_MAX");
+        m->cluster_max = 8;
+        if (cm && atoi(cm) == 16 && m->tc && allow_cluster16()) m->cluster_max = 16;
+        else if (cm && atoi(cm) >= 2 && atoi(cm) <= 8) m->cluster_max = atoi(cm);
         const char *sp = getenv("DBT_STACK");
         m->stack_planes = !(sp && strcmp(sp, "0") == 0);
         const char *ef = getenv("DBT_EVICT_FIRST");

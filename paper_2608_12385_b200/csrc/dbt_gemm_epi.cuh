@@ -24,6 +24,8 @@ enum : int { FE_NONE = 0, FE_QKV = 1, FE_RESID = 2, FE_GATEUP = 3, FE_DOWN = 4, 
 
 struct FusedEpi {
     int mode;
+    int cluster;      // FE_RESID / FE_DOWN: the splits of a tile form a thread-block cluster and reduce through
+                      // distributed shared memory (no tickets, no partials in global memory)
     int Bc, grouped;  // primary rows; branch rows Bc..2Bc-1 present
     RowMap rm;
     int *tickets;     // one counter per output tile (zero between launches)

@@ -105,6 +105,22 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map
         "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
         : "memory");
 }
+// Thread-block cluster helpers: rank, barrier, and a load from a peer CTA's shared memory.
+__device__ __forceinline__ uint32_t cluster_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ float ld_peer_smem(uint32_t local_addr, uint32_t rank) {
+    uint32_t ra;
+    float v;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(local_addr), "r"(rank));
+    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(ra) : "memory");
+    return v;
+}
 // L2 eviction policy for data that is read once per step (weight tiles, K/V pages): evict first, so
 // that the stream does not push the small reused data (activations, partials, gains, tables) out.
 __device__ __forceinline__ uint64_t l2_evict_first_policy() {
@@ -371,6 +387,79 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
                     if (c0 + i < rows) e.Z[(size_t)(c0 + i) * p.ldp + seg.col0 + f] = v[i] * scratch[c0 + i];
             }
         }
+    } else if (e.cluster) {
+        // The splits of this output tile are the CTAs of one cluster.  Each leaves its accumulator tile
+        // in its own shared memory; after a cluster barrier CTA r adds, in split order, the tiles of
+        // all ranks for the primary rows r, r + S, ... (and their branch twins) and finishes those rows:
+        // S-bar = S + . (FE_RESID) or M_2 += c * M_1, S += M (FE_DOWN, Eq. mlp), the next GEMM's input
+        // g * S as two bf16 planes, and this 128-column tile's share of sum(S^2) per row.  Every CTA
+        // takes part in both barriers whatever happened to it, so that nobody waits forever.
+        float *tile_s = scratch;                    // [N_TILE][128] fp32
+        float *red = scratch + N_TILE * kTcM;       // [8] block reduction
+        if (got) {
+#pragma unroll 1
+            for (int c0 = 0; c0 < N_TILE && c0 < rows; c0 += 16) {
+                float v[16];
+                ld_acc(c0, v);
+#pragma unroll
+                for (int i = 0; i < 16; i++) tile_s[(c0 + i) * kTcM + warp * 32 + lane] = v[i];
+            }
+        }
+        cluster_sync();
+        if (got) {
+            const uint32_t rank = cluster_rank(), S = gridDim.y;
+            const int fl = warp * 32 + lane, col = f0 + fl, d = e.ld_out;
+            const bool live = col < seg.n_out;
+            const uint32_t base = smem_u32(tile_s);
+            const float gn = (live && e.g_next) ? e.g_next[col] : 1.f;
+            const float cc = (live && e.mode == FE_DOWN && e.coup) ? e.coup[col] : 0.f;
+            for (int b = (int)rank; b < e.Bc; b += (int)S) {
+                const int r2 = e.Bc + b;
+                float s1 = 0.f, s2 = 0.f, m1 = 0.f, m2 = 0.f;
+                if (live) {
+                    s1 = __ldcg(e.S + (size_t)b * d + col);
+                    if (e.grouped) s2 = __ldcg(e.S + (size_t)r2 * d + col);
+                    float v1[16], v2[16];  // up to 16 ranks (the opt-in cluster size), all loads in flight
+#pragma unroll
+                    for (uint32_t j = 0; j < 16; j++) {
+                        v1[j] = j < S ? ld_peer_smem(base + (uint32_t)(b * kTcM + fl) * 4u, j) : 0.f;
+                        v2[j] = (j < S && e.grouped) ? ld_peer_smem(base + (uint32_t)(r2 * kTcM + fl) * 4u, j) : 0.f;
+                    }
+#pragma unroll
+                    for (int j = 0; j < 16; j++) {
+                        m1 += v1[j];
+                        m2 += v2[j];
+                    }
+                }
+                float q1 = 0.f, q2 = 0.f;
+                if (live) {
+                    s1 += m1;
+                    e.S[(size_t)b * d + col] = s1;
+                    epi_store_split(e.Xout, (size_t)b * d + col, e.lo_off, gn * s1);
+                    q1 = s1 * s1;
+                    if (e.grouped) {
+                        if (e.mode == FE_DOWN) m2 += cc * m1;
+                        s2 += m2;
+                        e.S[(size_t)r2 * d + col] = s2;
+                        epi_store_split(e.Xout, (size_t)r2 * d + col, e.lo_off, gn * s2);
+                        q2 = s2 * s2;
+                    }
+                }
+                q1 = warp_sum(q1);
+                q2 = warp_sum(q2);
+                __syncthreads();
+                if (lane == 0) {
+                    red[warp] = q1;
+                    red[4 + warp] = q2;
+                }
+                __syncthreads();
+                if (tid == 0) {
+                    e.ss_out[(size_t)tile * e.ss_ld + b] = red[0] + red[1] + red[2] + red[3];
+                    if (e.grouped) e.ss_out[(size_t)tile * e.ss_ld + r2] = red[4] + red[5] + red[6] + red[7];
+                }
+            }
+        }
+        cluster_sync();
     } else if (got) {
         int f = f0 + warp * 32 + lane;
         float *out = p.P + ((size_t)split * p.R + x_row0) * p.ldp + seg.col0 + f;

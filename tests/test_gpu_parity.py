@@ -309,12 +309,15 @@ def test_fresh_models_give_bitwise_identical_results():
             assert torch.equal(x["z1"], y["z1"]) and torch.equal(x["z2"], y["z2"])
 
 
-@pytest.mark.parametrize("knob,value", [("DBT_FUSED", "1"), ("DBT_WIDE", "0"), ("DBT_MEGA", "1"), ("DBT_L2_PREFETCH", "1")])
+@pytest.mark.parametrize("knob,value", [("DBT_FUSED", "1"), ("DBT_WIDE", "0"), ("DBT_MEGA", "1"), ("DBT_L2_PREFETCH", "1"),
+                                        ("DBT_CLUSTER", "1"), ("DBT_FUSE_QKV", "0"), ("DBT_STACK", "0"), ("DBT_EVICT_FIRST", "0")])
 def test_alternative_kernel_chains_match_oracle(monkeypatch, knob, value):
     """The variants of the dense chain that are not the default -- elementwise work folded into the
     GEMM epilogues (last-arriving CTA per output tile), a row-wide residual+RMSNorm kernel before
     each GEMM, the whole step as one persistent kernel, L2 prefetch requests riding on the GEMM
-    launches -- compute the same step."""
+    launches, the O / down projections reducing their splits inside a thread-block cluster, a
+    separate Q|K|V epilogue kernel, one MMA per activation plane, no L2 eviction hints -- compute
+    the same step."""
     monkeypatch.setenv(knob, value)
     cfg = small_bf16()
     w = make_weights(cfg, seed=5, matrix_std=0.05)
