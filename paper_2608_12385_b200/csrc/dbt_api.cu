@@ -94,7 +94,8 @@ struct dbt_model {
     std::map<const CUtensorMap *, ActBase> act_base;
     std::map<std::tuple<const CUtensorMap *, int, int>, CUtensorMap> act3d;
     int cluster_max;     // largest cluster the GEMM kernel may be launched with (16 when the opt-in size is granted, else 8)
-    int next_cluster_y;  // cluster size along y for the next launch (0: none); consumed by LAUNCH
+    int next_cluster_x = 1, next_cluster_y;  // cluster dims for the next launch (y 0: none); consumed by LAUNCH
+    bool cluster_gu;     // opt-in: gate|up GEMM as clusters of {gate tile, up tile} x splits that apply SwiGLU + b themselves
     bool cluster_epi;    // opt-in: O and down projections reduce their split-K partials inside a cluster and apply the residual there
     bool stack_planes;  // GEMM: one MMA per k16 step over both activation planes (DBT_STACK=0 issues two)
     bool evict_first;  // weight tiles and K/V pages carry the evict-first L2 hint (DBT_EVICT_FIRST=0 turns it off)
@@ -271,7 +272,7 @@ dbt_status fail(dbt_model *m, dbt_status st, const char *fmt, ...) {
 // stream-serialization attribute, so the kernel may start while its predecessor drains.  Each
 // kernel calls griddepcontrol.wait before it touches anything its predecessor produced.
 template <typename... Params, typename... Args>
-cudaError_t launch_kernel(cudaStream_t stream, bool pdl, int cluster_y, dim3 grid, dim3 block, size_t smem,
+cudaError_t launch_kernel(cudaStream_t stream, bool pdl, int cluster_x, int cluster_y, dim3 grid, dim3 block, size_t smem,
                           void (*kernel)(Params...), Args &&...args) {
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = grid;
@@ -285,9 +286,9 @@ cudaError_t launch_kernel(cudaStream_t stream, bool pdl, int cluster_y, dim3 gri
         attr[n].val.programmaticStreamSerializationAllowed = 1;
         n++;
     }
-    if (cluster_y > 1) {  // the CTAs (x, 0..cluster_y-1) of the grid form one thread-block cluster
+    if (cluster_x * cluster_y > 1) {  // cluster_x x cluster_y neighbouring CTAs of the grid form one thread-block cluster
         attr[n].id = cudaLaunchAttributeClusterDimension;
-        attr[n].val.clusterDim.x = 1;
+        attr[n].val.clusterDim.x = (unsigned)cluster_x;
         attr[n].val.clusterDim.y = (unsigned)cluster_y;
         attr[n].val.clusterDim.z = 1;
         n++;
@@ -330,8 +331,9 @@ cudaEvent_t prof_event(dbt_model *m) {
             p1_ = prof_event(m);                                                                         \
             cudaEventRecord(p0_, (m)->stream);                                                           \
         }                                                                                                \
-        cudaError_t e_ = launch_kernel((m)->stream, (m)->use_pdl && !pdl_disabled_for(m, tag), (m)->next_cluster_y,     \
-                                       dim3(grid), dim3(block), smem, kernel, __VA_ARGS__);               \
+        cudaError_t e_ = launch_kernel((m)->stream, (m)->use_pdl && !pdl_disabled_for(m, tag), (m)->next_cluster_x,     \
+                                       (m)->next_cluster_y, dim3(grid), dim3(block), smem, kernel, __VA_ARGS__); \
+        (m)->next_cluster_x = 1;                                                                         \
         (m)->next_cluster_y = 0;                                                                         \
         (m)->launches++;                                                                                 \
         if ((m)->prof_on) {                                                                              \
@@ -628,8 +630,9 @@ dbt_status run_gemm_tc(dbt_model *m, const TcCall &c, int n_tile, int *nsplit_ou
         split = 1;
         p.kt_per_split = total_kt;
     }
-    if (e.cluster) {  // the splits of a tile are one cluster: at most 16 CTAs (the opt-in cluster size)
-        int cap = m->cluster_max;
+    if (e.cluster) {  // the splits of a tile (of a gate tile and its up tile) are one cluster
+        int cap = e.mode == FE_GATEUP ? m->cluster_max / 2 : m->cluster_max;
+        if (e.mode == FE_GATEUP && split < cap) cap = split;  // keep the measured split where it fits
         split = total_kt < cap ? total_kt : cap;
         p.kt_per_split = (total_kt + split - 1) / split;
         split = (total_kt + p.kt_per_split - 1) / p.kt_per_split;
@@ -638,6 +641,7 @@ dbt_status run_gemm_tc(dbt_model *m, const TcCall &c, int n_tile, int *nsplit_ou
     if (e.mode != FE_NONE && tiles > 4096) return fail(m, DBT_ERR_UNSUPPORTED, "too many output tiles for %s", c.tag);
     dim3 grid(tiles, split, c.grp_cnt ? c.n_groups : 1);
     m->next_cluster_y = e.cluster ? split : 0;
+    m->next_cluster_x = e.cluster && e.mode == FE_GATEUP ? 2 : 1;
     if (nsplit_out) *nsplit_out = split;
     if (split_stride_out) *split_stride_out = (size_t)c.R * col;
     switch (n_tile) {
@@ -1178,9 +1182,15 @@ dbt_status run_layers_wide(dbt_model *m, const RowMap &rm, int grouped, int n_ti
         gu.W[0] = &mp.wg; gu.n_out[0] = F; gu.rows[0] = R;
         gu.W[1] = &mp.wu; gu.n_out[1] = F; gu.rows[1] = R;
         gu.nseg = 2;
-        if ((st = run_gemm_tc(m, gu, n_tile, &nsp, &sstride)) != DBT_OK) return st;
-        LAUNCH(m, "swiglu_couple", 0, swiglu_couple_kernel, dim3(Bc, (F + 255) / 256), 256, 0, w.P, nsp, sstride, F, Bc,
-               grouped, lw.coup_b, w.Hb, lo_h, (const float *)w.ss, ss_tiles, ss_ld, d, c.rms_eps);
+        if (m->cluster_gu && n_tile <= 64) {
+            FusedEpi eg = epi_base(m, rm, grouped, FE_GATEUP);
+            eg.cluster = 1; eg.ss_tiles = ss_tiles; eg.coup = lw.coup_b; eg.Xout = w.Hb; eg.lo_off = lo_h; eg.ld_out = F;
+            if ((st = run_gemm_tc(m, gu, n_tile, nullptr, nullptr, 0, eg)) != DBT_OK) return st;
+        } else {
+            if ((st = run_gemm_tc(m, gu, n_tile, &nsp, &sstride)) != DBT_OK) return st;
+            LAUNCH(m, "swiglu_couple", 0, swiglu_couple_kernel, dim3(Bc, (F + 255) / 256), 256, 0, w.P, nsp, sstride, F, Bc,
+                   grouped, lw.coup_b, w.Hb, lo_h, (const float *)w.ss, ss_tiles, ss_ld, d, c.rms_eps);
+        }
         TcCall dn = call("gemm_down", &m->map_Hb, F);
         dn.W[0] = &mp.wd; dn.n_out[0] = d; dn.rows[0] = R; dn.nseg = 1;
         const float *g_next = l + 1 < c.n_layers ? m->layers[l + 1].attn_norm_g
@@ -1696,6 +1706,12 @@ dbt_status dbt_create(const dbt_config *cfg, const dbt_weights *w, void *kv_pool
         // is at most 8 CTAs, so the projections run with 8 splits instead of 15-16 and their longer
         // chains cost what the removed kernel saves; 16-CTA clusters (DBT_CLUSTER_MAX=16) schedule
         // badly (1.29 ms).
+        // Opt-in (DBT_CLUSTER_GU=1): {gate tile, up tile} x splits as one cluster that applies SwiGLU and the
+        // b coupling itself.  Measured slower than the separate kernel (1.16 vs 1.12 ms per step at batch
+        // 16 on the 1B model): six CTAs finish 16 row pairs of a 128-feature tile on the GEMM's critical
+        // path, where the separate kernel spreads the same work over 352 blocks.
+        const char *cg = getenv("DBT_CLUSTER_GU");
+        m->cluster_gu = cg && strcmp(cg, "1") == 0;
         const char *cl = getenv("DBT_CLUSTER");
         m->cluster_epi = cl && strcmp(cl, "1") == 0;
         m->next_cluster_y = 0;

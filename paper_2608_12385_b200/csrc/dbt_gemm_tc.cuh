@@ -16,6 +16,7 @@
 #include <cuda.h>
 
 #include "dbt_common.cuh"
+#include "dbt_fused.cuh"
 #include "dbt_gemm_epi.cuh"
 
 namespace dbt {
@@ -229,6 +230,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
     DBT_TL_DECL;
     int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     int tile = blockIdx.x, split = blockIdx.y;
+    // Clustered gate|up: CTAs (2j, y) and (2j + 1, y) hold gate tile j and up tile j, so that a cluster
+    // of 2 x splits CTAs owns everything SwiGLU needs for 128 features.
+    if (e.cluster && e.mode == FE_GATEUP) tile = (int)(blockIdx.x & 1) * p.seg[1].tile0 + (int)(blockIdx.x >> 1);
     int x_row0 = 0, w_row0 = 0, grp_n = -1;
     if (p.grp_cnt) {
         // the expert's row list comes from the previous kernel: nothing can start before it is known
@@ -387,6 +391,61 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
                     if (c0 + i < rows) e.Z[(size_t)(c0 + i) * p.ldp + seg.col0 + f] = v[i] * scratch[c0 + i];
             }
         }
+    } else if (e.cluster && e.mode == FE_GATEUP) {
+        // The cluster is {gate tile j, up tile j} x splits (rank = x + 2 * y).  Each CTA leaves its
+        // accumulator tile in shared memory; after the barrier CTA r finishes the primary rows r, r + n,
+        // ... and their branch twins for the tile's 128 features: gate and up summed over the splits in
+        // split order, 1/rms of the GEMM input, H = SiLU(gate) * up, H~_2 = H_2 + b * H_1 (Eq. mlp), two
+        // bf16 planes for the down projection.
+        float *tile_s = scratch;  // [N_TILE][128] fp32
+        if (got) {
+#pragma unroll 1
+            for (int c0 = 0; c0 < N_TILE && c0 < rows; c0 += 16) {
+                float v[16];
+                ld_acc(c0, v);
+#pragma unroll
+                for (int i = 0; i < 16; i++) tile_s[(c0 + i) * kTcM + warp * 32 + lane] = v[i];
+            }
+        }
+        cluster_sync();
+        if (got) {
+            const uint32_t rank = cluster_rank(), S = gridDim.y, nranks = 2 * S;
+            const int fl = warp * 32 + lane, col = f0 + fl, F = e.ld_out;
+            const bool live = col < seg.n_out;
+            const uint32_t base = smem_u32(tile_s);
+            const float cb = (live && e.coup) ? e.coup[col] : 0.f;
+            for (int b = (int)rank; b < e.Bc; b += (int)nranks) {
+                const int r2 = e.Bc + b;
+                float rs1 = 1.f, rs2 = 1.f;
+                if (e.use_scale) row_scale2(e.ss_in, e.ss_tiles, e.ss_ld, b, e.grouped ? r2 : b, e.d_norm, e.eps, rs1, rs2);
+                if (live) {
+                    float g1 = 0.f, u1 = 0.f, g2 = 0.f, u2 = 0.f;
+                    float vg1[4], vu1[4], vg2[4], vu2[4];
+#pragma unroll
+                    for (uint32_t y = 0; y < 4; y++) {
+                        bool on = y < S;
+                        vg1[y] = on ? ld_peer_smem(base + (uint32_t)(b * kTcM + fl) * 4u, 2 * y) : 0.f;
+                        vu1[y] = on ? ld_peer_smem(base + (uint32_t)(b * kTcM + fl) * 4u, 2 * y + 1) : 0.f;
+                        vg2[y] = (on && e.grouped) ? ld_peer_smem(base + (uint32_t)(r2 * kTcM + fl) * 4u, 2 * y) : 0.f;
+                        vu2[y] = (on && e.grouped) ? ld_peer_smem(base + (uint32_t)(r2 * kTcM + fl) * 4u, 2 * y + 1) : 0.f;
+                    }
+#pragma unroll
+                    for (int y = 0; y < 4; y++) {
+                        g1 += vg1[y];
+                        u1 += vu1[y];
+                        g2 += vg2[y];
+                        u2 += vu2[y];
+                    }
+                    float h1 = silu(rs1 * g1) * (rs1 * u1);
+                    epi_store_split(e.Xout, (size_t)b * F + col, e.lo_off, h1);
+                    if (e.grouped) {
+                        float h2 = silu(rs2 * g2) * (rs2 * u2) + cb * h1;
+                        epi_store_split(e.Xout, (size_t)r2 * F + col, e.lo_off, h2);
+                    }
+                }
+            }
+        }
+        cluster_sync();
     } else if (e.cluster) {
         // The splits of this output tile are the CTAs of one cluster.  Each leaves its accumulator tile
         // in its own shared memory; after a cluster barrier CTA r adds, in split order, the tiles of
