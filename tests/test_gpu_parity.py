@@ -109,6 +109,36 @@ def test_1b_shape_full_width_grouped_step_with_synthetic_cache():
     assert_logits_close(g["z1"], o["z1"], "bf16", "1B primary-only z1")
 
 
+def test_1b_at_the_benchmarks_launch_configuration_on_sampled_sequences():
+    """The configuration bench.py times -- dense 1B, batch 16, context 2048 -- with the same launch
+    shapes (row tile 32, the attention split of 128 pairs of 33 stages).  The oracle cannot afford 16
+    sequences at this size in a test, so two of them (0 and 11) carry a seeded cache that both sides
+    receive; the other fourteen are filled on the device.  Sequences do not interact, so the sampled
+    rows must match the oracle run on those two sequences alone."""
+    cfg = dense_1b()
+    w = make_weights(cfg, seed=0)
+    B, ctx, pick = 16, 2048, [0, 11]
+    tok = make_tokens(cfg, B, 2, seed=2)
+    k, v = make_synthetic_kv(cfg, len(pick), ctx, seed=3)
+    gm = make_gpu_model(cfg, w, B, ctx + 3)
+    gen = torch.Generator(device=gm.device)
+    gen.manual_seed(5)
+    gm.kv_pool.normal_(0.0, 1.0, generator=gen)
+    gm.write_kv(k, v, page_table=gm.page_table[pick])
+    gm.set_seq_lens([ctx] * B)
+    om = oracle.OracleModel(cfg, w, len(pick), ctx + 3)
+    om.inject_kv(k, v, ctx)
+    for t in range(2):
+        o = om.decode_step(tok[pick, t].numpy())
+        g = gm.decode_full(tok[:, t].cuda().contiguous())
+        assert_logits_close(g["z1"][pick], o["z1"], "bf16", f"bench config step {t} z1")
+        assert_logits_close(g["z2"][pick], o["z2"], "bf16", f"bench config step {t} z2")
+    o = om.decode_step(tok[pick, 1].numpy(), grouped=False)
+    g = gm.decode_full(tok[:, 1].cuda().contiguous(), grouped=False)
+    assert_logits_close(g["z1"][pick], o["z1"], "bf16", "bench config primary-only z1")
+    assert gm.sync_status() == (0, 0)
+
+
 # ---- properties that hold at any size ---------------------------------------------------------------
 
 def _run_steps(gm, tok_dev, n_prefill, grouped):
