@@ -42,11 +42,12 @@ class OrcConfig(C.Structure):
     _fields_ += [("rope_base", C.c_float), ("rms_eps", C.c_float)]
     _fields_ += [(n, C.c_int32) for n in ("final_norm", "n_experts", "d_expert", "n_shared_experts",
                                          "k_primary", "k_branch", "router_mode", "moe_b_coupling",
-                                         "max_batch", "max_seq")]
+                                         "compute_matched", "max_batch", "max_seq")]
 
 
 _LAYER_FIELDS = ("attn_norm_g", "wq", "wk", "wv", "wo", "coup_a", "mlp_norm_g", "w_gate", "w_up", "w_down",
-                 "coup_b", "coup_c", "router", "exp_gate", "exp_up", "exp_down", "sh_gate", "sh_up", "sh_down")
+                 "coup_b", "coup_c", "router", "exp_gate", "exp_up", "exp_down", "sh_gate", "sh_up", "sh_down",
+                 "gate_a", "gate_g")
 
 
 class OrcLayer(C.Structure):
@@ -109,12 +110,13 @@ def _cfg_struct(cfg, max_batch: int, max_seq: int, kv_round_bf16: bool = False) 
                      rope_base=cfg.rope_base, rms_eps=cfg.rms_eps, final_norm=cfg.final_norm,
                      n_experts=cfg.n_experts, d_expert=cfg.d_expert, n_shared_experts=cfg.n_shared_experts,
                      k_primary=cfg.k_primary, k_branch=cfg.k_branch, router_mode=cfg.router_mode,
-                     moe_b_coupling=cfg.moe_b_coupling, max_batch=max_batch, max_seq=max_seq)
+                     moe_b_coupling=cfg.moe_b_coupling, compute_matched=cfg.compute_matched,
+                     max_batch=max_batch, max_seq=max_seq)
 
 
 def _weights_struct(cfg, w: dict):
     want = torch.float32 if cfg.weight_dtype == "fp32" else torch.bfloat16
-    vec = {"attn_norm_g", "coup_a", "mlp_norm_g", "coup_b", "coup_c"}
+    vec = {"attn_norm_g", "coup_a", "mlp_norm_g", "coup_b", "coup_c", "gate_a", "gate_g"}
     layers = (OrcLayer * cfg.n_layers)()
     for l, lw in enumerate(w["layers"]):
         for name in _LAYER_FIELDS:

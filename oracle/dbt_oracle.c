@@ -269,6 +269,8 @@ static void mlp_dense(const orc_config *c, const orc_layer_weights *lw, const fl
 
 /* Eq. moe_layer with per-path fan-out (Eq. moe_budget), un-gated shared experts
  * (M_i = R_i + G(N_i), Appendix B.3) and the c coupling on the total primary output.
+ * Compute-matched allocation (Appendix B.3, Eq. matched_shared_expert): the shared expert
+ * is evaluated on the primary state only, M_2 = R_2(N_2;k_2) + g_G * G(N_1), no b, no c.
  * forced / chosen: [2][n][kmax] slices for this layer (nullable). */
 static void mlp_moe(const orc_config *c, const orc_layer_weights *lw, const float *m1,
                     const float *m2, int n, const int32_t *forced, int32_t *chosen, float *M1,
@@ -284,6 +286,8 @@ static void mlp_moe(const orc_config *c, const orc_layer_weights *lw, const floa
     float *y = (float *)malloc(sizeof(float) * (size_t)d);
     double *acc = (double *)malloc(sizeof(double) * (size_t)d);
     float *Hs1 = (float *)malloc(sizeof(float) * (size_t)n * (Fs > 0 ? Fs : 1));
+    float *G1 = (float *)calloc((size_t)n * d, sizeof(float)); /* G(N_1), zero without shared experts */
+    int matched = c->compute_matched;
     int32_t idx[64];
     float wts[64];
     int32_t *idx1 = (int32_t *)malloc(sizeof(int32_t) * (size_t)n * kmax);
@@ -314,7 +318,9 @@ static void mlp_moe(const orc_config *c, const orc_layer_weights *lw, const floa
                 orc_linear(mat_offset(lw->exp_down, dt, e * (size_t)d * Fe), dt, d, Fe, h, 1, y);
                 for (int i = 0; i < d; i++) acc[i] += (double)wts[j] * (double)y[i];
             }
-            if (Fs > 0) { /* shared expert(s): every token, weight one */
+            if (p == 1 && matched) { /* the branch receives the gated primary shared-expert output */
+                for (int i = 0; i < d; i++) acc[i] += (double)lw->gate_g[i] * (double)G1[(size_t)r * d + i];
+            } else if (Fs > 0) { /* shared expert(s): every token, weight one */
                 orc_linear(lw->sh_gate, dt, Fs, d, m, 1, g);
                 orc_linear(lw->sh_up, dt, Fs, d, m, 1, u);
                 orc_swiglu(g, u, Fs, h);
@@ -322,14 +328,15 @@ static void mlp_moe(const orc_config *c, const orc_layer_weights *lw, const floa
                 if (p == 1 && c->moe_b_coupling)
                     for (int i = 0; i < Fs; i++) h[i] += lw->coup_b[i] * Hs1[(size_t)r * Fs + i];
                 orc_linear(lw->sh_down, dt, d, Fs, h, 1, y);
+                if (p == 0) memcpy(G1 + (size_t)r * d, y, sizeof(float) * (size_t)d);
                 for (int i = 0; i < d; i++) acc[i] += (double)y[i];
             }
-            if (p == 1)
+            if (p == 1 && !matched)
                 for (int i = 0; i < d; i++) acc[i] += (double)lw->coup_c[i] * (double)M1[(size_t)r * d + i];
             for (int i = 0; i < d; i++) M[i] = (float)acc[i];
         }
     }
-    free(logits); free(g); free(u); free(h); free(y); free(acc); free(Hs1); free(idx1);
+    free(logits); free(g); free(u); free(h); free(y); free(acc); free(Hs1); free(G1); free(idx1);
 }
 
 static void mlp_any(const orc_config *c, const orc_layer_weights *lw, const float *m1,
@@ -353,7 +360,7 @@ static int config_ok(const orc_config *c) {
         if (c->d_expert <= 0 || c->k_primary <= 0 || c->k_branch <= 0) return 0;
         if (c->k_primary > c->n_experts || c->k_branch > c->n_experts) return 0;
         if (c->k_primary > 64 || c->k_branch > 64 || c->n_shared_experts < 0) return 0;
-    } else if (c->d_ff <= 0) {
+    } else if (c->d_ff <= 0 || c->compute_matched) {
         return 0;
     }
     return 1;
@@ -403,6 +410,8 @@ static int step(orc_model *m, const int32_t *tokens, int B, int grouped, int wan
     int G = nq / nkv, dt = c->weight_dtype;
     size_t qd = q_dim_of(c), kvd = kv_dim_of(c);
     int R = grouped ? 2 * B : B;
+    /* rows that evaluate attention: the compute-matched branch has none (Eq. matched_attention) */
+    int Ra = (grouped && !c->compute_matched) ? 2 * B : B;
     int kmax = c->k_primary > c->k_branch ? c->k_primary : c->k_branch;
     if (B <= 0 || B > c->max_batch) return -1;
     for (int b = 0; b < B; b++) {
@@ -436,13 +445,13 @@ static int step(orc_model *m, const int32_t *tokens, int B, int grouped, int wan
         for (int r = 0; r < R; r++)
             orc_rmsnorm(S + (size_t)r * d, lw->attn_norm_g, d, c->rms_eps, N + (size_t)r * d);
         /* Q_i = RoPE(N_i W_Q) for both paths; K_1 = RoPE(N_1 W_K), V_1 = N_1 W_V: primary only */
-        orc_linear(lw->wq, dt, (int)qd, d, N, R, Q);
+        orc_linear(lw->wq, dt, (int)qd, d, N, Ra, Q);
         orc_linear(lw->wk, dt, (int)kvd, d, N, B, Kn);
         orc_linear(lw->wv, dt, (int)kvd, d, N, B, Vn);
-        for (int r = 0; r < R; r++) orc_rope(Q + (size_t)r * qd, nq, dh, m->len[r % B], c->rope_base);
+        for (int r = 0; r < Ra; r++) orc_rope(Q + (size_t)r * qd, nq, dh, m->len[r % B], c->rope_base);
         for (int b = 0; b < B; b++) orc_rope(Kn + (size_t)b * kvd, nkv, dh, m->len[b], c->rope_base);
         /* Q~_2 = Q_2 + a * Q_1 */
-        if (grouped)
+        if (Ra == 2 * B)
             for (int b = 0; b < B; b++)
                 for (size_t i = 0; i < qd; i++)
                     Q[(size_t)(B + b) * qd + i] += lw->coup_a[i] * Q[(size_t)b * qd + i];
@@ -457,14 +466,18 @@ static int step(orc_model *m, const int32_t *tokens, int B, int grouped, int wan
         }
         /* both queries attend to primary positions 0..t inclusive */
 #pragma omp parallel for schedule(static)
-        for (int rh = 0; rh < R * nq; rh++) {
+        for (int rh = 0; rh < Ra * nq; rh++) {
             int r = rh / nq, h = rh % nq, b = r % B, g = h / G;
             orc_attend(Q + (size_t)r * qd + (size_t)h * dh, m->kc + cache_index(c, l, b, 0) + (size_t)g * dh,
                        m->vc + cache_index(c, l, b, 0) + (size_t)g * dh, m->len[b] + 1, (int)kvd, dh,
                        O + (size_t)r * qd + (size_t)h * dh);
         }
         /* S-bar_i = S_i + Attn_i W_O */
-        orc_linear(lw->wo, dt, d, (int)qd, O, R, A);
+        orc_linear(lw->wo, dt, d, (int)qd, O, Ra, A);
+        if (grouped && c->compute_matched) /* A_2 = g_A * A_1 (Eq. matched_attention) */
+            for (int b = 0; b < B; b++)
+                for (int i = 0; i < d; i++)
+                    A[(size_t)(B + b) * d + i] = lw->gate_a[i] * A[(size_t)b * d + i];
         for (size_t i = 0; i < (size_t)R * d; i++) S[i] += A[i];
         /* MLP / MoE on RMSNorm(S-bar_i), then S_i^{l+1} = S-bar_i + M_i */
         for (int r = 0; r < R; r++)
@@ -568,10 +581,11 @@ int orc_full_forward(const orc_config *c, const orc_weights *w, const int32_t *t
             orc_linear(lw->wq, dt, (int)qd, d, N1, T, Q1);
             orc_linear(lw->wk, dt, (int)kvd, d, N1, T, K1);
             orc_linear(lw->wv, dt, (int)kvd, d, N1, T, V1);
-            orc_linear(lw->wq, dt, (int)qd, d, N2, T, Q2);
+            if (!c->compute_matched) orc_linear(lw->wq, dt, (int)qd, d, N2, T, Q2);
             for (int t = 0; t < T; t++) {
                 orc_rope(Q1 + (size_t)t * qd, nq, dh, t, c->rope_base);
                 orc_rope(K1 + (size_t)t * kvd, nkv, dh, t, c->rope_base);
+                if (c->compute_matched) continue;
                 orc_rope(Q2 + (size_t)t * qd, nq, dh, t, c->rope_base);
                 for (size_t i = 0; i < qd; i++) Q2[(size_t)t * qd + i] += lw->coup_a[i] * Q1[(size_t)t * qd + i];
             }
@@ -579,7 +593,7 @@ int orc_full_forward(const orc_config *c, const orc_weights *w, const int32_t *t
             if (v_out) memcpy(v_out + (((size_t)l * B + b) * T) * kvd, V1, sizeof(float) * (size_t)T * kvd);
             /* softmax(Q K^T / sqrt(d_h) + M_causal) V, the T x T form with an explicit mask */
 #pragma omp parallel for schedule(static)
-            for (int ph = 0; ph < 2 * nq; ph++) {
+            for (int ph = 0; ph < (c->compute_matched ? 1 : 2) * nq; ph++) {
                 int p = ph / nq, h = ph % nq, g = h / G;
                 const float *Qp = p ? Q2 : Q1;
                 float *Op = p ? O2 : O1;
@@ -608,7 +622,12 @@ int orc_full_forward(const orc_config *c, const orc_weights *w, const int32_t *t
                 free(P);
             }
             orc_linear(lw->wo, dt, d, (int)qd, O1, T, A1);
-            orc_linear(lw->wo, dt, d, (int)qd, O2, T, A2);
+            if (c->compute_matched) { /* A_2 = g_A * A_1 (Eq. matched_attention) */
+                for (int t = 0; t < T; t++)
+                    for (int i = 0; i < d; i++) A2[(size_t)t * d + i] = lw->gate_a[i] * A1[(size_t)t * d + i];
+            } else {
+                orc_linear(lw->wo, dt, d, (int)qd, O2, T, A2);
+            }
             for (size_t i = 0; i < (size_t)T * d; i++) {
                 S1[i] += A1[i];
                 S2[i] += A2[i];

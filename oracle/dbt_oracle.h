@@ -44,6 +44,11 @@ typedef struct {
     int32_t moe_b_coupling;    /* 1: b couples the shared expert's hidden state; 0: none.
                                   The paper defines b for a single MLP only -- parity
                                   unpinned for MoE layers.                                  */
+    int32_t compute_matched;   /* 1: compute-matched MoE allocation (Appendix B.3): the branch
+                                  evaluates no attention and no shared expert of its own,
+                                  A_2 = g_A * A_1 and M_2 = R_2(N_2;k_2) + g_G * G(N_1);
+                                  the a/b/c couplings do not appear in those equations and
+                                  are not applied.  MoE layers only.                       */
     int32_t max_batch, max_seq;
 } orc_config;
 
@@ -60,6 +65,7 @@ typedef struct {
     const void  *router;                      /* [E,d]                               */
     const void  *exp_gate, *exp_up, *exp_down;/* [E,Fe,d] [E,Fe,d] [E,d,Fe]          */
     const void  *sh_gate, *sh_up, *sh_down;   /* [Fs,d] [Fs,d] [d,Fs], Fs=n_shared*Fe*/
+    const float *gate_a, *gate_g;             /* [d] [d]   g_A, g_G of Appendix B.3 (compute_matched) */
 } orc_layer_weights;
 
 typedef struct {

@@ -37,6 +37,7 @@ class ModelConfig:
     k_branch: int = 0
     router_mode: int = 0  # 0 independent routing, 1 router replay
     moe_b_coupling: int = 1
+    compute_matched: int = 0  # 1: compute-matched MoE allocation (Appendix B.3): A_2 = g_A*A_1, shared expert gated
     page_size: int = 16
 
     @property
@@ -115,7 +116,7 @@ PRESETS = {"tiny": tiny_dense_fp32, "1b": dense_1b, "8b": dense_8b, "moe": moe_1
 LAYER_MATRICES_DENSE = ("wq", "wk", "wv", "wo", "w_gate", "w_up", "w_down")
 LAYER_MATRICES_MOE = ("wq", "wk", "wv", "wo", "router", "exp_gate", "exp_up", "exp_down",
                       "sh_gate", "sh_up", "sh_down")
-LAYER_VECTORS = ("attn_norm_g", "coup_a", "mlp_norm_g", "coup_b", "coup_c")
+LAYER_VECTORS = ("attn_norm_g", "coup_a", "mlp_norm_g", "coup_b", "coup_c", "gate_a", "gate_g")
 
 
 def _normal(gen: torch.Generator, shape, std: float, dtype: torch.dtype, mean: float = 0.0) -> torch.Tensor:
@@ -164,6 +165,9 @@ def make_weights(cfg: ModelConfig, seed: int = 0, coupling_std: float = 0.5,
                 lw["sh_up"] = _normal(gen, (Fs, d), matrix_std, wd)
                 lw["sh_down"] = _normal(gen, (d, Fs), matrix_std, wd)
             lw["coup_b"] = _normal(gen, (max(Fs, 1),), coupling_std, torch.float32)
+            if cfg.compute_matched:  # g_A, g_G: trained from one; spread so that a dropped gate shows
+                lw["gate_a"] = _normal(gen, (d,), coupling_std, torch.float32, 1.0)
+                lw["gate_g"] = _normal(gen, (d,), coupling_std, torch.float32, 1.0)
         else:
             F = cfg.d_ff
             lw["w_gate"] = _normal(gen, (F, d), matrix_std, wd)

@@ -84,8 +84,12 @@ def forward(cfg, w, tokens, branch: bool = True):
         v1 = n1 @ _w(lw["wv"]).T
         ks.append(k1)
         vs.append(v1)
-        s1 = s1 + _attn(q1, k1, v1, cfg) @ _w(lw["wo"]).T
-        if branch:
+        a1 = _attn(q1, k1, v1, cfg) @ _w(lw["wo"]).T
+        s1 = s1 + a1
+        matched = bool(getattr(cfg, "compute_matched", 0))
+        if branch and matched:  # Appendix B.3: a gated copy of the primary attention update
+            s2 = s2 + _w(lw["gate_a"]) * a1
+        elif branch:
             n2 = _norm(s2, lw["attn_norm_g"], eps)
             q2 = _rope_complex(n2 @ _w(lw["wq"]).T, cfg.n_q_heads, cfg.head_dim, cfg.rope_base)
             q2 = q2 + _w(lw["coup_a"]) * q1
@@ -102,11 +106,16 @@ def forward(cfg, w, tokens, branch: bool = True):
         else:
             M1, idx1 = _moe_routed(m1, lw, cfg, cfg.k_primary)
             hs1 = None
+            shared1 = torch.zeros_like(M1)
             if cfg.n_shared_experts > 0:
                 hs1 = _swiglu_hidden(m1, lw["sh_gate"], lw["sh_up"])
-                M1 = M1 + hs1 @ _w(lw["sh_down"]).T
+                shared1 = hs1 @ _w(lw["sh_down"]).T
+                M1 = M1 + shared1
             s1 = s1 + M1
-            if branch:
+            if branch and matched:  # Appendix B.3: own routed experts + gated primary shared expert
+                M2, _ = _moe_routed(m2, lw, cfg, cfg.k_branch)
+                s2 = s2 + M2 + _w(lw["gate_g"]) * shared1
+            elif branch:
                 if cfg.router_mode == 1:
                     M2, _ = _moe_routed(m2, lw, cfg, cfg.k_primary, idx_override=idx1)
                 else:
