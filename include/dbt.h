@@ -69,6 +69,10 @@ typedef struct {
     int32_t k_branch;         /* k_2 of Eq. moe_budget */
     int32_t router_mode;      /* DBT_ROUTER_* (replay: Section 4.3) */
     int32_t moe_b_coupling;   /* 1: b couples the shared expert's hidden state; 0: b unused in MoE */
+    int32_t compute_matched;  /* 1: compute-matched MoE allocation (Appendix B.3): the branch evaluates no
+                                 attention and no shared expert; A_2 = g_A*A_1 (Eq. matched_attention),
+                                 M_2 = R_2(N_2;k_2) + g_G*G(N_1) (Eq. matched_shared_expert); a, b, c are
+                                 not applied.  MoE models only (DBT_ERR_UNSUPPORTED otherwise). */
     int32_t max_batch, max_seq;
     int32_t page_size; /* tokens per KV page; 16 */
     int32_t num_pages; /* pages in the pool, per layer and per K/V */
@@ -86,6 +90,7 @@ typedef struct {
     const void *router;                        /* [E,d]                                       */
     const void *exp_gate, *exp_up, *exp_down;  /* [E,Fe,d] [E,Fe,d] [E,d,Fe]                  */
     const void *sh_gate, *sh_up, *sh_down;     /* [Fs,d] [Fs,d] [d,Fs], Fs = n_shared*Fe      */
+    const float *gate_a, *gate_g;              /* [d] [d]  g_A, g_G (compute_matched only)    */
 } dbt_layer_weights;
 
 typedef struct {

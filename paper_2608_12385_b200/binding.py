@@ -39,12 +39,12 @@ class DbtConfig(C.Structure):
                                          "vocab", "weight_dtype")]
     _fields_ += [("rope_base", C.c_float), ("rms_eps", C.c_float)]
     _fields_ += [(n, C.c_int32) for n in ("final_norm", "n_experts", "d_expert", "n_shared_experts", "k_primary",
-                                         "k_branch", "router_mode", "moe_b_coupling", "max_batch", "max_seq",
+                                         "k_branch", "router_mode", "moe_b_coupling", "compute_matched", "max_batch", "max_seq",
                                          "page_size", "num_pages")]
 
 
 LAYER_FIELDS = ("attn_norm_g", "wq", "wk", "wv", "wo", "coup_a", "mlp_norm_g", "w_gate", "w_up", "w_down", "coup_b",
-                "coup_c", "router", "exp_gate", "exp_up", "exp_down", "sh_gate", "sh_up", "sh_down")
+                "coup_c", "router", "exp_gate", "exp_up", "exp_down", "sh_gate", "sh_up", "sh_down", "gate_a", "gate_g")
 
 
 class DbtLayerWeights(C.Structure):
@@ -112,7 +112,8 @@ def make_config_struct(cfg: ModelConfig, max_batch: int, max_seq: int, num_pages
                      vocab=cfg.vocab, weight_dtype=0 if cfg.weight_dtype == "fp32" else 1, rope_base=cfg.rope_base,
                      rms_eps=cfg.rms_eps, final_norm=cfg.final_norm, n_experts=cfg.n_experts, d_expert=cfg.d_expert,
                      n_shared_experts=cfg.n_shared_experts, k_primary=cfg.k_primary, k_branch=cfg.k_branch,
-                     router_mode=cfg.router_mode, moe_b_coupling=cfg.moe_b_coupling, max_batch=max_batch,
+                     router_mode=cfg.router_mode, moe_b_coupling=cfg.moe_b_coupling,
+                     compute_matched=cfg.compute_matched, max_batch=max_batch,
                      max_seq=max_seq, page_size=cfg.page_size, num_pages=num_pages)
 
 

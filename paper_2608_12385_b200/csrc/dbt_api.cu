@@ -155,6 +155,7 @@ const char *check_config(const dbt_config *c, dbt_status *st) {
     if (2 * (c->n_q_heads / c->n_kv_heads) > 16) return "more than 16 queries per KV head over both paths";
     if (c->d_model % 8) return "d_model must be a multiple of 8";
     if (c->router_mode != DBT_ROUTER_INDEPENDENT && c->router_mode != DBT_ROUTER_REPLAY) return "unknown router_mode";
+    if (c->compute_matched && c->n_experts <= 0) return "compute_matched is defined for MoE models only";
     if (c->n_experts > 0) {
         if (c->d_expert <= 0 || c->d_expert % 8) return "d_expert must be a positive multiple of 8";
         if (c->k_primary <= 0 || c->k_branch <= 0) return "k_primary and k_branch must be positive";
@@ -430,17 +431,21 @@ dbt_status run_moe(dbt_model *m, int l, const RowMap &rm, int grouped, bool reco
     LAUNCH(m, "expert_down", 0, expert_down_kernel<WT>, g2, kLinWarps * 32, 0, (const WT *)lw.exp_down, Fe, d, w.Hexp, w.ecnt,
            w.elist, m->Rmax, w.Yexp);
     const float *Msh = nullptr;
+    // compute-matched allocation (Eq. matched_shared_expert): the shared expert runs on the primary rows only
+    const bool matched = grouped && c.compute_matched;
+    const int Rs = matched ? Bc : R;
     if (Fs > 0) {  // shared expert(s): every row of both paths; b couples its hidden state
         LinArgs gu{};
-        gu.W[0] = lw.sh_gate; gu.W[1] = lw.sh_up; gu.Y[0] = w.Hsh; gu.n_out[0] = Fs; gu.rows[0] = R;
-        gu.nseg = 2; gu.X = w.X; gu.K = d; gu.epi = EPI_SWIGLU; gu.Bc = Bc; gu.grouped = grouped;
+        gu.W[0] = lw.sh_gate; gu.W[1] = lw.sh_up; gu.Y[0] = w.Hsh; gu.n_out[0] = Fs; gu.rows[0] = Rs;
+        gu.nseg = 2; gu.X = w.X; gu.K = d; gu.epi = EPI_SWIGLU; gu.Bc = Bc; gu.grouped = matched ? 0 : grouped;
         gu.coup = c.moe_b_coupling ? lw.coup_b : nullptr;
         if ((st = run_linear<WT>(m, "shared_gateup", gu)) != DBT_OK) return st;
-        LinArgs dn = lin1(lw.sh_down, w.Msh, d, R, w.Hsh, Fs, EPI_STORE);
+        LinArgs dn = lin1(lw.sh_down, w.Msh, d, Rs, w.Hsh, Fs, EPI_STORE);
         if ((st = run_linear<WT>(m, "shared_down", dn)) != DBT_OK) return st;
         Msh = w.Msh;
     }
-    LAUNCH(m, "moe_combine", 0, moe_combine_kernel, Bc, 256, 0, w.Yexp, Msh, w.ridx, w.rwts, km, Bc, grouped, lw.coup_c, d, w.S);
+    LAUNCH(m, "moe_combine", 0, moe_combine_kernel, Bc, 256, 0, w.Yexp, Msh, w.ridx, w.rwts, km, Bc, grouped, lw.coup_c,
+           matched ? lw.gate_g : (const float *)nullptr, d, w.S);
     return DBT_OK;
 }
 
@@ -456,6 +461,9 @@ dbt_status run_layers(dbt_model *m, const RowMap &rm, int grouped, bool record_e
     size_t pool_kv_elems = pool_layer_elems / 2;
     int nsplit = (2 * 148 + Bc * c.n_kv_heads - 1) / (Bc * c.n_kv_heads);
     nsplit = nsplit < 1 ? 1 : nsplit > 16 ? 16 : nsplit;
+    // compute-matched allocation (Eq. matched_attention): attention is evaluated on the primary rows alone
+    const bool matched = grouped && c.compute_matched;
+    const int ga = matched ? 0 : grouped, Ra = ga ? 2 * Bc : Bc;
     double kv_bytes = 0;  // K and V of every visible position, once per layer
     for (int b = 0; b < rm.B; b++)
         for (int j = 0; j < rm.cn; j++) kv_bytes += (double)(m->len_host[b] + j + 1) * 2 * kvd * sizeof(WT);
@@ -468,22 +476,22 @@ dbt_status run_layers(dbt_model *m, const RowMap &rm, int grouped, bool record_e
         LAUNCH(m, "rmsnorm", 0, rmsnorm_kernel, R, 256, 0, w.S, lw.attn_norm_g, c.rms_eps, d, 1, 0, 1, w.X);
         // Q for all rows; K, V for the primary rows only (the branch produces only a query)
         LinArgs a{};
-        a.W[0] = lw.wq; a.Y[0] = w.Q; a.n_out[0] = qd; a.rows[0] = R;
+        a.W[0] = lw.wq; a.Y[0] = w.Q; a.n_out[0] = qd; a.rows[0] = Ra;
         a.W[1] = lw.wk; a.Y[1] = w.Kn; a.n_out[1] = kvd; a.rows[1] = Bc;
         a.W[2] = lw.wv; a.Y[2] = w.Vn; a.n_out[2] = kvd; a.rows[2] = Bc;
         a.nseg = 3; a.X = w.X; a.K = d; a.epi = EPI_STORE;
         if ((st = run_linear<WT>(m, "linear_qkv", a)) != DBT_OK) return st;
-        LAUNCH(m, "rope_append", 0, rope_couple_append_kernel<WT>, Bc, 256, 0, w.Q, w.Kn, w.Vn, rm, grouped, c.n_q_heads, c.n_kv_heads,
+        LAUNCH(m, "rope_append", 0, rope_couple_append_kernel<WT>, Bc, 256, 0, w.Q, w.Kn, w.Vn, rm, ga, c.n_q_heads, c.n_kv_heads,
                c.head_dim, lw.coup_a, w.rope, w.seq_len, w.page_table, m->pages_per_seq_max, c.num_pages, c.page_size,
                kpool, vpool, w.status);
         if (c.head_dim == 128)
-            st = run_attention<WT, 128>(m, rm, grouped, kpool, vpool, nsplit, kv_bytes);
+            st = run_attention<WT, 128>(m, rm, ga, kpool, vpool, nsplit, kv_bytes);
         else
-            st = run_attention<WT, 64>(m, rm, grouped, kpool, vpool, nsplit, kv_bytes);
+            st = run_attention<WT, 64>(m, rm, ga, kpool, vpool, nsplit, kv_bytes);
         if (st != DBT_OK) return st;
-        // S-bar_i = S_i + Attn_i W_O
-        LinArgs o = lin1(lw.wo, nullptr, d, R, w.O, qd, EPI_RESID);
-        o.S = w.S;
+        // S-bar_i = S_i + Attn_i W_O  (matched: S-bar_2 = S_2 + g_A * Attn_1 W_O)
+        LinArgs o = lin1(lw.wo, nullptr, d, Ra, w.O, qd, matched ? EPI_RESID_GATED : EPI_RESID);
+        o.S = w.S; o.Bc = Bc; o.coup = matched ? lw.gate_a : nullptr;
         if ((st = run_linear<WT>(m, "linear_o", o)) != DBT_OK) return st;
         LAUNCH(m, "rmsnorm", 0, rmsnorm_kernel, R, 256, 0, w.S, lw.mlp_norm_g, c.rms_eps, d, 1, 0, 1, w.X);
         if (c.n_experts == 0) {
@@ -764,25 +772,28 @@ dbt_status run_moe_tc(dbt_model *m, int l, const RowMap &rm, int grouped, bool r
     const float *Psh = nullptr;
     int nsp = 1;
     size_t sstride = 0;
+    // compute-matched allocation (Eq. matched_shared_expert): the shared expert runs on the primary rows only
+    const bool matched = grouped && c.compute_matched;
+    const int Rs = matched ? Bc : R;
     if (Fs > 0) {
         int nt = pad_rows(R);
         TcCall sg{};
-        sg.W[0] = &mp.wg; sg.n_out[0] = Fs; sg.rows[0] = R;
-        sg.W[1] = &mp.wu; sg.n_out[1] = Fs; sg.rows[1] = R;
-        sg.nseg = 2; sg.X = &m->map_Xb; sg.K = d; sg.R = R; sg.P = w.P; sg.P_floats = w.P_floats; sg.tag = "shared_gateup";
+        sg.W[0] = &mp.wg; sg.n_out[0] = Fs; sg.rows[0] = Rs;
+        sg.W[1] = &mp.wu; sg.n_out[1] = Fs; sg.rows[1] = Rs;
+        sg.nseg = 2; sg.X = &m->map_Xb; sg.K = d; sg.R = Rs; sg.P = w.P; sg.P_floats = w.P_floats; sg.tag = "shared_gateup";
         sg.parts = m->act_parts; sg.lo_row0 = m->Rmax;
         if ((st = run_gemm_tc(m, sg, nt, &nsp, &sstride)) != DBT_OK) return st;
         LAUNCH(m, "swiglu_couple", 0, swiglu_couple_kernel, dim3(Bc, (Fs + 255) / 256), 256, 0, w.P, nsp, sstride, Fs, Bc,
-               grouped, c.moe_b_coupling ? lw.coup_b : (const float *)nullptr, w.Hb,
+               matched ? 0 : grouped, c.moe_b_coupling ? lw.coup_b : (const float *)nullptr, w.Hb,
                m->act_parts == 2 ? (size_t)m->Rmax * Fs : (size_t)0, (const float *)nullptr, 0, 0, d, c.rms_eps);
         TcCall sd{};
-        sd.W[0] = &mp.wd; sd.n_out[0] = d; sd.rows[0] = R; sd.nseg = 1; sd.X = &m->map_Hb; sd.K = Fs; sd.R = R;
+        sd.W[0] = &mp.wd; sd.n_out[0] = d; sd.rows[0] = Rs; sd.nseg = 1; sd.X = &m->map_Hb; sd.K = Fs; sd.R = Rs;
         sd.P = w.P; sd.P_floats = w.P_floats; sd.tag = "shared_down"; sd.parts = m->act_parts; sd.lo_row0 = m->Rmax;
         if ((st = run_gemm_tc(m, sd, nt, &nsp, &sstride)) != DBT_OK) return st;
         Psh = w.P;
     }
     LAUNCH(m, "moe_combine", 0, moe_combine_sorted_kernel, dim3(Bc, (d + 255) / 256), 256, 0, w.Yexp, Psh, nsp, sstride, w.ridx, w.epos, w.rwts, km,
-           Bc, grouped, lw.coup_c, d, w.S);
+           Bc, grouped, lw.coup_c, matched ? lw.gate_g : (const float *)nullptr, d, w.S);
     return DBT_OK;
 }
 
@@ -804,6 +815,9 @@ dbt_status run_layers_tc(dbt_model *m, const RowMap &rm, int grouped, int n_tile
     for (int b = 0; b < rm.B; b++)
         for (int j = 0; j < rm.cn; j++) kv_bytes += (double)(m->len_host[b] + j + 1) * 2 * kvd * sizeof(WT);
     bool moe = c.n_experts > 0;
+    // compute-matched allocation (Eq. matched_attention): attention is evaluated on the primary rows alone
+    const bool matched = grouped && c.compute_matched;
+    const int ga = matched ? 0 : grouped, Ra = ga ? 2 * Bc : Bc;
     size_t lo_x = m->act_parts == 2 ? (size_t)m->Rmax * d : 0;
     dbt_status st;
     int mode = 0, nsp = 1;
@@ -818,36 +832,37 @@ dbt_status run_layers_tc(dbt_model *m, const RowMap &rm, int grouped, int n_tile
                l > 0 ? m->layers[l - 1].coup_c : nullptr, Bc, grouped, lw.attn_norm_g, c.rms_eps, d, 1, 1, 0, w.Xb,
                lo_x, (float *)nullptr);
         TcCall qkv{};
-        qkv.W[0] = &mp.wq; qkv.n_out[0] = qd; qkv.rows[0] = R;
+        qkv.W[0] = &mp.wq; qkv.n_out[0] = qd; qkv.rows[0] = Ra;
         qkv.W[1] = &mp.wk; qkv.n_out[1] = kvd; qkv.rows[1] = Bc;
         qkv.W[2] = &mp.wv; qkv.n_out[2] = kvd; qkv.rows[2] = Bc;
-        qkv.nseg = 3; qkv.X = &m->map_Xb; qkv.K = d; qkv.R = R; qkv.P = w.P; qkv.P_floats = w.P_floats; qkv.parts = m->act_parts; qkv.lo_row0 = m->Rmax; qkv.tag = "gemm_qkv";
+        qkv.nseg = 3; qkv.X = &m->map_Xb; qkv.K = d; qkv.R = Ra; qkv.P = w.P; qkv.P_floats = w.P_floats; qkv.parts = m->act_parts; qkv.lo_row0 = m->Rmax; qkv.tag = "gemm_qkv";
         qkv.pf_ptr[0] = lw.wo; qkv.pf_bytes[0] = (size_t)d * qd * sizeof(WT);
         if ((st = run_gemm_tc(m, qkv, n_tile, &nsp, &sstride)) != DBT_OK) return st;
         const bool fuse = m->fuse_qkv && m->att_fast && rm.cn == 1;
         QkvFuse qf{w.P, nsp, sstride, nullptr, 0, 0, lw.coup_a};
         if (!fuse)
-            LAUNCH(m, "qkv_epilogue", 0, qkv_epilogue_kernel<WT>, dim3(Bc, c.n_q_heads + c.n_kv_heads), 64, 0, w.P, nsp, sstride, w.Q, rm, grouped, c.n_q_heads,
+            LAUNCH(m, "qkv_epilogue", 0, qkv_epilogue_kernel<WT>, dim3(Bc, c.n_q_heads + c.n_kv_heads), 64, 0, w.P, nsp, sstride, w.Q, rm, ga, c.n_q_heads,
                    c.n_kv_heads, c.head_dim, lw.coup_a, w.rope, w.seq_len, w.page_table, m->pages_per_seq_max, c.num_pages,
                    c.page_size, kpool, vpool, w.status, (const float *)nullptr, 0, 0, d, c.rms_eps);
         if (m->att_fast)
-            st = c.head_dim == 128 ? run_attention_mma<128>(m, rm, grouped, l, kv_bytes, fuse ? &qf : nullptr)
-                                   : run_attention_mma<64>(m, rm, grouped, l, kv_bytes, fuse ? &qf : nullptr);
+            st = c.head_dim == 128 ? run_attention_mma<128>(m, rm, ga, l, kv_bytes, fuse ? &qf : nullptr)
+                                   : run_attention_mma<64>(m, rm, ga, l, kv_bytes, fuse ? &qf : nullptr);
         else if (c.head_dim == 128)
-            st = run_attention<WT, 128>(m, rm, grouped, kpool, vpool, att_split, kv_bytes, true);
+            st = run_attention<WT, 128>(m, rm, ga, kpool, vpool, att_split, kv_bytes, true);
         else
-            st = run_attention<WT, 64>(m, rm, grouped, kpool, vpool, att_split, kv_bytes, true);
+            st = run_attention<WT, 64>(m, rm, ga, kpool, vpool, att_split, kv_bytes, true);
         if (st != DBT_OK) return st;
         TcCall op{};
-        op.W[0] = &mp.wo; op.n_out[0] = d; op.rows[0] = R; op.nseg = 1; op.X = &m->map_Ob; op.K = qd; op.R = R;
+        op.W[0] = &mp.wo; op.n_out[0] = d; op.rows[0] = Ra; op.nseg = 1; op.X = &m->map_Ob; op.K = qd; op.R = Ra;
         op.P = w.P; op.P_floats = w.P_floats; op.parts = m->act_parts; op.lo_row0 = m->Rmax; op.tag = "gemm_o";
         if (!moe) {
             op.pf_ptr[0] = lw.w_gate; op.pf_bytes[0] = (size_t)c.d_ff * d * sizeof(WT);
             op.pf_ptr[1] = lw.w_up; op.pf_bytes[1] = (size_t)c.d_ff * d * sizeof(WT);
         }
         if ((st = run_gemm_tc(m, op, n_tile, &nsp, &sstride)) != DBT_OK) return st;
-        // S-bar_i = S_i + Attn_i W_O ; RMSNorm for the MLP
-        LAUNCH(m, "resid_norm", 0, resid_norm_kernel, Bc, norm_threads(d), 0, w.S, w.P, nsp, sstride, 1, (const float *)nullptr, Bc,
+        // S-bar_i = S_i + Attn_i W_O (matched: S-bar_2 = S_2 + g_A * Attn_1 W_O) ; RMSNorm for the MLP
+        LAUNCH(m, "resid_norm", 0, resid_norm_kernel, Bc, norm_threads(d), 0, w.S, w.P, nsp, sstride, matched ? 3 : 1,
+               matched ? lw.gate_a : (const float *)nullptr, Bc,
                grouped, lw.mlp_norm_g, c.rms_eps, d, 1, 1, 0, w.Xb, lo_x, moe ? w.X : (float *)nullptr);
         if (!moe) {
             int F = c.d_ff;
@@ -1664,6 +1679,7 @@ dbt_status dbt_create(const dbt_config *cfg, const dbt_weights *w, void *kv_pool
     for (int l = 0; l < cfg->n_layers; l++) {
         const dbt_layer_weights &lw = w->layers[l];
         bool ok = lw.attn_norm_g && lw.wq && lw.wk && lw.wv && lw.wo && lw.coup_a && lw.mlp_norm_g && lw.coup_c;
+        if (cfg->compute_matched) ok = ok && lw.gate_a && lw.gate_g;
         if (moe) {
             ok = ok && lw.router && lw.exp_gate && lw.exp_up && lw.exp_down;
             if (cfg->n_shared_experts > 0)

@@ -159,6 +159,7 @@ __global__ void __launch_bounds__(256) resid_wide_kernel(float *S, const float *
 //   mode 0: S unchanged                                   (after the embedding, after an MoE layer)
 //   mode 1: S += sum_s P[s]                               (S-bar_i = S_i + Attn_i W_O)
 //   mode 2: M = sum_s P[s]; M_2 += c * M_1; S += M        (Eq. mlp: M_2 = H~_2 W_D + c*M_1)
+//   mode 3: M_1 = sum_s P[s]; M_2 = g * M_1; S += M        (Eq. matched_attention; coup_c carries g_A)
 // then Xb = bf16(g * S / rms(S)) (apply_norm) or bf16(S).  Block j handles primary source row
 // j*src_mul + src_add and, in grouped mode, its branch twin; outputs go to rows j and n_out + j.
 __global__ void __launch_bounds__(1024) resid_norm_kernel(float *S, const float *P, int nsplit,
@@ -179,7 +180,7 @@ __global__ void __launch_bounds__(1024) resid_norm_kernel(float *S, const float 
         float v2 = grouped ? S[(size_t)r2 * d + i] : 0.f;
         float sm[2] = {0.f, 0.f};
         if (mode != 0) {
-            const size_t offs[2] = {(size_t)r1 * d + i, (size_t)(grouped ? r2 : r1) * d + i};
+            const size_t offs[2] = {(size_t)r1 * d + i, (size_t)(grouped && mode != 3 ? r2 : r1) * d + i};
             sum_splits_k<2, 8>(P, split_stride, nsplit, offs, sm);  // (1024 threads per block: 64 registers each)
             m1 = sm[0];
             v1 += m1;
@@ -190,6 +191,7 @@ __global__ void __launch_bounds__(1024) resid_norm_kernel(float *S, const float 
             if (mode != 0) {
                 float m2 = sm[1];
                 if (mode == 2) m2 += coup_c[i] * m1;
+                if (mode == 3) m2 = coup_c[i] * m1;
                 v2 += m2;
                 S[(size_t)r2 * d + i] = v2;
             }
@@ -446,11 +448,13 @@ __global__ void __launch_bounds__(256) moe_swiglu_kernel(const float *Pe, const 
 // M_1 = sum_j w_1j Expert_j(m_1) + G(m_1);  M_2 = sum_j w_2j Expert_j(m_2) + G~(m_2) + c*M_1;
 // S_i += M_i.  Ys: expert outputs at sorted positions; Psh: split-K partials of the shared
 // expert's down projection (nullptr: no shared expert).  One block per primary row.
+// gate_g != nullptr (Eq. matched_shared_expert): M_2 = sum_j w_2j Expert_j(m_2) + g_G * G(m_1), no c
+// term; Psh then holds primary rows only.
 __global__ void __launch_bounds__(256) moe_combine_sorted_kernel(const float *Ys, const float *Psh, int nsplit,
                                                                  size_t split_stride, const int32_t *idx,
                                                                  const int32_t *pos, const float *wts, int kmax, int Bc,
-                                                                 int grouped, const float *__restrict__ coup_c, int d,
-                                                                 float *S) {
+                                                                 int grouped, const float *__restrict__ coup_c,
+                                                                 const float *__restrict__ gate_g, int d, float *S) {
     DBT_TL_DECL;
     pdl_enter();
     DBT_TL_WAITED;
@@ -479,15 +483,15 @@ __global__ void __launch_bounds__(256) moe_combine_sorted_kernel(const float *Ys
             }
         }
         if (Psh) {
-            const size_t offs[2] = {(size_t)b * d + i, (size_t)(grouped ? r2 : b) * d + i};
+            const size_t offs[2] = {(size_t)b * d + i, (size_t)(grouped && !gate_g ? r2 : b) * d + i};
             float sm[2];
             sum_splits_k<2, 8>(Psh, split_stride, nsplit, offs, sm);
             m1 += sm[0];
-            m2 += sm[1];
+            m2 += gate_g ? gate_g[i] * sm[0] : sm[1];
         }
         S[(size_t)b * d + i] += m1;
         if (grouped) {
-            m2 += coup_c[i] * m1;
+            if (!gate_g) m2 += coup_c[i] * m1;
             S[(size_t)r2 * d + i] += m2;
         }
     }

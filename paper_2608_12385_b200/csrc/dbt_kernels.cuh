@@ -60,7 +60,7 @@ __global__ void rmsnorm_kernel(const float *S, const float *__restrict__ g, floa
 // One warp per output feature; the warp walks the weight row once per group of RT rows with
 // 128-bit loads.  Up to three weight segments share one launch (Q|K|V).
 
-enum : int { EPI_STORE = 0, EPI_RESID = 1, EPI_SWIGLU = 2, EPI_DOWN = 3 };
+enum : int { EPI_STORE = 0, EPI_RESID = 1, EPI_SWIGLU = 2, EPI_DOWN = 3, EPI_RESID_GATED = 4 };
 
 struct LinArgs {
     const void *W[3];
@@ -73,7 +73,7 @@ struct LinArgs {
     int epi;
     int Bc;       // primary rows in this launch
     int grouped;  // branch rows Bc..2Bc-1 present
-    const float *coup;  // b (EPI_SWIGLU) or c (EPI_DOWN); nullptr = no coupling
+    const float *coup;  // b (EPI_SWIGLU), c (EPI_DOWN) or g_A (EPI_RESID_GATED); nullptr = no coupling
     float *S;     // residual rows [.][n_out[0]] for EPI_RESID / EPI_DOWN
 };
 
@@ -138,9 +138,13 @@ __global__ void __launch_bounds__(kLinWarps * 32) linear_kernel(LinArgs a) {
         for (int r = 0; r < kLinRT; r++) {
             if (lane == r && r0 + r < rows) {
                 size_t o = (size_t)(r0 + r) * n_out + f;
-                if (a.epi == EPI_RESID)
+                if (a.epi == EPI_RESID) {
                     a.S[o] += acc[r];
-                else
+                } else if (a.epi == EPI_RESID_GATED) {
+                    // S-bar_1 = S_1 + A_1 ; S-bar_2 = S_2 + g_A * A_1 (Eq. matched_attention): primary rows only
+                    a.S[o] += acc[r];
+                    a.S[(size_t)(a.Bc + r0 + r) * n_out + f] += a.coup[f] * acc[r];
+                } else
                     Y[o] = acc[r];
             }
         }
@@ -618,16 +622,19 @@ __global__ void __launch_bounds__(kLinWarps * 32) expert_down_kernel(
 
 // M_1 = sum_j w_1j Expert_j(m_1) + G(m_1);  M_2 = sum_j w_2j Expert_j(m_2) + G~(m_2) + c*M_1;
 // S_i += M_i.  Slots are summed in slot order.  One block per primary row.
+// gate_g != nullptr (Eq. matched_shared_expert): M_2 = sum_j w_2j Expert_j(m_2) + g_G * G(m_1), no c term.
 __global__ void moe_combine_kernel(const float *Yexp, const float *Msh,
                                    const int32_t *idx, const float *wts, int kmax, int Bc,
-                                   int grouped, const float *__restrict__ coup_c, int d, float *S) {
+                                   int grouped, const float *__restrict__ coup_c,
+                                   const float *__restrict__ gate_g, int d, float *S) {
     pdl_enter();
     int b = blockIdx.x;
     for (int i = threadIdx.x; i < d; i += blockDim.x) {
         float m1 = 0.f;
         for (int j = 0; j < kmax; j++)
             if (idx[(size_t)b * kmax + j] >= 0) m1 = fmaf(wts[(size_t)b * kmax + j], Yexp[((size_t)b * kmax + j) * d + i], m1);
-        if (Msh) m1 += Msh[(size_t)b * d + i];
+        float sh1 = Msh ? Msh[(size_t)b * d + i] : 0.f;
+        if (Msh) m1 += sh1;
         S[(size_t)b * d + i] += m1;
         if (grouped) {
             int r = Bc + b;
@@ -635,8 +642,12 @@ __global__ void moe_combine_kernel(const float *Yexp, const float *Msh,
             for (int j = 0; j < kmax; j++)
                 if (idx[(size_t)r * kmax + j] >= 0)
                     m2 = fmaf(wts[(size_t)r * kmax + j], Yexp[((size_t)r * kmax + j) * d + i], m2);
-            if (Msh) m2 += Msh[(size_t)r * d + i];
-            m2 += coup_c[i] * m1;
+            if (gate_g)
+                m2 += gate_g[i] * sh1;
+            else {
+                if (Msh) m2 += Msh[(size_t)r * d + i];
+                m2 += coup_c[i] * m1;
+            }
             S[(size_t)r * d + i] += m2;
         }
     }

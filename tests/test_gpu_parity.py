@@ -149,7 +149,8 @@ def _run_steps(gm, tok_dev, n_prefill, grouped):
     return outs
 
 
-@pytest.mark.parametrize("cfg", [tiny_dense_fp32().replace(n_layers=2), small_bf16(), small_moe()])
+@pytest.mark.parametrize("cfg", [tiny_dense_fp32().replace(n_layers=2), small_bf16(), small_moe(),
+                                 small_moe(compute_matched=1)])
 def test_kv_cache_bit_identical_grouped_vs_primary_only(cfg):
     """The primary path never reads the branch: the cache written by grouped decode and by
     primary-only decode is the same bits, and so are the primary logits."""
@@ -284,6 +285,59 @@ def test_moe_1b_shape_two_layers():
     cfg = moe_1b(k_branch=4).replace(n_layers=2)
     flips = _moe_compare(cfg, B=2, T=8, npre=6, matrix_std=0.02)
     assert flips <= 2
+
+
+# ---- compute-matched MoE allocation (Appendix B.3) ---------------------------------------------------------
+
+@pytest.mark.parametrize("cfg", [small_moe(compute_matched=1, k_primary=3, k_branch=1),
+                                 small_moe(compute_matched=1, k_primary=2, k_branch=2, n_shared_experts=2),
+                                 small_moe(compute_matched=1, k_primary=1, k_branch=3, n_shared_experts=0),
+                                 small_moe(compute_matched=1, router_mode=1),
+                                 small_moe(compute_matched=1, n_q_heads=8, n_kv_heads=1, head_dim=128, d_model=384),
+                                 small_moe(compute_matched=1, weight_dtype="fp32")])
+def test_compute_matched_moe_decode_matches_oracle(cfg):
+    """The branch evaluates neither attention nor the shared expert: A_2 = g_A * A_1 and
+    M_2 = R_2(N_2; k_2) + g_G * G(N_1), compared element by element under the device's routing."""
+    flips = _moe_compare(cfg, B=3, T=14, npre=10)
+    assert flips <= 2
+
+
+@pytest.mark.parametrize("knob,value", [("DBT_FORCE_PATH", "simt"), ("DBT_ATTN", "simt"), ("DBT_MOE", "simt"),
+                                        ("DBT_FUSE_QKV", "0"), ("DBT_GRAPH", "0")])
+def test_compute_matched_moe_on_the_alternative_chains(monkeypatch, knob, value):
+    monkeypatch.setenv(knob, value)
+    flips = _moe_compare(small_moe(compute_matched=1, k_primary=2, k_branch=2), B=5, T=13, npre=9)
+    assert flips <= 2
+
+
+def test_compute_matched_moe_1b_shape_two_layers():
+    cfg = moe_1b(k_branch=2).replace(n_layers=2, compute_matched=1)
+    flips = _moe_compare(cfg, B=2, T=8, npre=6, matrix_std=0.02)
+    assert flips <= 2
+
+
+def test_compute_matched_unit_gates_same_embedding_equal_fanout_give_identical_paths():
+    """S_2^0 = S_1^0, A_2 = A_1, R_2 = R_1 and M_2 = R_1 + G(N_1): the two paths' logits are the same bits,
+    at the full MoE width and batch 16."""
+    cfg = moe_1b(k_branch=2).replace(n_layers=2, compute_matched=1)
+    w = make_weights(cfg, seed=31)
+    w["embed_branch"] = w["embed_primary"].clone()
+    for lw in w["layers"]:
+        lw["gate_a"] = torch.ones_like(lw["gate_a"])
+        lw["gate_g"] = torch.ones_like(lw["gate_g"])
+    B, T, npre = 16, 40, 37
+    tok = make_tokens(cfg, B, T, seed=32).cuda()
+    gm = make_gpu_model(cfg, w, B, T)
+    for o in _run_steps(gm, tok, npre, True):
+        assert torch.equal(o["z1"], o["z2"])
+        assert float(o["z1"].abs().max()) > 0
+
+
+def test_compute_matched_is_rejected_for_dense_models():
+    cfg = small_bf16(n_layers=1)
+    w = make_weights(cfg, seed=0)
+    with pytest.raises(binding.DbtError):
+        make_gpu_model(cfg.replace(compute_matched=1), w, 1, 16)
 
 
 # ---- error paths (host-detected, and device-detected without any fault) ---------------------------------
