@@ -106,6 +106,22 @@ def step_bytes(cfg, B: int, ctx_keys_first: int, steps: int, union=None) -> floa
     return mats + B * avg_keys * cfg.kv_bytes_per_token()
 
 
+def bench_config(args):
+    cfg = PRESETS[args.model]()
+    if cfg.is_moe:
+        cfg = cfg.replace(k_branch=args.k_branch, router_mode=args.router_mode, compute_matched=args.compute_matched)
+        if args.k_primary:
+            cfg = cfg.replace(k_primary=args.k_primary)
+    return cfg
+
+
+def workload_name(cfg, args) -> str:
+    if not cfg.is_moe:
+        return f"dense-{args.model}"
+    kind = "compute-matched " if cfg.compute_matched else ""
+    return f"{kind}moe-{args.model} (top-{cfg.k_primary} primary, top-{cfg.k_branch} branch)"
+
+
 def run_ours(args) -> dict | None:
     from paper_2608_12385_b200 import binding, build
 
@@ -113,9 +129,7 @@ def run_ours(args) -> dict | None:
     torch.cuda.set_device(local_rank)
     dev = f"cuda:{local_rank}"
     build.build()
-    cfg = PRESETS[args.model]()
-    if cfg.is_moe:
-        cfg = cfg.replace(k_branch=args.k_branch, router_mode=args.router_mode)
+    cfg = bench_config(args)
     B, S, K, W = args.batch, args.ctx, args.steps, args.warmup
     t0 = time.time()
     w = make_weights(cfg, seed=0)
@@ -224,7 +238,7 @@ def run_ours(args) -> dict | None:
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if cfg.weight_dtype == "bf16" else "f32", "data": "synthetic",
-        "config": {"workload": f"{'moe' if cfg.is_moe else 'dense'}-{args.model} bf16 grouped decode, batch {B}/GPU, prompt {S}, "
+        "config": {"workload": f"{workload_name(cfg, args)} bf16 grouped decode, batch {B}/GPU, prompt {S}, "
                                f"{K} steps (paged KV, 16-token pages)",
                    "batch_per_gpu": B, "prompt": S, "kv_population": kv_mode,
                    "l2_policy": "inputs larger than L2 (weights + KV >= 1.7 GB per step vs 126 MB)",
@@ -244,7 +258,8 @@ def run_ours(args) -> dict | None:
         "primary_only": {"ms_per_step": ms_po / K, "grouped_over_primary_only": (ms_total / K) / (ms_po / K),
                          "experts_loaded_per_layer": po_union_m},
         "moe": None if not cfg.is_moe else {"k_primary": cfg.k_primary, "k_branch": cfg.k_branch,
-                                            "router_mode": cfg.router_mode, "experts_loaded_per_layer": union,
+                                            "router_mode": cfg.router_mode, "compute_matched": cfg.compute_matched,
+                                            "experts_loaded_per_layer": union,
                                             "mean_union": sum(union) / len(union)},
         "kernels": [{"name": r["name"], "launches_per_step": r["launches"] / nprof,
                      "us_per_step": 1e3 * r["total_ms"] / nprof,
@@ -279,7 +294,7 @@ def run_reference(args) -> dict | None:
     rank, _, world = replicas.env_rank()
     if rank != 0:
         return None
-    cfg = PRESETS[args.model]()
+    cfg = bench_config(args)
     w = make_weights(cfg, seed=0)
     S, K, W = args.ctx, args.steps, min(args.warmup, 1)
     K = min(K, args.reference_max_steps)
@@ -288,7 +303,7 @@ def run_reference(args) -> dict | None:
         "impl": "reference", "metric": METRIC, "value": base["value"], "unit": UNIT, "n_gpus": world, "steps": K,
         "warmup": W, "ms_per_step": base["ms_per_step"], "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32 storage, f64 accumulate", "data": "synthetic",
-        "config": {"workload": f"dense-{args.model} grouped decode, CPU oracle, 1 sequence per step (bounded sample of "
+        "config": {"workload": f"{workload_name(cfg, args)} grouped decode, CPU oracle, 1 sequence per step (bounded sample of "
                                f"batch {args.batch}), context {S}"},
         "cpu_baseline": {"value": base["value"], "unit": UNIT, "kind": "oracle", "cores": base["cores"],
                          "sample": base["sample"]},
@@ -307,7 +322,10 @@ def main():
     ap.add_argument("--ctx", type=int, default=2048)
     ap.add_argument("--kv", default="prefill", choices=["prefill", "synthetic"])
     ap.add_argument("--k-branch", type=int, default=2, help="MoE: branch top-k")
+    ap.add_argument("--k-primary", type=int, default=0, help="MoE: primary top-k (0: the preset's)")
     ap.add_argument("--router-mode", type=int, default=0, help="MoE: 0 independent routing, 1 router replay")
+    ap.add_argument("--compute-matched", type=int, default=0,
+                    help="MoE: 1 = compute-matched allocation (attention and shared expert on the primary path only)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--reference-max-steps", type=int, default=128)
     args = ap.parse_args()
