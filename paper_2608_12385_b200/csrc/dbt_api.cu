@@ -42,6 +42,8 @@ struct Workspace {
     // MoE on tensor cores: activation rows sorted by expert
     __nv_bfloat16 *Xs, *Hs;
     float *Pe;
+    float *P2;       // split-K partials of the shared expert's GEMMs when they run beside the routed chain
+    size_t P2_floats;
     int32_t *epos, *eoff;
     size_t P_floats;
     // single-kernel decode step: plans (one per batch size and mode), descriptor array, counters
@@ -117,6 +119,11 @@ struct dbt_model {
     bool use_graph, use_pdl;
     std::string pdl_off;
     cudaStream_t cap_stream;
+    // MoE: the shared expert's three kernels run on a second stream beside the router / routed-expert
+    // chain of the same layer (DBT_MOE_OVERLAP=0 keeps one stream)
+    cudaStream_t side_stream;
+    cudaEvent_t ev_fork, ev_join;
+    bool moe_overlap;
     std::vector<GraphEntry> graphs;
 };
 
@@ -240,6 +247,11 @@ size_t carve(const dbt_config &c, char *base, Workspace *ws, int *Rmax_out, int 
             w.Xs = k.take<__nv_bfloat16>(2 * Rk * d);
             w.Hs = k.take<__nv_bfloat16>(2 * Rk * c.d_expert);
             w.Pe = k.take<float>(Rk * 2 * c.d_expert);
+            size_t wide2 = (size_t)(2 * Fs > d ? 2 * Fs : d);
+            w.P2_floats = Fs > 0 ? (size_t)Rmax * wide2 * 6 : 0;
+            if (w.P2_floats > ((size_t)8 << 20)) w.P2_floats = (size_t)8 << 20;
+            if (Fs > 0 && w.P2_floats < (size_t)Rmax * wide2) w.P2_floats = (size_t)Rmax * wide2;
+            w.P2 = k.take<float>(w.P2_floats);
             w.epos = k.take<int32_t>(Rk);
             w.eoff = k.take<int32_t>(c.n_experts + 1);
         }
@@ -738,6 +750,44 @@ dbt_status run_moe_tc(dbt_model *m, int l, const RowMap &rm, int grouped, bool r
     size_t lo_x = m->act_parts == 2 ? (size_t)m->Rmax * d : 0;
     size_t lo_xs = m->act_parts == 2 ? (size_t)Rk * d : 0, lo_hs = m->act_parts == 2 ? (size_t)Rk * Fe : 0;
     dbt_status st;
+    // shared expert(s) on every row of both paths; b couples its hidden state
+    const float *Psh = nullptr;
+    int nsp = 1;
+    size_t sstride = 0;
+    // compute-matched allocation (Eq. matched_shared_expert): the shared expert runs on the primary rows only
+    const bool matched = grouped && c.compute_matched;
+    const int Rs = matched ? Bc : R;
+    auto shared_expert = [&](float *Pbuf, size_t Pbuf_floats) -> dbt_status {
+        int nt = pad_rows(R);
+        TcCall sg{};
+        sg.W[0] = &mp.wg; sg.n_out[0] = Fs; sg.rows[0] = Rs;
+        sg.W[1] = &mp.wu; sg.n_out[1] = Fs; sg.rows[1] = Rs;
+        sg.nseg = 2; sg.X = &m->map_Xb; sg.K = d; sg.R = Rs; sg.P = Pbuf; sg.P_floats = Pbuf_floats; sg.tag = "shared_gateup";
+        sg.parts = m->act_parts; sg.lo_row0 = m->Rmax;
+        if ((st = run_gemm_tc(m, sg, nt, &nsp, &sstride)) != DBT_OK) return st;
+        LAUNCH(m, "swiglu_couple", 0, swiglu_couple_kernel, dim3(Bc, (Fs + 255) / 256), 256, 0, Pbuf, nsp, sstride, Fs, Bc,
+               matched ? 0 : grouped, c.moe_b_coupling ? lw.coup_b : (const float *)nullptr, w.Hb,
+               m->act_parts == 2 ? (size_t)m->Rmax * Fs : (size_t)0, (const float *)nullptr, 0, 0, d, c.rms_eps);
+        TcCall sd{};
+        sd.W[0] = &mp.wd; sd.n_out[0] = d; sd.rows[0] = Rs; sd.nseg = 1; sd.X = &m->map_Hb; sd.K = Fs; sd.R = Rs;
+        sd.P = Pbuf; sd.P_floats = Pbuf_floats; sd.tag = "shared_down"; sd.parts = m->act_parts; sd.lo_row0 = m->Rmax;
+        if ((st = run_gemm_tc(m, sd, nt, &nsp, &sstride)) != DBT_OK) return st;
+        Psh = Pbuf;
+        return DBT_OK;
+    };
+    // The shared expert depends on the normalised rows only: its three kernels run on a second stream
+    // beside the router, the routing kernels and the routed experts, and join before the combine.
+    const bool overlap = Fs > 0 && m->moe_overlap && m->side_stream;
+    cudaStream_t main_stream = m->stream;
+    if (overlap) {
+        CUDA_TRY(m, cudaEventRecord(m->ev_fork, main_stream));
+        CUDA_TRY(m, cudaStreamWaitEvent(m->side_stream, m->ev_fork, 0));
+        m->stream = m->side_stream;
+        st = shared_expert(w.P2, w.P2_floats);
+        m->stream = main_stream;
+        if (st != DBT_OK) return st;
+        CUDA_TRY(m, cudaEventRecord(m->ev_join, m->side_stream));
+    }
     // router logits on the tensor cores (split-K partials summed by the routing kernel), then
     // top-k per path and renormalised weights
     int rnsp = 1;
@@ -768,30 +818,8 @@ dbt_status run_moe_tc(dbt_model *m, int l, const RowMap &rm, int grouped, bool r
     dn.P = w.Yexp; dn.P_floats = (size_t)Rk * d; dn.tag = "expert_down"; dn.parts = m->act_parts; dn.lo_row0 = Rk;
     dn.grp_cnt = w.ecnt; dn.grp_off = w.eoff; dn.grp_w_rows = d; dn.n_groups = E;
     if ((st = run_gemm_tc(m, dn, n_tile, nullptr, nullptr)) != DBT_OK) return st;
-    // shared expert(s) on every row of both paths; b couples its hidden state
-    const float *Psh = nullptr;
-    int nsp = 1;
-    size_t sstride = 0;
-    // compute-matched allocation (Eq. matched_shared_expert): the shared expert runs on the primary rows only
-    const bool matched = grouped && c.compute_matched;
-    const int Rs = matched ? Bc : R;
-    if (Fs > 0) {
-        int nt = pad_rows(R);
-        TcCall sg{};
-        sg.W[0] = &mp.wg; sg.n_out[0] = Fs; sg.rows[0] = Rs;
-        sg.W[1] = &mp.wu; sg.n_out[1] = Fs; sg.rows[1] = Rs;
-        sg.nseg = 2; sg.X = &m->map_Xb; sg.K = d; sg.R = Rs; sg.P = w.P; sg.P_floats = w.P_floats; sg.tag = "shared_gateup";
-        sg.parts = m->act_parts; sg.lo_row0 = m->Rmax;
-        if ((st = run_gemm_tc(m, sg, nt, &nsp, &sstride)) != DBT_OK) return st;
-        LAUNCH(m, "swiglu_couple", 0, swiglu_couple_kernel, dim3(Bc, (Fs + 255) / 256), 256, 0, w.P, nsp, sstride, Fs, Bc,
-               matched ? 0 : grouped, c.moe_b_coupling ? lw.coup_b : (const float *)nullptr, w.Hb,
-               m->act_parts == 2 ? (size_t)m->Rmax * Fs : (size_t)0, (const float *)nullptr, 0, 0, d, c.rms_eps);
-        TcCall sd{};
-        sd.W[0] = &mp.wd; sd.n_out[0] = d; sd.rows[0] = Rs; sd.nseg = 1; sd.X = &m->map_Hb; sd.K = Fs; sd.R = Rs;
-        sd.P = w.P; sd.P_floats = w.P_floats; sd.tag = "shared_down"; sd.parts = m->act_parts; sd.lo_row0 = m->Rmax;
-        if ((st = run_gemm_tc(m, sd, nt, &nsp, &sstride)) != DBT_OK) return st;
-        Psh = w.P;
-    }
+    if (Fs > 0 && !overlap && (st = shared_expert(w.P, w.P_floats)) != DBT_OK) return st;
+    if (overlap) CUDA_TRY(m, cudaStreamWaitEvent(main_stream, m->ev_join, 0));
     LAUNCH(m, "moe_combine", 0, moe_combine_sorted_kernel, dim3(Bc, (d + 255) / 256), 256, 0, w.Yexp, Psh, nsp, sstride, w.ridx, w.epos, w.rwts, km,
            Bc, grouped, lw.coup_c, matched ? lw.gate_g : (const float *)nullptr, d, w.S);
     return DBT_OK;
@@ -863,7 +891,7 @@ dbt_status run_layers_tc(dbt_model *m, const RowMap &rm, int grouped, int n_tile
         // S-bar_i = S_i + Attn_i W_O (matched: S-bar_2 = S_2 + g_A * Attn_1 W_O) ; RMSNorm for the MLP
         LAUNCH(m, "resid_norm", 0, resid_norm_kernel, Bc, norm_threads(d), 0, w.S, w.P, nsp, sstride, matched ? 3 : 1,
                matched ? lw.gate_a : (const float *)nullptr, Bc,
-               grouped, lw.mlp_norm_g, c.rms_eps, d, 1, 1, 0, w.Xb, lo_x, moe ? w.X : (float *)nullptr);
+               grouped, lw.mlp_norm_g, c.rms_eps, d, 1, 1, 0, w.Xb, lo_x, moe && !m->moe_tc ? w.X : (float *)nullptr);
         if (!moe) {
             int F = c.d_ff;
             TcCall gu{};
@@ -1751,6 +1779,19 @@ dbt_status dbt_create(const dbt_config *cfg, const dbt_weights *w, void *kv_pool
     const char *gr = getenv("DBT_GRAPH");
     m->use_graph = !(gr && strcmp(gr, "0") == 0);
     m->cap_stream = nullptr;
+    m->side_stream = nullptr;
+    m->ev_fork = m->ev_join = nullptr;
+    {
+        const char *ov = getenv("DBT_MOE_OVERLAP");
+        m->moe_overlap = m->moe_tc && cfg->n_shared_experts > 0 && !(ov && strcmp(ov, "0") == 0);
+        if (m->moe_overlap &&
+            (cudaStreamCreateWithFlags(&m->side_stream, cudaStreamNonBlocking) != cudaSuccess ||
+             cudaEventCreateWithFlags(&m->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+             cudaEventCreateWithFlags(&m->ev_join, cudaEventDisableTiming) != cudaSuccess)) {
+            m->moe_overlap = false;  // one stream serves as well, only later
+            cudaGetLastError();
+        }
+    }
     if (m->use_graph && cudaStreamCreateWithFlags(&m->cap_stream, cudaStreamNonBlocking) != cudaSuccess) {
         m->use_graph = false;
         cudaGetLastError();
@@ -1826,6 +1867,9 @@ void dbt_destroy(dbt_model *m) {
         cudaGraphDestroy(g.graph);
     }
     if (m->cap_stream) cudaStreamDestroy(m->cap_stream);
+    if (m->side_stream) cudaStreamDestroy(m->side_stream);
+    if (m->ev_fork) cudaEventDestroy(m->ev_fork);
+    if (m->ev_join) cudaEventDestroy(m->ev_join);
     delete m;
 }
 

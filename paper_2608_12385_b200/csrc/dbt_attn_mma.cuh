@@ -65,6 +65,7 @@ constexpr int kAttMaxItems = 256;  // rows per launch (prefill chunks and batche
 constexpr int kAttMinUnits = 4;    // a CTA takes at least 4 tiles (256 tokens)
 constexpr int kAttMaxSeg = 256;    // most segments a (sequence, KV head) pair is split into
 constexpr int kAttGroup = 8;       // segments merged at once (one round of loads)
+constexpr int kAttSingle = 16;     // up to this many segments, one CTA merges them all (two rounds of loads)
 constexpr int kAttMaxGroups = kAttMaxSeg / kAttGroup;
 constexpr float kLog2e = 1.4426950408889634f;
 
@@ -837,7 +838,7 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
             }
         }
         if (sidx == (int)blockIdx.x) DBT_TL_MARK(1);
-        // ---- merging a pair's segments.  Up to kAttGroup segments: the last one to arrive merges them
+        // ---- merging a pair's segments.  Up to kAttSingle segments: the last one to arrive merges them
         // all, in segment order, and writes the output.  More: the segments form groups of kAttGroup;
         // the last arrival of a group merges it in place into the group's first slot, and the last
         // group to finish merges the group results: two short merges on several CTAs instead of one
@@ -935,7 +936,7 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
         };
         if (nseg > 1) {
             float *slot0 = p.part + (size_t)first_slot * 16 * (DH + 2);
-            if (nseg <= kAttGroup) {
+            if (nseg <= kAttSingle) {
                 if (arrive(p.tickets + pair, nseg)) merge(slot0, 1, nseg, true);
             } else {
                 int gi = seg / kAttGroup, ngroups = (nseg + kAttGroup - 1) / kAttGroup;

@@ -281,6 +281,12 @@ def test_moe_decode_matches_oracle_under_the_devices_routing(cfg):
     assert flips <= 2  # well-separated router logits: the free-running oracle picks the same experts
 
 
+def test_moe_at_batch_40():
+    """40 sequences: 80 stacked rows, a row tile of 128 in the per-expert GEMMs."""
+    flips = _moe_compare(small_moe(k_primary=2, k_branch=2), B=40, T=7, npre=5)
+    assert flips <= 6
+
+
 def test_moe_1b_shape_two_layers():
     cfg = moe_1b(k_branch=4).replace(n_layers=2)
     flips = _moe_compare(cfg, B=2, T=8, npre=6, matrix_std=0.02)
@@ -303,10 +309,19 @@ def test_compute_matched_moe_decode_matches_oracle(cfg):
 
 
 @pytest.mark.parametrize("knob,value", [("DBT_FORCE_PATH", "simt"), ("DBT_ATTN", "simt"), ("DBT_MOE", "simt"),
-                                        ("DBT_FUSE_QKV", "0"), ("DBT_GRAPH", "0")])
+                                        ("DBT_FUSE_QKV", "0"), ("DBT_GRAPH", "0"), ("DBT_MOE_OVERLAP", "0")])
 def test_compute_matched_moe_on_the_alternative_chains(monkeypatch, knob, value):
     monkeypatch.setenv(knob, value)
     flips = _moe_compare(small_moe(compute_matched=1, k_primary=2, k_branch=2), B=5, T=13, npre=9)
+    assert flips <= 2
+
+
+@pytest.mark.parametrize("knob,value", [("DBT_MOE_OVERLAP", "0"), ("DBT_GRAPH", "0"), ("DBT_MOE", "simt")])
+def test_moe_on_the_alternative_chains(monkeypatch, knob, value):
+    """The shared expert on the main stream instead of beside the routed chain, direct launches instead
+    of graph replay, the SIMT expert kernels."""
+    monkeypatch.setenv(knob, value)
+    flips = _moe_compare(small_moe(), B=5, T=13, npre=9)
     assert flips <= 2
 
 
