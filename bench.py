@@ -112,14 +112,17 @@ def bench_config(args):
         cfg = cfg.replace(k_branch=args.k_branch, router_mode=args.router_mode, compute_matched=args.compute_matched)
         if args.k_primary:
             cfg = cfg.replace(k_primary=args.k_primary)
+    if args.layers:  # profiler captures of one kernel: fewer layers, less device memory to save and restore
+        cfg = cfg.replace(n_layers=args.layers)
     return cfg
 
 
 def workload_name(cfg, args) -> str:
     if not cfg.is_moe:
-        return f"dense-{args.model}"
+        return f"dense-{args.model}" + (f" (cut to {cfg.n_layers} layers)" if args.layers else "")
     kind = "compute-matched " if cfg.compute_matched else ""
-    return f"{kind}moe-{args.model} (top-{cfg.k_primary} primary, top-{cfg.k_branch} branch)"
+    cut = f", cut to {cfg.n_layers} layers" if args.layers else ""
+    return f"{kind}moe-{args.model} (top-{cfg.k_primary} primary, top-{cfg.k_branch} branch{cut})"
 
 
 def run_ours(args) -> dict | None:
@@ -326,6 +329,7 @@ def main():
     ap.add_argument("--router-mode", type=int, default=0, help="MoE: 0 independent routing, 1 router replay")
     ap.add_argument("--compute-matched", type=int, default=0,
                     help="MoE: 1 = compute-matched allocation (attention and shared expert on the primary path only)")
+    ap.add_argument("--layers", type=int, default=0, help="cut the model to this many layers (profiler captures only)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--reference-max-steps", type=int, default=128)
     args = ap.parse_args()
