@@ -1,6 +1,6 @@
 """Batch x context sweep of the grouped decode step on one GPU.
 
-    python -m paper_2608_12385_b200.sweep --model 1b --out gpurun_out/sweep_1b.json
+    python -m paper_2608_12385_b200.sweep --model 1b --out sweep_1b.json
 
 For every (batch, context) cell: grouped and primary-only step time (CUDA events around a run of
 graph-replayed steps), algorithmic bytes (shared matrices once + visible K/V once), achieved
@@ -77,7 +77,7 @@ def main():
     ap.add_argument("--kv-cap-gb", type=float, default=100.0)
     ap.add_argument("--tiers", action="store_true", help="also run small cells through the CUDA-core GEMV path")
     ap.add_argument("--peak-gbs", type=float, default=None)
-    ap.add_argument("--out", default="gpurun_out/sweep.json")
+    ap.add_argument("--out", default="sweep.json")
     args = ap.parse_args()
     build.build()
     cfg = PRESETS[args.model]()

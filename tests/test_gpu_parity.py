@@ -293,6 +293,35 @@ def test_moe_1b_shape_two_layers():
     assert flips <= 2
 
 
+@pytest.mark.parametrize("matched", [0, 1])
+def test_moe_1b_at_the_benchmarks_launch_configuration_on_sampled_sequences(matched):
+    """The MoE configuration bench.py times -- 64 experts x 1408 + 1 shared, 16 layers, batch 8, context
+    4096, top-2 primary + top-2 branch -- with the same launch shapes (row tile 16, 32 attention pairs of 9
+    segments, the shared expert beside the routed chain).  Two sequences (0 and 5) carry a seeded cache that
+    both sides receive; the oracle runs them alone under the experts the device chose for them."""
+    cfg = moe_1b(k_branch=2).replace(compute_matched=matched)
+    w = make_weights(cfg, seed=0)
+    B, ctx, pick = 8, 4096, [0, 5]
+    tok = make_tokens(cfg, B, 2, seed=2)
+    k, v = make_synthetic_kv(cfg, len(pick), ctx, seed=3)
+    gm = make_gpu_model(cfg, w, B, ctx + 3)
+    gen = torch.Generator(device=gm.device)
+    gen.manual_seed(5)
+    gm.kv_pool.normal_(0.0, 1.0, generator=gen)
+    gm.write_kv(k, v, page_table=gm.page_table[pick])
+    gm.set_seq_lens([ctx] * B)
+    om = oracle.OracleModel(cfg, w, len(pick), ctx + 3)
+    om.inject_kv(k, v, ctx)
+    for t in range(2):
+        g = gm.decode_full(tok[:, t].cuda().contiguous())
+        ex = gm.last_experts(B).numpy()[:, :, pick]
+        o = om.decode_step(tok[pick, t].numpy(), forced_experts=np.ascontiguousarray(ex))
+        assert_logits_close(g["z1"][pick], o["z1"], "bf16", f"moe bench config step {t} z1")
+        assert_logits_close(g["z2"][pick], o["z2"], "bf16", f"moe bench config step {t} z2")
+        assert (ex[:, :, :, :2] >= 0).all()
+    assert gm.sync_status() == (0, 0)
+
+
 # ---- compute-matched MoE allocation (Appendix B.3) ---------------------------------------------------------
 
 @pytest.mark.parametrize("cfg", [small_moe(compute_matched=1, k_primary=3, k_branch=1),
