@@ -560,7 +560,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
                      "r"((uint32_t)Cfg::kTmemCols)
                      : "memory");
+#ifdef DBT_TL_GEMM_ALL
+    if (p.grp_cnt) tlx_[3] = blockIdx.z * 1000 + blockIdx.x;  // every per-expert CTA leaves a record
+    DBT_TL_END_IF(p.grp_cnt != nullptr, "gemmall");
+#else
     DBT_TL_END("gemm");
+#endif
 }
 
 // ---- host side: tensor maps -------------------------------------------------------------
