@@ -145,7 +145,7 @@ struct Carver {
 
 int elem_bytes(const dbt_config &c) { return c.weight_dtype == DBT_DTYPE_F32 ? 4 : 2; }
 int kmax_of(const dbt_config &c) { return c.k_primary > c.k_branch ? c.k_primary : c.k_branch; }
-int prefill_rows(const dbt_config &c) { return 2 * c.max_batch > 128 ? 2 * c.max_batch : 128; }
+int prefill_rows(const dbt_config &c) { return 2 * c.max_batch > 256 ? 2 * c.max_batch : 256; }
 
 const char *check_config(const dbt_config *c, dbt_status *st) {
     *st = DBT_ERR_INVALID_ARG;
