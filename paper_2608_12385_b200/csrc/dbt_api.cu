@@ -45,6 +45,7 @@ struct Workspace {
     float *P2;       // split-K partials of the shared expert's GEMMs when they run beside the routed chain
     size_t P2_floats;
     int32_t *epos, *eoff;
+    float *rs_sorted;  // 1/rms of each sorted row's source row (norm applied after the per-expert gate|up GEMM)
     size_t P_floats;
     // single-kernel decode step: plans (one per batch size and mode), descriptor array, counters
     char *mega_plans;
@@ -124,6 +125,7 @@ struct dbt_model {
     cudaStream_t side_stream;
     cudaEvent_t ev_fork, ev_join;
     bool moe_overlap;
+    bool moe_wide;  // MoE chain with the RMSNorm factor applied behind the GEMMs (DBT_MOE_WIDE=0: row-wide norm kernels)
     std::vector<GraphEntry> graphs;
 };
 
@@ -254,6 +256,7 @@ size_t carve(const dbt_config &c, char *base, Workspace *ws, int *Rmax_out, int 
             w.P2 = k.take<float>(w.P2_floats);
             w.epos = k.take<int32_t>(Rk);
             w.eoff = k.take<int32_t>(c.n_experts + 1);
+            w.rs_sorted = k.take<float>(Rk);
         }
     }
     if (ws) *ws = w;
@@ -432,7 +435,7 @@ dbt_status run_moe(dbt_model *m, int l, const RowMap &rm, int grouped, bool reco
         CUDA_TRY(m, cudaMemsetAsync(last + (size_t)c.max_batch * km, 0xff, sizeof(int32_t) * c.max_batch * km,
                                     m->stream));
     LAUNCH(m, "route", 0, route_kernel, R, 32, 2 * E * sizeof(float), w.rlogits, 1, (size_t)0, E, Bc, c.k_primary, c.k_branch, km,
-           c.router_mode == DBT_ROUTER_REPLAY, w.ridx, w.rwts, last, c.max_batch * km);
+           c.router_mode == DBT_ROUTER_REPLAY, w.ridx, w.rwts, last, c.max_batch * km, (const float *)nullptr, 0, 0, d, c.rms_eps);
     int32_t *ucnt = record_experts ? w.union_cnt + l : nullptr;
     if (ucnt) CUDA_TRY(m, cudaMemsetAsync(ucnt, 0, sizeof(int32_t), m->stream));
     LAUNCH(m, "moe_lists", 0, moe_lists_kernel, (E + 127) / 128, 128, 0, w.ridx, R, km, E, m->Rmax, w.ecnt, w.elist, ucnt);
@@ -738,7 +741,11 @@ dbt_status run_attention_mma(dbt_model *m, const RowMap &rm, int grouped, int la
 // paths are sorted by expert; one grouped GEMM launch covers all experts (blockIdx.z), CTAs of
 // experts nobody selected exit before touching their weights, so each selected expert's
 // matrices are read once for the union of the primary top-k_1 and branch top-k_2 rows.
-dbt_status run_moe_tc(dbt_model *m, int l, const RowMap &rm, int grouped, bool record_experts) {
+// wide: the rows in Xb are g * S, not yet divided by rms(S) (shares of sum(S^2) in ws.ss): every
+// consumer of a GEMM on them applies the row's factor itself, and the combine leaves the next layer's
+// input in the same form when it is given that layer's gain g_next.
+dbt_status run_moe_tc(dbt_model *m, int l, const RowMap &rm, int grouped, bool record_experts, bool wide,
+                      const float *g_next) {
     typedef __nv_bfloat16 WT;
     const dbt_config &c = m->cfg;
     const Workspace &w = m->ws;
@@ -749,6 +756,8 @@ dbt_status run_moe_tc(dbt_model *m, int l, const RowMap &rm, int grouped, bool r
     int n_tile = pad_rows(R);
     size_t lo_x = m->act_parts == 2 ? (size_t)m->Rmax * d : 0;
     size_t lo_xs = m->act_parts == 2 ? (size_t)Rk * d : 0, lo_hs = m->act_parts == 2 ? (size_t)Rk * Fe : 0;
+    const float *ssp = wide ? w.ss : nullptr;
+    const int ss_tiles = (d + 255) / 256, ss_ld = m->Rmax;
     dbt_status st;
     // shared expert(s) on every row of both paths; b couples its hidden state
     const float *Psh = nullptr;
@@ -767,7 +776,7 @@ dbt_status run_moe_tc(dbt_model *m, int l, const RowMap &rm, int grouped, bool r
         if ((st = run_gemm_tc(m, sg, nt, &nsp, &sstride)) != DBT_OK) return st;
         LAUNCH(m, "swiglu_couple", 0, swiglu_couple_kernel, dim3(Bc, (Fs + 255) / 256), 256, 0, Pbuf, nsp, sstride, Fs, Bc,
                matched ? 0 : grouped, c.moe_b_coupling ? lw.coup_b : (const float *)nullptr, w.Hb,
-               m->act_parts == 2 ? (size_t)m->Rmax * Fs : (size_t)0, (const float *)nullptr, 0, 0, d, c.rms_eps);
+               m->act_parts == 2 ? (size_t)m->Rmax * Fs : (size_t)0, ssp, ss_tiles, ss_ld, d, c.rms_eps);
         TcCall sd{};
         sd.W[0] = &mp.wd; sd.n_out[0] = d; sd.rows[0] = Rs; sd.nseg = 1; sd.X = &m->map_Hb; sd.K = Fs; sd.R = Rs;
         sd.P = Pbuf; sd.P_floats = Pbuf_floats; sd.tag = "shared_down"; sd.parts = m->act_parts; sd.lo_row0 = m->Rmax;
@@ -800,10 +809,11 @@ dbt_status run_moe_tc(dbt_model *m, int l, const RowMap &rm, int grouped, bool r
     if (last && !grouped)
         CUDA_TRY(m, cudaMemsetAsync(last + (size_t)c.max_batch * km, 0xff, sizeof(int32_t) * c.max_batch * km, m->stream));
     LAUNCH(m, "route", 0, route_kernel, R, 32, 2 * E * sizeof(float), w.P, rnsp, rstride, E, Bc, c.k_primary, c.k_branch, km,
-           c.router_mode == DBT_ROUTER_REPLAY, w.ridx, w.rwts, last, c.max_batch * km);
+           c.router_mode == DBT_ROUTER_REPLAY, w.ridx, w.rwts, last, c.max_batch * km, ssp, ss_tiles, ss_ld, d, c.rms_eps);
     LAUNCH(m, "moe_sort", 0, moe_sort_kernel, 1, 1024, 0, w.ridx, R, km, E, w.ecnt, w.eoff, w.epos,
            record_experts ? w.union_cnt + l : (int32_t *)nullptr);
-    LAUNCH(m, "moe_gather", 0, moe_gather_kernel, R * km, 256, 0, w.Xb, lo_x, w.ridx, w.epos, km, d, w.Xs, lo_xs);
+    LAUNCH(m, "moe_gather", 0, moe_gather_kernel, R * km, 256, 0, w.Xb, lo_x, w.ridx, w.epos, km, d, w.Xs, lo_xs, ssp, ss_tiles, ss_ld,
+           c.rms_eps, w.rs_sorted);
     // routed experts: gate|up, SwiGLU, down
     TcCall gu{};
     gu.W[0] = &mp.eg; gu.n_out[0] = Fe; gu.rows[0] = Rk;
@@ -812,7 +822,8 @@ dbt_status run_moe_tc(dbt_model *m, int l, const RowMap &rm, int grouped, bool r
     gu.tag = "expert_gateup"; gu.parts = m->act_parts; gu.lo_row0 = Rk;
     gu.grp_cnt = w.ecnt; gu.grp_off = w.eoff; gu.grp_w_rows = Fe; gu.n_groups = E;
     if ((st = run_gemm_tc(m, gu, n_tile, nullptr, nullptr)) != DBT_OK) return st;
-    LAUNCH(m, "moe_swiglu", 0, moe_swiglu_kernel, dim3(R * km, (Fe + 255) / 256), 256, 0, w.Pe, w.eoff + E, Fe, w.Hs, lo_hs);
+    LAUNCH(m, "moe_swiglu", 0, moe_swiglu_kernel, dim3(R * km, (Fe + 255) / 256), 256, 0, w.Pe, w.eoff + E, Fe, w.Hs, lo_hs,
+           wide ? (const float *)w.rs_sorted : (const float *)nullptr);
     TcCall dn{};
     dn.W[0] = &mp.ed; dn.n_out[0] = d; dn.rows[0] = Rk; dn.nseg = 1; dn.X = &m->map_Hs; dn.K = Fe; dn.R = Rk;
     dn.P = w.Yexp; dn.P_floats = (size_t)Rk * d; dn.tag = "expert_down"; dn.parts = m->act_parts; dn.lo_row0 = Rk;
@@ -820,8 +831,10 @@ dbt_status run_moe_tc(dbt_model *m, int l, const RowMap &rm, int grouped, bool r
     if ((st = run_gemm_tc(m, dn, n_tile, nullptr, nullptr)) != DBT_OK) return st;
     if (Fs > 0 && !overlap && (st = shared_expert(w.P, w.P_floats)) != DBT_OK) return st;
     if (overlap) CUDA_TRY(m, cudaStreamWaitEvent(main_stream, m->ev_join, 0));
+    const bool next_in = wide && g_next != nullptr;
     LAUNCH(m, "moe_combine", 0, moe_combine_sorted_kernel, dim3(Bc, (d + 255) / 256), 256, 0, w.Yexp, Psh, nsp, sstride, w.ridx, w.epos, w.rwts, km,
-           Bc, grouped, lw.coup_c, matched ? lw.gate_g : (const float *)nullptr, d, w.S);
+           Bc, grouped, lw.coup_c, matched ? lw.gate_g : (const float *)nullptr, d, w.S, next_in ? g_next : (const float *)nullptr,
+           next_in ? w.Xb : (__nv_bfloat16 *)nullptr, lo_x, next_in ? w.ss : (float *)nullptr, ss_ld);
     return DBT_OK;
 }
 
@@ -846,6 +859,9 @@ dbt_status run_layers_tc(dbt_model *m, const RowMap &rm, int grouped, int n_tile
     // compute-matched allocation (Eq. matched_attention): attention is evaluated on the primary rows alone
     const bool matched = grouped && c.compute_matched;
     const int ga = matched ? 0 : grouped, Ra = ga ? 2 * Bc : Bc;
+    // MoE on the tensor cores: norm factor behind the GEMMs, no row-wide reduction kernel (DBT_MOE_WIDE=0: before them)
+    const bool mwide = moe && m->moe_tc && m->moe_wide;
+    const int mss_tiles = (d + 255) / 256;
     size_t lo_x = m->act_parts == 2 ? (size_t)m->Rmax * d : 0;
     dbt_status st;
     int mode = 0, nsp = 1;
@@ -855,10 +871,18 @@ dbt_status run_layers_tc(dbt_model *m, const RowMap &rm, int grouped, int n_tile
         const LayerMaps &mp = m->maps[l];
         WT *kpool = reinterpret_cast<WT *>(m->kv_pool) + (size_t)l * pool_layer_elems;
         WT *vpool = kpool + pool_kv_elems;
-        // fold the previous layer's MLP output into S (Eq. mlp), N_i = RMSNorm(S_i)
-        LAUNCH(m, "resid_norm", 0, resid_norm_kernel, Bc, norm_threads(d), 0, w.S, w.P, nsp, sstride, mode,
-               l > 0 ? m->layers[l - 1].coup_c : nullptr, Bc, grouped, lw.attn_norm_g, c.rms_eps, d, 1, 1, 0, w.Xb,
-               lo_x, (float *)nullptr);
+        // fold the previous layer's MLP output into S (Eq. mlp), N_i = RMSNorm(S_i).  MoE, wide form: the
+        // GEMM input is g * S with the 1/rms factor applied behind the GEMM; the previous layer's combine
+        // has left it already, the first layer gets it from the residual kernel with nothing to add.
+        if (mwide) {
+            if (l == 0)
+                LAUNCH(m, "resid_wide", 0, resid_wide_kernel, dim3(Bc, mss_tiles), 256, 0, w.S, w.P, 0, (size_t)0, 1,
+                       (const float *)nullptr, Bc, grouped, lw.attn_norm_g, d, w.Xb, lo_x, w.ss, m->Rmax);
+        } else {
+            LAUNCH(m, "resid_norm", 0, resid_norm_kernel, Bc, norm_threads(d), 0, w.S, w.P, nsp, sstride, mode,
+                   l > 0 ? m->layers[l - 1].coup_c : nullptr, Bc, grouped, lw.attn_norm_g, c.rms_eps, d, 1, 1, 0, w.Xb,
+                   lo_x, (float *)nullptr);
+        }
         TcCall qkv{};
         qkv.W[0] = &mp.wq; qkv.n_out[0] = qd; qkv.rows[0] = Ra;
         qkv.W[1] = &mp.wk; qkv.n_out[1] = kvd; qkv.rows[1] = Bc;
@@ -867,11 +891,12 @@ dbt_status run_layers_tc(dbt_model *m, const RowMap &rm, int grouped, int n_tile
         qkv.pf_ptr[0] = lw.wo; qkv.pf_bytes[0] = (size_t)d * qd * sizeof(WT);
         if ((st = run_gemm_tc(m, qkv, n_tile, &nsp, &sstride)) != DBT_OK) return st;
         const bool fuse = m->fuse_qkv && m->att_fast && rm.cn == 1;
-        QkvFuse qf{w.P, nsp, sstride, nullptr, 0, 0, lw.coup_a};
+        QkvFuse qf{w.P, nsp, sstride, mwide ? w.ss : nullptr, mwide ? mss_tiles : 0, mwide ? m->Rmax : 0, lw.coup_a};
         if (!fuse)
             LAUNCH(m, "qkv_epilogue", 0, qkv_epilogue_kernel<WT>, dim3(Bc, c.n_q_heads + c.n_kv_heads), 64, 0, w.P, nsp, sstride, w.Q, rm, ga, c.n_q_heads,
                    c.n_kv_heads, c.head_dim, lw.coup_a, w.rope, w.seq_len, w.page_table, m->pages_per_seq_max, c.num_pages,
-                   c.page_size, kpool, vpool, w.status, (const float *)nullptr, 0, 0, d, c.rms_eps);
+                   c.page_size, kpool, vpool, w.status, mwide ? (const float *)w.ss : (const float *)nullptr, mwide ? mss_tiles : 0,
+                   mwide ? m->Rmax : 0, d, c.rms_eps);
         if (m->att_fast)
             st = c.head_dim == 128 ? run_attention_mma<128>(m, rm, ga, l, kv_bytes, fuse ? &qf : nullptr)
                                    : run_attention_mma<64>(m, rm, ga, l, kv_bytes, fuse ? &qf : nullptr);
@@ -889,6 +914,10 @@ dbt_status run_layers_tc(dbt_model *m, const RowMap &rm, int grouped, int n_tile
         }
         if ((st = run_gemm_tc(m, op, n_tile, &nsp, &sstride)) != DBT_OK) return st;
         // S-bar_i = S_i + Attn_i W_O (matched: S-bar_2 = S_2 + g_A * Attn_1 W_O) ; RMSNorm for the MLP
+        if (mwide)
+            LAUNCH(m, "resid_wide", 0, resid_wide_kernel, dim3(Bc, mss_tiles), 256, 0, w.S, w.P, nsp, sstride, matched ? 3 : 1,
+                   matched ? lw.gate_a : (const float *)nullptr, Bc, grouped, lw.mlp_norm_g, d, w.Xb, lo_x, w.ss, m->Rmax);
+        else
         LAUNCH(m, "resid_norm", 0, resid_norm_kernel, Bc, norm_threads(d), 0, w.S, w.P, nsp, sstride, matched ? 3 : 1,
                matched ? lw.gate_a : (const float *)nullptr, Bc,
                grouped, lw.mlp_norm_g, c.rms_eps, d, 1, 1, 0, w.Xb, lo_x, moe && !m->moe_tc ? w.X : (float *)nullptr);
@@ -919,7 +948,9 @@ dbt_status run_layers_tc(dbt_model *m, const RowMap &rm, int grouped, int n_tile
             if ((st = run_gemm_tc(m, dn, n_tile, &nsp, &sstride)) != DBT_OK) return st;
             mode = 2;
         } else {
-            st = m->moe_tc ? run_moe_tc(m, l, rm, grouped, record_experts) : run_moe<WT>(m, l, rm, grouped, record_experts);
+            st = m->moe_tc ? run_moe_tc(m, l, rm, grouped, record_experts, mwide,
+                                        l + 1 < c.n_layers ? m->layers[l + 1].attn_norm_g : nullptr)
+                           : run_moe<WT>(m, l, rm, grouped, record_experts);
             if (st != DBT_OK) return st;
             mode = 0;
         }
@@ -1784,6 +1815,8 @@ dbt_status dbt_create(const dbt_config *cfg, const dbt_weights *w, void *kv_pool
     {
         const char *ov = getenv("DBT_MOE_OVERLAP");
         m->moe_overlap = m->moe_tc && cfg->n_shared_experts > 0 && !(ov && strcmp(ov, "0") == 0);
+        const char *mw = getenv("DBT_MOE_WIDE");
+        m->moe_wide = m->moe_tc && m->act_parts == 2 && !(mw && strcmp(mw, "0") == 0);
         if (m->moe_overlap &&
             (cudaStreamCreateWithFlags(&m->side_stream, cudaStreamNonBlocking) != cudaSuccess ||
              cudaEventCreateWithFlags(&m->ev_fork, cudaEventDisableTiming) != cudaSuccess ||

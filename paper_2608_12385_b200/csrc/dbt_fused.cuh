@@ -117,8 +117,8 @@ __global__ void __launch_bounds__(256) resid_wide_kernel(float *S, const float *
         // coupling, and all splits of both rows' partials (up to 16 splits in one round)
         size_t o1 = (size_t)b * d + i, o2 = (size_t)(Bc + b) * d + i;
         float s1 = __ldcg(S + o1), s2 = grouped ? __ldcg(S + o2) : 0.f;
-        float gn = g_next ? g_next[i] : 1.f, cc = mode == 2 ? coup_c[i] : 0.f;
-        const size_t offs[2] = {o1, grouped ? o2 : o1};
+        float gn = g_next ? g_next[i] : 1.f, cc = mode >= 2 ? coup_c[i] : 0.f;
+        const size_t offs[2] = {o1, grouped && mode != 3 ? o2 : o1};
         float mm[2];
         sum_splits_k<2, 16>(P, split_stride, nsplit, offs, mm);
         s1 += mm[0];
@@ -128,6 +128,7 @@ __global__ void __launch_bounds__(256) resid_wide_kernel(float *S, const float *
         if (grouped) {
             float m2 = mm[1];
             if (mode == 2) m2 += cc * mm[0];
+            if (mode == 3) m2 = cc * mm[0];  // Eq. matched_attention: coup_c carries g_A
             s2 += m2;
             S[o2] = s2;
             store_split(Xb, o2, lo_off, gn * s2);
@@ -414,15 +415,24 @@ __global__ void __launch_bounds__(1024) moe_sort_kernel(const int32_t *idx, int 
     DBT_TL_END("moe_sort");
 }
 
-// Copy each entry's activation row (both bf16 planes) to its sorted position.
+// Copy each entry's activation row (both bf16 planes) to its sorted position.  ss != nullptr: the rows
+// hold g * S, not yet divided by rms(S); the row's factor 1/rms goes to rs_sorted[position] for the
+// SwiGLU kernel behind the per-expert gate|up GEMM.
 __global__ void __launch_bounds__(256) moe_gather_kernel(const __nv_bfloat16 *Xb, size_t lo_in, const int32_t *idx,
                                                          const int32_t *pos, int kmax, int d, __nv_bfloat16 *Xs,
-                                                         size_t lo_out) {
+                                                         size_t lo_out, const float *ss, int ss_tiles, int ss_ld,
+                                                         float eps, float *rs_sorted) {
     DBT_TL_DECL;
     pdl_enter();
     DBT_TL_WAITED;
     int entry = blockIdx.x;
     if (idx[entry] < 0) return;
+    if (ss && threadIdx.x < 32) {
+        float a = 0.f;
+        for (int t = threadIdx.x; t < ss_tiles; t += 32) a += __ldcg(ss + (size_t)t * ss_ld + entry / kmax);
+        a = warp_sum(a);
+        if (threadIdx.x == 0) rs_sorted[pos[entry]] = 1.f / sqrtf(a / (float)d + eps);
+    }
     const uint4 *src = reinterpret_cast<const uint4 *>(Xb + (size_t)(entry / kmax) * d);
     uint4 *dst = reinterpret_cast<uint4 *>(Xs + (size_t)pos[entry] * d);
     for (int i = threadIdx.x; i < d / 8; i += blockDim.x) {
@@ -432,15 +442,17 @@ __global__ void __launch_bounds__(256) moe_gather_kernel(const __nv_bfloat16 *Xb
     DBT_TL_END("moe_gath");
 }
 
-// H = SiLU(gate) * up on the sorted rows; Pe rows are [Fe gate | Fe up] (one split).
+// H = SiLU(gate) * up on the sorted rows; Pe rows are [Fe gate | Fe up] (one split).  rs (nullable):
+// the rows' 1/rms factors when the GEMM ran on inputs not yet divided by it.
 __global__ void __launch_bounds__(256) moe_swiglu_kernel(const float *Pe, const int32_t *off_total, int Fe,
-                                                         __nv_bfloat16 *Hs, size_t lo_off) {
+                                                         __nv_bfloat16 *Hs, size_t lo_off, const float *rs) {
     DBT_TL_DECL;
     pdl_enter();
     DBT_TL_WAITED;
     int p = blockIdx.x, f = blockIdx.y * blockDim.x + threadIdx.x;
     if (p >= *off_total || f >= Fe) return;
-    float h = silu(Pe[(size_t)p * 2 * Fe + f]) * Pe[(size_t)p * 2 * Fe + Fe + f];
+    const float sc = rs ? __ldcg(rs + p) : 1.f;
+    float h = silu(sc * Pe[(size_t)p * 2 * Fe + f]) * (sc * Pe[(size_t)p * 2 * Fe + Fe + f]);
     store_split(Hs, (size_t)p * Fe + f, lo_off, h);
     DBT_TL_END("moe_swig");
 }
@@ -450,14 +462,21 @@ __global__ void __launch_bounds__(256) moe_swiglu_kernel(const float *Pe, const 
 // expert's down projection (nullptr: no shared expert).  One block per primary row.
 // gate_g != nullptr (Eq. matched_shared_expert): M_2 = sum_j w_2j Expert_j(m_2) + g_G * G(m_1), no c
 // term; Psh then holds primary rows only.
+// Xn != nullptr (grid (Bc, ceil(d / 256)), 256 threads): the block also leaves the next layer's GEMM
+// input g_next * S (two bf16 planes, the 1/rms factor is applied after that GEMM) and its 256-column
+// share of sum(S^2) for both rows, as resid_wide_kernel does.
 __global__ void __launch_bounds__(256) moe_combine_sorted_kernel(const float *Ys, const float *Psh, int nsplit,
                                                                  size_t split_stride, const int32_t *idx,
                                                                  const int32_t *pos, const float *wts, int kmax, int Bc,
                                                                  int grouped, const float *__restrict__ coup_c,
-                                                                 const float *__restrict__ gate_g, int d, float *S) {
+                                                                 const float *__restrict__ gate_g, int d, float *S,
+                                                                 const float *__restrict__ g_next, __nv_bfloat16 *Xn,
+                                                                 size_t lo_off, float *ss_out, int ss_ld) {
     DBT_TL_DECL;
     pdl_enter();
     DBT_TL_WAITED;
+    __shared__ float scratch[64];
+    float q1 = 0.f, q2 = 0.f;
     int b = blockIdx.x;
     // the row's selections (weights, sorted positions) once, then all expert rows of a column in
     // flight together; terms are added in slot order
@@ -489,10 +508,36 @@ __global__ void __launch_bounds__(256) moe_combine_sorted_kernel(const float *Ys
             m1 += sm[0];
             m2 += gate_g ? gate_g[i] * sm[0] : sm[1];
         }
-        S[(size_t)b * d + i] += m1;
+        const float gn = Xn ? g_next[i] : 0.f;
+        const float v1 = S[(size_t)b * d + i] + m1;
+        S[(size_t)b * d + i] = v1;
+        if (Xn) store_split(Xn, (size_t)b * d + i, lo_off, gn * v1);
+        q1 += v1 * v1;
         if (grouped) {
             if (!gate_g) m2 += coup_c[i] * m1;
-            S[(size_t)r2 * d + i] += m2;
+            const float v2 = S[(size_t)r2 * d + i] + m2;
+            S[(size_t)r2 * d + i] = v2;
+            if (Xn) store_split(Xn, (size_t)r2 * d + i, lo_off, gn * v2);
+            q2 += v2 * v2;
+        }
+    }
+    if (Xn) {  // (uniform per launch) the block's share of both rows' sum(S^2)
+        q1 = warp_sum(q1);
+        q2 = warp_sum(q2);
+        const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+        if (lane == 0) {
+            scratch[warp] = q1;
+            scratch[32 + warp] = q2;
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            float a1 = 0.f, a2 = 0.f;
+            for (int w2 = 0; w2 < nw; w2++) {
+                a1 += scratch[w2];
+                a2 += scratch[32 + w2];
+            }
+            ss_out[(size_t)blockIdx.y * ss_ld + b] = a1;
+            if (grouped) ss_out[(size_t)blockIdx.y * ss_ld + r2] = a2;
         }
     }
     DBT_TL_END("moe_comb");

@@ -467,9 +467,12 @@ __global__ void advance_len_kernel(int32_t *seq_len, int B, int n) {
 // weights renormalised over the selection.  Replay: the branch row takes its primary twin's
 // selection and weighs it with its own probabilities.  One warp per row; logits may arrive
 // as split-K partials [nsplit][R][E] (summed in split order).
+// ss != nullptr: the router GEMM ran on g * S (not yet divided by rms(S)); the row's factor comes
+// from its per-tile shares of sum(S^2) and multiplies the logits here (the GEMM is linear).
 __global__ void __launch_bounds__(32) route_kernel(const float *logits, int nsplit, size_t split_stride, int E, int Bc,
                                                    int k_p, int k_b, int kmax, int replay, int32_t *idx, float *wts,
-                                                   int32_t *last, int last_stride_path) {
+                                                   int32_t *last, int last_stride_path, const float *ss, int ss_tiles,
+                                                   int ss_ld, int d_norm, float eps) {
     DBT_TL_DECL;
     pdl_enter();
     DBT_TL_WAITED;
@@ -479,6 +482,16 @@ __global__ void __launch_bounds__(32) route_kernel(const float *logits, int nspl
     int path = r >= Bc;
     int sel_row = (path && replay) ? r - Bc : r;
     int k = (path && !replay) ? k_b : k_p;
+    float inv_own = 1.f, inv_sel = 1.f;
+    if (ss) {
+        float a = 0.f, b2 = 0.f;
+        for (int t = lane; t < ss_tiles; t += 32) {
+            a += __ldcg(ss + (size_t)t * ss_ld + r);
+            b2 += __ldcg(ss + (size_t)t * ss_ld + sel_row);
+        }
+        inv_own = 1.f / sqrtf(warp_sum(a) / (float)d_norm + eps);
+        inv_sel = 1.f / sqrtf(warp_sum(b2) / (float)d_norm + eps);
+    }
     float mx = -INFINITY;
     for (int e = lane; e < E; e += 32) {
         float a = 0.f, b2 = 0.f;
@@ -496,6 +509,8 @@ __global__ void __launch_bounds__(32) route_kernel(const float *logits, int nspl
                 b2 += vb[j];
             }
         }
+        a *= inv_own;
+        b2 *= inv_sel;
         own[e] = a;
         sel[e] = b2;
         mx = fmaxf(mx, a);

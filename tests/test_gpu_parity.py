@@ -338,17 +338,20 @@ def test_compute_matched_moe_decode_matches_oracle(cfg):
 
 
 @pytest.mark.parametrize("knob,value", [("DBT_FORCE_PATH", "simt"), ("DBT_ATTN", "simt"), ("DBT_MOE", "simt"),
-                                        ("DBT_FUSE_QKV", "0"), ("DBT_GRAPH", "0"), ("DBT_MOE_OVERLAP", "0")])
+                                        ("DBT_FUSE_QKV", "0"), ("DBT_GRAPH", "0"), ("DBT_MOE_OVERLAP", "0"),
+                                        ("DBT_MOE_WIDE", "0")])
 def test_compute_matched_moe_on_the_alternative_chains(monkeypatch, knob, value):
     monkeypatch.setenv(knob, value)
     flips = _moe_compare(small_moe(compute_matched=1, k_primary=2, k_branch=2), B=5, T=13, npre=9)
     assert flips <= 2
 
 
-@pytest.mark.parametrize("knob,value", [("DBT_MOE_OVERLAP", "0"), ("DBT_GRAPH", "0"), ("DBT_MOE", "simt")])
+@pytest.mark.parametrize("knob,value", [("DBT_MOE_OVERLAP", "0"), ("DBT_GRAPH", "0"), ("DBT_MOE", "simt"),
+                                        ("DBT_MOE_WIDE", "0"), ("DBT_FUSE_QKV", "0"), ("DBT_ATTN", "simt")])
 def test_moe_on_the_alternative_chains(monkeypatch, knob, value):
     """The shared expert on the main stream instead of beside the routed chain, direct launches instead
-    of graph replay, the SIMT expert kernels."""
+    of graph replay, the SIMT expert kernels, row-wide norm kernels before the GEMMs instead of the norm
+    factor behind them, the separate Q|K|V epilogue kernel, the CUDA-core attention kernel."""
     monkeypatch.setenv(knob, value)
     flips = _moe_compare(small_moe(), B=5, T=13, npre=9)
     assert flips <= 2
