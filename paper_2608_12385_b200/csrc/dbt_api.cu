@@ -42,6 +42,8 @@ struct Workspace {
     // MoE on tensor cores: activation rows sorted by expert
     __nv_bfloat16 *Xs, *Hs;
     float *Pe;
+    float *ro_stats;      // readout: per (sequence, vocabulary chunk) softmax records and argmax candidates
+    int32_t *ro_tickets;  // readout: arrival counters per sequence
     float *P2;       // split-K partials of the shared expert's GEMMs when they run beside the routed chain
     size_t P2_floats;
     int32_t *epos, *eoff;
@@ -125,6 +127,7 @@ struct dbt_model {
     cudaStream_t side_stream;
     cudaEvent_t ev_fork, ev_join;
     bool moe_overlap;
+    bool readout_row;  // DBT_READOUT=row: the one-CTA-per-row readout kernel
     bool moe_wide;  // MoE chain with the RMSNorm factor applied behind the GEMMs (DBT_MOE_WIDE=0: row-wide norm kernels)
     std::vector<GraphEntry> graphs;
 };
@@ -206,6 +209,8 @@ size_t carve(const dbt_config &c, char *base, Workspace *ws, int *Rmax_out, int 
     w.status = k.take<int32_t>(4);
     w.att_tickets = k.take<int32_t>((size_t)Rmax * c.n_kv_heads);
     w.att_tickets2 = k.take<int32_t>((size_t)Rmax * c.n_kv_heads * kAttMaxGroups);
+    w.ro_stats = k.take<float>((size_t)c.max_batch * kRoMaxChunks * 8);
+    w.ro_tickets = k.take<int32_t>(c.max_batch);
     w.gemm_tickets = k.take<int32_t>(4096);
     w.tokens_stage = k.take<int32_t>(c.max_batch);
     w.next_stage = k.take<int32_t>(c.max_batch);
@@ -360,6 +365,24 @@ cudaEvent_t prof_event(dbt_model *m) {
     } while (0)
 
 // ---- launch helpers -------------------------------------------------------------------
+
+// Mixture readout (Eq. alpha, Eq. mixloss) and greedy token; also advances the sequence lengths.
+// Rows cut into chunks of at most 2048 logits, one CTA per (sequence, chunk): two short launches
+// instead of one CTA walking a row three times (DBT_READOUT=row keeps that kernel).
+dbt_status run_readout(dbt_model *m, int B, int grouped, int32_t *next_dev, float *alpha_dev) {
+    const dbt_config &c = m->cfg;
+    const Workspace &w = m->ws;
+    int nc = (c.vocab + kRoChunk - 1) / kRoChunk;
+    if (m->readout_row || nc > kRoMaxChunks) {
+        LAUNCH(m, "readout", 0, readout_kernel, B, 1024, 0, w.Z, B, c.vocab, grouped, next_dev, alpha_dev, w.seq_len, 1);
+        return DBT_OK;
+    }
+    int chunk = (c.vocab + nc - 1) / nc;
+    if (grouped) LAUNCH(m, "readout_stats", 0, readout_stats_kernel, dim3(B, nc), kRoThreads, 0, w.Z, B, c.vocab, chunk, w.ro_stats);
+    LAUNCH(m, "readout", 0, readout_pick_kernel, dim3(B, nc), kRoThreads, 0, w.Z, B, c.vocab, chunk, grouped, w.ro_stats, w.ro_tickets,
+           next_dev, alpha_dev, w.seq_len, 1);
+    return DBT_OK;
+}
 
 template <typename WT>
 dbt_status run_linear(dbt_model *m, const char *tag, const LinArgs &a) {
@@ -994,7 +1017,7 @@ dbt_status step_tc(dbt_model *m, const int32_t *tokens_dev, int B, int grouped, 
     if ((st = run_layers_tc(m, rm, grouped, n_tile, true, &mode, &nsp, &sstride)) != DBT_OK) return st;
     if ((st = run_head_tc(m, B, grouped, B, 1, 0, n_tile, mode, nsp, sstride)) != DBT_OK) return st;
     // the readout also bumps the sequence lengths: nothing after it in the step reads them
-    LAUNCH(m, "readout", 0, readout_kernel, B, 1024, 0, w.Z, B, c.vocab, grouped, next_dev, alpha_dev, w.seq_len, 1);
+    if ((st = run_readout(m, B, grouped, next_dev, alpha_dev)) != DBT_OK) return st;
     size_t zb = sizeof(float) * (size_t)B * c.vocab;
     if (z1_dev) CUDA_TRY(m, cudaMemcpyAsync(z1_dev, w.Z, zb, cudaMemcpyDeviceToDevice, m->stream));
     if (z2_dev && grouped)
@@ -1149,7 +1172,7 @@ dbt_status step_fused(dbt_model *m, const int32_t *tokens_dev, int B, int groupe
     if ((st = run_layers_fused(m, rm, grouped, n_tile)) != DBT_OK) return st;
     if ((st = run_head_fused(m, rm, grouped, n_tile)) != DBT_OK) return st;
     // the readout also bumps the sequence lengths: nothing after it in the step reads them
-    LAUNCH(m, "readout", 0, readout_kernel, B, 1024, 0, w.Z, B, c.vocab, grouped, next_dev, alpha_dev, w.seq_len, 1);
+    if ((st = run_readout(m, B, grouped, next_dev, alpha_dev)) != DBT_OK) return st;
     size_t zb = sizeof(float) * (size_t)B * c.vocab;
     if (z1_dev) CUDA_TRY(m, cudaMemcpyAsync(z1_dev, w.Z, zb, cudaMemcpyDeviceToDevice, m->stream));
     if (z2_dev && grouped)
@@ -1321,7 +1344,7 @@ dbt_status step_wide(dbt_model *m, const int32_t *tokens_dev, int B, int grouped
     if ((st = run_layers_wide(m, rm, grouped, n_tile)) != DBT_OK) return st;
     if ((st = run_head_wide(m, rm, grouped, n_tile)) != DBT_OK) return st;
     // the readout also bumps the sequence lengths: nothing after it in the step reads them
-    LAUNCH(m, "readout", 0, readout_kernel, B, 1024, 0, w.Z, B, c.vocab, grouped, next_dev, alpha_dev, w.seq_len, 1);
+    if ((st = run_readout(m, B, grouped, next_dev, alpha_dev)) != DBT_OK) return st;
     size_t zb = sizeof(float) * (size_t)B * c.vocab;
     if (z1_dev) CUDA_TRY(m, cudaMemcpyAsync(z1_dev, w.Z, zb, cudaMemcpyDeviceToDevice, m->stream));
     if (z2_dev && grouped)
@@ -1651,7 +1674,7 @@ dbt_status step_impl(dbt_model *m, const int32_t *tokens_dev, int B, int grouped
     if ((st = run_layers<WT>(m, rm, grouped, true)) != DBT_OK) return st;
     if ((st = run_head<WT>(m, R, 1, 0)) != DBT_OK) return st;
     // the readout also bumps the sequence lengths: nothing after it in the step reads them
-    LAUNCH(m, "readout", 0, readout_kernel, B, 1024, 0, w.Z, B, c.vocab, grouped, next_dev, alpha_dev, w.seq_len, 1);
+    if ((st = run_readout(m, B, grouped, next_dev, alpha_dev)) != DBT_OK) return st;
     size_t zb = sizeof(float) * (size_t)B * c.vocab;
     if (z1_dev) CUDA_TRY(m, cudaMemcpyAsync(z1_dev, w.Z, zb, cudaMemcpyDeviceToDevice, m->stream));
     if (z2_dev && grouped)
@@ -1803,6 +1826,8 @@ dbt_status dbt_create(const dbt_config *cfg, const dbt_weights *w, void *kv_pool
         const char *pf = getenv("DBT_L2_PREFETCH");
         m->l2_prefetch = pf && strcmp(pf, "1") == 0;
     }
+    const char *ro = getenv("DBT_READOUT");
+    m->readout_row = ro && strcmp(ro, "row") == 0;
     const char *pd = getenv("DBT_PDL");
     m->use_pdl = !(pd && strcmp(pd, "0") == 0);
     const char *po = getenv("DBT_PDL_OFF");
@@ -1855,6 +1880,7 @@ dbt_status dbt_create(const dbt_config *cfg, const dbt_weights *w, void *kv_pool
     if (e == cudaSuccess) e = cudaMemsetAsync(m->ws.status, 0, sizeof(int32_t) * 4, m->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(m->ws.att_tickets, 0, sizeof(int32_t) * (size_t)m->Rmax * cfg->n_kv_heads, m->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(m->ws.att_tickets2, 0, sizeof(int32_t) * (size_t)m->Rmax * cfg->n_kv_heads * kAttMaxGroups, m->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(m->ws.ro_tickets, 0, sizeof(int32_t) * (size_t)cfg->max_batch, m->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(m->ws.gemm_tickets, 0, sizeof(int32_t) * 4096, m->stream);
     if (e == cudaSuccess && moe) {
         e = cudaMemsetAsync(m->ws.last_experts, 0xff, sizeof(int32_t) * (size_t)cfg->n_layers * 2 * cfg->max_batch * kmax_of(*cfg), m->stream);
@@ -1976,6 +2002,7 @@ dbt_status dbt_reset(dbt_model *m) {
     CUDA_TRY(m, cudaMemsetAsync(m->ws.att_tickets, 0, sizeof(int32_t) * (size_t)m->Rmax * m->cfg.n_kv_heads, m->stream));
     CUDA_TRY(m, cudaMemsetAsync(m->ws.att_tickets2, 0, sizeof(int32_t) * (size_t)m->Rmax * m->cfg.n_kv_heads * kAttMaxGroups, m->stream));
     CUDA_TRY(m, cudaMemsetAsync(m->ws.gemm_tickets, 0, sizeof(int32_t) * 4096, m->stream));
+    CUDA_TRY(m, cudaMemsetAsync(m->ws.ro_tickets, 0, sizeof(int32_t) * (size_t)m->cfg.max_batch, m->stream));
     if (m->ws.mega_sync) CUDA_TRY(m, cudaMemsetAsync(m->ws.mega_sync, 0, sizeof(unsigned int) * 8, m->stream));
     std::fill(m->len_host.begin(), m->len_host.end(), 0);
     return DBT_OK;

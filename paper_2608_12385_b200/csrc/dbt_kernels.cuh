@@ -454,6 +454,153 @@ __global__ void __launch_bounds__(1024) readout_kernel(const float *Z, int B, in
     }
 }
 
+// ---- the readout on many CTAs -----------------------------------------------------------------
+// readout_kernel walks a row three times with one CTA.  Here a row is cut into NC chunks of at most
+// kRoChunk logits, a CTA per (row, chunk), each logit staged in registers:
+//   readout_stats_kernel: per chunk (m1, sum e^(z1-m1), sum e^(2(z1-m1)), m2, sum e^(z2-m2)) with the
+//     chunk's own maxima;
+//   readout_pick_kernel: every CTA folds the row's NC records in chunk order into p, q's normalisers
+//     and alpha (Eq. alpha), evaluates alpha p + (1 - alpha) q (Eq. mixloss) over its chunk, and leaves
+//     its best (value, index); the last CTA of the row to arrive picks among the NC candidates
+//     (lowest index on ties), writes the token and alpha and advances the sequence length.
+// Primary-only steps skip the first kernel: the pick is the argmax of z1.
+constexpr int kRoChunk = 2048, kRoThreads = 256, kRoPer = kRoChunk / kRoThreads, kRoMaxChunks = 128;
+
+__global__ void __launch_bounds__(kRoThreads) readout_stats_kernel(const float *Z, int B, int V, int chunk, float *stats) {
+    pdl_enter();
+    __shared__ float scratch[32];
+    const int b = blockIdx.x, ck = blockIdx.y, tid = threadIdx.x;
+    const int v0 = ck * chunk, v1 = min(V, v0 + chunk);
+    const float *z1 = Z + (size_t)b * V, *z2 = Z + (size_t)(B + b) * V;
+    float a[kRoPer], c[kRoPer];
+    float m1 = -INFINITY, m2 = -INFINITY;
+#pragma unroll
+    for (int j = 0; j < kRoPer; j++) {
+        const int v = v0 + j * kRoThreads + tid;
+        a[j] = v < v1 ? __ldcg(z1 + v) : -INFINITY;
+        c[j] = v < v1 ? __ldcg(z2 + v) : -INFINITY;
+    }
+#pragma unroll
+    for (int j = 0; j < kRoPer; j++) {
+        m1 = fmaxf(m1, a[j]);
+        m2 = fmaxf(m2, c[j]);
+    }
+    m1 = block_max(m1, scratch);
+    m2 = block_max(m2, scratch);
+    float s1 = 0.f, q1 = 0.f, s2 = 0.f;
+#pragma unroll
+    for (int j = 0; j < kRoPer; j++) {
+        const float e1 = a[j] == -INFINITY ? 0.f : expf(a[j] - m1);
+        s1 += e1;
+        q1 += e1 * e1;
+        s2 += c[j] == -INFINITY ? 0.f : expf(c[j] - m2);
+    }
+    s1 = block_sum(s1, scratch);
+    q1 = block_sum(q1, scratch);
+    s2 = block_sum(s2, scratch);
+    if (tid == 0) {
+        float *o = stats + ((size_t)b * gridDim.y + ck) * 8;
+        o[0] = m1; o[1] = s1; o[2] = q1; o[3] = m2; o[4] = s2;
+    }
+}
+
+__global__ void __launch_bounds__(kRoThreads) readout_pick_kernel(const float *Z, int B, int V, int chunk, int grouped,
+                                                                  float *stats, int32_t *tickets, int32_t *next,
+                                                                  float *alpha_out, int32_t *seq_len, int advance) {
+    pdl_enter();
+    __shared__ float bv[32];
+    __shared__ int bi[32];
+    __shared__ float glob[6];
+    __shared__ int last_s;
+    const int b = blockIdx.x, ck = blockIdx.y, nc = gridDim.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int v0 = ck * chunk, v1 = min(V, v0 + chunk);
+    const float *z1 = Z + (size_t)b * V, *z2 = Z + (size_t)(B + b) * V;
+    float a[kRoPer], c[kRoPer];
+#pragma unroll
+    for (int j = 0; j < kRoPer; j++) {  // the chunk's logits, requested before the row's records are folded
+        const int v = v0 + j * kRoThreads + tid;
+        a[j] = v < v1 ? __ldcg(z1 + v) : -INFINITY;
+        c[j] = (grouped && v < v1) ? __ldcg(z2 + v) : -INFINITY;
+    }
+    if (grouped && warp == 0) {
+        // fold the row's records: maxima first, then the sums rescaled to them, in chunk order (lane 0)
+        const float *rec = stats + (size_t)b * nc * 8;
+        float m1 = -INFINITY, m2 = -INFINITY;
+        for (int k = lane; k < nc; k += 32) {
+            m1 = fmaxf(m1, __ldcg(rec + (size_t)k * 8));
+            m2 = fmaxf(m2, __ldcg(rec + (size_t)k * 8 + 3));
+        }
+        m1 = warp_max(m1);
+        m2 = warp_max(m2);
+        if (lane == 0) {
+            float d1 = 0.f, c1 = 0.f, d2 = 0.f;
+            for (int k = 0; k < nc; k++) {
+                const float f1 = expf(__ldcg(rec + (size_t)k * 8) - m1), f2 = expf(__ldcg(rec + (size_t)k * 8 + 3) - m2);
+                d1 += __ldcg(rec + (size_t)k * 8 + 1) * f1;
+                c1 += __ldcg(rec + (size_t)k * 8 + 2) * f1 * f1;
+                d2 += __ldcg(rec + (size_t)k * 8 + 4) * f2;
+            }
+            glob[0] = m1; glob[1] = d1; glob[2] = m2; glob[3] = d2;
+            glob[4] = fminf(1.f, fmaxf(0.5f, c1 / (d1 * d1)));
+        }
+    }
+    __syncthreads();
+    const float m1 = glob[0], d1 = glob[1], m2 = glob[2], d2 = glob[3], alpha = glob[4];
+    ArgBest best = {-INFINITY, 0x7fffffff};
+#pragma unroll
+    for (int j = 0; j < kRoPer; j++) {
+        const int v = v0 + j * kRoThreads + tid;
+        if (v < v1) {
+            float val = grouped ? alpha * (expf(a[j] - m1) / d1) + (1.f - alpha) * (expf(c[j] - m2) / d2) : a[j];
+            best = better(best, ArgBest{val, v});
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        ArgBest other = {__shfl_xor_sync(0xffffffffu, best.v, o), __shfl_xor_sync(0xffffffffu, best.i, o)};
+        best = better(best, other);
+    }
+    if (lane == 0) {
+        bv[warp] = best.v;
+        bi[warp] = best.i;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        ArgBest t = lane < (kRoThreads >> 5) ? ArgBest{bv[lane], bi[lane]} : ArgBest{-INFINITY, 0x7fffffff};
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            ArgBest other = {__shfl_xor_sync(0xffffffffu, t.v, o), __shfl_xor_sync(0xffffffffu, t.i, o)};
+            t = better(t, other);
+        }
+        if (lane == 0) {
+            float *o2 = stats + ((size_t)b * nc + ck) * 8;
+            o2[5] = t.v;
+            o2[6] = __int_as_float(t.i);
+            __threadfence();
+            const int tk = atomicAdd(tickets + b, 1);
+            last_s = tk == nc - 1;
+            if (last_s) atomicExch(tickets + b, 0);
+        }
+    }
+    __syncthreads();
+    if (last_s && warp == 0) {
+        __threadfence();
+        const float *rec = stats + (size_t)b * nc * 8;
+        ArgBest t = {-INFINITY, 0x7fffffff};
+        for (int k = lane; k < nc; k += 32) t = better(t, ArgBest{__ldcg(rec + (size_t)k * 8 + 5), __float_as_int(__ldcg(rec + (size_t)k * 8 + 6))});
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            ArgBest other = {__shfl_xor_sync(0xffffffffu, t.v, o), __shfl_xor_sync(0xffffffffu, t.i, o)};
+            t = better(t, other);
+        }
+        if (lane == 0) {
+            if (next) next[b] = t.i;
+            if (alpha_out && grouped) alpha_out[b] = alpha;
+            if (seq_len) seq_len[b] += advance;  // the step's last use of the lengths was the last layer's attention
+        }
+    }
+}
+
 __global__ void advance_len_kernel(int32_t *seq_len, int B, int n) {
     pdl_enter();
     int b = blockIdx.x * blockDim.x + threadIdx.x;

@@ -440,7 +440,7 @@ def test_fresh_models_give_bitwise_identical_results():
             assert torch.equal(x["z1"], y["z1"]) and torch.equal(x["z2"], y["z2"])
 
 
-@pytest.mark.parametrize("knob,value", [("DBT_FUSED", "1"), ("DBT_WIDE", "0"), ("DBT_MEGA", "1"), ("DBT_L2_PREFETCH", "1"),
+@pytest.mark.parametrize("knob,value", [("DBT_READOUT", "row"), ("DBT_FUSED", "1"), ("DBT_WIDE", "0"), ("DBT_MEGA", "1"), ("DBT_L2_PREFETCH", "1"),
                                         ("DBT_CLUSTER", "1"), ("DBT_CLUSTER_GU", "1"), ("DBT_FUSE_QKV", "0"), ("DBT_STACK", "0"), ("DBT_EVICT_FIRST", "0")])
 def test_alternative_kernel_chains_match_oracle(monkeypatch, knob, value):
     """The variants of the dense chain that are not the default -- elementwise work folded into the
