@@ -81,3 +81,54 @@ def test_null_handle_calls_do_not_crash(lib):
     assert lib.dbt_seq_len(None, 0) == -1
     assert lib.dbt_launch_count(None) == 0
     lib.dbt_destroy(None)
+
+
+def _c_layout(header: str, structs: dict) -> dict:
+    """sizeof and field offsets as the C compiler sees them (gcc on the header itself)."""
+    import subprocess
+    import tempfile
+    lines = [f'#include "{header}"', "#include <stdio.h>", "#include <stddef.h>", "int main(void) {"]
+    for sname, fields in structs.items():
+        lines.append(f'printf("{sname} %zu\\n", sizeof({sname}));')
+        for f in fields:
+            lines.append(f'printf("{sname}.{f} %zu\\n", offsetof({sname}, {f}));')
+    lines += ["return 0;", "}"]
+    with tempfile.TemporaryDirectory() as td:
+        src, exe = os.path.join(td, "layout.c"), os.path.join(td, "layout")
+        open(src, "w").write("\n".join(lines))
+        subprocess.run(["gcc", "-I", os.path.dirname(header), "-o", exe, src], check=True)
+        out = subprocess.run([exe], check=True, capture_output=True, text=True).stdout
+    return {k: int(v) for k, v in (line.split() for line in out.splitlines())}
+
+
+def _ctypes_layout(name: str, struct) -> dict:
+    d = {name: C.sizeof(struct)}
+    for f, _ in struct._fields_:
+        d[f"{name}.{f}"] = getattr(struct, f).offset
+    return d
+
+
+def test_binding_structs_have_the_headers_layout():
+    """The ctypes mirrors of dbt_config / dbt_layer_weights / dbt_weights follow include/dbt.h field by field."""
+    pairs = {"dbt_config": binding.DbtConfig, "dbt_layer_weights": binding.DbtLayerWeights, "dbt_weights": binding.DbtWeights}
+    want = _c_layout(os.path.join(ROOT, "include", "dbt.h"), {n: [f for f, _ in s._fields_] for n, s in pairs.items()})
+    for n, s in pairs.items():
+        for k, v in _ctypes_layout(n, s).items():
+            assert want[k] == v, k
+
+
+def test_oracle_wrapper_structs_have_the_oracle_headers_layout():
+    import oracle
+    pairs = {"orc_config": oracle.OrcConfig, "orc_layer_weights": oracle.OrcLayer, "orc_weights": oracle.OrcWeights}
+    want = _c_layout(os.path.join(ROOT, "oracle", "dbt_oracle.h"), {n: [f for f, _ in s._fields_] for n, s in pairs.items()})
+    for n, s in pairs.items():
+        for k, v in _ctypes_layout(n, s).items():
+            assert want[k] == v, k
+
+
+def test_compute_matched_needs_an_moe_model(lib):
+    with pytest.raises(binding.DbtError) as e:
+        binding.query_sizes(dense_1b().replace(compute_matched=1), 1, 64, 8)
+    assert e.value.status == 2
+    kv, ws = binding.query_sizes(moe_1b().replace(compute_matched=1), 2, 64, 16)
+    assert kv > 0 and ws > 0
