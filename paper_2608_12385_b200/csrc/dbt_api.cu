@@ -128,6 +128,7 @@ struct dbt_model {
     cudaEvent_t ev_fork, ev_join;
     bool moe_overlap;
     bool readout_row;  // DBT_READOUT=row: the one-CTA-per-row readout kernel
+    int moe_row_tile;  // DBT_MOE_ROWTILE: row tile of the per-expert GEMMs (-1: chosen from the batch, 0: one tile of all rows)
     bool moe_wide;  // MoE chain with the RMSNorm factor applied behind the GEMMs (DBT_MOE_WIDE=0: row-wide norm kernels)
     std::vector<GraphEntry> graphs;
 };
@@ -576,6 +577,7 @@ struct TcCall {
     int lo_row0;  // row of the lo plane in the activation buffer
     const int *grp_cnt, *grp_off;  // per-expert mode (see TcParams); n_groups experts
     int grp_w_rows, n_groups;
+    int grp_row_tiles;  // per-expert mode: row tiles of n_tile rows per expert (0: one tile holds any list)
     const void *pf_ptr[3];  // L2 prefetch requests carried by this launch (the next GEMM's weights)
     size_t pf_bytes[3];
 };
@@ -658,6 +660,7 @@ dbt_status run_gemm_tc(dbt_model *m, const TcCall &c, int n_tile, int *nsplit_ou
     p.grp_cnt = c.grp_cnt;
     p.grp_off = c.grp_off;
     p.grp_w_rows = c.grp_w_rows;
+    p.grp_row_tiles = c.grp_cnt ? c.grp_row_tiles : 0;
     p.P = c.P;
     p.status = m->ws.status;
     p.evict_first = m->evict_first ? 1 : 0;
@@ -685,7 +688,7 @@ dbt_status run_gemm_tc(dbt_model *m, const TcCall &c, int n_tile, int *nsplit_ou
     }
     e.arrivals = (e.mode == FE_GATEUP ? 2 : 1) * split;
     if (e.mode != FE_NONE && tiles > 4096) return fail(m, DBT_ERR_UNSUPPORTED, "too many output tiles for %s", c.tag);
-    dim3 grid(tiles, split, c.grp_cnt ? c.n_groups : 1);
+    dim3 grid(tiles, c.grp_cnt && c.grp_row_tiles ? c.grp_row_tiles : split, c.grp_cnt ? c.n_groups : 1);
     m->next_cluster_y = e.cluster ? split : 0;
     m->next_cluster_x = e.cluster && e.mode == FE_GATEUP ? 2 : 1;
     if (nsplit_out) *nsplit_out = split;
@@ -844,14 +847,27 @@ dbt_status run_moe_tc(dbt_model *m, int l, const RowMap &rm, int grouped, bool r
     gu.nseg = 2; gu.X = &m->map_Xs; gu.K = d; gu.R = Rk; gu.P = w.Pe; gu.P_floats = (size_t)Rk * 2 * Fe;
     gu.tag = "expert_gateup"; gu.parts = m->act_parts; gu.lo_row0 = Rk;
     gu.grp_cnt = w.ecnt; gu.grp_off = w.eoff; gu.grp_w_rows = Fe; gu.n_groups = E;
-    if ((st = run_gemm_tc(m, gu, n_tile, nullptr, nullptr)) != DBT_OK) return st;
+    // An expert's list is short on average (rows x k / experts) but may hold every row: row tiles of
+    // 16 rows (32 from 64 sequences on; chosen from the batch, not the mode, so that grouped and
+    // primary-only steps use the same instruction shape), as many per expert as the rows of this step
+    // could need, keep two CTAs per SM and their deeper rings at large batches (measured: 4.86 -> 4.53 ms
+    // at batch 32, 6.43 -> 4.81 at batch 64).  DBT_MOE_ROWTILE=0: one tile of all rows; 16/32/64: that tile.
+    int gt = n_tile, grt = 0;
+    const int want_tile = m->moe_row_tile >= 0 ? m->moe_row_tile : (2 * Bc <= 64 ? 16 : 32);
+    if (want_tile > 0 && n_tile > want_tile) {
+        gt = want_tile;
+        grt = (R + gt - 1) / gt;
+    }
+    gu.grp_row_tiles = grt;
+    if ((st = run_gemm_tc(m, gu, gt, nullptr, nullptr)) != DBT_OK) return st;
     LAUNCH(m, "moe_swiglu", 0, moe_swiglu_kernel, dim3(R * km, (Fe + 255) / 256), 256, 0, w.Pe, w.eoff + E, Fe, w.Hs, lo_hs,
            wide ? (const float *)w.rs_sorted : (const float *)nullptr);
     TcCall dn{};
     dn.W[0] = &mp.ed; dn.n_out[0] = d; dn.rows[0] = Rk; dn.nseg = 1; dn.X = &m->map_Hs; dn.K = Fe; dn.R = Rk;
     dn.P = w.Yexp; dn.P_floats = (size_t)Rk * d; dn.tag = "expert_down"; dn.parts = m->act_parts; dn.lo_row0 = Rk;
     dn.grp_cnt = w.ecnt; dn.grp_off = w.eoff; dn.grp_w_rows = d; dn.n_groups = E;
-    if ((st = run_gemm_tc(m, dn, n_tile, nullptr, nullptr)) != DBT_OK) return st;
+    dn.grp_row_tiles = grt;
+    if ((st = run_gemm_tc(m, dn, gt, nullptr, nullptr)) != DBT_OK) return st;
     if (Fs > 0 && !overlap && (st = shared_expert(w.P, w.P_floats)) != DBT_OK) return st;
     if (overlap) CUDA_TRY(m, cudaStreamWaitEvent(main_stream, m->ev_join, 0));
     const bool next_in = wide && g_next != nullptr;
@@ -1840,6 +1856,9 @@ dbt_status dbt_create(const dbt_config *cfg, const dbt_weights *w, void *kv_pool
     {
         const char *ov = getenv("DBT_MOE_OVERLAP");
         m->moe_overlap = m->moe_tc && cfg->n_shared_experts > 0 && !(ov && strcmp(ov, "0") == 0);
+        const char *rt = getenv("DBT_MOE_ROWTILE");
+        m->moe_row_tile = rt ? atoi(rt) : -1;
+        if (m->moe_row_tile != 0 && m->moe_row_tile != 16 && m->moe_row_tile != 32 && m->moe_row_tile != 64) m->moe_row_tile = -1;
         const char *mw = getenv("DBT_MOE_WIDE");
         m->moe_wide = m->moe_tc && m->act_parts == 2 && !(mw && strcmp(mw, "0") == 0);
         if (m->moe_overlap &&

@@ -55,6 +55,9 @@ struct TcParams {
     // X and P starting at grp_off[e]; its weight rows start at e * grp_w_rows.  nullptr = off.
     const int *grp_cnt, *grp_off;
     int grp_w_rows;
+    // grouped mode with row tiles: blockIdx.y = which N_TILE rows of the expert's list (CTAs past the
+    // list's end leave at once); 0: the whole list fits one tile and blockIdx.y is the split as usual
+    int grp_row_tiles;
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -229,7 +232,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
 
     DBT_TL_DECL;
     int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    int tile = blockIdx.x, split = blockIdx.y;
+    int tile = blockIdx.x, split = p.grp_row_tiles ? 0 : blockIdx.y;
     // Clustered gate|up: CTAs (2j, y) and (2j + 1, y) hold gate tile j and up tile j, so that a cluster
     // of 2 x splits CTAs owns everything SwiGLU needs for 128 features.
     if (e.cluster && e.mode == FE_GATEUP) tile = (int)(blockIdx.x & 1) * p.seg[1].tile0 + (int)(blockIdx.x >> 1);
@@ -241,6 +244,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
         if (grp_n == 0) return;  // expert not selected by any row of either path: its weights are not read
         x_row0 = ld_mut(p.grp_off + blockIdx.z);
         w_row0 = blockIdx.z * p.grp_w_rows;
+        if (p.grp_row_tiles) {
+            const int r0 = (int)blockIdx.y * N_TILE;
+            if (r0 >= grp_n) return;  // the expert's rows end before this tile
+            x_row0 += r0;
+            grp_n -= r0;
+        }
     }
     int sg = 0;
     if (p.nseg > 1 && tile >= p.seg[1].tile0) sg = 1;

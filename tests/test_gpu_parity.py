@@ -173,6 +173,26 @@ def test_kv_cache_bit_identical_grouped_vs_primary_only(cfg):
     assert ka.float().abs().sum() > 0
 
 
+def test_moe_kv_cache_bit_identical_at_a_batch_with_row_tiled_expert_gemms():
+    """34 sequences: 68 stacked rows grouped, 34 primary-only; the per-expert GEMMs use the same row tile in
+    both modes, and the cache and the primary logits are the same bits."""
+    cfg = small_moe(k_primary=2, k_branch=2)
+    w = make_weights(cfg, seed=14, matrix_std=0.05)
+    B, T, npre = 34, 12, 8
+    tok = make_tokens(cfg, B, T, seed=15).cuda()
+    wd = binding.weights_to_device(w)
+    a = binding.Model(cfg, wd, B, T)
+    b = binding.Model(cfg, wd, B, T)
+    oa = _run_steps(a, tok, npre, True)
+    ob = _run_steps(b, tok, npre, False)
+    for x, y in zip(oa, ob):
+        assert torch.equal(x["z1"], y["z1"])
+    ka, va = a.read_kv(B, T)
+    kb, vb = b.read_kv(B, T)
+    assert torch.equal(ka.view(torch.int16), kb.view(torch.int16))
+    assert torch.equal(va.view(torch.int16), vb.view(torch.int16))
+
+
 def test_page_table_permutation_does_not_change_results():
     cfg = small_bf16(n_layers=2)
     w = make_weights(cfg, seed=14, matrix_std=0.05)
@@ -281,8 +301,12 @@ def test_moe_decode_matches_oracle_under_the_devices_routing(cfg):
     assert flips <= 2  # well-separated router logits: the free-running oracle picks the same experts
 
 
-def test_moe_at_batch_40():
-    """40 sequences: 80 stacked rows, a row tile of 128 in the per-expert GEMMs."""
+@pytest.mark.parametrize("rowtile", ["auto", "32", "16", "0"])
+def test_moe_at_batch_40(monkeypatch, rowtile):
+    """40 sequences: 80 stacked rows over 8 experts, so every expert's list is longer than a row tile of 16
+    or 32 and the per-expert GEMMs walk several row tiles per expert (0: one tile of 128 rows)."""
+    if rowtile != "auto":
+        monkeypatch.setenv("DBT_MOE_ROWTILE", rowtile)
     flips = _moe_compare(small_moe(k_primary=2, k_branch=2), B=40, T=7, npre=5)
     assert flips <= 6
 
