@@ -42,7 +42,7 @@ class OrcConfig(C.Structure):
     _fields_ += [("rope_base", C.c_float), ("rms_eps", C.c_float)]
     _fields_ += [(n, C.c_int32) for n in ("final_norm", "n_experts", "d_expert", "n_shared_experts",
                                          "k_primary", "k_branch", "router_mode", "moe_b_coupling",
-                                         "compute_matched", "max_batch", "max_seq")]
+                                         "compute_matched", "n_paths", "max_batch", "max_seq")]
 
 
 _LAYER_FIELDS = ("attn_norm_g", "wq", "wk", "wv", "wo", "coup_a", "mlp_norm_g", "w_gate", "w_up", "w_down",
@@ -75,6 +75,8 @@ def lib():
         L.orc_v_cache.argtypes = [vp]
         L.orc_v_cache.restype = vp
         L.orc_set_seq_len.argtypes = [vp, C.c_int, C.c_int]
+        L.orc_router_logits.argtypes = [vp]
+        L.orc_router_logits.restype = vp
         L.orc_prefill.argtypes = [vp, vp, C.c_int, C.c_int, vp]
         L.orc_decode_step.argtypes = [vp, vp, C.c_int, C.c_int, vp, vp, vp, vp, vp, vp, vp]
         L.orc_full_forward.argtypes = [C.POINTER(OrcConfig), C.POINTER(OrcWeights), vp, C.c_int, C.c_int,
@@ -87,6 +89,8 @@ def lib():
         L.orc_route.argtypes = [vp, C.c_int, C.c_int, vp, vp, vp]
         L.orc_readout.argtypes = [vp, vp, C.c_int, vp, vp]
         L.orc_readout.restype = C.c_int
+        L.orc_readout_multi.argtypes = [vp, vp, C.c_int, C.c_int, vp, vp]
+        L.orc_readout_multi.restype = C.c_int
         L.orc_set_threads.argtypes = [C.c_int]
         L.orc_get_threads.restype = C.c_int
         _lib = L
@@ -111,7 +115,7 @@ def _cfg_struct(cfg, max_batch: int, max_seq: int, kv_round_bf16: bool = False) 
                      n_experts=cfg.n_experts, d_expert=cfg.d_expert, n_shared_experts=cfg.n_shared_experts,
                      k_primary=cfg.k_primary, k_branch=cfg.k_branch, router_mode=cfg.router_mode,
                      moe_b_coupling=cfg.moe_b_coupling, compute_matched=cfg.compute_matched,
-                     max_batch=max_batch, max_seq=max_seq)
+                     n_paths=getattr(cfg, "n_paths", 2), max_batch=max_batch, max_seq=max_seq)
 
 
 def _weights_struct(cfg, w: dict):
@@ -126,6 +130,8 @@ def _weights_struct(cfg, w: dict):
             setattr(layers[l], name, _ptr(t))
     for name in ("embed_primary", "embed_branch", "lm_head"):
         assert w[name].dtype == want, name
+    nb = getattr(cfg, "n_paths", 2) - 1  # one embedding table per decode branch, stacked [K-1][V][d]
+    assert w["embed_branch"].numel() == nb * cfg.vocab * cfg.d_model, "embed_branch must hold K-1 tables"
     ws = OrcWeights(embed_primary=_ptr(w["embed_primary"]), embed_branch=_ptr(w["embed_branch"]),
                     embed_norm_g=_ptr(w["embed_norm_g"]), final_norm_g=_ptr(w["final_norm_g"]),
                     lm_head=_ptr(w["lm_head"]), layers=layers)
@@ -185,6 +191,16 @@ class OracleModel:
         for b in range(B):
             lib().orc_set_seq_len(self._h, b, length)
 
+    def router_logits(self, batch: int) -> np.ndarray:
+        """MoE: router logits of the last step, [L, K, batch, E] (a copy)."""
+        p = lib().orc_router_logits(self._h)
+        assert p, "not an MoE model"
+        K = getattr(self.cfg, "n_paths", 2)
+        shape = (self.cfg.n_layers, K, self.max_batch, self.cfg.n_experts)
+        n = int(np.prod(shape))
+        a = np.ctypeslib.as_array(C.cast(p, C.POINTER(C.c_float)), shape=(n,)).reshape(shape)
+        return a[:, :, :batch].copy()
+
     def prefill(self, tokens, want_logits: bool = True):
         tok = np.ascontiguousarray(np.asarray(tokens, dtype=np.int32))
         B, n = tok.shape
@@ -197,18 +213,19 @@ class OracleModel:
     def decode_step(self, tokens, grouped: bool = True, forced_experts=None, want_mix: bool = False):
         tok = np.ascontiguousarray(np.asarray(tokens, dtype=np.int32).reshape(-1))
         B, V, cfg = tok.shape[0], self.cfg.vocab, self.cfg
+        K = getattr(cfg, "n_paths", 2)
         out = {"next": np.empty(B, dtype=np.int32), "z1": np.empty((B, V), dtype=np.float32)}
-        if grouped:
-            out["z2"] = np.empty((B, V), dtype=np.float32)
+        if grouped:  # one decode branch: z2 [B, V]; more (Appendix C.1): [K-1, B, V]
+            out["z2"] = np.empty((B, V) if K == 2 else (K - 1, B, V), dtype=np.float32)
             out["alpha"] = np.empty(B, dtype=np.float32)
             if want_mix:
                 out["mix"] = np.empty((B, V), dtype=np.float32)
         if cfg.is_moe:
-            out["experts"] = np.full((cfg.n_layers, 2, B, cfg.kmax), -1, dtype=np.int32)
+            out["experts"] = np.full((cfg.n_layers, K, B, cfg.kmax), -1, dtype=np.int32)
         forced = None
         if forced_experts is not None:
             forced = np.ascontiguousarray(np.asarray(forced_experts, dtype=np.int32))
-            assert forced.shape == (cfg.n_layers, 2, B, cfg.kmax)
+            assert forced.shape == (cfg.n_layers, K, B, cfg.kmax)
         rc = lib().orc_decode_step(self._h, _ptr(tok), B, int(grouped), _ptr(forced), _ptr(out.get("experts")),
                                    _ptr(out["next"]), _ptr(out["z1"]), _ptr(out.get("z2")),
                                    _ptr(out.get("alpha")), _ptr(out.get("mix")))
@@ -218,13 +235,15 @@ class OracleModel:
 
 
 def full_forward(cfg, weights: dict, tokens, want_kv: bool = False):
-    """Non-incremental two-path forward: returns z1, z2 [B,T,V] (and K,V [L,B,T,kv_dim])."""
+    """Non-incremental forward of every path: returns z1 [B,T,V], z2 [B,T,V] (one decode branch)
+    or [K-1,B,T,V] (more), and K,V [L,B,T,kv_dim] on request."""
     tok = np.ascontiguousarray(np.asarray(tokens, dtype=np.int32))
     B, T = tok.shape
     c = _cfg_struct(cfg, B, T)
     ws, layers = _weights_struct(cfg, weights)
+    K = getattr(cfg, "n_paths", 2)
     z1 = np.empty((B, T, cfg.vocab), dtype=np.float32)
-    z2 = np.empty((B, T, cfg.vocab), dtype=np.float32)
+    z2 = np.empty((B, T, cfg.vocab) if K == 2 else (K - 1, B, T, cfg.vocab), dtype=np.float32)
     k = np.empty((cfg.n_layers, B, T, cfg.kv_dim), dtype=np.float32) if want_kv else None
     v = np.empty((cfg.n_layers, B, T, cfg.kv_dim), dtype=np.float32) if want_kv else None
     rc = lib().orc_full_forward(C.byref(c), C.byref(ws), _ptr(tok), B, T, _ptr(z1), _ptr(z2), _ptr(k), _ptr(v))
@@ -292,6 +311,15 @@ def readout(z1, z2, want_mix=True):
     alpha = np.empty(1, dtype=np.float32)
     mix = np.empty_like(z1) if want_mix else None
     tok = lib().orc_readout(_ptr(z1), _ptr(z2), z1.shape[0], _ptr(alpha), _ptr(mix))
+    return tok, float(alpha[0]), mix
+
+
+def readout_multi(z1, zb, want_mix=True):
+    """zb [nb, V]: the logits of nb decode branches (Appendix C.1)."""
+    z1, zb = _f32(z1), _f32(zb)
+    alpha = np.empty(1, dtype=np.float32)
+    mix = np.empty_like(z1) if want_mix else None
+    tok = lib().orc_readout_multi(_ptr(z1), _ptr(zb), zb.shape[0], z1.shape[0], _ptr(alpha), _ptr(mix))
     return tok, float(alpha[0]), mix
 
 

@@ -8,7 +8,9 @@
  * Notation follows the paper: S_1/S_2 primary and branch residual states, N_i normalised
  * states, Q_1,K_1,V_1 primary projections, Q_2 and Q~_2 the branch query before and after
  * the a coupling, H_i the activated MLP intermediate, M_i the MLP output, z_1/z_2 logits,
- * p/q their softmaxes.  Stacked rows are path-major: rows 0..n-1 primary, n..2n-1 branch.
+ * p/q their softmaxes.  Stacked rows are path-major: rows 0..n-1 primary, then n rows per
+ * decode branch (one branch in the main text; K-1 of them in Appendix C.1, "More decode
+ * branches": own embedding each, shared coupling vectors, branch distributions averaged).
  */
 #include "dbt_oracle.h"
 
@@ -25,7 +27,10 @@ struct orc_model {
     orc_layer_weights *layers; /* owned copy of the per-layer pointer table */
     float *kc, *vc;            /* [L][max_batch][max_seq][kv_dim]           */
     int32_t *len;              /* [max_batch] tokens already cached         */
+    float *rlog;               /* MoE: router logits of the last step, [L][K][max_batch][E] */
 };
+
+static inline int paths_of(const orc_config *c) { return c->n_paths >= 2 ? c->n_paths : 2; }
 
 /* ------------------------------------------------------------------------------------ */
 /* storage helpers                                                                       */
@@ -177,17 +182,24 @@ void orc_route(const float *logits, int E, int k, const int32_t *forced, int32_t
     free(p);
 }
 
-/* p = softmax(z1), q = softmax(z2), alpha = clip_[0.5,1](sum_v p_v^2),
- * mix = alpha p + (1-alpha) q, greedy token = argmax mix (lowest index on ties). */
-int orc_readout(const float *z1, const float *z2, int V, float *alpha, float *mix) {
-    double m1 = -INFINITY, m2 = -INFINITY, d1 = 0.0, d2 = 0.0;
-    for (int v = 0; v < V; v++) {
+/* p = softmax(z1), q_j = softmax(zb_j) for the nb decode branches, qbar = mean_j q_j
+ * (Appendix C.1; nb = 1 is the main text's single q), alpha = clip_[0.5,1](sum_v p_v^2),
+ * mix = alpha p + (1-alpha) qbar, greedy token = argmax mix (lowest index on ties).
+ * zb is [nb][V]. */
+int orc_readout_multi(const float *z1, const float *zb, int nb, int V, float *alpha, float *mix) {
+    double m1 = -INFINITY, d1 = 0.0;
+    double *mb = (double *)malloc(sizeof(double) * (size_t)nb);
+    double *db = (double *)malloc(sizeof(double) * (size_t)nb);
+    for (int v = 0; v < V; v++)
         if ((double)z1[v] > m1) m1 = z1[v];
-        if ((double)z2[v] > m2) m2 = z2[v];
-    }
-    for (int v = 0; v < V; v++) {
-        d1 += exp((double)z1[v] - m1);
-        d2 += exp((double)z2[v] - m2);
+    for (int v = 0; v < V; v++) d1 += exp((double)z1[v] - m1);
+    for (int j = 0; j < nb; j++) {
+        const float *z = zb + (size_t)j * V;
+        mb[j] = -INFINITY;
+        db[j] = 0.0;
+        for (int v = 0; v < V; v++)
+            if ((double)z[v] > mb[j]) mb[j] = z[v];
+        for (int v = 0; v < V; v++) db[j] += exp((double)z[v] - mb[j]);
     }
     double coll = 0.0;
     for (int v = 0; v < V; v++) {
@@ -201,8 +213,10 @@ int orc_readout(const float *z1, const float *z2, int V, float *alpha, float *mi
     double bestv = -1.0;
     for (int v = 0; v < V; v++) {
         double p = exp((double)z1[v] - m1) / d1;
-        double q = exp((double)z2[v] - m2) / d2;
-        double mv = a * p + (1.0 - a) * q;
+        double qbar = 0.0;
+        for (int j = 0; j < nb; j++) qbar += exp((double)zb[(size_t)j * V + v] - mb[j]) / db[j];
+        qbar /= (double)nb;
+        double mv = a * p + (1.0 - a) * qbar;
         if (mix) mix[v] = (float)mv;
         if (mv > bestv) {
             bestv = mv;
@@ -210,7 +224,13 @@ int orc_readout(const float *z1, const float *z2, int V, float *alpha, float *mi
         }
     }
     if (alpha) *alpha = (float)a;
+    free(mb); free(db);
     return best;
+}
+
+/* The main text's two-path readout (Eq. alpha, Eq. mixloss): one decode branch. */
+int orc_readout(const float *z1, const float *z2, int V, float *alpha, float *mix) {
+    return orc_readout_multi(z1, z2, 1, V, alpha, mix);
 }
 
 static int argmax_f32(const float *z, int n) {
@@ -236,49 +256,51 @@ int orc_get_threads(void) {
 }
 
 /* ------------------------------------------------------------------------------------ */
-/* MLP sub-layers on n primary rows (m1) and, when m2 != NULL, n branch rows (m2)        */
+/* MLP sub-layers on `paths` stacked groups of n rows: m = [N_1; N_2; ...] (group 0 primary) */
 
-/* Eq. mlp: M_1 = H_1 W_D ; H~_2 = H_2 + b*H_1 ; M_2 = H~_2 W_D + c*M_1 */
-static void mlp_dense(const orc_config *c, const orc_layer_weights *lw, const float *m1,
-                      const float *m2, int n, float *M1, float *M2) {
+/* Eq. mlp: M_1 = H_1 W_D ; H~_j = H_j + b*H_1 ; M_j = H~_j W_D + c*M_1 for every branch j
+ * (b, c shared by the branches: Appendix C.1). */
+static void mlp_dense(const orc_config *c, const orc_layer_weights *lw, const float *m, int paths,
+                      int n, float *M) {
     int d = c->d_model, F = c->d_ff, dt = c->weight_dtype;
-    int paths = m2 ? 2 : 1;
     float *g = (float *)malloc(sizeof(float) * (size_t)n * F);
     float *u = (float *)malloc(sizeof(float) * (size_t)n * F);
     float *H1 = (float *)malloc(sizeof(float) * (size_t)n * F);
-    float *H2 = (float *)malloc(sizeof(float) * (size_t)n * F);
-    for (int p = 0; p < paths; p++) {
-        const float *m = p ? m2 : m1;
-        float *H = p ? H2 : H1;
-        orc_linear(lw->w_gate, dt, F, d, m, n, g);
-        orc_linear(lw->w_up, dt, F, d, m, n, u);
-        orc_swiglu(g, u, n * F, H);
-    }
-    orc_linear(lw->w_down, dt, d, F, H1, n, M1);
-    if (m2) {
+    float *Hj = (float *)malloc(sizeof(float) * (size_t)n * F);
+    orc_linear(lw->w_gate, dt, F, d, m, n, g);
+    orc_linear(lw->w_up, dt, F, d, m, n, u);
+    orc_swiglu(g, u, n * F, H1);
+    orc_linear(lw->w_down, dt, d, F, H1, n, M);
+    for (int p = 1; p < paths; p++) {
+        const float *mj = m + (size_t)p * n * d;
+        float *Mj = M + (size_t)p * n * d;
+        orc_linear(lw->w_gate, dt, F, d, mj, n, g);
+        orc_linear(lw->w_up, dt, F, d, mj, n, u);
+        orc_swiglu(g, u, n * F, Hj);
         for (int r = 0; r < n; r++)
             for (int i = 0; i < F; i++)
-                H2[(size_t)r * F + i] += lw->coup_b[i] * H1[(size_t)r * F + i];
-        orc_linear(lw->w_down, dt, d, F, H2, n, M2);
+                Hj[(size_t)r * F + i] += lw->coup_b[i] * H1[(size_t)r * F + i];
+        orc_linear(lw->w_down, dt, d, F, Hj, n, Mj);
         for (int r = 0; r < n; r++)
             for (int i = 0; i < d; i++)
-                M2[(size_t)r * d + i] += lw->coup_c[i] * M1[(size_t)r * d + i];
+                Mj[(size_t)r * d + i] += lw->coup_c[i] * M[(size_t)r * d + i];
     }
-    free(g); free(u); free(H1); free(H2);
+    free(g); free(u); free(H1); free(Hj);
 }
 
 /* Eq. moe_layer with per-path fan-out (Eq. moe_budget), un-gated shared experts
  * (M_i = R_i + G(N_i), Appendix B.3) and the c coupling on the total primary output.
  * Compute-matched allocation (Appendix B.3, Eq. matched_shared_expert): the shared expert
- * is evaluated on the primary state only, M_2 = R_2(N_2;k_2) + g_G * G(N_1), no b, no c.
- * forced / chosen: [2][n][kmax] slices for this layer (nullable). */
-static void mlp_moe(const orc_config *c, const orc_layer_weights *lw, const float *m1,
-                    const float *m2, int n, const int32_t *forced, int32_t *chosen, float *M1,
-                    float *M2) {
+ * is evaluated on the primary state only, M_j = R_j(N_j;k_2) + g_G * G(N_1), no b, no c.
+ * Every decode branch routes for itself with fan-out k_2 (router replay: with the primary's
+ * expert set).  forced / chosen: [paths][n][kmax] slices for this layer (nullable);
+ * logits_out: [paths][ld_logits][E] router logits of this layer (nullable). */
+static void mlp_moe(const orc_config *c, const orc_layer_weights *lw, const float *m, int paths,
+                    int n, const int32_t *forced, int32_t *chosen, float *logits_out, int ld_logits,
+                    float *Mout) {
     int d = c->d_model, E = c->n_experts, Fe = c->d_expert, dt = c->weight_dtype;
     int Fs = c->n_shared_experts * Fe;
     int kmax = c->k_primary > c->k_branch ? c->k_primary : c->k_branch;
-    int paths = m2 ? 2 : 1;
     float *logits = (float *)malloc(sizeof(float) * (size_t)E);
     float *g = (float *)malloc(sizeof(float) * (size_t)(Fe > Fs ? Fe : Fs));
     float *u = (float *)malloc(sizeof(float) * (size_t)(Fe > Fs ? Fe : Fs));
@@ -291,15 +313,17 @@ static void mlp_moe(const orc_config *c, const orc_layer_weights *lw, const floa
     int32_t idx[64];
     float wts[64];
     int32_t *idx1 = (int32_t *)malloc(sizeof(int32_t) * (size_t)n * kmax);
+    const float *M1 = Mout;
 
     for (int p = 0; p < paths; p++) {
         for (int r = 0; r < n; r++) {
-            const float *m = (p ? m2 : m1) + (size_t)r * d;
-            float *M = (p ? M2 : M1) + (size_t)r * d;
+            const float *mr = m + ((size_t)p * n + r) * d;
+            float *M = Mout + ((size_t)p * n + r) * d;
             int k = p ? c->k_branch : c->k_primary;
             const int32_t *f = forced ? forced + ((size_t)p * n + r) * kmax : NULL;
-            orc_linear(lw->router, dt, E, d, m, 1, logits);
-            if (p == 1 && c->router_mode == 1) { /* router replay: I_2 := I_1, own weights */
+            orc_linear(lw->router, dt, E, d, mr, 1, logits);
+            if (logits_out) memcpy(logits_out + ((size_t)p * ld_logits + r) * E, logits, sizeof(float) * (size_t)E);
+            if (p >= 1 && c->router_mode == 1) { /* router replay: I_j := I_1, own weights */
                 k = c->k_primary;
                 f = idx1 + (size_t)r * kmax;
             }
@@ -312,26 +336,26 @@ static void mlp_moe(const orc_config *c, const orc_layer_weights *lw, const floa
             for (int i = 0; i < d; i++) acc[i] = 0.0;
             for (int j = 0; j < k; j++) { /* routed experts, weighted */
                 size_t e = (size_t)idx[j];
-                orc_linear(mat_offset(lw->exp_gate, dt, e * Fe * d), dt, Fe, d, m, 1, g);
-                orc_linear(mat_offset(lw->exp_up, dt, e * Fe * d), dt, Fe, d, m, 1, u);
+                orc_linear(mat_offset(lw->exp_gate, dt, e * Fe * d), dt, Fe, d, mr, 1, g);
+                orc_linear(mat_offset(lw->exp_up, dt, e * Fe * d), dt, Fe, d, mr, 1, u);
                 orc_swiglu(g, u, Fe, h);
                 orc_linear(mat_offset(lw->exp_down, dt, e * (size_t)d * Fe), dt, d, Fe, h, 1, y);
                 for (int i = 0; i < d; i++) acc[i] += (double)wts[j] * (double)y[i];
             }
-            if (p == 1 && matched) { /* the branch receives the gated primary shared-expert output */
+            if (p >= 1 && matched) { /* the branch receives the gated primary shared-expert output */
                 for (int i = 0; i < d; i++) acc[i] += (double)lw->gate_g[i] * (double)G1[(size_t)r * d + i];
             } else if (Fs > 0) { /* shared expert(s): every token, weight one */
-                orc_linear(lw->sh_gate, dt, Fs, d, m, 1, g);
-                orc_linear(lw->sh_up, dt, Fs, d, m, 1, u);
+                orc_linear(lw->sh_gate, dt, Fs, d, mr, 1, g);
+                orc_linear(lw->sh_up, dt, Fs, d, mr, 1, u);
                 orc_swiglu(g, u, Fs, h);
                 if (p == 0) memcpy(Hs1 + (size_t)r * Fs, h, sizeof(float) * (size_t)Fs);
-                if (p == 1 && c->moe_b_coupling)
+                if (p >= 1 && c->moe_b_coupling)
                     for (int i = 0; i < Fs; i++) h[i] += lw->coup_b[i] * Hs1[(size_t)r * Fs + i];
                 orc_linear(lw->sh_down, dt, d, Fs, h, 1, y);
                 if (p == 0) memcpy(G1 + (size_t)r * d, y, sizeof(float) * (size_t)d);
                 for (int i = 0; i < d; i++) acc[i] += (double)y[i];
             }
-            if (p == 1 && !matched)
+            if (p >= 1 && !matched)
                 for (int i = 0; i < d; i++) acc[i] += (double)lw->coup_c[i] * (double)M1[(size_t)r * d + i];
             for (int i = 0; i < d; i++) M[i] = (float)acc[i];
         }
@@ -339,13 +363,12 @@ static void mlp_moe(const orc_config *c, const orc_layer_weights *lw, const floa
     free(logits); free(g); free(u); free(h); free(y); free(acc); free(Hs1); free(G1); free(idx1);
 }
 
-static void mlp_any(const orc_config *c, const orc_layer_weights *lw, const float *m1,
-                    const float *m2, int n, const int32_t *forced, int32_t *chosen, float *M1,
-                    float *M2) {
+static void mlp_any(const orc_config *c, const orc_layer_weights *lw, const float *m, int paths, int n,
+                    const int32_t *forced, int32_t *chosen, float *logits_out, int ld_logits, float *M) {
     if (c->n_experts > 0)
-        mlp_moe(c, lw, m1, m2, n, forced, chosen, M1, M2);
+        mlp_moe(c, lw, m, paths, n, forced, chosen, logits_out, ld_logits, M);
     else
-        mlp_dense(c, lw, m1, m2, n, M1, M2);
+        mlp_dense(c, lw, m, paths, n, M);
 }
 
 /* ------------------------------------------------------------------------------------ */
@@ -356,6 +379,7 @@ static int config_ok(const orc_config *c) {
     if (c->head_dim <= 0 || (c->head_dim & 1) || c->vocab <= 0) return 0;
     if (c->n_q_heads % c->n_kv_heads) return 0;
     if (c->weight_dtype != 0 && c->weight_dtype != 1) return 0;
+    if (c->n_paths != 0 && (c->n_paths < 2 || c->n_paths > 16)) return 0;
     if (c->n_experts > 0) {
         if (c->d_expert <= 0 || c->k_primary <= 0 || c->k_branch <= 0) return 0;
         if (c->k_primary > c->n_experts || c->k_branch > c->n_experts) return 0;
@@ -378,7 +402,9 @@ orc_model *orc_create(const orc_config *cfg, const orc_weights *w) {
     m->kc = (float *)calloc(n, sizeof(float));
     m->vc = (float *)calloc(n, sizeof(float));
     m->len = (int32_t *)calloc((size_t)cfg->max_batch, sizeof(int32_t));
-    if (!m->kc || !m->vc) {
+    if (cfg->n_experts > 0)
+        m->rlog = (float *)calloc((size_t)cfg->n_layers * paths_of(cfg) * cfg->max_batch * cfg->n_experts, sizeof(float));
+    if (!m->kc || !m->vc || (cfg->n_experts > 0 && !m->rlog)) {
         orc_destroy(m);
         return NULL;
     }
@@ -387,13 +413,14 @@ orc_model *orc_create(const orc_config *cfg, const orc_weights *w) {
 
 void orc_destroy(orc_model *m) {
     if (!m) return;
-    free(m->layers); free(m->kc); free(m->vc); free(m->len); free(m);
+    free(m->layers); free(m->kc); free(m->vc); free(m->len); free(m->rlog); free(m);
 }
 void orc_reset(orc_model *m) { memset(m->len, 0, sizeof(int32_t) * (size_t)m->cfg.max_batch); }
 int orc_seq_len(const orc_model *m, int b) { return m->len[b]; }
 float *orc_k_cache(orc_model *m) { return m->kc; }
 float *orc_v_cache(orc_model *m) { return m->vc; }
 void orc_set_seq_len(orc_model *m, int b, int len) { m->len[b] = len; }
+const float *orc_router_logits(const orc_model *m) { return m->rlog; }
 
 static size_t cache_index(const orc_config *c, int l, int b, int t) {
     return (((size_t)l * c->max_batch + b) * c->max_seq + t) * kv_dim_of(c);
@@ -409,9 +436,11 @@ static int step(orc_model *m, const int32_t *tokens, int B, int grouped, int wan
     int d = c->d_model, dh = c->head_dim, nq = c->n_q_heads, nkv = c->n_kv_heads, V = c->vocab;
     int G = nq / nkv, dt = c->weight_dtype;
     size_t qd = q_dim_of(c), kvd = kv_dim_of(c);
-    int R = grouped ? 2 * B : B;
+    int K = paths_of(c);            /* residual paths: the primary and K-1 decode branches */
+    int P = grouped ? K : 1;        /* paths evaluated in this step                        */
+    int R = P * B;
     /* rows that evaluate attention: the compute-matched branch has none (Eq. matched_attention) */
-    int Ra = (grouped && !c->compute_matched) ? 2 * B : B;
+    int Pa = (grouped && !c->compute_matched) ? K : 1, Ra = Pa * B;
     int kmax = c->k_primary > c->k_branch ? c->k_primary : c->k_branch;
     if (B <= 0 || B > c->max_batch) return -1;
     for (int b = 0; b < B; b++) {
@@ -429,13 +458,14 @@ static int step(orc_model *m, const int32_t *tokens, int B, int grouped, int wan
     float *M = (float *)malloc(sizeof(float) * (size_t)R * d);
     float *row = (float *)malloc(sizeof(float) * (size_t)d);
 
-    /* Eq. embeddings: S_1^0 = RMSNorm(E_1[x]), S_2^0 = RMSNorm(E_2[x]) */
+    /* Eq. embeddings: S_1^0 = RMSNorm(E_1[x]), S_j^0 = RMSNorm(E_j[x]); every decode branch has
+     * its own table (Appendix C.1), stored one after another in embed_branch */
     for (int b = 0; b < B; b++) {
         fetch_row(m->w.embed_primary, dt, (size_t)tokens[b], d, row);
         orc_rmsnorm(row, m->w.embed_norm_g, d, c->rms_eps, S + (size_t)b * d);
-        if (grouped) {
-            fetch_row(m->w.embed_branch, dt, (size_t)tokens[b], d, row);
-            orc_rmsnorm(row, m->w.embed_norm_g, d, c->rms_eps, S + (size_t)(B + b) * d);
+        for (int j = 1; j < P; j++) {
+            fetch_row(m->w.embed_branch, dt, (size_t)(j - 1) * V + (size_t)tokens[b], d, row);
+            orc_rmsnorm(row, m->w.embed_norm_g, d, c->rms_eps, S + ((size_t)j * B + b) * d);
         }
     }
 
@@ -444,18 +474,18 @@ static int step(orc_model *m, const int32_t *tokens, int B, int grouped, int wan
         /* N_i = RMSNorm(S_i) */
         for (int r = 0; r < R; r++)
             orc_rmsnorm(S + (size_t)r * d, lw->attn_norm_g, d, c->rms_eps, N + (size_t)r * d);
-        /* Q_i = RoPE(N_i W_Q) for both paths; K_1 = RoPE(N_1 W_K), V_1 = N_1 W_V: primary only */
+        /* Q_i = RoPE(N_i W_Q) for all paths; K_1 = RoPE(N_1 W_K), V_1 = N_1 W_V: primary only */
         orc_linear(lw->wq, dt, (int)qd, d, N, Ra, Q);
         orc_linear(lw->wk, dt, (int)kvd, d, N, B, Kn);
         orc_linear(lw->wv, dt, (int)kvd, d, N, B, Vn);
         for (int r = 0; r < Ra; r++) orc_rope(Q + (size_t)r * qd, nq, dh, m->len[r % B], c->rope_base);
         for (int b = 0; b < B; b++) orc_rope(Kn + (size_t)b * kvd, nkv, dh, m->len[b], c->rope_base);
-        /* Q~_2 = Q_2 + a * Q_1 */
-        if (Ra == 2 * B)
+        /* Q~_j = Q_j + a * Q_1 (the same a for every branch) */
+        for (int j = 1; j < Pa; j++)
             for (int b = 0; b < B; b++)
                 for (size_t i = 0; i < qd; i++)
-                    Q[(size_t)(B + b) * qd + i] += lw->coup_a[i] * Q[(size_t)b * qd + i];
-        /* the primary path appends its key and value; the branch has none */
+                    Q[((size_t)j * B + b) * qd + i] += lw->coup_a[i] * Q[(size_t)b * qd + i];
+        /* the primary path appends its key and value; the branches have none */
         for (int b = 0; b < B; b++) {
             float *kd = m->kc + cache_index(c, l, b, m->len[b]);
             float *vd = m->vc + cache_index(c, l, b, m->len[b]);
@@ -464,7 +494,7 @@ static int step(orc_model *m, const int32_t *tokens, int B, int grouped, int wan
                 vd[i] = c->kv_round_bf16 ? round_through_bf16(Vn[(size_t)b * kvd + i]) : Vn[(size_t)b * kvd + i];
             }
         }
-        /* both queries attend to primary positions 0..t inclusive */
+        /* every query attends to primary positions 0..t inclusive */
 #pragma omp parallel for schedule(static)
         for (int rh = 0; rh < Ra * nq; rh++) {
             int r = rh / nq, h = rh % nq, b = r % B, g = h / G;
@@ -474,25 +504,28 @@ static int step(orc_model *m, const int32_t *tokens, int B, int grouped, int wan
         }
         /* S-bar_i = S_i + Attn_i W_O */
         orc_linear(lw->wo, dt, d, (int)qd, O, Ra, A);
-        if (grouped && c->compute_matched) /* A_2 = g_A * A_1 (Eq. matched_attention) */
-            for (int b = 0; b < B; b++)
-                for (int i = 0; i < d; i++)
-                    A[(size_t)(B + b) * d + i] = lw->gate_a[i] * A[(size_t)b * d + i];
+        if (grouped && c->compute_matched) /* A_j = g_A * A_1 (Eq. matched_attention) */
+            for (int j = 1; j < P; j++)
+                for (int b = 0; b < B; b++)
+                    for (int i = 0; i < d; i++)
+                        A[((size_t)j * B + b) * d + i] = lw->gate_a[i] * A[(size_t)b * d + i];
         for (size_t i = 0; i < (size_t)R * d; i++) S[i] += A[i];
         /* MLP / MoE on RMSNorm(S-bar_i), then S_i^{l+1} = S-bar_i + M_i */
         for (int r = 0; r < R; r++)
             orc_rmsnorm(S + (size_t)r * d, lw->mlp_norm_g, d, c->rms_eps, N + (size_t)r * d);
-        const int32_t *f = forced ? forced + (size_t)l * 2 * B * kmax : NULL;
-        int32_t *ch = chosen ? chosen + (size_t)l * 2 * B * kmax : NULL;
+        const int32_t *f = forced ? forced + (size_t)l * K * B * kmax : NULL;
+        int32_t *ch = chosen ? chosen + (size_t)l * K * B * kmax : NULL;
         if (ch && !grouped)
-            for (int i = 0; i < B * kmax; i++) ch[(size_t)B * kmax + i] = -1;
-        mlp_any(c, lw, N, grouped ? N + (size_t)B * d : NULL, B, f, ch, M, M + (size_t)B * d);
+            for (int i = 0; i < (K - 1) * B * kmax; i++) ch[(size_t)B * kmax + i] = -1;
+        float *lg = m->rlog ? m->rlog + (size_t)l * K * c->max_batch * c->n_experts : NULL;
+        mlp_any(c, lw, N, P, B, f, ch, lg, c->max_batch, M);
         for (size_t i = 0; i < (size_t)R * d; i++) S[i] += M[i];
     }
     for (int b = 0; b < B; b++) m->len[b] += 1;
 
     if (want_logits) {
         float *Z = (float *)malloc(sizeof(float) * (size_t)R * V);
+        float *zb = (float *)malloc(sizeof(float) * (size_t)(P > 1 ? P - 1 : 1) * V);
         for (int r = 0; r < R; r++) {
             if (c->final_norm)
                 orc_rmsnorm(S + (size_t)r * d, m->w.final_norm_g, d, c->rms_eps, N + (size_t)r * d);
@@ -504,17 +537,19 @@ static int step(orc_model *m, const int32_t *tokens, int B, int grouped, int wan
             const float *zb1 = Z + (size_t)b * V;
             if (z1) memcpy(z1 + (size_t)b * V, zb1, sizeof(float) * (size_t)V);
             if (grouped) {
-                const float *zb2 = Z + (size_t)(B + b) * V;
+                for (int j = 1; j < P; j++) { /* branch logits, branch-major: z2 [K-1][B][V] */
+                    memcpy(zb + (size_t)(j - 1) * V, Z + ((size_t)j * B + b) * V, sizeof(float) * (size_t)V);
+                    if (z2) memcpy(z2 + ((size_t)(j - 1) * B + b) * V, Z + ((size_t)j * B + b) * V, sizeof(float) * (size_t)V);
+                }
                 float al;
-                int tok = orc_readout(zb1, zb2, V, &al, mix ? mix + (size_t)b * V : NULL);
-                if (z2) memcpy(z2 + (size_t)b * V, zb2, sizeof(float) * (size_t)V);
+                int tok = orc_readout_multi(zb1, zb, P - 1, V, &al, mix ? mix + (size_t)b * V : NULL);
                 if (alpha) alpha[b] = al;
                 if (next) next[b] = tok;
             } else if (next) {
                 next[b] = argmax_f32(zb1, V);
             }
         }
-        free(Z);
+        free(Z); free(zb);
     }
     free(S); free(N); free(Q); free(Kn); free(Vn); free(O); free(A); free(M); free(row);
     return 0;
@@ -543,61 +578,66 @@ int orc_prefill(orc_model *m, const int32_t *tokens, int B, int n, float *last_l
 }
 
 /* ------------------------------------------------------------------------------------ */
-/* Non-incremental two-path forward over whole sequences (the training-time graph of      */
-/* Section 4: both paths at every position, ordinary causal mask, branch reads K_1,V_1).  */
+/* Non-incremental forward over whole sequences (the training-time graph of Section 4:   */
+/* every path at every position, ordinary causal mask, the branches read K_1,V_1).       */
+/* z2 is [K-1][B][T][V].                                                                 */
 
 int orc_full_forward(const orc_config *c, const orc_weights *w, const int32_t *tokens, int B, int T,
                      float *z1, float *z2, float *k_out, float *v_out) {
     if (!c || !w || !tokens || !config_ok(c) || B <= 0 || T <= 0) return -1;
     int d = c->d_model, dh = c->head_dim, nq = c->n_q_heads, nkv = c->n_kv_heads, V = c->vocab;
     int G = nq / nkv, dt = c->weight_dtype;
+    int K = paths_of(c), Pa = c->compute_matched ? 1 : K;
     size_t qd = q_dim_of(c), kvd = kv_dim_of(c);
     double scale = 1.0 / sqrt((double)dh);
+    for (size_t i = 0; i < (size_t)B * T; i++)
+        if (tokens[i] < 0 || tokens[i] >= V) return -1;
 
-    float *S1 = (float *)malloc(sizeof(float) * (size_t)T * d), *S2 = (float *)malloc(sizeof(float) * (size_t)T * d);
-    float *N1 = (float *)malloc(sizeof(float) * (size_t)T * d), *N2 = (float *)malloc(sizeof(float) * (size_t)T * d);
-    float *Q1 = (float *)malloc(sizeof(float) * (size_t)T * qd), *Q2 = (float *)malloc(sizeof(float) * (size_t)T * qd);
+    /* path-major stacks of T rows each: S = [S_1; S_2; ...] */
+    float *S = (float *)malloc(sizeof(float) * (size_t)K * T * d);
+    float *N = (float *)malloc(sizeof(float) * (size_t)K * T * d);
+    float *Q = (float *)malloc(sizeof(float) * (size_t)K * T * qd);
     float *K1 = (float *)malloc(sizeof(float) * (size_t)T * kvd), *V1 = (float *)malloc(sizeof(float) * (size_t)T * kvd);
-    float *O1 = (float *)malloc(sizeof(float) * (size_t)T * qd), *O2 = (float *)malloc(sizeof(float) * (size_t)T * qd);
-    float *A1 = (float *)malloc(sizeof(float) * (size_t)T * d), *A2 = (float *)malloc(sizeof(float) * (size_t)T * d);
-    float *M1 = (float *)malloc(sizeof(float) * (size_t)T * d), *M2 = (float *)malloc(sizeof(float) * (size_t)T * d);
+    float *O = (float *)malloc(sizeof(float) * (size_t)K * T * qd);
+    float *A = (float *)malloc(sizeof(float) * (size_t)K * T * d);
+    float *M = (float *)malloc(sizeof(float) * (size_t)K * T * d);
     float *row = (float *)malloc(sizeof(float) * (size_t)d);
 
     for (int b = 0; b < B; b++) {
         const int32_t *x = tokens + (size_t)b * T;
         for (int t = 0; t < T; t++) {
-            if (x[t] < 0 || x[t] >= V) return -1;
             fetch_row(w->embed_primary, dt, (size_t)x[t], d, row);
-            orc_rmsnorm(row, w->embed_norm_g, d, c->rms_eps, S1 + (size_t)t * d);
-            fetch_row(w->embed_branch, dt, (size_t)x[t], d, row);
-            orc_rmsnorm(row, w->embed_norm_g, d, c->rms_eps, S2 + (size_t)t * d);
+            orc_rmsnorm(row, w->embed_norm_g, d, c->rms_eps, S + (size_t)t * d);
+            for (int j = 1; j < K; j++) {
+                fetch_row(w->embed_branch, dt, (size_t)(j - 1) * V + (size_t)x[t], d, row);
+                orc_rmsnorm(row, w->embed_norm_g, d, c->rms_eps, S + ((size_t)j * T + t) * d);
+            }
         }
         for (int l = 0; l < c->n_layers; l++) {
             const orc_layer_weights *lw = &w->layers[l];
+            for (int r = 0; r < K * T; r++)
+                orc_rmsnorm(S + (size_t)r * d, lw->attn_norm_g, d, c->rms_eps, N + (size_t)r * d);
+            orc_linear(lw->wq, dt, (int)qd, d, N, Pa * T, Q);
+            orc_linear(lw->wk, dt, (int)kvd, d, N, T, K1);
+            orc_linear(lw->wv, dt, (int)kvd, d, N, T, V1);
             for (int t = 0; t < T; t++) {
-                orc_rmsnorm(S1 + (size_t)t * d, lw->attn_norm_g, d, c->rms_eps, N1 + (size_t)t * d);
-                orc_rmsnorm(S2 + (size_t)t * d, lw->attn_norm_g, d, c->rms_eps, N2 + (size_t)t * d);
-            }
-            orc_linear(lw->wq, dt, (int)qd, d, N1, T, Q1);
-            orc_linear(lw->wk, dt, (int)kvd, d, N1, T, K1);
-            orc_linear(lw->wv, dt, (int)kvd, d, N1, T, V1);
-            if (!c->compute_matched) orc_linear(lw->wq, dt, (int)qd, d, N2, T, Q2);
-            for (int t = 0; t < T; t++) {
-                orc_rope(Q1 + (size_t)t * qd, nq, dh, t, c->rope_base);
+                orc_rope(Q + (size_t)t * qd, nq, dh, t, c->rope_base);
                 orc_rope(K1 + (size_t)t * kvd, nkv, dh, t, c->rope_base);
-                if (c->compute_matched) continue;
-                orc_rope(Q2 + (size_t)t * qd, nq, dh, t, c->rope_base);
-                for (size_t i = 0; i < qd; i++) Q2[(size_t)t * qd + i] += lw->coup_a[i] * Q1[(size_t)t * qd + i];
+                for (int j = 1; j < Pa; j++) {
+                    float *Qj = Q + ((size_t)j * T + t) * qd;
+                    orc_rope(Qj, nq, dh, t, c->rope_base);
+                    for (size_t i = 0; i < qd; i++) Qj[i] += lw->coup_a[i] * Q[(size_t)t * qd + i];
+                }
             }
             if (k_out) memcpy(k_out + (((size_t)l * B + b) * T) * kvd, K1, sizeof(float) * (size_t)T * kvd);
             if (v_out) memcpy(v_out + (((size_t)l * B + b) * T) * kvd, V1, sizeof(float) * (size_t)T * kvd);
             /* softmax(Q K^T / sqrt(d_h) + M_causal) V, the T x T form with an explicit mask */
 #pragma omp parallel for schedule(static)
-            for (int ph = 0; ph < (c->compute_matched ? 1 : 2) * nq; ph++) {
+            for (int ph = 0; ph < Pa * nq; ph++) {
                 int p = ph / nq, h = ph % nq, g = h / G;
-                const float *Qp = p ? Q2 : Q1;
-                float *Op = p ? O2 : O1;
-                double *P = (double *)malloc(sizeof(double) * (size_t)T);
+                const float *Qp = Q + (size_t)p * T * qd;
+                float *Op = O + (size_t)p * T * qd;
+                double *Pr = (double *)malloc(sizeof(double) * (size_t)T);
                 for (int i = 0; i < T; i++) {
                     double mx = -INFINITY, den = 0.0;
                     for (int j = 0; j < T; j++) {
@@ -606,55 +646,44 @@ int orc_full_forward(const orc_config *c, const orc_weights *w, const int32_t *t
                             acc += (double)Qp[(size_t)i * qd + (size_t)h * dh + e] *
                                    (double)K1[(size_t)j * kvd + (size_t)g * dh + e];
                         double mask = (j <= i) ? 0.0 : -INFINITY;
-                        P[j] = acc * scale + mask;
-                        if (P[j] > mx) mx = P[j];
+                        Pr[j] = acc * scale + mask;
+                        if (Pr[j] > mx) mx = Pr[j];
                     }
                     for (int j = 0; j < T; j++) {
-                        P[j] = exp(P[j] - mx);
-                        den += P[j];
+                        Pr[j] = exp(Pr[j] - mx);
+                        den += Pr[j];
                     }
                     for (int e = 0; e < dh; e++) {
                         double acc = 0.0;
-                        for (int j = 0; j < T; j++) acc += P[j] * (double)V1[(size_t)j * kvd + (size_t)g * dh + e];
+                        for (int j = 0; j < T; j++) acc += Pr[j] * (double)V1[(size_t)j * kvd + (size_t)g * dh + e];
                         Op[(size_t)i * qd + (size_t)h * dh + e] = (float)(acc / den);
                     }
                 }
-                free(P);
+                free(Pr);
             }
-            orc_linear(lw->wo, dt, d, (int)qd, O1, T, A1);
-            if (c->compute_matched) { /* A_2 = g_A * A_1 (Eq. matched_attention) */
-                for (int t = 0; t < T; t++)
-                    for (int i = 0; i < d; i++) A2[(size_t)t * d + i] = lw->gate_a[i] * A1[(size_t)t * d + i];
-            } else {
-                orc_linear(lw->wo, dt, d, (int)qd, O2, T, A2);
-            }
-            for (size_t i = 0; i < (size_t)T * d; i++) {
-                S1[i] += A1[i];
-                S2[i] += A2[i];
-            }
-            for (int t = 0; t < T; t++) {
-                orc_rmsnorm(S1 + (size_t)t * d, lw->mlp_norm_g, d, c->rms_eps, N1 + (size_t)t * d);
-                orc_rmsnorm(S2 + (size_t)t * d, lw->mlp_norm_g, d, c->rms_eps, N2 + (size_t)t * d);
-            }
-            mlp_any(c, lw, N1, N2, T, NULL, NULL, M1, M2);
-            for (size_t i = 0; i < (size_t)T * d; i++) {
-                S1[i] += M1[i];
-                S2[i] += M2[i];
-            }
+            orc_linear(lw->wo, dt, d, (int)qd, O, Pa * T, A);
+            if (c->compute_matched) /* A_j = g_A * A_1 (Eq. matched_attention) */
+                for (int j = 1; j < K; j++)
+                    for (int t = 0; t < T; t++)
+                        for (int i = 0; i < d; i++)
+                            A[((size_t)j * T + t) * d + i] = lw->gate_a[i] * A[(size_t)t * d + i];
+            for (size_t i = 0; i < (size_t)K * T * d; i++) S[i] += A[i];
+            for (int r = 0; r < K * T; r++)
+                orc_rmsnorm(S + (size_t)r * d, lw->mlp_norm_g, d, c->rms_eps, N + (size_t)r * d);
+            mlp_any(c, lw, N, K, T, NULL, NULL, NULL, 0, M);
+            for (size_t i = 0; i < (size_t)K * T * d; i++) S[i] += M[i];
         }
-        for (int t = 0; t < T; t++) {
-            if (c->final_norm) {
-                orc_rmsnorm(S1 + (size_t)t * d, w->final_norm_g, d, c->rms_eps, N1 + (size_t)t * d);
-                orc_rmsnorm(S2 + (size_t)t * d, w->final_norm_g, d, c->rms_eps, N2 + (size_t)t * d);
-            } else {
-                memcpy(N1 + (size_t)t * d, S1 + (size_t)t * d, sizeof(float) * (size_t)d);
-                memcpy(N2 + (size_t)t * d, S2 + (size_t)t * d, sizeof(float) * (size_t)d);
-            }
+        for (int r = 0; r < K * T; r++) {
+            if (c->final_norm)
+                orc_rmsnorm(S + (size_t)r * d, w->final_norm_g, d, c->rms_eps, N + (size_t)r * d);
+            else
+                memcpy(N + (size_t)r * d, S + (size_t)r * d, sizeof(float) * (size_t)d);
         }
-        if (z1) orc_linear(w->lm_head, dt, V, d, N1, T, z1 + (size_t)b * T * V);
-        if (z2) orc_linear(w->lm_head, dt, V, d, N2, T, z2 + (size_t)b * T * V);
+        if (z1) orc_linear(w->lm_head, dt, V, d, N, T, z1 + (size_t)b * T * V);
+        if (z2)
+            for (int j = 1; j < K; j++)
+                orc_linear(w->lm_head, dt, V, d, N + (size_t)j * T * d, T, z2 + (((size_t)(j - 1) * B + b) * T) * V);
     }
-    free(S1); free(S2); free(N1); free(N2); free(Q1); free(Q2); free(K1); free(V1);
-    free(O1); free(O2); free(A1); free(A2); free(M1); free(M2); free(row);
+    free(S); free(N); free(Q); free(K1); free(V1); free(O); free(A); free(M); free(row);
     return 0;
 }

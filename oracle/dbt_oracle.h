@@ -49,6 +49,12 @@ typedef struct {
                                   A_2 = g_A * A_1 and M_2 = R_2(N_2;k_2) + g_G * G(N_1);
                                   the a/b/c couplings do not appear in those equations and
                                   are not applied.  MoE layers only.                       */
+    int32_t n_paths;           /* K of Appendix C.1 ("More decode branches"): residual paths in
+                                  all, the primary plus K-1 decode branches; each branch has
+                                  its own embedding table and same-position state, reads the
+                                  primary cache, shares a/b/c with the other branches, and the
+                                  readout uses the mean of the branch distributions.  2 (or 0)
+                                  is the main text's model.                                 */
     int32_t max_batch, max_seq;
 } orc_config;
 
@@ -69,7 +75,8 @@ typedef struct {
 } orc_layer_weights;
 
 typedef struct {
-    const void  *embed_primary, *embed_branch;   /* E_1, E_2 : [V,d]                 */
+    const void  *embed_primary, *embed_branch;   /* E_1 [V,d]; E_2..E_K one after another:
+                                                    [K-1][V,d]                        */
     const float *embed_norm_g, *final_norm_g;    /* [d]                              */
     const void  *lm_head;                        /* shared output matrix [V,d]       */
     const orc_layer_weights *layers;             /* [n_layers]                       */
@@ -89,6 +96,10 @@ int  orc_seq_len(const orc_model *m, int b);
 float *orc_k_cache(orc_model *m);
 float *orc_v_cache(orc_model *m);
 void orc_set_seq_len(orc_model *m, int b, int len);
+/* MoE models: the router logits r_i = N_i W_r the last step computed, [L][K][max_batch][E]
+ * (rows of paths the step did not evaluate keep older contents); NULL for dense models.
+ * Tests use them to check that an expert set chosen elsewhere is a valid top-k. */
+const float *orc_router_logits(const orc_model *m);
 
 /* Primary-only pass over n prompt positions of sequences 0..B-1 (tokens [B][n]),
  * position by position; appends K/V; logits of the last position to last_logits [B][V]
@@ -96,9 +107,9 @@ void orc_set_seq_len(orc_model *m, int b, int len);
 int orc_prefill(orc_model *m, const int32_t *tokens, int B, int n, float *last_logits);
 
 /* One step at position t_b = seq_len[b] for every sequence, token tokens[b].
- * grouped != 0: both paths; z2/alpha/mix are written; next = argmax of the mixture.
- * grouped == 0: the primary path alone; next = argmax z1.
- * forced_experts (nullable, MoE): [L][2][B][kmax] expert ids to use instead of top-k
+ * grouped != 0: all K paths; z2 ([K-1][B][V], branch-major), alpha, mix are written; next =
+ * argmax of the mixture.  grouped == 0: the primary path alone; next = argmax z1.
+ * forced_experts (nullable, MoE): [L][K][B][kmax] expert ids to use instead of top-k
  * selection (weights are still computed from this run's router probabilities), where
  * kmax = max(k_primary,k_branch); chosen_experts (nullable) receives the ids used,
  * same layout, -1 padded.  Any output pointer may be NULL. */
@@ -106,9 +117,9 @@ int orc_decode_step(orc_model *m, const int32_t *tokens, int B, int grouped,
                     const int32_t *forced_experts, int32_t *chosen_experts,
                     int32_t *next, float *z1, float *z2, float *alpha, float *mix);
 
-/* Non-incremental definition: both paths at every position of tokens [B][T] with an
+/* Non-incremental definition: every path at every position of tokens [B][T] with an
  * explicit causal mask (the training-time forward).  Touches no cache.  Outputs
- * z1,z2 [B][T][V] (nullable), k_out,v_out [L][B][T][kv_dim] (nullable). */
+ * z1 [B][T][V], z2 [K-1][B][T][V] (nullable), k_out,v_out [L][B][T][kv_dim] (nullable). */
 int orc_full_forward(const orc_config *cfg, const orc_weights *w, const int32_t *tokens,
                      int B, int T, float *z1, float *z2, float *k_out, float *v_out);
 
@@ -129,6 +140,9 @@ void orc_swiglu(const float *g, const float *u, int n, float *h);
 void orc_route(const float *logits, int E, int k, const int32_t *forced, int32_t *idx, float *wts);
 /* Readout of Eq. alpha / mixloss: p,q softmax; alpha; mix (nullable, [V]); returns argmax mix. */
 int orc_readout(const float *z1, const float *z2, int V, float *alpha, float *mix);
+/* The same with nb decode branches (Appendix C.1): zb [nb][V], q replaced by the mean of the
+ * branch distributions. */
+int orc_readout_multi(const float *z1, const float *zb, int nb, int V, float *alpha, float *mix);
 
 void orc_set_threads(int n);
 int  orc_get_threads(void);

@@ -38,6 +38,7 @@ class ModelConfig:
     router_mode: int = 0  # 0 independent routing, 1 router replay
     moe_b_coupling: int = 1
     compute_matched: int = 0  # 1: compute-matched MoE allocation (Appendix B.3): A_2 = g_A*A_1, shared expert gated
+    n_paths: int = 2  # K of Appendix C.1: the primary path plus K-1 decode branches (own embedding table each)
     page_size: int = 16
 
     @property
@@ -137,7 +138,8 @@ def make_weights(cfg: ModelConfig, seed: int = 0, coupling_std: float = 0.5,
     d, qd, kvd = cfg.d_model, cfg.q_dim, cfg.kv_dim
     w: dict = {
         "embed_primary": _normal(gen, (cfg.vocab, d), matrix_std, wd),
-        "embed_branch": _normal(gen, (cfg.vocab, d), matrix_std, wd),
+        # E_2 .. E_K, one table per decode branch, stacked [(K-1) * V, d]
+        "embed_branch": _normal(gen, ((cfg.n_paths - 1) * cfg.vocab, d), matrix_std, wd),
         "embed_norm_g": _normal(gen, (d,), 0.02, torch.float32, 1.0),
         "final_norm_g": _normal(gen, (d,), 0.02, torch.float32, 1.0),
         "lm_head": _normal(gen, (cfg.vocab, d), lm_head_std if lm_head_std is not None else matrix_std, wd),

@@ -321,3 +321,39 @@ def test_tiny_config_random_init_gives_alpha_half():
     tok = make_tokens(cfg, 1, 3, seed=1).numpy()
     _, outs, _ = run_incremental(cfg, w, tok, n_prefill=2)
     assert outs[0]["alpha"][0] == 0.5
+
+
+def test_recorded_router_logits_explain_the_chosen_experts():
+    """orc_router_logits exposes r_i = N_i W_r of the last step: the experts the step chose are the
+    brute-force top-k of those logits, the replayed branch reuses the primary's set, and the logits of
+    the first layer's primary rows equal the library-built float64 restatement."""
+    for cfg in (small_moe(), small_moe(router_mode=1)):
+        w = make_weights(cfg, seed=2, matrix_std=0.3)
+        tok = make_tokens(cfg, 3, 6, seed=3).numpy()
+        m = oracle.OracleModel(cfg, w, 3, 6)
+        m.prefill(tok[:, :4], want_logits=False)
+        o = m.decode_step(tok[:, 4])
+        r = m.router_logits(3)
+        assert r.shape == (cfg.n_layers, 2, 3, cfg.n_experts)
+        for l in range(cfg.n_layers):
+            for b in range(3):
+                top1 = set(np.argsort(-r[l, 0, b], kind="stable")[:cfg.k_primary].tolist())
+                assert set(o["experts"][l, 0, b, :cfg.k_primary].tolist()) == top1
+                if cfg.router_mode == 1:
+                    assert set(o["experts"][l, 1, b, :cfg.k_primary].tolist()) == top1
+                else:
+                    top2 = set(np.argsort(-r[l, 1, b], kind="stable")[:cfg.k_branch].tolist())
+                    assert set(o["experts"][l, 1, b, :cfg.k_branch].tolist()) == top2
+        # layer 0, primary rows, position 4: RMSNorm(S-bar_1) W_r rebuilt from library routines
+        import torch.nn.functional as F
+        lw = w["layers"][0]
+        tk = torch.as_tensor(tok[:, :5]).long()
+        s1 = F.rms_norm(w["embed_primary"].double()[tk], (cfg.d_model,), w["embed_norm_g"].double(), cfg.rms_eps)
+        n1 = F.rms_norm(s1, (cfg.d_model,), lw["attn_norm_g"].double(), cfg.rms_eps)
+        q1 = ref_torch._rope_complex(n1 @ lw["wq"].double().T, cfg.n_q_heads, cfg.head_dim, cfg.rope_base)
+        k1 = ref_torch._rope_complex(n1 @ lw["wk"].double().T, cfg.n_kv_heads, cfg.head_dim, cfg.rope_base)
+        v1 = n1 @ lw["wv"].double().T
+        sbar = s1 + ref_torch._attn(q1, k1, v1, cfg) @ lw["wo"].double().T
+        m1 = F.rms_norm(sbar, (cfg.d_model,), lw["mlp_norm_g"].double(), cfg.rms_eps)
+        want = (m1 @ lw["router"].double().T)[:, 4].numpy()
+        np.testing.assert_allclose(r[0, 0], want, rtol=2e-4, atol=2e-5)
