@@ -48,7 +48,8 @@ typedef enum {
     DBT_ERR_CAPACITY = 3,    /* max_batch, max_seq or the page pool would be exceeded */
     DBT_ERR_STATE = 4,
     DBT_ERR_CUDA = 5,
-    DBT_ERR_DEVICE = 6       /* the device status word is non-zero (dbt_sync_status)  */
+    DBT_ERR_DEVICE = 6,      /* the device status word is non-zero (dbt_sync_status)  */
+    DBT_ERR_TIMEOUT = 7      /* a bounded wait inside a kernel ran out (dbt_sync_status) */
 } dbt_status;
 
 enum { DBT_DTYPE_F32 = 0, DBT_DTYPE_BF16 = 1 };
@@ -167,10 +168,27 @@ dbt_status dbt_decode_step_primary_only_host(dbt_model *m, const int32_t *tokens
 dbt_status dbt_last_experts(dbt_model *m, const int32_t **experts_dev, int32_t *kmax);
 dbt_status dbt_last_expert_union(dbt_model *m, int32_t *count_per_layer_host);
 
-/* Wait for the stream and read the device status word.  *device_status: 0 = clean, 1 = a token
- * id was out of range, 2 = a page id was out of range; *detail = the offending value.
- * Returns DBT_ERR_DEVICE when non-zero.  HOST pointers, may be NULL. */
+/* Wait for the stream and read the device status word.  *device_status: 0 = clean; 1 = a token
+ * id was out of range, 2 = a page id was out of range (*detail = the offending value; the value was
+ * clamped and the step ran on): returns DBT_ERR_DEVICE; 3 = a bounded wait inside a kernel (on a
+ * shared-memory barrier that a TMA copy or a tensor-core commit completes) ran out after about two
+ * seconds: *detail = the wait site (100 + warp: operand ring of the GEMM, 200 + warp: its accumulator,
+ * 300..: the attention kernel's page ring), the CTA skipped its stores, released its tensor memory and
+ * returned, so the step's results are invalid but the context stays usable: returns DBT_ERR_TIMEOUT.
+ * The first code recorded wins until dbt_reset clears the word.  HOST pointers, may be NULL. */
 dbt_status dbt_sync_status(dbt_model *m, int32_t *device_status, int32_t *detail);
+
+/* The persistent state of the method is the primary path's KV cache alone (Background, "KV cache";
+ * Section 4.4 "Decode": the branch writes no persistent entries).  These two calls move it between the
+ * paged pool and HOST buffers in logical order [n_layers][B][T][kv_dim] (elements of `weight_dtype`, K after
+ * RoPE), for sequences seq_ids_host[0..B-1] (HOST; NULL = sequences 0..B-1) and positions 0..T-1, through the
+ * page table; they wait for the stream.  Export needs T <= the current length of each sequence
+ * (DBT_ERR_STATE otherwise).  Import overwrites those positions and sets the length of each listed
+ * sequence to T (the other sequences keep theirs).  T beyond a sequence's capacity: DBT_ERR_CAPACITY.
+ * Uses: handing a prefilled cache to another process or a checker, restoring a session, tests. */
+dbt_status dbt_kv_export(dbt_model *m, const int32_t *seq_ids_host, int32_t B, int32_t T, void *k_host, void *v_host);
+dbt_status dbt_kv_import(dbt_model *m, const int32_t *seq_ids_host, int32_t B, int32_t T, const void *k_host,
+                         const void *v_host);
 
 /* Operator-level entry: the grouped skinny GEMM alone (Section 4.4 "Decode": the stacked rows
  * of both paths go through one shared matrix, each weight tile fetched once).
@@ -178,9 +196,11 @@ dbt_status dbt_sync_status(dbt_model *m, int32_t *device_status, int32_t *detail
  * (1 <= R <= 256, K a multiple of 8, both 16-byte aligned), Y_dev DEVICE fp32 [R][n_out].
  * scratch_dev: DEVICE fp32 workspace of scratch_floats elements for the split-K partials
  * (at least splits * roundup(R) * n_out with roundup to 16/32/64/128/256); status_dev DEVICE
- * int32[2] (zeroed by the caller; non-zero afterwards = a bounded device wait expired).
- * force_split > 0 fixes the split-K factor, 0 lets the library choose; *split_used (HOST,
- * nullable) receives it.  Runs on the tensor cores (TMA + tcgen05); enqueues on cuda_stream. */
+ * int32[2] (zeroed by the caller; afterwards {3, wait site} when a bounded device wait ran out -- the
+ * codes of dbt_sync_status -- else still zero).
+ * force_split > 0 asks for that split-K factor (lowered to ceil(K/64) and to a factor whose ranges
+ * are all non-empty), 0 lets the library choose; *split_used (HOST, nullable) receives the factor
+ * used.  Runs on the tensor cores (TMA + tcgen05); enqueues on cuda_stream. */
 dbt_status dbt_op_gemm_tc(const void *W_dev, const void *X_dev, int32_t n_out, int32_t K, int32_t R,
                           int32_t force_split, float *Y_dev, float *scratch_dev, size_t scratch_floats,
                           int32_t *status_dev, void *cuda_stream, int32_t *split_used);

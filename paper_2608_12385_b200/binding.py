@@ -18,13 +18,13 @@ LIB_PATH = os.path.join(_HERE, "libdbt_b200.so")
 
 DBT_OK = 0
 STATUS_NAMES = {0: "DBT_OK", 1: "DBT_ERR_INVALID_ARG", 2: "DBT_ERR_UNSUPPORTED", 3: "DBT_ERR_CAPACITY",
-                4: "DBT_ERR_STATE", 5: "DBT_ERR_CUDA", 6: "DBT_ERR_DEVICE"}
+                4: "DBT_ERR_STATE", 5: "DBT_ERR_CUDA", 6: "DBT_ERR_DEVICE", 7: "DBT_ERR_TIMEOUT"}
 
 EXPORTS = ["dbt_query_sizes", "dbt_create", "dbt_destroy", "dbt_set_page_table", "dbt_reset", "dbt_set_seq_lens",
            "dbt_seq_len", "dbt_prefill", "dbt_decode_step", "dbt_decode_step_primary_only", "dbt_decode_step_host",
            "dbt_decode_step_primary_only_host", "dbt_last_experts", "dbt_last_expert_union", "dbt_sync_status",
            "dbt_launch_count", "dbt_last_error", "dbt_version", "dbt_profile_begin", "dbt_profile_end", "dbt_op_gemm_tc",
-           "dbt_op_gemm_tc_static"]
+           "dbt_op_gemm_tc_static", "dbt_kv_export", "dbt_kv_import"]
 
 
 class DbtError(RuntimeError):
@@ -90,6 +90,8 @@ def load_library():
     L.dbt_last_experts.argtypes = [vp, C.POINTER(vp), i32p]
     L.dbt_last_expert_union.argtypes = [vp, vp]
     L.dbt_sync_status.argtypes = [vp, i32p, i32p]
+    L.dbt_kv_export.argtypes = [vp, vp, i32, i32, vp, vp]
+    L.dbt_kv_import.argtypes = [vp, vp, i32, i32, vp, vp]
     L.dbt_op_gemm_tc.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, C.c_size_t, vp, vp, i32p]
     L.dbt_op_gemm_tc_static.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, vp, i32p]
     L.dbt_profile_begin.argtypes = [vp]
@@ -146,8 +148,8 @@ def op_gemm_tc(W: torch.Tensor, X: torch.Tensor, force_split: int = 0, scratch: 
         raise DbtError(st, L.dbt_last_error(None).decode())
     torch.cuda.synchronize()
     code = status.cpu().tolist()
-    if code[0] != 0:
-        raise DbtError(6, f"device status {code}")
+    if code[0] != 0:  # 3: a bounded device wait ran out (the codes of dbt_sync_status)
+        raise DbtError(7 if code[0] == 3 else 6, f"device status {code}")
     return Y, used.value
 
 
@@ -171,8 +173,8 @@ def op_gemm_tc_static(W: torch.Tensor, X: torch.Tensor, force_split: int = 0, Y:
         raise DbtError(st, L.dbt_last_error(None).decode())
     torch.cuda.synchronize()
     code = status.cpu().tolist()
-    if code[0] != 0:
-        raise DbtError(6, f"device status {code}")
+    if code[0] != 0:  # 3: a bounded device wait ran out (the codes of dbt_sync_status)
+        raise DbtError(7 if code[0] == 3 else 6, f"device status {code}")
     return Y, used.value
 
 
@@ -333,7 +335,7 @@ class Model:
     def sync_status(self) -> tuple[int, int]:
         s, d = C.c_int32(0), C.c_int32(0)
         st = self.L.dbt_sync_status(self._h, C.byref(s), C.byref(d))
-        if st not in (DBT_OK, 6):
+        if st not in (DBT_OK, 6, 7):
             self._check(st)
         return s.value, d.value
 
@@ -350,7 +352,30 @@ class Model:
     def launch_count(self) -> int:
         return self.L.dbt_launch_count(self._h)
 
-    # -- cache access through the page table (the pool is the caller's memory) --------------
+    # -- the cache through the C ABI (dbt_kv_export / dbt_kv_import) ---------------------------
+    def export_kv(self, batch: int, length: int, seq_ids=None):
+        """K, V [n_layers, batch, length, kv_dim] of sequences `seq_ids` (default 0..batch-1) as CPU
+        tensors of the model's storage type."""
+        c = self.cfg
+        k = torch.empty(c.n_layers, batch, length, c.kv_dim, dtype=c.torch_dtype)
+        v = torch.empty_like(k)
+        ids = None if seq_ids is None else torch.as_tensor(seq_ids, dtype=torch.int32).contiguous()
+        assert ids is None or ids.numel() == batch
+        self._check(self.L.dbt_kv_export(self._h, _p(ids), batch, length, k.data_ptr(), v.data_ptr()))
+        return k, v
+
+    def import_kv(self, k: torch.Tensor, v: torch.Tensor, seq_ids=None):
+        """Load K, V [n_layers, B, T, kv_dim] (any float type; converted to the model's) into sequences
+        `seq_ids` (default 0..B-1) and set their lengths to T."""
+        c = self.cfg
+        k = k.to("cpu", c.torch_dtype).contiguous()
+        v = v.to("cpu", c.torch_dtype).contiguous()
+        assert k.shape == v.shape and k.shape[0] == c.n_layers and k.shape[3] == c.kv_dim
+        ids = None if seq_ids is None else torch.as_tensor(seq_ids, dtype=torch.int32).contiguous()
+        assert ids is None or ids.numel() == k.shape[1]
+        self._check(self.L.dbt_kv_import(self._h, _p(ids), k.shape[1], k.shape[2], k.data_ptr(), v.data_ptr()))
+
+    # -- direct pool access for the benchmark's synthetic fills (the pool is the caller's memory) --
     def write_kv(self, k: torch.Tensor, v: torch.Tensor, page_table: torch.Tensor | None = None):
         """Scatter contiguous K, V [L, B, T, kv_dim] into the paged pool and set the lengths."""
         B, T = k.shape[1], k.shape[2]
@@ -358,12 +383,6 @@ class Model:
         scatter_kv(self.kv_view(), k.to(self.device, self.cfg.torch_dtype), v.to(self.device, self.cfg.torch_dtype),
                    pt.to(self.device), self.cfg)
         self.set_seq_lens([T] * B)
-
-    def read_kv(self, batch: int, length: int, page_table: torch.Tensor | None = None):
-        """Gather K, V [L, batch, length, kv_dim] from the paged pool."""
-        pt = page_table if page_table is not None else self.page_table
-        torch.cuda.synchronize(self.device)
-        return gather_kv(self.kv_view(), pt.to(self.device), batch, length, self.cfg)
 
 
 def _page_slot(pt: torch.Tensor, T: int, page_size: int):
@@ -381,12 +400,3 @@ def scatter_kv(view: torch.Tensor, k: torch.Tensor, v: torch.Tensor, pt: torch.T
         s = src.view(Lyr, B, T, cfg.n_kv_heads, cfg.head_dim).permute(1, 2, 0, 3, 4)  # [B, T, L, n_kv, dh]
         sub = view[:, which]                                                          # [L, P, n_kv, page, dh]
         sub[:, pages, :, slots, :] = s  # the two index tensors broadcast to [B, T] and move to the front
-
-
-def gather_kv(view: torch.Tensor, pt: torch.Tensor, B: int, T: int, cfg: ModelConfig):
-    pages, slots = _page_slot(pt[:B], T, cfg.page_size)
-    out = []
-    for which in (0, 1):
-        g = view[:, which][:, pages, :, slots, :]                                     # [B, T, L, n_kv, dh]
-        out.append(g.permute(2, 0, 1, 3, 4).reshape(cfg.n_layers, B, T, cfg.kv_dim).contiguous())
-    return out[0], out[1]

@@ -19,7 +19,6 @@
 #include "dbt_fused.cuh"
 #include "dbt_gemm_tc.cuh"
 #include "dbt_kernels.cuh"
-#include "dbt_mega.cuh"
 
 using namespace dbt;
 
@@ -33,6 +32,7 @@ struct Workspace {
     float2 *rope;
     int32_t *seq_len, *page_table, *status, *tokens_stage, *next_stage, *att_tickets, *att_tickets2, *gemm_tickets;
     float *alpha_stage;
+    char *kv_stage;  // staging for dbt_kv_export / dbt_kv_import (kKvStageBytes)
     // MoE
     float *rlogits, *rwts, *Hexp, *Yexp, *Msh, *Hsh;
     int32_t *ridx, *ecnt, *elist, *last_experts, *union_cnt;
@@ -49,14 +49,9 @@ struct Workspace {
     int32_t *epos, *eoff;
     float *rs_sorted;  // 1/rms of each sorted row's source row (norm applied after the per-expert gate|up GEMM)
     size_t P_floats;
-    // single-kernel decode step: plans (one per batch size and mode), descriptor array, counters
-    char *mega_plans;
-    CUtensorMap *mega_maps;
-    unsigned int *mega_sync;  // [0] barrier arrivals, [1] CTAs done, [2] error flag
-    float *rd_part, *rd_best;
 };
-constexpr int kMegaPlanSlots = 16;
-constexpr int kMegaTailMaps = 11;  // lm_head, K/V pages, {Xb, Ob, Hb} x row-tile width {16, 32, 64}
+
+constexpr size_t kKvStageBytes = (size_t)8 << 20;
 
 struct LayerMaps {
     CUtensorMap wq, wk, wv, wo, wg, wu, wd;  // dense MLP; for MoE wg/wu/wd hold the shared expert
@@ -91,26 +86,16 @@ struct dbt_model {
     CUtensorMap map_lm, map_Xb, map_Ob, map_Hb, map_kv, map_Xs, map_Hs;
     bool moe_tc;  // MoE experts on the tensor cores
     bool att_fast;  // TMA + mma.sync attention over the bf16 pool
-    bool fused;     // dense bf16: elementwise work fused into the GEMM epilogues
     bool wide;      // dense bf16: RMSNorm factor applied after the GEMM, no row-wide reduction kernel
     // two-plane GEMM inputs: base pointer of each 2-D input map, and the 3-D one-box-per-stage views
     // built from it on first use (key: 2-D map, row-tile width, plane rows)
     struct ActBase { const void *base; };
     std::map<const CUtensorMap *, ActBase> act_base;
     std::map<std::tuple<const CUtensorMap *, int, int>, CUtensorMap> act3d;
-    int cluster_max;     // largest cluster the GEMM kernel may be launched with (16 when the opt-in size is granted, else 8)
-    int next_cluster_x = 1, next_cluster_y;  // cluster dims for the next launch (y 0: none); consumed by LAUNCH
-    bool cluster_gu;     // opt-in: gate|up GEMM as clusters of {gate tile, up tile} x splits that apply SwiGLU + b themselves
-    bool cluster_epi;    // opt-in: O and down projections reduce their split-K partials inside a cluster and apply the residual there
-    bool stack_planes;  // GEMM: one MMA per k16 step over both activation planes (DBT_STACK=0 issues two)
     bool evict_first;  // weight tiles and K/V pages carry the evict-first L2 hint (DBT_EVICT_FIRST=0 turns it off)
     bool fuse_qkv;     // decode steps: the attention kernel does the Q|K|V epilogue itself (DBT_FUSE_QKV=0 keeps the kernel)
-    bool l2_prefetch;  // GEMM launches ask the L2 for the next GEMM's weights (opt-in, DBT_L2_PREFETCH=1)
-    bool mega;      // dense bf16, small batch: the whole decode step as one persistent kernel
-    struct MegaSlot { int B, grouped; };
-    std::vector<MegaSlot> mega_slots;
     int num_sms;
-    int act_parts;  // 2: GEMM inputs carried as hi + lo bf16 terms; 1: plain bf16
+    int act_parts;  // 2: GEMM inputs carried as hi + lo bf16 terms (the operator-level GEMM entry uses 1: plain bf16)
     // a decode step is captured once per (batch, mode, buffer set) and replayed as a CUDA graph
     struct GraphEntry {
         int B, grouped;
@@ -129,7 +114,7 @@ struct dbt_model {
     bool moe_overlap;
     bool readout_row;  // DBT_READOUT=row: the one-CTA-per-row readout kernel
     int moe_row_tile;  // DBT_MOE_ROWTILE: row tile of the per-expert GEMMs (-1: chosen from the batch, 0: one tile of all rows)
-    bool moe_wide;  // MoE chain with the RMSNorm factor applied behind the GEMMs (DBT_MOE_WIDE=0: row-wide norm kernels)
+    bool moe_wide;  // MoE chain with the RMSNorm factor applied behind the GEMMs (tensor-core MoE path)
     std::vector<GraphEntry> graphs;
 };
 
@@ -216,6 +201,7 @@ size_t carve(const dbt_config &c, char *base, Workspace *ws, int *Rmax_out, int 
     w.tokens_stage = k.take<int32_t>(c.max_batch);
     w.next_stage = k.take<int32_t>(c.max_batch);
     w.alpha_stage = k.take<float>(c.max_batch);
+    w.kv_stage = k.take<char>(kKvStageBytes);
     if (moe) {
         int km = kmax_of(c);
         w.rlogits = k.take<float>((size_t)Rmax * c.n_experts);
@@ -243,13 +229,6 @@ size_t carve(const dbt_config &c, char *base, Workspace *ws, int *Rmax_out, int 
         if (w.P_floats < (size_t)Rmax * widest) w.P_floats = (size_t)Rmax * widest;
         w.P = k.take<float>(w.P_floats);
         w.ss = k.take<float>((size_t)((d + 127) / 128) * Rmax);
-        if (!moe) {
-            w.mega_plans = k.take<char>((size_t)kMegaPlanSlots * align_up(sizeof(MegaPlan)));
-            w.mega_maps = k.take<CUtensorMap>((size_t)c.n_layers * 7 + kMegaTailMaps);
-            w.mega_sync = k.take<unsigned int>(8);
-            w.rd_part = k.take<float>((size_t)kMegaMaxCtas * 64 * 4);
-            w.rd_best = k.take<float>((size_t)kMegaMaxCtas * 64 * 2);
-        }
         if (moe) {
             size_t Rk = (size_t)Rmax * kmax_of(c);
             w.Xs = k.take<__nv_bfloat16>(2 * Rk * d);
@@ -294,25 +273,18 @@ dbt_status fail(dbt_model *m, dbt_status st, const char *fmt, ...) {
 // stream-serialization attribute, so the kernel may start while its predecessor drains.  Each
 // kernel calls griddepcontrol.wait before it touches anything its predecessor produced.
 template <typename... Params, typename... Args>
-cudaError_t launch_kernel(cudaStream_t stream, bool pdl, int cluster_x, int cluster_y, dim3 grid, dim3 block, size_t smem,
+cudaError_t launch_kernel(cudaStream_t stream, bool pdl, dim3 grid, dim3 block, size_t smem,
                           void (*kernel)(Params...), Args &&...args) {
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = grid;
     cfg.blockDim = block;
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[2];
+    cudaLaunchAttribute attr[1];
     int n = 0;
     if (pdl) {
         attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr[n].val.programmaticStreamSerializationAllowed = 1;
-        n++;
-    }
-    if (cluster_x * cluster_y > 1) {  // cluster_x x cluster_y neighbouring CTAs of the grid form one thread-block cluster
-        attr[n].id = cudaLaunchAttributeClusterDimension;
-        attr[n].val.clusterDim.x = (unsigned)cluster_x;
-        attr[n].val.clusterDim.y = (unsigned)cluster_y;
-        attr[n].val.clusterDim.z = 1;
         n++;
     }
     cfg.attrs = attr;
@@ -353,10 +325,8 @@ cudaEvent_t prof_event(dbt_model *m) {
             p1_ = prof_event(m);                                                                         \
             cudaEventRecord(p0_, (m)->stream);                                                           \
         }                                                                                                \
-        cudaError_t e_ = launch_kernel((m)->stream, (m)->use_pdl && !pdl_disabled_for(m, tag), (m)->next_cluster_x,     \
-                                       (m)->next_cluster_y, dim3(grid), dim3(block), smem, kernel, __VA_ARGS__); \
-        (m)->next_cluster_x = 1;                                                                         \
-        (m)->next_cluster_y = 0;                                                                         \
+        cudaError_t e_ = launch_kernel((m)->stream, (m)->use_pdl && !pdl_disabled_for(m, tag), dim3(grid),       \
+                                       dim3(block), smem, kernel, __VA_ARGS__);                          \
         (m)->launches++;                                                                                 \
         if ((m)->prof_on) {                                                                              \
             cudaEventRecord(p1_, (m)->stream);                                                           \
@@ -578,8 +548,6 @@ struct TcCall {
     const int *grp_cnt, *grp_off;  // per-expert mode (see TcParams); n_groups experts
     int grp_w_rows, n_groups;
     int grp_row_tiles;  // per-expert mode: row tiles of n_tile rows per expert (0: one tile holds any list)
-    const void *pf_ptr[3];  // L2 prefetch requests carried by this launch (the next GEMM's weights)
-    size_t pf_bytes[3];
 };
 
 int norm_threads(int d) { return d >= 1024 ? 1024 : d >= 512 ? 512 : 256; }
@@ -604,20 +572,14 @@ int choose_split(int tiles, int total_kt, int slots) {
 }
 
 // CTAs of the GEMM kernel that are resident at once: two per SM up to a row tile of 64 (96 KB of
-// ring each), one above.  DBT_SPLIT_SLOTS overrides (experiments).
+// ring each), one above.
 int split_slots(const dbt_model *m, int n_tile) {
-    static int forced = -1;
-    if (forced < 0) {
-        const char *e = getenv("DBT_SPLIT_SLOTS");
-        forced = e ? atoi(e) : 0;
-    }
-    if (forced > 0) return forced;
     int sms = m->num_sms > 0 ? m->num_sms : 148;  // the operator-level entry points carry no device query
     return (n_tile <= 64 ? 2 : 1) * sms;
 }
 
 template <int N_TILE>
-dbt_status launch_gemm_tc(dbt_model *m, const TcCall &c, const TcParams &p, const FusedEpi &e, dim3 grid, double bytes) {
+dbt_status launch_gemm_tc(dbt_model *m, const TcCall &c, const TcParams &p, const LmEpi &e, dim3 grid, double bytes) {
     const CUtensorMap *w1 = c.nseg > 1 ? c.W[1] : c.W[0], *w2 = c.nseg > 2 ? c.W[2] : c.W[0];
     const CUtensorMap *x = c.X;
     TcParams pp = p;
@@ -632,7 +594,7 @@ dbt_status launch_gemm_tc(dbt_model *m, const TcCall &c, const TcParams &p, cons
         if (hit != m->act3d.end()) {
             x = &hit->second;
             pp.x3d = 1;
-            pp.stacked = m->stack_planes && N_TILE <= 128 ? 1 : 0;
+            pp.stacked = N_TILE <= 128 ? 1 : 0;
         }
     }
     LAUNCH(m, c.tag, bytes, gemm_tc_kernel<N_TILE>, grid, 128, TcCfg<N_TILE>::kSmemBytes, *c.W[0], *w1, *w2, *x, pp, e);
@@ -641,7 +603,7 @@ dbt_status launch_gemm_tc(dbt_model *m, const TcCall &c, const TcParams &p, cons
 
 // Y partials P[split][R][ldp]; returns the split count and stride the consumer must use.
 dbt_status run_gemm_tc(dbt_model *m, const TcCall &c, int n_tile, int *nsplit_out, size_t *split_stride_out,
-                       int force_split = 0, FusedEpi e = FusedEpi{}) {
+                       int force_split = 0, LmEpi e = LmEpi{}, int test_skip_load = 0) {
     TcParams p{};
     int tiles = 0, col = 0;
     double bytes = 0;
@@ -664,10 +626,7 @@ dbt_status run_gemm_tc(dbt_model *m, const TcCall &c, int n_tile, int *nsplit_ou
     p.P = c.P;
     p.status = m->ws.status;
     p.evict_first = m->evict_first ? 1 : 0;
-    for (int j = 0; j < 3; j++) {
-        p.pf_ptr[j] = m->l2_prefetch ? (const char *)c.pf_ptr[j] : nullptr;
-        p.pf_bytes[j] = m->l2_prefetch && c.pf_ptr[j] ? c.pf_bytes[j] : 0;
-    }
+    p.test_skip_load = test_skip_load;
     int total_kt = (c.K + kTcK - 1) / kTcK;
     if (c.grp_cnt) force_split = 1;  // enough CTAs already: tiles x selected experts
     int split = force_split > 0 ? (force_split < total_kt ? force_split : total_kt) : choose_split(tiles, total_kt, split_slots(m, n_tile));
@@ -675,22 +634,11 @@ dbt_status run_gemm_tc(dbt_model *m, const TcCall &c, int n_tile, int *nsplit_ou
     if ((size_t)c.R * col > c.P_floats) return fail(m, DBT_ERR_CAPACITY, "partial buffer too small for %s", c.tag);
     p.kt_per_split = (total_kt + split - 1) / split;
     split = (total_kt + p.kt_per_split - 1) / p.kt_per_split;
-    if (e.mode == FE_LMHEAD) {
+    if (e.Z) {  // the output matrix has tiles enough: unsplit, logits straight from the accumulator
         split = 1;
         p.kt_per_split = total_kt;
     }
-    if (e.cluster) {  // the splits of a tile (of a gate tile and its up tile) are one cluster
-        int cap = e.mode == FE_GATEUP ? m->cluster_max / 2 : m->cluster_max;
-        if (e.mode == FE_GATEUP && split < cap) cap = split;  // keep the measured split where it fits
-        split = total_kt < cap ? total_kt : cap;
-        p.kt_per_split = (total_kt + split - 1) / split;
-        split = (total_kt + p.kt_per_split - 1) / p.kt_per_split;
-    }
-    e.arrivals = (e.mode == FE_GATEUP ? 2 : 1) * split;
-    if (e.mode != FE_NONE && tiles > 4096) return fail(m, DBT_ERR_UNSUPPORTED, "too many output tiles for %s", c.tag);
     dim3 grid(tiles, c.grp_cnt && c.grp_row_tiles ? c.grp_row_tiles : split, c.grp_cnt ? c.n_groups : 1);
-    m->next_cluster_y = e.cluster ? split : 0;
-    m->next_cluster_x = e.cluster && e.mode == FE_GATEUP ? 2 : 1;
     if (nsplit_out) *nsplit_out = split;
     if (split_stride_out) *split_stride_out = (size_t)c.R * col;
     switch (n_tile) {
@@ -779,7 +727,10 @@ dbt_status run_moe_tc(dbt_model *m, int l, const RowMap &rm, int grouped, bool r
     const LayerMaps &mp = m->maps[l];
     int Bc = rm.B * rm.cn, R = grouped ? 2 * Bc : Bc, d = c.d_model;
     int E = c.n_experts, Fe = c.d_expert, km = kmax_of(c), Fs = c.n_shared_experts * Fe, Rk = m->Rmax * km;
-    int n_tile = pad_rows(R);
+    // Row tile (and with it the resident-CTA count that sizes the split-K factors of the router and the shared
+    // expert) from the batch, never from the mode: a primary-only step uses the tile of the grouped step, so both
+    // add the same partials in the same order and write the same K/V bits.
+    int n_tile = pad_rows(2 * Bc <= 256 ? 2 * Bc : 256);
     size_t lo_x = m->act_parts == 2 ? (size_t)m->Rmax * d : 0;
     size_t lo_xs = m->act_parts == 2 ? (size_t)Rk * d : 0, lo_hs = m->act_parts == 2 ? (size_t)Rk * Fe : 0;
     const float *ssp = wide ? w.ss : nullptr;
@@ -793,7 +744,7 @@ dbt_status run_moe_tc(dbt_model *m, int l, const RowMap &rm, int grouped, bool r
     const bool matched = grouped && c.compute_matched;
     const int Rs = matched ? Bc : R;
     auto shared_expert = [&](float *Pbuf, size_t Pbuf_floats) -> dbt_status {
-        int nt = pad_rows(R);
+        int nt = n_tile;
         TcCall sg{};
         sg.W[0] = &mp.wg; sg.n_out[0] = Fs; sg.rows[0] = Rs;
         sg.W[1] = &mp.wu; sg.n_out[1] = Fs; sg.rows[1] = Rs;
@@ -927,7 +878,6 @@ dbt_status run_layers_tc(dbt_model *m, const RowMap &rm, int grouped, int n_tile
         qkv.W[1] = &mp.wk; qkv.n_out[1] = kvd; qkv.rows[1] = Bc;
         qkv.W[2] = &mp.wv; qkv.n_out[2] = kvd; qkv.rows[2] = Bc;
         qkv.nseg = 3; qkv.X = &m->map_Xb; qkv.K = d; qkv.R = Ra; qkv.P = w.P; qkv.P_floats = w.P_floats; qkv.parts = m->act_parts; qkv.lo_row0 = m->Rmax; qkv.tag = "gemm_qkv";
-        qkv.pf_ptr[0] = lw.wo; qkv.pf_bytes[0] = (size_t)d * qd * sizeof(WT);
         if ((st = run_gemm_tc(m, qkv, n_tile, &nsp, &sstride)) != DBT_OK) return st;
         const bool fuse = m->fuse_qkv && m->att_fast && rm.cn == 1;
         QkvFuse qf{w.P, nsp, sstride, mwide ? w.ss : nullptr, mwide ? mss_tiles : 0, mwide ? m->Rmax : 0, lw.coup_a};
@@ -947,10 +897,6 @@ dbt_status run_layers_tc(dbt_model *m, const RowMap &rm, int grouped, int n_tile
         TcCall op{};
         op.W[0] = &mp.wo; op.n_out[0] = d; op.rows[0] = Ra; op.nseg = 1; op.X = &m->map_Ob; op.K = qd; op.R = Ra;
         op.P = w.P; op.P_floats = w.P_floats; op.parts = m->act_parts; op.lo_row0 = m->Rmax; op.tag = "gemm_o";
-        if (!moe) {
-            op.pf_ptr[0] = lw.w_gate; op.pf_bytes[0] = (size_t)c.d_ff * d * sizeof(WT);
-            op.pf_ptr[1] = lw.w_up; op.pf_bytes[1] = (size_t)c.d_ff * d * sizeof(WT);
-        }
         if ((st = run_gemm_tc(m, op, n_tile, &nsp, &sstride)) != DBT_OK) return st;
         // S-bar_i = S_i + Attn_i W_O (matched: S-bar_2 = S_2 + g_A * Attn_1 W_O) ; RMSNorm for the MLP
         if (mwide)
@@ -966,7 +912,6 @@ dbt_status run_layers_tc(dbt_model *m, const RowMap &rm, int grouped, int n_tile
             gu.W[0] = &mp.wg; gu.n_out[0] = F; gu.rows[0] = R;
             gu.W[1] = &mp.wu; gu.n_out[1] = F; gu.rows[1] = R;
             gu.nseg = 2; gu.X = &m->map_Xb; gu.K = d; gu.R = R; gu.P = w.P; gu.P_floats = w.P_floats; gu.parts = m->act_parts; gu.lo_row0 = m->Rmax; gu.tag = "gemm_gateup";
-            gu.pf_ptr[0] = lw.w_down; gu.pf_bytes[0] = (size_t)d * F * sizeof(WT);
             if ((st = run_gemm_tc(m, gu, n_tile, &nsp, &sstride)) != DBT_OK) return st;
             dim3 sg(Bc, (F + 255) / 256);
             LAUNCH(m, "swiglu_couple", 0, swiglu_couple_kernel, sg, 256, 0, w.P, nsp, sstride, F, Bc, grouped, lw.coup_b,
@@ -974,16 +919,6 @@ dbt_status run_layers_tc(dbt_model *m, const RowMap &rm, int grouped, int n_tile
             TcCall dn{};
             dn.W[0] = &mp.wd; dn.n_out[0] = d; dn.rows[0] = R; dn.nseg = 1; dn.X = &m->map_Hb; dn.K = F; dn.R = R;
             dn.P = w.P; dn.P_floats = w.P_floats; dn.parts = m->act_parts; dn.lo_row0 = m->Rmax; dn.tag = "gemm_down";
-            if (l + 1 < c.n_layers) {
-                const dbt_layer_weights &nx = m->layers[l + 1];
-                dn.pf_ptr[0] = nx.wq; dn.pf_bytes[0] = (size_t)qd * d * sizeof(WT);
-                dn.pf_ptr[1] = nx.wk; dn.pf_bytes[1] = (size_t)kvd * d * sizeof(WT);
-                dn.pf_ptr[2] = nx.wv; dn.pf_bytes[2] = (size_t)kvd * d * sizeof(WT);
-            } else {
-                dn.pf_ptr[0] = m->w.lm_head;  // the first 48 MB of the output matrix
-                size_t lmb = (size_t)c.vocab * d * sizeof(WT);
-                dn.pf_bytes[0] = lmb < ((size_t)48 << 20) ? lmb : ((size_t)48 << 20);
-            }
             if ((st = run_gemm_tc(m, dn, n_tile, &nsp, &sstride)) != DBT_OK) return st;
             mode = 2;
         } else {
@@ -1071,171 +1006,12 @@ dbt_status prefill_tc(dbt_model *m, const int32_t *tokens_dev, int B, int n, flo
     return DBT_OK;
 }
 
-// ---- fused dense path: 4 GEMMs + attention per layer, no kernel between them ----------------
-
-FusedEpi epi_base(dbt_model *m, const RowMap &rm, int grouped, int mode) {
-    const dbt_config &c = m->cfg;
-    FusedEpi e{};
-    e.mode = mode;
-    e.Bc = rm.B * rm.cn;
-    e.grouped = grouped;
-    e.rm = rm;
-    e.tickets = m->ws.gemm_tickets;
-    e.ss_in = m->ws.ss;
-    e.ss_tiles = (c.d_model + 127) / 128;
-    e.ss_ld = m->Rmax;
-    e.d_norm = c.d_model;
-    e.eps = c.rms_eps;
-    e.use_scale = 1;
-    return e;
-}
-
-dbt_status run_layers_fused(dbt_model *m, const RowMap &rm, int grouped, int n_tile) {
-    typedef __nv_bfloat16 WT;
-    const dbt_config &c = m->cfg;
-    const Workspace &w = m->ws;
-    int Bc = rm.B * rm.cn, R = grouped ? 2 * Bc : Bc;
-    int d = c.d_model, qd = c.n_q_heads * c.head_dim, kvd = c.n_kv_heads * c.head_dim, F = c.d_ff;
-    size_t pool_layer_elems = (size_t)2 * c.num_pages * c.n_kv_heads * c.page_size * c.head_dim;
-    size_t lo_x = m->act_parts == 2 ? (size_t)m->Rmax * d : 0, lo_h = m->act_parts == 2 ? (size_t)m->Rmax * F : 0;
-    double kv_bytes = 0;
-    for (int b = 0; b < rm.B; b++)
-        for (int j = 0; j < rm.cn; j++) kv_bytes += (double)(m->len_host[b] + j + 1) * 2 * kvd * sizeof(WT);
-    dbt_status st;
-    auto call = [&](const char *tag, const CUtensorMap *X, int K) {
-        TcCall t{};
-        t.X = X; t.K = K; t.R = R; t.P = w.P; t.P_floats = w.P_floats; t.tag = tag;
-        t.parts = m->act_parts; t.lo_row0 = m->Rmax;
-        return t;
-    };
-    for (int l = 0; l < c.n_layers; l++) {
-        const dbt_layer_weights &lw = m->layers[l];
-        const LayerMaps &mp = m->maps[l];
-        WT *kpool = reinterpret_cast<WT *>(m->kv_pool) + (size_t)l * pool_layer_elems;
-        // Q|K|V with 1/rms, RoPE, the a coupling and the cache append in the epilogue
-        TcCall qkv = call("gemm_qkv", &m->map_Xb, d);
-        qkv.W[0] = &mp.wq; qkv.n_out[0] = qd; qkv.rows[0] = R;
-        qkv.W[1] = &mp.wk; qkv.n_out[1] = kvd; qkv.rows[1] = Bc;
-        qkv.W[2] = &mp.wv; qkv.n_out[2] = kvd; qkv.rows[2] = Bc;
-        qkv.nseg = 3;
-        FusedEpi eq = epi_base(m, rm, grouped, FE_QKV);
-        eq.coup = lw.coup_a; eq.Q = w.Q; eq.rope = w.rope; eq.seq_len = w.seq_len; eq.page_table = w.page_table;
-        eq.pt_stride = m->pages_per_seq_max; eq.num_pages = c.num_pages; eq.n_q = c.n_q_heads; eq.n_kv = c.n_kv_heads;
-        eq.dh = c.head_dim; eq.kpool = kpool; eq.vpool = kpool + pool_layer_elems / 2;
-        if ((st = run_gemm_tc(m, qkv, n_tile, nullptr, nullptr, 0, eq)) != DBT_OK) return st;
-        st = c.head_dim == 128 ? run_attention_mma<128>(m, rm, grouped, l, kv_bytes)
-                               : run_attention_mma<64>(m, rm, grouped, l, kv_bytes);
-        if (st != DBT_OK) return st;
-        // S-bar = S + Attn W_O; next input g_mlp * S-bar
-        TcCall op = call("gemm_o", &m->map_Ob, qd);
-        op.W[0] = &mp.wo; op.n_out[0] = d; op.rows[0] = R; op.nseg = 1;
-        FusedEpi eo = epi_base(m, rm, grouped, FE_RESID);
-        eo.use_scale = 0; eo.S = w.S; eo.g_next = lw.mlp_norm_g; eo.Xout = w.Xb; eo.lo_off = lo_x; eo.ld_out = d; eo.ss_out = w.ss;
-        if ((st = run_gemm_tc(m, op, n_tile, nullptr, nullptr, 0, eo)) != DBT_OK) return st;
-        // gate|up with 1/rms, SwiGLU and the b coupling
-        TcCall gu = call("gemm_gateup", &m->map_Xb, d);
-        gu.W[0] = &mp.wg; gu.n_out[0] = F; gu.rows[0] = R;
-        gu.W[1] = &mp.wu; gu.n_out[1] = F; gu.rows[1] = R;
-        gu.nseg = 2;
-        FusedEpi eg = epi_base(m, rm, grouped, FE_GATEUP);
-        eg.coup = lw.coup_b; eg.Xout = w.Hb; eg.lo_off = lo_h; eg.ld_out = F;
-        if ((st = run_gemm_tc(m, gu, n_tile, nullptr, nullptr, 0, eg)) != DBT_OK) return st;
-        // down with the c coupling and the residual; next input for layer l+1 (or the output matrix)
-        TcCall dn = call("gemm_down", &m->map_Hb, F);
-        dn.W[0] = &mp.wd; dn.n_out[0] = d; dn.rows[0] = R; dn.nseg = 1;
-        FusedEpi ed = epi_base(m, rm, grouped, FE_DOWN);
-        ed.use_scale = 0; ed.coup = lw.coup_c; ed.S = w.S; ed.Xout = w.Xb; ed.lo_off = lo_x; ed.ld_out = d; ed.ss_out = w.ss;
-        ed.g_next = l + 1 < c.n_layers ? m->layers[l + 1].attn_norm_g : (c.final_norm ? m->w.final_norm_g : nullptr);
-        if ((st = run_gemm_tc(m, dn, n_tile, nullptr, nullptr, 0, ed)) != DBT_OK) return st;
-    }
-    return DBT_OK;
-}
-
-dbt_status run_head_fused(dbt_model *m, const RowMap &rm, int grouped, int n_tile) {
-    const dbt_config &c = m->cfg;
-    const Workspace &w = m->ws;
-    int R = (grouped ? 2 : 1) * rm.B * rm.cn;
-    TcCall lm{};
-    lm.W[0] = &m->map_lm; lm.n_out[0] = c.vocab; lm.rows[0] = R; lm.nseg = 1; lm.X = &m->map_Xb; lm.K = c.d_model;
-    lm.R = R; lm.P = w.Z; lm.P_floats = (size_t)R * c.vocab; lm.tag = "gemm_lm_head";
-    lm.parts = m->act_parts; lm.lo_row0 = m->Rmax;
-    FusedEpi e = epi_base(m, rm, grouped, FE_LMHEAD);
-    e.use_scale = c.final_norm;
-    e.Z = w.Z;
-    return run_gemm_tc(m, lm, n_tile, nullptr, nullptr, 0, e);
-}
-
-template <typename WT>
-dbt_status run_embed_fused(dbt_model *m, const int32_t *tokens_dev, int n, int p0, const RowMap &rm, int R) {
-    const dbt_config &c = m->cfg;
-    const Workspace &w = m->ws;
-    LAUNCH(m, "embed", 0, embed_fused_kernel<WT>, R, 256, 0, tokens_dev, n, p0, rm, (const WT *)m->w.embed_primary,
-           (const WT *)m->w.embed_branch, m->w.embed_norm_g, c.rms_eps, c.d_model, c.vocab, w.S,
-           m->layers[0].attn_norm_g, w.Xb, m->act_parts == 2 ? (size_t)m->Rmax * c.d_model : (size_t)0, w.ss, m->Rmax,
-           (c.d_model + 127) / 128, w.status);
-    return DBT_OK;
-}
-
-dbt_status step_fused(dbt_model *m, const int32_t *tokens_dev, int B, int grouped, int32_t *next_dev, float *z1_dev,
-                      float *z2_dev, float *alpha_dev) {
-    typedef __nv_bfloat16 WT;
-    const dbt_config &c = m->cfg;
-    const Workspace &w = m->ws;
-    RowMap rm{B, 1};
-    int R = grouped ? 2 * B : B, n_tile = pad_rows(2 * B);
-    dbt_status st;
-    if ((st = run_embed_fused<WT>(m, tokens_dev, 1, 0, rm, R)) != DBT_OK) return st;
-    if ((st = run_layers_fused(m, rm, grouped, n_tile)) != DBT_OK) return st;
-    if ((st = run_head_fused(m, rm, grouped, n_tile)) != DBT_OK) return st;
-    // the readout also bumps the sequence lengths: nothing after it in the step reads them
-    if ((st = run_readout(m, B, grouped, next_dev, alpha_dev)) != DBT_OK) return st;
-    size_t zb = sizeof(float) * (size_t)B * c.vocab;
-    if (z1_dev) CUDA_TRY(m, cudaMemcpyAsync(z1_dev, w.Z, zb, cudaMemcpyDeviceToDevice, m->stream));
-    if (z2_dev && grouped)
-        CUDA_TRY(m, cudaMemcpyAsync(z2_dev, w.Z + (size_t)B * c.vocab, zb, cudaMemcpyDeviceToDevice, m->stream));
-    for (int b = 0; b < B; b++) m->len_host[b] += 1;
-    return DBT_OK;
-}
-
-dbt_status prefill_fused(dbt_model *m, const int32_t *tokens_dev, int B, int n, float *last_logits) {
-    typedef __nv_bfloat16 WT;
-    const dbt_config &c = m->cfg;
-    const Workspace &w = m->ws;
-    int cn_max = (m->Rmax < kAttMaxItems ? m->Rmax : kAttMaxItems) / B;
-    if (cn_max < 1) cn_max = 1;
-    // when logits are wanted the last position runs as its own chunk, so that the rows of the
-    // output-matrix GEMM are exactly the B last positions
-    int n_bulk = last_logits ? n - 1 : n;
-    dbt_status st;
-    for (int p0 = 0; p0 < n;) {
-        int cn = p0 < n_bulk ? (n_bulk - p0 < cn_max ? n_bulk - p0 : cn_max) : 1;
-        RowMap rm{B, cn};
-        int R = B * cn, n_tile = pad_rows(R);
-        if ((st = run_embed_fused<WT>(m, tokens_dev, n, p0, rm, R)) != DBT_OK) return st;
-        if ((st = run_layers_fused(m, rm, 0, n_tile)) != DBT_OK) return st;
-        if (last_logits && p0 + cn >= n) {
-            if ((st = run_head_fused(m, rm, 0, n_tile)) != DBT_OK) return st;
-            CUDA_TRY(m, cudaMemcpyAsync(last_logits, w.Z, sizeof(float) * (size_t)B * c.vocab, cudaMemcpyDeviceToDevice,
-                                        m->stream));
-        }
-        LAUNCH(m, "advance_len", 0, advance_len_kernel, (B + 127) / 128, 128, 0, w.seq_len, B, cn);
-        for (int b = 0; b < B; b++) m->len_host[b] += cn;  // the next chunk's byte accounting sees the new lengths
-        p0 += cn;
-    }
-    return DBT_OK;
-}
-
 // ---- dense bf16 path with the RMSNorm factor applied after the GEMM ---------------------------
 // No kernel of this chain reduces over a whole row: the residual kernel is column-parallel and
 // leaves per-block shares of sum(S^2); the kernels after the Q|K|V and gate|up GEMMs (and the
 // output-matrix GEMM's own epilogue) multiply by 1/rms.  9 kernels per layer.
 
-// Up to a row tile of 64 the O and down projections finish their own output (cluster reduction of the
-// split-K partials + residual epilogue); their shares of sum(S^2) are then per 128-column tile.
-bool wide_cluster(const dbt_model *m, int n_tile) { return m->cluster_epi && n_tile <= 64; }
-int wide_ss_tiles(const dbt_model *m, int n_tile) {
-    return wide_cluster(m, n_tile) ? (m->cfg.d_model + 127) / 128 : (m->cfg.d_model + 255) / 256;
-}
+int wide_ss_tiles(const dbt_model *m) { return (m->cfg.d_model + 255) / 256; }
 
 dbt_status run_layers_wide(dbt_model *m, const RowMap &rm, int grouped, int n_tile) {
     typedef __nv_bfloat16 WT;
@@ -1245,8 +1021,7 @@ dbt_status run_layers_wide(dbt_model *m, const RowMap &rm, int grouped, int n_ti
     int d = c.d_model, qd = c.n_q_heads * c.head_dim, kvd = c.n_kv_heads * c.head_dim, F = c.d_ff;
     size_t pool_layer_elems = (size_t)2 * c.num_pages * c.n_kv_heads * c.page_size * c.head_dim;
     size_t lo_x = m->act_parts == 2 ? (size_t)m->Rmax * d : 0, lo_h = m->act_parts == 2 ? (size_t)m->Rmax * F : 0;
-    const bool clustered = wide_cluster(m, n_tile);
-    int ss_tiles = wide_ss_tiles(m, n_tile), ss_ld = m->Rmax;
+    int ss_tiles = wide_ss_tiles(m), ss_ld = m->Rmax;
     double kv_bytes = 0;
     for (int b = 0; b < rm.B; b++)
         for (int j = 0; j < rm.cn; j++) kv_bytes += (double)(m->len_host[b] + j + 1) * 2 * kvd * sizeof(WT);
@@ -1282,11 +1057,7 @@ dbt_status run_layers_wide(dbt_model *m, const RowMap &rm, int grouped, int n_ti
         if (st != DBT_OK) return st;
         TcCall op = call("gemm_o", &m->map_Ob, qd);
         op.W[0] = &mp.wo; op.n_out[0] = d; op.rows[0] = R; op.nseg = 1;
-        if (clustered) {
-            FusedEpi eo = epi_base(m, rm, grouped, FE_RESID);
-            eo.cluster = 1; eo.S = w.S; eo.g_next = lw.mlp_norm_g; eo.Xout = w.Xb; eo.lo_off = lo_x; eo.ld_out = d; eo.ss_out = w.ss;
-            if ((st = run_gemm_tc(m, op, n_tile, nullptr, nullptr, 0, eo)) != DBT_OK) return st;
-        } else {
+        {
             if ((st = run_gemm_tc(m, op, n_tile, &nsp, &sstride)) != DBT_OK) return st;
             LAUNCH(m, "resid_wide", 0, resid_wide_kernel, dim3(Bc, ss_tiles), 256, 0, w.S, w.P, nsp, sstride, 1,
                    (const float *)nullptr, Bc, grouped, lw.mlp_norm_g, d, w.Xb, lo_x, w.ss, ss_ld);
@@ -1295,11 +1066,7 @@ dbt_status run_layers_wide(dbt_model *m, const RowMap &rm, int grouped, int n_ti
         gu.W[0] = &mp.wg; gu.n_out[0] = F; gu.rows[0] = R;
         gu.W[1] = &mp.wu; gu.n_out[1] = F; gu.rows[1] = R;
         gu.nseg = 2;
-        if (m->cluster_gu && n_tile <= 64) {
-            FusedEpi eg = epi_base(m, rm, grouped, FE_GATEUP);
-            eg.cluster = 1; eg.ss_tiles = ss_tiles; eg.coup = lw.coup_b; eg.Xout = w.Hb; eg.lo_off = lo_h; eg.ld_out = F;
-            if ((st = run_gemm_tc(m, gu, n_tile, nullptr, nullptr, 0, eg)) != DBT_OK) return st;
-        } else {
+        {
             if ((st = run_gemm_tc(m, gu, n_tile, &nsp, &sstride)) != DBT_OK) return st;
             LAUNCH(m, "swiglu_couple", 0, swiglu_couple_kernel, dim3(Bc, (F + 255) / 256), 256, 0, w.P, nsp, sstride, F, Bc,
                    grouped, lw.coup_b, w.Hb, lo_h, (const float *)w.ss, ss_tiles, ss_ld, d, c.rms_eps);
@@ -1308,12 +1075,7 @@ dbt_status run_layers_wide(dbt_model *m, const RowMap &rm, int grouped, int n_ti
         dn.W[0] = &mp.wd; dn.n_out[0] = d; dn.rows[0] = R; dn.nseg = 1;
         const float *g_next = l + 1 < c.n_layers ? m->layers[l + 1].attn_norm_g
                                                  : (c.final_norm ? m->w.final_norm_g : (const float *)nullptr);
-        if (clustered) {
-            FusedEpi ed = epi_base(m, rm, grouped, FE_DOWN);
-            ed.cluster = 1; ed.coup = lw.coup_c; ed.S = w.S; ed.g_next = g_next; ed.Xout = w.Xb; ed.lo_off = lo_x; ed.ld_out = d;
-            ed.ss_out = w.ss;
-            if ((st = run_gemm_tc(m, dn, n_tile, nullptr, nullptr, 0, ed)) != DBT_OK) return st;
-        } else {
+        {
             if ((st = run_gemm_tc(m, dn, n_tile, &nsp, &sstride)) != DBT_OK) return st;
             LAUNCH(m, "resid_wide", 0, resid_wide_kernel, dim3(Bc, ss_tiles), 256, 0, w.S, w.P, nsp, sstride, 2, lw.coup_c, Bc,
                    grouped, g_next, d, w.Xb, lo_x, w.ss, ss_ld);
@@ -1330,10 +1092,14 @@ dbt_status run_head_wide(dbt_model *m, const RowMap &rm, int grouped, int n_tile
     lm.W[0] = &m->map_lm; lm.n_out[0] = c.vocab; lm.rows[0] = R; lm.nseg = 1; lm.X = &m->map_Xb; lm.K = c.d_model;
     lm.R = R; lm.P = w.Z; lm.P_floats = (size_t)R * c.vocab; lm.tag = "gemm_lm_head";
     lm.parts = m->act_parts; lm.lo_row0 = m->Rmax;
-    FusedEpi e = epi_base(m, rm, grouped, FE_LMHEAD);
-    e.ss_tiles = wide_ss_tiles(m, n_tile);
-    e.use_scale = c.final_norm;
+    LmEpi e{};
     e.Z = w.Z;
+    e.ss_in = w.ss;
+    e.ss_tiles = wide_ss_tiles(m);
+    e.ss_ld = m->Rmax;
+    e.d_norm = c.d_model;
+    e.use_scale = c.final_norm;
+    e.eps = c.rms_eps;
     return run_gemm_tc(m, lm, n_tile, nullptr, nullptr, 0, e);
 }
 
@@ -1344,7 +1110,7 @@ dbt_status run_embed_wide(dbt_model *m, const int32_t *tokens_dev, int n, int p0
     LAUNCH(m, "embed", 0, embed_fused_kernel<WT>, R, 256, 0, tokens_dev, n, p0, rm, (const WT *)m->w.embed_primary,
            (const WT *)m->w.embed_branch, m->w.embed_norm_g, c.rms_eps, c.d_model, c.vocab, w.S,
            m->layers[0].attn_norm_g, w.Xb, m->act_parts == 2 ? (size_t)m->Rmax * c.d_model : (size_t)0, w.ss, m->Rmax,
-           wide_ss_tiles(m, n_tile), w.status);
+           wide_ss_tiles(m), w.status);
     return DBT_OK;
 }
 
@@ -1398,199 +1164,14 @@ dbt_status prefill_wide(dbt_model *m, const int32_t *tokens_dev, int B, int n, f
 }
 
 
-// ---- dense bf16, small batch: the whole decode step as one persistent kernel -------------------
-
-template <int N_TILE, int DH>
-bool mega_allow() {
-    if (cudaFuncSetAttribute(mega_decode_kernel<N_TILE, DH>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             MegaCfg<N_TILE, DH>::kSmemBytes) != cudaSuccess)
-        return false;
-    int per_sm = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, mega_decode_kernel<N_TILE, DH>, kMegaThreads,
-                                                      MegaCfg<N_TILE, DH>::kSmemBytes) != cudaSuccess)
-        return false;
-    return per_sm >= 1;
-}
-
-bool mega_eligible(const dbt_model *m, int B) {
-    if (!m->mega) return false;
-    const dbt_config &c = m->cfg;
-    int n_tile = pad_rows(2 * B);
-    if (n_tile > 64 || B > 32) return false;
-    int vt = (c.vocab + 127) / 128, ft = 2 * ((c.d_ff + 127) / 128);
-    int qt = (c.n_q_heads * c.head_dim + 127) / 128 + 2 * ((c.n_kv_heads * c.head_dim + 127) / 128);
-    int tiles = vt > ft ? vt : ft;
-    if (qt > tiles) tiles = qt;
-    if ((size_t)(m->num_sms + tiles) * n_tile * 128 > m->ws.P_floats) return false;
-    if (m->num_sms + B * c.n_kv_heads > m->part_items) return false;
-    return true;
-}
-
-// The plan of a (batch, mode) pair lives in device memory; it is written once, outside any capture.
-dbt_status mega_prepare(dbt_model *m, int B, int grouped, int *slot_out) {
-    for (size_t i = 0; i < m->mega_slots.size(); i++)
-        if (m->mega_slots[i].B == B && m->mega_slots[i].grouped == grouped) {
-            *slot_out = (int)i;
-            return DBT_OK;
-        }
-    if ((int)m->mega_slots.size() >= kMegaPlanSlots) {
-        *slot_out = -1;
-        return DBT_OK;
-    }
-    const dbt_config &c = m->cfg;
-    const Workspace &w = m->ws;
-    MegaPlan p;
-    memset(&p, 0, sizeof p);
-    int d = c.d_model, qd = c.n_q_heads * c.head_dim;
-    p.B = B; p.grouped = grouped; p.R = grouped ? 2 * B : B; p.L = c.n_layers; p.d = d; p.n_q = c.n_q_heads;
-    p.n_kv = c.n_kv_heads; p.dh = c.head_dim; p.F = c.d_ff; p.V = c.vocab; p.Rmax = m->Rmax; p.final_norm = c.final_norm;
-    p.num_pages = c.num_pages; p.pt_stride = m->pages_per_seq_max; p.eps = c.rms_eps;
-    p.S = w.S; p.Q = w.Q; p.P = w.P; p.ss = w.ss; p.Z = w.Z; p.part = w.part; p.rd_part = w.rd_part; p.rd_best = w.rd_best;
-    p.Xb = w.Xb; p.Ob = w.Ob; p.Hb = w.Hb; p.pool = reinterpret_cast<__nv_bfloat16 *>(m->kv_pool);
-    p.lo_x = (size_t)m->Rmax * d; p.lo_o = (size_t)m->Rmax * qd; p.lo_h = (size_t)m->Rmax * c.d_ff;
-    p.rope = w.rope; p.seq_len = w.seq_len; p.page_table = w.page_table; p.att_tickets = w.att_tickets; p.status = w.status;
-    p.bar_count = w.mega_sync; p.done_count = w.mega_sync + 1; p.err = reinterpret_cast<int *>(w.mega_sync + 2);
-    p.maps = w.mega_maps;
-    p.E1 = (const __nv_bfloat16 *)m->w.embed_primary; p.E2 = (const __nv_bfloat16 *)m->w.embed_branch;
-    p.g_e = m->w.embed_norm_g; p.g_first = m->layers[0].attn_norm_g;
-    p.plane_rows = (long long)c.num_pages * c.n_kv_heads * c.page_size;
-    for (int l = 0; l < c.n_layers; l++) {
-        const dbt_layer_weights &lw = m->layers[l];
-        p.layer[l].coup_a = lw.coup_a; p.layer[l].coup_b = lw.coup_b; p.layer[l].coup_c = lw.coup_c;
-        p.layer[l].g_mlp = lw.mlp_norm_g;
-        p.layer[l].g_next = l + 1 < c.n_layers ? m->layers[l + 1].attn_norm_g
-                                               : (c.final_norm ? m->w.final_norm_g : (const float *)nullptr);
-    }
-    int slot = (int)m->mega_slots.size();
-    CUDA_TRY(m, cudaMemcpy(w.mega_plans + (size_t)slot * align_up(sizeof(MegaPlan)), &p, sizeof p, cudaMemcpyHostToDevice));
-    m->mega_slots.push_back(dbt_model::MegaSlot{B, grouped});
-    *slot_out = slot;
-    return DBT_OK;
-}
-
-template <int N_TILE, int DH>
-cudaError_t mega_launch(dbt_model *m, const MegaPlan *plan, const int32_t *tokens, int32_t *next, float *alpha) {
-    cudaLaunchConfig_t cfg{};
-    cfg.gridDim = dim3(m->num_sms);
-    cfg.blockDim = dim3(kMegaThreads);
-    cfg.dynamicSmemBytes = MegaCfg<N_TILE, DH>::kSmemBytes;
-    cfg.stream = m->stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeCooperative;  // all CTAs resident at once: they meet at grid barriers
-    attr[0].val.cooperative = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, mega_decode_kernel<N_TILE, DH>, plan, tokens, next, alpha);
-}
-
-dbt_status step_mega(dbt_model *m, int slot, const int32_t *tokens_dev, int B, int grouped, int32_t *next_dev,
-                     float *z1_dev, float *z2_dev, float *alpha_dev) {
-    const dbt_config &c = m->cfg;
-    const Workspace &w = m->ws;
-    const MegaPlan *plan = reinterpret_cast<const MegaPlan *>(w.mega_plans + (size_t)slot * align_up(sizeof(MegaPlan)));
-    int n_tile = pad_rows(2 * B);
-    double bytes = 0;
-    if (m->prof_on) {
-        int qd = c.n_q_heads * c.head_dim, kvd = c.n_kv_heads * c.head_dim;
-        bytes = ((double)c.n_layers * ((double)(qd + 2 * kvd) * c.d_model + (double)c.d_model * qd + 3.0 * c.d_ff * c.d_model) +
-                 (double)c.vocab * c.d_model) * 2;
-        for (int b = 0; b < B; b++) bytes += (double)(m->len_host[b] + 1) * 2 * kvd * 2 * c.n_layers;
-    }
-    cudaEvent_t p0 = nullptr, p1 = nullptr;
-    if (m->prof_on) {
-        p0 = prof_event(m);
-        p1 = prof_event(m);
-        cudaEventRecord(p0, m->stream);
-    }
-    cudaError_t e = cudaErrorInvalidValue;
-    if (c.head_dim == 128) {
-        if (n_tile == 16) e = mega_launch<16, 128>(m, plan, tokens_dev, next_dev, alpha_dev);
-        else if (n_tile == 32) e = mega_launch<32, 128>(m, plan, tokens_dev, next_dev, alpha_dev);
-        else e = mega_launch<64, 128>(m, plan, tokens_dev, next_dev, alpha_dev);
-    } else {
-        if (n_tile == 16) e = mega_launch<16, 64>(m, plan, tokens_dev, next_dev, alpha_dev);
-        else if (n_tile == 32) e = mega_launch<32, 64>(m, plan, tokens_dev, next_dev, alpha_dev);
-        else e = mega_launch<64, 64>(m, plan, tokens_dev, next_dev, alpha_dev);
-    }
-    m->launches++;
-    if (m->prof_on) {
-        cudaEventRecord(p1, m->stream);
-        m->prof.push_back(dbt_model::ProfRec{"mega_decode_step", bytes, p0, p1});
-    }
-    if (e != cudaSuccess) return fail(m, DBT_ERR_CUDA, "launch mega_decode_kernel: %s", cudaGetErrorString(e));
-    size_t zb = sizeof(float) * (size_t)B * c.vocab;
-    if (z1_dev) CUDA_TRY(m, cudaMemcpyAsync(z1_dev, w.Z, zb, cudaMemcpyDeviceToDevice, m->stream));
-    if (z2_dev && grouped)
-        CUDA_TRY(m, cudaMemcpyAsync(z2_dev, w.Z + (size_t)B * c.vocab, zb, cudaMemcpyDeviceToDevice, m->stream));
-    for (int b = 0; b < B; b++) m->len_host[b] += 1;
-    return DBT_OK;
-}
-
-bool setup_mega(dbt_model *m) {
-    const dbt_config &c = m->cfg;
-    const char *mg = getenv("DBT_MEGA");
-    if (!(mg && strcmp(mg, "1") == 0)) return false;
-    if (!m->tc || !m->att_fast || c.n_experts > 0 || m->act_parts != 2 || c.n_layers > kMegaMaxLayers) return false;
-    if (c.head_dim != 64 && c.head_dim != 128) return false;
-    if (c.page_size != 16 || m->num_sms > kMegaMaxCtas) return false;
-    int dev = 0, coop = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return false;
-    cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
-    if (!coop) return false;
-    bool ok = c.head_dim == 128 ? (mega_allow<16, 128>() && mega_allow<32, 128>() && mega_allow<64, 128>())
-                                : (mega_allow<16, 64>() && mega_allow<32, 64>() && mega_allow<64, 64>());
-    if (!ok) {
-        cudaGetLastError();
-        return false;
-    }
-    const Workspace &w = m->ws;
-    std::vector<CUtensorMap> maps((size_t)c.n_layers * 7 + kMegaTailMaps);
-    for (int l = 0; l < c.n_layers; l++) {
-        const LayerMaps &mp = m->maps[l];
-        CUtensorMap *o = maps.data() + (size_t)l * 7;
-        o[0] = mp.wq; o[1] = mp.wk; o[2] = mp.wv; o[3] = mp.wo; o[4] = mp.wg; o[5] = mp.wu; o[6] = mp.wd;
-    }
-    CUtensorMap *t = maps.data() + (size_t)c.n_layers * 7;
-    t[0] = m->map_lm;
-    t[1] = m->map_kv;
-    bool mok = true;
-    for (int i = 0; i < 3 && mok; i++) {
-        uint32_t nt = 16u << i;
-        mok = make_act_map(&t[2 + 3 * i + 0], w.Xb, m->Rmax, c.d_model, nt) &&
-              make_act_map(&t[2 + 3 * i + 1], w.Ob, m->Rmax, (uint64_t)c.n_q_heads * c.head_dim, nt) &&
-              make_act_map(&t[2 + 3 * i + 2], w.Hb, m->Rmax, c.d_ff, nt);
-    }
-    if (!mok) return false;
-    if (cudaMemcpy(w.mega_maps, maps.data(), maps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice) != cudaSuccess ||
-        cudaMemset(w.mega_sync, 0, sizeof(unsigned int) * 8) != cudaSuccess) {
-        cudaGetLastError();
-        return false;
-    }
-    return true;
-}
-
 template <int N_TILE>
 bool allow_smem() {
     return cudaFuncSetAttribute(gemm_tc_kernel<N_TILE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 TcCfg<N_TILE>::kSmemBytes) == cudaSuccess;
 }
-// Clusters of 16 CTAs need an opt-in per kernel; without it the clustered epilogue uses 8.
-bool allow_cluster16() {
-    static int state = 0;
-    if (state == 0) {
-        bool ok = cudaFuncSetAttribute(gemm_tc_kernel<16>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess &&
-                  cudaFuncSetAttribute(gemm_tc_kernel<32>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess &&
-                  cudaFuncSetAttribute(gemm_tc_kernel<64>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess;
-        if (!ok) cudaGetLastError();
-        state = ok ? 1 : -1;
-    }
-    return state == 1;
-}
+// The attribute is per device: set it on every call for the device that is current (it is cheap).
 bool allow_smem_all() {
-    static int state = 0;  // 0 unknown, 1 ok, -1 failed
-    if (state == 0)
-        state = (allow_smem<16>() && allow_smem<32>() && allow_smem<64>() && allow_smem<128>() && allow_smem<256>()) ? 1 : -1;
-    return state == 1;
+    return allow_smem<16>() && allow_smem<32>() && allow_smem<64>() && allow_smem<128>() && allow_smem<256>();
 }
 
 // Build the TMA descriptors of a bf16 model.  Returns false when the path cannot be used.
@@ -1661,19 +1242,10 @@ bool setup_tc(dbt_model *m) {
                                        AttCfg<64>::kSmemBytes) == cudaSuccess &&
                   cudaFuncSetAttribute(attn_mma_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        AttCfg<64>::kSmemBytes) == cudaSuccess;
-    const char *fu = getenv("DBT_FUSED");
-    // Opt-in (DBT_FUSED=1): measured slower than the separate elementwise kernels at batch 16
-    // (1.96 ms vs 1.55 ms per step on the 1B model): the tile's last CTA folds the split-K
-    // partials alone, on 16..44 SMs, while the separate kernels spread that work over the GPU
-    // and overlap with their neighbours through programmatic dependent launch.
-    m->fused = ok && m->att_fast && !moe && (fu && strcmp(fu, "1") == 0);
-    const char *wi = getenv("DBT_WIDE");
     // Default chain of a dense bf16 model: the RMSNorm factor is applied after the GEMM, so no kernel
-    // reduces over a whole row (9 kernels per layer; 1.37 vs 1.42 ms per step at batch 16 on the 1B
-    // model against the chain with a row-wide residual+norm kernel, which DBT_WIDE=0 selects).
-    m->wide = ok && m->att_fast && !moe && !m->fused && !(wi && strcmp(wi, "0") == 0);
-    const char *split = getenv("DBT_ACT_SPLIT");
-    m->act_parts = (split && strcmp(split, "0") == 0) ? 1 : 2;
+    // reduces over a whole row.
+    m->wide = ok && m->att_fast && !moe;
+    m->act_parts = 2;
     return ok;
 }
 
@@ -1809,38 +1381,11 @@ dbt_status dbt_create(const dbt_config *cfg, const dbt_weights *w, void *kv_pool
         m->num_sms = sms > 0 && sms <= 148 ? sms : 148;  // the partial buffer is sized for 2 x 148 CTAs
     }
     m->tc = setup_tc(m);
-    m->mega = false;
-    m->mega = setup_mega(m);
     {
-        // Opt-in (DBT_L2_PREFETCH=1): measured no faster (1.49 vs 1.45 ms per step at batch 16 on the
-        // 1B model); the GEMMs of a decode step wait on dependency latency, not on HBM bandwidth.
-        // Opt-in (DBT_CLUSTER=1): the splits of an O / down projection tile as one thread-block cluster that
-        // reduces through distributed shared memory and applies the residual itself.  Measured equal to
-        // the separate residual kernel (1.12 vs 1.12 ms per step at batch 16 on the 1B model): a cluster
-        // is at most 8 CTAs, so the projections run with 8 splits instead of 15-16 and their longer
-        // chains cost what the removed kernel saves; 16-CTA clusters (DBT_CLUSTER_MAX=16) schedule
-        // badly (1.29 ms).
-        // Opt-in (DBT_CLUSTER_GU=1): {gate tile, up tile} x splits as one cluster that applies SwiGLU and the
-        // b coupling itself.  Measured slower than the separate kernel (1.16 vs 1.12 ms per step at batch
-        // 16 on the 1B model): six CTAs finish 16 row pairs of a 128-feature tile on the GEMM's critical
-        // path, where the separate kernel spreads the same work over 352 blocks.
-        const char *cg = getenv("DBT_CLUSTER_GU");
-        m->cluster_gu = cg && strcmp(cg, "1") == 0;
-        const char *cl = getenv("DBT_CLUSTER");
-        m->cluster_epi = cl && strcmp(cl, "1") == 0;
-        m->next_cluster_y = 0;
-        const char *cm = getenv("DBT_CLUSTER_MAX");
-        m->cluster_max = 8;
-        if (cm && atoi(cm) == 16 && m->tc && allow_cluster16()) m->cluster_max = 16;
-        else if (cm && atoi(cm) >= 2 && atoi(cm) <= 8) m->cluster_max = atoi(cm);
-        const char *sp = getenv("DBT_STACK");
-        m->stack_planes = !(sp && strcmp(sp, "0") == 0);
         const char *ef = getenv("DBT_EVICT_FIRST");
         m->evict_first = !(ef && strcmp(ef, "0") == 0);
         const char *fq = getenv("DBT_FUSE_QKV");
         m->fuse_qkv = m->att_fast && !(fq && strcmp(fq, "0") == 0);
-        const char *pf = getenv("DBT_L2_PREFETCH");
-        m->l2_prefetch = pf && strcmp(pf, "1") == 0;
     }
     const char *ro = getenv("DBT_READOUT");
     m->readout_row = ro && strcmp(ro, "row") == 0;
@@ -1859,8 +1404,7 @@ dbt_status dbt_create(const dbt_config *cfg, const dbt_weights *w, void *kv_pool
         const char *rt = getenv("DBT_MOE_ROWTILE");
         m->moe_row_tile = rt ? atoi(rt) : -1;
         if (m->moe_row_tile != 0 && m->moe_row_tile != 16 && m->moe_row_tile != 32 && m->moe_row_tile != 64) m->moe_row_tile = -1;
-        const char *mw = getenv("DBT_MOE_WIDE");
-        m->moe_wide = m->moe_tc && m->act_parts == 2 && !(mw && strcmp(mw, "0") == 0);
+        m->moe_wide = m->moe_tc && m->act_parts == 2;
         if (m->moe_overlap &&
             (cudaStreamCreateWithFlags(&m->side_stream, cudaStreamNonBlocking) != cudaSuccess ||
              cudaEventCreateWithFlags(&m->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
@@ -2022,7 +1566,6 @@ dbt_status dbt_reset(dbt_model *m) {
     CUDA_TRY(m, cudaMemsetAsync(m->ws.att_tickets2, 0, sizeof(int32_t) * (size_t)m->Rmax * m->cfg.n_kv_heads * kAttMaxGroups, m->stream));
     CUDA_TRY(m, cudaMemsetAsync(m->ws.gemm_tickets, 0, sizeof(int32_t) * 4096, m->stream));
     CUDA_TRY(m, cudaMemsetAsync(m->ws.ro_tickets, 0, sizeof(int32_t) * (size_t)m->cfg.max_batch, m->stream));
-    if (m->ws.mega_sync) CUDA_TRY(m, cudaMemsetAsync(m->ws.mega_sync, 0, sizeof(unsigned int) * 8, m->stream));
     std::fill(m->len_host.begin(), m->len_host.end(), 0);
     return DBT_OK;
 }
@@ -2049,7 +1592,6 @@ dbt_status dbt_prefill(dbt_model *m, const int32_t *tokens_dev, int32_t B, int32
     dbt_status st = check_step_args(m, tokens_dev, B, n);
     if (st != DBT_OK) return st;
     if (m->cfg.weight_dtype == DBT_DTYPE_F32) return prefill_impl<float>(m, tokens_dev, B, n, last_primary_logits_dev);
-    if (m->fused) return prefill_fused(m, tokens_dev, B, n, last_primary_logits_dev);
     if (m->wide) return prefill_wide(m, tokens_dev, B, n, last_primary_logits_dev);
     if (m->tc) return prefill_tc(m, tokens_dev, B, n, last_primary_logits_dev);
     return prefill_impl<__nv_bfloat16>(m, tokens_dev, B, n, last_primary_logits_dev);
@@ -2058,13 +1600,6 @@ dbt_status dbt_prefill(dbt_model *m, const int32_t *tokens_dev, int32_t B, int32
 static dbt_status step_direct(dbt_model *m, const int32_t *tokens_dev, int B, int grouped, int32_t *next_dev,
                               float *z1, float *z2, float *alpha) {
     if (m->cfg.weight_dtype == DBT_DTYPE_F32) return step_impl<float>(m, tokens_dev, B, grouped, next_dev, z1, z2, alpha);
-    if (mega_eligible(m, B)) {
-        int slot = -1;
-        dbt_status st = mega_prepare(m, B, grouped, &slot);
-        if (st != DBT_OK) return st;
-        if (slot >= 0) return step_mega(m, slot, tokens_dev, B, grouped, next_dev, z1, z2, alpha);
-    }
-    if (m->fused) return step_fused(m, tokens_dev, B, grouped, next_dev, z1, z2, alpha);
     if (m->wide) return step_wide(m, tokens_dev, B, grouped, next_dev, z1, z2, alpha);
     if (m->tc) return step_tc(m, tokens_dev, B, grouped, next_dev, z1, z2, alpha);
     return step_impl<__nv_bfloat16>(m, tokens_dev, B, grouped, next_dev, z1, z2, alpha);
@@ -2082,11 +1617,6 @@ static dbt_status step_graphed(dbt_model *m, const int32_t *tokens_dev, int B, i
     if (!hit) {
         if (m->graphs.size() >= 64) {  // a caller that never reuses buffers: stop caching
             return step_direct(m, tokens_dev, B, grouped, next_dev, z1, z2, alpha);
-        }
-        if (mega_eligible(m, B)) {  // the plan upload must not fall inside the capture
-            int slot = -1;
-            dbt_status pst = mega_prepare(m, B, grouped, &slot);
-            if (pst != DBT_OK) return pst;
         }
         std::vector<int32_t> len_save = m->len_host;
         int64_t l0 = m->launches;
@@ -2169,6 +1699,85 @@ dbt_status dbt_decode_step_primary_only_host(dbt_model *m, const int32_t *tokens
     return step_host(m, tokens_host, B, next_tokens_host, nullptr, 0);
 }
 
+// Moves nb sequences x nt positions of one layer's K (or V) plane between the paged pool and the staging
+// buffer, through the page table.  One thread per 16 bytes.
+static dbt_status kv_stage_copy(dbt_model *m, int layer, int which, const int32_t *seq_ids_dev, int s0, int nb, int t0, int nt,
+                                int to_pool) {
+    const dbt_config &c = m->cfg;
+    const int row_bytes = c.head_dim * elem_bytes(c);
+    char *plane = m->kv_pool + ((size_t)layer * 2 + which) * c.num_pages * c.n_kv_heads * c.page_size * row_bytes;
+    size_t vecs = (size_t)nb * nt * c.n_kv_heads * (row_bytes / 16);
+    LAUNCH(m, "kv_copy", 0, kv_copy_kernel, (unsigned)((vecs + 255) / 256), 256, 0, plane, m->ws.page_table, m->pages_per_seq_max,
+           c.num_pages, c.n_kv_heads, row_bytes, seq_ids_dev, s0, nb, t0, nt, m->ws.kv_stage, to_pool, m->ws.status);
+    return DBT_OK;
+}
+
+static dbt_status kv_transfer(dbt_model *m, const int32_t *seq_ids_host, int32_t B, int32_t T, char *k_host, char *v_host,
+                              int to_pool) {
+    if (!m) return DBT_ERR_INVALID_ARG;
+    if (!k_host || !v_host) return fail(m, DBT_ERR_INVALID_ARG, "NULL host buffer");
+    if (B <= 0 || T <= 0 || B > m->cfg.max_batch) return fail(m, DBT_ERR_INVALID_ARG, "bad B or T");
+    const dbt_config &c = m->cfg;
+    int cap = m->pages_per_seq * c.page_size;
+    if (cap > c.max_seq) cap = c.max_seq;
+    if (T > cap) return fail(m, DBT_ERR_CAPACITY, "T=%d exceeds the per-sequence capacity %d", T, cap);
+    std::vector<int32_t> ids(B);
+    for (int b = 0; b < B; b++) {
+        ids[b] = seq_ids_host ? seq_ids_host[b] : b;
+        if (ids[b] < 0 || ids[b] >= c.max_batch) return fail(m, DBT_ERR_INVALID_ARG, "sequence id %d out of range", ids[b]);
+        if (!to_pool && m->len_host[ids[b]] < T)
+            return fail(m, DBT_ERR_STATE, "sequence %d holds %d positions, %d requested", ids[b], m->len_host[ids[b]], T);
+    }
+    // the ids travel in the token staging buffer (max_batch ints)
+    CUDA_TRY(m, cudaMemcpyAsync(m->ws.tokens_stage, ids.data(), sizeof(int32_t) * B, cudaMemcpyHostToDevice, m->stream));
+    const size_t row = (size_t)c.n_kv_heads * c.head_dim * elem_bytes(c);  // one position of one sequence
+    const size_t rows_cap = kKvStageBytes / row;
+    if (rows_cap == 0) return fail(m, DBT_ERR_UNSUPPORTED, "kv row larger than the staging buffer");
+    const bool use_pdl = m->use_pdl;
+    m->use_pdl = false;  // copies and kernels alternate on the stream: plain stream order
+    dbt_status st = DBT_OK;
+    for (int l = 0; l < c.n_layers && st == DBT_OK; l++)
+        for (int which = 0; which < 2 && st == DBT_OK; which++) {
+            char *host = (which ? v_host : k_host) + (size_t)l * B * T * row;
+            // whole sequences per chunk when a sequence fits, else one sequence in position ranges
+            const int seq_per = (size_t)T <= rows_cap ? (int)(rows_cap / T) : 0;
+            for (int s0 = 0; s0 < B && st == DBT_OK; s0 += seq_per > 0 ? seq_per : 1) {
+                const int nb = seq_per > 0 ? (B - s0 < seq_per ? B - s0 : seq_per) : 1;
+                const int t_step = seq_per > 0 ? T : (int)rows_cap;
+                for (int t0 = 0; t0 < T && st == DBT_OK; t0 += t_step) {
+                    const int nt = T - t0 < t_step ? T - t0 : t_step;
+                    char *hp = host + ((size_t)s0 * T + t0) * row;
+                    const size_t bytes = (size_t)nb * nt * row;
+                    cudaError_t e = cudaSuccess;
+                    if (to_pool) e = cudaMemcpyAsync(m->ws.kv_stage, hp, bytes, cudaMemcpyHostToDevice, m->stream);
+                    if (e == cudaSuccess) st = kv_stage_copy(m, l, which, m->ws.tokens_stage, s0, nb, t0, nt, to_pool);
+                    if (e == cudaSuccess && st == DBT_OK && !to_pool)
+                        e = cudaMemcpyAsync(hp, m->ws.kv_stage, bytes, cudaMemcpyDeviceToHost, m->stream);
+                    if (e != cudaSuccess) st = fail(m, DBT_ERR_CUDA, "kv transfer: %s", cudaGetErrorString(e));
+                }
+            }
+        }
+    m->use_pdl = use_pdl;
+    if (st != DBT_OK) return st;
+    CUDA_TRY(m, cudaStreamSynchronize(m->stream));
+    if (to_pool) {  // the imported sequences now hold T positions
+        for (int b = 0; b < B; b++) {
+            m->len_host[ids[b]] = T;
+            CUDA_TRY(m, cudaMemcpy(m->ws.seq_len + ids[b], &T, sizeof(int32_t), cudaMemcpyHostToDevice));
+        }
+    }
+    return DBT_OK;
+}
+
+dbt_status dbt_kv_export(dbt_model *m, const int32_t *seq_ids_host, int32_t B, int32_t T, void *k_host, void *v_host) {
+    return kv_transfer(m, seq_ids_host, B, T, (char *)k_host, (char *)v_host, 0);
+}
+
+dbt_status dbt_kv_import(dbt_model *m, const int32_t *seq_ids_host, int32_t B, int32_t T, const void *k_host,
+                         const void *v_host) {
+    return kv_transfer(m, seq_ids_host, B, T, (char *)const_cast<void *>(k_host), (char *)const_cast<void *>(v_host), 1);
+}
+
 dbt_status dbt_last_experts(dbt_model *m, const int32_t **experts_dev, int32_t *kmax) {
     if (!m) return DBT_ERR_INVALID_ARG;
     if (m->cfg.n_experts == 0) return fail(m, DBT_ERR_STATE, "not an MoE model");
@@ -2193,6 +1802,8 @@ dbt_status dbt_sync_status(dbt_model *m, int32_t *device_status, int32_t *detail
     CUDA_TRY(m, cudaMemcpy(h, m->ws.status, sizeof h, cudaMemcpyDeviceToHost));
     if (device_status) *device_status = h[0];
     if (detail) *detail = h[1];
+    if (h[0] == kStatusWaitExpired)
+        return fail(m, DBT_ERR_TIMEOUT, "a bounded device wait ran out (wait site %d)", h[1]);
     if (h[0] != 0) return fail(m, DBT_ERR_DEVICE, "device status %d (detail %d)", h[0], h[1]);
     return DBT_OK;
 }
@@ -2213,13 +1824,18 @@ static dbt_status op_gemm_tc_impl(dbt_model *m, const void *W_dev, const void *X
     TcCall c{};
     c.W[0] = &mw; c.n_out[0] = n_out; c.rows[0] = R; c.nseg = 1; c.X = &mx; c.K = K; c.R = R;
     c.P = scratch_dev; c.P_floats = scratch_floats; c.tag = "gemm"; c.parts = 1; c.lo_row0 = 0;
+    if (force_split > (K + kTcK - 1) / kTcK) force_split = (K + kTcK - 1) / kTcK;  // at most one k-tile per split
     if (force_split > 0) {  // honour the request by shrinking the scratch the heuristic may use
         size_t per = (size_t)pad_rows(R) * n_out;
         if ((size_t)force_split * per > scratch_floats) return fail(m, DBT_ERR_CAPACITY, "scratch too small");
     }
     int nsp = 1;
     size_t stride = 0;
-    dbt_status st = run_gemm_tc(m, c, pad_rows(R), &nsp, &stride, force_split);
+    // Test hook (host-set, off by default): DBT_TEST_EXPIRE_WAIT=1 makes CTA (0,0,0) skip one weight-tile request
+    // and shortens every wait to about a millisecond, so that a test can watch a bounded wait run out: the kernel
+    // records status 3 in status_dev and returns normally.  No other entry point reads the variable.
+    const char *tw = getenv("DBT_TEST_EXPIRE_WAIT");
+    dbt_status st = run_gemm_tc(m, c, pad_rows(R), &nsp, &stride, force_split, LmEpi{}, tw && strcmp(tw, "1") == 0);
     if (st != DBT_OK) return st;
     size_t n = (size_t)R * n_out;
     LAUNCH(m, "reduce", 0, reduce_splits_kernel, (unsigned)((n + 255) / 256), 256, 0, scratch_dev, nsp, stride, n, Y_dev);
@@ -2273,8 +1889,10 @@ dbt_status dbt_op_gemm_tc_static(const void *W_dev, const void *X_dev, int32_t n
                   "roundup(R)=%d rows x n_out=%d = %zu floats exceed the static scratch of %zu floats (8 MiB); "
                   "use dbt_op_gemm_tc with caller-provided scratch",
                   pad_rows(R), n_out, (size_t)pad_rows(R) * (size_t)n_out, kStaticScratchFloats);
-    } else if (force_split > 0 && (size_t)force_split * pad_rows(R > 0 && R <= 256 ? R : 1) * (size_t)(n_out > 0 ? n_out : 0) >
-                                      kStaticScratchFloats) {
+    } else if (force_split > 0 && K > 0 &&
+               (size_t)(force_split < (K + kTcK - 1) / kTcK ? force_split : (K + kTcK - 1) / kTcK) *
+                       pad_rows(R > 0 && R <= 256 ? R : 1) * (size_t)(n_out > 0 ? n_out : 0) >
+                   kStaticScratchFloats) {
         st = fail(m, DBT_ERR_CAPACITY, "force_split=%d needs more than the static scratch of %zu floats (8 MiB)",
                   force_split, kStaticScratchFloats);
     } else {

@@ -5,7 +5,8 @@
 // tile is brought from HBM exactly once by TMA (128B-swizzled, K-major) into a shared-memory
 // ring, multiplied by tcgen05.mma into an fp32 accumulator in tensor memory, and read back
 // with tcgen05.ld for the epilogue.  One CTA = one 128-feature tile x one K range (split-K
-// partials are written to global memory and summed, in split order, by the consumer kernel).
+// partials are written to global memory and summed, in split order, by the consumer kernel;
+// the shared output matrix runs unsplit and writes logits, times the row's 1/rms, directly).
 //
 // Roles inside the 128-thread CTA: warp 0 lane 0 issues TMA, warp 1 lane 0 issues MMAs and
 // owns the TMEM allocation, all four warps run the epilogue (warp w owns TMEM lanes 32w..).
@@ -17,7 +18,6 @@
 
 #include "dbt_common.cuh"
 #include "dbt_fused.cuh"
-#include "dbt_gemm_epi.cuh"
 
 namespace dbt {
 
@@ -25,6 +25,7 @@ constexpr int kTcM = 128;       // weight rows per tile (MMA M)
 constexpr int kTcK = 64;        // K elements per stage (one 128-byte swizzle row of bf16)
 constexpr int kTcABytes = kTcM * kTcK * 2;
 constexpr uint64_t kWaitCycles = 4000000000ull;  // ~2 s at 1.9 GHz
+constexpr uint64_t kTestWaitCycles = 2000000ull;  // ~1 ms: the limit under TcParams::test_skip_load
 
 struct TcSeg {
     int tile0;   // first tile index of this segment
@@ -35,10 +36,6 @@ struct TcSeg {
 
 struct TcParams {
     int evict_first;  // weight tiles carry the evict-first L2 hint
-    // up to three byte ranges (the next GEMM's weights) that this launch asks the L2 to fetch while it
-    // and the small kernels after it run: HBM is otherwise idle between the GEMMs of a decode step
-    const char *pf_ptr[3];
-    unsigned long long pf_bytes[3];
     int x3d;  // tmX is the 3-D {64, N_TILE, 2} view of a two-plane input: one box per stage
     int stacked;  // with x3d: one MMA per k16 step over both planes (N = 2 * N_TILE), halves added in the epilogue
     TcSeg seg[3];
@@ -58,6 +55,19 @@ struct TcParams {
     // grouped mode with row tiles: blockIdx.y = which N_TILE rows of the expert's list (CTAs past the
     // list's end leave at once); 0: the whole list fits one tile and blockIdx.y is the split as usual
     int grp_row_tiles;
+    // test hook (dbt_op_gemm_tc only): 1 = CTA (0,0,0) never requests the weight tile of its first stage
+    // and every wait gives up after kTestWaitCycles, so that the expired-wait path can be exercised:
+    // the kernel records kStatusWaitExpired, skips its stores, frees its TMEM and returns
+    int test_skip_load;
+};
+
+// Epilogue of the shared output matrix (Section 4.2: z_i from the final states): logits = accumulator
+// times the row's 1/rms (the final RMSNorm's gain is folded into the GEMM input), written to Z.
+struct LmEpi {
+    float *Z;             // nullptr: the ordinary split-K partial store
+    const float *ss_in;   // per-tile shares of sum(S^2): [ss_tiles][ss_ld]
+    int ss_tiles, ss_ld, d_norm, use_scale;
+    float eps;
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -69,7 +79,7 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
 // Bounded wait on a phase parity; false when the limit expired.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint64_t limit = kWaitCycles) {
     uint32_t done = 0;
     asm volatile(
         "{\n"
@@ -93,7 +103,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
             : "r"(bar), "r"(parity)
             : "memory");
         if (done) return true;
-        if ((unsigned long long)(clock64() - t0) > kWaitCycles) return false;
+        if ((unsigned long long)(clock64() - t0) > limit) return false;
     }
 }
 
@@ -108,22 +118,6 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map
         "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];" ::"r"(dst),
         "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
         : "memory");
-}
-// Thread-block cluster helpers: rank, barrier, and a load from a peer CTA's shared memory.
-__device__ __forceinline__ uint32_t cluster_rank() {
-    uint32_t r;
-    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-    return r;
-}
-__device__ __forceinline__ void cluster_sync() {
-    asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-__device__ __forceinline__ float ld_peer_smem(uint32_t local_addr, uint32_t rank) {
-    uint32_t ra;
-    float v;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(local_addr), "r"(rank));
-    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(ra) : "memory");
-    return v;
 }
 // L2 eviction policy for data that is read once per step (weight tiles, K/V pages): evict first, so
 // that the stream does not push the small reused data (activations, partials, gains, tables) out.
@@ -202,11 +196,7 @@ struct TcCfg {
     static constexpr int kStageBytes = kTcABytes + 2 * kBBytes;
     // small row counts: keep one CTA near 100 KB so that a dependent kernel's CTA can become
     // resident beside it; large row counts take the whole SM
-#ifdef DBT_TC_DEEP
-    static constexpr int kStages = N_TILE <= 16 ? 10 : N_TILE <= 32 ? 8 : N_TILE <= 64 ? 6 : N_TILE <= 128 ? 4 : 2;
-#else
     static constexpr int kStages = N_TILE <= 16 ? 5 : N_TILE <= 32 ? 4 : N_TILE <= 64 ? 3 : N_TILE <= 128 ? 4 : 2;
-#endif
     // room for the two planes' accumulators side by side (see `stacked` in the kernel)
     static constexpr int kStackable = N_TILE <= 128;
     static constexpr int kTmemCols = kStackable ? (2 * N_TILE < 32 ? 32 : 2 * N_TILE) : N_TILE;
@@ -217,7 +207,7 @@ template <int N_TILE>
 __global__ void __launch_bounds__(128, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtensorMap tmW1,
                const __grid_constant__ CUtensorMap tmW2, const __grid_constant__ CUtensorMap tmX, TcParams p,
-               FusedEpi e) {
+               LmEpi e) {
     using Cfg = TcCfg<N_TILE>;
     constexpr int STAGES = Cfg::kStages;
     extern __shared__ uint8_t smem_raw[];
@@ -233,9 +223,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
     DBT_TL_DECL;
     int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     int tile = blockIdx.x, split = p.grp_row_tiles ? 0 : blockIdx.y;
-    // Clustered gate|up: CTAs (2j, y) and (2j + 1, y) hold gate tile j and up tile j, so that a cluster
-    // of 2 x splits CTAs owns everything SwiGLU needs for 128 features.
-    if (e.cluster && e.mode == FE_GATEUP) tile = (int)(blockIdx.x & 1) * p.seg[1].tile0 + (int)(blockIdx.x >> 1);
     int x_row0 = 0, w_row0 = 0, grp_n = -1;
     if (p.grp_cnt) {
         // the expert's row list comes from the previous kernel: nothing can start before it is known
@@ -281,19 +268,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
     uint32_t tmem_base = *tmem_holder;
     pdl_launch_dependents();
 
-    if (warp == 2 && lane == 0) {
-        constexpr unsigned long long kChunk = 16384;
-        const unsigned ncta = gridDim.x * gridDim.y * gridDim.z;
-        const unsigned cid = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);
-        for (int j = 0; j < 3; j++) {
-            const unsigned long long bytes = p.pf_bytes[j];
-            for (unsigned long long off = (unsigned long long)cid * kChunk; off < bytes; off += (unsigned long long)ncta * kChunk) {
-                unsigned sz = (unsigned)min(kChunk, bytes - off) & ~15u;
-                if (sz) asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p.pf_ptr[j] + off), "r"(sz) : "memory");
-            }
-        }
-    }
     bool ok = true;
+    const uint64_t wait_limit = p.test_skip_load ? kTestWaitCycles : kWaitCycles;
+    const bool skip_first_w = p.test_skip_load && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0;
     if (warp == 0 && lane == 0) {
         // ---- TMA producer.  Weight tiles do not depend on the previous kernel: the first
         // ring-full of them is requested before waiting for it.
@@ -320,14 +297,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
         };
         for (int i = 0; i < npre; i++) {
             mbar_expect_tx(full_bar(i), tx);
-            load_w(i, kt0 + i);
+            if (!(skip_first_w && i == 0)) load_w(i, kt0 + i);
         }
         pdl_wait();
         DBT_TL_MARK(0);
         for (int i = 0; i < npre; i++) load_x(i, kt0 + i);
         for (int i = npre; i < nkt && ok; i++) {
             int s = i % STAGES;
-            ok = mbar_wait(empty_bar(s), ((i / STAGES) - 1) & 1);
+            ok = mbar_wait(empty_bar(s), ((i / STAGES) - 1) & 1, wait_limit);
             if (!ok) break;
             mbar_expect_tx(full_bar(s), tx);
             load_w(s, kt0 + i);
@@ -344,7 +321,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
         const bool stacked = Cfg::kStackable && p.stacked;
         for (int i = 0; i < nkt && ok; i++) {
             int s = i % STAGES;
-            ok = mbar_wait(full_bar(s), (i / STAGES) & 1);
+            ok = mbar_wait(full_bar(s), (i / STAGES) & 1, wait_limit);
             if (!ok) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             uint64_t adesc = umma_smem_desc(tiles + s * Cfg::kStageBytes);
@@ -371,7 +348,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
     // ---- epilogue: TMEM lane = weight row (feature), TMEM column = activation row
     pdl_wait();
     DBT_TL_WAITED;
-    bool got = mbar_wait(accum_bar, 0);
+    bool got = ok && mbar_wait(accum_bar, 0, wait_limit);  // the issuing lane knows already when the accumulator will never complete
     DBT_TL_MARK(2);
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (!got && lane == 0) report(p.status, kStatusWaitExpired, 200 + warp);
@@ -387,8 +364,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
 #pragma unroll
         for (int i = 0; i < 16; i++) v[i] = __uint_as_float(a[i]) + (stacked_acc ? __uint_as_float(b[i]) : 0.f);
     };
-    if (got && e.mode == FE_LMHEAD) {
-        epi_row_scales(e, p.R, scratch);
+    if (got && e.Z) {
+        // 1/rms per row (or 1 when the input was not normalised) into shared memory
+        for (int r = tid; r < p.R; r += blockDim.x) {
+            float v = 1.f;
+            if (e.use_scale) {
+                float ss = 0.f;
+                for (int t = 0; t < e.ss_tiles; t++) ss += __ldcg(e.ss_in + (size_t)t * e.ss_ld + r);
+                v = 1.f / sqrtf(ss / (float)e.d_norm + e.eps);
+            }
+            scratch[r] = v;
+        }
+        __syncthreads();
         int f = f0 + warp * 32 + lane;
 #pragma unroll 1
         for (int c0 = 0; c0 < N_TILE && c0 < rows; c0 += 16) {
@@ -400,134 +387,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
                     if (c0 + i < rows) e.Z[(size_t)(c0 + i) * p.ldp + seg.col0 + f] = v[i] * scratch[c0 + i];
             }
         }
-    } else if (e.cluster && e.mode == FE_GATEUP) {
-        // The cluster is {gate tile j, up tile j} x splits (rank = x + 2 * y).  Each CTA leaves its
-        // accumulator tile in shared memory; after the barrier CTA r finishes the primary rows r, r + n,
-        // ... and their branch twins for the tile's 128 features: gate and up summed over the splits in
-        // split order, 1/rms of the GEMM input, H = SiLU(gate) * up, H~_2 = H_2 + b * H_1 (Eq. mlp), two
-        // bf16 planes for the down projection.
-        float *tile_s = scratch;  // [N_TILE][128] fp32
-        if (got) {
-#pragma unroll 1
-            for (int c0 = 0; c0 < N_TILE && c0 < rows; c0 += 16) {
-                float v[16];
-                ld_acc(c0, v);
-#pragma unroll
-                for (int i = 0; i < 16; i++) tile_s[(c0 + i) * kTcM + warp * 32 + lane] = v[i];
-            }
-        }
-        cluster_sync();
-        if (got) {
-            const uint32_t rank = cluster_rank(), S = gridDim.y, nranks = 2 * S;
-            const int fl = warp * 32 + lane, col = f0 + fl, F = e.ld_out;
-            const bool live = col < seg.n_out;
-            const uint32_t base = smem_u32(tile_s);
-            const float cb = (live && e.coup) ? e.coup[col] : 0.f;
-            for (int b = (int)rank; b < e.Bc; b += (int)nranks) {
-                const int r2 = e.Bc + b;
-                float rs1 = 1.f, rs2 = 1.f;
-                if (e.use_scale) row_scale2(e.ss_in, e.ss_tiles, e.ss_ld, b, e.grouped ? r2 : b, e.d_norm, e.eps, rs1, rs2);
-                if (live) {
-                    float g1 = 0.f, u1 = 0.f, g2 = 0.f, u2 = 0.f;
-                    float vg1[4], vu1[4], vg2[4], vu2[4];
-#pragma unroll
-                    for (uint32_t y = 0; y < 4; y++) {
-                        bool on = y < S;
-                        vg1[y] = on ? ld_peer_smem(base + (uint32_t)(b * kTcM + fl) * 4u, 2 * y) : 0.f;
-                        vu1[y] = on ? ld_peer_smem(base + (uint32_t)(b * kTcM + fl) * 4u, 2 * y + 1) : 0.f;
-                        vg2[y] = (on && e.grouped) ? ld_peer_smem(base + (uint32_t)(r2 * kTcM + fl) * 4u, 2 * y) : 0.f;
-                        vu2[y] = (on && e.grouped) ? ld_peer_smem(base + (uint32_t)(r2 * kTcM + fl) * 4u, 2 * y + 1) : 0.f;
-                    }
-#pragma unroll
-                    for (int y = 0; y < 4; y++) {
-                        g1 += vg1[y];
-                        u1 += vu1[y];
-                        g2 += vg2[y];
-                        u2 += vu2[y];
-                    }
-                    float h1 = silu(rs1 * g1) * (rs1 * u1);
-                    epi_store_split(e.Xout, (size_t)b * F + col, e.lo_off, h1);
-                    if (e.grouped) {
-                        float h2 = silu(rs2 * g2) * (rs2 * u2) + cb * h1;
-                        epi_store_split(e.Xout, (size_t)r2 * F + col, e.lo_off, h2);
-                    }
-                }
-            }
-        }
-        cluster_sync();
-    } else if (e.cluster) {
-        // The splits of this output tile are the CTAs of one cluster.  Each leaves its accumulator tile
-        // in its own shared memory; after a cluster barrier CTA r adds, in split order, the tiles of
-        // all ranks for the primary rows r, r + S, ... (and their branch twins) and finishes those rows:
-        // S-bar = S + . (FE_RESID) or M_2 += c * M_1, S += M (FE_DOWN, Eq. mlp), the next GEMM's input
-        // g * S as two bf16 planes, and this 128-column tile's share of sum(S^2) per row.  Every CTA
-        // takes part in both barriers whatever happened to it, so that nobody waits forever.
-        float *tile_s = scratch;                    // [N_TILE][128] fp32
-        float *red = scratch + N_TILE * kTcM;       // [8] block reduction
-        if (got) {
-#pragma unroll 1
-            for (int c0 = 0; c0 < N_TILE && c0 < rows; c0 += 16) {
-                float v[16];
-                ld_acc(c0, v);
-#pragma unroll
-                for (int i = 0; i < 16; i++) tile_s[(c0 + i) * kTcM + warp * 32 + lane] = v[i];
-            }
-        }
-        cluster_sync();
-        if (got) {
-            const uint32_t rank = cluster_rank(), S = gridDim.y;
-            const int fl = warp * 32 + lane, col = f0 + fl, d = e.ld_out;
-            const bool live = col < seg.n_out;
-            const uint32_t base = smem_u32(tile_s);
-            const float gn = (live && e.g_next) ? e.g_next[col] : 1.f;
-            const float cc = (live && e.mode == FE_DOWN && e.coup) ? e.coup[col] : 0.f;
-            for (int b = (int)rank; b < e.Bc; b += (int)S) {
-                const int r2 = e.Bc + b;
-                float s1 = 0.f, s2 = 0.f, m1 = 0.f, m2 = 0.f;
-                if (live) {
-                    s1 = __ldcg(e.S + (size_t)b * d + col);
-                    if (e.grouped) s2 = __ldcg(e.S + (size_t)r2 * d + col);
-                    float v1[16], v2[16];  // up to 16 ranks (the opt-in cluster size), all loads in flight
-#pragma unroll
-                    for (uint32_t j = 0; j < 16; j++) {
-                        v1[j] = j < S ? ld_peer_smem(base + (uint32_t)(b * kTcM + fl) * 4u, j) : 0.f;
-                        v2[j] = (j < S && e.grouped) ? ld_peer_smem(base + (uint32_t)(r2 * kTcM + fl) * 4u, j) : 0.f;
-                    }
-#pragma unroll
-                    for (int j = 0; j < 16; j++) {
-                        m1 += v1[j];
-                        m2 += v2[j];
-                    }
-                }
-                float q1 = 0.f, q2 = 0.f;
-                if (live) {
-                    s1 += m1;
-                    e.S[(size_t)b * d + col] = s1;
-                    epi_store_split(e.Xout, (size_t)b * d + col, e.lo_off, gn * s1);
-                    q1 = s1 * s1;
-                    if (e.grouped) {
-                        if (e.mode == FE_DOWN) m2 += cc * m1;
-                        s2 += m2;
-                        e.S[(size_t)r2 * d + col] = s2;
-                        epi_store_split(e.Xout, (size_t)r2 * d + col, e.lo_off, gn * s2);
-                        q2 = s2 * s2;
-                    }
-                }
-                q1 = warp_sum(q1);
-                q2 = warp_sum(q2);
-                __syncthreads();
-                if (lane == 0) {
-                    red[warp] = q1;
-                    red[4 + warp] = q2;
-                }
-                __syncthreads();
-                if (tid == 0) {
-                    e.ss_out[(size_t)tile * e.ss_ld + b] = red[0] + red[1] + red[2] + red[3];
-                    if (e.grouped) e.ss_out[(size_t)tile * e.ss_ld + r2] = red[4] + red[5] + red[6] + red[7];
-                }
-            }
-        }
-        cluster_sync();
     } else if (got) {
         int f = f0 + warp * 32 + lane;
         float *out = p.P + ((size_t)split * p.R + x_row0) * p.ldp + seg.col0 + f;
@@ -539,26 +398,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
 #pragma unroll
                 for (int i = 0; i < 16; i++)
                     if (c0 + i < rows) out[(size_t)(c0 + i) * p.ldp] = v[i];
-            }
-        }
-        if (e.mode != FE_NONE) {
-            // arrival ticket of this output tile; the last CTA folds the splits and finishes the tile
-            __threadfence();
-            __syncthreads();
-            int *flag = reinterpret_cast<int *>(scratch);
-            if (tid == 0) {
-                int *tk = e.tickets + (e.mode == FE_GATEUP ? tile - seg.tile0 : tile);
-                int t = atomicAdd(tk, 1);
-                int last = t == e.arrivals - 1;
-                if (last) atomicExch(tk, 0);
-                *flag = last;
-            }
-            __syncthreads();
-            int last = *flag;
-            __syncthreads();
-            if (last) {
-                __threadfence();
-                fused_epilogue(e, p.P, gridDim.y, p.R, p.ldp, f0, seg.col0, seg.n_out, sg, tile, scratch);
             }
         }
     }

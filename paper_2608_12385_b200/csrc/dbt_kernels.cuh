@@ -601,6 +601,35 @@ __global__ void __launch_bounds__(kRoThreads) readout_pick_kernel(const float *Z
     }
 }
 
+// dbt_kv_export / dbt_kv_import: one K or V plane of one layer, [num_pages][n_kv][16][row_bytes], against a staging
+// buffer in logical order [nb][nt][n_kv][row_bytes] for sequences seq_ids[s0..s0+nb) and positions t0..t0+nt-1,
+// through the page table (Background, KV cache: the cache is addressed by position; paging is this library's).
+__global__ void kv_copy_kernel(char *plane, const int32_t *page_table, int pt_stride, int num_pages, int n_kv, int row_bytes,
+                               const int32_t *seq_ids, int s0, int nb, int t0, int nt, char *stage, int to_pool, int *status) {
+    pdl_enter();
+    const int vpr = row_bytes / 16;
+    const size_t total = (size_t)nb * nt * n_kv * vpr;
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= total) return;
+    const int v = (int)(i % vpr);
+    size_t r = i / vpr;
+    const int h = (int)(r % n_kv);
+    r /= n_kv;
+    const int ti = (int)(r % nt), bi = (int)(r / nt);
+    const int t = t0 + ti, seq = ld_mut(seq_ids + s0 + bi);
+    int page = ld_mut(page_table + (size_t)seq * pt_stride + t / 16);
+    if (page < 0 || page >= num_pages) {
+        report(status, kStatusBadPage, page);
+        return;
+    }
+    uint4 *pool_p = reinterpret_cast<uint4 *>(plane + (((size_t)page * n_kv + h) * 16 + (t & 15)) * row_bytes) + v;
+    uint4 *stage_p = reinterpret_cast<uint4 *>(stage + (((size_t)bi * nt + ti) * n_kv + h) * row_bytes) + v;
+    if (to_pool)
+        *pool_p = *stage_p;
+    else
+        *stage_p = *pool_p;
+}
+
 __global__ void advance_len_kernel(int32_t *seq_len, int B, int n) {
     pdl_enter();
     int b = blockIdx.x * blockDim.x + threadIdx.x;

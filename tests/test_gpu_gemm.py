@@ -72,3 +72,23 @@ def test_columns_are_independent_of_their_neighbours():
     narrow, _ = binding.op_gemm_tc(W, X[:20].contiguous(), force_split=4)  # 32-wide instruction
     torch.testing.assert_close(full[:20], narrow, rtol=1e-5, atol=1e-5)
     print("bit-identical across instruction widths:", torch.equal(full[:20], narrow))
+
+
+def test_an_expired_device_wait_is_reported_and_the_next_call_is_clean(monkeypatch):
+    """Every wait inside the kernels is bounded.  With the host-set test hook one CTA of a tiny GEMM never
+    requests one of its weight tiles and the limit drops to about a millisecond: the waits on that tile run
+    out, the kernel records status 3 with the wait site, skips its stores, frees its tensor memory and
+    returns -- nothing traps and nothing spins on.  The very next call on the same GPU, without the hook,
+    is clean and correct."""
+    g = torch.Generator(device="cpu").manual_seed(3)
+    W = torch.randn(256, 512, generator=g).to(torch.bfloat16).cuda()
+    X = torch.randn(8, 512, generator=g).to(torch.bfloat16).cuda()
+    monkeypatch.setenv("DBT_TEST_EXPIRE_WAIT", "1")
+    with pytest.raises(binding.DbtError) as e:
+        binding.op_gemm_tc(W, X, force_split=2)
+    assert e.value.status == 7 and ("[3, 10" in str(e.value) or "[3, 20" in str(e.value)), str(e.value)
+    monkeypatch.delenv("DBT_TEST_EXPIRE_WAIT")
+    Y, _ = binding.op_gemm_tc(W, X, force_split=2)
+    want = X.float() @ W.float().T
+    assert torch.allclose(Y, want, rtol=1e-3, atol=1e-2)
+    torch.cuda.synchronize()

@@ -78,7 +78,7 @@ def test_context_lengths_around_page_and_chunk_boundaries(ctx):
     if ctx > 0:
         k, v = make_synthetic_kv(cfg, B, ctx, seed=11)
         om.inject_kv(k, v, ctx)
-        gm.write_kv(k, v)
+        gm.import_kv(k, v)
     for t in range(2):
         o = om.decode_step(tok[:, t].numpy())
         g = gm.decode_full(tok[:, t].cuda().contiguous())
@@ -97,7 +97,7 @@ def test_1b_shape_full_width_grouped_step_with_synthetic_cache():
     om = oracle.OracleModel(cfg, w, B, ctx + 3)
     gm = make_gpu_model(cfg, w, B, ctx + 3)
     om.inject_kv(k, v, ctx)
-    gm.write_kv(k, v)
+    gm.import_kv(k, v)
     for t in range(2):
         o = om.decode_step(tok[:, t].numpy())
         g = gm.decode_full(tok[:, t].cuda().contiguous())
@@ -124,7 +124,7 @@ def test_1b_at_the_benchmarks_launch_configuration_on_sampled_sequences():
     gen = torch.Generator(device=gm.device)
     gen.manual_seed(5)
     gm.kv_pool.normal_(0.0, 1.0, generator=gen)
-    gm.write_kv(k, v, page_table=gm.page_table[pick])
+    gm.import_kv(k, v, seq_ids=pick)
     gm.set_seq_lens([ctx] * B)
     om = oracle.OracleModel(cfg, w, len(pick), ctx + 3)
     om.inject_kv(k, v, ctx)
@@ -136,6 +136,59 @@ def test_1b_at_the_benchmarks_launch_configuration_on_sampled_sequences():
     o = om.decode_step(tok[pick, 1].numpy(), grouped=False)
     g = gm.decode_full(tok[:, 1].cuda().contiguous(), grouped=False)
     assert_logits_close(g["z1"][pick], o["z1"], "bf16", "bench config primary-only z1")
+    assert gm.sync_status() == (0, 0)
+
+
+# ---- readout off the clip of alpha (Eq. alpha, Eq. mixloss) ---------------------------------------------------
+
+@pytest.mark.parametrize("cfg,matrix_std", [(small_bf16(), 0.05), (tiny_dense_fp32(), 0.02)])
+def test_readout_with_alpha_between_the_clips_and_at_one(cfg, matrix_std):
+    """Random-init models have sum p^2 ~ 1e-3, so alpha sits on its lower clip and the mixture is symmetric
+    in p and q.  An output matrix drawn with standard deviation 2.0 makes p peaked: over these 6 sequences x 4
+    steps alpha lands strictly between the clips for some rows, at 1.0 for others, and argmax p != argmax q
+    everywhere, so a readout that swapped p and q, used sum q^2, or mis-folded a chunk would fail here.
+    The logits and their rounding errors scale with the output matrix, so the absolute bar scales by the same
+    factor f; d(alpha)/dz_j = 2 p_j (p_j - alpha), hence |d alpha| <= max|dz_1|.  The readout kernels alone are
+    then checked tightly: the oracle's readout of the DEVICE's own logits must reproduce the device's alpha
+    and, where the mixture's top two are apart, its token."""
+    dt = cfg.weight_dtype
+    head_std = 2.0
+    f = head_std / matrix_std
+    w = make_weights(cfg, seed=41, matrix_std=matrix_std, lm_head_std=head_std)
+    B, T, npre = 6, 12, 8
+    tok = make_tokens(cfg, B, T, seed=42)
+    om = oracle.OracleModel(cfg, w, B, T)
+    gm = make_gpu_model(cfg, w, B, T)
+    om.prefill(tok[:, :npre].numpy(), want_logits=False)
+    gm.prefill(tok[:, :npre].cuda().contiguous())
+    alphas, swapped_would_differ = [], 0
+    for t in range(npre, T):
+        o = om.decode_step(tok[:, t].numpy(), want_mix=True)
+        g = gm.decode_full(tok[:, t].cuda().contiguous())
+        z1, z2 = g["z1"].cpu().numpy(), g["z2"].cpu().numpy()
+        errs = []
+        for name, got in (("z1", z1), ("z2", z2)):
+            d = np.abs(got.astype(np.float64) - o[name])
+            rel = np.linalg.norm(got.astype(np.float64) - o[name]) / np.linalg.norm(o[name])
+            assert d.max() <= TOL[dt]["max_abs"] * f and rel <= TOL[dt]["rel_l2"], (name, t, d.max(), rel)
+            errs.append(d.max())
+        a_dev = g["alpha"].cpu().numpy()
+        np.testing.assert_allclose(a_dev, o["alpha"], rtol=1e-3, atol=errs[0])
+        nxt = g["next"].cpu().numpy()
+        for b in range(B):
+            tok_o, a_o, mix_o = oracle.readout(z1[b], z2[b])
+            assert a_dev[b] == pytest.approx(a_o, rel=2e-5), (t, b, a_dev[b], a_o)
+            top = np.sort(mix_o)[-2:]
+            if top[1] - top[0] > 1e-4 * top[1]:
+                assert nxt[b] == tok_o, (t, b, nxt[b], tok_o)
+            # what a p <-> q swap would have produced
+            _, a_sw, _ = oracle.readout(z2[b], z1[b])
+            swapped_would_differ += int(abs(a_sw - a_o) > 1e-3)
+        assert (o["z1"].argmax(-1) != o["z2"].argmax(-1)).all()
+        alphas.append(o["alpha"])
+    alphas = np.stack(alphas)
+    assert ((alphas > 0.5) & (alphas < 1.0)).sum() >= 5 and (alphas == 1.0).sum() >= 1, alphas
+    assert swapped_would_differ >= 5
     assert gm.sync_status() == (0, 0)
 
 
@@ -164,8 +217,8 @@ def test_kv_cache_bit_identical_grouped_vs_primary_only(cfg):
     ob = _run_steps(b, tok, npre, False)
     for x, y in zip(oa, ob):
         assert torch.equal(x["z1"], y["z1"])
-    ka, va = a.read_kv(B, T)
-    kb, vb = b.read_kv(B, T)
+    ka, va = a.export_kv(B, T)
+    kb, vb = b.export_kv(B, T)
     assert torch.equal(ka.view(torch.int16 if cfg.weight_dtype == "bf16" else torch.int32),
                        kb.view(torch.int16 if cfg.weight_dtype == "bf16" else torch.int32))
     assert torch.equal(va.view(torch.int16 if cfg.weight_dtype == "bf16" else torch.int32),
@@ -187,10 +240,70 @@ def test_moe_kv_cache_bit_identical_at_a_batch_with_row_tiled_expert_gemms():
     ob = _run_steps(b, tok, npre, False)
     for x, y in zip(oa, ob):
         assert torch.equal(x["z1"], y["z1"])
-    ka, va = a.read_kv(B, T)
-    kb, vb = b.read_kv(B, T)
+    ka, va = a.export_kv(B, T)
+    kb, vb = b.export_kv(B, T)
     assert torch.equal(ka.view(torch.int16), kb.view(torch.int16))
     assert torch.equal(va.view(torch.int16), vb.view(torch.int16))
+
+
+def test_moe_kv_bit_identical_at_full_width_where_the_resident_cta_count_changes_with_the_tile():
+    """One layer at the MoE model's width (d 2048, experts of 1408) and 34 sequences: the grouped step's 68
+    stacked rows need a row tile of 128 (one GEMM CTA per SM), the 34 primary-only rows alone would fit a tile
+    of 64 (two per SM) and a split-K search over twice the slots picks other factors for the shared expert
+    (11 vs 6 and 11 vs 8).  Both modes therefore size their tiles from the batch, not from the rows present,
+    and the primary logits and the cache come out bit-identical."""
+    cfg = moe_1b(k_branch=2).replace(n_layers=1, vocab=2048)
+    w = make_weights(cfg, seed=16)
+    B, T, npre = 34, 6, 4
+    tok = make_tokens(cfg, B, T, seed=17).cuda()
+    wd = binding.weights_to_device(w)
+    a = binding.Model(cfg, wd, B, T)
+    b = binding.Model(cfg, wd, B, T)
+    oa = _run_steps(a, tok, npre, True)
+    ob = _run_steps(b, tok, npre, False)
+    for x, y in zip(oa, ob):
+        assert torch.equal(x["z1"], y["z1"])
+    ka, va = a.export_kv(B, T)
+    kb, vb = b.export_kv(B, T)
+    assert torch.equal(ka.view(torch.int16), kb.view(torch.int16))
+    assert torch.equal(va.view(torch.int16), vb.view(torch.int16))
+
+
+def test_kv_export_import_round_trip_through_a_shuffled_page_table():
+    """dbt_kv_export returns what dbt_kv_import stored, in logical order, whatever the page table; importing
+    into a subset of the sequences leaves the others' lengths and contents alone; bad requests are refused."""
+    cfg = small_bf16(n_layers=2)
+    w = make_weights(cfg, seed=14, matrix_std=0.05)
+    B, T = 3, 45
+    gm = make_gpu_model(cfg, w, B, 64, num_pages=20)
+    gm.set_page_table(make_page_table(B, 4, 20, seed=16))
+    k, v = make_synthetic_kv(cfg, B, T, seed=3)
+    gm.import_kv(k, v)
+    assert [gm.seq_len(b) for b in range(B)] == [T] * B
+    k2, v2 = gm.export_kv(B, T)
+    assert torch.equal(k2.view(torch.int16), k.view(torch.int16)) and torch.equal(v2.view(torch.int16), v.view(torch.int16))
+    # positions live where the page table says
+    view = gm.kv_view()
+    pt = gm.page_table
+    for (l, b, t) in [(0, 0, 0), (1, 2, 17), (1, 1, 44)]:
+        page, slot = int(pt[b, t // 16]), t % 16
+        got = view[l, 0, page, :, slot, :].reshape(-1).cpu()
+        assert torch.equal(got.view(torch.int16), k[l, b, t].view(torch.int16))
+    # a subset, shorter: only sequence 2 changes
+    k3, v3 = make_synthetic_kv(cfg, 1, 10, seed=5)
+    gm.import_kv(k3, v3, seq_ids=[2])
+    assert [gm.seq_len(b) for b in range(B)] == [T, T, 10]
+    k4, _ = gm.export_kv(2, T)
+    assert torch.equal(k4.view(torch.int16), k[:, :2].contiguous().view(torch.int16))
+    k5, _ = gm.export_kv(1, 10, seq_ids=[2])
+    assert torch.equal(k5.view(torch.int16), k3.view(torch.int16))
+    with pytest.raises(binding.DbtError) as e:
+        gm.export_kv(1, 11, seq_ids=[2])  # longer than the sequence
+    assert e.value.status == 4
+    with pytest.raises(binding.DbtError) as e:
+        gm.import_kv(*make_synthetic_kv(cfg, 1, 65, seed=6))  # beyond four pages
+    assert e.value.status == 3
+    assert gm.sync_status() == (0, 0)
 
 
 def test_page_table_permutation_does_not_change_results():
@@ -207,8 +320,8 @@ def test_page_table_permutation_does_not_change_results():
     ob = _run_steps(b, tok, npre, True)
     for x, y in zip(oa, ob):
         assert torch.equal(x["z1"], y["z1"]) and torch.equal(x["z2"], y["z2"]) and torch.equal(x["next"], y["next"])
-    ka, _ = a.read_kv(B, T)
-    kb, _ = b.read_kv(B, T)
+    ka, _ = a.export_kv(B, T)
+    kb, _ = b.export_kv(B, T)
     assert torch.equal(ka.float(), kb.float())
 
 
@@ -258,6 +371,37 @@ def test_host_buffer_entry_points_match_device_entry_points():
 
 # ---- MoE ----------------------------------------------------------------------------------------------
 
+ROUTER_EPS = {"bf16": 1e-2, "fp32": 1e-4}  # router logits are O(1); half the bar on model logits
+
+
+def assert_routing_is_a_valid_topk(cfg, ex, rlog, what=""):
+    """ex [L, 2, B, kmax]: the device's expert ids; rlog [L, 2, B, E]: the oracle's router logits for the same
+    rows (computed under the device's choice in the earlier layers).  Eq. moe_layer fixes the selected set
+    only up to rounding at near-ties, so what must hold is: k distinct experts per row, none of them below
+    an unselected expert by more than the logit tolerance (softmax is monotone, so logits order as the
+    probabilities do), the unused slots -1, and under router replay (Section 4.3) the branch's set is the
+    primary's."""
+    eps = ROUTER_EPS[cfg.weight_dtype]
+    L, _, B, _ = ex.shape
+    replay = cfg.router_mode == 1
+    for l in range(L):
+        for p in range(2):
+            k = cfg.k_primary if (p == 0 or replay) else cfg.k_branch
+            for b in range(B):
+                chosen = ex[l, p, b, :k]
+                assert (ex[l, p, b, k:] == -1).all(), f"{what} layer {l} path {p} row {b}: unused slots"
+                assert ((chosen >= 0) & (chosen < cfg.n_experts)).all() and len(set(chosen.tolist())) == k, \
+                    f"{what} layer {l} path {p} row {b}: {chosen}"
+                if p == 1 and replay:
+                    assert chosen.tolist() == ex[l, 0, b, :k].tolist(), f"{what} layer {l} row {b}: replay set"
+                    continue
+                r = rlog[l, p, b]
+                rest = np.delete(r, chosen)
+                if rest.size:
+                    assert r[chosen].min() >= rest.max() - eps, \
+                        f"{what} layer {l} path {p} row {b}: chose {chosen} with logits {r[chosen]}, left {rest.max()}"
+
+
 def _moe_compare(cfg, B, T, npre, matrix_std=0.05):
     w = make_weights(cfg, seed=21, matrix_std=matrix_std)
     tok = make_tokens(cfg, B, T, seed=22)
@@ -265,40 +409,29 @@ def _moe_compare(cfg, B, T, npre, matrix_std=0.05):
     gm = make_gpu_model(cfg, w, B, T)
     z1_full, _, k_full, v_full = oracle.full_forward(cfg, w, tok[:, :npre].numpy(), want_kv=True)
     om.inject_kv(k_full, v_full, npre)
-    got = gm.prefill(tok[:, :npre].cuda().contiguous(), want_logits=True)
-    # prefill routes the primary path by top-k too; near-ties can flip, so compare loosely here
-    # and exactly (forced routing) in the decode steps below, which restart from the oracle's cache
-    gm.write_kv(torch.from_numpy(k_full), torch.from_numpy(v_full))
-    flips = 0
+    # the decode steps below start from the oracle's cache on both sides and impose the device's routing
+    # on the oracle; the prefill itself is compared in test_moe_prefill_matches_the_oracle
+    gm.import_kv(torch.from_numpy(k_full), torch.from_numpy(v_full))
     for t in range(npre, T):
         g = gm.decode_full(tok[:, t].cuda().contiguous())
         ex = gm.last_experts(B).numpy()
-        # the device's choice must be a valid top-k of the oracle's router up to rounding:
-        o_free = oracle.OracleModel(cfg, w, B, T)
-        o_free.inject_kv(om.k_cache[:, :B, :t], om.v_cache[:, :B, :t], t)
-        of = o_free.decode_step(tok[:, t].numpy())
-        flips += int((np.sort(of["experts"], -1) != np.sort(ex, -1)).any())
         o = om.decode_step(tok[:, t].numpy(), forced_experts=ex)
-        assert_logits_close(g["z1"], o["z1"], "bf16", f"moe step {t} z1")
-        assert_logits_close(g["z2"], o["z2"], "bf16", f"moe step {t} z2")
-        kp, kb = cfg.k_primary, (cfg.k_primary if cfg.router_mode == 1 else cfg.k_branch)
-        assert (ex[:, 0, :, :kp] >= 0).all() and (ex[:, 0, :, kp:] == -1).all()
-        assert (ex[:, 1, :, :kb] >= 0).all() and (ex[:, 1, :, kb:] == -1).all()
+        assert_routing_is_a_valid_topk(cfg, ex, om.router_logits(B), f"step {t}")
+        assert_logits_close(g["z1"], o["z1"], cfg.weight_dtype, f"moe step {t} z1")
+        assert_logits_close(g["z2"], o["z2"], cfg.weight_dtype, f"moe step {t} z2")
         union = gm.last_expert_union()
         for l in range(cfg.n_layers):
             assert union[l] == len(set(ex[l][ex[l] >= 0].tolist()))
-    assert got is not None
-    return flips
+    assert gm.sync_status() == (0, 0)
 
 
 @pytest.mark.parametrize("cfg", [small_moe(), small_moe(router_mode=1), small_moe(n_shared_experts=0, k_branch=8),
                                  small_moe(moe_b_coupling=0, k_primary=1, k_branch=1)])
 def test_moe_decode_matches_oracle_under_the_devices_routing(cfg):
-    """Router near-ties are decided by rounding, so the device's expert choice is read back,
-    checked for shape and union count, and imposed on the oracle; everything else is compared
-    element by element."""
-    flips = _moe_compare(cfg, B=3, T=14, npre=10)
-    assert flips <= 2  # well-separated router logits: the free-running oracle picks the same experts
+    """Router near-ties are decided by rounding, so the device's expert choice is read back, checked
+    row by row against the oracle's router logits (a valid top-k up to the logit tolerance), and imposed
+    on the oracle; everything else is compared element by element."""
+    _moe_compare(cfg, B=3, T=14, npre=10)
 
 
 @pytest.mark.parametrize("rowtile", ["auto", "32", "16", "0"])
@@ -307,14 +440,51 @@ def test_moe_at_batch_40(monkeypatch, rowtile):
     or 32 and the per-expert GEMMs walk several row tiles per expert (0: one tile of 128 rows)."""
     if rowtile != "auto":
         monkeypatch.setenv("DBT_MOE_ROWTILE", rowtile)
-    flips = _moe_compare(small_moe(k_primary=2, k_branch=2), B=40, T=7, npre=5)
-    assert flips <= 6
+    _moe_compare(small_moe(k_primary=2, k_branch=2), B=40, T=7, npre=5)
 
 
 def test_moe_1b_shape_two_layers():
     cfg = moe_1b(k_branch=4).replace(n_layers=2)
-    flips = _moe_compare(cfg, B=2, T=8, npre=6, matrix_std=0.02)
-    assert flips <= 2
+    _moe_compare(cfg, B=2, T=8, npre=6, matrix_std=0.02)
+
+
+@pytest.mark.parametrize("cfg", [small_moe(), small_moe(weight_dtype="fp32"), small_moe(compute_matched=1)])
+def test_moe_prefill_matches_the_oracle(cfg):
+    """dbt_prefill of an MoE model (Section 4.4 item 1: the primary path alone, fan-out k_1) against the
+    oracle's position-by-position primary pass: last-position logits and every cached K and V.  The router
+    matrix is scaled by 8 so that the k_1-th and (k_1+1)-th logits of every prompt row are far apart
+    (checked below on the oracle's logits): the selected sets are then unique and both sides must agree."""
+    w = make_weights(cfg, seed=79, matrix_std=0.05)
+    for lw in w["layers"]:
+        lw["router"] = (lw["router"].float() * 8).to(cfg.torch_dtype)
+    B, n = 3, 40
+    tok = make_tokens(cfg, B, n + 2, seed=179)
+    om = oracle.OracleModel(cfg, w, B, n + 2)
+    margin = np.inf
+    for t in range(n):  # the oracle's prefill is this loop (orc_prefill walks the prompt the same way)
+        o = om.decode_step(tok[:, t].numpy(), grouped=False)
+        r = -np.sort(-om.router_logits(B)[:, 0], axis=-1)
+        margin = min(margin, float((r[..., cfg.k_primary - 1] - r[..., cfg.k_primary]).min()))
+    # device router logits at this scale are good to ~8e-3 (8 x the error on unit-scale logits)
+    assert margin > 0.03, f"router logits not separated: {margin}"
+    gm = make_gpu_model(cfg, w, B, n + 2)
+    got = gm.prefill(tok[:, :n].cuda().contiguous(), want_logits=True)
+    assert_logits_close(got, o["z1"], cfg.weight_dtype, "moe prefill logits")
+    k_dev, v_dev = gm.export_kv(B, n)
+    # the device stores K and V in the model's type: bf16 rounding (2^-9 relative) on top of the logit-level error
+    rtol, atol = (2.0 ** -8, 5e-3) if cfg.weight_dtype == "bf16" else (1e-4, 1e-5)
+    np.testing.assert_allclose(k_dev.float().numpy(), om.k_cache[:, :B, :n], rtol=rtol, atol=atol)
+    np.testing.assert_allclose(v_dev.float().numpy(), om.v_cache[:, :B, :n], rtol=rtol, atol=atol)
+    assert float(k_dev.float().abs().max()) > 0.1
+    # and the caches are interchangeable: a grouped step on top of the device's own prefill
+    o2 = om.decode_step(tok[:, n].numpy())
+    g2 = gm.decode_full(tok[:, n].cuda().contiguous())
+    ex = gm.last_experts(B).numpy()
+    assert_routing_is_a_valid_topk(cfg, ex, om.router_logits(B), "step after prefill")
+    if (np.sort(ex, -1) == np.sort(o2["experts"], -1)).all():
+        assert_logits_close(g2["z1"], o2["z1"], cfg.weight_dtype, "step after moe prefill z1")
+        assert_logits_close(g2["z2"], o2["z2"], cfg.weight_dtype, "step after moe prefill z2")
+    assert gm.sync_status() == (0, 0)
 
 
 @pytest.mark.parametrize("matched", [0, 1])
@@ -332,7 +502,7 @@ def test_moe_1b_at_the_benchmarks_launch_configuration_on_sampled_sequences(matc
     gen = torch.Generator(device=gm.device)
     gen.manual_seed(5)
     gm.kv_pool.normal_(0.0, 1.0, generator=gen)
-    gm.write_kv(k, v, page_table=gm.page_table[pick])
+    gm.import_kv(k, v, seq_ids=pick)
     gm.set_seq_lens([ctx] * B)
     om = oracle.OracleModel(cfg, w, len(pick), ctx + 3)
     om.inject_kv(k, v, ctx)
@@ -340,9 +510,9 @@ def test_moe_1b_at_the_benchmarks_launch_configuration_on_sampled_sequences(matc
         g = gm.decode_full(tok[:, t].cuda().contiguous())
         ex = gm.last_experts(B).numpy()[:, :, pick]
         o = om.decode_step(tok[pick, t].numpy(), forced_experts=np.ascontiguousarray(ex))
+        assert_routing_is_a_valid_topk(cfg, np.ascontiguousarray(ex), om.router_logits(len(pick)), f"step {t}")
         assert_logits_close(g["z1"][pick], o["z1"], "bf16", f"moe bench config step {t} z1")
         assert_logits_close(g["z2"][pick], o["z2"], "bf16", f"moe bench config step {t} z2")
-        assert (ex[:, :, :, :2] >= 0).all()
     assert gm.sync_status() == (0, 0)
 
 
@@ -357,34 +527,29 @@ def test_moe_1b_at_the_benchmarks_launch_configuration_on_sampled_sequences(matc
 def test_compute_matched_moe_decode_matches_oracle(cfg):
     """The branch evaluates neither attention nor the shared expert: A_2 = g_A * A_1 and
     M_2 = R_2(N_2; k_2) + g_G * G(N_1), compared element by element under the device's routing."""
-    flips = _moe_compare(cfg, B=3, T=14, npre=10)
-    assert flips <= 2
+    _moe_compare(cfg, B=3, T=14, npre=10)
 
 
 @pytest.mark.parametrize("knob,value", [("DBT_FORCE_PATH", "simt"), ("DBT_ATTN", "simt"), ("DBT_MOE", "simt"),
-                                        ("DBT_FUSE_QKV", "0"), ("DBT_GRAPH", "0"), ("DBT_MOE_OVERLAP", "0"),
-                                        ("DBT_MOE_WIDE", "0")])
+                                        ("DBT_FUSE_QKV", "0"), ("DBT_GRAPH", "0"), ("DBT_MOE_OVERLAP", "0")])
 def test_compute_matched_moe_on_the_alternative_chains(monkeypatch, knob, value):
     monkeypatch.setenv(knob, value)
-    flips = _moe_compare(small_moe(compute_matched=1, k_primary=2, k_branch=2), B=5, T=13, npre=9)
-    assert flips <= 2
+    _moe_compare(small_moe(compute_matched=1, k_primary=2, k_branch=2), B=5, T=13, npre=9)
 
 
 @pytest.mark.parametrize("knob,value", [("DBT_MOE_OVERLAP", "0"), ("DBT_GRAPH", "0"), ("DBT_MOE", "simt"),
-                                        ("DBT_MOE_WIDE", "0"), ("DBT_FUSE_QKV", "0"), ("DBT_ATTN", "simt")])
+                                        ("DBT_FUSE_QKV", "0"), ("DBT_ATTN", "simt")])
 def test_moe_on_the_alternative_chains(monkeypatch, knob, value):
     """The shared expert on the main stream instead of beside the routed chain, direct launches instead
-    of graph replay, the SIMT expert kernels, row-wide norm kernels before the GEMMs instead of the norm
-    factor behind them, the separate Q|K|V epilogue kernel, the CUDA-core attention kernel."""
+    of graph replay, the CUDA-core expert kernels, the separate Q|K|V epilogue kernel, the CUDA-core
+    attention kernel."""
     monkeypatch.setenv(knob, value)
-    flips = _moe_compare(small_moe(), B=5, T=13, npre=9)
-    assert flips <= 2
+    _moe_compare(small_moe(), B=5, T=13, npre=9)
 
 
 def test_compute_matched_moe_1b_shape_two_layers():
     cfg = moe_1b(k_branch=2).replace(n_layers=2, compute_matched=1)
-    flips = _moe_compare(cfg, B=2, T=8, npre=6, matrix_std=0.02)
-    assert flips <= 2
+    _moe_compare(cfg, B=2, T=8, npre=6, matrix_std=0.02)
 
 
 def test_compute_matched_unit_gates_same_embedding_equal_fanout_give_identical_paths():
@@ -464,39 +629,20 @@ def test_fresh_models_give_bitwise_identical_results():
             assert torch.equal(x["z1"], y["z1"]) and torch.equal(x["z2"], y["z2"])
 
 
-@pytest.mark.parametrize("knob,value", [("DBT_READOUT", "row"), ("DBT_FUSED", "1"), ("DBT_WIDE", "0"), ("DBT_MEGA", "1"), ("DBT_L2_PREFETCH", "1"),
-                                        ("DBT_CLUSTER", "1"), ("DBT_CLUSTER_GU", "1"), ("DBT_FUSE_QKV", "0"), ("DBT_STACK", "0"), ("DBT_EVICT_FIRST", "0")])
+@pytest.mark.parametrize("knob,value", [("DBT_READOUT", "row"), ("DBT_FUSE_QKV", "0"), ("DBT_EVICT_FIRST", "0"),
+                                        ("DBT_GRAPH", "0"), ("DBT_PDL", "0"), ("DBT_ATTN", "simt"),
+                                        ("DBT_FORCE_PATH", "simt")])
 def test_alternative_kernel_chains_match_oracle(monkeypatch, knob, value):
-    """The variants of the dense chain that are not the default -- elementwise work folded into the
-    GEMM epilogues (last-arriving CTA per output tile), a row-wide residual+RMSNorm kernel before
-    each GEMM, the whole step as one persistent kernel, L2 prefetch requests riding on the GEMM
-    launches, the O / down projections reducing their splits inside a thread-block cluster, a
-    separate Q|K|V epilogue kernel, one MMA per activation plane, no L2 eviction hints -- compute
-    the same step."""
+    """The fallbacks of the dense chain -- the one-CTA-per-row readout (vocabularies beyond the chunked
+    kernel's reach), a separate Q|K|V epilogue kernel (the one prefill uses), no L2 eviction hints, direct
+    launches instead of graph replay, no programmatic dependent launch, the CUDA-core attention and GEMM
+    kernels (what fp32 models run on) -- compute the same step."""
     monkeypatch.setenv(knob, value)
     cfg = small_bf16()
     w = make_weights(cfg, seed=5, matrix_std=0.05)
     tok = make_tokens(cfg, 3, 40, seed=6)
     teacher_forced_compare(cfg, w, tok, n_prefill=35, grouped=True)
     teacher_forced_compare(cfg, w, tok, n_prefill=35, grouped=False)
-
-
-def test_single_kernel_step_across_row_tile_widths(monkeypatch):
-    """The persistent single-kernel step at batch sizes that select each of its row-tile widths
-    (16, 32, 64), with enough context for several attention stages per CTA."""
-    monkeypatch.setenv("DBT_MEGA", "1")
-    cfg = small_bf16(n_q_heads=2, n_kv_heads=1, head_dim=128, d_model=128, vocab=777, n_layers=2)
-    w = make_weights(cfg, seed=5, matrix_std=0.05)
-    for B, T, npre in [(5, 140, 132), (12, 24, 20), (30, 24, 20)]:
-        tok = make_tokens(cfg, B, T, seed=6)
-        teacher_forced_compare(cfg, w, tok, n_prefill=npre, grouped=True)
-    # and it is the path that ran: one launch per decode step
-    gm = make_gpu_model(cfg, w, 5, 32)
-    tok = make_tokens(cfg, 5, 8, seed=6).cuda()
-    gm.prefill(tok[:, :6].contiguous())
-    before = gm.launch_count()
-    gm.decode_step(tok[:, 6].contiguous())
-    assert gm.launch_count() - before == 1
 
 
 def test_8b_shape_two_layers_paged_with_shuffled_pages():
@@ -514,7 +660,7 @@ def test_8b_shape_two_layers_paged_with_shuffled_pages():
     pt = make_page_table(B, (ctx + 2 + 15) // 16, 40, seed=4)
     gm.set_page_table(pt)
     om.inject_kv(k, v, ctx)
-    gm.write_kv(k, v)
+    gm.import_kv(k, v)
     for t in range(2):
         o = om.decode_step(tok[:, t].numpy())
         g = gm.decode_full(tok[:, t].cuda().contiguous())
