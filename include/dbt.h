@@ -18,7 +18,7 @@
  *    never frees it and never writes the weights.  It must outlive the handle.
  *  - Matrices are row-major [out_features, in_features] (the paper's H W with W stored
  *    transposed), in `weight_dtype`.  Norm gains and the coupling vectors a, b, c are fp32.
- *  - Stacked activations are path-major: rows 0..B-1 primary, B..2B-1 branch.
+ *  - Stacked activations are path-major: rows 0..B-1 primary, then B rows per decode branch.
  *  - KV pool layout: [n_layers][2 (K,V)][num_pages][n_kv_heads][page_size][head_dim] in
  *    `weight_dtype`; K is stored after RoPE.  Logical position t of sequence b lives in
  *    physical page page_table[b][t / page_size], slot t % page_size.
@@ -74,6 +74,12 @@ typedef struct {
                                  attention and no shared expert; A_2 = g_A*A_1 (Eq. matched_attention),
                                  M_2 = R_2(N_2;k_2) + g_G*G(N_1) (Eq. matched_shared_expert); a, b, c are
                                  not applied.  MoE models only (DBT_ERR_UNSUPPORTED otherwise). */
+    int32_t n_paths;          /* K of Appendix C.1 ("More decode branches"): residual paths in all, the primary plus
+                                 K-1 decode branches.  Each branch has its own embedding table and same-position
+                                 state, reads the primary cache, shares a, b, c (and g_A, g_G) with the other
+                                 branches, routes for itself in MoE layers; the readout mixes p with the mean of
+                                 the branch distributions.  2 (or 0) is the main text's model; at most 8, and
+                                 n_paths * n_q_heads / n_kv_heads <= 16 (DBT_ERR_UNSUPPORTED otherwise). */
     int32_t max_batch, max_seq;
     int32_t page_size; /* tokens per KV page; 16 */
     int32_t num_pages; /* pages in the pool, per layer and per K/V */
@@ -95,7 +101,8 @@ typedef struct {
 } dbt_layer_weights;
 
 typedef struct {
-    const void *embed_primary, *embed_branch;  /* DEVICE E_1, E_2 [V,d]                       */
+    const void *embed_primary, *embed_branch;  /* DEVICE E_1 [V,d]; E_2..E_K one after another
+                                                  [n_paths-1][V,d]                            */
     const float *embed_norm_g, *final_norm_g;  /* DEVICE [d]                                  */
     const void *lm_head;                       /* DEVICE shared output matrix [V,d]           */
     const dbt_layer_weights *layers;           /* HOST array [n_layers] of DEVICE pointers    */
@@ -139,8 +146,9 @@ dbt_status dbt_prefill(dbt_model *m, const int32_t *tokens_dev, int32_t B, int32
  * tokens_dev[b] at position t_b = its length; the primary appends K_1,V_1[t_b]; both paths'
  * queries read positions 0..t_b of the primary cache; the shared matrices are applied to
  * the stacked rows; next_tokens_dev[b] = argmax of alpha*p + (1-alpha)*q (lowest index on
- * ties).  Lengths advance by one.  All pointers DEVICE; outputs may be NULL:
- * next_tokens_dev int32 [B] (may alias tokens_dev), logits_* fp32 [B][V], alpha_dev fp32 [B].
+ * ties; with more than one decode branch q is the mean of the branch distributions, Appendix C.1).
+ * Lengths advance by one.  All pointers DEVICE; outputs may be NULL: next_tokens_dev int32 [B] (may alias
+ * tokens_dev), logits_primary_dev fp32 [B][V], logits_branch_dev fp32 [n_paths-1][B][V], alpha_dev fp32 [B].
  * To start from a prompt x_1..x_S: prefill x_1..x_{S-1}, then pass x_S to the first step
  * (the boundary step of Section 4.4 item 2). */
 dbt_status dbt_decode_step(dbt_model *m, const int32_t *tokens_dev, int32_t B, int32_t *next_tokens_dev,
@@ -160,7 +168,7 @@ dbt_status dbt_decode_step_host(dbt_model *m, const int32_t *tokens_host, int32_
 dbt_status dbt_decode_step_primary_only_host(dbt_model *m, const int32_t *tokens_host, int32_t B,
                                              int32_t *next_tokens_host);
 
-/* MoE only: DEVICE int32 [n_layers][2][max_batch][kmax] (kmax = max(k_primary,k_branch)),
+/* MoE only: DEVICE int32 [n_layers][n_paths][max_batch][kmax] (kmax = max(k_primary,k_branch)),
  * the expert ids each row used in the last decode step (-1 padded); and the number of
  * distinct experts loaded per layer in the last step, HOST int32 [n_layers] (waits for the
  * stream).  Equation moe_layer leaves near-ties in the router to rounding, so tests read the

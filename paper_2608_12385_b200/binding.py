@@ -39,7 +39,7 @@ class DbtConfig(C.Structure):
                                          "vocab", "weight_dtype")]
     _fields_ += [("rope_base", C.c_float), ("rms_eps", C.c_float)]
     _fields_ += [(n, C.c_int32) for n in ("final_norm", "n_experts", "d_expert", "n_shared_experts", "k_primary",
-                                         "k_branch", "router_mode", "moe_b_coupling", "compute_matched", "max_batch", "max_seq",
+                                         "k_branch", "router_mode", "moe_b_coupling", "compute_matched", "n_paths", "max_batch", "max_seq",
                                          "page_size", "num_pages")]
 
 
@@ -115,7 +115,7 @@ def make_config_struct(cfg: ModelConfig, max_batch: int, max_seq: int, num_pages
                      rms_eps=cfg.rms_eps, final_norm=cfg.final_norm, n_experts=cfg.n_experts, d_expert=cfg.d_expert,
                      n_shared_experts=cfg.n_shared_experts, k_primary=cfg.k_primary, k_branch=cfg.k_branch,
                      router_mode=cfg.router_mode, moe_b_coupling=cfg.moe_b_coupling,
-                     compute_matched=cfg.compute_matched, max_batch=max_batch,
+                     compute_matched=cfg.compute_matched, n_paths=cfg.n_paths, max_batch=max_batch,
                      max_seq=max_seq, page_size=cfg.page_size, num_pages=num_pages)
 
 
@@ -304,7 +304,8 @@ class Model:
             buf = {"tok": torch.empty(B, dtype=torch.int32, device=self.device),
                    "next": torch.empty(B, dtype=torch.int32, device=self.device),
                    "z1": torch.empty(B, V, dtype=torch.float32, device=self.device),
-                   "z2": torch.empty(B, V, dtype=torch.float32, device=self.device),
+                   "z2": torch.empty((B, V) if self.cfg.n_paths == 2 else (self.cfg.n_paths - 1, B, V),
+                                     dtype=torch.float32, device=self.device),
                    "alpha": torch.empty(B, dtype=torch.float32, device=self.device)}
             cache[B] = buf
         buf["tok"].copy_(tokens_dev)
@@ -316,16 +317,16 @@ class Model:
 
     # -- diagnostics ----------------------------------------------------------------------
     def last_experts(self, batch: int) -> torch.Tensor:
-        """[n_layers, 2, batch, kmax] expert ids used by the last decode step."""
+        """[n_layers, n_paths, batch, kmax] expert ids used by the last decode step."""
         ptr, km = C.c_void_p(None), C.c_int32(0)
         self._check(self.L.dbt_last_experts(self._h, C.byref(ptr), C.byref(km)))
-        n = self.cfg.n_layers * 2 * self.max_batch * km.value
+        n = self.cfg.n_layers * self.cfg.n_paths * self.max_batch * km.value
         torch.cuda.synchronize(self.device)
         host = torch.empty(n, dtype=torch.int32)
         # the ids live inside the workspace tensor: locate them by address
         off = ptr.value - self.workspace.data_ptr()
         host.copy_(self.workspace[off:off + 4 * n].view(torch.int32).cpu())
-        return host.view(self.cfg.n_layers, 2, self.max_batch, km.value)[:, :, :batch].contiguous()
+        return host.view(self.cfg.n_layers, self.cfg.n_paths, self.max_batch, km.value)[:, :, :batch].contiguous()
 
     def last_expert_union(self) -> list[int]:
         buf = (C.c_int32 * self.cfg.n_layers)()

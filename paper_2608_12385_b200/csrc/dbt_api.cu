@@ -135,8 +135,14 @@ struct Carver {
 };
 
 int elem_bytes(const dbt_config &c) { return c.weight_dtype == DBT_DTYPE_F32 ? 4 : 2; }
+// Residual paths of the model: the primary and K-1 decode branches (Appendix C.1; 2 in the main text).
+int paths_of(const dbt_config &c) { return c.n_paths >= 2 ? c.n_paths : 2; }
+// The `grouped` argument of the step functions: 0 = the primary path alone, K >= 2 = all K paths stacked.
+int npaths(int grouped) { return grouped > 1 ? grouped : 1; }
+// Kernels that pair a primary row with one branch row run a block per branch in grid.z.
+unsigned branch_blocks(int grouped) { return grouped > 1 ? (unsigned)(grouped - 1) : 1u; }
 int kmax_of(const dbt_config &c) { return c.k_primary > c.k_branch ? c.k_primary : c.k_branch; }
-int prefill_rows(const dbt_config &c) { return 2 * c.max_batch > 256 ? 2 * c.max_batch : 256; }
+int prefill_rows(const dbt_config &c) { return paths_of(c) * c.max_batch > 256 ? paths_of(c) * c.max_batch : 256; }
 
 const char *check_config(const dbt_config *c, dbt_status *st) {
     *st = DBT_ERR_INVALID_ARG;
@@ -150,7 +156,8 @@ const char *check_config(const dbt_config *c, dbt_status *st) {
     if (c->head_dim != 64 && c->head_dim != 128) return "head_dim must be 64 or 128";
     if (c->page_size != 16) return "page_size must be 16";
     if (c->n_q_heads % c->n_kv_heads) return "n_q_heads must be a multiple of n_kv_heads";
-    if (2 * (c->n_q_heads / c->n_kv_heads) > 16) return "more than 16 queries per KV head over both paths";
+    if (c->n_paths != 0 && (c->n_paths < 2 || c->n_paths > 8)) return "n_paths must be 2..8 (0 = 2)";
+    if (paths_of(*c) * (c->n_q_heads / c->n_kv_heads) > 16) return "more than 16 queries per KV head over all paths";
     if (c->d_model % 8) return "d_model must be a multiple of 8";
     if (c->router_mode != DBT_ROUTER_INDEPENDENT && c->router_mode != DBT_ROUTER_REPLAY) return "unknown router_mode";
     if (c->compute_matched && c->n_experts <= 0) return "compute_matched is defined for MoE models only";
@@ -186,8 +193,8 @@ size_t carve(const dbt_config &c, char *base, Workspace *ws, int *Rmax_out, int 
     w.O = k.take<float>((size_t)Rmax * qd);
     w.G1 = k.take<float>((size_t)Rmax * F);
     w.M = k.take<float>((size_t)Rmax * d);
-    w.Z = k.take<float>((size_t)2 * c.max_batch * c.vocab);
-    w.Zrows = k.take<float>((size_t)2 * c.max_batch * d);
+    w.Z = k.take<float>((size_t)paths_of(c) * c.max_batch * c.vocab);
+    w.Zrows = k.take<float>((size_t)paths_of(c) * c.max_batch * d);
     w.part = k.take<float>((size_t)part_items * 16 * (c.head_dim + 2));
     w.rope = k.take<float2>((size_t)c.max_seq * (c.head_dim / 2));
     w.seq_len = k.take<int32_t>(c.max_batch);
@@ -195,7 +202,7 @@ size_t carve(const dbt_config &c, char *base, Workspace *ws, int *Rmax_out, int 
     w.status = k.take<int32_t>(4);
     w.att_tickets = k.take<int32_t>((size_t)Rmax * c.n_kv_heads);
     w.att_tickets2 = k.take<int32_t>((size_t)Rmax * c.n_kv_heads * kAttMaxGroups);
-    w.ro_stats = k.take<float>((size_t)c.max_batch * kRoMaxChunks * 8);
+    w.ro_stats = k.take<float>((size_t)c.max_batch * kRoMaxChunks * kRoRec);
     w.ro_tickets = k.take<int32_t>(c.max_batch);
     w.gemm_tickets = k.take<int32_t>(4096);
     w.tokens_stage = k.take<int32_t>(c.max_batch);
@@ -213,7 +220,7 @@ size_t carve(const dbt_config &c, char *base, Workspace *ws, int *Rmax_out, int 
         w.Hsh = k.take<float>((size_t)Rmax * (Fs > 0 ? Fs : 8));
         w.ecnt = k.take<int32_t>(c.n_experts);
         w.elist = k.take<int32_t>((size_t)c.n_experts * Rmax);
-        w.last_experts = k.take<int32_t>((size_t)c.n_layers * 2 * c.max_batch * km);
+        w.last_experts = k.take<int32_t>((size_t)c.n_layers * paths_of(c) * c.max_batch * km);
         w.union_cnt = k.take<int32_t>(c.n_layers);
     }
     if (c.weight_dtype == DBT_DTYPE_BF16) {
@@ -349,7 +356,7 @@ dbt_status run_readout(dbt_model *m, int B, int grouped, int32_t *next_dev, floa
         return DBT_OK;
     }
     int chunk = (c.vocab + nc - 1) / nc;
-    if (grouped) LAUNCH(m, "readout_stats", 0, readout_stats_kernel, dim3(B, nc), kRoThreads, 0, w.Z, B, c.vocab, chunk, w.ro_stats);
+    if (grouped) LAUNCH(m, "readout_stats", 0, readout_stats_kernel, dim3(B, nc), kRoThreads, 0, w.Z, B, c.vocab, grouped, chunk, w.ro_stats);
     LAUNCH(m, "readout", 0, readout_pick_kernel, dim3(B, nc), kRoThreads, 0, w.Z, B, c.vocab, chunk, grouped, w.ro_stats, w.ro_tickets,
            next_dev, alpha_dev, w.seq_len, 1);
     return DBT_OK;
@@ -386,7 +393,7 @@ template <typename KT, int DH>
 dbt_status run_attention(dbt_model *m, const RowMap &rm, int grouped, const KT *kpool, const KT *vpool, int nsplit,
                          double kv_bytes, bool out_bf16 = false) {
     const dbt_config &c = m->cfg;
-    int G = c.n_q_heads / c.n_kv_heads, nq = grouped ? 2 * G : G;
+    int G = c.n_q_heads / c.n_kv_heads, nq = npaths(grouped) * G;
     dim3 grid(rm.B * rm.cn, c.n_kv_heads, nsplit);
     int NQ = nq <= 1 ? 1 : nq <= 2 ? 2 : nq <= 4 ? 4 : nq <= 8 ? 8 : 16;
     const Workspace &w = m->ws;
@@ -419,15 +426,15 @@ dbt_status run_moe(dbt_model *m, int l, const RowMap &rm, int grouped, bool reco
     const dbt_config &c = m->cfg;
     const Workspace &w = m->ws;
     const dbt_layer_weights &lw = m->layers[l];
-    int Bc = rm.B * rm.cn, R = grouped ? 2 * Bc : Bc, d = c.d_model;
+    int Bc = rm.B * rm.cn, R = npaths(grouped) * Bc, d = c.d_model;
     dbt_status st;
     int E = c.n_experts, Fe = c.d_expert, km = kmax_of(c), Fs = c.n_shared_experts * Fe;
     LinArgs rl = lin1(lw.router, w.rlogits, E, R, w.X, d);
     if ((st = run_linear<WT>(m, "router", rl)) != DBT_OK) return st;
-    int32_t *last = record_experts ? w.last_experts + (size_t)l * 2 * c.max_batch * km : nullptr;
+    int32_t *last = record_experts ? w.last_experts + (size_t)l * paths_of(c) * c.max_batch * km : nullptr;
     if (last && !grouped)
-        CUDA_TRY(m, cudaMemsetAsync(last + (size_t)c.max_batch * km, 0xff, sizeof(int32_t) * c.max_batch * km,
-                                    m->stream));
+        CUDA_TRY(m, cudaMemsetAsync(last + (size_t)c.max_batch * km, 0xff,
+                                    sizeof(int32_t) * (paths_of(c) - 1) * c.max_batch * km, m->stream));
     LAUNCH(m, "route", 0, route_kernel, R, 32, 2 * E * sizeof(float), w.rlogits, 1, (size_t)0, E, Bc, c.k_primary, c.k_branch, km,
            c.router_mode == DBT_ROUTER_REPLAY, w.ridx, w.rwts, last, c.max_batch * km, (const float *)nullptr, 0, 0, d, c.rms_eps);
     int32_t *ucnt = record_experts ? w.union_cnt + l : nullptr;
@@ -464,7 +471,7 @@ template <typename WT>
 dbt_status run_layers(dbt_model *m, const RowMap &rm, int grouped, bool record_experts) {
     const dbt_config &c = m->cfg;
     const Workspace &w = m->ws;
-    int Bc = rm.B * rm.cn, R = grouped ? 2 * Bc : Bc;
+    int Bc = rm.B * rm.cn, R = npaths(grouped) * Bc;
     int d = c.d_model, qd = c.n_q_heads * c.head_dim, kvd = c.n_kv_heads * c.head_dim;
     size_t pool_layer_elems = (size_t)2 * c.num_pages * c.n_kv_heads * c.page_size * c.head_dim;
     size_t pool_kv_elems = pool_layer_elems / 2;
@@ -472,7 +479,7 @@ dbt_status run_layers(dbt_model *m, const RowMap &rm, int grouped, bool record_e
     nsplit = nsplit < 1 ? 1 : nsplit > 16 ? 16 : nsplit;
     // compute-matched allocation (Eq. matched_attention): attention is evaluated on the primary rows alone
     const bool matched = grouped && c.compute_matched;
-    const int ga = matched ? 0 : grouped, Ra = ga ? 2 * Bc : Bc;
+    const int ga = matched ? 0 : grouped, Ra = npaths(ga) * Bc;
     double kv_bytes = 0;  // K and V of every visible position, once per layer
     for (int b = 0; b < rm.B; b++)
         for (int j = 0; j < rm.cn; j++) kv_bytes += (double)(m->len_host[b] + j + 1) * 2 * kvd * sizeof(WT);
@@ -500,7 +507,7 @@ dbt_status run_layers(dbt_model *m, const RowMap &rm, int grouped, bool record_e
         if (st != DBT_OK) return st;
         // S-bar_i = S_i + Attn_i W_O  (matched: S-bar_2 = S_2 + g_A * Attn_1 W_O)
         LinArgs o = lin1(lw.wo, nullptr, d, Ra, w.O, qd, matched ? EPI_RESID_GATED : EPI_RESID);
-        o.S = w.S; o.Bc = Bc; o.coup = matched ? lw.gate_a : nullptr;
+        o.S = w.S; o.Bc = Bc; o.grouped = grouped; o.coup = matched ? lw.gate_a : nullptr;
         if ((st = run_linear<WT>(m, "linear_o", o)) != DBT_OK) return st;
         LAUNCH(m, "rmsnorm", 0, rmsnorm_kernel, R, 256, 0, w.S, lw.mlp_norm_g, c.rms_eps, d, 1, 0, 1, w.X);
         if (c.n_experts == 0) {
@@ -704,7 +711,7 @@ dbt_status run_attention_mma(dbt_model *m, const RowMap &rm, int grouped, int la
     dim3 grid(2 * m->num_sms);  // two resident CTAs per SM; each takes an equal share of all K/V tiles
     // up to 8 query rows per KV head over both paths: the transposed-product variant (fixed per
     // model, so that grouped and primary-only steps run the same arithmetic on the primary rows)
-    if (2 * G <= 8)
+    if (paths_of(c) * G <= 8)
         LAUNCH(m, "attention", kv_bytes, (attn_mma_kernel<DH, true>), grid, 160, AttCfg<DH>::kSmemBytes, m->map_kv, p);
     else
         LAUNCH(m, "attention", kv_bytes, (attn_mma_kernel<DH, false>), grid, 160, AttCfg<DH>::kSmemBytes, m->map_kv, p);
@@ -725,12 +732,12 @@ dbt_status run_moe_tc(dbt_model *m, int l, const RowMap &rm, int grouped, bool r
     const Workspace &w = m->ws;
     const dbt_layer_weights &lw = m->layers[l];
     const LayerMaps &mp = m->maps[l];
-    int Bc = rm.B * rm.cn, R = grouped ? 2 * Bc : Bc, d = c.d_model;
+    int Bc = rm.B * rm.cn, R = npaths(grouped) * Bc, d = c.d_model;
     int E = c.n_experts, Fe = c.d_expert, km = kmax_of(c), Fs = c.n_shared_experts * Fe, Rk = m->Rmax * km;
     // Row tile (and with it the resident-CTA count that sizes the split-K factors of the router and the shared
     // expert) from the batch, never from the mode: a primary-only step uses the tile of the grouped step, so both
     // add the same partials in the same order and write the same K/V bits.
-    int n_tile = pad_rows(2 * Bc <= 256 ? 2 * Bc : 256);
+    int n_tile = pad_rows(paths_of(c) * Bc <= 256 ? paths_of(c) * Bc : 256);
     size_t lo_x = m->act_parts == 2 ? (size_t)m->Rmax * d : 0;
     size_t lo_xs = m->act_parts == 2 ? (size_t)Rk * d : 0, lo_hs = m->act_parts == 2 ? (size_t)Rk * Fe : 0;
     const float *ssp = wide ? w.ss : nullptr;
@@ -751,7 +758,7 @@ dbt_status run_moe_tc(dbt_model *m, int l, const RowMap &rm, int grouped, bool r
         sg.nseg = 2; sg.X = &m->map_Xb; sg.K = d; sg.R = Rs; sg.P = Pbuf; sg.P_floats = Pbuf_floats; sg.tag = "shared_gateup";
         sg.parts = m->act_parts; sg.lo_row0 = m->Rmax;
         if ((st = run_gemm_tc(m, sg, nt, &nsp, &sstride)) != DBT_OK) return st;
-        LAUNCH(m, "swiglu_couple", 0, swiglu_couple_kernel, dim3(Bc, (Fs + 255) / 256), 256, 0, Pbuf, nsp, sstride, Fs, Bc,
+        LAUNCH(m, "swiglu_couple", 0, swiglu_couple_kernel, dim3(Bc, (Fs + 255) / 256, branch_blocks(matched ? 0 : grouped)), 256, 0, Pbuf, nsp, sstride, Fs, Bc,
                matched ? 0 : grouped, c.moe_b_coupling ? lw.coup_b : (const float *)nullptr, w.Hb,
                m->act_parts == 2 ? (size_t)m->Rmax * Fs : (size_t)0, ssp, ss_tiles, ss_ld, d, c.rms_eps);
         TcCall sd{};
@@ -782,9 +789,10 @@ dbt_status run_moe_tc(dbt_model *m, int l, const RowMap &rm, int grouped, bool r
     rt.W[0] = &mp.rt; rt.n_out[0] = E; rt.rows[0] = R; rt.nseg = 1; rt.X = &m->map_Xb; rt.K = d; rt.R = R;
     rt.P = w.P; rt.P_floats = w.P_floats; rt.tag = "router"; rt.parts = m->act_parts; rt.lo_row0 = m->Rmax;
     if ((st = run_gemm_tc(m, rt, n_tile, &rnsp, &rstride)) != DBT_OK) return st;
-    int32_t *last = record_experts ? w.last_experts + (size_t)l * 2 * c.max_batch * km : nullptr;
+    int32_t *last = record_experts ? w.last_experts + (size_t)l * paths_of(c) * c.max_batch * km : nullptr;
     if (last && !grouped)
-        CUDA_TRY(m, cudaMemsetAsync(last + (size_t)c.max_batch * km, 0xff, sizeof(int32_t) * c.max_batch * km, m->stream));
+        CUDA_TRY(m, cudaMemsetAsync(last + (size_t)c.max_batch * km, 0xff, sizeof(int32_t) * (paths_of(c) - 1) * c.max_batch * km,
+                                    m->stream));
     LAUNCH(m, "route", 0, route_kernel, R, 32, 2 * E * sizeof(float), w.P, rnsp, rstride, E, Bc, c.k_primary, c.k_branch, km,
            c.router_mode == DBT_ROUTER_REPLAY, w.ridx, w.rwts, last, c.max_batch * km, ssp, ss_tiles, ss_ld, d, c.rms_eps);
     LAUNCH(m, "moe_sort", 0, moe_sort_kernel, 1, 1024, 0, w.ridx, R, km, E, w.ecnt, w.eoff, w.epos,
@@ -804,7 +812,7 @@ dbt_status run_moe_tc(dbt_model *m, int l, const RowMap &rm, int grouped, bool r
     // could need, keep two CTAs per SM and their deeper rings at large batches (measured: 4.86 -> 4.53 ms
     // at batch 32, 6.43 -> 4.81 at batch 64).  DBT_MOE_ROWTILE=0: one tile of all rows; 16/32/64: that tile.
     int gt = n_tile, grt = 0;
-    const int want_tile = m->moe_row_tile >= 0 ? m->moe_row_tile : (2 * Bc <= 64 ? 16 : 32);
+    const int want_tile = m->moe_row_tile >= 0 ? m->moe_row_tile : (paths_of(c) * Bc <= 64 ? 16 : 32);
     if (want_tile > 0 && n_tile > want_tile) {
         gt = want_tile;
         grt = (R + gt - 1) / gt;
@@ -822,7 +830,7 @@ dbt_status run_moe_tc(dbt_model *m, int l, const RowMap &rm, int grouped, bool r
     if (Fs > 0 && !overlap && (st = shared_expert(w.P, w.P_floats)) != DBT_OK) return st;
     if (overlap) CUDA_TRY(m, cudaStreamWaitEvent(main_stream, m->ev_join, 0));
     const bool next_in = wide && g_next != nullptr;
-    LAUNCH(m, "moe_combine", 0, moe_combine_sorted_kernel, dim3(Bc, (d + 255) / 256), 256, 0, w.Yexp, Psh, nsp, sstride, w.ridx, w.epos, w.rwts, km,
+    LAUNCH(m, "moe_combine", 0, moe_combine_sorted_kernel, dim3(Bc, (d + 255) / 256, branch_blocks(grouped)), 256, 0, w.Yexp, Psh, nsp, sstride, w.ridx, w.epos, w.rwts, km,
            Bc, grouped, lw.coup_c, matched ? lw.gate_g : (const float *)nullptr, d, w.S, next_in ? g_next : (const float *)nullptr,
            next_in ? w.Xb : (__nv_bfloat16 *)nullptr, lo_x, next_in ? w.ss : (float *)nullptr, ss_ld);
     return DBT_OK;
@@ -836,7 +844,7 @@ dbt_status run_layers_tc(dbt_model *m, const RowMap &rm, int grouped, int n_tile
     typedef __nv_bfloat16 WT;
     const dbt_config &c = m->cfg;
     const Workspace &w = m->ws;
-    int Bc = rm.B * rm.cn, R = grouped ? 2 * Bc : Bc;
+    int Bc = rm.B * rm.cn, R = npaths(grouped) * Bc;
     int d = c.d_model, qd = c.n_q_heads * c.head_dim, kvd = c.n_kv_heads * c.head_dim;
     size_t pool_layer_elems = (size_t)2 * c.num_pages * c.n_kv_heads * c.page_size * c.head_dim;
     size_t pool_kv_elems = pool_layer_elems / 2;
@@ -848,7 +856,7 @@ dbt_status run_layers_tc(dbt_model *m, const RowMap &rm, int grouped, int n_tile
     bool moe = c.n_experts > 0;
     // compute-matched allocation (Eq. matched_attention): attention is evaluated on the primary rows alone
     const bool matched = grouped && c.compute_matched;
-    const int ga = matched ? 0 : grouped, Ra = ga ? 2 * Bc : Bc;
+    const int ga = matched ? 0 : grouped, Ra = npaths(ga) * Bc;
     // MoE on the tensor cores: norm factor behind the GEMMs, no row-wide reduction kernel (DBT_MOE_WIDE=0: before them)
     const bool mwide = moe && m->moe_tc && m->moe_wide;
     const int mss_tiles = (d + 255) / 256;
@@ -866,10 +874,10 @@ dbt_status run_layers_tc(dbt_model *m, const RowMap &rm, int grouped, int n_tile
         // has left it already, the first layer gets it from the residual kernel with nothing to add.
         if (mwide) {
             if (l == 0)
-                LAUNCH(m, "resid_wide", 0, resid_wide_kernel, dim3(Bc, mss_tiles), 256, 0, w.S, w.P, 0, (size_t)0, 1,
+                LAUNCH(m, "resid_wide", 0, resid_wide_kernel, dim3(Bc, mss_tiles, branch_blocks(grouped)), 256, 0, w.S, w.P, 0, (size_t)0, 1,
                        (const float *)nullptr, Bc, grouped, lw.attn_norm_g, d, w.Xb, lo_x, w.ss, m->Rmax);
         } else {
-            LAUNCH(m, "resid_norm", 0, resid_norm_kernel, Bc, norm_threads(d), 0, w.S, w.P, nsp, sstride, mode,
+            LAUNCH(m, "resid_norm", 0, resid_norm_kernel, dim3(Bc, 1, branch_blocks(grouped)), norm_threads(d), 0, w.S, w.P, nsp, sstride, mode,
                    l > 0 ? m->layers[l - 1].coup_c : nullptr, Bc, grouped, lw.attn_norm_g, c.rms_eps, d, 1, 1, 0, w.Xb,
                    lo_x, (float *)nullptr);
         }
@@ -882,7 +890,7 @@ dbt_status run_layers_tc(dbt_model *m, const RowMap &rm, int grouped, int n_tile
         const bool fuse = m->fuse_qkv && m->att_fast && rm.cn == 1;
         QkvFuse qf{w.P, nsp, sstride, mwide ? w.ss : nullptr, mwide ? mss_tiles : 0, mwide ? m->Rmax : 0, lw.coup_a};
         if (!fuse)
-            LAUNCH(m, "qkv_epilogue", 0, qkv_epilogue_kernel<WT>, dim3(Bc, c.n_q_heads + c.n_kv_heads), 64, 0, w.P, nsp, sstride, w.Q, rm, ga, c.n_q_heads,
+            LAUNCH(m, "qkv_epilogue", 0, qkv_epilogue_kernel<WT>, dim3(Bc, c.n_q_heads + c.n_kv_heads, branch_blocks(ga)), 64, 0, w.P, nsp, sstride, w.Q, rm, ga, c.n_q_heads,
                    c.n_kv_heads, c.head_dim, lw.coup_a, w.rope, w.seq_len, w.page_table, m->pages_per_seq_max, c.num_pages,
                    c.page_size, kpool, vpool, w.status, mwide ? (const float *)w.ss : (const float *)nullptr, mwide ? mss_tiles : 0,
                    mwide ? m->Rmax : 0, d, c.rms_eps);
@@ -900,10 +908,10 @@ dbt_status run_layers_tc(dbt_model *m, const RowMap &rm, int grouped, int n_tile
         if ((st = run_gemm_tc(m, op, n_tile, &nsp, &sstride)) != DBT_OK) return st;
         // S-bar_i = S_i + Attn_i W_O (matched: S-bar_2 = S_2 + g_A * Attn_1 W_O) ; RMSNorm for the MLP
         if (mwide)
-            LAUNCH(m, "resid_wide", 0, resid_wide_kernel, dim3(Bc, mss_tiles), 256, 0, w.S, w.P, nsp, sstride, matched ? 3 : 1,
+            LAUNCH(m, "resid_wide", 0, resid_wide_kernel, dim3(Bc, mss_tiles, branch_blocks(grouped)), 256, 0, w.S, w.P, nsp, sstride, matched ? 3 : 1,
                    matched ? lw.gate_a : (const float *)nullptr, Bc, grouped, lw.mlp_norm_g, d, w.Xb, lo_x, w.ss, m->Rmax);
         else
-        LAUNCH(m, "resid_norm", 0, resid_norm_kernel, Bc, norm_threads(d), 0, w.S, w.P, nsp, sstride, matched ? 3 : 1,
+        LAUNCH(m, "resid_norm", 0, resid_norm_kernel, dim3(Bc, 1, branch_blocks(grouped)), norm_threads(d), 0, w.S, w.P, nsp, sstride, matched ? 3 : 1,
                matched ? lw.gate_a : (const float *)nullptr, Bc,
                grouped, lw.mlp_norm_g, c.rms_eps, d, 1, 1, 0, w.Xb, lo_x, moe && !m->moe_tc ? w.X : (float *)nullptr);
         if (!moe) {
@@ -913,7 +921,7 @@ dbt_status run_layers_tc(dbt_model *m, const RowMap &rm, int grouped, int n_tile
             gu.W[1] = &mp.wu; gu.n_out[1] = F; gu.rows[1] = R;
             gu.nseg = 2; gu.X = &m->map_Xb; gu.K = d; gu.R = R; gu.P = w.P; gu.P_floats = w.P_floats; gu.parts = m->act_parts; gu.lo_row0 = m->Rmax; gu.tag = "gemm_gateup";
             if ((st = run_gemm_tc(m, gu, n_tile, &nsp, &sstride)) != DBT_OK) return st;
-            dim3 sg(Bc, (F + 255) / 256);
+            dim3 sg(Bc, (F + 255) / 256, branch_blocks(grouped));
             LAUNCH(m, "swiglu_couple", 0, swiglu_couple_kernel, sg, 256, 0, w.P, nsp, sstride, F, Bc, grouped, lw.coup_b,
                    w.Hb, m->act_parts == 2 ? (size_t)m->Rmax * F : (size_t)0, (const float *)nullptr, 0, 0, d, c.rms_eps);
             TcCall dn{};
@@ -940,10 +948,10 @@ dbt_status run_head_tc(dbt_model *m, int Bc_src, int grouped, int n_rows_out, in
                        int mode, int nsp, size_t sstride) {
     const dbt_config &c = m->cfg;
     const Workspace &w = m->ws;
-    LAUNCH(m, "resid_norm", 0, resid_norm_kernel, n_rows_out, norm_threads(c.d_model), 0, w.S, w.P, nsp, sstride, mode,
+    LAUNCH(m, "resid_norm", 0, resid_norm_kernel, dim3(n_rows_out, 1, branch_blocks(grouped)), norm_threads(c.d_model), 0, w.S, w.P, nsp, sstride, mode,
            m->layers[c.n_layers - 1].coup_c, Bc_src, grouped, m->w.final_norm_g, c.rms_eps, c.d_model, c.final_norm,
            src_mul, src_add, w.Xb, m->act_parts == 2 ? (size_t)m->Rmax * c.d_model : (size_t)0, (float *)nullptr);
-    int R = grouped ? 2 * n_rows_out : n_rows_out;
+    int R = npaths(grouped) * n_rows_out;
     TcCall lm{};
     lm.W[0] = &m->map_lm; lm.n_out[0] = c.vocab; lm.rows[0] = R; lm.nseg = 1; lm.X = &m->map_Xb; lm.K = c.d_model;
     lm.R = R; lm.P = w.Z; lm.P_floats = (size_t)R * c.vocab;  // exactly one split: Z is the output itself
@@ -958,8 +966,8 @@ dbt_status step_tc(dbt_model *m, const int32_t *tokens_dev, int B, int grouped, 
     const dbt_config &c = m->cfg;
     const Workspace &w = m->ws;
     RowMap rm{B, 1};
-    int R = grouped ? 2 * B : B;
-    int n_tile = pad_rows(2 * B);  // the same instruction shape in both modes
+    int R = npaths(grouped) * B;
+    int n_tile = pad_rows(paths_of(c) * B);  // the same instruction shape in both modes
     dbt_status st;
     LAUNCH(m, "embed", 0, embed_norm_kernel<WT>, R, 256, 0, tokens_dev, 1, 0, rm, (const WT *)m->w.embed_primary,
            (const WT *)m->w.embed_branch, m->w.embed_norm_g, c.rms_eps, c.d_model, c.vocab, w.S, w.status);
@@ -971,8 +979,8 @@ dbt_status step_tc(dbt_model *m, const int32_t *tokens_dev, int B, int grouped, 
     if ((st = run_readout(m, B, grouped, next_dev, alpha_dev)) != DBT_OK) return st;
     size_t zb = sizeof(float) * (size_t)B * c.vocab;
     if (z1_dev) CUDA_TRY(m, cudaMemcpyAsync(z1_dev, w.Z, zb, cudaMemcpyDeviceToDevice, m->stream));
-    if (z2_dev && grouped)
-        CUDA_TRY(m, cudaMemcpyAsync(z2_dev, w.Z + (size_t)B * c.vocab, zb, cudaMemcpyDeviceToDevice, m->stream));
+    if (z2_dev && grouped)  // the branches' logits, branch-major [K-1][B][V]
+        CUDA_TRY(m, cudaMemcpyAsync(z2_dev, w.Z + (size_t)B * c.vocab, zb * (npaths(grouped) - 1), cudaMemcpyDeviceToDevice, m->stream));
     for (int b = 0; b < B; b++) m->len_host[b] += 1;
     m->pending_union = c.n_experts > 0;
     return DBT_OK;
@@ -1017,7 +1025,7 @@ dbt_status run_layers_wide(dbt_model *m, const RowMap &rm, int grouped, int n_ti
     typedef __nv_bfloat16 WT;
     const dbt_config &c = m->cfg;
     const Workspace &w = m->ws;
-    int Bc = rm.B * rm.cn, R = grouped ? 2 * Bc : Bc;
+    int Bc = rm.B * rm.cn, R = npaths(grouped) * Bc;
     int d = c.d_model, qd = c.n_q_heads * c.head_dim, kvd = c.n_kv_heads * c.head_dim, F = c.d_ff;
     size_t pool_layer_elems = (size_t)2 * c.num_pages * c.n_kv_heads * c.page_size * c.head_dim;
     size_t lo_x = m->act_parts == 2 ? (size_t)m->Rmax * d : 0, lo_h = m->act_parts == 2 ? (size_t)m->Rmax * F : 0;
@@ -1048,7 +1056,7 @@ dbt_status run_layers_wide(dbt_model *m, const RowMap &rm, int grouped, int n_ti
         const bool fuse = m->fuse_qkv && rm.cn == 1;
         QkvFuse qf{w.P, nsp, sstride, w.ss, ss_tiles, ss_ld, lw.coup_a};
         if (!fuse)
-            LAUNCH(m, "qkv_epilogue", 0, qkv_epilogue_kernel<WT>, dim3(Bc, c.n_q_heads + c.n_kv_heads), 64, 0, w.P, nsp, sstride,
+            LAUNCH(m, "qkv_epilogue", 0, qkv_epilogue_kernel<WT>, dim3(Bc, c.n_q_heads + c.n_kv_heads, branch_blocks(grouped)), 64, 0, w.P, nsp, sstride,
                    w.Q, rm, grouped, c.n_q_heads, c.n_kv_heads, c.head_dim, lw.coup_a, w.rope, w.seq_len, w.page_table,
                    m->pages_per_seq_max, c.num_pages, c.page_size, kpool, vpool, w.status, (const float *)w.ss, ss_tiles, ss_ld, d,
                    c.rms_eps);
@@ -1059,7 +1067,7 @@ dbt_status run_layers_wide(dbt_model *m, const RowMap &rm, int grouped, int n_ti
         op.W[0] = &mp.wo; op.n_out[0] = d; op.rows[0] = R; op.nseg = 1;
         {
             if ((st = run_gemm_tc(m, op, n_tile, &nsp, &sstride)) != DBT_OK) return st;
-            LAUNCH(m, "resid_wide", 0, resid_wide_kernel, dim3(Bc, ss_tiles), 256, 0, w.S, w.P, nsp, sstride, 1,
+            LAUNCH(m, "resid_wide", 0, resid_wide_kernel, dim3(Bc, ss_tiles, branch_blocks(grouped)), 256, 0, w.S, w.P, nsp, sstride, 1,
                    (const float *)nullptr, Bc, grouped, lw.mlp_norm_g, d, w.Xb, lo_x, w.ss, ss_ld);
         }
         TcCall gu = call("gemm_gateup", &m->map_Xb, d);
@@ -1068,7 +1076,7 @@ dbt_status run_layers_wide(dbt_model *m, const RowMap &rm, int grouped, int n_ti
         gu.nseg = 2;
         {
             if ((st = run_gemm_tc(m, gu, n_tile, &nsp, &sstride)) != DBT_OK) return st;
-            LAUNCH(m, "swiglu_couple", 0, swiglu_couple_kernel, dim3(Bc, (F + 255) / 256), 256, 0, w.P, nsp, sstride, F, Bc,
+            LAUNCH(m, "swiglu_couple", 0, swiglu_couple_kernel, dim3(Bc, (F + 255) / 256, branch_blocks(grouped)), 256, 0, w.P, nsp, sstride, F, Bc,
                    grouped, lw.coup_b, w.Hb, lo_h, (const float *)w.ss, ss_tiles, ss_ld, d, c.rms_eps);
         }
         TcCall dn = call("gemm_down", &m->map_Hb, F);
@@ -1077,7 +1085,7 @@ dbt_status run_layers_wide(dbt_model *m, const RowMap &rm, int grouped, int n_ti
                                                  : (c.final_norm ? m->w.final_norm_g : (const float *)nullptr);
         {
             if ((st = run_gemm_tc(m, dn, n_tile, &nsp, &sstride)) != DBT_OK) return st;
-            LAUNCH(m, "resid_wide", 0, resid_wide_kernel, dim3(Bc, ss_tiles), 256, 0, w.S, w.P, nsp, sstride, 2, lw.coup_c, Bc,
+            LAUNCH(m, "resid_wide", 0, resid_wide_kernel, dim3(Bc, ss_tiles, branch_blocks(grouped)), 256, 0, w.S, w.P, nsp, sstride, 2, lw.coup_c, Bc,
                    grouped, g_next, d, w.Xb, lo_x, w.ss, ss_ld);
         }
     }
@@ -1087,7 +1095,7 @@ dbt_status run_layers_wide(dbt_model *m, const RowMap &rm, int grouped, int n_ti
 dbt_status run_head_wide(dbt_model *m, const RowMap &rm, int grouped, int n_tile) {
     const dbt_config &c = m->cfg;
     const Workspace &w = m->ws;
-    int R = (grouped ? 2 : 1) * rm.B * rm.cn;
+    int R = npaths(grouped) * rm.B * rm.cn;
     TcCall lm{};
     lm.W[0] = &m->map_lm; lm.n_out[0] = c.vocab; lm.rows[0] = R; lm.nseg = 1; lm.X = &m->map_Xb; lm.K = c.d_model;
     lm.R = R; lm.P = w.Z; lm.P_floats = (size_t)R * c.vocab; lm.tag = "gemm_lm_head";
@@ -1120,7 +1128,7 @@ dbt_status step_wide(dbt_model *m, const int32_t *tokens_dev, int B, int grouped
     const dbt_config &c = m->cfg;
     const Workspace &w = m->ws;
     RowMap rm{B, 1};
-    int R = grouped ? 2 * B : B, n_tile = pad_rows(2 * B);
+    int R = npaths(grouped) * B, n_tile = pad_rows(paths_of(c) * B);
     dbt_status st;
     if ((st = run_embed_wide<WT>(m, tokens_dev, 1, 0, rm, R, n_tile)) != DBT_OK) return st;
     if ((st = run_layers_wide(m, rm, grouped, n_tile)) != DBT_OK) return st;
@@ -1129,8 +1137,8 @@ dbt_status step_wide(dbt_model *m, const int32_t *tokens_dev, int B, int grouped
     if ((st = run_readout(m, B, grouped, next_dev, alpha_dev)) != DBT_OK) return st;
     size_t zb = sizeof(float) * (size_t)B * c.vocab;
     if (z1_dev) CUDA_TRY(m, cudaMemcpyAsync(z1_dev, w.Z, zb, cudaMemcpyDeviceToDevice, m->stream));
-    if (z2_dev && grouped)
-        CUDA_TRY(m, cudaMemcpyAsync(z2_dev, w.Z + (size_t)B * c.vocab, zb, cudaMemcpyDeviceToDevice, m->stream));
+    if (z2_dev && grouped)  // the branches' logits, branch-major [K-1][B][V]
+        CUDA_TRY(m, cudaMemcpyAsync(z2_dev, w.Z + (size_t)B * c.vocab, zb * (npaths(grouped) - 1), cudaMemcpyDeviceToDevice, m->stream));
     for (int b = 0; b < B; b++) m->len_host[b] += 1;
     return DBT_OK;
 }
@@ -1255,7 +1263,7 @@ dbt_status step_impl(dbt_model *m, const int32_t *tokens_dev, int B, int grouped
     const dbt_config &c = m->cfg;
     const Workspace &w = m->ws;
     RowMap rm{B, 1};
-    int R = grouped ? 2 * B : B;
+    int R = npaths(grouped) * B;
     dbt_status st;
     LAUNCH(m, "embed", 0, embed_norm_kernel<WT>, R, 256, 0, tokens_dev, 1, 0, rm, (const WT *)m->w.embed_primary,
            (const WT *)m->w.embed_branch, m->w.embed_norm_g, c.rms_eps, c.d_model, c.vocab, w.S, w.status);
@@ -1265,8 +1273,8 @@ dbt_status step_impl(dbt_model *m, const int32_t *tokens_dev, int B, int grouped
     if ((st = run_readout(m, B, grouped, next_dev, alpha_dev)) != DBT_OK) return st;
     size_t zb = sizeof(float) * (size_t)B * c.vocab;
     if (z1_dev) CUDA_TRY(m, cudaMemcpyAsync(z1_dev, w.Z, zb, cudaMemcpyDeviceToDevice, m->stream));
-    if (z2_dev && grouped)
-        CUDA_TRY(m, cudaMemcpyAsync(z2_dev, w.Z + (size_t)B * c.vocab, zb, cudaMemcpyDeviceToDevice, m->stream));
+    if (z2_dev && grouped)  // the branches' logits, branch-major [K-1][B][V]
+        CUDA_TRY(m, cudaMemcpyAsync(z2_dev, w.Z + (size_t)B * c.vocab, zb * (npaths(grouped) - 1), cudaMemcpyDeviceToDevice, m->stream));
     for (int b = 0; b < B; b++) m->len_host[b] += 1;
     m->pending_union = c.n_experts > 0;
     return DBT_OK;
@@ -1446,7 +1454,7 @@ dbt_status dbt_create(const dbt_config *cfg, const dbt_weights *w, void *kv_pool
     if (e == cudaSuccess) e = cudaMemsetAsync(m->ws.ro_tickets, 0, sizeof(int32_t) * (size_t)cfg->max_batch, m->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(m->ws.gemm_tickets, 0, sizeof(int32_t) * 4096, m->stream);
     if (e == cudaSuccess && moe) {
-        e = cudaMemsetAsync(m->ws.last_experts, 0xff, sizeof(int32_t) * (size_t)cfg->n_layers * 2 * cfg->max_batch * kmax_of(*cfg), m->stream);
+        e = cudaMemsetAsync(m->ws.last_experts, 0xff, sizeof(int32_t) * (size_t)cfg->n_layers * paths_of(*cfg) * cfg->max_batch * kmax_of(*cfg), m->stream);
         if (e == cudaSuccess) e = cudaMemsetAsync(m->ws.union_cnt, 0, sizeof(int32_t) * cfg->n_layers, m->stream);
     }
     if (e == cudaSuccess) e = cudaStreamSynchronize(m->stream);  // the host vectors go out of scope
@@ -1662,7 +1670,7 @@ dbt_status dbt_decode_step(dbt_model *m, const int32_t *tokens_dev, int32_t B, i
                            float *logits_primary_dev, float *logits_branch_dev, float *alpha_dev) {
     dbt_status st = check_step_args(m, tokens_dev, B, 1);
     if (st != DBT_OK) return st;
-    return step_graphed(m, tokens_dev, B, 1, next_tokens_dev, logits_primary_dev, logits_branch_dev, alpha_dev);
+    return step_graphed(m, tokens_dev, B, paths_of(m->cfg), next_tokens_dev, logits_primary_dev, logits_branch_dev, alpha_dev);
 }
 
 dbt_status dbt_decode_step_primary_only(dbt_model *m, const int32_t *tokens_dev, int32_t B, int32_t *next_tokens_dev,

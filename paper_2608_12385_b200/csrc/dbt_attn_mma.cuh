@@ -34,7 +34,8 @@ namespace dbt {
 struct AttnParams {
     const float *Q;  // [rows][q_dim] fp32, post-RoPE, branch rows already coupled
     RowMap rm;
-    int grouped, G, n_kv, num_pages, pt_stride;
+    int grouped;  // paths present: 0 or 1 = the primary alone, P >= 2 = the primary and P-1 decode branches
+    int G, n_kv, num_pages, pt_stride;
     long long k_row0;  // first row of this layer's K plane in the pool's row numbering (the V plane is one plane further)
     const int32_t *page_table, *seq_len;
     float *part;        // [CTAs + pairs][16][DH + 2] segment partials
@@ -78,7 +79,7 @@ struct AttCfg {
     // scratch: one [16][DH + 8] fp32 slot (Q tile / warp fold; the padding keeps the fold's
     // fragment-shaped accesses off a single bank), m, l, flag, row tables
     static constexpr int kFoldStride = DH + 8;
-    static constexpr int kScratchBytes = (16 * kFoldStride + 2 * 16 + 8 + 3 * kAttMaxItems + 12) * 4 + 2 * DH * 2 + 32;
+    static constexpr int kScratchBytes = (16 * kFoldStride + 2 * 16 + 16 + 3 * kAttMaxItems + 12) * 4 + 2 * DH * 2 + 32;
     static constexpr int kSmemBytes = kStages * kStageBytes + 1024 + 128 + kScratchBytes;
 };
 
@@ -140,8 +141,8 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
     float *sc_o = reinterpret_cast<float *>(gen + STAGES * Cfg::kStageBytes + 128);  // [16][FS]
     float *sc_m = sc_o + 16 * FS;                                                   // [16]
     float *sc_l = sc_m + 16;                                                        // [16]
-    int *flag = reinterpret_cast<int *>(sc_l + 16);                                 // [0] last?, [1] longest pair
-    int *cum = flag + 8;                 // [items + 1] prefix of tiles per row
+    int *flag = reinterpret_cast<int *>(sc_l + 16);                                 // [0] last?, [1] longest pair, [8..15] 1/rms per path
+    int *cum = flag + 16;                // [items + 1] prefix of tiles per row
     int *nk_s = cum + kAttMaxItems + 1;  // [items] visible keys per row
     int *segcum = nk_s + kAttMaxItems;   // [items + 1] prefix of segments per row (per KV head)
     __nv_bfloat16 *kv_new =  // [2][DH] this step's K, V row (16-byte aligned)
@@ -150,7 +151,8 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
     DBT_TL_DECL;
     int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     int items = p.rm.Bc(), Bc = items;
-    int nq_act = p.grouped ? 2 * p.G : p.G, q_dim = p.n_kv * p.G * DH;
+    const int P = p.grouped > 1 ? p.grouped : 1;  // query rows of a KV head: G heads of every path, path-major
+    int nq_act = P * p.G, q_dim = p.n_kv * p.G * DH;
 
     if (tid == 0) {
         for (int s = 0; s < STAGES; s++) {
@@ -338,8 +340,8 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
                 int q = idx / (DH / 4), c4 = idx % (DH / 4);
                 float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (q < nq_act) {
-                    int row = q < p.G ? item : Bc + item;
-                    int h = g * p.G + (q < p.G ? q : q - p.G);
+                    int row = (q / p.G) * Bc + item;
+                    int h = g * p.G + q % p.G;
                     v = __ldcg(reinterpret_cast<const float4 *>(p.Q + (size_t)row * q_dim + (size_t)h * DH) + c4);
                 }
                 reinterpret_cast<float4 *>(sc_o)[idx] = v;
@@ -347,12 +349,14 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
         } else {
             constexpr int half = DH / 2;
             const int kv_dim = p.n_kv * DH, ldp = q_dim + 2 * kv_dim, pos = nkeys - 1;
-            const int twin = p.grouped ? Bc + item : item;
+            const bool grp = P > 1;
+            const int twin = grp ? Bc + item : item;  // the first branch's row travels with the primary's loads
             const size_t p1 = (size_t)item * ldp, p2 = (size_t)twin * ldp;
-            // One round of loads: the first warp requests the norm shares of the two rows (lanes
-            // 0..15 the primary row, 16..31 its twin) and hands 1/rms to the others through shared
-            // memory; every thread requests the partials, the rotation and the coupling of its
-            // outputs before anyone waits.
+            // One round of loads: the first warp requests the norm shares of the pair's rows (lanes
+            // 0..15 the primary row, 16..31 the first branch's) and hands 1/rms to the others through
+            // shared memory; every thread requests the partials, the rotation and the coupling of its
+            // outputs before anyone waits.  Further decode branches (Appendix C.1) follow in rounds of
+            // their own.
             float myss = 0.f;
             if (p.ss && warp == 0)
                 for (int t = lane & 15; t < p.ss_tiles; t += 16) myss += __ldcg(p.ss + (size_t)t * p.ss_ld + (lane < 16 ? item : twin));
@@ -360,7 +364,7 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
                 reinterpret_cast<float4 *>(sc_o + (size_t)nq_act * DH)[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
             const int nitems = p.G * half;
             const bool do_kv = owns_last && tid < half;
-            float *rs_s = reinterpret_cast<float *>(flag + 2);
+            float *rs_s = reinterpret_cast<float *>(flag + 8);  // [path]
             float rs1 = 1.f, rs2 = 1.f, kvs[4] = {0.f, 0.f, 0.f, 0.f};
             float2 t_kv = make_float2(1.f, 0.f);
             for (int it0 = 0; it0 * 128 < nitems; it0++) {
@@ -369,7 +373,7 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
                 int j = act ? idx / half : 0, i = act ? idx % half : tid % half;
                 int o0 = (g * p.G + j) * DH + i, o1 = o0 + half;
                 float2 t = p.rope[(size_t)pos * half + i];
-                float ca0 = p.grouped ? p.coup_a[o0] : 0.f, ca1 = p.grouped ? p.coup_a[o1] : 0.f;
+                float ca0 = grp ? p.coup_a[o0] : 0.f, ca1 = grp ? p.coup_a[o1] : 0.f;
                 const size_t offs[4] = {p1 + o0, p1 + o1, p2 + o0, p2 + o1};
                 float sm[4] = {0.f, 0.f, 0.f, 0.f};
                 if (act) sum_splits_k<4, 12>(p.qkv_P, p.qkv_stride, p.qkv_nsplit, offs, sm);
@@ -388,6 +392,19 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
                             for (int k = 0; k < 16; k++) a += sc_m[lane + k];
                             rs_s[lane >> 4] = p.ss ? 1.f / sqrtf(a / (float)p.d_norm + p.eps) : 1.f;
                         }
+                        for (int jp = 2; jp < P; jp++) {  // further branches: the whole warp per row
+                            float a = 0.f;
+                            if (p.ss)
+                                for (int t2 = lane; t2 < p.ss_tiles; t2 += 32) a += __ldcg(p.ss + (size_t)t2 * p.ss_ld + jp * Bc + item);
+                            sc_m[lane] = a;
+                            __syncwarp();
+                            if (lane == 0) {
+                                float tot = 0.f;
+                                for (int k = 0; k < 32; k++) tot += sc_m[k];
+                                rs_s[jp] = p.ss ? 1.f / sqrtf(tot / (float)p.d_norm + p.eps) : 1.f;
+                            }
+                            __syncwarp();
+                        }
                     }
                     consumer_sync();
                     rs1 = rs_s[0];
@@ -398,10 +415,20 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
                     float r0 = x0 * t.x - x1 * t.y, r1 = x1 * t.x + x0 * t.y;
                     sc_o[(size_t)j * DH + i] = r0;
                     sc_o[(size_t)j * DH + i + half] = r1;
-                    if (p.grouped) {
+                    if (grp) {
                         float y0 = rs2 * sm[2], y1 = rs2 * sm[3];
                         sc_o[(size_t)(p.G + j) * DH + i] = (y0 * t.x - y1 * t.y) + ca0 * r0;
                         sc_o[(size_t)(p.G + j) * DH + i + half] = (y1 * t.x + y0 * t.y) + ca1 * r1;
+                    }
+                    for (int jp = 2; jp < P; jp++) {  // Q~_j = Q_j + a * Q_1 for the further branches
+                        const size_t pj = (size_t)(jp * Bc + item) * ldp;
+                        const size_t offj[2] = {pj + o0, pj + o1};
+                        float sj[2];
+                        sum_splits_k<2, 12>(p.qkv_P, p.qkv_stride, p.qkv_nsplit, offj, sj);
+                        const float rsj = rs_s[jp];
+                        float y0 = rsj * sj[0], y1 = rsj * sj[1];
+                        sc_o[(size_t)(jp * p.G + j) * DH + i] = (y0 * t.x - y1 * t.y) + ca0 * r0;
+                        sc_o[(size_t)(jp * p.G + j) * DH + i + half] = (y1 * t.x + y0 * t.y) + ca1 * r1;
                     }
                 }
             }
@@ -610,8 +637,8 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
                         if (q < nq_act) {
                             if (nseg == 1) {
                                 // the pair's only segment: normalise and write the head's output
-                                int row = q < p.G ? item : Bc + item;
-                                int hq = g * p.G + (q < p.G ? q : q - p.G);
+                                int row = (q / p.G) * Bc + item;
+                                int hq = g * p.G + q % p.G;
                                 size_t ob = (size_t)row * q_dim + (size_t)hq * DH;
                                 float inv = 1.f / l_run[h];
     #pragma unroll
@@ -806,8 +833,8 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
                         int q = c + j;
                         if (q < nq_act) {
                             if (nseg == 1) {
-                                int row = q < p.G ? item : Bc + item;
-                                int hq = g * p.G + (q < p.G ? q : q - p.G);
+                                int row = (q / p.G) * Bc + item;
+                                int hq = g * p.G + q % p.G;
                                 size_t ob = (size_t)row * q_dim + (size_t)hq * DH;
                                 float inv = 1.f / l_run[j];
 #pragma unroll
@@ -894,8 +921,8 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
                 for (int a = 0; a < 2; a++) {
                     if (!act[a]) continue;
                     if (final) {
-                        int row = qq[a] < p.G ? item : Bc + item;
-                        int h = g * p.G + (qq[a] < p.G ? qq[a] : qq[a] - p.G);
+                        int row = (qq[a] / p.G) * Bc + item;
+                        int h = g * p.G + qq[a] % p.G;
                         size_t o_idx = (size_t)row * q_dim + (size_t)h * DH + ee[a];
                         float x = X[a] / L[a];
                         __nv_bfloat16 hi = __float2bfloat16_rn(x);

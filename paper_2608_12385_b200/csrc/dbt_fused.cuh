@@ -1,5 +1,11 @@
 // Elementwise kernels that sit between the tensor-core GEMMs of the bf16 path.  Each one also
 // sums the split-K partials of the GEMM before it, in split order (deterministic).
+//
+// Rows are path-major: Bc primary rows, then Bc rows per decode branch (one branch in the main text, K-1 with
+// more decode branches, Appendix C.1).  A kernel that couples a branch row to its primary twin runs one block
+// per (primary row, ..., branch): blockIdx.z is the branch, its row is (blockIdx.z + 1) * Bc + b.  Every block
+// recomputes what it needs of the primary row from the partials (a pure function of them); only the blocks of
+// the first branch store the primary row's results.
 #pragma once
 
 #include "dbt_common.cuh"
@@ -111,19 +117,23 @@ __global__ void __launch_bounds__(256) resid_wide_kernel(float *S, const float *
     DBT_TL_WAITED;
     __shared__ float scratch[64];
     int b = blockIdx.x, i = blockIdx.y * blockDim.x + threadIdx.x;
+    const bool first = blockIdx.z == 0;  // the first branch's blocks also own the primary row
+    const int r2 = ((int)blockIdx.z + 1) * Bc + b;
     float q1 = 0.f, q2 = 0.f;
     if (i < d) {
         // every load of this thread goes out before the first use: S of both rows, the gain, the
         // coupling, and all splits of both rows' partials (up to 16 splits in one round)
-        size_t o1 = (size_t)b * d + i, o2 = (size_t)(Bc + b) * d + i;
-        float s1 = __ldcg(S + o1), s2 = grouped ? __ldcg(S + o2) : 0.f;
+        size_t o1 = (size_t)b * d + i, o2 = (size_t)r2 * d + i;
+        float s1 = first ? __ldcg(S + o1) : 0.f, s2 = grouped ? __ldcg(S + o2) : 0.f;
         float gn = g_next ? g_next[i] : 1.f, cc = mode >= 2 ? coup_c[i] : 0.f;
         const size_t offs[2] = {o1, grouped && mode != 3 ? o2 : o1};
         float mm[2];
         sum_splits_k<2, 16>(P, split_stride, nsplit, offs, mm);
         s1 += mm[0];
-        S[o1] = s1;
-        store_split(Xb, o1, lo_off, gn * s1);
+        if (first) {
+            S[o1] = s1;
+            store_split(Xb, o1, lo_off, gn * s1);
+        }
         q1 = s1 * s1;
         if (grouped) {
             float m2 = mm[1];
@@ -150,8 +160,8 @@ __global__ void __launch_bounds__(256) resid_wide_kernel(float *S, const float *
             a1 += scratch[w2];
             a2 += scratch[32 + w2];
         }
-        ss_out[(size_t)blockIdx.y * ss_ld + b] = a1;
-        if (grouped) ss_out[(size_t)blockIdx.y * ss_ld + Bc + b] = a2;
+        if (first) ss_out[(size_t)blockIdx.y * ss_ld + b] = a1;
+        if (grouped) ss_out[(size_t)blockIdx.y * ss_ld + r2] = a2;
     }
     DBT_TL_END("resid_wide");
 }
@@ -161,8 +171,8 @@ __global__ void __launch_bounds__(256) resid_wide_kernel(float *S, const float *
 //   mode 1: S += sum_s P[s]                               (S-bar_i = S_i + Attn_i W_O)
 //   mode 2: M = sum_s P[s]; M_2 += c * M_1; S += M        (Eq. mlp: M_2 = H~_2 W_D + c*M_1)
 //   mode 3: M_1 = sum_s P[s]; M_2 = g * M_1; S += M        (Eq. matched_attention; coup_c carries g_A)
-// then Xb = bf16(g * S / rms(S)) (apply_norm) or bf16(S).  Block j handles primary source row
-// j*src_mul + src_add and, in grouped mode, its branch twin; outputs go to rows j and n_out + j.
+// then Xb = bf16(g * S / rms(S)) (apply_norm) or bf16(S).  Block (j, 0, z) handles primary source row
+// j*src_mul + src_add and, in grouped mode, its twin of branch z; outputs go to rows j and (z+1)*n_out + j.
 __global__ void __launch_bounds__(1024) resid_norm_kernel(float *S, const float *P, int nsplit,
                                                          size_t split_stride, int mode,
                                                          const float *__restrict__ coup_c, int Bc, int grouped,
@@ -174,10 +184,12 @@ __global__ void __launch_bounds__(1024) resid_norm_kernel(float *S, const float 
     DBT_TL_WAITED;
     __shared__ float scratch[32];
     int j = blockIdx.x, n_out = gridDim.x;
-    int r1 = j * src_mul + src_add, r2 = Bc + r1;
+    const bool first = blockIdx.z == 0;
+    const int zb = (int)blockIdx.z + 1;
+    int r1 = j * src_mul + src_add, r2 = zb * Bc + r1;
     float ss1 = 0.f, ss2 = 0.f;
     for (int i = threadIdx.x; i < d; i += blockDim.x) {
-        float v1 = S[(size_t)r1 * d + i], m1 = 0.f;
+        float v1 = first ? S[(size_t)r1 * d + i] : 0.f, m1 = 0.f;
         float v2 = grouped ? S[(size_t)r2 * d + i] : 0.f;
         float sm[2] = {0.f, 0.f};
         if (mode != 0) {
@@ -185,7 +197,7 @@ __global__ void __launch_bounds__(1024) resid_norm_kernel(float *S, const float 
             sum_splits_k<2, 8>(P, split_stride, nsplit, offs, sm);  // (1024 threads per block: 64 registers each)
             m1 = sm[0];
             v1 += m1;
-            S[(size_t)r1 * d + i] = v1;
+            if (first) S[(size_t)r1 * d + i] = v1;
         }
         ss1 += v1 * v1;
         if (grouped) {
@@ -211,13 +223,15 @@ __global__ void __launch_bounds__(1024) resid_norm_kernel(float *S, const float 
     // each thread re-reads only the elements of S it wrote itself (same index stride)
     for (int i = threadIdx.x; i < d; i += blockDim.x) {
         float gi = apply_norm ? g[i] : 1.f;
-        float x1 = gi * S[(size_t)r1 * d + i] * inv1;
-        store_split(Xb, (size_t)j * d + i, lo_off, x1);
-        if (Xf) Xf[(size_t)j * d + i] = x1;
+        if (first) {
+            float x1 = gi * S[(size_t)r1 * d + i] * inv1;
+            store_split(Xb, (size_t)j * d + i, lo_off, x1);
+            if (Xf) Xf[(size_t)j * d + i] = x1;
+        }
         if (grouped) {
             float x2 = gi * S[(size_t)r2 * d + i] * inv2;
-            store_split(Xb, (size_t)(n_out + j) * d + i, lo_off, x2);
-            if (Xf) Xf[(size_t)(n_out + j) * d + i] = x2;
+            store_split(Xb, (size_t)(zb * n_out + j) * d + i, lo_off, x2);
+            if (Xf) Xf[(size_t)(zb * n_out + j) * d + i] = x2;
         }
     }
     DBT_TL_END("resid_norm");
@@ -238,14 +252,16 @@ __global__ void __launch_bounds__(64) qkv_epilogue_kernel(
     pdl_enter();
     DBT_TL_WAITED;
     int item = blockIdx.x, hh = blockIdx.y, i = threadIdx.x, Bc = rm.Bc();
+    const bool first = blockIdx.z == 0;
+    const int twin = ((int)blockIdx.z + 1) * Bc + item;
     int half = dh / 2;
     if (i >= half) return;
     int seq = rm.seq(item), pos = ld_mut(seq_len + seq) + rm.off(item);
     int q_dim = n_q * dh, kv_dim = n_kv * dh, ldp = q_dim + 2 * kv_dim;
     float2 t = rope_tab[(size_t)pos * half + i];
-    size_t p1 = (size_t)item * ldp, p2 = (size_t)(Bc + item) * ldp;
+    size_t p1 = (size_t)item * ldp, p2 = (size_t)twin * ldp;
     float rs1, rs2;  // 1/rms when the GEMM input was g*S
-    row_scale2(ss, ss_tiles, ss_ld, item, grouped ? Bc + item : item, d_norm, eps, rs1, rs2);
+    row_scale2(ss, ss_tiles, ss_ld, item, grouped ? twin : item, d_norm, eps, rs1, rs2);
     if (hh < n_q) {
         int o0 = hh * dh + i, o1 = o0 + half;
         const size_t offs[4] = {p1 + o0, p1 + o1, grouped ? p2 + o0 : p1 + o0, grouped ? p2 + o1 : p1 + o1};
@@ -254,17 +270,20 @@ __global__ void __launch_bounds__(64) qkv_epilogue_kernel(
         float x0 = rs1 * sm[0], x1 = rs1 * sm[1];
         float r0 = x0 * t.x - x1 * t.y, r1 = x1 * t.x + x0 * t.y;
         float *q1 = Q + (size_t)item * q_dim;
-        q1[o0] = r0;
-        q1[o1] = r1;
+        if (first) {
+            q1[o0] = r0;
+            q1[o1] = r1;
+        }
         if (grouped) {
             float y0 = rs2 * sm[2], y1 = rs2 * sm[3];
-            float *q2 = Q + (size_t)(Bc + item) * q_dim;
+            float *q2 = Q + (size_t)twin * q_dim;
             q2[o0] = (y0 * t.x - y1 * t.y) + coup_a[o0] * r0;
             q2[o1] = (y1 * t.x + y0 * t.y) + coup_a[o1] * r1;
         }
         DBT_TL_END("qkv_epilogue");
         return;
     }
+    if (!first) return;  // K_1, V_1 exist once: the branches have none
     int gk = hh - n_q;
     int page = page_table[(size_t)seq * pt_stride + pos / page_size];
     if (page < 0 || page >= num_pages) {
@@ -297,7 +316,8 @@ __global__ void __launch_bounds__(256) swiglu_couple_kernel(const float *P, int 
     __shared__ float sh[34];
     int b = blockIdx.x, f = blockIdx.y * blockDim.x + threadIdx.x;
     const bool act = f < F;
-    const int rb = grouped ? Bc + b : b, lane = threadIdx.x & 31;
+    const bool first = blockIdx.z == 0;
+    const int rb = grouped ? ((int)blockIdx.z + 1) * Bc + b : b, lane = threadIdx.x & 31;
     // The norm shares of the block's two rows are fetched once, by the first warp (lanes 0..15 the
     // primary row, 16..31 its twin), requested before the partials so that they travel together,
     // and handed to the block through shared memory: a few hundred blocks would otherwise all
@@ -306,7 +326,7 @@ __global__ void __launch_bounds__(256) swiglu_couple_kernel(const float *P, int 
     if (ss && threadIdx.x < 32)
         for (int t = lane & 15; t < ss_tiles; t += 16) myss += __ldcg(ss + (size_t)t * ss_ld + (lane < 16 ? b : rb));
     size_t p1 = (size_t)b * 2 * F + (act ? f : 0);
-    size_t p2 = grouped ? (size_t)(Bc + b) * 2 * F + (act ? f : 0) : p1;
+    size_t p2 = grouped ? (size_t)rb * 2 * F + (act ? f : 0) : p1;
     const size_t offs[4] = {p1, p1 + F, p2, p2 + F};
     float sm[4] = {0.f, 0.f, 0.f, 0.f};
     if (act) sum_splits_k<4, 4>(P, split_stride, nsplit, offs, sm);
@@ -323,11 +343,11 @@ __global__ void __launch_bounds__(256) swiglu_couple_kernel(const float *P, int 
     if (act) {
         float rs1 = sh[32], rs2 = sh[33];
         float h1 = silu(rs1 * sm[0]) * (rs1 * sm[1]);
-        store_split(Hb, (size_t)b * F + f, lo_off, h1);
+        if (first) store_split(Hb, (size_t)b * F + f, lo_off, h1);
         if (grouped) {
             float h2 = silu(rs2 * sm[2]) * (rs2 * sm[3]);
             if (coup_b) h2 += coup_b[f] * h1;
-            store_split(Hb, (size_t)(Bc + b) * F + f, lo_off, h2);
+            store_split(Hb, (size_t)rb * F + f, lo_off, h2);
         }
     }
     DBT_TL_END("swiglu");
@@ -346,13 +366,13 @@ __global__ void __launch_bounds__(256) embed_fused_kernel(const int32_t *tokens,
     pdl_enter();
     __shared__ float scratch[32];
     int r = blockIdx.x;
-    int path = r >= rm.Bc();
+    int path = r / rm.Bc();  // 0 primary; j >= 1: decode branch j with its own table E2[j-1] (Appendix C.1)
     int tok = ld_mut(tokens + (size_t)rm.seq(r) * n + p0 + rm.off(r));
     if (tok < 0 || tok >= V) {
         if (threadIdx.x == 0) report(status, kStatusBadToken, tok);
         tok = min(max(tok, 0), V - 1);
     }
-    const WT *e = (path ? E2 : E1) + (size_t)tok * d;
+    const WT *e = (path ? E2 + (size_t)(path - 1) * V * d : E1) + (size_t)tok * d;
     float ss = 0.f;
     for (int i = threadIdx.x; i < d; i += blockDim.x) {
         float x = load1(e + i);
@@ -481,7 +501,8 @@ __global__ void __launch_bounds__(256) moe_combine_sorted_kernel(const float *Ys
     // the row's selections (weights, sorted positions) once, then all expert rows of a column in
     // flight together; terms are added in slot order
     constexpr int KM = 16;
-    const int r2 = Bc + b;
+    const bool first = blockIdx.z == 0;
+    const int r2 = ((int)blockIdx.z + 1) * Bc + b;
     for (int i = blockIdx.y * blockDim.x + threadIdx.x; i < d; i += gridDim.y * blockDim.x) {
         float m1 = 0.f, m2 = 0.f;
         for (int j0 = 0; j0 < kmax; j0 += KM) {
@@ -509,10 +530,12 @@ __global__ void __launch_bounds__(256) moe_combine_sorted_kernel(const float *Ys
             m2 += gate_g ? gate_g[i] * sm[0] : sm[1];
         }
         const float gn = Xn ? g_next[i] : 0.f;
-        const float v1 = S[(size_t)b * d + i] + m1;
-        S[(size_t)b * d + i] = v1;
-        if (Xn) store_split(Xn, (size_t)b * d + i, lo_off, gn * v1);
-        q1 += v1 * v1;
+        if (first) {
+            const float v1 = S[(size_t)b * d + i] + m1;
+            S[(size_t)b * d + i] = v1;
+            if (Xn) store_split(Xn, (size_t)b * d + i, lo_off, gn * v1);
+            q1 += v1 * v1;
+        }
         if (grouped) {
             if (!gate_g) m2 += coup_c[i] * m1;
             const float v2 = S[(size_t)r2 * d + i] + m2;
@@ -536,7 +559,7 @@ __global__ void __launch_bounds__(256) moe_combine_sorted_kernel(const float *Ys
                 a1 += scratch[w2];
                 a2 += scratch[32 + w2];
             }
-            ss_out[(size_t)blockIdx.y * ss_ld + b] = a1;
+            if (first) ss_out[(size_t)blockIdx.y * ss_ld + b] = a1;
             if (grouped) ss_out[(size_t)blockIdx.y * ss_ld + r2] = a2;
         }
     }

@@ -19,13 +19,13 @@ __global__ void embed_norm_kernel(const int32_t *tokens, int n, int p0, RowMap r
     pdl_enter();
     __shared__ float scratch[32];
     int r = blockIdx.x;
-    int path = r >= rm.Bc();
+    int path = r / rm.Bc();  // 0 primary; j >= 1: decode branch j with its own table E2[j-1] (Appendix C.1)
     int tok = ld_mut(tokens + (size_t)rm.seq(r) * n + p0 + rm.off(r));
     if (tok < 0 || tok >= V) {
         if (threadIdx.x == 0) report(status, kStatusBadToken, tok);
         tok = min(max(tok, 0), V - 1);
     }
-    const WT *e = (path ? E2 : E1) + (size_t)tok * d;
+    const WT *e = (path ? E2 + (size_t)(path - 1) * V * d : E1) + (size_t)tok * d;
     float ss = 0.f;
     for (int i = threadIdx.x; i < d; i += blockDim.x) {
         float x = load1(e + i);
@@ -72,7 +72,7 @@ struct LinArgs {
     int K;
     int epi;
     int Bc;       // primary rows in this launch
-    int grouped;  // branch rows Bc..2Bc-1 present
+    int grouped;  // paths present: 0 or 1 = the primary alone; P >= 2 = branch rows j*Bc .. (j+1)*Bc-1, j = 1..P-1
     const float *coup;  // b (EPI_SWIGLU), c (EPI_DOWN) or g_A (EPI_RESID_GATED); nullptr = no coupling
     float *S;     // residual rows [.][n_out[0]] for EPI_RESID / EPI_DOWN
 };
@@ -143,25 +143,27 @@ __global__ void __launch_bounds__(kLinWarps * 32) linear_kernel(LinArgs a) {
                 } else if (a.epi == EPI_RESID_GATED) {
                     // S-bar_1 = S_1 + A_1 ; S-bar_2 = S_2 + g_A * A_1 (Eq. matched_attention): primary rows only
                     a.S[o] += acc[r];
-                    a.S[(size_t)(a.Bc + r0 + r) * n_out + f] += a.coup[f] * acc[r];
+                    for (int j = 1; j < a.grouped; j++) a.S[(size_t)(j * a.Bc + r0 + r) * n_out + f] += a.coup[f] * acc[r];
                 } else
                     Y[o] = acc[r];
             }
         }
     }
-    if (a.epi == EPI_SWIGLU && a.grouped && a.coup != nullptr) {
-        // H~_2 = H_2 + b * H_1 (Eq. mlp), feature f of every sequence
+    if (a.epi == EPI_SWIGLU && a.grouped > 1 && a.coup != nullptr) {
+        // H~_j = H_j + b * H_1 (Eq. mlp), feature f of every sequence and branch
         __syncwarp();
         float bf = a.coup[f];
-        for (int b = lane; b < a.Bc; b += 32) Y[(size_t)(a.Bc + b) * n_out + f] += bf * Y[(size_t)b * n_out + f];
+        for (int b = lane; b < a.Bc; b += 32)
+            for (int j = 1; j < a.grouped; j++) Y[(size_t)(j * a.Bc + b) * n_out + f] += bf * Y[(size_t)b * n_out + f];
     } else if (a.epi == EPI_DOWN) {
-        // M_2 += c * M_1 ; S_i^{l+1} = S-bar_i + M_i (Eq. mlp)
+        // M_j += c * M_1 ; S_i^{l+1} = S-bar_i + M_i (Eq. mlp)
         __syncwarp();
-        float cf = (a.grouped && a.coup != nullptr) ? a.coup[f] : 0.f;
+        float cf = (a.grouped > 1 && a.coup != nullptr) ? a.coup[f] : 0.f;
         for (int b = lane; b < a.Bc; b += 32) {
             float m1 = Y[(size_t)b * n_out + f];
             a.S[(size_t)b * n_out + f] += m1;
-            if (a.grouped) a.S[(size_t)(a.Bc + b) * n_out + f] += Y[(size_t)(a.Bc + b) * n_out + f] + cf * m1;
+            for (int j = 1; j < a.grouped; j++)
+                a.S[(size_t)(j * a.Bc + b) * n_out + f] += Y[(size_t)(j * a.Bc + b) * n_out + f] + cf * m1;
         }
     }
 }
@@ -183,7 +185,6 @@ __global__ void rope_couple_append_kernel(float *Q, const float *Kn,
     int half = dh / 2, q_dim = n_q * dh, kv_dim = n_kv * dh;
     const float2 *cs = rope_tab + (size_t)pos * half;
     float *q1 = Q + (size_t)item * q_dim;
-    float *q2 = Q + (size_t)(Bc + item) * q_dim;
     for (int idx = threadIdx.x; idx < n_q * half; idx += blockDim.x) {
         int h = idx / half, i = idx % half;
         float2 t = cs[i];
@@ -192,7 +193,8 @@ __global__ void rope_couple_append_kernel(float *Q, const float *Kn,
         float r0 = x0 * t.x - x1 * t.y, r1 = x1 * t.x + x0 * t.y;
         q1[o0] = r0;
         q1[o1] = r1;
-        if (grouped) {
+        for (int j = 1; j < grouped; j++) {  // `grouped` counts the paths present: every branch row, the same a
+            float *q2 = Q + (size_t)(j * Bc + item) * q_dim;
             float y0 = q2[o0], y1 = q2[o1];
             q2[o0] = (y0 * t.x - y1 * t.y) + coup_a[o0] * r0;
             q2[o1] = (y1 * t.x + y0 * t.y) + coup_a[o1] * r1;
@@ -238,14 +240,14 @@ __global__ void __launch_bounds__(128) attn_partial_kernel(
     int item = blockIdx.x, g = blockIdx.y, sp = blockIdx.z;
     int Bc = rm.Bc(), seq = rm.seq(item);
     int nkeys = ld_mut(seq_len + seq) + rm.off(item) + 1;
-    int nq_act = grouped ? 2 * G : G, q_dim = n_kv * G * DH;
+    int nq_act = (grouped > 1 ? grouped : 1) * G, q_dim = n_kv * G * DH;  // `grouped`: paths present
     float scale = 1.f / sqrtf((float)DH);
     for (int idx = tid; idx < NQ * DH; idx += TPB) {
         int q = idx / DH, e = idx % DH;
         float v = 0.f;
         if (q < nq_act) {
-            int row = q < G ? item : Bc + item;
-            int h = g * G + (q < G ? q : q - G);
+            int row = (q / G) * Bc + item;
+            int h = g * G + q % G;
             v = Q[(size_t)row * q_dim + h * DH + e] * scale;
         }
         qs[q][e] = v;
@@ -356,7 +358,7 @@ __global__ void attn_merge_kernel(const float *part, int nsplit, int NQ, int DH,
                                   size_t lo_off) {
     pdl_enter();
     int item = blockIdx.x, g = blockIdx.y, e = threadIdx.x;
-    int nq_act = grouped ? 2 * G : G, q_dim = n_kv * G * DH;
+    int nq_act = (grouped > 1 ? grouped : 1) * G, q_dim = n_kv * G * DH;  // `grouped`: paths present
     const float *base = part + ((size_t)item * n_kv + g) * nsplit * NQ * (DH + 2);
     for (int q = 0; q < nq_act; q++) {
         float M = -INFINITY;
@@ -369,8 +371,8 @@ __global__ void attn_merge_kernel(const float *part, int nsplit, int NQ, int DH,
             L += p[DH + 1] * w;
             o += p[e] * w;
         }
-        int row = q < G ? item : Bc + item;
-        int h = g * G + (q < G ? q : q - G);
+        int row = (q / G) * Bc + item;
+        int h = g * G + q % G;
         if (O) O[(size_t)row * q_dim + h * DH + e] = o / L;
         if (Ob) {
             float x = o / L;
@@ -382,10 +384,11 @@ __global__ void attn_merge_kernel(const float *part, int nsplit, int NQ, int DH,
 }
 
 // ---------------------------------------------------------------------------------------
-// Readout (Eq. alpha, Eq. mixloss): p = softmax(z_1), q = softmax(z_2),
-// alpha = clip_[0.5,1](sum p^2), next = argmax(alpha p + (1-alpha) q), lowest index on ties.
-// Primary-only: next = argmax z_1.  One block per sequence; the block also advances its sequence's
-// length when asked to (the last kernel of a decode step).
+// Readout (Eq. alpha, Eq. mixloss): p = softmax(z_1), q_j = softmax(z_j) for the decode branches
+// j = 2..P (one in the main text; Appendix C.1 averages several: qbar = mean_j q_j),
+// alpha = clip_[0.5,1](sum p^2), next = argmax(alpha p + (1-alpha) qbar), lowest index on ties.
+// Primary-only (P = 1): next = argmax z_1.  Z rows are path-major: row j*B + b.  One block per
+// sequence; the block also advances its sequence's length when asked to (the last kernel of a step).
 struct ArgBest {
     float v;
     int i;
@@ -394,38 +397,58 @@ __device__ __forceinline__ ArgBest better(ArgBest a, ArgBest b) {
     if (b.v > a.v || (b.v == a.v && b.i < a.i)) return b;
     return a;
 }
+constexpr int kMaxBranches = 7;  // decode branches per model (P <= 8 paths)
 
-__global__ void __launch_bounds__(1024) readout_kernel(const float *Z, int B, int V, int grouped,
+__global__ void __launch_bounds__(1024) readout_kernel(const float *Z, int B, int V, int P,
                                                        int32_t *next, float *alpha_out, int32_t *seq_len, int advance) {
     pdl_enter();
     __shared__ float scratch[32];
     __shared__ float bv[32];
     __shared__ int bi[32];
     int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nw = blockDim.x >> 5;
-    const float *z1 = Z + (size_t)b * V, *z2 = Z + (size_t)(B + b) * V;
-    float m1 = -INFINITY, m2 = -INFINITY, d1 = 1.f, d2 = 1.f, alpha = 1.f;
+    const bool grouped = P > 1;
+    const int nb = grouped ? P - 1 : 0;
+    const float *z1 = Z + (size_t)b * V;
+    float m1 = -INFINITY, d1 = 1.f, alpha = 1.f;
+    float mb[kMaxBranches], db[kMaxBranches];
     if (grouped) {
-        for (int v = tid; v < V; v += blockDim.x) {
-            m1 = fmaxf(m1, z1[v]);
-            m2 = fmaxf(m2, z2[v]);
-        }
+        for (int v = tid; v < V; v += blockDim.x) m1 = fmaxf(m1, z1[v]);
         m1 = block_max(m1, scratch);
-        m2 = block_max(m2, scratch);
-        float s1 = 0.f, s2 = 0.f, c1 = 0.f;
+        float s1 = 0.f, c1 = 0.f;
         for (int v = tid; v < V; v += blockDim.x) {
             float e1 = expf(z1[v] - m1);
             s1 += e1;
             c1 += e1 * e1;
-            s2 += expf(z2[v] - m2);
         }
         d1 = block_sum(s1, scratch);
-        d2 = block_sum(s2, scratch);
         c1 = block_sum(c1, scratch);
         alpha = fminf(1.f, fmaxf(0.5f, c1 / (d1 * d1)));
+#pragma unroll
+        for (int jb = 0; jb < kMaxBranches; jb++) {
+            mb[jb] = 0.f;
+            db[jb] = 1.f;
+            if (jb < nb) {
+                const float *zj = Z + (size_t)((jb + 1) * B + b) * V;
+                float mj = -INFINITY, sj = 0.f;
+                for (int v = tid; v < V; v += blockDim.x) mj = fmaxf(mj, zj[v]);
+                mj = block_max(mj, scratch);
+                for (int v = tid; v < V; v += blockDim.x) sj += expf(zj[v] - mj);
+                mb[jb] = mj;
+                db[jb] = block_sum(sj, scratch);
+            }
+        }
     }
+    const float inv_nb = grouped ? 1.f / (float)nb : 0.f;
     ArgBest best = {-INFINITY, 0x7fffffff};
     for (int v = tid; v < V; v += blockDim.x) {
-        float val = grouped ? alpha * (expf(z1[v] - m1) / d1) + (1.f - alpha) * (expf(z2[v] - m2) / d2) : z1[v];
+        float val = z1[v];
+        if (grouped) {
+            float qs = 0.f;
+#pragma unroll
+            for (int jb = 0; jb < kMaxBranches; jb++)
+                if (jb < nb) qs += expf(Z[(size_t)((jb + 1) * B + b) * V + v] - mb[jb]) / db[jb];
+            val = alpha * (expf(z1[v] - m1) / d1) + (1.f - alpha) * (qs * inv_nb);
+        }
         best = better(best, ArgBest{val, v});
     }
 #pragma unroll
@@ -457,16 +480,20 @@ __global__ void __launch_bounds__(1024) readout_kernel(const float *Z, int B, in
 // ---- the readout on many CTAs -----------------------------------------------------------------
 // readout_kernel walks a row three times with one CTA.  Here a row is cut into NC chunks of at most
 // kRoChunk logits, a CTA per (row, chunk), each logit staged in registers:
-//   readout_stats_kernel: per chunk (m1, sum e^(z1-m1), sum e^(2(z1-m1)), m2, sum e^(z2-m2)) with the
-//     chunk's own maxima;
-//   readout_pick_kernel: every CTA folds the row's NC records in chunk order into p, q's normalisers
-//     and alpha (Eq. alpha), evaluates alpha p + (1 - alpha) q (Eq. mixloss) over its chunk, and leaves
-//     its best (value, index); the last CTA of the row to arrive picks among the NC candidates
-//     (lowest index on ties), writes the token and alpha and advances the sequence length.
+//   readout_stats_kernel: per chunk a record (m1, sum e^(z1-m1), sum e^(2(z1-m1)), and per decode branch
+//     (m_j, sum e^(z_j-m_j))) with the chunk's own maxima;
+//   readout_pick_kernel: every CTA folds the row's NC records in chunk order into p's and the q_j's
+//     normalisers and alpha (Eq. alpha), evaluates alpha p + (1 - alpha) mean_j q_j (Eq. mixloss;
+//     Appendix C.1 for several branches) over its chunk, and leaves its best (value, index); the last
+//     CTA of the row to arrive picks among the NC candidates (lowest index on ties), writes the token and
+//     alpha and advances the sequence length.
 // Primary-only steps skip the first kernel: the pick is the argmax of z1.
+// Record layout (kRoRec floats): [0] m1, [1] s1, [2] sum of squares, [3] best value, [4] best index,
+// [5 + 2j] m of branch j, [6 + 2j] s of branch j.
 constexpr int kRoChunk = 2048, kRoThreads = 256, kRoPer = kRoChunk / kRoThreads, kRoMaxChunks = 128;
+constexpr int kRoRec = 5 + 2 * kMaxBranches + 1;
 
-__global__ void __launch_bounds__(kRoThreads) readout_stats_kernel(const float *Z, int B, int V, int chunk, float *stats) {
+__global__ void __launch_bounds__(kRoThreads) readout_stats_kernel(const float *Z, int B, int V, int P, int chunk, float *stats) {
     pdl_enter();
     __shared__ float scratch[32];
     const int b = blockIdx.x, ck = blockIdx.y, tid = threadIdx.x;
@@ -498,22 +525,42 @@ __global__ void __launch_bounds__(kRoThreads) readout_stats_kernel(const float *
     s1 = block_sum(s1, scratch);
     q1 = block_sum(q1, scratch);
     s2 = block_sum(s2, scratch);
+    float *o = stats + ((size_t)b * gridDim.y + ck) * kRoRec;
     if (tid == 0) {
-        float *o = stats + ((size_t)b * gridDim.y + ck) * 8;
-        o[0] = m1; o[1] = s1; o[2] = q1; o[3] = m2; o[4] = s2;
+        o[0] = m1; o[1] = s1; o[2] = q1; o[5] = m2; o[6] = s2;
+    }
+    for (int jb = 1; jb < P - 1; jb++) {  // further decode branches, one after the other
+        const float *zj = Z + (size_t)((jb + 1) * B + b) * V;
+        float mj = -INFINITY, sj = 0.f;
+#pragma unroll
+        for (int j = 0; j < kRoPer; j++) {
+            const int v = v0 + j * kRoThreads + tid;
+            c[j] = v < v1 ? __ldcg(zj + v) : -INFINITY;
+            mj = fmaxf(mj, c[j]);
+        }
+        mj = block_max(mj, scratch);
+#pragma unroll
+        for (int j = 0; j < kRoPer; j++) sj += c[j] == -INFINITY ? 0.f : expf(c[j] - mj);
+        sj = block_sum(sj, scratch);
+        if (tid == 0) {
+            o[5 + 2 * jb] = mj;
+            o[6 + 2 * jb] = sj;
+        }
     }
 }
 
-__global__ void __launch_bounds__(kRoThreads) readout_pick_kernel(const float *Z, int B, int V, int chunk, int grouped,
+__global__ void __launch_bounds__(kRoThreads) readout_pick_kernel(const float *Z, int B, int V, int chunk, int P,
                                                                   float *stats, int32_t *tickets, int32_t *next,
                                                                   float *alpha_out, int32_t *seq_len, int advance) {
     pdl_enter();
     __shared__ float bv[32];
     __shared__ int bi[32];
-    __shared__ float glob[6];
+    __shared__ float glob[4 + 2 * kMaxBranches];  // m1, d1, alpha, -, then (m_j, d_j) per branch
     __shared__ int last_s;
     const int b = blockIdx.x, ck = blockIdx.y, nc = gridDim.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int v0 = ck * chunk, v1 = min(V, v0 + chunk);
+    const bool grouped = P > 1;
+    const int nb = grouped ? P - 1 : 0;
     const float *z1 = Z + (size_t)b * V, *z2 = Z + (size_t)(B + b) * V;
     float a[kRoPer], c[kRoPer];
 #pragma unroll
@@ -524,34 +571,57 @@ __global__ void __launch_bounds__(kRoThreads) readout_pick_kernel(const float *Z
     }
     if (grouped && warp == 0) {
         // fold the row's records: maxima first, then the sums rescaled to them, in chunk order (lane 0)
-        const float *rec = stats + (size_t)b * nc * 8;
-        float m1 = -INFINITY, m2 = -INFINITY;
-        for (int k = lane; k < nc; k += 32) {
-            m1 = fmaxf(m1, __ldcg(rec + (size_t)k * 8));
-            m2 = fmaxf(m2, __ldcg(rec + (size_t)k * 8 + 3));
-        }
+        const float *rec = stats + (size_t)b * nc * kRoRec;
+        float m1 = -INFINITY;
+        for (int k = lane; k < nc; k += 32) m1 = fmaxf(m1, __ldcg(rec + (size_t)k * kRoRec));
         m1 = warp_max(m1);
-        m2 = warp_max(m2);
         if (lane == 0) {
-            float d1 = 0.f, c1 = 0.f, d2 = 0.f;
+            float d1 = 0.f, c1 = 0.f;
             for (int k = 0; k < nc; k++) {
-                const float f1 = expf(__ldcg(rec + (size_t)k * 8) - m1), f2 = expf(__ldcg(rec + (size_t)k * 8 + 3) - m2);
-                d1 += __ldcg(rec + (size_t)k * 8 + 1) * f1;
-                c1 += __ldcg(rec + (size_t)k * 8 + 2) * f1 * f1;
-                d2 += __ldcg(rec + (size_t)k * 8 + 4) * f2;
+                const float f1 = expf(__ldcg(rec + (size_t)k * kRoRec) - m1);
+                d1 += __ldcg(rec + (size_t)k * kRoRec + 1) * f1;
+                c1 += __ldcg(rec + (size_t)k * kRoRec + 2) * f1 * f1;
             }
-            glob[0] = m1; glob[1] = d1; glob[2] = m2; glob[3] = d2;
-            glob[4] = fminf(1.f, fmaxf(0.5f, c1 / (d1 * d1)));
+            glob[0] = m1; glob[1] = d1;
+            glob[2] = fminf(1.f, fmaxf(0.5f, c1 / (d1 * d1)));
+        }
+        for (int jb = 0; jb < nb; jb++) {
+            float mj = -INFINITY;
+            for (int k = lane; k < nc; k += 32) mj = fmaxf(mj, __ldcg(rec + (size_t)k * kRoRec + 5 + 2 * jb));
+            mj = warp_max(mj);
+            if (lane == 0) {
+                float dj = 0.f;
+                for (int k = 0; k < nc; k++)
+                    dj += __ldcg(rec + (size_t)k * kRoRec + 6 + 2 * jb) * expf(__ldcg(rec + (size_t)k * kRoRec + 5 + 2 * jb) - mj);
+                glob[4 + 2 * jb] = mj;
+                glob[5 + 2 * jb] = dj;
+            }
         }
     }
     __syncthreads();
-    const float m1 = glob[0], d1 = glob[1], m2 = glob[2], d2 = glob[3], alpha = glob[4];
+    const float m1 = glob[0], d1 = glob[1], alpha = glob[2];
+    const float inv_nb = grouped ? 1.f / (float)nb : 0.f;
+    float qs[kRoPer];
+    if (grouped) {
+        const float m2 = glob[4], d2 = glob[5];
+#pragma unroll
+        for (int j = 0; j < kRoPer; j++) qs[j] = c[j] == -INFINITY ? 0.f : expf(c[j] - m2) / d2;
+        for (int jb = 1; jb < nb; jb++) {
+            const float *zj = Z + (size_t)((jb + 1) * B + b) * V;
+            const float mj = glob[4 + 2 * jb], dj = glob[5 + 2 * jb];
+#pragma unroll
+            for (int j = 0; j < kRoPer; j++) {
+                const int v = v0 + j * kRoThreads + tid;
+                if (v < v1) qs[j] += expf(__ldcg(zj + v) - mj) / dj;
+            }
+        }
+    }
     ArgBest best = {-INFINITY, 0x7fffffff};
 #pragma unroll
     for (int j = 0; j < kRoPer; j++) {
         const int v = v0 + j * kRoThreads + tid;
         if (v < v1) {
-            float val = grouped ? alpha * (expf(a[j] - m1) / d1) + (1.f - alpha) * (expf(c[j] - m2) / d2) : a[j];
+            float val = grouped ? alpha * (expf(a[j] - m1) / d1) + (1.f - alpha) * (qs[j] * inv_nb) : a[j];
             best = better(best, ArgBest{val, v});
         }
     }
@@ -573,9 +643,9 @@ __global__ void __launch_bounds__(kRoThreads) readout_pick_kernel(const float *Z
             t = better(t, other);
         }
         if (lane == 0) {
-            float *o2 = stats + ((size_t)b * nc + ck) * 8;
-            o2[5] = t.v;
-            o2[6] = __int_as_float(t.i);
+            float *o2 = stats + ((size_t)b * nc + ck) * kRoRec;
+            o2[3] = t.v;
+            o2[4] = __int_as_float(t.i);
             __threadfence();
             const int tk = atomicAdd(tickets + b, 1);
             last_s = tk == nc - 1;
@@ -585,9 +655,10 @@ __global__ void __launch_bounds__(kRoThreads) readout_pick_kernel(const float *Z
     __syncthreads();
     if (last_s && warp == 0) {
         __threadfence();
-        const float *rec = stats + (size_t)b * nc * 8;
+        const float *rec = stats + (size_t)b * nc * kRoRec;
         ArgBest t = {-INFINITY, 0x7fffffff};
-        for (int k = lane; k < nc; k += 32) t = better(t, ArgBest{__ldcg(rec + (size_t)k * 8 + 5), __float_as_int(__ldcg(rec + (size_t)k * 8 + 6))});
+        for (int k = lane; k < nc; k += 32)
+            t = better(t, ArgBest{__ldcg(rec + (size_t)k * kRoRec + 3), __float_as_int(__ldcg(rec + (size_t)k * kRoRec + 4))});
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
             ArgBest other = {__shfl_xor_sync(0xffffffffu, t.v, o), __shfl_xor_sync(0xffffffffu, t.i, o)};
@@ -655,8 +726,8 @@ __global__ void __launch_bounds__(32) route_kernel(const float *logits, int nspl
     extern __shared__ float smem[];
     float *own = smem, *sel = smem + E;  // own-row logits -> probabilities; selection-row logits
     int r = blockIdx.x, lane = threadIdx.x;
-    int path = r >= Bc;
-    int sel_row = (path && replay) ? r - Bc : r;
+    int path = r / Bc;  // 0 primary, j >= 1 decode branch j (each branch routes for itself, fan-out k_b)
+    int sel_row = (path && replay) ? r % Bc : r;
     int k = (path && !replay) ? k_b : k_p;
     float inv_own = 1.f, inv_sel = 1.f;
     if (ss) {
@@ -827,8 +898,8 @@ __global__ void moe_combine_kernel(const float *Yexp, const float *Msh,
         float sh1 = Msh ? Msh[(size_t)b * d + i] : 0.f;
         if (Msh) m1 += sh1;
         S[(size_t)b * d + i] += m1;
-        if (grouped) {
-            int r = Bc + b;
+        for (int jp = 1; jp < grouped; jp++) {  // `grouped` counts the paths present
+            int r = jp * Bc + b;
             float m2 = 0.f;
             for (int j = 0; j < kmax; j++)
                 if (idx[(size_t)r * kmax + j] >= 0)

@@ -141,7 +141,7 @@ def test_1b_at_the_benchmarks_launch_configuration_on_sampled_sequences():
 
 # ---- readout off the clip of alpha (Eq. alpha, Eq. mixloss) ---------------------------------------------------
 
-@pytest.mark.parametrize("cfg,matrix_std", [(small_bf16(), 0.05), (tiny_dense_fp32(), 0.02)])
+@pytest.mark.parametrize("cfg,matrix_std", [(small_bf16(), 0.05), (tiny_dense_fp32(), 0.02), (small_bf16(n_paths=3), 0.05)])
 def test_readout_with_alpha_between_the_clips_and_at_one(cfg, matrix_std):
     """Random-init models have sum p^2 ~ 1e-3, so alpha sits on its lower clip and the mixture is symmetric
     in p and q.  An output matrix drawn with standard deviation 2.0 makes p peaked: over these 6 sequences x 4
@@ -175,16 +175,17 @@ def test_readout_with_alpha_between_the_clips_and_at_one(cfg, matrix_std):
         a_dev = g["alpha"].cpu().numpy()
         np.testing.assert_allclose(a_dev, o["alpha"], rtol=1e-3, atol=errs[0])
         nxt = g["next"].cpu().numpy()
+        zb = z2 if z2.ndim == 3 else z2[None]  # [branches, B, V]
         for b in range(B):
-            tok_o, a_o, mix_o = oracle.readout(z1[b], z2[b])
+            tok_o, a_o, mix_o = oracle.readout_multi(z1[b], np.ascontiguousarray(zb[:, b]))
             assert a_dev[b] == pytest.approx(a_o, rel=2e-5), (t, b, a_dev[b], a_o)
             top = np.sort(mix_o)[-2:]
             if top[1] - top[0] > 1e-4 * top[1]:
                 assert nxt[b] == tok_o, (t, b, nxt[b], tok_o)
             # what a p <-> q swap would have produced
-            _, a_sw, _ = oracle.readout(z2[b], z1[b])
+            _, a_sw, _ = oracle.readout(zb[0, b], z1[b])
             swapped_would_differ += int(abs(a_sw - a_o) > 1e-3)
-        assert (o["z1"].argmax(-1) != o["z2"].argmax(-1)).all()
+        assert (o["z1"].argmax(-1) != o["z2"].argmax(-1)).all()  # (every branch, when there are several)
         alphas.append(o["alpha"])
     alphas = np.stack(alphas)
     assert ((alphas > 0.5) & (alphas < 1.0)).sum() >= 5 and (alphas == 1.0).sum() >= 1, alphas
@@ -203,7 +204,8 @@ def _run_steps(gm, tok_dev, n_prefill, grouped):
 
 
 @pytest.mark.parametrize("cfg", [tiny_dense_fp32().replace(n_layers=2), small_bf16(), small_moe(),
-                                 small_moe(compute_matched=1)])
+                                 small_moe(compute_matched=1), small_bf16(n_paths=3), small_moe(n_paths=4),
+                                 tiny_dense_fp32().replace(n_layers=2, n_paths=3)])
 def test_kv_cache_bit_identical_grouped_vs_primary_only(cfg):
     """The primary path never reads the branch: the cache written by grouped decode and by
     primary-only decode is the same bits, and so are the primary logits."""
@@ -375,24 +377,25 @@ ROUTER_EPS = {"bf16": 1e-2, "fp32": 1e-4}  # router logits are O(1); half the ba
 
 
 def assert_routing_is_a_valid_topk(cfg, ex, rlog, what=""):
-    """ex [L, 2, B, kmax]: the device's expert ids; rlog [L, 2, B, E]: the oracle's router logits for the same
+    """ex [L, K, B, kmax]: the device's expert ids; rlog [L, K, B, E]: the oracle's router logits for the same
     rows (computed under the device's choice in the earlier layers).  Eq. moe_layer fixes the selected set
     only up to rounding at near-ties, so what must hold is: k distinct experts per row, none of them below
     an unselected expert by more than the logit tolerance (softmax is monotone, so logits order as the
     probabilities do), the unused slots -1, and under router replay (Section 4.3) the branch's set is the
     primary's."""
     eps = ROUTER_EPS[cfg.weight_dtype]
-    L, _, B, _ = ex.shape
+    L, K, B, _ = ex.shape
+    assert K == cfg.n_paths
     replay = cfg.router_mode == 1
     for l in range(L):
-        for p in range(2):
+        for p in range(K):
             k = cfg.k_primary if (p == 0 or replay) else cfg.k_branch
             for b in range(B):
                 chosen = ex[l, p, b, :k]
                 assert (ex[l, p, b, k:] == -1).all(), f"{what} layer {l} path {p} row {b}: unused slots"
                 assert ((chosen >= 0) & (chosen < cfg.n_experts)).all() and len(set(chosen.tolist())) == k, \
                     f"{what} layer {l} path {p} row {b}: {chosen}"
-                if p == 1 and replay:
+                if p >= 1 and replay:
                     assert chosen.tolist() == ex[l, 0, b, :k].tolist(), f"{what} layer {l} row {b}: replay set"
                     continue
                 r = rlog[l, p, b]
@@ -514,6 +517,48 @@ def test_moe_1b_at_the_benchmarks_launch_configuration_on_sampled_sequences(matc
         assert_logits_close(g["z1"][pick], o["z1"], "bf16", f"moe bench config step {t} z1")
         assert_logits_close(g["z2"][pick], o["z2"], "bf16", f"moe bench config step {t} z2")
     assert gm.sync_status() == (0, 0)
+
+
+# ---- more decode branches (Appendix C.1) ----------------------------------------------------------------------
+
+@pytest.mark.parametrize("cfg,B,T,npre", [
+    (small_bf16(n_paths=3), 3, 40, 35),                                        # 3 paths x 4 queries per KV head: 12 of 16 rows
+    (small_bf16(n_paths=4, n_q_heads=4, n_kv_heads=4), 2, 24, 20),             # MHA, 4 paths
+    (small_bf16(n_paths=8, n_q_heads=2, n_kv_heads=1, head_dim=128, d_model=128, vocab=777), 5, 50, 47),  # 8 paths, 16 rows
+    (tiny_dense_fp32().replace(n_paths=3), 2, 30, 25),                         # the fp32 kernels
+    (small_bf16(n_paths=3, n_q_heads=8, n_kv_heads=2), 33, 20, 18),            # 99 stacked rows: row tile 128
+])
+def test_more_decode_branches_dense(cfg, B, T, npre):
+    """K > 2: every branch's logits, alpha and the token of alpha p + (1-alpha) mean_j q_j against the oracle."""
+    w = make_weights(cfg, seed=5, matrix_std=0.05 if cfg.weight_dtype == "bf16" else 0.02)
+    tok = make_tokens(cfg, B, T, seed=6)
+    teacher_forced_compare(cfg, w, tok, n_prefill=npre, grouped=True)
+
+
+@pytest.mark.parametrize("cfg", [small_moe(n_paths=3), small_moe(n_paths=3, router_mode=1),
+                                 small_moe(n_paths=4, compute_matched=1), small_moe(n_paths=3, weight_dtype="fp32")])
+def test_more_decode_branches_moe(cfg):
+    """Every branch routes for itself (fan-out k_2; router replay: the primary's set), checked row by row."""
+    _moe_compare(cfg, B=3, T=14, npre=10)
+
+
+def test_identical_branch_tables_give_identical_branch_logits_on_the_device():
+    cfg = small_bf16(n_paths=3)
+    w = make_weights(cfg, seed=5, matrix_std=0.05)
+    V = cfg.vocab
+    w["embed_branch"] = torch.cat([w["embed_branch"][:V], w["embed_branch"][:V]]).contiguous()
+    tok = make_tokens(cfg, 3, 24, seed=6).cuda()
+    gm = make_gpu_model(cfg, w, 3, 24)
+    for o in _run_steps(gm, tok, 20, True):
+        assert torch.equal(o["z2"][0], o["z2"][1]) and float(o["z2"].abs().max()) > 0
+
+
+def test_too_many_query_rows_over_all_paths_are_rejected():
+    cfg = small_bf16(n_paths=5)  # 5 paths x 4 queries per KV head > 16
+    w = make_weights(cfg, seed=0)
+    with pytest.raises(binding.DbtError) as e:
+        make_gpu_model(cfg, w, 1, 16)
+    assert e.value.status == 2
 
 
 # ---- compute-matched MoE allocation (Appendix B.3) ---------------------------------------------------------
