@@ -42,8 +42,23 @@ def load_peaks() -> dict:
     if os.path.exists(path):
         with open(path) as f:
             p = json.load(f)
-        return {"hbm_gbs": float(p["hbm_gbs"]), "source": "measured"}
-    return {"hbm_gbs": 6650.0, "source": "fallback"}
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", 1400.0)),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def prefill_flops(cfg, B: int, n: int) -> float:
+    """Useful FLOPs of a primary-only prefill of n positions for B sequences: every layer matrix once per token
+    (2 FLOP per weight; MoE: k_primary routed experts + the shared ones) plus causal attention
+    (Q K^T and P V over n (n + 1) / 2 query-key pairs per head)."""
+    per_layer = (cfg.q_dim + 2 * cfg.kv_dim) * cfg.d_model + cfg.d_model * cfg.q_dim
+    if cfg.is_moe:
+        per_layer += 3 * cfg.d_expert * cfg.d_model * (cfg.k_primary + cfg.n_shared_experts) + cfg.n_experts * cfg.d_model
+    else:
+        per_layer += 3 * cfg.d_ff * cfg.d_model
+    gemm = 2.0 * per_layer * cfg.n_layers * B * n
+    attn = 4.0 * cfg.q_dim * cfg.n_layers * B * (n * (n + 1) / 2.0)
+    return gemm + attn
 
 
 class ClockSampler:
@@ -112,6 +127,8 @@ def bench_config(args):
         cfg = cfg.replace(k_branch=args.k_branch, router_mode=args.router_mode, compute_matched=args.compute_matched)
         if args.k_primary:
             cfg = cfg.replace(k_primary=args.k_primary)
+    if args.paths != 2:  # more decode branches (Appendix C.1)
+        cfg = cfg.replace(n_paths=args.paths)
     if args.layers:  # profiler captures of one kernel: fewer layers, less device memory to save and restore
         cfg = cfg.replace(n_layers=args.layers)
     return cfg
@@ -119,7 +136,8 @@ def bench_config(args):
 
 def workload_name(cfg, args) -> str:
     if not cfg.is_moe:
-        return f"dense-{args.model}" + (f" (cut to {cfg.n_layers} layers)" if args.layers else "")
+        return (f"dense-{args.model}" + (f" (cut to {cfg.n_layers} layers)" if args.layers else "")
+                + (f" with {cfg.n_paths - 1} decode branches" if cfg.n_paths != 2 else ""))
     kind = "compute-matched " if cfg.compute_matched else ""
     cut = f", cut to {cfg.n_layers} layers" if args.layers else ""
     return f"{kind}moe-{args.model} (top-{cfg.k_primary} primary, top-{cfg.k_branch} branch{cut})"
@@ -157,32 +175,45 @@ def run_ours(args) -> dict | None:
     tok_a = torch.empty(B, dtype=torch.int32, device=dev)
     tok_b = torch.empty(B, dtype=torch.int32, device=dev)
 
-    def timed(grouped: bool, steps: int, warmup: int, sample_clocks: bool):
-        m.set_seq_lens([S - 1] * B)
-        tok_a.copy_(first)
-        cur, nxt = tok_a, tok_b
+    def timed(grouped: bool, steps: int, warmup: int, sample_clocks: bool, min_total_ms: float = 500.0, max_regions: int = 200):
+        """Regions of exactly `steps` steps (every region restarts from the prompt's end, after `warmup` untimed
+        steps), each bracketed by barrier + synchronize and timed with CUDA events on the launching stream;
+        repeated until at least min_total_ms of device time has been timed, so that the clock sampler sees the
+        GPU under load for several samples whatever `steps` is.  Returns the MEDIAN region."""
         step = m.decode_step if grouped else m.decode_step_primary_only
-        for _ in range(warmup):
-            step(cur, nxt)
-            cur, nxt = nxt, cur
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        replicas.barrier()
-        torch.cuda.synchronize()
         sampler = ClockSampler(local_rank) if sample_clocks else None
-        launches0 = m.launch_count()
-        e0.record(stream)
-        for _ in range(steps):
-            step(cur, nxt)
-            cur, nxt = nxt, cur
-        e1.record(stream)
-        torch.cuda.synchronize()
-        replicas.barrier()
+        regions, launches = [], 0
+        while True:
+            m.set_seq_lens([S - 1] * B)
+            tok_a.copy_(first)
+            cur, nxt = tok_a, tok_b
+            for _ in range(warmup):
+                step(cur, nxt)
+                cur, nxt = nxt, cur
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            replicas.barrier()
+            torch.cuda.synchronize()
+            launches0 = m.launch_count()
+            e0.record(stream)
+            for _ in range(steps):
+                step(cur, nxt)
+                cur, nxt = nxt, cur
+            e1.record(stream)
+            torch.cuda.synchronize()
+            replicas.barrier()
+            regions.append(e0.elapsed_time(e1))
+            launches = m.launch_count() - launches0
+            # every rank must leave the loop in the same round: decide on rank-uniform data
+            done = replicas.all_agree(sum(regions) >= min_total_ms or len(regions) >= max_regions, dev)
+            if done:
+                break
         clocks = sampler.stop() if sampler else None
-        return e0.elapsed_time(e1), m.launch_count() - launches0, clocks
+        regions.sort()
+        return regions[len(regions) // 2], launches, clocks, len(regions)
 
-    ms_po, _, _ = timed(False, K, W, False)
+    ms_po, _, _, _ = timed(False, K, W, False, min_total_ms=200.0)
     po_union_m = m.last_expert_union() if cfg.is_moe else None
-    ms_total, launches, clocks = timed(True, K, W, True)
+    ms_total, launches, clocks, n_regions = timed(True, K, W, True)
     value, ms_max = replicas.aggregate_throughput(B * K, ms_total, dev)
     ms_step = ms_max / K
     union = po_union = None
@@ -232,7 +263,9 @@ def run_ours(args) -> dict | None:
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        cpu = cpu_baseline(cfg, w, S, steps=2)
+        cpu = cpu_baseline(cfg, w, S, steps=4, warm=1)
+        one = cpu_baseline(cfg, w, S, steps=1, warm=1, threads=1)
+        cpu["one_thread"] = {"value": one["value"], "ms_per_step": one["ms_per_step"]}
     if rank != 0:
         return None
     hbm = peaks["hbm_gbs"]
@@ -245,7 +278,8 @@ def run_ours(args) -> dict | None:
                                f"{K} steps (paged KV, 16-token pages)",
                    "batch_per_gpu": B, "prompt": S, "kv_population": kv_mode,
                    "l2_policy": "inputs larger than L2 (weights + KV >= 1.7 GB per step vs 126 MB)",
-                   "replicas": world, "device_status": status[0]},
+                   "replicas": world, "device_status": status[0],
+                   "timed_regions": n_regions, "region_reported": "median of the K-step regions"},
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": 4 * B, "d2h_bytes_per_step": 8 * B,
                 "ms_per_step": e2e_ms / K},
@@ -269,13 +303,24 @@ def run_ours(args) -> dict | None:
                      "gbs": (r["bytes"] / (r["total_ms"] * 1e-3) / 1e9) if r["bytes"] > 0 and r["total_ms"] > 0 else None}
                     for r in prof],
         "cpu_baseline": cpu, "setup_s": setup_s, "prefill_s": t_prefill,
+        "prefill": None if t_prefill is None else {
+            "tokens": B * (S - 1), "tokens_per_s": B * (S - 1) / t_prefill,
+            "useful_tflops": prefill_flops(cfg, B, S - 1) / t_prefill / 1e12,
+            "frac_of_bf16_sustained": prefill_flops(cfg, B, S - 1) / t_prefill / 1e12 / peaks["bf16_tflops_sustained"],
+            "bound": "tensor", "note": "primary path only (Section 4.4 item 1); wall clock of one dbt_prefill call "
+                                       "including its launches; activations as two bf16 planes double the tensor work"},
     }
 
 
-def cpu_baseline(cfg, w, S: int, steps: int, batch: int = 1, warm: int = 0) -> dict:
+def cpu_baseline(cfg, w, S: int, steps: int, batch: int = 1, warm: int = 0, threads: int = 0) -> dict:
     """The oracle as it stands, timed on this machine's host cores on a bounded sample of the
-    workload: `batch` sequence(s) with an S-1 position synthetic cache, `steps` grouped steps."""
+    workload: `batch` sequence(s) with an S-1 position synthetic cache, `warm` untimed and `steps`
+    timed grouped steps (threads: 0 = all cores)."""
     import oracle
+
+    all_threads = oracle.get_threads()
+    if threads:
+        oracle.set_threads(threads)
 
     k, v = make_synthetic_kv(cfg, batch, S - 1, seed=3)
     om = oracle.OracleModel(cfg, w, batch, S + steps + warm + 1)
@@ -287,8 +332,12 @@ def cpu_baseline(cfg, w, S: int, steps: int, batch: int = 1, warm: int = 0) -> d
     for i in range(steps):
         om.decode_step(tok[:, warm + i])
     dt = time.perf_counter() - t0
-    return {"value": batch * steps / dt, "unit": UNIT, "cores": oracle.get_threads(), "kind": "oracle",
-            "sample": f"{steps} grouped steps of {batch} sequence(s) at context {S} (synthetic cache), full model",
+    used = oracle.get_threads()
+    if threads:
+        oracle.set_threads(all_threads)
+    return {"value": batch * steps / dt, "unit": UNIT, "cores": used, "kind": "oracle",
+            "sample": f"{steps} grouped steps (after {warm} warm) of {batch} sequence(s) at context {S} "
+                      f"(synthetic cache), full model",
             "ms_per_step": 1e3 * dt / steps}
 
 
@@ -329,6 +378,7 @@ def main():
     ap.add_argument("--router-mode", type=int, default=0, help="MoE: 0 independent routing, 1 router replay")
     ap.add_argument("--compute-matched", type=int, default=0,
                     help="MoE: 1 = compute-matched allocation (attention and shared expert on the primary path only)")
+    ap.add_argument("--paths", type=int, default=2, help="residual paths K: the primary plus K-1 decode branches (Appendix C.1)")
     ap.add_argument("--layers", type=int, default=0, help="cut the model to this many layers (profiler captures only)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--reference-max-steps", type=int, default=128)

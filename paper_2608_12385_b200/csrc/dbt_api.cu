@@ -142,7 +142,13 @@ int npaths(int grouped) { return grouped > 1 ? grouped : 1; }
 // Kernels that pair a primary row with one branch row run a block per branch in grid.z.
 unsigned branch_blocks(int grouped) { return grouped > 1 ? (unsigned)(grouped - 1) : 1u; }
 int kmax_of(const dbt_config &c) { return c.k_primary > c.k_branch ? c.k_primary : c.k_branch; }
-int prefill_rows(const dbt_config &c) { return paths_of(c) * c.max_batch > 256 ? paths_of(c) * c.max_batch : 256; }
+// Rows of the activation buffers: all paths of a full batch in a decode step, or one prompt chunk of the
+// prefill (2048 rows for dense bf16 models, whose GEMMs sweep several row tiles per weight tile and whose
+// causal attention packs consecutive positions into a query tile; 256 otherwise).
+int prefill_rows(const dbt_config &c) {
+    int chunk = (c.weight_dtype == DBT_DTYPE_BF16 && c.n_experts == 0) ? 2048 : 256;
+    return paths_of(c) * c.max_batch > chunk ? paths_of(c) * c.max_batch : chunk;
+}
 
 const char *check_config(const dbt_config *c, dbt_status *st) {
     *st = DBT_ERR_INVALID_ARG;
@@ -174,6 +180,9 @@ const char *check_config(const dbt_config *c, dbt_status *st) {
     return nullptr;
 }
 
+// Rows whose attention may be split into segments: a decode step's, or an unpacked prompt chunk's (<= 256).
+int att_rows_of(const dbt_config &c) { return paths_of(c) * c.max_batch > 256 ? paths_of(c) * c.max_batch : 256; }
+
 // One pass over the workspace layout; with base == nullptr it only measures.
 size_t carve(const dbt_config &c, char *base, Workspace *ws, int *Rmax_out, int *part_items_out) {
     Carver k{base, 0};
@@ -184,7 +193,8 @@ size_t carve(const dbt_config &c, char *base, Workspace *ws, int *Rmax_out, int 
     int Fs = moe ? c.n_shared_experts * c.d_expert : 0;
     int F = moe ? (Fs > 0 ? Fs : 8) : c.d_ff;
     int pps = (c.max_seq + c.page_size - 1) / c.page_size;
-    int part_items = Rmax * c.n_kv_heads + 8 * 148;  // attention partial slots: up to three rounds of 2 x 148 segments plus one per pair
+    int att_rows = att_rows_of(c);
+    int part_items = att_rows * c.n_kv_heads + 8 * 148;  // attention partial slots: up to three rounds of 2 x 148 segments plus one per pair
     w.S = k.take<float>((size_t)Rmax * d);
     w.X = k.take<float>((size_t)Rmax * d);
     w.Q = k.take<float>((size_t)Rmax * qd);
@@ -200,8 +210,8 @@ size_t carve(const dbt_config &c, char *base, Workspace *ws, int *Rmax_out, int 
     w.seq_len = k.take<int32_t>(c.max_batch);
     w.page_table = k.take<int32_t>((size_t)c.max_batch * pps);
     w.status = k.take<int32_t>(4);
-    w.att_tickets = k.take<int32_t>((size_t)Rmax * c.n_kv_heads);
-    w.att_tickets2 = k.take<int32_t>((size_t)Rmax * c.n_kv_heads * kAttMaxGroups);
+    w.att_tickets = k.take<int32_t>((size_t)att_rows * c.n_kv_heads);
+    w.att_tickets2 = k.take<int32_t>((size_t)att_rows * c.n_kv_heads * kAttMaxGroups);
     w.ro_stats = k.take<float>((size_t)c.max_batch * kRoMaxChunks * kRoRec);
     w.ro_tickets = k.take<int32_t>(c.max_batch);
     w.gemm_tickets = k.take<int32_t>(4096);
@@ -340,6 +350,15 @@ cudaEvent_t prof_event(dbt_model *m) {
             (m)->prof.push_back(dbt_model::ProfRec{tag, (double)(bytes), p0_, p1_});                     \
         }                                                                                                \
         if (e_ != cudaSuccess) return fail(m, DBT_ERR_CUDA, "launch %s: %s", #kernel, cudaGetErrorString(e_)); \
+    } while (0)
+
+// Kernels templated on "more than one decode branch" (see resid_wide_kernel).
+#define LAUNCH_BR(m, grouped, tag, bytes, kernel, grid, block, smem, ...)                \
+    do {                                                                                 \
+        if ((grouped) > 2)                                                               \
+            LAUNCH(m, tag, bytes, kernel<true>, grid, block, smem, __VA_ARGS__);         \
+        else                                                                             \
+            LAUNCH(m, tag, bytes, kernel<false>, grid, block, smem, __VA_ARGS__);        \
     } while (0)
 
 // ---- launch helpers -------------------------------------------------------------------
@@ -634,6 +653,15 @@ dbt_status run_gemm_tc(dbt_model *m, const TcCall &c, int n_tile, int *nsplit_ou
     p.status = m->ws.status;
     p.evict_first = m->evict_first ? 1 : 0;
     p.test_skip_load = test_skip_load;
+    // more rows than the widest tile (prompt chunks): several row tiles per weight tile, no split-K
+    int row_tiles = 1;
+    if (!c.grp_cnt && c.R > 256) {
+        if (e.Z) return fail(m, DBT_ERR_UNSUPPORTED, "the output-matrix epilogue takes at most 256 rows");
+        n_tile = 256;
+        row_tiles = (c.R + 255) / 256;
+        force_split = 1;
+    }
+    p.row_tiles = row_tiles;
     int total_kt = (c.K + kTcK - 1) / kTcK;
     if (c.grp_cnt) force_split = 1;  // enough CTAs already: tiles x selected experts
     int split = force_split > 0 ? (force_split < total_kt ? force_split : total_kt) : choose_split(tiles, total_kt, split_slots(m, n_tile));
@@ -645,7 +673,7 @@ dbt_status run_gemm_tc(dbt_model *m, const TcCall &c, int n_tile, int *nsplit_ou
         split = 1;
         p.kt_per_split = total_kt;
     }
-    dim3 grid(tiles, c.grp_cnt && c.grp_row_tiles ? c.grp_row_tiles : split, c.grp_cnt ? c.n_groups : 1);
+    dim3 grid(tiles * row_tiles, c.grp_cnt && c.grp_row_tiles ? c.grp_row_tiles : split, c.grp_cnt ? c.n_groups : 1);
     if (nsplit_out) *nsplit_out = split;
     if (split_stride_out) *split_stride_out = (size_t)c.R * col;
     switch (n_tile) {
@@ -670,7 +698,7 @@ struct QkvFuse {
 
 template <int DH>
 dbt_status run_attention_mma(dbt_model *m, const RowMap &rm, int grouped, int layer, double kv_bytes,
-                             const QkvFuse *qf = nullptr) {
+                             const QkvFuse *qf = nullptr, bool pack_prompt = false) {
     const dbt_config &c = m->cfg;
     const Workspace &w = m->ws;
     int items = rm.B * rm.cn, G = c.n_q_heads / c.n_kv_heads;
@@ -707,11 +735,18 @@ dbt_status run_attention_mma(dbt_model *m, const RowMap &rm, int grouped, int la
         p.kpool = reinterpret_cast<__nv_bfloat16 *>(m->kv_pool) + (size_t)layer * 2 * plane * c.head_dim;
         p.vpool = p.kpool + (size_t)plane * c.head_dim;
     }
-    if (items > kAttMaxItems) return fail(m, DBT_ERR_CAPACITY, "attention rows %d exceed %d", items, kAttMaxItems);
+    // prompt chunks: 16 / G consecutive positions of a sequence share a query tile (the 16-row kernel)
+    const bool packed = pack_prompt && !grouped && !qf && rm.cn > 1;
+    if (packed) {
+        p.pack = 16 / G;
+        p.cn = rm.cn;
+        p.nbk = (rm.cn + p.pack - 1) / p.pack;
+    }
+    if (!packed && items > kAttMaxItems) return fail(m, DBT_ERR_CAPACITY, "attention rows %d exceed %d", items, kAttMaxItems);
     dim3 grid(2 * m->num_sms);  // two resident CTAs per SM; each takes an equal share of all K/V tiles
     // up to 8 query rows per KV head over both paths: the transposed-product variant (fixed per
     // model, so that grouped and primary-only steps run the same arithmetic on the primary rows)
-    if (paths_of(c) * G <= 8)
+    if (paths_of(c) * G <= 8 && !packed)
         LAUNCH(m, "attention", kv_bytes, (attn_mma_kernel<DH, true>), grid, 160, AttCfg<DH>::kSmemBytes, m->map_kv, p);
     else
         LAUNCH(m, "attention", kv_bytes, (attn_mma_kernel<DH, false>), grid, 160, AttCfg<DH>::kSmemBytes, m->map_kv, p);
@@ -830,7 +865,7 @@ dbt_status run_moe_tc(dbt_model *m, int l, const RowMap &rm, int grouped, bool r
     if (Fs > 0 && !overlap && (st = shared_expert(w.P, w.P_floats)) != DBT_OK) return st;
     if (overlap) CUDA_TRY(m, cudaStreamWaitEvent(main_stream, m->ev_join, 0));
     const bool next_in = wide && g_next != nullptr;
-    LAUNCH(m, "moe_combine", 0, moe_combine_sorted_kernel, dim3(Bc, (d + 255) / 256, branch_blocks(grouped)), 256, 0, w.Yexp, Psh, nsp, sstride, w.ridx, w.epos, w.rwts, km,
+    LAUNCH_BR(m, grouped, "moe_combine", 0, moe_combine_sorted_kernel, dim3(Bc, (d + 255) / 256, branch_blocks(grouped)), 256, 0, w.Yexp, Psh, nsp, sstride, w.ridx, w.epos, w.rwts, km,
            Bc, grouped, lw.coup_c, matched ? lw.gate_g : (const float *)nullptr, d, w.S, next_in ? g_next : (const float *)nullptr,
            next_in ? w.Xb : (__nv_bfloat16 *)nullptr, lo_x, next_in ? w.ss : (float *)nullptr, ss_ld);
     return DBT_OK;
@@ -874,7 +909,7 @@ dbt_status run_layers_tc(dbt_model *m, const RowMap &rm, int grouped, int n_tile
         // has left it already, the first layer gets it from the residual kernel with nothing to add.
         if (mwide) {
             if (l == 0)
-                LAUNCH(m, "resid_wide", 0, resid_wide_kernel, dim3(Bc, mss_tiles, branch_blocks(grouped)), 256, 0, w.S, w.P, 0, (size_t)0, 1,
+                LAUNCH_BR(m, grouped, "resid_wide", 0, resid_wide_kernel, dim3(Bc, mss_tiles, branch_blocks(grouped)), 256, 0, w.S, w.P, 0, (size_t)0, 1,
                        (const float *)nullptr, Bc, grouped, lw.attn_norm_g, d, w.Xb, lo_x, w.ss, m->Rmax);
         } else {
             LAUNCH(m, "resid_norm", 0, resid_norm_kernel, dim3(Bc, 1, branch_blocks(grouped)), norm_threads(d), 0, w.S, w.P, nsp, sstride, mode,
@@ -908,7 +943,7 @@ dbt_status run_layers_tc(dbt_model *m, const RowMap &rm, int grouped, int n_tile
         if ((st = run_gemm_tc(m, op, n_tile, &nsp, &sstride)) != DBT_OK) return st;
         // S-bar_i = S_i + Attn_i W_O (matched: S-bar_2 = S_2 + g_A * Attn_1 W_O) ; RMSNorm for the MLP
         if (mwide)
-            LAUNCH(m, "resid_wide", 0, resid_wide_kernel, dim3(Bc, mss_tiles, branch_blocks(grouped)), 256, 0, w.S, w.P, nsp, sstride, matched ? 3 : 1,
+            LAUNCH_BR(m, grouped, "resid_wide", 0, resid_wide_kernel, dim3(Bc, mss_tiles, branch_blocks(grouped)), 256, 0, w.S, w.P, nsp, sstride, matched ? 3 : 1,
                    matched ? lw.gate_a : (const float *)nullptr, Bc, grouped, lw.mlp_norm_g, d, w.Xb, lo_x, w.ss, m->Rmax);
         else
         LAUNCH(m, "resid_norm", 0, resid_norm_kernel, dim3(Bc, 1, branch_blocks(grouped)), norm_threads(d), 0, w.S, w.P, nsp, sstride, matched ? 3 : 1,
@@ -1060,14 +1095,14 @@ dbt_status run_layers_wide(dbt_model *m, const RowMap &rm, int grouped, int n_ti
                    w.Q, rm, grouped, c.n_q_heads, c.n_kv_heads, c.head_dim, lw.coup_a, w.rope, w.seq_len, w.page_table,
                    m->pages_per_seq_max, c.num_pages, c.page_size, kpool, vpool, w.status, (const float *)w.ss, ss_tiles, ss_ld, d,
                    c.rms_eps);
-        st = c.head_dim == 128 ? run_attention_mma<128>(m, rm, grouped, l, kv_bytes, fuse ? &qf : nullptr)
-                               : run_attention_mma<64>(m, rm, grouped, l, kv_bytes, fuse ? &qf : nullptr);
+        st = c.head_dim == 128 ? run_attention_mma<128>(m, rm, grouped, l, kv_bytes, fuse ? &qf : nullptr, true)
+                               : run_attention_mma<64>(m, rm, grouped, l, kv_bytes, fuse ? &qf : nullptr, true);
         if (st != DBT_OK) return st;
         TcCall op = call("gemm_o", &m->map_Ob, qd);
         op.W[0] = &mp.wo; op.n_out[0] = d; op.rows[0] = R; op.nseg = 1;
         {
             if ((st = run_gemm_tc(m, op, n_tile, &nsp, &sstride)) != DBT_OK) return st;
-            LAUNCH(m, "resid_wide", 0, resid_wide_kernel, dim3(Bc, ss_tiles, branch_blocks(grouped)), 256, 0, w.S, w.P, nsp, sstride, 1,
+            LAUNCH_BR(m, grouped, "resid_wide", 0, resid_wide_kernel, dim3(Bc, ss_tiles, branch_blocks(grouped)), 256, 0, w.S, w.P, nsp, sstride, 1,
                    (const float *)nullptr, Bc, grouped, lw.mlp_norm_g, d, w.Xb, lo_x, w.ss, ss_ld);
         }
         TcCall gu = call("gemm_gateup", &m->map_Xb, d);
@@ -1085,7 +1120,7 @@ dbt_status run_layers_wide(dbt_model *m, const RowMap &rm, int grouped, int n_ti
                                                  : (c.final_norm ? m->w.final_norm_g : (const float *)nullptr);
         {
             if ((st = run_gemm_tc(m, dn, n_tile, &nsp, &sstride)) != DBT_OK) return st;
-            LAUNCH(m, "resid_wide", 0, resid_wide_kernel, dim3(Bc, ss_tiles, branch_blocks(grouped)), 256, 0, w.S, w.P, nsp, sstride, 2, lw.coup_c, Bc,
+            LAUNCH_BR(m, grouped, "resid_wide", 0, resid_wide_kernel, dim3(Bc, ss_tiles, branch_blocks(grouped)), 256, 0, w.S, w.P, nsp, sstride, 2, lw.coup_c, Bc,
                    grouped, g_next, d, w.Xb, lo_x, w.ss, ss_ld);
         }
     }
@@ -1147,7 +1182,7 @@ dbt_status prefill_wide(dbt_model *m, const int32_t *tokens_dev, int B, int n, f
     typedef __nv_bfloat16 WT;
     const dbt_config &c = m->cfg;
     const Workspace &w = m->ws;
-    int cn_max = (m->Rmax < kAttMaxItems ? m->Rmax : kAttMaxItems) / B;
+    int cn_max = m->Rmax / B;  // a chunk of up to Rmax rows: GEMMs over several row tiles, packed causal attention
     if (cn_max < 1) cn_max = 1;
     // when logits are wanted the last position runs as its own chunk, so that the rows of the
     // output-matrix GEMM are exactly the B last positions
@@ -1156,7 +1191,7 @@ dbt_status prefill_wide(dbt_model *m, const int32_t *tokens_dev, int B, int n, f
     for (int p0 = 0; p0 < n;) {
         int cn = p0 < n_bulk ? (n_bulk - p0 < cn_max ? n_bulk - p0 : cn_max) : 1;
         RowMap rm{B, cn};
-        int R = B * cn, n_tile = pad_rows(R);
+        int R = B * cn, n_tile = pad_rows(R < 256 ? R : 256);
         if ((st = run_embed_wide<WT>(m, tokens_dev, n, p0, rm, R, n_tile)) != DBT_OK) return st;
         if ((st = run_layers_wide(m, rm, 0, n_tile)) != DBT_OK) return st;
         if (last_logits && p0 + cn >= n) {
@@ -1188,7 +1223,7 @@ bool setup_tc(dbt_model *m) {
     const Workspace &w = m->ws;
     const char *force = getenv("DBT_FORCE_PATH");
     if (force && strcmp(force, "simt") == 0) return false;
-    if (c.weight_dtype != DBT_DTYPE_BF16 || m->Rmax > 256) return false;
+    if (c.weight_dtype != DBT_DTYPE_BF16) return false;
     if (!allow_smem_all()) return false;
     int d = c.d_model, qd = c.n_q_heads * c.head_dim, kvd = c.n_kv_heads * c.head_dim;
     bool moe = c.n_experts > 0;
@@ -1449,8 +1484,8 @@ dbt_status dbt_create(const dbt_config *cfg, const dbt_weights *w, void *kv_pool
         e = cudaMemcpyAsync(m->ws.page_table, pt.data(), pt.size() * sizeof(int32_t), cudaMemcpyHostToDevice, m->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(m->ws.seq_len, 0, sizeof(int32_t) * cfg->max_batch, m->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(m->ws.status, 0, sizeof(int32_t) * 4, m->stream);
-    if (e == cudaSuccess) e = cudaMemsetAsync(m->ws.att_tickets, 0, sizeof(int32_t) * (size_t)m->Rmax * cfg->n_kv_heads, m->stream);
-    if (e == cudaSuccess) e = cudaMemsetAsync(m->ws.att_tickets2, 0, sizeof(int32_t) * (size_t)m->Rmax * cfg->n_kv_heads * kAttMaxGroups, m->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(m->ws.att_tickets, 0, sizeof(int32_t) * (size_t)att_rows_of(*cfg) * cfg->n_kv_heads, m->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(m->ws.att_tickets2, 0, sizeof(int32_t) * (size_t)att_rows_of(*cfg) * cfg->n_kv_heads * kAttMaxGroups, m->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(m->ws.ro_tickets, 0, sizeof(int32_t) * (size_t)cfg->max_batch, m->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(m->ws.gemm_tickets, 0, sizeof(int32_t) * 4096, m->stream);
     if (e == cudaSuccess && moe) {
@@ -1570,8 +1605,8 @@ dbt_status dbt_reset(dbt_model *m) {
     if (!m) return DBT_ERR_INVALID_ARG;
     CUDA_TRY(m, cudaMemsetAsync(m->ws.seq_len, 0, sizeof(int32_t) * m->cfg.max_batch, m->stream));
     CUDA_TRY(m, cudaMemsetAsync(m->ws.status, 0, sizeof(int32_t) * 4, m->stream));
-    CUDA_TRY(m, cudaMemsetAsync(m->ws.att_tickets, 0, sizeof(int32_t) * (size_t)m->Rmax * m->cfg.n_kv_heads, m->stream));
-    CUDA_TRY(m, cudaMemsetAsync(m->ws.att_tickets2, 0, sizeof(int32_t) * (size_t)m->Rmax * m->cfg.n_kv_heads * kAttMaxGroups, m->stream));
+    CUDA_TRY(m, cudaMemsetAsync(m->ws.att_tickets, 0, sizeof(int32_t) * (size_t)att_rows_of(m->cfg) * m->cfg.n_kv_heads, m->stream));
+    CUDA_TRY(m, cudaMemsetAsync(m->ws.att_tickets2, 0, sizeof(int32_t) * (size_t)att_rows_of(m->cfg) * m->cfg.n_kv_heads * kAttMaxGroups, m->stream));
     CUDA_TRY(m, cudaMemsetAsync(m->ws.gemm_tickets, 0, sizeof(int32_t) * 4096, m->stream));
     CUDA_TRY(m, cudaMemsetAsync(m->ws.ro_tickets, 0, sizeof(int32_t) * (size_t)m->cfg.max_batch, m->stream));
     std::fill(m->len_host.begin(), m->len_host.end(), 0);

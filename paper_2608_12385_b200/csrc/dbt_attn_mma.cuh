@@ -58,6 +58,11 @@ struct AttnParams {
     const float *coup_a;
     const float2 *rope;
     __nv_bfloat16 *kpool, *vpool;  // this layer's K and V planes
+    // Prompt chunks (Section 4.4 item 1, the primary path alone): pack > 0 packs `pack` consecutive positions of
+    // a sequence (times the G heads of the KV head) into one 16-row query tile, each row with its own causal
+    // limit; a chunk holds cn positions per sequence, nbk = ceil(cn / pack) tiles per sequence, one CTA pass per
+    // (tile, KV head) over all its keys, no split.  Q rows and output rows are seq * cn + position.
+    int pack, cn, nbk;
 };
 
 constexpr int kAttTile = 64;       // tokens per pipeline stage (4 pages)
@@ -153,6 +158,12 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
     int items = p.rm.Bc(), Bc = items;
     const int P = p.grouped > 1 ? p.grouped : 1;  // query rows of a KV head: G heads of every path, path-major
     int nq_act = P * p.G, q_dim = p.n_kv * p.G * DH;
+    const bool packed = p.pack > 0;
+    if (packed) items = p.rm.B * p.nbk;
+    // geometry of an item: its sequence, the keys visible to its last row, the positions it holds
+    auto item_seq = [&](int i) { return packed ? i / p.nbk : p.rm.seq(i); };
+    auto item_npos = [&](int i) { return packed ? min(p.pack, p.cn - (i % p.nbk) * p.pack) : 1; };
+    auto item_row0 = [&](int i) { return packed ? (i / p.nbk) * p.cn + (i % p.nbk) * p.pack : i; };  // first Q / output row
 
     if (tid == 0) {
         for (int s = 0; s < STAGES; s++) {
@@ -164,7 +175,7 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
     pdl_launch_dependents();
     pdl_wait();  // sequence lengths, Q and the freshly appended K/V come from earlier kernels of the step
     DBT_TL_WAITED;
-    if (warp == 0) {
+    if (warp == 0 && !packed) {
         int running = 0, longest = 0;
         if (lane == 0) cum[0] = 0;
         for (int base = 0; base < items; base += 32) {
@@ -244,11 +255,25 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
         }
     }
     __syncthreads();
-    const int C = gridDim.x, Sg = segcum[items] * p.n_kv;  // all segments, ordered (row, KV head, segment)
+    const int C = gridDim.x, Sg = packed ? items * p.n_kv : segcum[items] * p.n_kv;  // all segments, ordered (row, KV head, segment)
     DBT_TL_MARK(3);
     if ((int)blockIdx.x >= Sg) return;
     // segment sidx -> its row, KV head, stage range and the pair's segment count
+    auto item_nkeys = [&](int i) {
+        if (!packed) return nk_s[i];
+        return ld_mut(p.seq_len + i / p.nbk) + (i % p.nbk) * p.pack + item_npos(i);
+    };
     auto locate = [&](int sidx, int &item, int &g, int &seg, int &n, int &ui, int &t0, int &t1) {
+        if (packed) {  // one pass per (tile, KV head) over all its keys
+            item = sidx / p.n_kv;
+            g = sidx % p.n_kv;
+            seg = 0;
+            n = 1;
+            ui = (item_nkeys(item) + kAttTile - 1) / kAttTile;
+            t0 = 0;
+            t1 = ui;
+            return;
+        }
         int lo = 0, hi = items - 1;
         while (lo < hi) {  // largest row whose first segment is <= sidx
             int mid = (lo + hi + 1) >> 1;
@@ -275,7 +300,7 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
         for (int sidx = blockIdx.x; sidx < Sg && ok; sidx += C) {
             int item, g, seg, n, ui, t0, t1;
             locate(sidx, item, g, seg, n, ui, t0, t1);
-            int seq = p.rm.seq(item), total_pages = (nk_s[item] + 15) >> 4;
+            int seq = item_seq(item), total_pages = (item_nkeys(item) + 15) >> 4;
             for (int t = t0; t < t1; t++, it++) {
                 int s = it % STAGES;
                 int p0 = t * 4, np = min(4, total_pages - p0);
@@ -329,7 +354,8 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
     for (int sidx = blockIdx.x; sidx < Sg; sidx += C) {
         int item, g, seg, nseg, ui, t0, t1;
         locate(sidx, item, g, seg, nseg, ui, t0, t1);
-        int nkeys = nk_s[item];
+        int nkeys = item_nkeys(item);
+        if (packed) nq_act = item_npos(item) * p.G;  // rows: position-major, the G heads of each position
 
         // Query tile (16 rows x DH, fp32) into shared memory, then mma A fragments (bf16),
         // pre-scaled by log2(e)/sqrt(d_h).  Rows: G primary heads, then G coupled branch heads.
@@ -340,7 +366,7 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
                 int q = idx / (DH / 4), c4 = idx % (DH / 4);
                 float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (q < nq_act) {
-                    int row = (q / p.G) * Bc + item;
+                    int row = packed ? item_row0(item) + q / p.G : (q / p.G) * Bc + item;
                     int h = g * p.G + q % p.G;
                     v = __ldcg(reinterpret_cast<const float4 *>(p.Q + (size_t)row * q_dim + (size_t)h * DH) + c4);
                 }
@@ -521,12 +547,19 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
                     // mask, online softmax (base 2), pack P as the A operand of P V
                     int col = (lane & 3) * 2;
                     float rmax[2] = {-INFINITY, -INFINITY};
+                    // packed prompt tiles: the row of position pp sees the keys up to its own position only
+                    int vrow[2] = {valid, valid};
+                    if (packed) {
+                        const int npos = nq_act / p.G, rem = nkeys - (t * kAttTile + warp * 16);
+    #pragma unroll
+                        for (int h = 0; h < 2; h++) vrow[h] = min(16, rem - max(npos - 1 - ((lane >> 2) + 8 * h) / p.G, 0));
+                    }
     #pragma unroll
                     for (int nb = 0; nb < 2; nb++)
     #pragma unroll
                         for (int e = 0; e < 4; e++) {
                             int tk = nb * 8 + col + (e & 1);
-                            if (tk >= valid) sacc[nb][e] = -INFINITY;
+                            if (tk >= vrow[e >> 1]) sacc[nb][e] = -INFINITY;
                             rmax[e >> 1] = fmaxf(rmax[e >> 1], sacc[nb][e]);
                         }
                     float corr[2], msub[2];
@@ -637,7 +670,7 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
                         if (q < nq_act) {
                             if (nseg == 1) {
                                 // the pair's only segment: normalise and write the head's output
-                                int row = (q / p.G) * Bc + item;
+                                int row = packed ? item_row0(item) + q / p.G : (q / p.G) * Bc + item;
                                 int hq = g * p.G + q % p.G;
                                 size_t ob = (size_t)row * q_dim + (size_t)hq * DH;
                                 float inv = 1.f / l_run[h];
@@ -833,7 +866,7 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
                         int q = c + j;
                         if (q < nq_act) {
                             if (nseg == 1) {
-                                int row = (q / p.G) * Bc + item;
+                                int row = packed ? item_row0(item) + q / p.G : (q / p.G) * Bc + item;
                                 int hq = g * p.G + q % p.G;
                                 size_t ob = (size_t)row * q_dim + (size_t)hq * DH;
                                 float inv = 1.f / l_run[j];
@@ -921,7 +954,7 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
                 for (int a = 0; a < 2; a++) {
                     if (!act[a]) continue;
                     if (final) {
-                        int row = (qq[a] / p.G) * Bc + item;
+                        int row = packed ? item_row0(item) + qq[a] / p.G : (qq[a] / p.G) * Bc + item;
                         int h = g * p.G + qq[a] % p.G;
                         size_t o_idx = (size_t)row * q_dim + (size_t)h * DH + ee[a];
                         float x = X[a] / L[a];

@@ -107,7 +107,10 @@ __device__ __forceinline__ void row_scale2(const float *ss, int ss_tiles, int ss
 // coupling, M_2 += c*M_1 first (mode 2); the next GEMM's input is g * S (un-normalised, two bf16
 // planes) and each 256-column block leaves its share of sum(S^2) per row in ss_out[tile][row].
 // The consumer of that GEMM multiplies by 1/rms (the GEMM is linear), see row_scale.
-// grid (primary rows, d / 256): every thread owns one column of a row and of its branch twin.
+// grid (primary rows, d / 256, branches): every thread owns one column of a row and of its branch twin.
+// MULTI = false (at most one decode branch): the block index of the branch is a compile-time zero -- with it
+// a run-time value the compiler orders this kernel's loads worse and a launch takes 3.5 us longer.
+template <bool MULTI>
 __global__ void __launch_bounds__(256) resid_wide_kernel(float *S, const float *P, int nsplit, size_t split_stride,
                                                          int mode, const float *__restrict__ coup_c, int Bc, int grouped,
                                                          const float *__restrict__ g_next, int d, __nv_bfloat16 *Xb,
@@ -117,8 +120,8 @@ __global__ void __launch_bounds__(256) resid_wide_kernel(float *S, const float *
     DBT_TL_WAITED;
     __shared__ float scratch[64];
     int b = blockIdx.x, i = blockIdx.y * blockDim.x + threadIdx.x;
-    const bool first = blockIdx.z == 0;  // the first branch's blocks also own the primary row
-    const int r2 = ((int)blockIdx.z + 1) * Bc + b;
+    const bool first = MULTI ? blockIdx.z == 0 : true;  // the first branch's blocks also own the primary row
+    const int r2 = MULTI ? ((int)blockIdx.z + 1) * Bc + b : Bc + b;
     float q1 = 0.f, q2 = 0.f;
     if (i < d) {
         // every load of this thread goes out before the first use: S of both rows, the gain, the
@@ -485,6 +488,7 @@ __global__ void __launch_bounds__(256) moe_swiglu_kernel(const float *Pe, const 
 // Xn != nullptr (grid (Bc, ceil(d / 256)), 256 threads): the block also leaves the next layer's GEMM
 // input g_next * S (two bf16 planes, the 1/rms factor is applied after that GEMM) and its 256-column
 // share of sum(S^2) for both rows, as resid_wide_kernel does.
+template <bool MULTI>
 __global__ void __launch_bounds__(256) moe_combine_sorted_kernel(const float *Ys, const float *Psh, int nsplit,
                                                                  size_t split_stride, const int32_t *idx,
                                                                  const int32_t *pos, const float *wts, int kmax, int Bc,
@@ -501,8 +505,8 @@ __global__ void __launch_bounds__(256) moe_combine_sorted_kernel(const float *Ys
     // the row's selections (weights, sorted positions) once, then all expert rows of a column in
     // flight together; terms are added in slot order
     constexpr int KM = 16;
-    const bool first = blockIdx.z == 0;
-    const int r2 = ((int)blockIdx.z + 1) * Bc + b;
+    const bool first = MULTI ? blockIdx.z == 0 : true;
+    const int r2 = MULTI ? ((int)blockIdx.z + 1) * Bc + b : Bc + b;
     for (int i = blockIdx.y * blockDim.x + threadIdx.x; i < d; i += gridDim.y * blockDim.x) {
         float m1 = 0.f, m2 = 0.f;
         for (int j0 = 0; j0 < kmax; j0 += KM) {

@@ -55,6 +55,10 @@ struct TcParams {
     // grouped mode with row tiles: blockIdx.y = which N_TILE rows of the expert's list (CTAs past the
     // list's end leave at once); 0: the whole list fits one tile and blockIdx.y is the split as usual
     int grp_row_tiles;
+    // dense mode with more rows than one tile holds (prompt chunks): blockIdx.x = weight tile * row_tiles + row
+    // tile, so that the CTAs sharing a weight tile are neighbours in launch order and all but the first find it
+    // in L2; 0 or 1: blockIdx.x is the weight tile
+    int row_tiles;
     // test hook (dbt_op_gemm_tc only): 1 = CTA (0,0,0) never requests the weight tile of its first stage
     // and every wait gives up after kTestWaitCycles, so that the expired-wait path can be exercised:
     // the kernel records kStatusWaitExpired, skips its stores, frees its TMEM and returns
@@ -224,6 +228,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
     int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     int tile = blockIdx.x, split = p.grp_row_tiles ? 0 : blockIdx.y;
     int x_row0 = 0, w_row0 = 0, grp_n = -1;
+    if (p.row_tiles > 1) {
+        x_row0 = (int)(blockIdx.x % p.row_tiles) * N_TILE;
+        tile = blockIdx.x / p.row_tiles;
+    }
     if (p.grp_cnt) {
         // the expert's row list comes from the previous kernel: nothing can start before it is known
         pdl_wait();
@@ -354,7 +362,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
     if (!got && lane == 0) report(p.status, kStatusWaitExpired, 200 + warp);
     got = __syncthreads_and(got);  // the ring is idle from here on: its memory serves as scratch
     float *scratch = reinterpret_cast<float *>(gen_tiles);
-    int rows = grp_n >= 0 ? min(grp_n, N_TILE) : min(seg.rows, p.R);
+    int rows = grp_n >= 0 ? min(grp_n, N_TILE) : min(min(seg.rows, p.R) - x_row0, N_TILE);
     const bool stacked_acc = Cfg::kStackable && p.stacked;
     auto ld_acc = [&](int c0, float (&v)[16]) {  // 16 accumulator columns of this thread's feature
         uint32_t a[16], b[16];

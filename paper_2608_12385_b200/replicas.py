@@ -50,6 +50,15 @@ def sum_over_ranks(value: float, device: str = "cpu") -> float:
     return float(t.item())
 
 
+def all_agree(flag: bool, device: str = "cpu") -> bool:
+    """True when `flag` holds on every rank (a rank-uniform decision, e.g. when to leave a timing loop)."""
+    if not (dist.is_available() and dist.is_initialized()):
+        return bool(flag)
+    t = torch.tensor([1.0 if flag else 0.0], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MIN)
+    return bool(t.item() > 0.5)
+
+
 def aggregate_throughput(units_this_rank: float, ms_this_rank: float, device: str = "cpu") -> tuple[float, float]:
     """Whole-job throughput: units processed by all ranks / the slowest rank's time.
     Returns (units per second, max ms)."""

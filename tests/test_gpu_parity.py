@@ -66,6 +66,75 @@ def test_prefill_longer_than_one_chunk_and_page_boundaries():
     teacher_forced_compare(cfg, w, tok, n_prefill=300, grouped=True)
 
 
+@pytest.mark.parametrize("cfg,B,n", [
+    (small_bf16(n_layers=2), 2, 2100),                                    # three chunks of <= 1024 positions, 4 positions per query tile
+    (small_bf16(n_layers=2), 3, 700),                                     # ragged chunks (682 + 18) and tail tiles
+    (small_bf16(n_layers=1, n_q_heads=4, n_kv_heads=4), 1, 2500),         # MHA: 16 positions per tile, 2048 + 452
+    (small_bf16(n_layers=1, n_q_heads=2, n_kv_heads=1, head_dim=128, d_model=128, vocab=777), 5, 1000),  # 8 per tile
+    (small_bf16(n_layers=1, n_q_heads=8, n_kv_heads=1), 2, 333),          # 2 positions per tile
+])
+def test_long_prompt_prefill_matches_the_oracle(cfg, B, n):
+    """Section 4.4 item 1, prompt-wide prefill: prompts of up to 2500 positions go through in chunks of up to
+    2048 rows (GEMMs over several row tiles per weight tile, causal attention with 16 / G consecutive positions
+    per query tile).  Last-position logits and the whole cache against the oracle's position-by-position
+    primary pass, then two grouped steps on top of the device's own cache."""
+    w = make_weights(cfg, seed=51, matrix_std=0.05)
+    tok = make_tokens(cfg, B, n + 2, seed=52)
+    om = oracle.OracleModel(cfg, w, B, n + 2)
+    gm = make_gpu_model(cfg, w, B, n + 2)
+    want = om.prefill(tok[:, :n].numpy())
+    got = gm.prefill(tok[:, :n].cuda().contiguous(), want_logits=True)
+    assert_logits_close(got, want, "bf16", "prefill logits")
+    k_dev, v_dev = gm.export_kv(B, n)
+    np.testing.assert_allclose(k_dev.float().numpy(), om.k_cache[:, :B, :n], rtol=2.0 ** -8, atol=5e-3)
+    np.testing.assert_allclose(v_dev.float().numpy(), om.v_cache[:, :B, :n], rtol=2.0 ** -8, atol=5e-3)
+    for t in range(n, n + 2):
+        o = om.decode_step(tok[:, t].numpy())
+        g = gm.decode_full(tok[:, t].cuda().contiguous())
+        assert_logits_close(g["z1"], o["z1"], "bf16", f"step {t} z1")
+        assert_logits_close(g["z2"], o["z2"], "bf16", f"step {t} z2")
+    assert gm.sync_status() == (0, 0)
+
+
+def test_prefill_in_one_call_equals_prefill_in_pieces():
+    """The cache does not depend on how the prompt is cut into calls: 1500 positions at once (one chunk, six
+    row tiles) and as 700 + 800 give the same logits within tolerance and caches equal to bf16 rounding."""
+    cfg = small_bf16(n_layers=2)
+    w = make_weights(cfg, seed=53, matrix_std=0.05)
+    tok = make_tokens(cfg, 1, 1500, seed=54).cuda()
+    wd = binding.weights_to_device(w)
+    a, b = binding.Model(cfg, wd, 1, 1500), binding.Model(cfg, wd, 1, 1500)
+    za = a.prefill(tok.contiguous(), want_logits=True)
+    b.prefill(tok[:, :700].contiguous())
+    zb = b.prefill(tok[:, 700:].contiguous(), want_logits=True)
+    assert_logits_close(za, zb.cpu().numpy(), "bf16", "one call vs two")
+    ka, va = a.export_kv(1, 1500)
+    kb, vb = b.export_kv(1, 1500)
+    np.testing.assert_allclose(ka.float().numpy(), kb.float().numpy(), rtol=2.0 ** -7, atol=5e-3)
+    np.testing.assert_allclose(va.float().numpy(), vb.float().numpy(), rtol=2.0 ** -7, atol=5e-3)
+
+
+def test_1b_width_prompt_of_2100_positions_on_a_sampled_sequence():
+    """The 1B model's width (two of its layers, to keep the oracle's 2100 positions within a minute): three
+    sequences prefilled together on the device, sequence 1 checked against the oracle run on it alone."""
+    cfg = dense_1b().replace(n_layers=2)
+    w = make_weights(cfg, seed=0)
+    B, n, pick = 3, 2100, 1
+    tok = make_tokens(cfg, B, n + 1, seed=2)
+    gm = make_gpu_model(cfg, w, B, n + 1)
+    got = gm.prefill(tok[:, :n].cuda().contiguous(), want_logits=True)
+    om = oracle.OracleModel(cfg, w, 1, n + 1)
+    want = om.prefill(tok[pick:pick + 1, :n].numpy())
+    assert_logits_close(got[pick:pick + 1], want, "bf16", "1B-width prefill logits")
+    k_dev, v_dev = gm.export_kv(1, n, seq_ids=[pick])
+    np.testing.assert_allclose(k_dev.float().numpy(), om.k_cache[:, :1, :n], rtol=2.0 ** -8, atol=5e-3)
+    np.testing.assert_allclose(v_dev.float().numpy(), om.v_cache[:, :1, :n], rtol=2.0 ** -8, atol=5e-3)
+    o = om.decode_step(tok[pick:pick + 1, n].numpy())
+    g = gm.decode_full(tok[:, n].cuda().contiguous())
+    assert_logits_close(g["z1"][pick:pick + 1], o["z1"], "bf16", "step after prefill z1")
+    assert_logits_close(g["z2"][pick:pick + 1], o["z2"], "bf16", "step after prefill z2")
+
+
 @pytest.mark.parametrize("ctx", [0, 1, 15, 16, 17, 63, 64, 65, 255, 256, 257, 2047, 4100, 8200])
 def test_context_lengths_around_page_and_chunk_boundaries(ctx):
     """Synthetic cache of `ctx` positions, then two grouped steps."""
