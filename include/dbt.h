@@ -142,6 +142,18 @@ int32_t dbt_seq_len(const dbt_model *m, int32_t b);
 dbt_status dbt_prefill(dbt_model *m, const int32_t *tokens_dev, int32_t B, int32_t n,
                        float *last_primary_logits_dev);
 
+/* Section 4.4 items 1 and 2 in one call: the primary path alone processes the whole prompt x_1..x_S
+ * (tokens_dev DEVICE int32 [B][S], sequences 0..B-1 from their current lengths), and the continuation boundary
+ * -- one branch evaluation at the final prompt token, coupled to the primary's Q_1, H_1, M_1 of that position
+ * and read against the completed cache -- predicts x_{S+1} from the mixture.  Outputs as dbt_decode_step.
+ * How it runs: positions 1..S-1 as the prompt-wide prefill, position S as one grouped step.  The boundary
+ * evaluation has to stream every shared matrix once for the branch row anyway; letting the primary row of
+ * position S ride in that same pass produces the "retained intermediates" where they are consumed, costs no
+ * extra memory traffic and needs no per-layer retention buffers.  The values are those of the paper's form
+ * (prefill all S positions, then a branch-only evaluation).  Lengths advance by S. */
+dbt_status dbt_prefill_boundary(dbt_model *m, const int32_t *tokens_dev, int32_t B, int32_t S, int32_t *next_tokens_dev,
+                                float *logits_primary_dev, float *logits_branch_dev, float *alpha_dev);
+
 /* Section 4.4 items 2-3, one grouped step ("Decode" paragraph): for each sequence b the token
  * tokens_dev[b] at position t_b = its length; the primary appends K_1,V_1[t_b]; both paths'
  * queries read positions 0..t_b of the primary cache; the shared matrices are applied to

@@ -24,7 +24,7 @@ EXPORTS = ["dbt_query_sizes", "dbt_create", "dbt_destroy", "dbt_set_page_table",
            "dbt_seq_len", "dbt_prefill", "dbt_decode_step", "dbt_decode_step_primary_only", "dbt_decode_step_host",
            "dbt_decode_step_primary_only_host", "dbt_last_experts", "dbt_last_expert_union", "dbt_sync_status",
            "dbt_launch_count", "dbt_last_error", "dbt_version", "dbt_profile_begin", "dbt_profile_end", "dbt_op_gemm_tc",
-           "dbt_op_gemm_tc_static", "dbt_kv_export", "dbt_kv_import"]
+           "dbt_op_gemm_tc_static", "dbt_kv_export", "dbt_kv_import", "dbt_prefill_boundary"]
 
 
 class DbtError(RuntimeError):
@@ -84,6 +84,7 @@ def load_library():
     L.dbt_seq_len.restype = i32
     L.dbt_prefill.argtypes = [vp, vp, i32, i32, vp]
     L.dbt_decode_step.argtypes = [vp, vp, i32, vp, vp, vp, vp]
+    L.dbt_prefill_boundary.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp]
     L.dbt_decode_step_primary_only.argtypes = [vp, vp, i32, vp, vp]
     L.dbt_decode_step_host.argtypes = [vp, vp, i32, vp, vp]
     L.dbt_decode_step_primary_only_host.argtypes = [vp, vp, i32, vp]
@@ -274,6 +275,19 @@ class Model:
         B, n = tokens_dev.shape
         out = torch.empty(B, self.cfg.vocab, dtype=torch.float32, device=self.device) if want_logits else None
         self._check(self.L.dbt_prefill(self._h, tokens_dev.data_ptr(), B, n, _p(out)))
+        return out
+
+    def prefill_boundary(self, tokens_dev: torch.Tensor) -> dict:
+        """The whole prompt [B, S] and the boundary evaluation at its last token (Section 4.4 items 1-2)."""
+        assert tokens_dev.dtype == torch.int32 and tokens_dev.is_cuda and tokens_dev.is_contiguous()
+        B, S = tokens_dev.shape
+        V, K = self.cfg.vocab, self.cfg.n_paths
+        out = {"next": torch.empty(B, dtype=torch.int32, device=self.device),
+               "z1": torch.empty(B, V, dtype=torch.float32, device=self.device),
+               "z2": torch.empty((B, V) if K == 2 else (K - 1, B, V), dtype=torch.float32, device=self.device),
+               "alpha": torch.empty(B, dtype=torch.float32, device=self.device)}
+        self._check(self.L.dbt_prefill_boundary(self._h, tokens_dev.data_ptr(), B, S, _p(out["next"]), _p(out["z1"]),
+                                                _p(out["z2"]), _p(out["alpha"])))
         return out
 
     def decode_step(self, tokens_dev: torch.Tensor, next_dev: torch.Tensor | None = None, z1=None, z2=None,

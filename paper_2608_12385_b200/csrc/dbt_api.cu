@@ -116,6 +116,8 @@ struct dbt_model {
     int moe_row_tile;  // DBT_MOE_ROWTILE: row tile of the per-expert GEMMs (-1: chosen from the batch, 0: one tile of all rows)
     bool moe_wide;  // MoE chain with the RMSNorm factor applied behind the GEMMs (tensor-core MoE path)
     std::vector<GraphEntry> graphs;
+    // where a decode step finds sequence b's token: tokens[b * tok_stride + tok_p0] (1, 0 except inside dbt_prefill_boundary)
+    int tok_stride = 1, tok_p0 = 0;
 };
 
 namespace {
@@ -744,6 +746,15 @@ dbt_status run_attention_mma(dbt_model *m, const RowMap &rm, int grouped, int la
     }
     if (!packed && items > kAttMaxItems) return fail(m, DBT_ERR_CAPACITY, "attention rows %d exceed %d", items, kAttMaxItems);
     dim3 grid(2 * m->num_sms);  // two resident CTAs per SM; each takes an equal share of all K/V tiles
+    // When the (sequence, KV head) pairs fill one wave of SMs, every pair goes to one CTA with a ring twice as deep,
+    // one CTA per SM: no pair is split, so there are no partials to write, no tickets and no merge.  Chosen from
+    // the batch and the model, never from the mode or the lengths (a captured step serves every length).
+    const int pairs = items * c.n_kv_heads;
+    if (!packed && paths_of(c) * G <= 8 && 2 * pairs > m->num_sms && pairs <= m->num_sms) {
+        dim3 g1(m->num_sms);
+        LAUNCH(m, "attention", kv_bytes, (attn_mma_kernel<DH, true, true>), g1, 160, (AttCfg<DH, true>::kSmemBytes), m->map_kv, p);
+        return DBT_OK;
+    }
     // up to 8 query rows per KV head over both paths: the transposed-product variant (fixed per
     // model, so that grouped and primary-only steps run the same arithmetic on the primary rows)
     if (paths_of(c) * G <= 8 && !packed)
@@ -1004,7 +1015,7 @@ dbt_status step_tc(dbt_model *m, const int32_t *tokens_dev, int B, int grouped, 
     int R = npaths(grouped) * B;
     int n_tile = pad_rows(paths_of(c) * B);  // the same instruction shape in both modes
     dbt_status st;
-    LAUNCH(m, "embed", 0, embed_norm_kernel<WT>, R, 256, 0, tokens_dev, 1, 0, rm, (const WT *)m->w.embed_primary,
+    LAUNCH(m, "embed", 0, embed_norm_kernel<WT>, R, 256, 0, tokens_dev, m->tok_stride, m->tok_p0, rm, (const WT *)m->w.embed_primary,
            (const WT *)m->w.embed_branch, m->w.embed_norm_g, c.rms_eps, c.d_model, c.vocab, w.S, w.status);
     int mode, nsp;
     size_t sstride;
@@ -1032,7 +1043,7 @@ dbt_status prefill_tc(dbt_model *m, const int32_t *tokens_dev, int B, int n, flo
         int cn = n - p0 < cn_max ? n - p0 : cn_max;
         RowMap rm{B, cn};
         int R = B * cn, n_tile = pad_rows(R);
-        LAUNCH(m, "embed", 0, embed_norm_kernel<WT>, R, 256, 0, tokens_dev, n, p0, rm, (const WT *)m->w.embed_primary,
+        LAUNCH(m, "embed", 0, embed_norm_kernel<WT>, R, 256, 0, tokens_dev, m->tok_stride > 1 ? m->tok_stride : n, p0, rm, (const WT *)m->w.embed_primary,
                (const WT *)m->w.embed_branch, m->w.embed_norm_g, c.rms_eps, c.d_model, c.vocab, w.S, w.status);
         int mode, nsp;
         size_t sstride;
@@ -1165,7 +1176,7 @@ dbt_status step_wide(dbt_model *m, const int32_t *tokens_dev, int B, int grouped
     RowMap rm{B, 1};
     int R = npaths(grouped) * B, n_tile = pad_rows(paths_of(c) * B);
     dbt_status st;
-    if ((st = run_embed_wide<WT>(m, tokens_dev, 1, 0, rm, R, n_tile)) != DBT_OK) return st;
+    if ((st = run_embed_wide<WT>(m, tokens_dev, m->tok_stride, m->tok_p0, rm, R, n_tile)) != DBT_OK) return st;
     if ((st = run_layers_wide(m, rm, grouped, n_tile)) != DBT_OK) return st;
     if ((st = run_head_wide(m, rm, grouped, n_tile)) != DBT_OK) return st;
     // the readout also bumps the sequence lengths: nothing after it in the step reads them
@@ -1192,7 +1203,7 @@ dbt_status prefill_wide(dbt_model *m, const int32_t *tokens_dev, int B, int n, f
         int cn = p0 < n_bulk ? (n_bulk - p0 < cn_max ? n_bulk - p0 : cn_max) : 1;
         RowMap rm{B, cn};
         int R = B * cn, n_tile = pad_rows(R < 256 ? R : 256);
-        if ((st = run_embed_wide<WT>(m, tokens_dev, n, p0, rm, R, n_tile)) != DBT_OK) return st;
+        if ((st = run_embed_wide<WT>(m, tokens_dev, m->tok_stride > 1 ? m->tok_stride : n, p0, rm, R, n_tile)) != DBT_OK) return st;
         if ((st = run_layers_wide(m, rm, 0, n_tile)) != DBT_OK) return st;
         if (last_logits && p0 + cn >= n) {
             if ((st = run_head_wide(m, rm, 0, n_tile)) != DBT_OK) return st;
@@ -1277,6 +1288,10 @@ bool setup_tc(dbt_model *m) {
     m->att_fast = ok && !(fa && strcmp(fa, "simt") == 0) &&
                   make_kv_page_map(&m->map_kv, m->kv_pool, (uint64_t)c.n_layers * 2 * c.num_pages * c.n_kv_heads * c.page_size,
                                    (uint64_t)c.num_pages * c.n_kv_heads * c.page_size, c.head_dim) &&
+                  cudaFuncSetAttribute(attn_mma_kernel<128, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       AttCfg<128, true>::kSmemBytes) == cudaSuccess &&
+                  cudaFuncSetAttribute(attn_mma_kernel<64, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       AttCfg<64, true>::kSmemBytes) == cudaSuccess &&
                   cudaFuncSetAttribute(attn_mma_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        AttCfg<128>::kSmemBytes) == cudaSuccess &&
                   cudaFuncSetAttribute(attn_mma_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -1300,7 +1315,7 @@ dbt_status step_impl(dbt_model *m, const int32_t *tokens_dev, int B, int grouped
     RowMap rm{B, 1};
     int R = npaths(grouped) * B;
     dbt_status st;
-    LAUNCH(m, "embed", 0, embed_norm_kernel<WT>, R, 256, 0, tokens_dev, 1, 0, rm, (const WT *)m->w.embed_primary,
+    LAUNCH(m, "embed", 0, embed_norm_kernel<WT>, R, 256, 0, tokens_dev, m->tok_stride, m->tok_p0, rm, (const WT *)m->w.embed_primary,
            (const WT *)m->w.embed_branch, m->w.embed_norm_g, c.rms_eps, c.d_model, c.vocab, w.S, w.status);
     if ((st = run_layers<WT>(m, rm, grouped, true)) != DBT_OK) return st;
     if ((st = run_head<WT>(m, R, 1, 0)) != DBT_OK) return st;
@@ -1326,7 +1341,7 @@ dbt_status prefill_impl(dbt_model *m, const int32_t *tokens_dev, int B, int n, f
         int cn = n - p0 < cn_max ? n - p0 : cn_max;
         RowMap rm{B, cn};
         int R = B * cn;
-        LAUNCH(m, "embed", 0, embed_norm_kernel<WT>, R, 256, 0, tokens_dev, n, p0, rm, (const WT *)m->w.embed_primary,
+        LAUNCH(m, "embed", 0, embed_norm_kernel<WT>, R, 256, 0, tokens_dev, m->tok_stride > 1 ? m->tok_stride : n, p0, rm, (const WT *)m->w.embed_primary,
                (const WT *)m->w.embed_branch, m->w.embed_norm_g, c.rms_eps, c.d_model, c.vocab, w.S, w.status);
         if ((st = run_layers<WT>(m, rm, 0, false)) != DBT_OK) return st;
         bool last = p0 + cn >= n;
@@ -1706,6 +1721,30 @@ dbt_status dbt_decode_step(dbt_model *m, const int32_t *tokens_dev, int32_t B, i
     dbt_status st = check_step_args(m, tokens_dev, B, 1);
     if (st != DBT_OK) return st;
     return step_graphed(m, tokens_dev, B, paths_of(m->cfg), next_tokens_dev, logits_primary_dev, logits_branch_dev, alpha_dev);
+}
+
+dbt_status dbt_prefill_boundary(dbt_model *m, const int32_t *tokens_dev, int32_t B, int32_t S, int32_t *next_tokens_dev,
+                                float *logits_primary_dev, float *logits_branch_dev, float *alpha_dev) {
+    dbt_status st = check_step_args(m, tokens_dev, B, S);
+    if (st != DBT_OK) return st;
+    if (S > 1) {
+        // positions 1..S-1 of every row of tokens_dev [B][S]: the prompt-wide prefill walks rows of stride S
+        m->tok_stride = S;
+        st = m->cfg.weight_dtype == DBT_DTYPE_F32 ? prefill_impl<float>(m, tokens_dev, B, S - 1, nullptr)
+             : m->wide                             ? prefill_wide(m, tokens_dev, B, S - 1, nullptr)
+             : m->tc                               ? prefill_tc(m, tokens_dev, B, S - 1, nullptr)
+                                                   : prefill_impl<__nv_bfloat16>(m, tokens_dev, B, S - 1, nullptr);
+        m->tok_stride = 1;
+        if (st != DBT_OK) return st;
+    }
+    // position S: the primary's step and the branch's boundary evaluation in one grouped pass (launched
+    // directly: the token addressing differs from a decode step's, so the captured graphs do not apply)
+    m->tok_stride = S;
+    m->tok_p0 = S - 1;
+    st = step_direct(m, tokens_dev, B, paths_of(m->cfg), next_tokens_dev, logits_primary_dev, logits_branch_dev, alpha_dev);
+    m->tok_stride = 1;
+    m->tok_p0 = 0;
+    return st;
 }
 
 dbt_status dbt_decode_step_primary_only(dbt_model *m, const int32_t *tokens_dev, int32_t B, int32_t *next_tokens_dev,

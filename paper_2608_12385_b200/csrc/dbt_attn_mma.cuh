@@ -75,12 +75,15 @@ constexpr int kAttSingle = 16;     // up to this many segments, one CTA merges t
 constexpr int kAttMaxGroups = kAttMaxSeg / kAttGroup;
 constexpr float kLog2e = 1.4426950408889634f;
 
-template <int DH>
+// DEEP: one CTA per SM with a ring twice as deep instead of two CTAs per SM: the same bytes in flight per SM,
+// half as many segments (fewer query builds, partials and merges).  (A second group of four consumer warps
+// taking alternate stages of the deep ring was measured 1 % slower: the stream, not the consumers, sets the pace.)
+template <int DH, bool DEEP = false>
 struct AttCfg {
     static constexpr int kHalves = DH / 64;                 // 128-byte column groups per row
     static constexpr int kPageBytes = 16 * DH * 2;          // one page of K (or V) for one head
     static constexpr int kStageBytes = 2 * 4 * kPageBytes;  // K + V, 4 pages
-    static constexpr int kStages = DH == 128 ? 3 : 6;       // 96 KB ring: two CTAs keep ~190 KB in flight per SM
+    static constexpr int kStages = (DH == 128 ? 3 : 6) * (DEEP ? 2 : 1);  // 96 KB ring: two CTAs keep ~190 KB in flight per SM
     // scratch: one [16][DH + 8] fp32 slot (Q tile / warp fold; the padding keeps the fold's
     // fragment-shaped accesses off a single bank), m, l, flag, row tables
     static constexpr int kFoldStride = DH + 8;
@@ -131,9 +134,9 @@ __device__ __forceinline__ void tma_load_4d_hint(uint32_t dst, const CUtensorMap
 }
 __device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
-template <int DH, bool NARROW>
-__global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant__ CUtensorMap tmKV, AttnParams p) {
-    using Cfg = AttCfg<DH>;
+template <int DH, bool NARROW, bool DEEP = false>
+__global__ void __launch_bounds__(160, DEEP ? 1 : 2) attn_mma_kernel(const __grid_constant__ CUtensorMap tmKV, AttnParams p) {
+    using Cfg = AttCfg<DH, DEEP>;
     constexpr int STAGES = Cfg::kStages, HALVES = Cfg::kHalves, KS = DH / 16, NB = DH / 8;
     extern __shared__ uint8_t smem_raw[];
     uint32_t raw = smem_u32(smem_raw);
@@ -301,17 +304,24 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
             int item, g, seg, n, ui, t0, t1;
             locate(sidx, item, g, seg, n, ui, t0, t1);
             int seq = item_seq(item), total_pages = (item_nkeys(item) + 15) >> 4;
+            // page ids 32 at a time (eight stages' worth, one coalesced load): a lookup per stage would put an
+            // L2 round trip on every stage of this loop and cap a CTA at one stage per ~0.7 us
+            int pt_base = -(1 << 30), my_page = 0;
             for (int t = t0; t < t1; t++, it++) {
                 int s = it % STAGES;
                 int p0 = t * 4, np = min(4, total_pages - p0);
+                if (p0 + 4 > pt_base + 32) {
+                    pt_base = p0;
+                    my_page = p0 + lane < total_pages ? __ldg(p.page_table + (size_t)seq * p.pt_stride + p0 + lane) : 0;
+                }
                 if (lane == 0) {
                     if (it >= STAGES) ok = mbar_wait(empty_bar(s), ((it / STAGES) - 1) & 1);
                     if (ok) mbar_expect_tx(full_bar(s), (uint32_t)np * 2 * Cfg::kPageBytes);
                 }
                 ok = __shfl_sync(0xffffffffu, ok, 0);
                 if (!ok) break;
+                int page = __shfl_sync(0xffffffffu, my_page, (p0 - pt_base + lane) & 31);
                 if (lane < np) {
-                    int page = __ldg(p.page_table + (size_t)seq * p.pt_stride + p0 + lane);
                     if (page < 0 || page >= p.num_pages) {
                         report(p.status, kStatusBadPage, page);
                         page = 0;
@@ -326,7 +336,9 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
                 }
                 // After the first stage the stream pauses until the consumers have their queries: their
                 // few small loads would otherwise queue behind hundreds of CTAs' page traffic for several
-                // microseconds, and nothing can be consumed before they return anyway.
+                // microseconds, and nothing can be consumed before they return anyway.  (Letting the ring fill
+                // at once instead, with the small loads issued first, was measured slower: the queries are ready
+                // 0.8 us sooner but the stream then runs 10 % slower.)
                 if (it == 0) asm volatile("bar.sync 2, 160;" ::: "memory");
             }
         }
@@ -1009,7 +1021,16 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(const __grid_constant_
         }
         if (sidx == (int)blockIdx.x) DBT_TL_MARK(2);
     }
-    DBT_TL_END_IF(blockIdx.x == 0 || blockIdx.x == 99 || blockIdx.x == 200 || blockIdx.x == 281, blockIdx.x == 0 ? "attentio" : blockIdx.x == 99 ? "att99" : blockIdx.x == 200 ? "att200" : "att281");
+#ifdef DBT_TL_ATT_ALL
+    {  // every CTA leaves a record: mark 3 carries (SM id << 16 | block index)
+        unsigned smid;
+        asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+        tlx_[3] = ((unsigned long long)smid << 16) | blockIdx.x;
+    }
+    DBT_TL_END_IF(true, "attall");
+#else
+    DBT_TL_END("attentio");
+#endif
 }
 
 // The K/V pool as a 4-D bf16 tensor (64 columns, 64-column piece of a row, row, K|V plane of a

@@ -96,6 +96,37 @@ def test_long_prompt_prefill_matches_the_oracle(cfg, B, n):
     assert gm.sync_status() == (0, 0)
 
 
+@pytest.mark.parametrize("cfg", [small_bf16(n_layers=2), tiny_dense_fp32().replace(n_layers=2), small_moe(),
+                                 small_bf16(n_layers=2, n_paths=3)])
+def test_prefill_boundary_is_prefill_of_all_but_one_plus_the_grouped_step(cfg):
+    """Section 4.4 items 1-2 in one call: the same bits as dbt_prefill over x_1..x_{S-1} followed by
+    dbt_decode_step on x_S, the same cache, and (dense models) the oracle's values for that boundary."""
+    w = make_weights(cfg, seed=61, matrix_std=0.05)
+    B, S = 3, 37
+    tok = make_tokens(cfg, B, S + 1, seed=62)
+    wd = binding.weights_to_device(w)
+    a, b = binding.Model(cfg, wd, B, S + 1), binding.Model(cfg, wd, B, S + 1)
+    ga = a.prefill_boundary(tok[:, :S].cuda().contiguous())
+    b.prefill(tok[:, :S - 1].cuda().contiguous())
+    gb = b.decode_full(tok[:, S - 1].cuda().contiguous())
+    for k in ("next", "z1", "z2", "alpha"):
+        assert torch.equal(ga[k], gb[k]), k
+    assert [a.seq_len(i) for i in range(B)] == [S] * B
+    ka, va = a.export_kv(B, S)
+    kb, vb = b.export_kv(B, S)
+    assert torch.equal(ka.float(), kb.float()) and torch.equal(va.float(), vb.float())
+    if not cfg.is_moe:
+        om = oracle.OracleModel(cfg, w, B, S + 1)
+        om.prefill(tok[:, :S - 1].numpy(), want_logits=False)
+        o = om.decode_step(tok[:, S - 1].numpy())
+        assert_logits_close(ga["z1"], o["z1"], cfg.weight_dtype, "boundary z1")
+        assert_logits_close(ga["z2"], o["z2"], cfg.weight_dtype, "boundary z2")
+    # and the next step continues from there on both handles alike
+    ga2 = a.decode_full(tok[:, S].cuda().contiguous())
+    gb2 = b.decode_full(tok[:, S].cuda().contiguous())
+    assert torch.equal(ga2["z1"], gb2["z1"]) and torch.equal(ga2["z2"], gb2["z2"])
+
+
 def test_prefill_in_one_call_equals_prefill_in_pieces():
     """The cache does not depend on how the prompt is cut into calls: 1500 positions at once (one chunk, six
     row tiles) and as 700 + 800 give the same logits within tolerance and caches equal to bf16 rounding."""
