@@ -33,6 +33,7 @@ struct Workspace {
     int32_t *seq_len, *page_table, *status, *tokens_stage, *next_stage, *att_tickets, *att_tickets2, *gemm_tickets;
     float *alpha_stage;
     char *kv_stage;  // staging for dbt_kv_export / dbt_kv_import (kKvStageBytes)
+    int32_t *att_plan;  // a decode step's attention work split (attn_plan_kernel), kAttPlanInts
     // MoE
     float *rlogits, *rwts, *Hexp, *Yexp, *Msh, *Hsh;
     int32_t *ridx, *ecnt, *elist, *last_experts, *union_cnt;
@@ -118,6 +119,7 @@ struct dbt_model {
     std::vector<GraphEntry> graphs;
     // where a decode step finds sequence b's token: tokens[b * tok_stride + tok_p0] (1, 0 except inside dbt_prefill_boundary)
     int tok_stride = 1, tok_p0 = 0;
+    bool att_planned = false;  // inside a decode step whose attention work split has been computed (run_attention_plan)
 };
 
 namespace {
@@ -221,6 +223,7 @@ size_t carve(const dbt_config &c, char *base, Workspace *ws, int *Rmax_out, int 
     w.next_stage = k.take<int32_t>(c.max_batch);
     w.alpha_stage = k.take<float>(c.max_batch);
     w.kv_stage = k.take<char>(kKvStageBytes);
+    w.att_plan = k.take<int32_t>(kAttPlanInts);
     if (moe) {
         int km = kmax_of(c);
         w.rlogits = k.take<float>((size_t)Rmax * c.n_experts);
@@ -698,9 +701,29 @@ struct QkvFuse {
     const float *coup_a;
 };
 
+// One deep-ring CTA per SM instead of two CTAs per SM: when the (sequence, KV head) pairs fill one wave of SMs,
+// every pair goes to one CTA, so no pair is split and there are no partials to write, no tickets and no merge.
+// Chosen from the batch and the model, never from the mode or the lengths (a captured step serves every length).
+bool attn_deep(const dbt_model *m, int items) {
+    const dbt_config &c = m->cfg;
+    const int pairs = items * c.n_kv_heads, G = c.n_q_heads / c.n_kv_heads;
+    return paths_of(c) * G <= 8 && 2 * pairs > m->num_sms && pairs <= m->num_sms;
+}
+
+// The attention work split of a decode step, once for all its layers.
+dbt_status run_attention_plan(dbt_model *m, const RowMap &rm) {
+    const dbt_config &c = m->cfg;
+    const int items = rm.B * rm.cn;
+    if (items > kAttMaxItems) return DBT_OK;  // (the attention launch reports the capacity error)
+    LAUNCH(m, "attn_plan", 0, attn_plan_kernel, 1, 32, 0, rm, m->ws.seq_len, c.n_kv_heads,
+           attn_deep(m, items) ? m->num_sms : 2 * m->num_sms, m->ws.att_plan);
+    m->att_planned = true;  // cleared by the step function when its layers have been enqueued
+    return DBT_OK;
+}
+
 template <int DH>
 dbt_status run_attention_mma(dbt_model *m, const RowMap &rm, int grouped, int layer, double kv_bytes,
-                             const QkvFuse *qf = nullptr, bool pack_prompt = false) {
+                             const QkvFuse *qf = nullptr, bool pack_prompt = false, bool planned = false) {
     const dbt_config &c = m->cfg;
     const Workspace &w = m->ws;
     int items = rm.B * rm.cn, G = c.n_q_heads / c.n_kv_heads;
@@ -744,13 +767,13 @@ dbt_status run_attention_mma(dbt_model *m, const RowMap &rm, int grouped, int la
         p.cn = rm.cn;
         p.nbk = (rm.cn + p.pack - 1) / p.pack;
     }
+    if (planned && !packed) {  // from the second layer on the plan may be read before the dependency wait
+        p.plan = m->ws.att_plan;
+        p.plan_prewait = layer > 0 ? 1 : 0;
+    }
     if (!packed && items > kAttMaxItems) return fail(m, DBT_ERR_CAPACITY, "attention rows %d exceed %d", items, kAttMaxItems);
     dim3 grid(2 * m->num_sms);  // two resident CTAs per SM; each takes an equal share of all K/V tiles
-    // When the (sequence, KV head) pairs fill one wave of SMs, every pair goes to one CTA with a ring twice as deep,
-    // one CTA per SM: no pair is split, so there are no partials to write, no tickets and no merge.  Chosen from
-    // the batch and the model, never from the mode or the lengths (a captured step serves every length).
-    const int pairs = items * c.n_kv_heads;
-    if (!packed && paths_of(c) * G <= 8 && 2 * pairs > m->num_sms && pairs <= m->num_sms) {
+    if (!packed && attn_deep(m, items)) {
         dim3 g1(m->num_sms);
         LAUNCH(m, "attention", kv_bytes, (attn_mma_kernel<DH, true, true>), g1, 160, (AttCfg<DH, true>::kSmemBytes), m->map_kv, p);
         return DBT_OK;
@@ -941,8 +964,8 @@ dbt_status run_layers_tc(dbt_model *m, const RowMap &rm, int grouped, int n_tile
                    c.page_size, kpool, vpool, w.status, mwide ? (const float *)w.ss : (const float *)nullptr, mwide ? mss_tiles : 0,
                    mwide ? m->Rmax : 0, d, c.rms_eps);
         if (m->att_fast)
-            st = c.head_dim == 128 ? run_attention_mma<128>(m, rm, ga, l, kv_bytes, fuse ? &qf : nullptr)
-                                   : run_attention_mma<64>(m, rm, ga, l, kv_bytes, fuse ? &qf : nullptr);
+            st = c.head_dim == 128 ? run_attention_mma<128>(m, rm, ga, l, kv_bytes, fuse ? &qf : nullptr, false, m->att_planned)
+                                   : run_attention_mma<64>(m, rm, ga, l, kv_bytes, fuse ? &qf : nullptr, false, m->att_planned);
         else if (c.head_dim == 128)
             st = run_attention<WT, 128>(m, rm, ga, kpool, vpool, att_split, kv_bytes, true);
         else
@@ -1015,11 +1038,14 @@ dbt_status step_tc(dbt_model *m, const int32_t *tokens_dev, int B, int grouped, 
     int R = npaths(grouped) * B;
     int n_tile = pad_rows(paths_of(c) * B);  // the same instruction shape in both modes
     dbt_status st;
+    if (m->att_fast && (st = run_attention_plan(m, rm)) != DBT_OK) return st;
     LAUNCH(m, "embed", 0, embed_norm_kernel<WT>, R, 256, 0, tokens_dev, m->tok_stride, m->tok_p0, rm, (const WT *)m->w.embed_primary,
            (const WT *)m->w.embed_branch, m->w.embed_norm_g, c.rms_eps, c.d_model, c.vocab, w.S, w.status);
     int mode, nsp;
     size_t sstride;
-    if ((st = run_layers_tc(m, rm, grouped, n_tile, true, &mode, &nsp, &sstride)) != DBT_OK) return st;
+    st = run_layers_tc(m, rm, grouped, n_tile, true, &mode, &nsp, &sstride);
+    m->att_planned = false;
+    if (st != DBT_OK) return st;
     if ((st = run_head_tc(m, B, grouped, B, 1, 0, n_tile, mode, nsp, sstride)) != DBT_OK) return st;
     // the readout also bumps the sequence lengths: nothing after it in the step reads them
     if ((st = run_readout(m, B, grouped, next_dev, alpha_dev)) != DBT_OK) return st;
@@ -1106,8 +1132,8 @@ dbt_status run_layers_wide(dbt_model *m, const RowMap &rm, int grouped, int n_ti
                    w.Q, rm, grouped, c.n_q_heads, c.n_kv_heads, c.head_dim, lw.coup_a, w.rope, w.seq_len, w.page_table,
                    m->pages_per_seq_max, c.num_pages, c.page_size, kpool, vpool, w.status, (const float *)w.ss, ss_tiles, ss_ld, d,
                    c.rms_eps);
-        st = c.head_dim == 128 ? run_attention_mma<128>(m, rm, grouped, l, kv_bytes, fuse ? &qf : nullptr, true)
-                               : run_attention_mma<64>(m, rm, grouped, l, kv_bytes, fuse ? &qf : nullptr, true);
+        st = c.head_dim == 128 ? run_attention_mma<128>(m, rm, grouped, l, kv_bytes, fuse ? &qf : nullptr, true, m->att_planned)
+                               : run_attention_mma<64>(m, rm, grouped, l, kv_bytes, fuse ? &qf : nullptr, true, m->att_planned);
         if (st != DBT_OK) return st;
         TcCall op = call("gemm_o", &m->map_Ob, qd);
         op.W[0] = &mp.wo; op.n_out[0] = d; op.rows[0] = R; op.nseg = 1;
@@ -1176,8 +1202,11 @@ dbt_status step_wide(dbt_model *m, const int32_t *tokens_dev, int B, int grouped
     RowMap rm{B, 1};
     int R = npaths(grouped) * B, n_tile = pad_rows(paths_of(c) * B);
     dbt_status st;
+    if ((st = run_attention_plan(m, rm)) != DBT_OK) return st;
     if ((st = run_embed_wide<WT>(m, tokens_dev, m->tok_stride, m->tok_p0, rm, R, n_tile)) != DBT_OK) return st;
-    if ((st = run_layers_wide(m, rm, grouped, n_tile)) != DBT_OK) return st;
+    st = run_layers_wide(m, rm, grouped, n_tile);
+    m->att_planned = false;
+    if (st != DBT_OK) return st;
     if ((st = run_head_wide(m, rm, grouped, n_tile)) != DBT_OK) return st;
     // the readout also bumps the sequence lengths: nothing after it in the step reads them
     if ((st = run_readout(m, B, grouped, next_dev, alpha_dev)) != DBT_OK) return st;

@@ -63,6 +63,8 @@ struct AttnParams {
     // limit; a chunk holds cn positions per sequence, nbk = ceil(cn / pack) tiles per sequence, one CTA pass per
     // (tile, KV head) over all its keys, no split.  Q rows and output rows are seq * cn + position.
     int pack, cn, nbk;
+    const int *plan;   // the step's precomputed work split (attn_plan_kernel), or nullptr
+    int plan_prewait;  // the plan may be read before the dependency wait
 };
 
 constexpr int kAttTile = 64;       // tokens per pipeline stage (4 pages)
@@ -134,6 +136,97 @@ __device__ __forceinline__ void tma_load_4d_hint(uint32_t dst, const CUtensorMap
 }
 __device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
+// The work split of one attention launch, computed by one warp from the sequence lengths: cum[i] = stages of the
+// rows before row i, nk[i] = keys visible to row i, segcum[i] = segments (per KV head) of the rows before row i.
+// The same for every layer of a decode step, so a step computes it once (attn_plan_kernel) and the attention
+// launches copy it; launches without a plan (prompt chunks) compute it themselves.
+__device__ __forceinline__ void att_plan_warp(int lane, int items, RowMap rm, const int32_t *seq_len, int n_kv, int C0_arg,
+                                              int *cum, int *nk_s, int *segcum) {
+    int running = 0, longest = 0;
+    if (lane == 0) cum[0] = 0;
+    for (int base = 0; base < items; base += 32) {
+        int i = base + lane, nk = 0, u = 0;
+        if (i < items) {
+            nk = ld_mut(seq_len + rm.seq(i)) + rm.off(i) + 1;
+            u = (nk + kAttTile - 1) / kAttTile;
+            nk_s[i] = nk;
+        }
+        int incl = u, mx = u;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            int t = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += t;
+            mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        }
+        longest = max(longest, mx);
+        if (i < items) cum[i + 1] = running + incl;
+        running += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    __syncwarp();
+    // Work split: a (row, KV head) pair of u stages is cut into n equal segments and CTA c takes
+    // segments c, c + C0_arg, ...: a CTA never straddles two pairs, and the split depends on
+    // the lengths only.  n = round or floor of u / q for a target segment length q = all stages /
+    // (k * CTAs), k = 1..3 rounds; of these six candidates the one with the smallest estimated
+    // time (rounds x (longest segment + a fixed per-segment cost of ~6 stages)) is taken, fewer
+    // segments on ties.
+    const int C0 = C0_arg, U0 = cum[items] * n_kv;
+    auto seg_count = [&](int u, int q, int mode) {  // mode 0: round, 1: floor
+        int n = mode == 0 ? (2 * u + q) / (2 * q) : u / q;
+        return min(max(n, 1), min(max(u, 1), kAttMaxSeg));
+    };
+    int best_q = max((U0 + C0 - 1) / C0, kAttMinUnits), best_mode = 0;
+    int best_cost = -1, best_sg = 0;
+    for (int cand = 0; cand < 6; cand++) {
+        const int k = cand / 2 + 1, mode = cand & 1;
+        const int q = max((U0 + k * C0 - 1) / (k * C0), kAttMinUnits);
+        int sg = 0, longest_seg = 0;
+        for (int base = 0; base < items; base += 32) {
+            int i = base + lane;
+            if (i < items) {
+                int u = cum[i + 1] - cum[i], n = seg_count(u, q, mode);
+                sg += n;
+                longest_seg = max(longest_seg, (u + n - 1) / n);
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            sg += __shfl_xor_sync(0xffffffffu, sg, o);
+            longest_seg = max(longest_seg, __shfl_xor_sync(0xffffffffu, longest_seg, o));
+        }
+        sg *= n_kv;
+        int rounds = (sg + C0 - 1) / C0, cost = rounds * (longest_seg + 6);
+        if (best_cost < 0 || cost < best_cost || (cost == best_cost && sg < best_sg)) {
+            best_cost = cost;
+            best_q = q;
+            best_mode = mode;
+            best_sg = sg;
+        }
+        // the plain split fits one round, or every pair is already whole: take it (the common cases)
+        if (cand == 0 && (rounds == 1 || sg == items * n_kv)) break;
+    }
+    int run2 = 0;
+    if (lane == 0) segcum[0] = 0;
+    for (int base = 0; base < items; base += 32) {
+        int i = base + lane, n = 0;
+        if (i < items) n = seg_count(cum[i + 1] - cum[i], best_q, best_mode);
+        int incl = n;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            int t = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += t;
+        }
+        if (i < items) segcum[i + 1] = run2 + incl;
+        run2 += __shfl_sync(0xffffffffu, incl, 31);
+    }
+}
+
+constexpr int kAttPlanInts = 3 * kAttMaxItems + 2;  // cum [items + 1] | nk [items] | segcum [items + 1], at fixed offsets
+
+__global__ void __launch_bounds__(32) attn_plan_kernel(RowMap rm, const int32_t *seq_len, int n_kv, int C0, int *plan) {
+    pdl_enter();
+    att_plan_warp(threadIdx.x, rm.Bc(), rm, seq_len, n_kv, C0, plan, plan + kAttMaxItems + 1, plan + 2 * kAttMaxItems + 1);
+}
+
 template <int DH, bool NARROW, bool DEEP = false>
 __global__ void __launch_bounds__(160, DEEP ? 1 : 2) attn_mma_kernel(const __grid_constant__ CUtensorMap tmKV, AttnParams p) {
     using Cfg = AttCfg<DH, DEEP>;
@@ -176,88 +269,24 @@ __global__ void __launch_bounds__(160, DEEP ? 1 : 2) attn_mma_kernel(const __gri
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     pdl_launch_dependents();
-    pdl_wait();  // sequence lengths, Q and the freshly appended K/V come from earlier kernels of the step
-    DBT_TL_WAITED;
-    if (warp == 0 && !packed) {
-        int running = 0, longest = 0;
-        if (lane == 0) cum[0] = 0;
-        for (int base = 0; base < items; base += 32) {
-            int i = base + lane, nk = 0, u = 0;
-            if (i < items) {
-                nk = ld_mut(p.seq_len + p.rm.seq(i)) + p.rm.off(i) + 1;
-                u = (nk + kAttTile - 1) / kAttTile;
-                nk_s[i] = nk;
-            }
-            int incl = u, mx = u;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                int t = __shfl_up_sync(0xffffffffu, incl, o);
-                if (lane >= o) incl += t;
-                mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-            }
-            longest = max(longest, mx);
-            if (i < items) cum[i + 1] = running + incl;
-            running += __shfl_sync(0xffffffffu, incl, 31);
+    // A decode step's work split comes precomputed (the same for all its layers).  From the second layer on
+    // it is read before the dependency wait: the kernel that wrote it finished long before any kernel that
+    // could still be running now; in the first layer that kernel may still be running, so the wait comes first.
+    const bool use_plan = p.plan != nullptr && !packed;
+    if (!(use_plan && p.plan_prewait)) pdl_wait();  // sequence lengths, Q and the freshly appended K/V come from earlier kernels of the step
+    if (use_plan) {
+        if (!p.plan_prewait) pdl_wait();
+        for (int i = tid; i <= items; i += blockDim.x) {
+            cum[i] = ld_mut(p.plan + i);
+            segcum[i] = ld_mut(p.plan + 2 * kAttMaxItems + 1 + i);
+            if (i < items) nk_s[i] = ld_mut(p.plan + kAttMaxItems + 1 + i);
         }
-        if (lane == 0) flag[1] = longest;
-        __syncwarp();
-        // Work split: a (row, KV head) pair of u stages is cut into n equal segments and CTA c takes
-        // segments c, c + gridDim.x, ...: a CTA never straddles two pairs, and the split depends on
-        // the lengths only.  n = round or floor of u / q for a target segment length q = all stages /
-        // (k * CTAs), k = 1..3 rounds; of these six candidates the one with the smallest estimated
-        // time (rounds x (longest segment + a fixed per-segment cost of ~6 stages)) is taken, fewer
-        // segments on ties.
-        const int C0 = gridDim.x, U0 = cum[items] * p.n_kv;
-        auto seg_count = [&](int u, int q, int mode) {  // mode 0: round, 1: floor
-            int n = mode == 0 ? (2 * u + q) / (2 * q) : u / q;
-            return min(max(n, 1), min(max(u, 1), kAttMaxSeg));
-        };
-        int best_q = max((U0 + C0 - 1) / C0, kAttMinUnits), best_mode = 0;
-        int best_cost = -1, best_sg = 0;
-        for (int cand = 0; cand < 6; cand++) {
-            const int k = cand / 2 + 1, mode = cand & 1;
-            const int q = max((U0 + k * C0 - 1) / (k * C0), kAttMinUnits);
-            int sg = 0, longest_seg = 0;
-            for (int base = 0; base < items; base += 32) {
-                int i = base + lane;
-                if (i < items) {
-                    int u = cum[i + 1] - cum[i], n = seg_count(u, q, mode);
-                    sg += n;
-                    longest_seg = max(longest_seg, (u + n - 1) / n);
-                }
-            }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-                sg += __shfl_xor_sync(0xffffffffu, sg, o);
-                longest_seg = max(longest_seg, __shfl_xor_sync(0xffffffffu, longest_seg, o));
-            }
-            sg *= p.n_kv;
-            int rounds = (sg + C0 - 1) / C0, cost = rounds * (longest_seg + 6);
-            if (best_cost < 0 || cost < best_cost || (cost == best_cost && sg < best_sg)) {
-                best_cost = cost;
-                best_q = q;
-                best_mode = mode;
-                best_sg = sg;
-            }
-            // the plain split fits one round, or every pair is already whole: take it (the common cases)
-            if (cand == 0 && (rounds == 1 || sg == items * p.n_kv)) break;
-        }
-        int run2 = 0;
-        if (lane == 0) segcum[0] = 0;
-        for (int base = 0; base < items; base += 32) {
-            int i = base + lane, n = 0;
-            if (i < items) n = seg_count(cum[i + 1] - cum[i], best_q, best_mode);
-            int incl = n;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                int t = __shfl_up_sync(0xffffffffu, incl, o);
-                if (lane >= o) incl += t;
-            }
-            if (i < items) segcum[i + 1] = run2 + incl;
-            run2 += __shfl_sync(0xffffffffu, incl, 31);
-        }
+    } else if (warp == 0 && !packed) {
+        att_plan_warp(lane, items, p.rm, p.seq_len, p.n_kv, (int)gridDim.x, cum, nk_s, segcum);
     }
     __syncthreads();
+    if (use_plan && p.plan_prewait) pdl_wait();
+    DBT_TL_WAITED;
     const int C = gridDim.x, Sg = packed ? items * p.n_kv : segcum[items] * p.n_kv;  // all segments, ordered (row, KV head, segment)
     DBT_TL_MARK(3);
     if ((int)blockIdx.x >= Sg) return;
