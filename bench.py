@@ -31,7 +31,7 @@ from paper_2608_12385_b200.inputs import PRESETS, make_synthetic_kv, make_tokens
 # ncu DRAM traffic / algorithmic bytes per launch (captures summarised under profiles/): attention 140.8 MB
 # read+written for 134.6 MB of visible K/V (the rest is the Q|K|V partials it consumes and its output); the GEMMs
 # read their weights once (46.47 MB for 46.14 MB of gate|up weights).
-NCU_TRAFFIC_OVER_ALGORITHMIC = {"attention": 140.8 / 134.58, "gemm_gateup": 1.007, "gemm_down": 1.034, "gemm_qkv": 1.02,
+NCU_TRAFFIC_OVER_ALGORITHMIC = {"attention": 141.9 / 134.45, "gemm_gateup": 1.007, "gemm_down": 1.034, "gemm_qkv": 1.02,
                                 "gemm_o": 1.04}
 METRIC = "grouped_decode_tokens_per_s"
 UNIT = "tokens/s"
@@ -211,9 +211,9 @@ def run_ours(args) -> dict | None:
         regions.sort()
         return regions[len(regions) // 2], launches, clocks, len(regions)
 
-    ms_po, _, _, _ = timed(False, K, W, False, min_total_ms=200.0)
+    ms_po, _, _, _ = timed(False, K, W, False, min_total_ms=0.4 * args.min_timed_ms)
     po_union_m = m.last_expert_union() if cfg.is_moe else None
-    ms_total, launches, clocks, n_regions = timed(True, K, W, True)
+    ms_total, launches, clocks, n_regions = timed(True, K, W, True, min_total_ms=args.min_timed_ms)
     value, ms_max = replicas.aggregate_throughput(B * K, ms_total, dev)
     ms_step = ms_max / K
     union = po_union = None
@@ -381,6 +381,9 @@ def main():
     ap.add_argument("--paths", type=int, default=2, help="residual paths K: the primary plus K-1 decode branches (Appendix C.1)")
     ap.add_argument("--layers", type=int, default=0, help="cut the model to this many layers (profiler captures only)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--min-timed-ms", type=float, default=500.0,
+                    help="repeat the K-step timed region until this much device time has been timed (0: one region; "
+                         "profiler captures)")
     ap.add_argument("--reference-max-steps", type=int, default=128)
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup

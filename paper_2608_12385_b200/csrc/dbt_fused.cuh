@@ -116,19 +116,26 @@ __global__ void __launch_bounds__(256) resid_wide_kernel(float *S, const float *
                                                          const float *__restrict__ g_next, int d, __nv_bfloat16 *Xb,
                                                          size_t lo_off, float *ss_out, int ss_ld) {
     DBT_TL_DECL;
-    pdl_enter();
-    DBT_TL_WAITED;
+    pdl_launch_dependents();
     __shared__ float scratch[64];
     int b = blockIdx.x, i = blockIdx.y * blockDim.x + threadIdx.x;
+    // The gain and the coupling are weights: they are read once per step, so they come from HBM, not from L2.
+    // Requested before the dependency wait, that latency passes while the GEMM before this kernel still runs.
+    float gn = 1.f, cc = 0.f;
+    if (i < d) {
+        gn = g_next ? g_next[i] : 1.f;
+        cc = mode >= 2 ? coup_c[i] : 0.f;
+    }
+    pdl_wait();
+    DBT_TL_WAITED;
     const bool first = MULTI ? blockIdx.z == 0 : true;  // the first branch's blocks also own the primary row
     const int r2 = MULTI ? ((int)blockIdx.z + 1) * Bc + b : Bc + b;
     float q1 = 0.f, q2 = 0.f;
     if (i < d) {
-        // every load of this thread goes out before the first use: S of both rows, the gain, the
-        // coupling, and all splits of both rows' partials (up to 16 splits in one round)
+        // every load of this thread goes out before the first use: S of both rows and all splits of both
+        // rows' partials (up to 16 splits in one round)
         size_t o1 = (size_t)b * d + i, o2 = (size_t)r2 * d + i;
         float s1 = first ? __ldcg(S + o1) : 0.f, s2 = grouped ? __ldcg(S + o2) : 0.f;
-        float gn = g_next ? g_next[i] : 1.f, cc = mode >= 2 ? coup_c[i] : 0.f;
         const size_t offs[2] = {o1, grouped && mode != 3 ? o2 : o1};
         float mm[2];
         sum_splits_k<2, 16>(P, split_stride, nsplit, offs, mm);
@@ -314,11 +321,13 @@ __global__ void __launch_bounds__(256) swiglu_couple_kernel(const float *P, int 
                                                             __nv_bfloat16 *Hb, size_t lo_off, const float *ss,
                                                             int ss_tiles, int ss_ld, int d_norm, float eps) {
     DBT_TL_DECL;
-    pdl_enter();
-    DBT_TL_WAITED;
+    pdl_launch_dependents();
     __shared__ float sh[34];
     int b = blockIdx.x, f = blockIdx.y * blockDim.x + threadIdx.x;
     const bool act = f < F;
+    const float cb = (act && grouped && coup_b) ? coup_b[f] : 0.f;  // a weight, from HBM: requested before the wait
+    pdl_wait();
+    DBT_TL_WAITED;
     const bool first = blockIdx.z == 0;
     const int rb = grouped ? ((int)blockIdx.z + 1) * Bc + b : b, lane = threadIdx.x & 31;
     // The norm shares of the block's two rows are fetched once, by the first warp (lanes 0..15 the
@@ -349,7 +358,7 @@ __global__ void __launch_bounds__(256) swiglu_couple_kernel(const float *P, int 
         if (first) store_split(Hb, (size_t)b * F + f, lo_off, h1);
         if (grouped) {
             float h2 = silu(rs2 * sm[2]) * (rs2 * sm[3]);
-            if (coup_b) h2 += coup_b[f] * h1;
+            h2 += cb * h1;
             store_split(Hb, (size_t)rb * F + f, lo_off, h2);
         }
     }
