@@ -1102,6 +1102,9 @@ dbt_status run_layers_wide(dbt_model *m, const RowMap &rm, int grouped, int n_ti
     size_t pool_layer_elems = (size_t)2 * c.num_pages * c.n_kv_heads * c.page_size * c.head_dim;
     size_t lo_x = m->act_parts == 2 ? (size_t)m->Rmax * d : 0, lo_h = m->act_parts == 2 ? (size_t)m->Rmax * F : 0;
     int ss_tiles = wide_ss_tiles(m), ss_ld = m->Rmax;
+    // prompt chunks of more than one row tile: the kernels between the GEMMs stream tens of MB and take
+    // their vector form (four elements per thread)
+    const bool rows_form = !grouped && rm.cn > 1 && Bc > 256 && d % 4 == 0 && F % 4 == 0 && c.head_dim % 8 == 0 && ((size_t)m->Rmax * d) % 4 == 0;
     double kv_bytes = 0;
     for (int b = 0; b < rm.B; b++)
         for (int j = 0; j < rm.cn; j++) kv_bytes += (double)(m->len_host[b] + j + 1) * 2 * kvd * sizeof(WT);
@@ -1127,7 +1130,12 @@ dbt_status run_layers_wide(dbt_model *m, const RowMap &rm, int grouped, int n_ti
         if ((st = run_gemm_tc(m, qkv, n_tile, &nsp, &sstride)) != DBT_OK) return st;
         const bool fuse = m->fuse_qkv && rm.cn == 1;
         QkvFuse qf{w.P, nsp, sstride, w.ss, ss_tiles, ss_ld, lw.coup_a};
-        if (!fuse)
+        if (rows_form)
+            LAUNCH(m, "qkv_epilogue", 0, qkv_rows_kernel, dim3(Bc, ((c.n_q_heads + c.n_kv_heads) * (c.head_dim / 8) + 255) / 256), 256, 0,
+                   w.P, nsp, sstride, w.Q, rm, c.n_q_heads, c.n_kv_heads, c.head_dim, w.rope, w.seq_len, w.page_table,
+                   m->pages_per_seq_max, c.num_pages, c.page_size, kpool, vpool, w.status, (const float *)w.ss, ss_tiles, ss_ld, d,
+                   c.rms_eps);
+        else if (!fuse)
             LAUNCH(m, "qkv_epilogue", 0, qkv_epilogue_kernel<WT>, dim3(Bc, c.n_q_heads + c.n_kv_heads, branch_blocks(grouped)), 64, 0, w.P, nsp, sstride,
                    w.Q, rm, grouped, c.n_q_heads, c.n_kv_heads, c.head_dim, lw.coup_a, w.rope, w.seq_len, w.page_table,
                    m->pages_per_seq_max, c.num_pages, c.page_size, kpool, vpool, w.status, (const float *)w.ss, ss_tiles, ss_ld, d,
@@ -1139,6 +1147,10 @@ dbt_status run_layers_wide(dbt_model *m, const RowMap &rm, int grouped, int n_ti
         op.W[0] = &mp.wo; op.n_out[0] = d; op.rows[0] = R; op.nseg = 1;
         {
             if ((st = run_gemm_tc(m, op, n_tile, &nsp, &sstride)) != DBT_OK) return st;
+            if (rows_form)
+                LAUNCH(m, "resid_wide", 0, resid_rows_kernel, dim3((Bc + 3) / 4, ss_tiles), 256, 0, w.S, w.P, nsp, sstride, lw.mlp_norm_g, Bc, d,
+                       w.Xb, lo_x, w.ss, ss_ld);
+            else
             LAUNCH_BR(m, grouped, "resid_wide", 0, resid_wide_kernel, dim3(Bc, ss_tiles, branch_blocks(grouped)), 256, 0, w.S, w.P, nsp, sstride, 1,
                    (const float *)nullptr, Bc, grouped, lw.mlp_norm_g, d, w.Xb, lo_x, w.ss, ss_ld);
         }
@@ -1148,6 +1160,10 @@ dbt_status run_layers_wide(dbt_model *m, const RowMap &rm, int grouped, int n_ti
         gu.nseg = 2;
         {
             if ((st = run_gemm_tc(m, gu, n_tile, &nsp, &sstride)) != DBT_OK) return st;
+            if (rows_form)
+                LAUNCH(m, "swiglu_couple", 0, swiglu_rows_kernel, dim3(Bc, (F + 1023) / 1024), 256, 0, w.P, nsp, sstride, F, w.Hb, lo_h,
+                       (const float *)w.ss, ss_tiles, ss_ld, d, c.rms_eps);
+            else
             LAUNCH(m, "swiglu_couple", 0, swiglu_couple_kernel, dim3(Bc, (F + 255) / 256, branch_blocks(grouped)), 256, 0, w.P, nsp, sstride, F, Bc,
                    grouped, lw.coup_b, w.Hb, lo_h, (const float *)w.ss, ss_tiles, ss_ld, d, c.rms_eps);
         }
@@ -1157,6 +1173,10 @@ dbt_status run_layers_wide(dbt_model *m, const RowMap &rm, int grouped, int n_ti
                                                  : (c.final_norm ? m->w.final_norm_g : (const float *)nullptr);
         {
             if ((st = run_gemm_tc(m, dn, n_tile, &nsp, &sstride)) != DBT_OK) return st;
+            if (rows_form)
+                LAUNCH(m, "resid_wide", 0, resid_rows_kernel, dim3((Bc + 3) / 4, ss_tiles), 256, 0, w.S, w.P, nsp, sstride, g_next, Bc, d, w.Xb,
+                       lo_x, w.ss, ss_ld);
+            else
             LAUNCH_BR(m, grouped, "resid_wide", 0, resid_wide_kernel, dim3(Bc, ss_tiles, branch_blocks(grouped)), 256, 0, w.S, w.P, nsp, sstride, 2, lw.coup_c, Bc,
                    grouped, g_next, d, w.Xb, lo_x, w.ss, ss_ld);
         }

@@ -365,6 +365,166 @@ __global__ void __launch_bounds__(256) swiglu_couple_kernel(const float *P, int 
     DBT_TL_END("swiglu");
 }
 
+// ---- prompt chunks: many primary rows, no branch --------------------------------------------------
+// The three kernels above give every thread one output element (latency counts there: a decode step has a
+// few dozen rows).  A prompt chunk has up to a few thousand rows and these kernels become streams of
+// 10..140 MB: here every thread takes four consecutive elements (16-byte loads, 8-byte bf16 stores) of a
+// primary row.  Same arithmetic per element; the partial sums of sum(S^2) are added in another order.
+
+__device__ __forceinline__ float4 ldcg4(const float *p) { return __ldcg(reinterpret_cast<const float4 *>(p)); }
+
+// Four values as two bf16 planes (see store_split), 8 bytes per plane.
+__device__ __forceinline__ void store_split4(__nv_bfloat16 *dst, size_t idx, size_t lo_off, float4 x) {
+    __nv_bfloat162 h0 = __floats2bfloat162_rn(x.x, x.y), h1 = __floats2bfloat162_rn(x.z, x.w);
+    uint2 hv = make_uint2(*reinterpret_cast<uint32_t *>(&h0), *reinterpret_cast<uint32_t *>(&h1));
+    *reinterpret_cast<uint2 *>(dst + idx) = hv;
+    if (lo_off) {
+        __nv_bfloat162 l0 = __floats2bfloat162_rn(x.x - __low2float(h0), x.y - __high2float(h0));
+        __nv_bfloat162 l1 = __floats2bfloat162_rn(x.z - __low2float(h1), x.w - __high2float(h1));
+        *reinterpret_cast<uint2 *>(dst + idx + lo_off) =
+            make_uint2(*reinterpret_cast<uint32_t *>(&l0), *reinterpret_cast<uint32_t *>(&l1));
+    }
+}
+
+__device__ __forceinline__ float4 sum_splits4(const float *P, size_t split_stride, int nsplit, size_t off) {
+    float4 m = ldcg4(P + off);
+    for (int s = 1; s < nsplit; s++) {
+        float4 v = ldcg4(P + (size_t)s * split_stride + off);
+        m.x += v.x, m.y += v.y, m.z += v.z, m.w += v.w;
+    }
+    return m;
+}
+
+// resid_wide_kernel for R primary rows: S += sum_s P[s]; Xb = g_next * S as two planes; the share of
+// sum(S^2) of every (row, 256-column tile).  grid (ceil(R / 4), d / 256), 64 threads per row.  d % 4 == 0.
+__global__ void __launch_bounds__(256) resid_rows_kernel(float *S, const float *P, int nsplit, size_t split_stride,
+                                                         const float *__restrict__ g_next, int R, int d,
+                                                         __nv_bfloat16 *Xb, size_t lo_off, float *ss_out, int ss_ld) {
+    pdl_launch_dependents();
+    __shared__ float scratch[8];
+    const int sub = threadIdx.x >> 6, row = blockIdx.x * 4 + sub, i = blockIdx.y * 256 + (threadIdx.x & 63) * 4;
+    const bool act = row < R && i < d;
+    float4 gn = make_float4(1.f, 1.f, 1.f, 1.f);
+    if (act && g_next) gn = *reinterpret_cast<const float4 *>(g_next + i);
+    pdl_wait();
+    float q = 0.f;
+    if (act) {
+        size_t o = (size_t)row * d + i;
+        float4 s = ldcg4(S + o), m = sum_splits4(P, split_stride, nsplit, o);
+        s.x += m.x, s.y += m.y, s.z += m.z, s.w += m.w;
+        *reinterpret_cast<float4 *>(S + o) = s;
+        store_split4(Xb, o, lo_off, make_float4(gn.x * s.x, gn.y * s.y, gn.z * s.z, gn.w * s.w));
+        q = s.x * s.x + s.y * s.y + s.z * s.z + s.w * s.w;
+    }
+    q = warp_sum(q);
+    if ((threadIdx.x & 31) == 0) scratch[threadIdx.x >> 5] = q;
+    __syncthreads();
+    if ((threadIdx.x & 63) == 0 && row < R) ss_out[(size_t)blockIdx.y * ss_ld + row] = scratch[2 * sub] + scratch[2 * sub + 1];
+}
+
+// swiglu_couple_kernel for R primary rows: H = SiLU(rs * gate) * (rs * up) as two planes.
+// grid (R, ceil(F / 1024)).  F % 4 == 0.
+__global__ void __launch_bounds__(256) swiglu_rows_kernel(const float *P, int nsplit, size_t split_stride, int F,
+                                                          __nv_bfloat16 *Hb, size_t lo_off, const float *ss, int ss_tiles,
+                                                          int ss_ld, int d_norm, float eps) {
+    pdl_launch_dependents();
+    __shared__ float rs_s;
+    const int row = blockIdx.x, f = (blockIdx.y * 256 + threadIdx.x) * 4;
+    pdl_wait();
+    float a = 0.f;
+    if (ss && threadIdx.x < 32)
+        for (int t = threadIdx.x; t < ss_tiles; t += 32) a += __ldcg(ss + (size_t)t * ss_ld + row);
+    float4 gt = make_float4(0.f, 0.f, 0.f, 0.f), up = gt;
+    if (f < F) {
+        size_t o = (size_t)row * 2 * F + f;
+        gt = sum_splits4(P, split_stride, nsplit, o);
+        up = sum_splits4(P, split_stride, nsplit, o + F);
+    }
+    if (threadIdx.x < 32) {
+        a = warp_sum(a);
+        if (threadIdx.x == 0) rs_s = ss ? 1.f / sqrtf(a / (float)d_norm + eps) : 1.f;
+    }
+    __syncthreads();
+    if (f < F) {
+        const float rs = rs_s;
+        float4 h = make_float4(silu(rs * gt.x) * (rs * up.x), silu(rs * gt.y) * (rs * up.y), silu(rs * gt.z) * (rs * up.z),
+                               silu(rs * gt.w) * (rs * up.w));
+        store_split4(Hb, (size_t)row * F + f, lo_off, h);
+    }
+}
+
+// qkv_epilogue_kernel for R primary rows of a bf16 cache: 1/rms, RoPE on Q and K, append K_1, V_1.
+// grid (R, ceil((n_q + n_kv) * (dh / 8) / 256)): a thread takes four consecutive rotation pairs of a head.
+__global__ void __launch_bounds__(256) qkv_rows_kernel(const float *P, int nsplit, size_t split_stride, float *Q, RowMap rm,
+                                                       int n_q, int n_kv, int dh, const float2 *__restrict__ rope_tab,
+                                                       const int32_t *seq_len, const int32_t *__restrict__ page_table,
+                                                       int pt_stride, int num_pages, int page_size, __nv_bfloat16 *kpool,
+                                                       __nv_bfloat16 *vpool, int *status, const float *ss, int ss_tiles,
+                                                       int ss_ld, int d_norm, float eps) {
+    pdl_launch_dependents();
+    __shared__ float rs_s;
+    const int item = blockIdx.x, half = dh / 2, per_head = half / 4;
+    const int w = blockIdx.y * 256 + threadIdx.x, hh = w / per_head, i = (w % per_head) * 4;
+    const bool act = hh < n_q + n_kv;
+    pdl_wait();
+    float a = 0.f;
+    if (ss && threadIdx.x < 32)
+        for (int t = threadIdx.x; t < ss_tiles; t += 32) a += __ldcg(ss + (size_t)t * ss_ld + item);
+    const int seq = rm.seq(item), pos = ld_mut(seq_len + seq) + rm.off(item);
+    const int q_dim = n_q * dh, kv_dim = n_kv * dh, ldp = q_dim + 2 * kv_dim;
+    const size_t p1 = (size_t)item * ldp;
+    const bool is_q = hh < n_q;
+    float4 x0 = make_float4(0.f, 0.f, 0.f, 0.f), x1 = x0, v0 = x0, v1 = x0, c = x0, sn = x0;
+    int page = 0;
+    size_t o0 = 0;
+    if (act) {
+        const float4 t0 = *reinterpret_cast<const float4 *>(rope_tab + (size_t)pos * half + i);
+        const float4 t1 = *reinterpret_cast<const float4 *>(rope_tab + (size_t)pos * half + i + 2);
+        c = make_float4(t0.x, t0.z, t1.x, t1.z);
+        sn = make_float4(t0.y, t0.w, t1.y, t1.w);
+        o0 = is_q ? (size_t)hh * dh + i : (size_t)q_dim + (size_t)(hh - n_q) * dh + i;
+        x0 = sum_splits4(P, split_stride, nsplit, p1 + o0);
+        x1 = sum_splits4(P, split_stride, nsplit, p1 + o0 + half);
+        if (!is_q) {
+            v0 = sum_splits4(P, split_stride, nsplit, p1 + o0 + kv_dim);
+            v1 = sum_splits4(P, split_stride, nsplit, p1 + o0 + kv_dim + half);
+            page = page_table[(size_t)seq * pt_stride + pos / page_size];
+        }
+    }
+    if (threadIdx.x < 32) {
+        a = warp_sum(a);
+        if (threadIdx.x == 0) rs_s = ss ? 1.f / sqrtf(a / (float)d_norm + eps) : 1.f;
+    }
+    __syncthreads();
+    if (!act) return;
+    const float rs = rs_s;
+    x0 = make_float4(rs * x0.x, rs * x0.y, rs * x0.z, rs * x0.w);
+    x1 = make_float4(rs * x1.x, rs * x1.y, rs * x1.z, rs * x1.w);
+    const float4 r0 = make_float4(x0.x * c.x - x1.x * sn.x, x0.y * c.y - x1.y * sn.y, x0.z * c.z - x1.z * sn.z,
+                                  x0.w * c.w - x1.w * sn.w);
+    const float4 r1 = make_float4(x1.x * c.x + x0.x * sn.x, x1.y * c.y + x0.y * sn.y, x1.z * c.z + x0.z * sn.z,
+                                  x1.w * c.w + x0.w * sn.w);
+    if (is_q) {
+        float *q1 = Q + (size_t)item * q_dim + o0;
+        *reinterpret_cast<float4 *>(q1) = r0;
+        *reinterpret_cast<float4 *>(q1 + half) = r1;
+        return;
+    }
+    if (page < 0 || page >= num_pages) {
+        if (i == 0) report(status, kStatusBadPage, page);
+        return;
+    }
+    const size_t base = (((size_t)page * n_kv + (hh - n_q)) * page_size + pos % page_size) * dh + i;
+    auto st4 = [](__nv_bfloat16 *dst, float4 v) {
+        __nv_bfloat162 a2 = __floats2bfloat162_rn(v.x, v.y), b2 = __floats2bfloat162_rn(v.z, v.w);
+        *reinterpret_cast<uint2 *>(dst) = make_uint2(*reinterpret_cast<uint32_t *>(&a2), *reinterpret_cast<uint32_t *>(&b2));
+    };
+    st4(kpool + base, r0);
+    st4(kpool + base + half, r1);
+    st4(vpool + base, make_float4(rs * v0.x, rs * v0.y, rs * v0.z, rs * v0.w));
+    st4(vpool + base + half, make_float4(rs * v1.x, rs * v1.y, rs * v1.z, rs * v1.w));
+}
+
 // Eq. embeddings for the fused path: S^0 = RMSNorm(E[x]) and, for the first layer's Q|K|V GEMM,
 // the input g_next * S^0 as two bf16 planes plus sum(S^0 ^2) per row (tile 0 carries the whole
 // sum, the other tile slots are zeroed).  One block per row.
