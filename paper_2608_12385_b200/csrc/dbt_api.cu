@@ -16,6 +16,7 @@
 #include <vector>
 
 #include "dbt_attn_mma.cuh"
+#include "dbt_attn_prompt.cuh"
 #include "dbt_fused.cuh"
 #include "dbt_gemm_tc.cuh"
 #include "dbt_kernels.cuh"
@@ -94,6 +95,7 @@ struct dbt_model {
     std::map<const CUtensorMap *, ActBase> act_base;
     std::map<std::tuple<const CUtensorMap *, int, int>, CUtensorMap> act3d;
     bool evict_first;  // weight tiles and K/V pages carry the evict-first L2 hint (DBT_EVICT_FIRST=0 turns it off)
+    bool prompt_attn_off;  // DBT_PROMPT_ATTN=tile: prompt chunks through the 16-row kernel's packed tiles (the earlier form)
     bool fuse_qkv;     // decode steps: the attention kernel does the Q|K|V epilogue itself (DBT_FUSE_QKV=0 keeps the kernel)
     int num_sms;
     int act_parts;  // 2: GEMM inputs carried as hi + lo bf16 terms (the operator-level GEMM entry uses 1: plain bf16)
@@ -762,6 +764,27 @@ dbt_status run_attention_mma(dbt_model *m, const RowMap &rm, int grouped, int la
     }
     // prompt chunks: 16 / G consecutive positions of a sequence share a query tile (the 16-row kernel)
     const bool packed = pack_prompt && !grouped && !qf && rm.cn > 1;
+    if (packed && 16 % G == 0 && !m->prompt_attn_off) {
+        // the prompt kernel: eight query tiles per CTA share every page the CTA brings in
+        PromptAttnParams q{};
+        q.Q = w.Q;
+        q.B = rm.B;
+        q.cn = rm.cn;
+        q.G = G;
+        q.n_kv = c.n_kv_heads;
+        q.num_pages = c.num_pages;
+        q.pt_stride = m->pages_per_seq_max;
+        q.k_row0 = p.k_row0;
+        q.page_table = w.page_table;
+        q.seq_len = w.seq_len;
+        q.Ob = w.Ob;
+        q.lo_off = p.lo_off;
+        q.status = w.status;
+        q.nqb = (rm.cn + kPaWarps * (16 / G) - 1) / (kPaWarps * (16 / G));
+        dim3 gp(rm.B * c.n_kv_heads * q.nqb);
+        LAUNCH(m, "attention", kv_bytes, attn_prompt_kernel<DH>, gp, (kPaWarps + 1) * 32, PromptAttCfg<DH>::kSmemBytes, m->map_kv, q);
+        return DBT_OK;
+    }
     if (packed) {
         p.pack = 16 / G;
         p.cn = rm.cn;
@@ -1337,6 +1360,10 @@ bool setup_tc(dbt_model *m) {
     m->att_fast = ok && !(fa && strcmp(fa, "simt") == 0) &&
                   make_kv_page_map(&m->map_kv, m->kv_pool, (uint64_t)c.n_layers * 2 * c.num_pages * c.n_kv_heads * c.page_size,
                                    (uint64_t)c.num_pages * c.n_kv_heads * c.page_size, c.head_dim) &&
+                  cudaFuncSetAttribute(attn_prompt_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       PromptAttCfg<128>::kSmemBytes) == cudaSuccess &&
+                  cudaFuncSetAttribute(attn_prompt_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       PromptAttCfg<64>::kSmemBytes) == cudaSuccess &&
                   cudaFuncSetAttribute(attn_mma_kernel<128, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        AttCfg<128, true>::kSmemBytes) == cudaSuccess &&
                   cudaFuncSetAttribute(attn_mma_kernel<64, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -1493,6 +1520,8 @@ dbt_status dbt_create(const dbt_config *cfg, const dbt_weights *w, void *kv_pool
         m->evict_first = !(ef && strcmp(ef, "0") == 0);
         const char *fq = getenv("DBT_FUSE_QKV");
         m->fuse_qkv = m->att_fast && !(fq && strcmp(fq, "0") == 0);
+        const char *pa = getenv("DBT_PROMPT_ATTN");
+        m->prompt_attn_off = pa && strcmp(pa, "tile") == 0;
     }
     const char *ro = getenv("DBT_READOUT");
     m->readout_row = ro && strcmp(ro, "row") == 0;

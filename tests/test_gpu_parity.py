@@ -72,12 +72,14 @@ def test_prefill_longer_than_one_chunk_and_page_boundaries():
     (small_bf16(n_layers=1, n_q_heads=4, n_kv_heads=4), 1, 2500),         # MHA: 16 positions per tile, 2048 + 452
     (small_bf16(n_layers=1, n_q_heads=2, n_kv_heads=1, head_dim=128, d_model=128, vocab=777), 5, 1000),  # 8 per tile
     (small_bf16(n_layers=1, n_q_heads=8, n_kv_heads=1), 2, 333),          # 2 positions per tile
+    (small_bf16(n_layers=1, n_q_heads=3, n_kv_heads=1), 2, 400),          # 3 heads per KV head: 5 positions per tile (the 16-row kernel)
 ])
 def test_long_prompt_prefill_matches_the_oracle(cfg, B, n):
     """Section 4.4 item 1, prompt-wide prefill: prompts of up to 2500 positions go through in chunks of up to
-    2048 rows (GEMMs over several row tiles per weight tile, causal attention with 16 / G consecutive positions
-    per query tile).  Last-position logits and the whole cache against the oracle's position-by-position
-    primary pass, then two grouped steps on top of the device's own cache."""
+    2048 rows (GEMMs over several row tiles per weight tile, vector kernels between them, causal attention
+    with 16 / G consecutive positions per query tile and eight tiles per CTA).  Last-position logits and the
+    whole cache against the oracle's position-by-position primary pass, then two grouped steps on top of the
+    device's own cache."""
     w = make_weights(cfg, seed=51, matrix_std=0.05)
     tok = make_tokens(cfg, B, n + 2, seed=52)
     om = oracle.OracleModel(cfg, w, B, n + 2)
@@ -125,6 +127,13 @@ def test_prefill_boundary_is_prefill_of_all_but_one_plus_the_grouped_step(cfg):
     ga2 = a.decode_full(tok[:, S].cuda().contiguous())
     gb2 = b.decode_full(tok[:, S].cuda().contiguous())
     assert torch.equal(ga2["z1"], gb2["z1"]) and torch.equal(ga2["z2"], gb2["z2"])
+
+
+def test_prompt_chunks_through_the_16_row_attention_kernel(monkeypatch):
+    """DBT_PROMPT_ATTN=tile: the earlier form of the prompt attention (one 16-row tile per CTA pass) still
+    serves head ratios that do not divide 16, and computes the same prefill."""
+    monkeypatch.setenv("DBT_PROMPT_ATTN", "tile")
+    test_long_prompt_prefill_matches_the_oracle(small_bf16(n_layers=2), 3, 700)
 
 
 def test_prefill_in_one_call_equals_prefill_in_pieces():
