@@ -611,7 +611,7 @@ int split_slots(const dbt_model *m, int n_tile) {
     return (n_tile <= 64 ? 2 : 1) * sms;
 }
 
-template <int N_TILE>
+template <int N_TILE, int MT = 1>
 dbt_status launch_gemm_tc(dbt_model *m, const TcCall &c, const TcParams &p, const LmEpi &e, dim3 grid, double bytes) {
     const CUtensorMap *w1 = c.nseg > 1 ? c.W[1] : c.W[0], *w2 = c.nseg > 2 ? c.W[2] : c.W[0];
     const CUtensorMap *x = c.X;
@@ -630,7 +630,7 @@ dbt_status launch_gemm_tc(dbt_model *m, const TcCall &c, const TcParams &p, cons
             pp.stacked = N_TILE <= 128 ? 1 : 0;
         }
     }
-    LAUNCH(m, c.tag, bytes, gemm_tc_kernel<N_TILE>, grid, 128, TcCfg<N_TILE>::kSmemBytes, *c.W[0], *w1, *w2, *x, pp, e);
+    LAUNCH(m, c.tag, bytes, (gemm_tc_kernel<N_TILE, MT>), grid, 128, (TcCfg<N_TILE, MT>::kSmemBytes), *c.W[0], *w1, *w2, *x, pp, e);
     return DBT_OK;
 }
 
@@ -640,9 +640,22 @@ dbt_status run_gemm_tc(dbt_model *m, const TcCall &c, int n_tile, int *nsplit_ou
     TcParams p{};
     int tiles = 0, col = 0;
     double bytes = 0;
+    // prompt chunks (more rows than the widest tile): two weight tiles per CTA share every activation box where
+    // that pays -- such a CTA takes ~1.6x as long as a one-tile CTA, so the choice goes by full waves of CTAs
+    int mt = 1;
+    if (!c.grp_cnt && c.R > 256) {
+        int t1 = 0, t2 = 0;
+        for (int s = 0; s < c.nseg; s++) {
+            t1 += (c.n_out[s] + kTcM - 1) / kTcM;
+            t2 += (c.n_out[s] + 2 * kTcM - 1) / (2 * kTcM);
+        }
+        const int rt = (c.R + 255) / 256, sms = m->num_sms;
+        const int w1 = (t1 * rt + sms - 1) / sms, w2 = (t2 * rt + sms - 1) / sms;
+        if (16 * w2 < 10 * w1) mt = 2;
+    }
     for (int s = 0; s < c.nseg; s++) {
         p.seg[s] = TcSeg{tiles, c.n_out[s], c.rows[s], col};
-        tiles += (c.n_out[s] + kTcM - 1) / kTcM;
+        tiles += (c.n_out[s] + kTcM * mt - 1) / (kTcM * mt);
         col += c.n_out[s];
         if (!c.grp_cnt) bytes += (double)c.n_out[s] * c.K * 2;  // per-expert launches: the loaded set is known on the device only
     }
@@ -688,7 +701,7 @@ dbt_status run_gemm_tc(dbt_model *m, const TcCall &c, int n_tile, int *nsplit_ou
         case 32: return launch_gemm_tc<32>(m, c, p, e, grid, bytes);
         case 64: return launch_gemm_tc<64>(m, c, p, e, grid, bytes);
         case 128: return launch_gemm_tc<128>(m, c, p, e, grid, bytes);
-        case 256: return launch_gemm_tc<256>(m, c, p, e, grid, bytes);
+        case 256: return mt == 2 ? launch_gemm_tc<256, 2>(m, c, p, e, grid, bytes) : launch_gemm_tc<256>(m, c, p, e, grid, bytes);
     }
     return fail(m, DBT_ERR_UNSUPPORTED, "row tile %d", n_tile);
 }
@@ -1297,7 +1310,9 @@ bool allow_smem() {
 }
 // The attribute is per device: set it on every call for the device that is current (it is cheap).
 bool allow_smem_all() {
-    return allow_smem<16>() && allow_smem<32>() && allow_smem<64>() && allow_smem<128>() && allow_smem<256>();
+    return allow_smem<16>() && allow_smem<32>() && allow_smem<64>() && allow_smem<128>() && allow_smem<256>() &&
+           cudaFuncSetAttribute(gemm_tc_kernel<256, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcCfg<256, 2>::kSmemBytes) ==
+               cudaSuccess;
 }
 
 // Build the TMA descriptors of a bf16 model.  Returns false when the path cannot be used.

@@ -194,26 +194,32 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
 // Activations may arrive as two bf16 terms, x = hi + lo (hi = bf16(x), lo = bf16(x - hi)): the
 // weight tile is then multiplied by both and the two products land in the same fp32
 // accumulator, which restores fp32-level accuracy of the activations at no extra HBM traffic.
-template <int N_TILE>
+// MT: weight tiles per CTA.  A prompt chunk's GEMM (256-row activation tiles, no split-K) is bound by the
+// bytes its CTAs pull from L2 per MMA; with two weight tiles (two accumulators, 2 x 256 TMEM columns) sharing
+// every activation box, a stage carries 96 KB for twice the MMAs of the 80 KB stage of one tile.
+template <int N_TILE, int MT = 1>
 struct TcCfg {
     static constexpr int kBBytes = N_TILE * kTcK * 2;        // one term of the activation tile
-    static constexpr int kStageBytes = kTcABytes + 2 * kBBytes;
+    static constexpr int kStageBytes = MT * kTcABytes + 2 * kBBytes;
     // small row counts: keep one CTA near 100 KB so that a dependent kernel's CTA can become
     // resident beside it; large row counts take the whole SM
     static constexpr int kStages = N_TILE <= 16 ? 5 : N_TILE <= 32 ? 4 : N_TILE <= 64 ? 3 : N_TILE <= 128 ? 4 : 2;
     // room for the two planes' accumulators side by side (see `stacked` in the kernel)
     static constexpr int kStackable = N_TILE <= 128;
-    static constexpr int kTmemCols = kStackable ? (2 * N_TILE < 32 ? 32 : 2 * N_TILE) : N_TILE;
+    static constexpr int kAccCols = kStackable ? 2 * N_TILE : N_TILE;  // accumulator columns of one weight tile
+    static constexpr int kTmemCols = MT * kAccCols < 32 ? 32 : MT * kAccCols;
+    static_assert(MT * kAccCols <= 512, "tensor memory has 512 columns");
     static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
 
-template <int N_TILE>
+template <int N_TILE, int MT = 1>
 __global__ void __launch_bounds__(128, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtensorMap tmW1,
                const __grid_constant__ CUtensorMap tmW2, const __grid_constant__ CUtensorMap tmX, TcParams p,
                LmEpi e) {
-    using Cfg = TcCfg<N_TILE>;
+    using Cfg = TcCfg<N_TILE, MT>;
     constexpr int STAGES = Cfg::kStages;
+    constexpr int kBOff = MT * kTcABytes;  // the activation box follows the weight tiles of a stage
     extern __shared__ uint8_t smem_raw[];
     uint32_t raw = smem_u32(smem_raw);
     uint32_t tiles = (raw + 1023u) & ~1023u;  // 1024-byte aligned operand tiles
@@ -251,7 +257,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
     if (p.nseg > 2 && tile >= p.seg[2].tile0) sg = 2;
     const TcSeg seg = p.seg[sg];
     const CUtensorMap *tmW = sg == 0 ? &tmW0 : sg == 1 ? &tmW1 : &tmW2;
-    int f0 = (tile - seg.tile0) * kTcM;
+    int f0 = (tile - seg.tile0) * kTcM * MT;
     int total_kt = (p.K + kTcK - 1) / kTcK;
     int kt0 = split * p.kt_per_split;
     int nkt = min(p.kt_per_split, total_kt - kt0);
@@ -285,23 +291,28 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
         tma_prefetch_desc(tmW);
         tma_prefetch_desc(&tmX);
         int npre = min(STAGES, nkt);
-        const uint32_t tx = kTcABytes + p.parts * Cfg::kBBytes;
+        const uint32_t tx = MT * kTcABytes + p.parts * Cfg::kBBytes;
         auto load_x = [&](int s, int kt) {
             if (p.x3d) {
-                tma_load_3d(tiles + s * Cfg::kStageBytes + kTcABytes, &tmX, full_bar(s), kt * kTcK, x_row0, 0);
+                tma_load_3d(tiles + s * Cfg::kStageBytes + kBOff, &tmX, full_bar(s), kt * kTcK, x_row0, 0);
                 return;
             }
             for (int part = 0; part < p.parts; part++)
                 for (int j = 0; j < N_TILE / 16; j++)
-                    tma_load_2d(tiles + s * Cfg::kStageBytes + kTcABytes + part * Cfg::kBBytes + j * 2048, &tmX,
+                    tma_load_2d(tiles + s * Cfg::kStageBytes + kBOff + part * Cfg::kBBytes + j * 2048, &tmX,
                                 full_bar(s), kt * kTcK, part * p.lo_row0 + x_row0 + j * 16);
         };
         const uint64_t pol = l2_evict_first_policy();
         auto load_w = [&](int s, int kt) {
-            if (p.evict_first)
-                tma_load_2d_hint(tiles + s * Cfg::kStageBytes, tmW, full_bar(s), kt * kTcK, w_row0 + f0, pol);
-            else
-                tma_load_2d(tiles + s * Cfg::kStageBytes, tmW, full_bar(s), kt * kTcK, w_row0 + f0);
+#pragma unroll
+            for (int mt = 0; mt < MT; mt++) {  // a tile past the matrix's last row arrives as zeros
+                if (p.evict_first)
+                    tma_load_2d_hint(tiles + s * Cfg::kStageBytes + mt * kTcABytes, tmW, full_bar(s), kt * kTcK,
+                                     w_row0 + f0 + mt * kTcM, pol);
+                else
+                    tma_load_2d(tiles + s * Cfg::kStageBytes + mt * kTcABytes, tmW, full_bar(s), kt * kTcK,
+                                w_row0 + f0 + mt * kTcM);
+            }
         };
         for (int i = 0; i < npre; i++) {
             mbar_expect_tx(full_bar(i), tx);
@@ -332,17 +343,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
             ok = mbar_wait(full_bar(s), (i / STAGES) & 1, wait_limit);
             if (!ok) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            uint64_t adesc = umma_smem_desc(tiles + s * Cfg::kStageBytes);
-            if (stacked) {
-                uint64_t bdesc = umma_smem_desc(tiles + s * Cfg::kStageBytes + kTcABytes);
 #pragma unroll
-                for (int k = 0; k < kTcK / 16; k++) umma_f16(tmem_base, adesc + 2 * k, bdesc + 2 * k, idesc2, (i | k) != 0);
-            } else {
-                for (int part = 0; part < p.parts; part++) {
-                    uint64_t bdesc = umma_smem_desc(tiles + s * Cfg::kStageBytes + kTcABytes + part * Cfg::kBBytes);
+            for (int mt = 0; mt < MT; mt++) {
+                const uint32_t acc = tmem_base + mt * Cfg::kAccCols;
+                uint64_t adesc = umma_smem_desc(tiles + s * Cfg::kStageBytes + mt * kTcABytes);
+                if (stacked) {
+                    uint64_t bdesc = umma_smem_desc(tiles + s * Cfg::kStageBytes + kBOff);
 #pragma unroll
-                    for (int k = 0; k < kTcK / 16; k++)  // advance 16 elements = 32 bytes inside the swizzle row
-                        umma_f16(tmem_base, adesc + 2 * k, bdesc + 2 * k, idesc, (i | k | part) != 0);
+                    for (int k = 0; k < kTcK / 16; k++) umma_f16(acc, adesc + 2 * k, bdesc + 2 * k, idesc2, (i | k) != 0);
+                } else {
+                    for (int part = 0; part < p.parts; part++) {
+                        uint64_t bdesc = umma_smem_desc(tiles + s * Cfg::kStageBytes + kBOff + part * Cfg::kBBytes);
+#pragma unroll
+                        for (int k = 0; k < kTcK / 16; k++)  // advance 16 elements = 32 bytes inside the swizzle row
+                            umma_f16(acc, adesc + 2 * k, bdesc + 2 * k, idesc, (i | k | part) != 0);
+                    }
                 }
             }
             umma_commit(empty_bar(s));
@@ -364,10 +379,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
     float *scratch = reinterpret_cast<float *>(gen_tiles);
     int rows = grp_n >= 0 ? min(grp_n, N_TILE) : min(min(seg.rows, p.R) - x_row0, N_TILE);
     const bool stacked_acc = Cfg::kStackable && p.stacked;
-    auto ld_acc = [&](int c0, float (&v)[16]) {  // 16 accumulator columns of this thread's feature
+    auto ld_acc = [&](int mt, int c0, float (&v)[16]) {  // 16 accumulator columns of this thread's feature
         uint32_t a[16], b[16];
-        tmem_ld16_issue(tmem_base + ((uint32_t)(warp * 32) << 16) + c0, a);
-        if (stacked_acc) tmem_ld16_issue(tmem_base + ((uint32_t)(warp * 32) << 16) + N_TILE + c0, b);
+        const uint32_t base = tmem_base + ((uint32_t)(warp * 32) << 16) + mt * Cfg::kAccCols;
+        tmem_ld16_issue(base + c0, a);
+        if (stacked_acc) tmem_ld16_issue(base + N_TILE + c0, b);
         tmem_ld_wait();  // both halves travel together
 #pragma unroll
         for (int i = 0; i < 16; i++) v[i] = __uint_as_float(a[i]) + (stacked_acc ? __uint_as_float(b[i]) : 0.f);
@@ -388,7 +404,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
 #pragma unroll 1
         for (int c0 = 0; c0 < N_TILE && c0 < rows; c0 += 16) {
             float v[16];
-            ld_acc(c0, v);
+            ld_acc(0, c0, v);
             if (f < seg.n_out) {
 #pragma unroll
                 for (int i = 0; i < 16; i++)
@@ -396,16 +412,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
             }
         }
     } else if (got) {
-        int f = f0 + warp * 32 + lane;
-        float *out = p.P + ((size_t)split * p.R + x_row0) * p.ldp + seg.col0 + f;
 #pragma unroll 1
-        for (int c0 = 0; c0 < N_TILE && c0 < rows; c0 += 16) {
-            float v[16];
-            ld_acc(c0, v);
-            if (f < seg.n_out) {
+        for (int mt = 0; mt < MT; mt++) {
+            int f = f0 + mt * kTcM + warp * 32 + lane;
+            float *out = p.P + ((size_t)split * p.R + x_row0) * p.ldp + seg.col0 + f;
+#pragma unroll 1
+            for (int c0 = 0; c0 < N_TILE && c0 < rows; c0 += 16) {
+                float v[16];
+                ld_acc(mt, c0, v);
+                if (f < seg.n_out) {
 #pragma unroll
-                for (int i = 0; i < 16; i++)
-                    if (c0 + i < rows) out[(size_t)(c0 + i) * p.ldp] = v[i];
+                    for (int i = 0; i < 16; i++)
+                        if (c0 + i < rows) out[(size_t)(c0 + i) * p.ldp] = v[i];
+                }
             }
         }
     }
