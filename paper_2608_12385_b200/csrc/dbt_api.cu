@@ -900,7 +900,7 @@ dbt_status run_moe_tc(dbt_model *m, int l, const RowMap &rm, int grouped, bool r
                                     m->stream));
     LAUNCH(m, "route", 0, route_kernel, R, 32, 2 * E * sizeof(float), w.P, rnsp, rstride, E, Bc, c.k_primary, c.k_branch, km,
            c.router_mode == DBT_ROUTER_REPLAY, w.ridx, w.rwts, last, c.max_batch * km, ssp, ss_tiles, ss_ld, d, c.rms_eps);
-    LAUNCH(m, "moe_sort", 0, moe_sort_kernel, 1, 1024, 0, w.ridx, R, km, E, w.ecnt, w.eoff, w.epos,
+    LAUNCH(m, "moe_sort", 0, moe_sort_kernel, 1, (E + 31) / 32 * 32 < 64 ? 64 : (E + 31) / 32 * 32, 0, w.ridx, R, km, E, w.ecnt, w.eoff, w.epos,
            record_experts ? w.union_cnt + l : (int32_t *)nullptr);
     LAUNCH(m, "moe_gather", 0, moe_gather_kernel, R * km, 256, 0, w.Xb, lo_x, w.ridx, w.epos, km, d, w.Xs, lo_xs, ssp, ss_tiles, ss_ld,
            c.rms_eps, w.rs_sorted);

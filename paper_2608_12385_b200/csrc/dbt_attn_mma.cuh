@@ -71,6 +71,7 @@ constexpr int kAttTile = 64;       // tokens per pipeline stage (4 pages)
 constexpr int kAttWarps = 4;       // consumer warps, one page each
 constexpr int kAttMaxItems = 256;  // rows per launch (prefill chunks and batches stay below)
 constexpr int kAttMinUnits = 4;    // a CTA takes at least 4 tiles (256 tokens)
+constexpr int kAttPauseAt = 1;     // the producer pauses after stage 1 (the second) until the queries are built
 constexpr int kAttMaxSeg = 256;    // most segments a (sequence, KV head) pair is split into
 constexpr int kAttGroup = 8;       // segments merged at once (one round of loads)
 constexpr int kAttSingle = 16;     // up to this many segments, one CTA merges them all (two rounds of loads)
@@ -363,12 +364,13 @@ __global__ void __launch_bounds__(160, DEEP ? 1 : 2) attn_mma_kernel(const __gri
                         tma_load_4d(tiles + s * Cfg::kStageBytes + lane * 2 * Cfg::kPageBytes, &tmKV, full_bar(s), 0, 0,
                                     (int)(p.k_row0 + row), 0);
                 }
-                // After the first stage the stream pauses until the consumers have their queries: their
+                // After the first two stages the stream pauses until the consumers have their queries: their
                 // few small loads would otherwise queue behind hundreds of CTAs' page traffic for several
                 // microseconds, and nothing can be consumed before they return anyway.  (Letting the ring fill
                 // at once instead, with the small loads issued first, was measured slower: the queries are ready
-                // 0.8 us sooner but the stream then runs 10 % slower.)
-                if (it == 0) asm volatile("bar.sync 2, 160;" ::: "memory");
+                // 0.8 us sooner but the stream then runs 10 % slower; pausing after one, two, four or six stages
+                // gave 1.0446, 1.0384, 1.0420 and 1.0462 ms per step of the 1B model at batch 16.)
+                if (it == kAttPauseAt || (it < kAttPauseAt && sidx + C >= Sg && t == t1 - 1)) asm volatile("bar.sync 2, 160;" ::: "memory");
             }
         }
         if (!ok && lane == 0) report(p.status, kStatusWaitExpired, 300);

@@ -566,13 +566,13 @@ __global__ void __launch_bounds__(256) embed_fused_kernel(const int32_t *tokens,
 
 // Per-expert row lists -> offsets and the sorted position of every (row, slot) entry.  Entries of
 // one expert keep ascending (row, slot) order; experts follow each other in index order.
-// One block, one thread per expert (E <= 1024).
+// One block, one thread per expert (E <= blockDim.x <= 1024); the offsets come from a two-level shuffle scan.
 __global__ void __launch_bounds__(1024) moe_sort_kernel(const int32_t *idx, int R, int kmax, int E, int32_t *cnt,
                                                         int32_t *off, int32_t *pos, int32_t *union_count) {
     DBT_TL_DECL;
     pdl_enter();
     DBT_TL_WAITED;
-    __shared__ int s_cnt[1024], s_off[1025];
+    __shared__ int s_wsum[32];
     __shared__ int s_idx[4096];  // the selections, staged once (larger lists are read from global memory)
     const int n = R * kmax;
     const bool staged = n <= 4096;
@@ -580,30 +580,38 @@ __global__ void __launch_bounds__(1024) moe_sort_kernel(const int32_t *idx, int 
         for (int i = threadIdx.x; i < n; i += blockDim.x) s_idx[i] = idx[i];
     __syncthreads();
     const int32_t *src = staged ? s_idx : idx;
-    int e = threadIdx.x, c = 0;
+    const int e = threadIdx.x, lane = e & 31, wp = e >> 5;
+    int c = 0;
     if (e < E)
         for (int i = 0; i < n; i++) c += src[i] == e;
-    s_cnt[e] = e < E ? c : 0;
-    __syncthreads();
-    if (e == 0) {
-        int run = 0, uni = 0;
-        for (int i = 0; i < E; i++) {
-            s_off[i] = run;
-            run += s_cnt[i];
-            uni += s_cnt[i] > 0;
+    int incl = c;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        int t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    if (lane == 31) s_wsum[wp] = incl;
+    const int uni = __syncthreads_count(c > 0);
+    if (wp == 0) {
+        int v = lane < (int)(blockDim.x >> 5) ? s_wsum[lane] : 0, w = v;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            int t = __shfl_up_sync(0xffffffffu, w, o);
+            if (lane >= o) w += t;
         }
-        s_off[E] = run;
-        if (union_count) *union_count = uni;
+        s_wsum[lane] = w - v;  // experts before this warp's
     }
     __syncthreads();
+    const int my_off = s_wsum[wp] + incl - c;
     if (e < E) {
         cnt[e] = c;
-        off[e] = s_off[e];
+        off[e] = my_off;
         int k = 0;
         for (int i = 0; i < n && k < c; i++)
-            if (src[i] == e) pos[i] = s_off[e] + k++;
+            if (src[i] == e) pos[i] = my_off + k++;
     }
-    if (e == 0) off[E] = s_off[E];
+    if (e == E - 1) off[E] = my_off + c;
+    if (e == 0 && union_count) *union_count = uni;
     DBT_TL_END("moe_sort");
 }
 
@@ -673,21 +681,43 @@ __global__ void __launch_bounds__(256) moe_combine_sorted_kernel(const float *Ys
     int b = blockIdx.x;
     // the row's selections (weights, sorted positions) once, then all expert rows of a column in
     // flight together; terms are added in slot order
-    constexpr int KM = 16;
+    constexpr int KM = 8;
     const bool first = MULTI ? blockIdx.z == 0 : true;
     const int r2 = MULTI ? ((int)blockIdx.z + 1) * Bc + b : Bc + b;
     for (int i = blockIdx.y * blockDim.x + threadIdx.x; i < d; i += gridDim.y * blockDim.x) {
         float m1 = 0.f, m2 = 0.f;
+        // Everything that does not depend on the routing is requested first: the residual rows and (up to 8
+        // splits of) the shared expert's partials; they travel while the selections, then the expert rows, arrive.
+        const float s1_in = first ? __ldcg(S + (size_t)b * d + i) : 0.f, s2_in = grouped ? __ldcg(S + (size_t)r2 * d + i) : 0.f;
+        const size_t offs[2] = {(size_t)b * d + i, (size_t)(grouped && !gate_g ? r2 : b) * d + i};
+        const bool early = Psh && nsplit <= 8;
+        float pv[8][2];
+#pragma unroll
+        for (int sp = 0; sp < 8; sp++) {
+            pv[sp][0] = early && sp < nsplit ? __ldcg(Psh + (size_t)sp * split_stride + offs[0]) : 0.f;
+            pv[sp][1] = early && sp < nsplit ? __ldcg(Psh + (size_t)sp * split_stride + offs[1]) : 0.f;
+        }
         for (int j0 = 0; j0 < kmax; j0 += KM) {
+            // selections, weights and sorted positions of both rows in one round, the expert rows in the next
+            int e1[KM], e2[KM], p1[KM], p2[KM];
             float y1[KM], w1[KM], y2[KM], w2[KM];
 #pragma unroll
             for (int j = 0; j < KM; j++) {
-                bool on1 = j0 + j < kmax && idx[(size_t)b * kmax + j0 + j] >= 0;
-                bool on2 = grouped && j0 + j < kmax && idx[(size_t)r2 * kmax + j0 + j] >= 0;
-                w1[j] = on1 ? wts[(size_t)b * kmax + j0 + j] : 0.f;
-                y1[j] = on1 ? __ldcg(Ys + (size_t)pos[(size_t)b * kmax + j0 + j] * d + i) : 0.f;
-                w2[j] = on2 ? wts[(size_t)r2 * kmax + j0 + j] : 0.f;
-                y2[j] = on2 ? __ldcg(Ys + (size_t)pos[(size_t)r2 * kmax + j0 + j] * d + i) : 0.f;
+                const bool in = j0 + j < kmax;
+                const size_t o1 = (size_t)b * kmax + j0 + j, o2 = (size_t)r2 * kmax + j0 + j;
+                e1[j] = in ? idx[o1] : -1;
+                p1[j] = in ? pos[o1] : 0;
+                w1[j] = in ? wts[o1] : 0.f;
+                e2[j] = in && grouped ? idx[o2] : -1;
+                p2[j] = in && grouped ? pos[o2] : 0;
+                w2[j] = in && grouped ? wts[o2] : 0.f;
+            }
+#pragma unroll
+            for (int j = 0; j < KM; j++) {
+                if (e1[j] < 0) w1[j] = 0.f;
+                if (e2[j] < 0) w2[j] = 0.f;
+                y1[j] = e1[j] >= 0 ? __ldcg(Ys + (size_t)p1[j] * d + i) : 0.f;
+                y2[j] = e2[j] >= 0 ? __ldcg(Ys + (size_t)p2[j] * d + i) : 0.f;
             }
 #pragma unroll
             for (int j = 0; j < KM; j++) {
@@ -696,22 +726,29 @@ __global__ void __launch_bounds__(256) moe_combine_sorted_kernel(const float *Ys
             }
         }
         if (Psh) {
-            const size_t offs[2] = {(size_t)b * d + i, (size_t)(grouped && !gate_g ? r2 : b) * d + i};
-            float sm[2];
-            sum_splits_k<2, 8>(Psh, split_stride, nsplit, offs, sm);
+            float sm[2] = {0.f, 0.f};
+            if (early) {
+#pragma unroll
+                for (int sp = 0; sp < 8; sp++) {
+                    sm[0] += pv[sp][0];
+                    sm[1] += pv[sp][1];
+                }
+            } else {
+                sum_splits_k<2, 8>(Psh, split_stride, nsplit, offs, sm);
+            }
             m1 += sm[0];
             m2 += gate_g ? gate_g[i] * sm[0] : sm[1];
         }
         const float gn = Xn ? g_next[i] : 0.f;
         if (first) {
-            const float v1 = S[(size_t)b * d + i] + m1;
+            const float v1 = s1_in + m1;
             S[(size_t)b * d + i] = v1;
             if (Xn) store_split(Xn, (size_t)b * d + i, lo_off, gn * v1);
             q1 += v1 * v1;
         }
         if (grouped) {
             if (!gate_g) m2 += coup_c[i] * m1;
-            const float v2 = S[(size_t)r2 * d + i] + m2;
+            const float v2 = s2_in + m2;
             S[(size_t)r2 * d + i] = v2;
             if (Xn) store_split(Xn, (size_t)r2 * d + i, lo_off, gn * v2);
             q2 += v2 * v2;

@@ -729,38 +729,57 @@ __global__ void __launch_bounds__(32) route_kernel(const float *logits, int nspl
     int path = r / Bc;  // 0 primary, j >= 1 decode branch j (each branch routes for itself, fan-out k_b)
     int sel_row = (path && replay) ? r % Bc : r;
     int k = (path && !replay) ? k_b : k_p;
+    // One round of loads: the row's norm shares and every split of this lane's experts are requested before
+    // anything is added (16 splits x 2 experts in flight; the sums still run in split order).  Replay reads the
+    // primary twin's logits too; otherwise the selection row is the row itself.
+    const bool twin = sel_row != r;
+    float ssa = 0.f, ssb = 0.f;
+    if (ss)
+        for (int t = lane; t < ss_tiles; t += 32) {
+            ssa += __ldcg(ss + (size_t)t * ss_ld + r);
+            if (twin) ssb += __ldcg(ss + (size_t)t * ss_ld + sel_row);
+        }
+    for (int e0 = 0; e0 < E; e0 += 64) {
+        float a[2] = {0.f, 0.f}, b2[2] = {0.f, 0.f};
+        for (int s0 = 0; s0 < nsplit; s0 += 16) {
+            float va[2][16], vb[2][16];
+#pragma unroll
+            for (int u = 0; u < 2; u++)
+#pragma unroll
+                for (int j = 0; j < 16; j++) {
+                    const int e = e0 + u * 32 + lane;
+                    const bool on = e < E && s0 + j < nsplit;
+                    va[u][j] = on ? __ldcg(logits + (size_t)(s0 + j) * split_stride + (size_t)r * E + e) : 0.f;
+                    vb[u][j] = on && twin ? __ldcg(logits + (size_t)(s0 + j) * split_stride + (size_t)sel_row * E + e) : 0.f;
+                }
+#pragma unroll
+            for (int u = 0; u < 2; u++)
+#pragma unroll
+                for (int j = 0; j < 16; j++) {
+                    a[u] += va[u][j];
+                    b2[u] += vb[u][j];
+                }
+        }
+#pragma unroll
+        for (int u = 0; u < 2; u++) {
+            const int e = e0 + u * 32 + lane;
+            if (e < E) {
+                own[e] = a[u];
+                sel[e] = twin ? b2[u] : a[u];
+            }
+        }
+    }
     float inv_own = 1.f, inv_sel = 1.f;
     if (ss) {
-        float a = 0.f, b2 = 0.f;
-        for (int t = lane; t < ss_tiles; t += 32) {
-            a += __ldcg(ss + (size_t)t * ss_ld + r);
-            b2 += __ldcg(ss + (size_t)t * ss_ld + sel_row);
-        }
-        inv_own = 1.f / sqrtf(warp_sum(a) / (float)d_norm + eps);
-        inv_sel = 1.f / sqrtf(warp_sum(b2) / (float)d_norm + eps);
+        inv_own = 1.f / sqrtf(warp_sum(ssa) / (float)d_norm + eps);
+        inv_sel = twin ? 1.f / sqrtf(warp_sum(ssb) / (float)d_norm + eps) : inv_own;
     }
     float mx = -INFINITY;
     for (int e = lane; e < E; e += 32) {
-        float a = 0.f, b2 = 0.f;
-        for (int s0 = 0; s0 < nsplit; s0 += 8) {  // eight splits of both rows in flight, added in split order
-            float va[8], vb[8];
-#pragma unroll
-            for (int j = 0; j < 8; j++) {
-                bool on = s0 + j < nsplit;
-                va[j] = on ? __ldcg(logits + (size_t)(s0 + j) * split_stride + (size_t)r * E + e) : 0.f;
-                vb[j] = on ? __ldcg(logits + (size_t)(s0 + j) * split_stride + (size_t)sel_row * E + e) : 0.f;
-            }
-#pragma unroll
-            for (int j = 0; j < 8; j++) {
-                a += va[j];
-                b2 += vb[j];
-            }
-        }
-        a *= inv_own;
-        b2 *= inv_sel;
-        own[e] = a;
-        sel[e] = b2;
-        mx = fmaxf(mx, a);
+        const float x = own[e] * inv_own;
+        own[e] = x;
+        sel[e] *= inv_sel;
+        mx = fmaxf(mx, x);
     }
     mx = warp_max(mx);
     float sum = 0.f;
