@@ -581,6 +581,7 @@ struct TcCall {
     const int *grp_cnt, *grp_off;  // per-expert mode (see TcParams); n_groups experts
     int grp_w_rows, n_groups;
     int grp_row_tiles;  // per-expert mode: row tiles of n_tile rows per expert (0: one tile holds any list)
+    int grp_prewait;    // per-expert mode: the lists are final before this launch can be resident (see TcParams)
 };
 
 int norm_threads(int d) { return d >= 1024 ? 1024 : d >= 512 ? 512 : 256; }
@@ -669,6 +670,7 @@ dbt_status run_gemm_tc(dbt_model *m, const TcCall &c, int n_tile, int *nsplit_ou
     p.grp_off = c.grp_off;
     p.grp_w_rows = c.grp_w_rows;
     p.grp_row_tiles = c.grp_cnt ? c.grp_row_tiles : 0;
+    p.grp_prewait = c.grp_cnt ? c.grp_prewait : 0;
     p.P = c.P;
     p.status = m->ws.status;
     p.evict_first = m->evict_first ? 1 : 0;
@@ -923,6 +925,7 @@ dbt_status run_moe_tc(dbt_model *m, int l, const RowMap &rm, int grouped, bool r
         grt = (R + gt - 1) / gt;
     }
     gu.grp_row_tiles = grt;
+    gu.grp_prewait = m->use_pdl ? 1 : 0;  // the gather kernel before it lets its dependents in only after its own wait
     if ((st = run_gemm_tc(m, gu, gt, nullptr, nullptr)) != DBT_OK) return st;
     LAUNCH(m, "moe_swiglu", 0, moe_swiglu_kernel, dim3(R * km, (Fe + 255) / 256), 256, 0, w.Pe, w.eoff + E, Fe, w.Hs, lo_hs,
            wide ? (const float *)w.rs_sorted : (const float *)nullptr);
@@ -931,6 +934,10 @@ dbt_status run_moe_tc(dbt_model *m, int l, const RowMap &rm, int grouped, bool r
     dn.P = w.Yexp; dn.P_floats = (size_t)Rk * d; dn.tag = "expert_down"; dn.parts = m->act_parts; dn.lo_row0 = Rk;
     dn.grp_cnt = w.ecnt; dn.grp_off = w.eoff; dn.grp_w_rows = d; dn.n_groups = E;
     dn.grp_row_tiles = grt;
+    // The lists come from the sort kernel, four launches back.  A CTA of this launch can only be resident once every
+    // CTA of the SwiGLU kernel has started, hence once every CTA of the gate|up GEMM has passed its own dependency
+    // wait (it waits before anything else), hence after the gather kernel -- and the sort kernel before it -- ended.
+    dn.grp_prewait = m->use_pdl ? 1 : 0;
     if ((st = run_gemm_tc(m, dn, gt, nullptr, nullptr)) != DBT_OK) return st;
     if (Fs > 0 && !overlap && (st = shared_expert(w.P, w.P_floats)) != DBT_OK) return st;
     if (overlap) CUDA_TRY(m, cudaStreamWaitEvent(main_stream, m->ev_join, 0));

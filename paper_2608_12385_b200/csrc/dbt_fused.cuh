@@ -623,7 +623,10 @@ __global__ void __launch_bounds__(256) moe_gather_kernel(const __nv_bfloat16 *Xb
                                                          size_t lo_out, const float *ss, int ss_tiles, int ss_ld,
                                                          float eps, float *rs_sorted) {
     DBT_TL_DECL;
-    pdl_enter();
+    // Wait first, then let the per-expert GEMM in: by the time one of its CTAs is resident the sort kernel's lists
+    // are final, so it may read them (and request its first weight tiles) before its own dependency wait.
+    pdl_wait();
+    pdl_launch_dependents();
     DBT_TL_WAITED;
     int entry = blockIdx.x;
     if (idx[entry] < 0) return;

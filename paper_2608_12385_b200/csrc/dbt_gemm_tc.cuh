@@ -55,6 +55,10 @@ struct TcParams {
     // grouped mode with row tiles: blockIdx.y = which N_TILE rows of the expert's list (CTAs past the
     // list's end leave at once); 0: the whole list fits one tile and blockIdx.y is the split as usual
     int grp_row_tiles;
+    // grouped mode: 1 = the row lists were written at least three kernels before this one (by a kernel that the
+    // launch chain guarantees complete before any CTA of this launch can be resident), so they may be read, and
+    // the first ring of weight tiles requested, before the dependency wait
+    int grp_prewait;
     // dense mode with more rows than one tile holds (prompt chunks): blockIdx.x = weight tile * row_tiles + row
     // tile, so that the CTAs sharing a weight tile are neighbours in launch order and all but the first find it
     // in L2; 0 or 1: blockIdx.x is the weight tile
@@ -239,8 +243,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
         tile = blockIdx.x / p.row_tiles;
     }
     if (p.grp_cnt) {
-        // the expert's row list comes from the previous kernel: nothing can start before it is known
-        pdl_wait();
+        // the expert's row list comes from an earlier kernel: nothing can start before it is known
+        if (!p.grp_prewait) pdl_wait();
         grp_n = ld_mut(p.grp_cnt + blockIdx.z);
         if (grp_n == 0) return;  // expert not selected by any row of either path: its weights are not read
         x_row0 = ld_mut(p.grp_off + blockIdx.z);
