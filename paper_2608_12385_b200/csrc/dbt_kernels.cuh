@@ -769,6 +769,7 @@ __global__ void __launch_bounds__(32) route_kernel(const float *logits, int nspl
             }
         }
     }
+    DBT_TL_MARK(0);
     float inv_own = 1.f, inv_sel = 1.f;
     if (ss) {
         inv_own = 1.f / sqrtf(warp_sum(ssa) / (float)d_norm + eps);
@@ -790,6 +791,7 @@ __global__ void __launch_bounds__(32) route_kernel(const float *logits, int nspl
     }
     sum = warp_sum(sum);
     __syncwarp();
+    DBT_TL_MARK(1);
     float tot = 0.f;
     int mine = -1;  // lane j keeps the j-th selection (k <= 64: two rounds of lanes at most)
     int mine2 = -1;
@@ -818,6 +820,7 @@ __global__ void __launch_bounds__(32) route_kernel(const float *logits, int nspl
         if (j == lane) mine = bi;
         if (j == lane + 32) mine2 = bi;
     }
+    DBT_TL_MARK(2);
     for (int j = lane; j < kmax; j += 32) {
         int e = j < k ? (j < 32 ? mine : mine2) : -1;
         idx[(size_t)r * kmax + j] = e;
