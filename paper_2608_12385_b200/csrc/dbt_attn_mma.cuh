@@ -434,6 +434,8 @@ __global__ void __launch_bounds__(160, DEEP ? 1 : 2) attn_mma_kernel(const __gri
             const int nitems = p.G * half;
             const bool do_kv = owns_last && tid < half;
             float *rs_s = reinterpret_cast<float *>(flag + 8);  // [path]
+            // the page of this step's position: requested with the first round of loads, used after it
+            const int page_new = do_kv ? __ldg(p.page_table + (size_t)p.rm.seq(item) * p.pt_stride + (pos >> 4)) : 0;
             float rs1 = 1.f, rs2 = 1.f, kvs[4] = {0.f, 0.f, 0.f, 0.f};
             float2 t_kv = make_float2(1.f, 0.f);
             for (int it0 = 0; it0 * 128 < nitems; it0++) {
@@ -511,7 +513,7 @@ __global__ void __launch_bounds__(160, DEEP ? 1 : 2) attn_mma_kernel(const __gri
                 kv_new[i + half] = k1;
                 kv_new[DH + i] = v0;
                 kv_new[DH + i + half] = v1;
-                int page = __ldg(p.page_table + (size_t)p.rm.seq(item) * p.pt_stride + (pos >> 4));
+                const int page = page_new;
                 if (page < 0 || page >= p.num_pages) {
                     if (i == 0) report(p.status, kStatusBadPage, page);
                 } else {

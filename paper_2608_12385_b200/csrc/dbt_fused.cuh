@@ -135,7 +135,9 @@ __global__ void __launch_bounds__(256) resid_wide_kernel(float *S, const float *
         // every load of this thread goes out before the first use: S of both rows and all splits of both
         // rows' partials (up to 16 splits in one round)
         size_t o1 = (size_t)b * d + i, o2 = (size_t)r2 * d + i;
-        float s1 = first ? __ldcg(S + o1) : 0.f, s2 = grouped ? __ldcg(S + o2) : 0.f;
+        // (the primary row is loaded by every branch's block, stored by the first: a predicate on the load would
+        // split this round of loads)
+        float s1 = __ldcg(S + o1), s2 = grouped ? __ldcg(S + o2) : 0.f;
         const size_t offs[2] = {o1, grouped && mode != 3 ? o2 : o1};
         float mm[2];
         sum_splits_k<2, 16>(P, split_stride, nsplit, offs, mm);

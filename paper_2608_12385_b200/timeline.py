@@ -66,6 +66,7 @@ def main():
     ap.add_argument("--batch", type=int, default=16)
     ap.add_argument("--ctx", type=int, default=2048)
     ap.add_argument("--layers", type=int, default=0)
+    ap.add_argument("--paths", type=int, default=2, help="residual paths K (the primary plus K-1 decode branches)")
     ap.add_argument("--primary-only", action="store_true")
     ap.add_argument("--out", default="")
     args = ap.parse_args()
@@ -74,6 +75,8 @@ def main():
     cfg = PRESETS[args.model]()
     if args.layers:
         cfg = cfg.replace(n_layers=args.layers)
+    if args.paths != 2:
+        cfg = cfg.replace(n_paths=args.paths)
     w = make_weights(cfg, seed=0)
     B, S = args.batch, args.ctx
     m = binding.Model(cfg, binding.weights_to_device(w), B, S + 64)
