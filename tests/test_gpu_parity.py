@@ -692,13 +692,43 @@ def test_compute_matched_moe_on_the_alternative_chains(monkeypatch, knob, value)
 
 
 @pytest.mark.parametrize("knob,value", [("DBT_MOE_OVERLAP", "0"), ("DBT_GRAPH", "0"), ("DBT_MOE", "simt"),
-                                        ("DBT_FUSE_QKV", "0"), ("DBT_ATTN", "simt")])
+                                        ("DBT_FUSE_QKV", "0"), ("DBT_ATTN", "simt"), ("DBT_MOE_PERSIST", "0"),
+                                        ("DBT_MOE_PERSIST", "1")])
 def test_moe_on_the_alternative_chains(monkeypatch, knob, value):
     """The shared expert on the main stream instead of beside the routed chain, direct launches instead
     of graph replay, the CUDA-core expert kernels, the separate Q|K|V epilogue kernel, the CUDA-core
-    attention kernel."""
+    attention kernel, the per-expert GEMMs as one CTA per unit / as persistent CTAs (the default takes the
+    persistent form up to 16 stacked rows)."""
     monkeypatch.setenv(knob, value)
     _moe_compare(small_moe(), B=5, T=13, npre=9)
+
+
+@pytest.mark.parametrize("cfg,B", [(small_moe(), 5), (small_moe(k_branch=8, n_shared_experts=0), 3),
+                                   (moe_1b(k_branch=2).replace(n_layers=2), 12), (small_moe(n_paths=3), 20)])
+def test_persistent_per_expert_gemm_gives_the_same_bits(monkeypatch, cfg, B):
+    """Both forms of the per-expert GEMM launch add the same products in the same order: logits, expert choice
+    and cache are the same bits (row tiles of 16 and of 32 rows, several row tiles per expert at batch 20 x 3
+    paths, grouped and primary-only steps)."""
+    w = make_weights(cfg, seed=71, matrix_std=0.02 if cfg.d_model > 1000 else 0.05)
+    T, npre = 9, 6
+    tok = make_tokens(cfg, B, T, seed=72).cuda()
+    wd = binding.weights_to_device(w)
+    runs = {}
+    for value in ("0", "1"):
+        monkeypatch.setenv("DBT_MOE_PERSIST", value)
+        for grouped in (True, False):
+            gm = binding.Model(cfg, wd, B, T)
+            outs = _run_steps(gm, tok, npre, grouped)
+            runs[value, grouped] = (outs, gm.export_kv(B, T), gm.last_experts(B))
+            assert gm.sync_status() == (0, 0)
+    for grouped in (True, False):
+        (oa, kva, ea), (ob, kvb, eb) = runs["0", grouped], runs["1", grouped]
+        for x, y in zip(oa, ob):
+            assert torch.equal(x["z1"], y["z1"])
+            if grouped:
+                assert torch.equal(x["z2"], y["z2"])
+        assert torch.equal(kva[0].float(), kvb[0].float()) and torch.equal(kva[1].float(), kvb[1].float())
+        assert torch.equal(ea, eb)
 
 
 def test_compute_matched_moe_1b_shape_two_layers():
