@@ -248,6 +248,60 @@ def test_1b_at_the_benchmarks_launch_configuration_on_sampled_sequences():
     assert gm.sync_status() == (0, 0)
 
 
+def test_1b_width_three_paths_at_batch_16_on_sampled_sequences():
+    """Appendix C.1 at the benchmark's batch and the 1B model's width (four of its layers, context 700): three
+    residual paths, i.e. 48 stacked rows in 64-row GEMM tiles, six query rows per KV head in the one-wave
+    attention form, a block per branch in the kernels between the GEMMs, two branch distributions in the
+    readout.  Sequences 3 and 14 against the oracle run on them alone."""
+    cfg = dense_1b().replace(n_layers=4, n_paths=3)
+    w = make_weights(cfg, seed=0)
+    B, ctx, pick = 16, 700, [3, 14]
+    tok = make_tokens(cfg, B, 2, seed=2)
+    k, v = make_synthetic_kv(cfg, len(pick), ctx, seed=3)
+    gm = make_gpu_model(cfg, w, B, ctx + 3)
+    gen = torch.Generator(device=gm.device)
+    gen.manual_seed(5)
+    gm.kv_pool.normal_(0.0, 1.0, generator=gen)
+    gm.import_kv(k, v, seq_ids=pick)
+    gm.set_seq_lens([ctx] * B)
+    om = oracle.OracleModel(cfg, w, len(pick), ctx + 3)
+    om.inject_kv(k, v, ctx)
+    for t in range(2):
+        o = om.decode_step(tok[pick, t].numpy())
+        g = gm.decode_full(tok[:, t].cuda().contiguous())
+        assert_logits_close(g["z1"][pick], o["z1"], "bf16", f"K=3 step {t} z1")
+        for j in range(2):
+            assert_logits_close(g["z2"][j][pick], o["z2"][j], "bf16", f"K=3 step {t} branch {j + 2}")
+        np.testing.assert_allclose(g["alpha"][pick].cpu().numpy(), o["alpha"], rtol=1e-3)
+    assert gm.sync_status() == (0, 0)
+
+
+def test_8b_width_prompt_pass_with_two_weight_tiles_per_cta():
+    """The prompt pass at the 8B shape's width (one layer; d 4096, 32 query / 8 KV heads of 128, F 14336): two
+    sequences of 520 positions are one chunk of 1040 rows = five row tiles, where every GEMM of the layer takes
+    two weight tiles per CTA (the Q|K|V launch across its three weight matrices), and the prompt attention
+    kernel runs four heads per KV head.  Last-position logits and the cache against the oracle, then a grouped
+    step on the device's cache."""
+    from paper_2608_12385_b200.inputs import dense_8b
+    cfg = dense_8b().replace(n_layers=1)
+    w = make_weights(cfg, seed=0)
+    B, n = 2, 520
+    tok = make_tokens(cfg, B, n + 1, seed=2)
+    om = oracle.OracleModel(cfg, w, B, n + 1)
+    gm = make_gpu_model(cfg, w, B, n + 1)
+    want = om.prefill(tok[:, :n].numpy())
+    got = gm.prefill(tok[:, :n].cuda().contiguous(), want_logits=True)
+    assert_logits_close(got, want, "bf16", "8B-width prefill logits")
+    k_dev, v_dev = gm.export_kv(B, n)
+    np.testing.assert_allclose(k_dev.float().numpy(), om.k_cache[:, :B, :n], rtol=2.0 ** -8, atol=5e-3)
+    np.testing.assert_allclose(v_dev.float().numpy(), om.v_cache[:, :B, :n], rtol=2.0 ** -8, atol=5e-3)
+    o = om.decode_step(tok[:, n].numpy())
+    g = gm.decode_full(tok[:, n].cuda().contiguous())
+    assert_logits_close(g["z1"], o["z1"], "bf16", "step after prefill z1")
+    assert_logits_close(g["z2"], o["z2"], "bf16", "step after prefill z2")
+    assert gm.sync_status() == (0, 0)
+
+
 # ---- readout off the clip of alpha (Eq. alpha, Eq. mixloss) ---------------------------------------------------
 
 @pytest.mark.parametrize("cfg,matrix_std", [(small_bf16(), 0.05), (tiny_dense_fp32(), 0.02), (small_bf16(n_paths=3), 0.05)])
