@@ -155,7 +155,8 @@ int kmax_of(const dbt_config &c) { return c.k_primary > c.k_branch ? c.k_primary
 // prefill (2048 rows for dense bf16 models, whose GEMMs sweep several row tiles per weight tile and whose
 // causal attention packs consecutive positions into a query tile; 256 otherwise).
 int prefill_rows(const dbt_config &c) {
-    int chunk = (c.weight_dtype == DBT_DTYPE_BF16 && c.n_experts == 0) ? 2048 : 256;
+    // rows of a prompt chunk: bf16 models 2048, everything else 256
+    int chunk = c.weight_dtype != DBT_DTYPE_BF16 ? 256 : 2048;
     return paths_of(c) * c.max_batch > chunk ? paths_of(c) * c.max_batch : chunk;
 }
 
@@ -585,6 +586,7 @@ struct TcCall {
     int grp_w_rows, n_groups;
     int grp_row_tiles;  // per-expert mode: row tiles of n_tile rows per expert (0: one tile holds any list)
     int grp_prewait;    // per-expert mode: the lists are final before this launch can be resident (see TcParams)
+    int grp_mt2;        // per-expert mode, 64-row tiles: two weight tiles per CTA share each activation box (prompt chunks)
 };
 
 int norm_threads(int d) { return d >= 1024 ? 1024 : d >= 512 ? 512 : 256; }
@@ -671,6 +673,7 @@ dbt_status run_gemm_tc(dbt_model *m, const TcCall &c, int n_tile, int *nsplit_ou
         const int w1 = (t1 * rt + sms - 1) / sms, w2 = (t2 * rt + sms - 1) / sms;
         if (16 * w2 < 10 * w1) mt = 2;
     }
+    if (c.grp_cnt && c.grp_mt2 && n_tile == 64) mt = 2;
     for (int s = 0; s < c.nseg; s++) {
         p.seg[s] = TcSeg{tiles, c.n_out[s], c.rows[s], col};
         tiles += (c.n_out[s] + kTcM * mt - 1) / (kTcM * mt);
@@ -718,7 +721,7 @@ dbt_status run_gemm_tc(dbt_model *m, const TcCall &c, int n_tile, int *nsplit_ou
     switch (n_tile) {
         case 16: return launch_gemm_tc<16>(m, c, p, e, grid, bytes);
         case 32: return launch_gemm_tc<32>(m, c, p, e, grid, bytes);
-        case 64: return launch_gemm_tc<64>(m, c, p, e, grid, bytes);
+        case 64: return mt == 2 ? launch_gemm_tc<64, 2>(m, c, p, e, grid, bytes) : launch_gemm_tc<64>(m, c, p, e, grid, bytes);
         case 128: return launch_gemm_tc<128>(m, c, p, e, grid, bytes);
         case 256: return mt == 2 ? launch_gemm_tc<256, 2>(m, c, p, e, grid, bytes) : launch_gemm_tc<256>(m, c, p, e, grid, bytes);
     }
@@ -920,7 +923,7 @@ dbt_status run_moe_tc(dbt_model *m, int l, const RowMap &rm, int grouped, bool r
                                     m->stream));
     LAUNCH(m, "route", 0, route_kernel, R, 32, 2 * E * sizeof(float), w.P, rnsp, rstride, E, Bc, c.k_primary, c.k_branch, km,
            c.router_mode == DBT_ROUTER_REPLAY, w.ridx, w.rwts, last, c.max_batch * km, ssp, ss_tiles, ss_ld, d, c.rms_eps);
-    LAUNCH(m, "moe_sort", 0, moe_sort_kernel, 1, (E + 31) / 32 * 32 < 64 ? 64 : (E + 31) / 32 * 32, 0, w.ridx, R, km, E, w.ecnt, w.eoff, w.epos,
+    LAUNCH(m, "moe_sort", 0, moe_sort_kernel, 1, R * km > 512 ? 1024 : (E + 31) / 32 * 32 < 64 ? 64 : (E + 31) / 32 * 32, 0, w.ridx, R, km, E, w.ecnt, w.eoff, w.epos,
            record_experts ? w.union_cnt + l : (int32_t *)nullptr);
     LAUNCH(m, "moe_gather", 0, moe_gather_kernel, R * km, 256, 0, w.Xb, lo_x, w.ridx, w.epos, km, d, w.Xs, lo_xs, ssp, ss_tiles, ss_ld,
            c.rms_eps, w.rs_sorted);
@@ -937,12 +940,14 @@ dbt_status run_moe_tc(dbt_model *m, int l, const RowMap &rm, int grouped, bool r
     // could need, keep two CTAs per SM and their deeper rings at large batches (measured: 4.86 -> 4.53 ms
     // at batch 32, 6.43 -> 4.81 at batch 64).  DBT_MOE_ROWTILE=0: one tile of all rows; 16/32/64: that tile.
     int gt = n_tile, grt = 0;
-    const int want_tile = m->moe_row_tile >= 0 ? m->moe_row_tile : (paths_of(c) * Bc <= 64 ? 16 : 32);
+    // (prompt chunks of more than 256 rows: tiles of 64 rows, an expert's share of such a chunk)
+    const int want_tile = m->moe_row_tile >= 0 ? m->moe_row_tile : (paths_of(c) * Bc <= 64 ? 16 : Bc <= 256 ? 32 : 64);
     if (want_tile > 0 && n_tile > want_tile) {
         gt = want_tile;
         grt = (R + gt - 1) / gt;
     }
     gu.grp_row_tiles = grt;
+    gu.grp_mt2 = (gt == 64 && Bc > 256) ? 1 : 0;
     gu.grp_prewait = m->use_pdl ? 1 : 0;  // the gather kernel before it lets its dependents in only after its own wait
     if ((st = run_gemm_tc(m, gu, gt, nullptr, nullptr)) != DBT_OK) return st;
     LAUNCH(m, "moe_swiglu", 0, moe_swiglu_kernel, dim3(R * km, (Fe + 255) / 256), 256, 0, w.Pe, w.eoff + E, Fe, w.Hs, lo_hs,
@@ -952,6 +957,7 @@ dbt_status run_moe_tc(dbt_model *m, int l, const RowMap &rm, int grouped, bool r
     dn.P = w.Yexp; dn.P_floats = (size_t)Rk * d; dn.tag = "expert_down"; dn.parts = m->act_parts; dn.lo_row0 = Rk;
     dn.grp_cnt = w.ecnt; dn.grp_off = w.eoff; dn.grp_w_rows = d; dn.n_groups = E;
     dn.grp_row_tiles = grt;
+    dn.grp_mt2 = gu.grp_mt2;
     // The lists come from the sort kernel, four launches back.  A CTA of this launch can only be resident once every
     // CTA of the SwiGLU kernel has started, hence once every CTA of the gate|up GEMM has passed its own dependency
     // wait (it waits before anything else), hence after the gather kernel -- and the sort kernel before it -- ended.
@@ -960,6 +966,12 @@ dbt_status run_moe_tc(dbt_model *m, int l, const RowMap &rm, int grouped, bool r
     if (Fs > 0 && !overlap && (st = shared_expert(w.P, w.P_floats)) != DBT_OK) return st;
     if (overlap) CUDA_TRY(m, cudaStreamWaitEvent(main_stream, m->ev_join, 0));
     const bool next_in = wide && g_next != nullptr;
+    if (!grouped && wide && rm.cn > 1 && Bc > 256 && d % 4 == 0 && ((size_t)m->Rmax * d) % 4 == 0) {  // prompt chunks: the vector form
+        LAUNCH(m, "moe_combine", 0, moe_combine_rows_kernel, dim3((Bc + 3) / 4, (d + 255) / 256), 256, 0, w.Yexp, Psh, nsp, sstride, w.ridx,
+               w.epos, w.rwts, km, Bc, d, w.S, next_in ? g_next : (const float *)nullptr, next_in ? w.Xb : (__nv_bfloat16 *)nullptr, lo_x,
+               next_in ? w.ss : (float *)nullptr, ss_ld);
+        return DBT_OK;
+    }
     LAUNCH_BR(m, grouped, "moe_combine", 0, moe_combine_sorted_kernel, dim3(Bc, (d + 255) / 256, branch_blocks(grouped)), 256, 0, w.Yexp, Psh, nsp, sstride, w.ridx, w.epos, w.rwts, km,
            Bc, grouped, lw.coup_c, matched ? lw.gate_g : (const float *)nullptr, d, w.S, next_in ? g_next : (const float *)nullptr,
            next_in ? w.Xb : (__nv_bfloat16 *)nullptr, lo_x, next_in ? w.ss : (float *)nullptr, ss_ld);
@@ -991,6 +1003,10 @@ dbt_status run_layers_tc(dbt_model *m, const RowMap &rm, int grouped, int n_tile
     const bool mwide = moe && m->moe_tc && m->moe_wide;
     const int mss_tiles = (d + 255) / 256;
     size_t lo_x = m->act_parts == 2 ? (size_t)m->Rmax * d : 0;
+    // prompt chunks of more than one row tile (MoE models): the prompt attention kernel and the vector forms of the
+    // kernels around it, as in the dense prompt pass
+    const bool rows_form = mwide && m->att_fast && !grouped && rm.cn > 1 && Bc > 256 && d % 4 == 0 && c.head_dim % 8 == 0 &&
+                           ((size_t)m->Rmax * d) % 4 == 0;
     dbt_status st;
     int mode = 0, nsp = 1;
     size_t sstride = 0;
@@ -1019,14 +1035,19 @@ dbt_status run_layers_tc(dbt_model *m, const RowMap &rm, int grouped, int n_tile
         if ((st = run_gemm_tc(m, qkv, n_tile, &nsp, &sstride)) != DBT_OK) return st;
         const bool fuse = m->fuse_qkv && m->att_fast && rm.cn == 1;
         QkvFuse qf{w.P, nsp, sstride, mwide ? w.ss : nullptr, mwide ? mss_tiles : 0, mwide ? m->Rmax : 0, lw.coup_a};
-        if (!fuse)
+        if (rows_form)
+            LAUNCH(m, "qkv_epilogue", 0, qkv_rows_kernel, dim3(Bc, ((c.n_q_heads + c.n_kv_heads) * (c.head_dim / 8) + 255) / 256), 256, 0,
+                   w.P, nsp, sstride, w.Q, rm, c.n_q_heads, c.n_kv_heads, c.head_dim, w.rope, w.seq_len, w.page_table,
+                   m->pages_per_seq_max, c.num_pages, c.page_size, kpool, vpool, w.status, (const float *)w.ss, mss_tiles, m->Rmax, d,
+                   c.rms_eps);
+        else if (!fuse)
             LAUNCH(m, "qkv_epilogue", 0, qkv_epilogue_kernel<WT>, dim3(Bc, c.n_q_heads + c.n_kv_heads, branch_blocks(ga)), 64, 0, w.P, nsp, sstride, w.Q, rm, ga, c.n_q_heads,
                    c.n_kv_heads, c.head_dim, lw.coup_a, w.rope, w.seq_len, w.page_table, m->pages_per_seq_max, c.num_pages,
                    c.page_size, kpool, vpool, w.status, mwide ? (const float *)w.ss : (const float *)nullptr, mwide ? mss_tiles : 0,
                    mwide ? m->Rmax : 0, d, c.rms_eps);
         if (m->att_fast)
-            st = c.head_dim == 128 ? run_attention_mma<128>(m, rm, ga, l, kv_bytes, fuse ? &qf : nullptr, false, m->att_planned)
-                                   : run_attention_mma<64>(m, rm, ga, l, kv_bytes, fuse ? &qf : nullptr, false, m->att_planned);
+            st = c.head_dim == 128 ? run_attention_mma<128>(m, rm, ga, l, kv_bytes, fuse ? &qf : nullptr, rows_form, m->att_planned)
+                                   : run_attention_mma<64>(m, rm, ga, l, kv_bytes, fuse ? &qf : nullptr, rows_form, m->att_planned);
         else if (c.head_dim == 128)
             st = run_attention<WT, 128>(m, rm, ga, kpool, vpool, att_split, kv_bytes, true);
         else
@@ -1037,7 +1058,10 @@ dbt_status run_layers_tc(dbt_model *m, const RowMap &rm, int grouped, int n_tile
         op.P = w.P; op.P_floats = w.P_floats; op.parts = m->act_parts; op.lo_row0 = m->Rmax; op.tag = "gemm_o";
         if ((st = run_gemm_tc(m, op, n_tile, &nsp, &sstride)) != DBT_OK) return st;
         // S-bar_i = S_i + Attn_i W_O (matched: S-bar_2 = S_2 + g_A * Attn_1 W_O) ; RMSNorm for the MLP
-        if (mwide)
+        if (rows_form)
+            LAUNCH(m, "resid_wide", 0, resid_rows_kernel, dim3((Bc + 3) / 4, mss_tiles), 256, 0, w.S, w.P, nsp, sstride, lw.mlp_norm_g, Bc, d,
+                   w.Xb, lo_x, w.ss, m->Rmax);
+        else if (mwide)
             LAUNCH_BR(m, grouped, "resid_wide", 0, resid_wide_kernel, dim3(Bc, mss_tiles, branch_blocks(grouped)), 256, 0, w.S, w.P, nsp, sstride, matched ? 3 : 1,
                    matched ? lw.gate_a : (const float *)nullptr, Bc, grouped, lw.mlp_norm_g, d, w.Xb, lo_x, w.ss, m->Rmax);
         else
@@ -1123,7 +1147,10 @@ dbt_status prefill_tc(dbt_model *m, const int32_t *tokens_dev, int B, int n, flo
     typedef __nv_bfloat16 WT;
     const dbt_config &c = m->cfg;
     const Workspace &w = m->ws;
-    int cn_max = m->Rmax / B;
+    // chunks of up to Rmax rows where every kernel of the chain takes more than one row tile (the tensor-core MoE
+    // chain with the norm factor behind the GEMMs); 256 rows otherwise
+    const bool big = c.n_experts > 0 && m->moe_tc && m->moe_wide && m->att_fast;
+    int cn_max = (big ? m->Rmax : (m->Rmax < 256 ? m->Rmax : 256)) / B;
     if (cn_max < 1) cn_max = 1;
     dbt_status st;
     for (int p0 = 0; p0 < n; p0 += cn_max) {
@@ -1337,6 +1364,8 @@ bool allow_smem() {
 bool allow_smem_all() {
     return allow_smem<16>() && allow_smem<32>() && allow_smem<64>() && allow_smem<128>() && allow_smem<256>() &&
            cudaFuncSetAttribute(gemm_tc_kernel<256, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcCfg<256, 2>::kSmemBytes) ==
+               cudaSuccess &&
+           cudaFuncSetAttribute(gemm_tc_kernel<64, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcCfg<64, 2>::kSmemBytes) ==
                cudaSuccess;
 }
 

@@ -577,15 +577,31 @@ __global__ void __launch_bounds__(1024) moe_sort_kernel(const int32_t *idx, int 
     __shared__ int s_wsum[32];
     __shared__ int s_idx[4096];  // the selections, staged once (larger lists are read from global memory)
     const int n = R * kmax;
-    const bool staged = n <= 4096;
+    // Long lists (prompt chunks, large batches): counts and positions through shared-memory atomics by all
+    // threads.  The order of an expert's rows is then arbitrary, which no value depends on (every row's products
+    // are its own, whatever its place in the tile).  Short lists keep the ascending order below.
+    const bool parallel = n > 512;
+    __shared__ int s_cnt[1024], s_fill[1024];
+    const bool staged = !parallel && n <= 4096;
     if (staged)
         for (int i = threadIdx.x; i < n; i += blockDim.x) s_idx[i] = idx[i];
+    if (parallel) {
+        for (int i = threadIdx.x; i < 1024; i += blockDim.x) s_cnt[i] = 0;
+        __syncthreads();
+        for (int i = threadIdx.x; i < n; i += blockDim.x) {
+            const int ex = idx[i];
+            if (ex >= 0 && ex < E) atomicAdd(&s_cnt[ex], 1);
+        }
+    }
     __syncthreads();
     const int32_t *src = staged ? s_idx : idx;
     const int e = threadIdx.x, lane = e & 31, wp = e >> 5;
     int c = 0;
-    if (e < E)
+    if (parallel) {
+        c = e < E ? s_cnt[e] : 0;
+    } else if (e < E) {
         for (int i = 0; i < n; i++) c += src[i] == e;
+    }
     int incl = c;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -608,9 +624,20 @@ __global__ void __launch_bounds__(1024) moe_sort_kernel(const int32_t *idx, int 
     if (e < E) {
         cnt[e] = c;
         off[e] = my_off;
-        int k = 0;
-        for (int i = 0; i < n && k < c; i++)
-            if (src[i] == e) pos[i] = my_off + k++;
+        if (parallel) {
+            s_fill[e] = my_off;
+        } else {
+            int k = 0;
+            for (int i = 0; i < n && k < c; i++)
+                if (src[i] == e) pos[i] = my_off + k++;
+        }
+    }
+    if (parallel) {
+        __syncthreads();
+        for (int i = threadIdx.x; i < n; i += blockDim.x) {
+            const int ex = idx[i];
+            if (ex >= 0 && ex < E) pos[i] = atomicAdd(&s_fill[ex], 1);
+        }
     }
     if (e == E - 1) off[E] = my_off + c;
     if (e == 0 && union_count) *union_count = uni;
@@ -779,6 +806,66 @@ __global__ void __launch_bounds__(256) moe_combine_sorted_kernel(const float *Ys
         }
     }
     DBT_TL_END("moe_comb");
+}
+
+// moe_combine_sorted_kernel for R primary rows of a prompt chunk (no branch): S += sum_j w_j Expert_j(m) + G(m); the next
+// layer's GEMM input g_next * S as two planes and the shares of sum(S^2).  grid (ceil(R / 4), d / 256), 64 threads
+// per row, four consecutive columns per thread.  d % 4 == 0.
+__global__ void __launch_bounds__(256) moe_combine_rows_kernel(const float *Ys, const float *Psh, int nsplit, size_t split_stride,
+                                                               const int32_t *idx, const int32_t *pos, const float *wts,
+                                                               int kmax, int R, int d, float *S,
+                                                               const float *__restrict__ g_next, __nv_bfloat16 *Xn,
+                                                               size_t lo_off, float *ss_out, int ss_ld) {
+    pdl_launch_dependents();
+    __shared__ float scratch[8];
+    const int sub = threadIdx.x >> 6, row = blockIdx.x * 4 + sub, i = blockIdx.y * 256 + (threadIdx.x & 63) * 4;
+    const bool act = row < R && i < d;
+    float4 gn = make_float4(1.f, 1.f, 1.f, 1.f);
+    if (act && Xn) gn = *reinterpret_cast<const float4 *>(g_next + i);
+    pdl_wait();
+    float q = 0.f;
+    if (act) {
+        const size_t o = (size_t)row * d + i;
+        float4 s = ldcg4(S + o), m = make_float4(0.f, 0.f, 0.f, 0.f);
+        constexpr int KM = 8;
+        for (int j0 = 0; j0 < kmax; j0 += KM) {
+            int e1[KM], p1[KM];
+            float w1[KM];
+            float4 y[KM];
+#pragma unroll
+            for (int j = 0; j < KM; j++) {
+                const bool in = j0 + j < kmax;
+                const size_t oj = (size_t)row * kmax + j0 + j;
+                e1[j] = in ? idx[oj] : -1;
+                p1[j] = in ? pos[oj] : 0;
+                w1[j] = in ? wts[oj] : 0.f;
+            }
+#pragma unroll
+            for (int j = 0; j < KM; j++) y[j] = e1[j] >= 0 ? ldcg4(Ys + (size_t)p1[j] * d + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int j = 0; j < KM; j++)
+                if (e1[j] >= 0 && w1[j] != 0.f) {
+                    m.x = fmaf(w1[j], y[j].x, m.x);
+                    m.y = fmaf(w1[j], y[j].y, m.y);
+                    m.z = fmaf(w1[j], y[j].z, m.z);
+                    m.w = fmaf(w1[j], y[j].w, m.w);
+                }
+        }
+        if (Psh) {
+            float4 sh = sum_splits4(Psh, split_stride, nsplit, o);
+            m.x += sh.x, m.y += sh.y, m.z += sh.z, m.w += sh.w;
+        }
+        s.x += m.x, s.y += m.y, s.z += m.z, s.w += m.w;
+        *reinterpret_cast<float4 *>(S + o) = s;
+        if (Xn) store_split4(Xn, o, lo_off, make_float4(gn.x * s.x, gn.y * s.y, gn.z * s.z, gn.w * s.w));
+        q = s.x * s.x + s.y * s.y + s.z * s.z + s.w * s.w;
+    }
+    if (Xn) {
+        q = warp_sum(q);
+        if ((threadIdx.x & 31) == 0) scratch[threadIdx.x >> 5] = q;
+        __syncthreads();
+        if ((threadIdx.x & 63) == 0 && row < R) ss_out[(size_t)blockIdx.y * ss_ld + row] = scratch[2 * sub] + scratch[2 * sub + 1];
+    }
 }
 
 // Sum split partials into a plain fp32 matrix (used by the operator-level GEMM entry point).

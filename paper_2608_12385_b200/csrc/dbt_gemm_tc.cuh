@@ -207,7 +207,9 @@ struct TcCfg {
     static constexpr int kStageBytes = MT * kTcABytes + 2 * kBBytes;
     // small row counts: keep one CTA near 100 KB so that a dependent kernel's CTA can become
     // resident beside it; large row counts take the whole SM
-    static constexpr int kStages = N_TILE <= 16 ? 5 : N_TILE <= 32 ? 4 : N_TILE <= 64 ? 3 : N_TILE <= 128 ? 4 : 2;
+    // (64-row tiles with two weight tiles per CTA -- the per-expert GEMMs of a prompt chunk -- keep two CTAs per SM
+    // with two stages of 48 KB each)
+    static constexpr int kStages = N_TILE <= 16 ? 5 : N_TILE <= 32 ? 4 : N_TILE <= 64 ? (MT == 2 ? 2 : 3) : N_TILE <= 128 ? 4 : 2;
     // room for the two planes' accumulators side by side (see `stacked` in the kernel)
     static constexpr int kStackable = N_TILE <= 128;
     static constexpr int kAccCols = kStackable ? 2 * N_TILE : N_TILE;  // accumulator columns of one weight tile
