@@ -248,31 +248,87 @@ def test_1b_at_the_benchmarks_launch_configuration_on_sampled_sequences():
     assert gm.sync_status() == (0, 0)
 
 
+@pytest.mark.parametrize("cfg,lens", [
+    (small_bf16(n_layers=2), [0, 5, 17, 300, 64, 63]),                        # from an empty cache to 19 pages
+    (small_bf16(n_layers=2, n_paths=3), [1, 1000, 16, 15, 129]),              # three paths
+    (small_bf16(n_layers=1), [7 * i % 211 for i in range(40)]),               # 80 (sequence, KV head) pairs: the one-wave attention form
+    (small_moe(), [3, 90, 0, 31, 32, 33, 500]),
+])
+def test_sequences_of_different_lengths_in_one_batch(cfg, lens):
+    """A serving batch is ragged: every sequence at its own position (its own RoPE angle, page count and share of
+    the attention work split).  Each sequence gets a seeded cache of its own length through dbt_kv_import;
+    sequences do not interact, so row b must match the oracle run on sequence b alone (dense models: two grouped
+    steps and a primary-only one; the MoE model under the device's routing, checked as a valid top-k)."""
+    B, steps = len(lens), 2
+    w = make_weights(cfg, seed=41, matrix_std=0.05)
+    tok = make_tokens(cfg, B, steps + 1, seed=42)
+    T = max(lens) + steps + 2
+    gm = make_gpu_model(cfg, w, B, T)
+    oms = []
+    for b, n in enumerate(lens):
+        om = oracle.OracleModel(cfg, w, 1, T)
+        if n:
+            k, v = make_synthetic_kv(cfg, 1, n, seed=100 + b)
+            gm.import_kv(k, v, seq_ids=[b])
+            om.inject_kv(k, v, n)
+        oms.append(om)
+    gm.set_seq_lens(lens)
+    for t in range(steps + 1):
+        grouped = t < steps or cfg.is_moe  # (the MoE model: grouped steps only, the routing of every path is read back)
+        g = gm.decode_full(tok[:, t].cuda().contiguous(), grouped=grouped)
+        ex = gm.last_experts(B).numpy() if cfg.is_moe else None
+        for b, om in enumerate(oms):
+            forced = np.ascontiguousarray(ex[:, :, b:b + 1]) if cfg.is_moe else None
+            o = om.decode_step(tok[b:b + 1, t].numpy(), grouped=grouped, forced_experts=forced)
+            if cfg.is_moe:
+                assert_routing_is_a_valid_topk(cfg, forced, om.router_logits(1), f"seq {b} step {t}")
+            assert_logits_close(g["z1"][b:b + 1], o["z1"], cfg.weight_dtype, f"seq {b} (length {lens[b] + t}) z1")
+            if grouped:
+                z2 = g["z2"][:, b:b + 1] if cfg.n_paths > 2 else g["z2"][b:b + 1]
+                assert_logits_close(z2, o["z2"], cfg.weight_dtype, f"seq {b} (length {lens[b] + t}) z2")
+    assert [gm.seq_len(b) for b in range(B)] == [n + steps + 1 for n in lens]
+    assert gm.sync_status() == (0, 0)
+
+
+@pytest.mark.parametrize("cfg,B", [(small_bf16(n_layers=1), 128), (small_bf16(n_layers=1), 77),
+                                   (small_bf16(n_layers=1, n_paths=3), 85)])
+def test_large_batches_up_to_256_stacked_rows(cfg, B):
+    """The widest decode tiles: 256 stacked rows (128 sequences x 2 paths), an odd 154, and 255 rows over three
+    paths; prefill of 20 positions (a chunk of more than 2048 rows is cut), three grouped steps."""
+    w = make_weights(cfg, seed=43, matrix_std=0.05)
+    tok = make_tokens(cfg, B, 23, seed=44)
+    teacher_forced_compare(cfg, w, tok, n_prefill=20, grouped=True)
+
+
 def test_1b_width_three_paths_at_batch_16_on_sampled_sequences():
-    """Appendix C.1 at the benchmark's batch and the 1B model's width (four of its layers, context 700): three
-    residual paths, i.e. 48 stacked rows in 64-row GEMM tiles, six query rows per KV head in the one-wave
-    attention form, a block per branch in the kernels between the GEMMs, two branch distributions in the
-    readout.  Sequences 3 and 14 against the oracle run on them alone."""
+    """Appendix C.1 at the benchmark's batch and the 1B model's width (four of its layers): three residual paths,
+    i.e. 48 stacked rows in 64-row GEMM tiles, six query rows per KV head in the one-wave attention form (128
+    pairs of different lengths: sequence b holds 100 + 40 b positions), a block per branch in the kernels between
+    the GEMMs, two branch distributions in the readout.  Sequences 3 and 14 against the oracle run on each alone."""
     cfg = dense_1b().replace(n_layers=4, n_paths=3)
     w = make_weights(cfg, seed=0)
-    B, ctx, pick = 16, 700, [3, 14]
+    B, pick = 16, [3, 14]
+    lens = [100 + 40 * b for b in range(B)]
     tok = make_tokens(cfg, B, 2, seed=2)
-    k, v = make_synthetic_kv(cfg, len(pick), ctx, seed=3)
-    gm = make_gpu_model(cfg, w, B, ctx + 3)
+    gm = make_gpu_model(cfg, w, B, max(lens) + 3)
     gen = torch.Generator(device=gm.device)
     gen.manual_seed(5)
     gm.kv_pool.normal_(0.0, 1.0, generator=gen)
-    gm.import_kv(k, v, seq_ids=pick)
-    gm.set_seq_lens([ctx] * B)
-    om = oracle.OracleModel(cfg, w, len(pick), ctx + 3)
-    om.inject_kv(k, v, ctx)
+    oms = {}
+    for b in pick:
+        k, v = make_synthetic_kv(cfg, 1, lens[b], seed=3 + b)
+        gm.import_kv(k, v, seq_ids=[b])
+        oms[b] = oracle.OracleModel(cfg, w, 1, lens[b] + 3)
+        oms[b].inject_kv(k, v, lens[b])
+    gm.set_seq_lens(lens)
     for t in range(2):
-        o = om.decode_step(tok[pick, t].numpy())
         g = gm.decode_full(tok[:, t].cuda().contiguous())
-        assert_logits_close(g["z1"][pick], o["z1"], "bf16", f"K=3 step {t} z1")
-        for j in range(2):
-            assert_logits_close(g["z2"][j][pick], o["z2"][j], "bf16", f"K=3 step {t} branch {j + 2}")
-        np.testing.assert_allclose(g["alpha"][pick].cpu().numpy(), o["alpha"], rtol=1e-3)
+        for b in pick:
+            o = oms[b].decode_step(tok[b:b + 1, t].numpy())
+            assert_logits_close(g["z1"][b:b + 1], o["z1"], "bf16", f"K=3 seq {b} step {t} z1")
+            for j in range(2):
+                assert_logits_close(g["z2"][j][b:b + 1], o["z2"][j], "bf16", f"K=3 seq {b} step {t} branch {j + 2}")
+            np.testing.assert_allclose(g["alpha"][b:b + 1].cpu().numpy(), o["alpha"], rtol=1e-3)
     assert gm.sync_status() == (0, 0)
 
 
