@@ -193,7 +193,8 @@ dbt_status dbt_last_expert_union(dbt_model *m, int32_t *count_per_layer_host);
  * clamped and the step ran on): returns DBT_ERR_DEVICE; 3 = a bounded wait inside a kernel (on a
  * shared-memory barrier that a TMA copy or a tensor-core commit completes) ran out after about two
  * seconds: *detail = the wait site (100 + warp: operand ring of the GEMM, 200 + warp: its accumulator,
- * 300..: the attention kernel's page ring), the CTA skipped its stores, released its tensor memory and
+ * 300..: the decode attention kernel's page ring, 400..: the prompt attention kernel's, 500..: the
+ * persistent per-expert GEMM's rings and accumulators), the CTA skipped its stores, released its tensor memory and
  * returned, so the step's results are invalid but the context stays usable: returns DBT_ERR_TIMEOUT.
  * The first code recorded wins until dbt_reset clears the word.  HOST pointers, may be NULL. */
 dbt_status dbt_sync_status(dbt_model *m, int32_t *device_status, int32_t *detail);
