@@ -91,7 +91,10 @@ struct AttCfg {
     // fragment-shaped accesses off a single bank), m, l, flag, row tables
     static constexpr int kFoldStride = DH + 8;
     static constexpr int kScratchBytes = (16 * kFoldStride + 2 * 16 + 16 + 3 * kAttMaxItems + 12) * 4 + 2 * DH * 2 + 32;
-    static constexpr int kSmemBytes = kStages * kStageBytes + 1024 + 128 + kScratchBytes;
+    // room for the ring's barriers (two per stage, up to 12 stages) ahead of the scratch
+    static constexpr int kBarBytes = 256;
+    static_assert(2 * kStages * 8 <= kBarBytes, "the barriers must not reach into the scratch");
+    static constexpr int kSmemBytes = kStages * kStageBytes + 1024 + kBarBytes + kScratchBytes;
 };
 
 __device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4]) {
@@ -240,7 +243,7 @@ __global__ void __launch_bounds__(160, DEEP ? 1 : 2) attn_mma_kernel(const __gri
     auto full_bar = [&](int s) { return bars + 8u * s; };
     auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
     constexpr int FS = Cfg::kFoldStride;
-    float *sc_o = reinterpret_cast<float *>(gen + STAGES * Cfg::kStageBytes + 128);  // [16][FS]
+    float *sc_o = reinterpret_cast<float *>(gen + STAGES * Cfg::kStageBytes + Cfg::kBarBytes);  // [16][FS]
     float *sc_m = sc_o + 16 * FS;                                                   // [16]
     float *sc_l = sc_m + 16;                                                        // [16]
     int *flag = reinterpret_cast<int *>(sc_l + 16);                                 // [0] last?, [1] longest pair, [8..15] 1/rms per path

@@ -252,6 +252,7 @@ def test_1b_at_the_benchmarks_launch_configuration_on_sampled_sequences():
     (small_bf16(n_layers=2), [0, 5, 17, 300, 64, 63]),                        # from an empty cache to 19 pages
     (small_bf16(n_layers=2, n_paths=3), [1, 1000, 16, 15, 129]),              # three paths
     (small_bf16(n_layers=1), [7 * i % 211 for i in range(40)]),               # 80 (sequence, KV head) pairs: the one-wave attention form
+    (small_bf16(n_layers=1), [900 + 13 * i for i in range(40)]),              # the same with more stages per pair than its ring holds
     (small_moe(), [3, 90, 0, 31, 32, 33, 500]),
 ])
 def test_sequences_of_different_lengths_in_one_batch(cfg, lens):
