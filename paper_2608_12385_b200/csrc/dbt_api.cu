@@ -98,6 +98,7 @@ struct dbt_model {
     bool evict_first;  // weight tiles and K/V pages carry the evict-first L2 hint (DBT_EVICT_FIRST=0 turns it off)
     int moe_persist;       // per-expert GEMMs as persistent CTAs over the units that have work: -1 by the batch, DBT_MOE_PERSIST=0/1 off/on
     int cur_rows;          // primary rows (sequences x positions) of the launch plan being built
+    bool moe_fuse_swiglu;  // the persistent per-expert gate|up launch applies the SwiGLU itself (DBT_MOE_FUSE_SWIGLU=0: a kernel of its own)
     bool prompt_attn_off;  // DBT_PROMPT_ATTN=tile: prompt chunks through the 16-row kernel's packed tiles (the earlier form)
     bool fuse_qkv;     // decode steps: the attention kernel does the Q|K|V epilogue itself (DBT_FUSE_QKV=0 keeps the kernel)
     int num_sms;
@@ -587,6 +588,10 @@ struct TcCall {
     int grp_row_tiles;  // per-expert mode: row tiles of n_tile rows per expert (0: one tile holds any list)
     int grp_prewait;    // per-expert mode: the lists are final before this launch can be resident (see TcParams)
     int grp_mt2;        // per-expert mode, 64-row tiles: two weight tiles per CTA share each activation box (prompt chunks)
+    // per-expert gate|up launch: where it runs as persistent CTAs it may apply the SwiGLU itself (see SwigluEpi);
+    // *fused tells the caller whether it did
+    const SwigluEpi *swiglu;
+    bool *fused;
 };
 
 int norm_threads(int d) { return d >= 1024 ? 1024 : d >= 512 ? 512 : 256; }
@@ -642,11 +647,21 @@ dbt_status launch_gemm_tc(dbt_model *m, const TcCall &c, const TcParams &p, cons
         // stacked rows, within +-2 % of the one-CTA-per-unit launch above that; same bits either way)
         const bool want = m->moe_persist < 0 ? paths_of(m->cfg) * m->cur_rows <= 16 : m->moe_persist > 0;
         if (c.grp_cnt && want && pp.x3d && pp.stacked && c.nseg <= 2 && c.n_groups <= kPersistMaxGroups) {
+            if (N_TILE == 16 && c.swiglu && c.fused && c.nseg == 2 && c.n_out[0] == c.n_out[1] && m->moe_fuse_swiglu) {
+                const int smem = TcPersistCfg<N_TILE, true>::smem_bytes(c.n_groups);
+                if (cudaFuncSetAttribute(gemm_tc_persist_kernel<N_TILE, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) !=
+                    cudaSuccess)
+                    return fail(m, DBT_ERR_CUDA, "shared memory opt-in for the persistent per-expert GEMM");
+                LAUNCH(m, c.tag, bytes, (gemm_tc_persist_kernel<N_TILE, true>), dim3(2 * m->num_sms), 192, smem, *c.W[0], *w1, *x, pp,
+                       c.n_groups, (int)grid.x / 2, *c.swiglu);
+                *c.fused = true;
+                return DBT_OK;
+            }
             const int smem = TcPersistCfg<N_TILE>::smem_bytes(c.n_groups);
             if (cudaFuncSetAttribute(gemm_tc_persist_kernel<N_TILE>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
                 return fail(m, DBT_ERR_CUDA, "shared memory opt-in for the persistent per-expert GEMM");
             LAUNCH(m, c.tag, bytes, gemm_tc_persist_kernel<N_TILE>, dim3(2 * m->num_sms), 192, smem, *c.W[0], *w1, *x, pp, c.n_groups,
-                   (int)grid.x);
+                   (int)grid.x, SwigluEpi{});
             return DBT_OK;
         }
     }
@@ -949,18 +964,24 @@ dbt_status run_moe_tc(dbt_model *m, int l, const RowMap &rm, int grouped, bool r
     gu.grp_row_tiles = grt;
     gu.grp_mt2 = (gt == 64 && Bc > 256) ? 1 : 0;
     gu.grp_prewait = m->use_pdl ? 1 : 0;  // the gather kernel before it lets its dependents in only after its own wait
+    const SwigluEpi se{w.Hs, lo_hs, wide ? (const float *)w.rs_sorted : (const float *)nullptr, Fe};
+    bool swiglu_done = false;
+    gu.swiglu = &se;
+    gu.fused = &swiglu_done;
     if ((st = run_gemm_tc(m, gu, gt, nullptr, nullptr)) != DBT_OK) return st;
-    LAUNCH(m, "moe_swiglu", 0, moe_swiglu_kernel, dim3(R * km, (Fe + 255) / 256), 256, 0, w.Pe, w.eoff + E, Fe, w.Hs, lo_hs,
-           wide ? (const float *)w.rs_sorted : (const float *)nullptr);
+    if (!swiglu_done)
+        LAUNCH(m, "moe_swiglu", 0, moe_swiglu_kernel, dim3(R * km, (Fe + 255) / 256), 256, 0, w.Pe, w.eoff + E, Fe, w.Hs, lo_hs,
+               wide ? (const float *)w.rs_sorted : (const float *)nullptr);
     TcCall dn{};
     dn.W[0] = &mp.ed; dn.n_out[0] = d; dn.rows[0] = Rk; dn.nseg = 1; dn.X = &m->map_Hs; dn.K = Fe; dn.R = Rk;
     dn.P = w.Yexp; dn.P_floats = (size_t)Rk * d; dn.tag = "expert_down"; dn.parts = m->act_parts; dn.lo_row0 = Rk;
     dn.grp_cnt = w.ecnt; dn.grp_off = w.eoff; dn.grp_w_rows = d; dn.n_groups = E;
     dn.grp_row_tiles = grt;
     dn.grp_mt2 = gu.grp_mt2;
-    // The lists come from the sort kernel, four launches back.  A CTA of this launch can only be resident once every
-    // CTA of the SwiGLU kernel has started, hence once every CTA of the gate|up GEMM has passed its own dependency
-    // wait (it waits before anything else), hence after the gather kernel -- and the sort kernel before it -- ended.
+    // The lists come from the sort kernel, several launches back.  A CTA of this launch can only be resident once
+    // every CTA of the launch before it has started (the SwiGLU kernel, or the gate|up GEMM where that applies the
+    // SwiGLU itself), hence once every CTA of the gate|up GEMM is resident, hence once every CTA of the gather kernel
+    // has let its dependents in -- which it does only after its own wait on the sort kernel.
     dn.grp_prewait = m->use_pdl ? 1 : 0;
     if ((st = run_gemm_tc(m, dn, gt, nullptr, nullptr)) != DBT_OK) return st;
     if (Fs > 0 && !overlap && (st = shared_expert(w.P, w.P_floats)) != DBT_OK) return st;
@@ -1591,6 +1612,8 @@ dbt_status dbt_create(const dbt_config *cfg, const dbt_weights *w, void *kv_pool
         m->fuse_qkv = m->att_fast && !(fq && strcmp(fq, "0") == 0);
         const char *mp = getenv("DBT_MOE_PERSIST");
         m->moe_persist = !mp ? -1 : strcmp(mp, "1") == 0 ? 1 : 0;
+        const char *fs = getenv("DBT_MOE_FUSE_SWIGLU");
+        m->moe_fuse_swiglu = !(fs && strcmp(fs, "0") == 0);
         const char *pa = getenv("DBT_PROMPT_ATTN");
         m->prompt_attn_off = pa && strcmp(pa, "tile") == 0;
     }

@@ -17,34 +17,48 @@ namespace dbt {
 
 constexpr int kPersistMaxGroups = 1024;
 
-template <int N_TILE>
-struct TcPersistCfg {
-    using Base = TcCfg<N_TILE>;
-    static constexpr int kAccCols = Base::kAccCols;
-    static constexpr int kTmemCols = 2 * kAccCols < 32 ? 32 : 2 * kAccCols;  // two accumulators
-    // ring + alignment slack + barriers + three tables of E (+1) ints: counts, row offsets, tile offsets
-    static constexpr int smem_bytes(int n_groups) { return Base::kStages * Base::kStageBytes + 1024 + 256 + (3 * n_groups + 8) * 4; }
+// The gate|up launch may also do the SwiGLU (Eq. moe_layer's expert MLP): FUSE = a unit takes the gate tile and the
+// up tile of the same 128 features (two accumulators), and its epilogue -- which overlaps the next unit's MMAs --
+// writes H = SiLU(rs * gate) * (rs * up) as the down projection's two bf16 planes: no kernel in between.
+struct SwigluEpi {
+    __nv_bfloat16 *Hs;  // [rows][Fe] hi plane (+ lo plane at lo_off)
+    size_t lo_off;
+    const float *rs;    // per sorted row: 1/rms of the row the GEMM input was not yet divided by (nullptr: 1)
+    int Fe;
 };
 
-template <int N_TILE>
+template <int N_TILE, bool FUSE = false>
+struct TcPersistCfg {
+    using Base = TcCfg<N_TILE>;
+    static constexpr int kWTiles = FUSE ? 2 : 1;
+    static constexpr int kStageBytes = kWTiles * kTcABytes + 2 * Base::kBBytes;
+    static constexpr int kStages = FUSE ? 3 : Base::kStages;  // both forms keep two CTAs per SM
+    static constexpr int kAccCols = kWTiles * Base::kAccCols;  // accumulator columns of one unit
+    static constexpr int kTmemCols = 2 * kAccCols < 32 ? 32 : 2 * kAccCols;  // two units' accumulators
+    // ring + alignment slack + barriers + three tables of E (+1) ints: counts, row offsets, tile offsets
+    static constexpr int smem_bytes(int n_groups) { return kStages * kStageBytes + 1024 + 256 + (3 * n_groups + 8) * 4; }
+};
+
+template <int N_TILE, bool FUSE = false>
 __global__ void __launch_bounds__(192, 2)
 gemm_tc_persist_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtensorMap tmW1,
-                       const __grid_constant__ CUtensorMap tmX, TcParams p, int n_groups, int tiles) {
+                       const __grid_constant__ CUtensorMap tmX, TcParams p, int n_groups, int tiles, SwigluEpi se) {
     using Cfg = TcCfg<N_TILE>;
-    using PCfg = TcPersistCfg<N_TILE>;
+    using PCfg = TcPersistCfg<N_TILE, FUSE>;
     static_assert(N_TILE <= 32, "the epilogue holds a whole accumulator row in registers");
-    constexpr int STAGES = Cfg::kStages;
+    constexpr int STAGES = PCfg::kStages;
+    constexpr int kXOff = PCfg::kWTiles * kTcABytes;  // the activation box follows the weight tile(s) of a stage
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles_s = (raw + 1023u) & ~1023u;  // 1024-byte aligned operand tiles
     uint8_t *gen = smem_raw + (tiles_s - raw);
-    const uint32_t bars = tiles_s + STAGES * Cfg::kStageBytes;
+    const uint32_t bars = tiles_s + STAGES * PCfg::kStageBytes;
     auto full_bar = [&](int s) { return bars + 8u * s; };
     auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
     auto acc_full = [&](int b) { return bars + 8u * (2 * STAGES + b); };
     auto acc_empty = [&](int b) { return bars + 8u * (2 * STAGES + 2 + b); };
-    uint32_t *tmem_holder = reinterpret_cast<uint32_t *>(gen + STAGES * Cfg::kStageBytes + 8 * (2 * STAGES + 4));
-    int *cnt_s = reinterpret_cast<int *>(gen + STAGES * Cfg::kStageBytes + 256);  // [E]
+    uint32_t *tmem_holder = reinterpret_cast<uint32_t *>(gen + STAGES * PCfg::kStageBytes + 8 * (2 * STAGES + 4));
+    int *cnt_s = reinterpret_cast<int *>(gen + STAGES * PCfg::kStageBytes + 256);  // [E]
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, E = n_groups;
     int *roff = cnt_s + E;      // [E + 1] first sorted row of an expert
     int *toff = roff + E + 1;   // [E + 1] row tiles before an expert
@@ -116,7 +130,7 @@ gemm_tc_persist_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_co
         Unit un;
         un.x_row0 = roff[lo] + rt * N_TILE;
         un.rows = min(N_TILE, cnt_s[lo] - rt * N_TILE);
-        un.sg = (p.nseg > 1 && ft >= p.seg[1].tile0) ? 1 : 0;
+        un.sg = (!FUSE && p.nseg > 1 && ft >= p.seg[1].tile0) ? 1 : 0;  // FUSE: `tiles` counts one segment's tiles
         un.f0 = (ft - p.seg[un.sg].tile0) * kTcM;
         un.w_row = lo * p.grp_w_rows + un.f0;
         return un;
@@ -128,17 +142,21 @@ gemm_tc_persist_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_co
         tma_prefetch_desc(&tmW0);
         tma_prefetch_desc(&tmW1);
         tma_prefetch_desc(&tmX);
-        const uint32_t tx = kTcABytes + 2 * Cfg::kBBytes;
+        const uint32_t tx = PCfg::kWTiles * kTcABytes + 2 * Cfg::kBBytes;
         const uint64_t pol = l2_evict_first_policy();
         auto load_w = [&](int s, int kt, const Unit &un) {
-            const CUtensorMap *tmW = un.sg == 0 ? &tmW0 : &tmW1;
-            if (p.evict_first)
-                tma_load_2d_hint(tiles_s + s * Cfg::kStageBytes, tmW, full_bar(s), kt * kTcK, un.w_row, pol);
-            else
-                tma_load_2d(tiles_s + s * Cfg::kStageBytes, tmW, full_bar(s), kt * kTcK, un.w_row);
+#pragma unroll
+            for (int wt = 0; wt < PCfg::kWTiles; wt++) {  // FUSE: the gate tile, then the up tile of the same features
+                const CUtensorMap *tmW = (FUSE ? wt : un.sg) == 0 ? &tmW0 : &tmW1;
+                const uint32_t dst = tiles_s + s * PCfg::kStageBytes + wt * kTcABytes;
+                if (p.evict_first)
+                    tma_load_2d_hint(dst, tmW, full_bar(s), kt * kTcK, un.w_row, pol);
+                else
+                    tma_load_2d(dst, tmW, full_bar(s), kt * kTcK, un.w_row);
+            }
         };
         auto load_x = [&](int s, int kt, const Unit &un) {
-            tma_load_3d(tiles_s + s * Cfg::kStageBytes + kTcABytes, &tmX, full_bar(s), kt * kTcK, un.x_row0, 0);
+            tma_load_3d(tiles_s + s * PCfg::kStageBytes + kXOff, &tmX, full_bar(s), kt * kTcK, un.x_row0, 0);
         };
         int it = 0;
         bool first = true;
@@ -183,10 +201,14 @@ gemm_tc_persist_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_co
                 ok = mbar_wait(full_bar(s), (it / STAGES) & 1);
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint64_t adesc = umma_smem_desc(tiles_s + s * Cfg::kStageBytes);
-                const uint64_t bdesc = umma_smem_desc(tiles_s + s * Cfg::kStageBytes + kTcABytes);
+                const uint64_t bdesc = umma_smem_desc(tiles_s + s * PCfg::kStageBytes + kXOff);
 #pragma unroll
-                for (int k = 0; k < kTcK / 16; k++) umma_f16(acc, adesc + 2 * k, bdesc + 2 * k, idesc2, (kt | k) != 0);
+                for (int wt = 0; wt < PCfg::kWTiles; wt++) {
+                    const uint64_t adesc = umma_smem_desc(tiles_s + s * PCfg::kStageBytes + wt * kTcABytes);
+#pragma unroll
+                    for (int k = 0; k < kTcK / 16; k++)
+                        umma_f16(acc + wt * Cfg::kAccCols, adesc + 2 * k, bdesc + 2 * k, idesc2, (kt | k) != 0);
+                }
                 umma_commit(empty_bar(s));
             }
             if (ok) umma_commit(acc_full(buf));
@@ -205,7 +227,7 @@ gemm_tc_persist_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_co
             if (!ok) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint32_t base = tmem_base + ((uint32_t)(q * 32) << 16) + buf * PCfg::kAccCols;
-            float v[N_TILE];
+            float v[N_TILE], vu[FUSE ? N_TILE : 1];
 #pragma unroll
             for (int c0 = 0; c0 < N_TILE; c0 += 16) {
                 uint32_t a[16], b[16];
@@ -214,13 +236,30 @@ gemm_tc_persist_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_co
                 tmem_ld_wait();
 #pragma unroll
                 for (int i = 0; i < 16; i++) v[c0 + i] = __uint_as_float(a[i]) + __uint_as_float(b[i]);
+                if constexpr (FUSE) {  // the up tile's accumulator
+                    tmem_ld16_issue(base + Cfg::kAccCols + c0, a);
+                    tmem_ld16_issue(base + Cfg::kAccCols + N_TILE + c0, b);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 16; i++) vu[c0 + i] = __uint_as_float(a[i]) + __uint_as_float(b[i]);
+                }
             }
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
             if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(acc_empty(buf)) : "memory");
             const TcSeg seg = p.seg[un.sg];
             const int f = un.f0 + q * 32 + lane;
-            if (f < seg.n_out) {
+            if constexpr (FUSE) {
+                if (f < se.Fe) {
+#pragma unroll
+                    for (int i = 0; i < N_TILE; i++)
+                        if (i < un.rows) {
+                            const int row = un.x_row0 + i;
+                            const float sc = se.rs ? __ldcg(se.rs + row) : 1.f;
+                            store_split(se.Hs, (size_t)row * se.Fe + f, se.lo_off, silu(sc * v[i]) * (sc * vu[i]));
+                        }
+                }
+            } else if (f < seg.n_out) {
                 float *out = p.P + (size_t)un.x_row0 * p.ldp + seg.col0 + f;
 #pragma unroll
                 for (int i = 0; i < N_TILE; i++)
