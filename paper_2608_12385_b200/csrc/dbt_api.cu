@@ -99,6 +99,7 @@ struct dbt_model {
     int moe_persist;       // per-expert GEMMs as persistent CTAs over the units that have work: -1 by the batch, DBT_MOE_PERSIST=0/1 off/on
     int cur_rows;          // primary rows (sequences x positions) of the launch plan being built
     bool moe_fuse_swiglu;  // the persistent per-expert gate|up launch applies the SwiGLU itself (DBT_MOE_FUSE_SWIGLU=0: a kernel of its own)
+    bool prompt_fuse_swiglu;  // prompt chunks: SwiGLU in the gate|up GEMM's epilogue (DBT_PROMPT_FUSE_SWIGLU=0: a kernel of its own)
     bool prompt_attn_off;  // DBT_PROMPT_ATTN=tile: prompt chunks through the 16-row kernel's packed tiles (the earlier form)
     bool fuse_qkv;     // decode steps: the attention kernel does the Q|K|V epilogue itself (DBT_FUSE_QKV=0 keeps the kernel)
     int num_sms;
@@ -592,6 +593,10 @@ struct TcCall {
     // *fused tells the caller whether it did
     const SwigluEpi *swiglu;
     bool *fused;
+    // dense gate|up launch over a prompt chunk: gate and up tiles of the same features in one CTA, SwiGLU in the
+    // epilogue (see GuEpi); *gu_fused tells the caller whether it was taken
+    const GuEpi *gu;
+    bool *gu_fused;
 };
 
 int norm_threads(int d) { return d >= 1024 ? 1024 : d >= 512 ? 512 : 256; }
@@ -689,6 +694,9 @@ dbt_status run_gemm_tc(dbt_model *m, const TcCall &c, int n_tile, int *nsplit_ou
         if (16 * w2 < 10 * w1) mt = 2;
     }
     if (c.grp_cnt && c.grp_mt2 && n_tile == 64) mt = 2;
+    const bool gu_pair = !c.grp_cnt && c.R > 256 && c.gu && c.gu_fused && c.nseg == 2 && c.n_out[0] == c.n_out[1] && c.n_out[0] % 8 == 0 &&
+                         m->prompt_fuse_swiglu;
+    if (gu_pair) mt = 2;
     for (int s = 0; s < c.nseg; s++) {
         p.seg[s] = TcSeg{tiles, c.n_out[s], c.rows[s], col};
         tiles += (c.n_out[s] + kTcM * mt - 1) / (kTcM * mt);
@@ -696,6 +704,14 @@ dbt_status run_gemm_tc(dbt_model *m, const TcCall &c, int n_tile, int *nsplit_ou
         if (!c.grp_cnt) bytes += (double)c.n_out[s] * c.K * 2;  // per-expert launches: the loaded set is known on the device only
     }
     p.nseg = c.nseg;
+    if (gu_pair) {  // tiles of 128 features, each with its gate and its up rows
+        p.seg[0] = TcSeg{0, c.n_out[0], c.rows[0], 0};
+        p.nseg = 1;
+        tiles = (c.n_out[0] + kTcM - 1) / kTcM;
+        p.gu = *c.gu;
+        p.gu.on = 1;
+        *c.gu_fused = true;
+    }
     p.K = c.K;
     p.ldp = col;
     p.R = c.R;
@@ -1268,8 +1284,17 @@ dbt_status run_layers_wide(dbt_model *m, const RowMap &rm, int grouped, int n_ti
         gu.W[1] = &mp.wu; gu.n_out[1] = F; gu.rows[1] = R;
         gu.nseg = 2;
         {
+            bool gu_done = false;
+            GuEpi ge{};
+            if (rows_form) {
+                ge.Hb = w.Hb; ge.lo_off = lo_h; ge.ss = w.ss; ge.ss_tiles = ss_tiles; ge.ss_ld = ss_ld; ge.d_norm = d; ge.F = F;
+                ge.eps = c.rms_eps;
+                gu.gu = &ge;
+                gu.gu_fused = &gu_done;
+            }
             if ((st = run_gemm_tc(m, gu, n_tile, &nsp, &sstride)) != DBT_OK) return st;
-            if (rows_form)
+            if (gu_done) {
+            } else if (rows_form)
                 LAUNCH(m, "swiglu_couple", 0, swiglu_rows_kernel, dim3(Bc, (F + 1023) / 1024), 256, 0, w.P, nsp, sstride, F, w.Hb, lo_h,
                        (const float *)w.ss, ss_tiles, ss_ld, d, c.rms_eps);
             else
@@ -1614,6 +1639,8 @@ dbt_status dbt_create(const dbt_config *cfg, const dbt_weights *w, void *kv_pool
         m->moe_persist = !mp ? -1 : strcmp(mp, "1") == 0 ? 1 : 0;
         const char *fs = getenv("DBT_MOE_FUSE_SWIGLU");
         m->moe_fuse_swiglu = !(fs && strcmp(fs, "0") == 0);
+        const char *pf = getenv("DBT_PROMPT_FUSE_SWIGLU");
+        m->prompt_fuse_swiglu = !(pf && strcmp(pf, "0") == 0);
         const char *pa = getenv("DBT_PROMPT_ATTN");
         m->prompt_attn_off = pa && strcmp(pa, "tile") == 0;
     }

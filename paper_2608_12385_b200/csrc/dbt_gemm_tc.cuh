@@ -34,7 +34,20 @@ struct TcSeg {
     int col0;    // first output column of this segment in P
 };
 
+// Prompt chunks, gate|up launch with two weight tiles per CTA: the two tiles are the gate tile and the up tile of
+// the same 128 features, and the epilogue applies the SwiGLU (Eq. mlp: H = SiLU(m W_g) * (m W_u), with the row's
+// 1/rms from its shares of sum(S^2)) and writes the down projection's input planes: no partials, no kernel between.
+struct GuEpi {
+    int on;
+    __nv_bfloat16 *Hb;  // [rows][F] hi plane (+ lo plane at lo_off)
+    size_t lo_off;
+    const float *ss;    // nullptr: the GEMM input was already normalised
+    int ss_tiles, ss_ld, d_norm, F;
+    float eps;
+};
+
 struct TcParams {
+    GuEpi gu;
     int evict_first;  // weight tiles carry the evict-first L2 hint
     int x3d;  // tmX is the 3-D {64, N_TILE, 2} view of a two-plane input: one box per stage
     int stacked;  // with x3d: one MMA per k16 step over both planes (N = 2 * N_TILE), halves added in the epilogue
@@ -263,7 +276,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
     if (p.nseg > 2 && tile >= p.seg[2].tile0) sg = 2;
     const TcSeg seg = p.seg[sg];
     const CUtensorMap *tmW = sg == 0 ? &tmW0 : sg == 1 ? &tmW1 : &tmW2;
-    int f0 = (tile - seg.tile0) * kTcM * MT;
+    const bool gu_pair = MT == 2 && p.gu.on;
+    int f0 = (tile - seg.tile0) * kTcM * (gu_pair ? 1 : MT);
     int total_kt = (p.K + kTcK - 1) / kTcK;
     int kt0 = split * p.kt_per_split;
     int nkt = min(p.kt_per_split, total_kt - kt0);
@@ -312,12 +326,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
         auto load_w = [&](int s, int kt) {
 #pragma unroll
             for (int mt = 0; mt < MT; mt++) {  // a tile past the matrix's last row arrives as zeros
+                // (gate|up pairs: tile 0 from the gate matrix, tile 1 the same rows of the up matrix)
+                const CUtensorMap *tw = gu_pair ? (mt == 0 ? &tmW0 : &tmW1) : tmW;
+                const int wrow = w_row0 + f0 + (gu_pair ? 0 : mt * kTcM);
                 if (p.evict_first)
-                    tma_load_2d_hint(tiles + s * Cfg::kStageBytes + mt * kTcABytes, tmW, full_bar(s), kt * kTcK,
-                                     w_row0 + f0 + mt * kTcM, pol);
+                    tma_load_2d_hint(tiles + s * Cfg::kStageBytes + mt * kTcABytes, tw, full_bar(s), kt * kTcK, wrow, pol);
                 else
-                    tma_load_2d(tiles + s * Cfg::kStageBytes + mt * kTcABytes, tmW, full_bar(s), kt * kTcK,
-                                w_row0 + f0 + mt * kTcM);
+                    tma_load_2d(tiles + s * Cfg::kStageBytes + mt * kTcABytes, tw, full_bar(s), kt * kTcK, wrow);
             }
         };
         for (int i = 0; i < npre; i++) {
@@ -415,6 +430,43 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
 #pragma unroll
                 for (int i = 0; i < 16; i++)
                     if (c0 + i < rows) e.Z[(size_t)(c0 + i) * p.ldp + seg.col0 + f] = v[i] * scratch[c0 + i];
+            }
+        }
+    } else if (got && gu_pair) {
+        if constexpr (MT == 2) {
+            // H goes through shared memory (the idle ring: [row][128 features] per plane) so that it leaves in
+            // 16-byte pieces of a row instead of 2-byte elements of a column.  F % 8 == 0.
+            __nv_bfloat16 *st_hi = reinterpret_cast<__nv_bfloat16 *>(gen_tiles), *st_lo = st_hi + N_TILE * kTcM;
+            float *rs_s = reinterpret_cast<float *>(st_lo + N_TILE * kTcM);
+            for (int r = tid; r < rows; r += blockDim.x)
+                rs_s[r] = row_scale(p.gu.ss, p.gu.ss_tiles, p.gu.ss_ld, x_row0 + r, p.gu.d_norm, p.gu.eps);
+            __syncthreads();
+            const int fl = warp * 32 + lane;
+#pragma unroll 1
+            for (int c0 = 0; c0 < N_TILE && c0 < rows; c0 += 16) {
+                float vg[16], vu[16];
+                ld_acc(0, c0, vg);
+                ld_acc(1, c0, vu);
+#pragma unroll
+                for (int i = 0; i < 16; i++) {
+                    const float rs = rs_s[min(c0 + i, N_TILE - 1)];
+                    const float h = silu(rs * vg[i]) * (rs * vu[i]);
+                    const __nv_bfloat16 hi = __float2bfloat16_rn(h);
+                    st_hi[(c0 + i) * kTcM + fl] = hi;
+                    st_lo[(c0 + i) * kTcM + fl] = __float2bfloat16_rn(h - __bfloat162float(hi));
+                }
+            }
+            __syncthreads();
+            const int nf8 = max(0, min(kTcM, p.gu.F - f0)) / 8;  // 16-byte pieces of this tile's features
+            for (int idx = tid; idx < rows * (kTcM / 8); idx += blockDim.x) {
+                const int r = idx / (kTcM / 8), c8 = idx % (kTcM / 8);
+                if (c8 < nf8) {
+                    const size_t o = (size_t)(x_row0 + r) * p.gu.F + f0 + c8 * 8;
+                    *reinterpret_cast<uint4 *>(p.gu.Hb + o) = *reinterpret_cast<const uint4 *>(st_hi + r * kTcM + c8 * 8);
+                    if (p.gu.lo_off)
+                        *reinterpret_cast<uint4 *>(p.gu.Hb + o + p.gu.lo_off) =
+                            *reinterpret_cast<const uint4 *>(st_lo + r * kTcM + c8 * 8);
+                }
             }
         }
     } else if (got) {
