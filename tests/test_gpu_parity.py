@@ -136,6 +136,13 @@ def test_prompt_chunks_through_the_16_row_attention_kernel(monkeypatch):
     test_long_prompt_prefill_matches_the_oracle(small_bf16(n_layers=2), 3, 700)
 
 
+def test_prompt_chunks_with_the_swiglu_as_a_kernel_of_its_own(monkeypatch):
+    """DBT_PROMPT_FUSE_SWIGLU=0: the gate|up GEMM of a prompt chunk leaves fp32 partials and the vector SwiGLU
+    kernel follows (the default applies it in the GEMM's epilogue)."""
+    monkeypatch.setenv("DBT_PROMPT_FUSE_SWIGLU", "0")
+    test_long_prompt_prefill_matches_the_oracle(small_bf16(n_layers=2), 3, 700)
+
+
 def test_prefill_in_one_call_equals_prefill_in_pieces():
     """The cache does not depend on how the prompt is cut into calls: 1500 positions at once (one chunk, six
     row tiles) and as 700 + 800 give the same logits within tolerance and caches equal to bf16 rounding."""
@@ -838,7 +845,7 @@ def test_compute_matched_moe_on_the_alternative_chains(monkeypatch, knob, value)
 
 @pytest.mark.parametrize("knob,value", [("DBT_MOE_OVERLAP", "0"), ("DBT_GRAPH", "0"), ("DBT_MOE", "simt"),
                                         ("DBT_FUSE_QKV", "0"), ("DBT_ATTN", "simt"), ("DBT_MOE_PERSIST", "0"),
-                                        ("DBT_MOE_PERSIST", "1")])
+                                        ("DBT_MOE_PERSIST", "1"), ("DBT_MOE_FUSE_SWIGLU", "0")])
 def test_moe_on_the_alternative_chains(monkeypatch, knob, value):
     """The shared expert on the main stream instead of beside the routed chain, direct launches instead
     of graph replay, the CUDA-core expert kernels, the separate Q|K|V epilogue kernel, the CUDA-core
